@@ -1,0 +1,337 @@
+/*
+ * SKVQ CPU oracle -- TEST INFRASTRUCTURE, NOT THE PRODUCT.
+ *
+ * A plain, slow, deliberately unoptimised restatement of the SKVQ runtime path
+ * (arXiv 2405.06219): channel reorder, group-wise clipped dynamic asymmetric
+ * quantization with a full-precision sliding window, and softmax attention of a
+ * single decode query over the mixed [quantized prefix || fp16 window] cache.
+ * It exists so that the CUDA library can be checked against something written
+ * straight from the paper.  Only the test-suite, the smoke check and the
+ * benchmark's CPU-baseline leg may call it.  It shares no code, header, table or
+ * helper with the CUDA path, and the CUDA path never calls it.
+ *
+ * Precision contract
+ *   - quantizer: IEEE fp32, one rounding per operation (build with
+ *     -ffp-contract=off, never -ffast-math), round-half-to-even via rintf();
+ *     scale and zero point are stored in fp16 (round-to-nearest-even) and the
+ *     codes are computed against the *stored* (rounded) parameters.
+ *   - attention: fp64 everywhere; dequantized values are never rounded.
+ *
+ * Layout (all row-major, host memory)
+ *   codes  uint8  [B][Hkv][cap_q][D*bits/8]   code j of a row sits in bits
+ *                                             [(j*bits) mod 8, +bits) of byte (j*bits)/8
+ *   meta   uint16 [B][Hkv][cap_q][D/G][2]     {h, z} as fp16 bit patterns
+ *   win    uint16 [B][Hkv][W][D]              ring: token t lives in slot t mod W,
+ *                                             channels already in reordered order
+ *   lengths int32 [B]                         tokens appended so far
+ *
+ * Pins (tests/test_oracle_*.py): round-trip error bound, reduction to textbook
+ * per-token min-max quantization, closed-form groups, permutation invariance,
+ * single-append == bulk-append, brute-force attention, convexity, q = 0 mean.
+ * End-to-end accuracy versus the paper's benchmark tables: parity unpinned (the
+ * datasets and model weights those tables need are not available).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* ---------------------------------------------------------------- fp16 <-> fp32 */
+
+/* IEEE binary16 -> binary32, exact. */
+float orc_f16_to_f32(uint16_t hbits)
+{
+    uint32_t sign = (uint32_t)(hbits >> 15) & 1u;
+    uint32_t expo = (uint32_t)(hbits >> 10) & 0x1Fu;
+    uint32_t mant = (uint32_t)hbits & 0x3FFu;
+    double mag;
+    if (expo == 0)
+        mag = ldexp((double)mant, -24);                 /* subnormal or zero */
+    else if (expo == 31)
+        mag = mant ? (double)NAN : (double)INFINITY;
+    else
+        mag = ldexp((double)(mant + 1024u), (int)expo - 25);
+    return (float)(sign ? -mag : mag);
+}
+
+/* IEEE binary32 -> binary16, round to nearest, ties to even. */
+uint16_t orc_f32_to_f16(float f)
+{
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    uint16_t sign = (uint16_t)((u >> 16) & 0x8000u);
+    if (isnan(f)) return (uint16_t)(sign | 0x7E00u);
+    double a = fabs((double)f);
+    if (a >= 65520.0) return (uint16_t)(sign | 0x7C00u); /* rounds past the largest finite half */
+    if (a == 0.0) return sign;
+    int e;
+    (void)frexp(a, &e);                                   /* a = m * 2^e, 0.5 <= m < 1 */
+    int ulp_exp = (e - 1) - 10;                           /* exponent of one unit in the last place */
+    if (ulp_exp < -24) ulp_exp = -24;                     /* subnormal spacing */
+    double scaled = ldexp(a, -ulp_exp);                   /* exact: a power-of-two scaling */
+    double r = nearbyint(scaled);                         /* default mode: ties to even */
+    double v = ldexp(r, ulp_exp);                         /* the rounded magnitude, exact */
+    if (v >= 65536.0) return (uint16_t)(sign | 0x7C00u);
+    /* encode v */
+    if (v < ldexp(1.0, -14)) {
+        uint32_t m = (uint32_t)ldexp(v, 24);
+        return (uint16_t)(sign | m);
+    }
+    int e2;
+    double m2 = frexp(v, &e2);                            /* v = m2 * 2^e2 */
+    uint32_t mant = (uint32_t)ldexp(m2, 11) - 1024u;      /* 10 explicit bits */
+    uint32_t expo = (uint32_t)(e2 - 1 + 15);
+    return (uint16_t)(sign | (expo << 10) | mant);
+}
+
+/* ---------------------------------------------------------------- quantizer */
+
+/* Channel reorder (Sec. 3.1, Eq. 1): stored[j] = src[idx[j]]. */
+void orc_reorder_row(const uint16_t *src, const int32_t *idx, int D, uint16_t *dst)
+{
+    for (int j = 0; j < D; ++j) dst[j] = src[idx[j]];
+}
+
+/*
+ * Clipped dynamic asymmetric quantization of one already-reordered row
+ * (Sec. 3.1 uniform quantizer, Eq. 2, and clipping_quant of Algorithm 1):
+ * per group of G consecutive channels take min and max, multiply both by the
+ * group's clip factor, derive scale h and zero point z, round both to fp16,
+ * then code = clamp(rint((x - z) / h), 0, 2^bits - 1).
+ * A zero is canonicalised to +0 before it is used so that the sign of a zero
+ * minimum or maximum (which depends on the order elements are visited) cannot
+ * leak into the stored parameters.
+ */
+void orc_quantize_reordered_row(const uint16_t *xr, const float *alpha, int D, int G, int bits,
+                                uint8_t *codes, uint16_t *meta)
+{
+    const int qmax = (1 << bits) - 1;
+    const int ng = D / G;
+    memset(codes, 0, (size_t)(D * bits / 8));
+    for (int g = 0; g < ng; ++g) {
+        float mn = INFINITY, mx = -INFINITY;
+        for (int j = g * G; j < (g + 1) * G; ++j) {
+            float v = orc_f16_to_f32(xr[j]);
+            if (v < mn) mn = v;
+            if (v > mx) mx = v;
+        }
+        float lo = alpha[g] * mn;
+        float hi = alpha[g] * mx;
+        lo = lo + 0.0f;
+        hi = hi + 0.0f;
+        float h32 = (hi - lo) / (float)qmax;
+        uint16_t h16 = orc_f32_to_f16(h32);
+        uint16_t z16 = orc_f32_to_f16(lo);
+        float hf = orc_f16_to_f32(h16);
+        float zf = orc_f16_to_f32(z16);
+        meta[2 * g + 0] = h16;
+        meta[2 * g + 1] = z16;
+        for (int j = g * G; j < (g + 1) * G; ++j) {
+            int c = 0;
+            if (hf != 0.0f) {
+                float x = orc_f16_to_f32(xr[j]);
+                float d = x - zf;
+                float r = rintf(d / hf);
+                if (r < 0.0f) r = 0.0f;
+                if (r > (float)qmax) r = (float)qmax;
+                c = (int)r;
+            }
+            int bit = j * bits;
+            codes[bit >> 3] |= (uint8_t)(c << (bit & 7));
+        }
+    }
+}
+
+/* Code j of a packed row. */
+static int orc_code_at(const uint8_t *codes, int j, int bits)
+{
+    int bit = j * bits;
+    return (codes[bit >> 3] >> (bit & 7)) & ((1 << bits) - 1);
+}
+
+/* Dequantize one row to fp64 without rounding: x^ = h*c + z. */
+void orc_dequant_row(const uint8_t *codes, const uint16_t *meta, int D, int G, int bits, double *out)
+{
+    for (int j = 0; j < D; ++j) {
+        int g = j / G;
+        double h = (double)orc_f16_to_f32(meta[2 * g + 0]);
+        double z = (double)orc_f16_to_f32(meta[2 * g + 1]);
+        out[j] = h * (double)orc_code_at(codes, j, bits) + z;
+    }
+}
+
+/* Reorder then quantize n independent rows (no cache state); for unit tests. */
+void orc_quantize_rows(const uint16_t *x, int n, const int32_t *idx, const float *alpha, int D, int G,
+                       int bits, uint8_t *codes, uint16_t *meta)
+{
+    uint16_t *tmp = (uint16_t *)malloc(sizeof(uint16_t) * (size_t)D);
+    for (int r = 0; r < n; ++r) {
+        orc_reorder_row(x + (size_t)r * D, idx, D, tmp);
+        orc_quantize_reordered_row(tmp, alpha, D, G, bits, codes + (size_t)r * (D * bits / 8),
+                                   meta + (size_t)r * (D / G) * 2);
+    }
+    free(tmp);
+}
+
+/* ---------------------------------------------------------------- cache state */
+
+typedef struct {
+    int B, Hkv, D, G, W, cap_q; /* cap_q: rows available in the quantized segment */
+    int k_bits, v_bits;
+    uint8_t *k_codes, *v_codes;
+    uint16_t *k_meta, *v_meta;
+    uint16_t *k_win, *v_win;
+    int32_t *lengths;
+    const int32_t *reorder_k, *reorder_v; /* [Hkv][D] */
+    const float *alpha_k, *alpha_v;       /* [Hkv][D/G] */
+} orc_cache;
+
+static size_t orc_row_index(const orc_cache *c, int b, int h, int t, int rows)
+{
+    return ((size_t)b * c->Hkv + h) * (size_t)rows + (size_t)t;
+}
+
+/*
+ * Sliding-window append (Sec. 3.2 and the body of Algorithm 1).  The n_new[b]
+ * new tokens of sequence b are concatenated after the L0 tokens already there;
+ * every token in [processed, L1 - W) is quantized, where processed =
+ * max(0, L0 - W) is what earlier calls already quantized, and the last
+ * min(L1, W) tokens are left in full precision in the ring.
+ * k, v: fp16 bits [B][n_stride][Hkv][D] in the model's original channel order.
+ * Returns 0, or -1 if a sequence would exceed its capacity (nothing is changed
+ * for that sequence).
+ */
+int orc_append(orc_cache *c, const uint16_t *k, const uint16_t *v, const int32_t *n_new, int n_stride)
+{
+    const int D = c->D, W = c->W, ng = c->D / c->G;
+    int status = 0;
+    for (int b = 0; b < c->B; ++b) {
+        const int L0 = c->lengths[b];
+        const int L1 = L0 + n_new[b];
+        const int processed = L0 - W > 0 ? L0 - W : 0;
+        const int q_end = L1 - W > 0 ? L1 - W : 0;
+        if (q_end > c->cap_q || n_new[b] > n_stride || n_new[b] < 0) {
+            status = -1;
+            continue;
+        }
+#pragma omp parallel for schedule(static)
+        for (int h = 0; h < c->Hkv; ++h) {
+            uint16_t *rowk = (uint16_t *)malloc(sizeof(uint16_t) * (size_t)D);
+            uint16_t *rowv = (uint16_t *)malloc(sizeof(uint16_t) * (size_t)D);
+            /* 1. quantize what slides out of the window, oldest first */
+            for (int t = processed; t < q_end; ++t) {
+                if (t < L0) { /* still sitting in the ring, already reordered */
+                    size_t s = orc_row_index(c, b, h, t % W, W) * (size_t)D;
+                    memcpy(rowk, c->k_win + s, sizeof(uint16_t) * (size_t)D);
+                    memcpy(rowv, c->v_win + s, sizeof(uint16_t) * (size_t)D);
+                } else {      /* one of the new tokens */
+                    size_t s = (((size_t)b * n_stride + (size_t)(t - L0)) * c->Hkv + h) * (size_t)D;
+                    orc_reorder_row(k + s, c->reorder_k + (size_t)h * D, D, rowk);
+                    orc_reorder_row(v + s, c->reorder_v + (size_t)h * D, D, rowv);
+                }
+                size_t r = orc_row_index(c, b, h, t, c->cap_q);
+                orc_quantize_reordered_row(rowk, c->alpha_k + (size_t)h * ng, D, c->G, c->k_bits,
+                                           c->k_codes + r * (size_t)(D * c->k_bits / 8),
+                                           c->k_meta + r * (size_t)ng * 2);
+                orc_quantize_reordered_row(rowv, c->alpha_v + (size_t)h * ng, D, c->G, c->v_bits,
+                                           c->v_codes + r * (size_t)(D * c->v_bits / 8),
+                                           c->v_meta + r * (size_t)ng * 2);
+            }
+            /* 2. the new tokens that remain inside the window go to the ring */
+            int first_kept = q_end > L0 ? q_end : L0;
+            for (int t = first_kept; t < L1; ++t) {
+                size_t s = (((size_t)b * n_stride + (size_t)(t - L0)) * c->Hkv + h) * (size_t)D;
+                size_t d = orc_row_index(c, b, h, t % W, W) * (size_t)D;
+                orc_reorder_row(k + s, c->reorder_k + (size_t)h * D, D, c->k_win + d);
+                orc_reorder_row(v + s, c->reorder_v + (size_t)h * D, D, c->v_win + d);
+            }
+            free(rowk);
+            free(rowv);
+        }
+        c->lengths[b] = L1;
+    }
+    return status;
+}
+
+/*
+ * Decode attention for one query per sequence (Eq. 1 and the first lines of
+ * Algorithm 1, with the softmax and its scale written out):
+ *   q'      = q[reorder_k]                       (same permutation as the keys)
+ *   s_t     = sm_scale * sum_j q'_j K~_{t,j}      K~ = h*c+z for t < L-W, fp16 window otherwise
+ *   p       = softmax(s) over all t < L
+ *   o'_j    = sum_t p_t V~_{t,j}
+ *   out[reorder_v[j]] = o'_j                      (undo the value permutation)
+ * q: fp16 bits [B][Hq][D]; out: fp64 [B][Hq][D].  Query head hq reads KV head
+ * hq / (Hq / Hkv).  A sequence of length 0 yields zeros.
+ */
+void orc_attention(const orc_cache *c, int Hq, const uint16_t *q, double sm_scale, double *out)
+{
+    const int D = c->D, W = c->W, ng = c->D / c->G;
+    const int rep = Hq / c->Hkv;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int b = 0; b < c->B; ++b) {
+        for (int hq = 0; hq < Hq; ++hq) {
+            const int hk = hq / rep;
+            const int L = c->lengths[b];
+            const int Lq = L - W > 0 ? L - W : 0;
+            double *o = out + ((size_t)b * Hq + hq) * (size_t)D;
+            for (int j = 0; j < D; ++j) o[j] = 0.0;
+            if (L <= 0) continue;
+            double *qp = (double *)malloc(sizeof(double) * (size_t)D);
+            double *row = (double *)malloc(sizeof(double) * (size_t)D);
+            double *s = (double *)malloc(sizeof(double) * (size_t)L);
+            double *acc = (double *)calloc((size_t)D, sizeof(double));
+            const int32_t *ik = c->reorder_k + (size_t)hk * D;
+            const int32_t *iv = c->reorder_v + (size_t)hk * D;
+            for (int j = 0; j < D; ++j)
+                qp[j] = (double)orc_f16_to_f32(q[((size_t)b * Hq + hq) * (size_t)D + ik[j]]);
+            /* scores */
+            for (int t = 0; t < L; ++t) {
+                if (t < Lq) {
+                    size_t r = orc_row_index(c, b, hk, t, c->cap_q);
+                    orc_dequant_row(c->k_codes + r * (size_t)(D * c->k_bits / 8),
+                                    c->k_meta + r * (size_t)ng * 2, D, c->G, c->k_bits, row);
+                } else {
+                    size_t w = orc_row_index(c, b, hk, t % W, W) * (size_t)D;
+                    for (int j = 0; j < D; ++j) row[j] = (double)orc_f16_to_f32(c->k_win[w + j]);
+                }
+                double d = 0.0;
+                for (int j = 0; j < D; ++j) d += qp[j] * row[j];
+                s[t] = sm_scale * d;
+            }
+            /* softmax */
+            double m = s[0];
+            for (int t = 1; t < L; ++t) if (s[t] > m) m = s[t];
+            double denom = 0.0;
+            for (int t = 0; t < L; ++t) { s[t] = exp(s[t] - m); denom += s[t]; }
+            /* weighted sum of values */
+            for (int t = 0; t < L; ++t) {
+                if (t < Lq) {
+                    size_t r = orc_row_index(c, b, hk, t, c->cap_q);
+                    orc_dequant_row(c->v_codes + r * (size_t)(D * c->v_bits / 8),
+                                    c->v_meta + r * (size_t)ng * 2, D, c->G, c->v_bits, row);
+                } else {
+                    size_t w = orc_row_index(c, b, hk, t % W, W) * (size_t)D;
+                    for (int j = 0; j < D; ++j) row[j] = (double)orc_f16_to_f32(c->v_win[w + j]);
+                }
+                double p = s[t] / denom;
+                for (int j = 0; j < D; ++j) acc[j] += p * row[j];
+            }
+            for (int j = 0; j < D; ++j) o[iv[j]] = acc[j];
+            free(qp); free(row); free(s); free(acc);
+        }
+    }
+}
+
+/* Threads the parallel loops above will use (1 without OpenMP). */
+int orc_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}

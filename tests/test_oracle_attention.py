@@ -1,0 +1,245 @@
+"""Pins for the CPU oracle's sliding-window cache and its fp64 attention.
+
+The cache semantics are checked against the paper's statement (latest W tokens stay
+fp16, everything older is quantized, single appends equal one bulk append); the
+attention against library routines (scipy softmax + einsum, torch SDPA in fp64),
+and against properties that hold for any softmax attention.
+"""
+import numpy as np
+import pytest
+import scipy.special
+
+from oracle import skvq_oracle as orc
+from paper_2405_06219_b200 import workloads
+from test_oracle_quantizer import unpack_codes
+
+D = 128
+
+
+def make_cache(B, Hq, Hkv, W, cap, bits=2, group=128, alpha=0.9, seed=0, identity=False):
+    rng = np.random.default_rng(seed)
+    if identity:
+        rk = rv = np.tile(np.arange(D, dtype=np.int32), (Hkv, 1))
+    else:
+        rk = np.stack([rng.permutation(D) for _ in range(Hkv)]).astype(np.int32)
+        rv = np.stack([rng.permutation(D) for _ in range(Hkv)]).astype(np.int32)
+    a = np.full((Hkv, D // group), alpha, np.float32)
+    return orc.OracleCache(B, Hq, Hkv, D, bits, bits, group, W, cap, rk, rv, a, a)
+
+
+def rand_kv(B, n, Hkv, seed):
+    rng = np.random.default_rng(seed)
+    sigma = np.exp(0.5 * rng.standard_normal((Hkv, D))).astype(np.float32)
+    sigma[:, :3] *= 15
+    k = (rng.standard_normal((B, n, Hkv, D)).astype(np.float32) * sigma).astype(np.float16)
+    v = rng.standard_normal((B, n, Hkv, D)).astype(np.float16)
+    return k, v
+
+
+def cache_state(c):
+    return [c.k_codes.copy(), c.v_codes.copy(), c.k_meta.view(np.uint16).copy(), c.v_meta.view(np.uint16).copy(),
+            c.k_win.view(np.uint16).copy(), c.v_win.view(np.uint16).copy(), c.lengths.copy()]
+
+
+def mixed_cache_dense(c, b, hk):
+    """Independent numpy reconstruction of K~ and V~ (reordered order) for one (sequence, KV head)."""
+    L = int(c.lengths[b])
+    Lq = max(L - c.W, 0)
+    out = []
+    for codes, meta, win, bits in ((c.k_codes, c.k_meta, c.k_win, c.k_bits), (c.v_codes, c.v_meta, c.v_win, c.v_bits)):
+        code = unpack_codes(codes[b, hk, :Lq], bits).astype(np.float64)
+        h = np.repeat(meta[b, hk, :Lq, :, 0].astype(np.float64), c.G, axis=1)
+        z = np.repeat(meta[b, hk, :Lq, :, 1].astype(np.float64), c.G, axis=1)
+        dense = np.zeros((L, D))
+        dense[:Lq] = h * code + z
+        for t in range(Lq, L):
+            dense[t] = win[b, hk, t % c.W].astype(np.float64)
+        out.append(dense)
+    return out
+
+
+def brute_attention(c, q, sm_scale):
+    out = np.zeros((c.B, c.Hq, D))
+    rep = c.Hq // c.Hkv
+    for b in range(c.B):
+        if c.lengths[b] == 0:
+            continue
+        for hq in range(c.Hq):
+            hk = hq // rep
+            Kt, Vt = mixed_cache_dense(c, b, hk)
+            qp = q[b, hq].astype(np.float64)[c.reorder_k[hk]]
+            p = scipy.special.softmax(float(np.float32(sm_scale)) * (Kt @ qp))
+            o = np.einsum("t,td->d", p, Vt)
+            out[b, hq, c.reorder_v[hk]] = o
+    return out
+
+
+# ------------------------------------------------------------------ window semantics (Sec. 3.2, Algorithm 1)
+@pytest.mark.parametrize("W,n", [(8, 5), (8, 8), (8, 9), (8, 37), (0, 6), (16, 40)])
+def test_window_keeps_last_w_tokens_and_quantizes_the_rest(W, n):
+    c = make_cache(2, 4, 2, W, 64, group=32, seed=1)
+    k, v = rand_kv(2, n, 2, 2)
+    assert c.append(k, v) == 0
+    assert np.all(c.lengths == n)
+    Lq = max(n - W, 0)
+    for b in range(2):
+        for h in range(2):
+            for t in range(Lq, n):                       # window: reordered fp16, slot t mod W
+                assert np.array_equal(c.k_win[b, h, t % W], k[b, t, h][c.reorder_k[h]])
+                assert np.array_equal(c.v_win[b, h, t % W], v[b, t, h][c.reorder_v[h]])
+            if Lq:
+                ck, mk = orc.quantize_rows(k[b, :Lq, h], c.reorder_k[h], c.alpha_k[h], 2, 32)
+                cv, mv = orc.quantize_rows(v[b, :Lq, h], c.reorder_v[h], c.alpha_v[h], 2, 32)
+                assert np.array_equal(c.k_codes[b, h, :Lq], ck) and np.array_equal(c.v_codes[b, h, :Lq], cv)
+                assert np.array_equal(c.k_meta[b, h, :Lq].view(np.uint16), mk.view(np.uint16))
+                assert np.array_equal(c.v_meta[b, h, :Lq].view(np.uint16), mv.view(np.uint16))
+            assert not c.k_codes[b, h, Lq:].any() and not c.v_meta[b, h, Lq:].view(np.uint16).any()
+
+
+@pytest.mark.parametrize("W", [0, 8, 16])
+def test_single_appends_equal_bulk_and_any_chunking(W):
+    n = 45
+    k, v = rand_kv(2, n, 2, 3)
+    bulk = make_cache(2, 2, 2, W, 64, seed=4)
+    bulk.append(k, v)
+    one = make_cache(2, 2, 2, W, 64, seed=4)
+    for t in range(n):
+        one.append(k[:, t:t + 1], v[:, t:t + 1])
+    chunked = make_cache(2, 2, 2, W, 64, seed=4)
+    t = 0
+    for step in (1, 7, 2, 20, 15):
+        chunked.append(k[:, t:t + step], v[:, t:t + step])
+        t += step
+    assert t == n
+    for other in (one, chunked):
+        for a, b in zip(cache_state(bulk), cache_state(other)):
+            assert np.array_equal(a, b)
+
+
+def test_ragged_append_counts_and_capacity():
+    c = make_cache(3, 2, 2, 8, 32, seed=5)
+    k, v = rand_kv(3, 30, 2, 6)
+    assert c.append(k, v, np.array([30, 0, 11], np.int32)) == 0
+    assert c.lengths.tolist() == [30, 0, 11]
+    ref = make_cache(1, 2, 2, 8, 32, seed=5)
+    ref.append(k[2:3, :11], v[2:3, :11])
+    assert np.array_equal(c.k_codes[2], ref.k_codes[0]) and np.array_equal(c.k_win[2], ref.k_win[0])
+    before = cache_state(c)
+    assert c.append(k[:, :5], v[:, :5], np.array([5, 0, 0], np.int32)) == -1      # 35 > capacity 32
+    assert c.lengths.tolist() == [30, 0, 11]
+    for a, b in zip(before, cache_state(c)):
+        assert np.array_equal(a, b)
+
+
+# ------------------------------------------------------------------ attention
+@pytest.mark.parametrize("Hq,Hkv,bits,group,W,L", [(2, 2, 2, 128, 16, 300), (4, 1, 2, 32, 8, 150),
+                                                  (4, 2, 4, 64, 32, 100), (2, 2, 2, 128, 0, 64)])
+def test_attention_matches_library_brute_force(Hq, Hkv, bits, group, W, L):
+    c = make_cache(2, Hq, Hkv, W, 320, bits=bits, group=group, seed=7)
+    k, v = rand_kv(2, L, Hkv, 8)
+    c.append(k, v, np.array([L, L - 37], np.int32))
+    q = np.random.default_rng(9).standard_normal((2, Hq, D)).astype(np.float16)
+    got = c.attention(q, 1 / np.sqrt(D))
+    want = brute_attention(c, q, 1 / np.sqrt(D))
+    assert np.abs(got - want).max() < 1e-12
+
+
+def test_all_fp16_window_reduces_to_torch_sdpa():
+    """W >= L: nothing is quantized and the call is plain attention; torch's fp64 SDPA is the reference."""
+    import torch
+    L, Hq, Hkv = 50, 4, 2
+    c = make_cache(2, Hq, Hkv, 64, 64, seed=10)
+    k, v = rand_kv(2, L, Hkv, 11)
+    c.append(k, v)
+    assert not c.k_codes.any()
+    q = np.random.default_rng(12).standard_normal((2, Hq, D)).astype(np.float16)
+    got = c.attention(q, 0.11)
+    tq = torch.from_numpy(q.astype(np.float64))[:, :, None, :]                        # [B,Hq,1,D]
+    tk = torch.from_numpy(k.astype(np.float64)).permute(0, 2, 1, 3).repeat_interleave(Hq // Hkv, 1)
+    tv = torch.from_numpy(v.astype(np.float64)).permute(0, 2, 1, 3).repeat_interleave(Hq // Hkv, 1)
+    want = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, scale=float(np.float32(0.11)))[:, :, 0].numpy()
+    assert np.abs(got - want).max() < 1e-12
+
+
+def test_reorder_leaves_attention_unchanged_when_nothing_is_quantized():
+    """Eq. 1: permuting q and K channels alike, and un-permuting the V output, changes nothing."""
+    L, H = 40, 2
+    k, v = rand_kv(1, L, H, 13)
+    q = np.random.default_rng(14).standard_normal((1, H, D)).astype(np.float16)
+    a = make_cache(1, H, H, 64, 64, seed=15)
+    b = make_cache(1, H, H, 64, 64, identity=True)
+    a.append(k, v)
+    b.append(k, v)
+    assert np.abs(a.attention(q, 0.1) - b.attention(q, 0.1)).max() < 1e-13
+
+
+def test_zero_query_gives_mean_of_values_and_outputs_are_convex():
+    c = make_cache(1, 2, 2, 16, 128, seed=16)
+    k, v = rand_kv(1, 90, 2, 17)
+    c.append(k, v)
+    out0 = c.attention(np.zeros((1, 2, D), np.float16), 0.3)
+    q = np.random.default_rng(18).standard_normal((1, 2, D)).astype(np.float16)
+    out = c.attention(q, 0.3)
+    for h in range(2):
+        _, Vt = mixed_cache_dense(c, 0, h)
+        inv = np.empty(D, np.int64)
+        inv[c.reorder_v[h]] = np.arange(D)
+        Vorig = Vt[:, inv]                                                          # back to original channel order
+        assert np.abs(out0[0, h] - Vorig.mean(0)).max() < 1e-12
+        assert np.all(out[0, h] <= Vorig.max(0) + 1e-12) and np.all(out[0, h] >= Vorig.min(0) - 1e-12)
+
+
+def test_dominant_key_selects_its_value_row_and_score_shift_is_invisible():
+    H, L, W = 1, 70, 8
+    k, v = rand_kv(1, L, H, 19)
+    k = (k.astype(np.float32) * 0.05).astype(np.float16)
+    k[:, :, :, 0] = 1.0                      # a channel on which all keys agree
+    k[0, 20] = 0
+    k[0, 20, 0, 0] = 1.0
+    k[0, 20, 0, 1] = 40.0                    # token 20 dominates for a query along channel 1
+    c = make_cache(1, H, H, W, 128, alpha=1.0, identity=True)
+    c.append(k, v)
+    q = np.zeros((1, H, D), np.float16)
+    q[0, 0, 1] = 30.0
+    out = c.attention(q, 1.0)
+    _, Vt = mixed_cache_dense(c, 0, 0)
+    assert np.abs(out[0, 0] - Vt[20]).max() < 1e-9
+    # adding a multiple of a channel on which all keys agree shifts every score alike (nothing quantized here)
+    c2 = make_cache(1, H, H, 128, 128, alpha=1.0, seed=22)
+    c2.append(k, v)
+    q2 = q.copy()
+    q2[0, 0, 0] = 7.0
+    q[0, 0, 1] = 0.5
+    q2[0, 0, 1] = 0.5
+    assert np.abs(c2.attention(q, 1.0) - c2.attention(q2, 1.0)).max() < 1e-9
+
+
+def test_empty_sequence_gives_zeros():
+    c = make_cache(2, 2, 2, 8, 32, seed=20)
+    k, v = rand_kv(2, 12, 2, 21)
+    c.append(k, v, np.array([0, 12], np.int32))
+    out = c.attention(np.ones((2, 2, D), np.float16), 0.1)
+    assert not out[0].any() and out[1].any()
+
+
+# ------------------------------------------------------------------ workload generator (no method arithmetic)
+def test_workload_generator_is_deterministic_and_chunk_invariant():
+    w = workloads.configs()[2].scaled(context=10000, batch=2)
+    a = w.tokens("k", 1, 4000, 9000)
+    b = np.concatenate([w.tokens("k", 1, 4000, 4096), w.tokens("k", 1, 4096, 8192), w.tokens("k", 1, 8192, 9000)])
+    assert np.array_equal(a.view(np.uint16), b.view(np.uint16))
+    assert not np.array_equal(w.tokens("k", 0, 0, 16), w.tokens("v", 0, 0, 16))
+    idx = w.reorder_index("k")
+    assert idx.shape == (8, 128) and all(sorted(r.tolist()) == list(range(128)) for r in idx)
+    sig = w.key_sigma()
+    assert ((sig > 4).sum(1) >= 8).all() and (sig > 4).sum() < 8 * 12
+    lens = workloads.configs()[4].lengths()
+    assert lens.shape == (64,) and lens.min() >= 1024 and lens.max() <= 16384
+
+
+def test_algorithmic_bytes_match_stated_sizes():
+    cf = workloads.configs()
+    assert abs(workloads.algorithmic_bytes(cf[0]) / 1e6 - 11.26) < 0.02
+    assert abs(workloads.algorithmic_bytes(cf[1]) / 1e6 - 618.5) < 0.5
+    assert abs(workloads.algorithmic_bytes(cf[2]) / 1e6 - 404.4) < 0.5
+    assert abs(workloads.algorithmic_bytes(cf[3]) / 1e6 - 2417.7) < 0.5

@@ -1,0 +1,268 @@
+"""Pins for the CPU oracle's quantizer: what the paper and plain mathematics fix.
+
+Each test checks the oracle against something other than itself: numpy's own fp16
+conversion, hand-derived closed forms, a brute-force nearest-level search, the
+paper's printed average-bit arithmetic, or a property of the definition.
+"""
+import os
+
+import numpy as np
+import pytest
+
+from oracle import skvq_oracle as orc
+
+D = 128
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def unpack_codes(codes: np.ndarray, bits: int) -> np.ndarray:
+    """Independent numpy unpack: code j = bits [(j*bits) mod 8, +bits) of byte (j*bits)//8."""
+    n, nbytes = codes.shape
+    bitsarr = np.unpackbits(codes, axis=1, bitorder="little")          # [n, nbytes*8], LSB first
+    bitsarr = bitsarr.reshape(n, nbytes * 8 // bits, bits)
+    weights = (1 << np.arange(bits)).astype(np.int64)
+    return (bitsarr * weights).sum(axis=2)
+
+
+def ident():
+    return np.arange(D, dtype=np.int32)
+
+
+# ------------------------------------------------------------------ fp16 conversions
+def test_f16_to_f32_all_patterns_match_numpy():
+    bits = np.arange(65536, dtype=np.uint16)
+    want = bits.view(np.float16).astype(np.float32)
+    got = np.array([orc.f16_bits_to_f32(int(b)) for b in bits], dtype=np.float32)
+    nan = np.isnan(want)
+    assert np.array_equal(np.isnan(got), nan)
+    assert np.array_equal(got[~nan].view(np.uint32), want[~nan].view(np.uint32))
+
+
+def test_f32_to_f16_matches_numpy_round_to_nearest_even():
+    rng = np.random.default_rng(1)
+    xs = np.concatenate([
+        rng.standard_normal(20000).astype(np.float32) * np.float32(10.0) ** rng.integers(-9, 5, 20000),
+        np.array([0.0, -0.0, 65504.0, 65519.9, 65520.0, 70000.0, -65520.0, 2.0 ** -24, 2.0 ** -25,
+                  1.5 * 2.0 ** -25, 2.0 ** -14, 6.1e-5, 1.00048828125, 1.000732421875, 2049.0, 2051.0],
+                 dtype=np.float32),
+        # exact ties between neighbouring halves: (2k+1) * 2^-11 around 1.0
+        (1.0 + (2 * np.arange(64) + 1) * 2.0 ** -11).astype(np.float32),
+    ]).astype(np.float32)
+    with np.errstate(over="ignore"):
+        want = xs.astype(np.float16).view(np.uint16)
+    got = np.array([orc.f32_to_f16_bits(float(x)) for x in xs], dtype=np.uint16)
+    assert np.array_equal(got, want)
+
+
+# ------------------------------------------------------------------ closed forms
+@pytest.mark.parametrize("bits", [2, 4])
+def test_lossless_arithmetic_progression(bits):
+    """A group holding exactly the 2^bits levels a + k*d (d a power of two), alpha = 1: h = d, z = a, code = k."""
+    qmax = (1 << bits) - 1
+    a, d = -1.5, 0.25
+    ks = np.arange(D) % (qmax + 1)
+    x = (a + ks * d).astype(np.float16)[None]
+    codes, meta = orc.quantize_rows(x, ident(), np.ones(1, np.float32), bits, D)
+    assert np.array_equal(unpack_codes(codes, bits)[0], ks)
+    assert float(meta[0, 0, 0]) == d and float(meta[0, 0, 1]) == a
+    assert np.array_equal(orc.dequant_rows(codes, meta, bits, D)[0], x[0].astype(np.float64))
+
+
+def test_pack_layout_golden_bytes():
+    """Codes 0,1,2,3 repeated: every 2-bit byte is 0b11100100; 4-bit codes 0..15: bytes 0x10, 0x32, ..."""
+    x2 = (np.arange(D) % 4).astype(np.float16)[None]
+    codes, _ = orc.quantize_rows(x2, ident(), np.ones(1, np.float32), 2, D)
+    assert codes.shape == (1, 32) and np.all(codes == 0xE4)
+    x4 = (np.arange(D) % 16).astype(np.float16)[None]
+    codes, _ = orc.quantize_rows(x4, ident(), np.ones(1, np.float32), 4, D)
+    want = np.array([0x10, 0x32, 0x54, 0x76, 0x98, 0xBA, 0xDC, 0xFE] * 8, dtype=np.uint8)
+    assert codes.shape == (1, 64) and np.array_equal(codes[0], want)
+
+
+@pytest.mark.parametrize("bits", [2, 4])
+def test_constant_group_is_degenerate(bits):
+    x = np.full((1, D), 0.7314, dtype=np.float16)
+    codes, meta = orc.quantize_rows(x, ident(), np.full(1, 1.0, np.float32), bits, D)
+    assert np.all(codes == 0)
+    assert float(meta[0, 0, 0]) == 0.0 and meta[0, 0, 1] == x[0, 0]
+    assert np.all(orc.dequant_rows(codes, meta, bits, D) == float(x[0, 0]))
+
+
+@pytest.mark.parametrize("bits", [2, 4])
+def test_two_valued_group_hits_both_ends(bits):
+    qmax = (1 << bits) - 1
+    rng = np.random.default_rng(3)
+    pick = rng.integers(0, 2, D)
+    pick[:2] = [0, 1]
+    x = np.where(pick == 1, 3.0, -1.5).astype(np.float16)[None]
+    codes, _ = orc.quantize_rows(x, ident(), np.ones(1, np.float32), bits, D)
+    assert np.array_equal(unpack_codes(codes, bits)[0], pick * qmax)
+
+
+def test_zero_sign_is_canonical():
+    """A group whose minimum is -0 or +0 stores the same (positive) zero point."""
+    x = np.zeros((2, D), dtype=np.float16)
+    x[0, :] = np.float16(-0.0)
+    x[0, 5] = 1.0
+    x[1, 5] = 1.0
+    x[1, 9] = np.float16(-0.0)
+    _, meta = orc.quantize_rows(x, ident(), np.ones(1, np.float32), 2, D)
+    assert meta.view(np.uint16)[0, 0, 1] == 0 and meta.view(np.uint16)[1, 0, 1] == 0
+
+
+# ------------------------------------------------------------------ definition-level properties
+def random_rows(n, seed, outliers=True):
+    rng = np.random.default_rng(seed)
+    sigma = np.exp(0.5 * rng.standard_normal(D)).astype(np.float32)
+    if outliers:
+        sigma[rng.choice(D, 4, replace=False)] *= 15.0
+    return (rng.standard_normal((n, D)).astype(np.float32) * sigma).astype(np.float16)
+
+
+@pytest.mark.parametrize("bits,group,alpha", [(2, 128, 0.9), (2, 32, 0.85), (4, 64, 0.95), (2, 64, 1.0), (4, 128, 1.0)])
+def test_stored_parameters_follow_eq2(bits, group, alpha):
+    """h = alpha*(max-min)/qmax and z = alpha*min (Eq. 2 / clipping_quant), stored as fp16.
+    The expected values are formed in fp64 straight from the definition; fp32 intermediate
+    rounding can move the fp16 result by at most one unit in the last place."""
+    qmax = (1 << bits) - 1
+    x = random_rows(64, 10 + bits + group)
+    ng = D // group
+    _, meta = orc.quantize_rows(x, ident(), np.full(ng, alpha, np.float32), bits, group)
+    xg = x.astype(np.float64).reshape(64, ng, group)
+    a = float(np.float32(alpha))
+    h_want = (a * (xg.max(2) - xg.min(2)) / qmax)
+    z_want = a * xg.min(2)
+    h_got, z_got = meta[..., 0].astype(np.float64), meta[..., 1].astype(np.float64)
+    ulp_h = np.spacing(np.abs(h_want).astype(np.float16)).astype(np.float64)
+    ulp_z = np.spacing(np.abs(z_want).astype(np.float16)).astype(np.float64)
+    assert np.all(np.abs(h_got - h_want) <= 0.5 * ulp_h * 1.01 + 1e-12)
+    assert np.all(np.abs(z_got - z_want) <= 0.5 * ulp_z * 1.01 + 1e-12)
+    exact = (h_got == h_want.astype(np.float16).astype(np.float64)).mean()
+    assert exact > 0.99
+    assert np.all(h_got >= 0)
+
+
+@pytest.mark.parametrize("bits,group,alpha", [(2, 128, 0.9), (2, 32, 0.85), (4, 64, 0.95), (2, 128, 1.0), (4, 32, 1.0)])
+def test_codes_are_nearest_level_brute_force(bits, group, alpha):
+    """Brute force over all 2^bits levels: the stored code is (one of) the nearest reconstruction
+    levels h*c+z to x, which also gives |x^ - x| <= h/2 inside the clipped range and the end
+    point outside it (uniform quantizer of Sec. 3.1)."""
+    qmax = (1 << bits) - 1
+    x = random_rows(96, 20 + bits + group)
+    ng = D // group
+    codes, meta = orc.quantize_rows(x, ident(), np.full(ng, alpha, np.float32), bits, group)
+    c = unpack_codes(codes, bits)
+    assert c.min() >= 0 and c.max() <= qmax
+    h = np.repeat(meta[..., 0].astype(np.float64), group, axis=1)
+    z = np.repeat(meta[..., 1].astype(np.float64), group, axis=1)
+    xd = x.astype(np.float64)
+    levels = h[..., None] * np.arange(qmax + 1) + z[..., None]            # [n, D, levels]
+    err_all = np.abs(levels - xd[..., None])
+    err_got = np.abs(h * c + z - xd)
+    slack = 4 * np.finfo(np.float32).eps * (np.abs(xd) + np.abs(z) + qmax * h) + 1e-30
+    assert np.all(err_got <= err_all.min(axis=2) + slack)
+    inside = (xd >= z) & (xd <= z + qmax * h)
+    assert np.all(err_got[inside] <= 0.5 * h[inside] + slack[inside])
+    below, above = xd < z, xd > z + qmax * h
+    assert np.all(c[below & (h > 0)] == 0) and np.all(c[above & (h > 0)] == qmax)
+    if alpha < 1.0:
+        assert above.any() or below.any()                                  # clipping really clips
+    # dequantization is exactly h*c+z in fp64
+    assert np.array_equal(orc.dequant_rows(codes, meta, bits, group), h * c + z)
+
+
+@pytest.mark.parametrize("bits", [2, 4])
+def test_alpha_one_full_group_is_textbook_per_token_minmax(bits):
+    """alpha = 1, one group per token, identity order: plain per-token asymmetric min-max
+    round-to-nearest (the dynamic quantization of Sec. 3.1).  Away from rounding ties the codes
+    equal round((x - min) / ((max - min) / qmax)) evaluated in fp64."""
+    qmax = (1 << bits) - 1
+    x = random_rows(128, 5, outliers=False)
+    codes, _ = orc.quantize_rows(x, ident(), np.ones(1, np.float32), bits, D)
+    c = unpack_codes(codes, bits)
+    xd = x.astype(np.float64)
+    mn, mx = xd.min(1, keepdims=True), xd.max(1, keepdims=True)
+    u = (xd - mn) / ((mx - mn) / qmax)
+    want = np.clip(np.rint(u), 0, qmax).astype(np.int64)
+    near_tie = np.abs(u - np.floor(u) - 0.5) < 2e-3 * (qmax + 1)          # fp16 rounding of h moves these
+    assert near_tie.mean() < 0.15
+    assert np.array_equal(c[~near_tie], want[~near_tie])
+    assert np.all(np.abs(c - want)[near_tie] <= 1)
+    # the row minimum and maximum land on the end codes
+    assert np.all(c[np.arange(128), xd.argmin(1)] == 0) and np.all(c[np.arange(128), xd.argmax(1)] == qmax)
+
+
+def test_codes_monotone_within_group():
+    x = random_rows(32, 7)
+    codes, _ = orc.quantize_rows(x, ident(), np.full(4, 0.85, np.float32), 2, 32)
+    c = unpack_codes(codes, 2).reshape(32, 4, 32)
+    xg = x.astype(np.float64).reshape(32, 4, 32)
+    order = np.argsort(xg, axis=2, kind="stable")
+    assert np.all(np.diff(np.take_along_axis(c, order, axis=2), axis=2) >= 0)
+
+
+def test_groups_are_independent_and_contiguous():
+    """Changing channels of one group changes only that group's codes and parameters."""
+    x = random_rows(4, 8)
+    y = x.copy()
+    y[:, 32:64] = (y[:, 32:64].astype(np.float32) * 3 + 1).astype(np.float16)
+    a = np.full(4, 0.9, np.float32)
+    c1, m1 = orc.quantize_rows(x, ident(), a, 2, 32)
+    c2, m2 = orc.quantize_rows(y, ident(), a, 2, 32)
+    same_bytes = np.ones(32, bool)
+    same_bytes[8:16] = False                                              # channels 32..63 = bytes 8..15
+    assert np.array_equal(c1[:, same_bytes], c2[:, same_bytes])
+    assert np.array_equal(m1[:, [0, 2, 3]], m2[:, [0, 2, 3]]) and not np.array_equal(m1[:, 1], m2[:, 1])
+
+
+def test_per_group_alpha_is_used_per_group():
+    x = random_rows(8, 9)
+    a = np.array([1.0, 0.5, 0.75, 0.9], np.float32)
+    _, m = orc.quantize_rows(x, ident(), a, 2, 32)
+    xg = x.astype(np.float64).reshape(8, 4, 32)
+    z_want = (a[None].astype(np.float64) * xg.min(2)).astype(np.float32).astype(np.float16)
+    assert np.array_equal(m[..., 1], z_want)
+
+
+# ------------------------------------------------------------------ reorder
+def test_reorder_is_a_gather_by_index():
+    """stored[j] = src[idx[j]]: with one group per channel-pair the parameters expose the order."""
+    rng = np.random.default_rng(11)
+    idx = rng.permutation(D).astype(np.int32)
+    x = random_rows(16, 12)
+    a = np.full(D // 32, 0.9, np.float32)
+    c_re, m_re = orc.quantize_rows(x, idx, a, 4, 32)
+    c_id, m_id = orc.quantize_rows(np.ascontiguousarray(x[:, idx]), ident(), a, 4, 32)
+    assert np.array_equal(c_re, c_id) and np.array_equal(m_re.view(np.uint16), m_id.view(np.uint16))
+    # and it is not the scatter direction
+    inv = np.argsort(idx).astype(np.int32)
+    c_sc, _ = orc.quantize_rows(np.ascontiguousarray(x[:, inv]), ident(), a, 4, 32)
+    assert not np.array_equal(c_re, c_sc)
+
+
+def test_reorder_with_single_group_only_permutes_codes():
+    """With G = D the group statistics ignore order, so reordering permutes the codes and nothing else."""
+    rng = np.random.default_rng(13)
+    idx = rng.permutation(D).astype(np.int32)
+    x = random_rows(16, 14)
+    a = np.full(1, 0.9, np.float32)
+    c_re, m_re = orc.quantize_rows(x, idx, a, 2, D)
+    c_id, m_id = orc.quantize_rows(x, ident(), a, 2, D)
+    assert np.array_equal(m_re.view(np.uint16), m_id.view(np.uint16))
+    assert np.array_equal(unpack_codes(c_re, 2), unpack_codes(c_id, 2)[:, idx])
+
+
+# ------------------------------------------------------------------ the paper's storage arithmetic
+def test_average_bits_match_paper():
+    """bits/element of what the cache stores = N + (bits of h + bits of z) / G; the golden file holds
+    the figures the paper prints (ablation text and group-size table)."""
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "avg_bits.txt")) if l.strip() and not l.startswith("#")]
+    for bits, group, param_bits, want in rows:
+        bits, group, param_bits, want = int(bits), int(group), int(param_bits), float(want)
+        x = random_rows(2, 15)
+        codes, meta = orc.quantize_rows(x, ident(), np.ones(D // group, np.float32), bits, group)
+        n_params = meta.shape[1] * meta.shape[2]
+        stored_bits = codes.shape[1] * 8 + n_params * param_bits          # per row, params at the stated width
+        assert stored_bits / D == pytest.approx(want, abs=1e-12)
+        if param_bits == 16:                                              # what the oracle really stores
+            assert (codes[0].nbytes + meta[0].nbytes) * 8 / D == pytest.approx(want, abs=1e-12)
