@@ -1,0 +1,166 @@
+/*
+ * skvq.h -- C ABI of the B200-native SKVQ hot path (sliding-window KV-cache
+ * quantization, arXiv 2405.06219): append tokens to a cache whose older part is
+ * 2/4-bit group-quantized, and run decode attention directly on that cache.
+ *
+ * General rules
+ *   - Every pointer is a DEVICE pointer owned by the caller unless its comment
+ *     says "host".  The library allocates nothing, frees nothing and keeps no
+ *     pointer after a call returns.
+ *   - Every device buffer must be 16-byte aligned.
+ *   - Calls only enqueue work on `cuda_stream` (a cudaStream_t passed as void*,
+ *     NULL = the default stream); they never synchronise.  Lengths are read on
+ *     the device.
+ *   - Return value: SKVQ_OK or a negative SKVQ_ERR_* code.  On an error nothing
+ *     is launched.  Conditions only the device can see (a sequence that would
+ *     exceed its capacity) leave that sequence untouched and OR a bit into
+ *     skvq_cache::status.
+ *   - Compiled for sm_100a only; there is no CPU path.
+ *
+ * Notation: B sequences, Hq query heads, Hkv KV heads (Hq % Hkv == 0, query head
+ * hq reads KV head hq / (Hq/Hkv)), D = head_dim, W = window, G = group size,
+ * ng = D/G groups per row, L_b = lengths[b], Lq_b = max(L_b - W, 0) quantized
+ * tokens of sequence b.
+ */
+#ifndef SKVQ_H_
+#define SKVQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SKVQ_OK 0
+#define SKVQ_ERR_INVALID_ARG (-1) /* NULL where a buffer is required, negative size, ... */
+#define SKVQ_ERR_UNSUPPORTED (-2) /* head_dim != 128, bits not in {2,4}, G not in {32,64,128}, Hq % Hkv != 0, Hq/Hkv > 8 */
+#define SKVQ_ERR_MISALIGNED (-3)  /* a device buffer is not 16-byte aligned */
+#define SKVQ_ERR_CAPACITY (-4)    /* host-visible overflow: n_new or max_len_hint beyond max_tokens */
+#define SKVQ_ERR_WORKSPACE (-5)   /* workspace missing or smaller than skvq_workspace_size() */
+#define SKVQ_ERR_CUDA (-6)        /* the CUDA runtime reported an error at launch */
+
+#define SKVQ_STATUS_OVERFLOW 1    /* bit set in *status when a sequence would have exceeded max_tokens */
+
+/* Rows of the quantized segment are allocated in multiples of this many tokens so
+ * that a kernel may stage whole tiles; see skvq_quant_capacity(). */
+#define SKVQ_TOKEN_ALIGN 64
+
+/* Shape and quantization settings (host struct). */
+typedef struct skvq_config {
+    int32_t batch;       /* B >= 1 */
+    int32_t n_q_heads;   /* Hq */
+    int32_t n_kv_heads;  /* Hkv */
+    int32_t head_dim;    /* D, must be 128 */
+    int32_t k_bits;      /* 2 or 4 */
+    int32_t v_bits;      /* 2 or 4 */
+    int32_t group_size;  /* G: 32, 64 or 128 consecutive (reordered) channels share scale/zero */
+    int32_t window;      /* W >= 0 latest tokens kept in fp16 (Sec. 3.2); 0 quantizes everything */
+    int32_t max_tokens;  /* per-sequence capacity (quantized segment + window) */
+} skvq_config;
+
+/*
+ * The cache (host struct of device pointers).  cap = skvq_quant_capacity(cfg).
+ * Layouts are row-major:
+ *   k_codes/v_codes  uint8   [B][Hkv][cap][D*bits/8]  code j of a row = bits [(j*bits)%8, +bits) of
+ *                                                     byte (j*bits)/8, j counted in reordered order
+ *   k_meta/v_meta    half2   [B][Hkv][cap][ng]        {scale h, zero z}; dequantized x^ = h*code + z
+ *   k_win/v_win      half    [B][Hkv][W][D]           ring; token t sits in slot t % W, reordered order
+ *   lengths          int32   [B]                      tokens appended so far (start at 0)
+ *   reorder_k/_v     int32   [Hkv][D]                 gather index: stored[j] = source[idx[j]]; each
+ *                                                     row must be a permutation of 0..D-1 (Eq. 1)
+ *   alpha_k/_v       float   [Hkv][ng]                clip factor per group in (0,1] (Eq. 2)
+ *   status           int32   [1]                      optional (may be NULL); SKVQ_STATUS_* bits are OR-ed in
+ * Rows at or beyond Lq_b hold unspecified bytes.  The buffers fully describe the state:
+ * copying them is a checkpoint.
+ */
+typedef struct skvq_cache {
+    void *k_codes, *v_codes;
+    void *k_meta, *v_meta;
+    void *k_win, *v_win;
+    int32_t *lengths;
+    const int32_t *reorder_k, *reorder_v;
+    const float *alpha_k, *alpha_v;
+    int32_t *status;
+} skvq_cache;
+
+/* Options of one decode-attention call (host struct). */
+typedef struct skvq_attn_args {
+    float sm_scale;         /* softmax scale, e.g. 1/sqrt(D) */
+    int32_t max_len_hint;   /* host upper bound on lengths[] (sizes the grid); <= max_tokens */
+    int32_t n_splits;       /* sequence partitions per (sequence, KV head); 0 = library chooses */
+    void *workspace;        /* device scratch for the split partials, >= skvq_workspace_size() bytes */
+    size_t workspace_bytes;
+    void *ev_begin, *ev_end;/* optional cudaEvent_t (else NULL) recorded on the stream immediately
+                               before / after the partition kernel, for profiling */
+} skvq_attn_args;
+
+/* Library version (major*100 + minor). */
+int skvq_version(void);
+
+/* Static text for a return code. */
+const char *skvq_strerror(int code);
+
+/* Number of CUDA kernels this library has launched in this process (monotonic). */
+uint64_t skvq_launch_count(void);
+
+/* Validate cfg (host only).  Returns SKVQ_OK or the error a call with it would return. */
+int skvq_check_config(const skvq_config *cfg);
+
+/* Rows per (sequence, KV head) in the quantized segment:
+ * round_up(max(max_tokens - W, 0), SKVQ_TOKEN_ALIGN), at least SKVQ_TOKEN_ALIGN.  Negative on a bad cfg. */
+int32_t skvq_quant_capacity(const skvq_config *cfg);
+
+/* Bytes of k_codes, v_codes, k_meta, v_meta, k_win, v_win (in that order) for cfg.  Host only. */
+int skvq_cache_sizes(const skvq_config *cfg, size_t bytes_out[6]);
+
+/*
+ * Append tokens (Sec. 3.2, Algorithm 1 body, clipping_quant; Eq. 2).
+ * Sequence b receives n_b = n_new_per_seq ? n_new_per_seq[b] : n_new tokens (0 <= n_b <= n_new).
+ * With L0 = lengths[b], L1 = L0 + n_b: every token in [max(L0-W,0), max(L1-W,0)) is reordered
+ * (stored[j] = x[idx[j]]), split into groups of G channels and quantized per group:
+ *   lo = alpha*min, hi = alpha*max, h = fp16((hi-lo)/(2^bits-1)), z = fp16(lo),
+ *   code = clamp(rint((x - z)/h), 0, 2^bits-1)   (fp32, IEEE division, ties to even; h == 0 -> code 0)
+ * the last min(L1, W) tokens are kept in fp16 in the ring, and lengths[b] becomes L1.
+ * One bulk call equals the same tokens appended one at a time.
+ *   k, v           half [B][n_new][Hkv][D], original channel order (rows beyond n_b are ignored)
+ *   n_new_per_seq  device int32 [B] or NULL
+ * If L1 > max_tokens the sequence is left unchanged and SKVQ_STATUS_OVERFLOW is set in *status.
+ * NaN/Inf inputs give unspecified codes.
+ */
+int skvq_quantize_append(const skvq_config *cfg, const skvq_cache *cache, const void *k, const void *v,
+                         const int32_t *n_new_per_seq, int32_t n_new, void *cuda_stream);
+
+/* Scratch bytes skvq_decode_attention needs for lengths up to max_len_hint and the given n_splits
+ * (0 = the library's choice for that hint).  0 on a bad cfg. */
+size_t skvq_workspace_size(const skvq_config *cfg, int32_t max_len_hint, int32_t n_splits);
+
+/*
+ * Decode attention of one query per sequence over [quantized prefix || fp16 window]
+ * (Eq. 1 and the first lines of Algorithm 1; softmax and its scale written out):
+ *   q' = q[reorder_k],  s_t = sm_scale * sum_j q'_j K~[t][j],  p = softmax_t(s),
+ *   o'_j = sum_t p_t V~[t][j],  out[reorder_v[j]] = o'_j,
+ * where K~/V~ are h*code+z for t < Lq_b and the ring value for Lq_b <= t < L_b.  Dequantization
+ * happens in registers; no dequantized cache is written.  A sequence of length 0 yields zeros.
+ *   q    half [B][Hq][D]      out  half [B][Hq][D]
+ * The workspace contents are overwritten; calls sharing a workspace must be stream-ordered.
+ */
+int skvq_decode_attention(const skvq_config *cfg, const skvq_cache *cache, const void *q, void *out,
+                          const skvq_attn_args *args, void *cuda_stream);
+
+/*
+ * One decode step driven from HOST buffers: copies k_new, v_new (half [B][1][Hkv][D]) and q
+ * (half [B][Hq][D]) from host memory into `staging`, appends the token, runs decode attention and
+ * copies out (half [B][Hq][D]) back to host memory, all enqueued on the stream (the caller
+ * synchronises before reading out_host).  Pinned host memory keeps the copies asynchronous.
+ *   staging  device scratch of at least skvq_step_staging_size(cfg) bytes
+ */
+size_t skvq_step_staging_size(const skvq_config *cfg);
+int skvq_decode_step_host(const skvq_config *cfg, const skvq_cache *cache, const void *k_new_host,
+                          const void *v_new_host, const void *q_host, void *out_host, void *staging,
+                          const skvq_attn_args *args, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SKVQ_H_ */

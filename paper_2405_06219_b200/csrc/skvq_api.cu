@@ -1,0 +1,216 @@
+// C-ABI entry points of libskvq: argument validation, sizing helpers and the host-buffer decode step.
+#include <atomic>
+
+#include "skvq_internal.cuh"
+
+namespace skvq {
+
+static std::atomic<uint64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+static int check_cfg(const skvq_config *c)
+{
+    if (!c) return SKVQ_ERR_INVALID_ARG;
+    if (c->batch < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1 || c->window < 0 || c->max_tokens < 1)
+        return SKVQ_ERR_INVALID_ARG;
+    if (c->batch > 65535 || c->n_kv_heads > 65535) return SKVQ_ERR_UNSUPPORTED;
+    if (c->head_dim != kHeadDim) return SKVQ_ERR_UNSUPPORTED;
+    if ((c->k_bits != 2 && c->k_bits != 4) || (c->v_bits != 2 && c->v_bits != 4)) return SKVQ_ERR_UNSUPPORTED;
+    if (c->group_size != 32 && c->group_size != 64 && c->group_size != 128) return SKVQ_ERR_UNSUPPORTED;
+    if (c->n_q_heads % c->n_kv_heads != 0) return SKVQ_ERR_UNSUPPORTED;
+    if (c->n_q_heads / c->n_kv_heads > kMaxRep) return SKVQ_ERR_UNSUPPORTED;
+    return SKVQ_OK;
+}
+
+static int quant_capacity(const skvq_config *c)
+{
+    long rows = (long)c->max_tokens - c->window;
+    if (rows < 0) rows = 0;
+    rows = (rows + SKVQ_TOKEN_ALIGN - 1) / SKVQ_TOKEN_ALIGN * SKVQ_TOKEN_ALIGN;
+    if (rows < SKVQ_TOKEN_ALIGN) rows = SKVQ_TOKEN_ALIGN;
+    return (int)rows;
+}
+
+static Shape make_shape(const skvq_config *c)
+{
+    Shape s;
+    s.B = c->batch;
+    s.Hq = c->n_q_heads;
+    s.Hkv = c->n_kv_heads;
+    s.rep = s.Hq / s.Hkv;
+    s.k_bits = c->k_bits;
+    s.v_bits = c->v_bits;
+    s.G = c->group_size;
+    s.ng = kHeadDim / s.G;
+    s.W = c->window;
+    s.cap = quant_capacity(c);
+    s.max_tokens = c->max_tokens;
+    return s;
+}
+
+static bool misaligned(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+static int check_cache(const skvq_config *cfg, const skvq_cache *c, CachePtrs *out)
+{
+    if (!c) return SKVQ_ERR_INVALID_ARG;
+    if (!c->k_codes || !c->v_codes || !c->k_meta || !c->v_meta || !c->lengths || !c->reorder_k || !c->reorder_v ||
+        !c->alpha_k || !c->alpha_v)
+        return SKVQ_ERR_INVALID_ARG;
+    if (cfg->window > 0 && (!c->k_win || !c->v_win)) return SKVQ_ERR_INVALID_ARG;
+    const void *ptrs[] = {c->k_codes, c->v_codes, c->k_meta, c->v_meta, c->k_win, c->v_win,
+                          c->lengths, c->reorder_k, c->reorder_v, c->alpha_k, c->alpha_v};
+    for (const void *p : ptrs)
+        if (p && misaligned(p)) return SKVQ_ERR_MISALIGNED;
+    out->k_codes = static_cast<uint8_t *>(c->k_codes);
+    out->v_codes = static_cast<uint8_t *>(c->v_codes);
+    out->k_meta = static_cast<__half2 *>(c->k_meta);
+    out->v_meta = static_cast<__half2 *>(c->v_meta);
+    out->k_win = static_cast<__half *>(c->k_win);
+    out->v_win = static_cast<__half *>(c->v_win);
+    out->lengths = c->lengths;
+    out->reorder_k = c->reorder_k;
+    out->reorder_v = c->reorder_v;
+    out->alpha_k = c->alpha_k;
+    out->alpha_v = c->alpha_v;
+    out->status = c->status;
+    return SKVQ_OK;
+}
+
+static size_t workspace_bytes(const Shape &s, const SplitPlan &p)
+{
+    return (size_t)s.B * s.Hq * p.n_splits * kPartialStride * sizeof(float);
+}
+
+}  // namespace skvq
+
+using namespace skvq;
+
+extern "C" {
+
+int skvq_version(void) { return 100; }
+
+const char *skvq_strerror(int code)
+{
+    switch (code) {
+        case SKVQ_OK: return "ok";
+        case SKVQ_ERR_INVALID_ARG: return "invalid argument";
+        case SKVQ_ERR_UNSUPPORTED: return "unsupported configuration";
+        case SKVQ_ERR_MISALIGNED: return "device buffer is not 16-byte aligned";
+        case SKVQ_ERR_CAPACITY: return "token count exceeds the cache capacity";
+        case SKVQ_ERR_WORKSPACE: return "workspace missing or too small";
+        case SKVQ_ERR_CUDA: return "CUDA runtime error at launch";
+        default: return "unknown error code";
+    }
+}
+
+uint64_t skvq_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int skvq_check_config(const skvq_config *cfg) { return check_cfg(cfg); }
+
+int32_t skvq_quant_capacity(const skvq_config *cfg)
+{
+    const int rc = check_cfg(cfg);
+    return rc != SKVQ_OK ? rc : quant_capacity(cfg);
+}
+
+int skvq_cache_sizes(const skvq_config *cfg, size_t bytes_out[6])
+{
+    const int rc = check_cfg(cfg);
+    if (rc != SKVQ_OK) return rc;
+    if (!bytes_out) return SKVQ_ERR_INVALID_ARG;
+    const Shape s = make_shape(cfg);
+    const size_t rows = (size_t)s.B * s.Hkv * s.cap;
+    bytes_out[0] = rows * (kHeadDim * s.k_bits / 8);
+    bytes_out[1] = rows * (kHeadDim * s.v_bits / 8);
+    bytes_out[2] = rows * s.ng * sizeof(__half2);
+    bytes_out[3] = rows * s.ng * sizeof(__half2);
+    bytes_out[4] = (size_t)s.B * s.Hkv * s.W * kHeadDim * sizeof(__half);
+    bytes_out[5] = bytes_out[4];
+    return SKVQ_OK;
+}
+
+int skvq_quantize_append(const skvq_config *cfg, const skvq_cache *cache, const void *k, const void *v,
+                         const int32_t *n_new_per_seq, int32_t n_new, void *cuda_stream)
+{
+    int rc = check_cfg(cfg);
+    if (rc != SKVQ_OK) return rc;
+    CachePtrs c;
+    rc = check_cache(cfg, cache, &c);
+    if (rc != SKVQ_OK) return rc;
+    if (n_new < 0) return SKVQ_ERR_INVALID_ARG;
+    if (n_new == 0) return SKVQ_OK;
+    if (!k || !v) return SKVQ_ERR_INVALID_ARG;
+    if (misaligned(k) || misaligned(v) || (n_new_per_seq && (reinterpret_cast<uintptr_t>(n_new_per_seq) & 3u)))
+        return SKVQ_ERR_MISALIGNED;
+    if (n_new > cfg->max_tokens) return SKVQ_ERR_CAPACITY;
+    const Shape s = make_shape(cfg);
+    const cudaError_t e = launch_append(s, c, static_cast<const __half *>(k), static_cast<const __half *>(v),
+                                        n_new_per_seq, n_new, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? SKVQ_OK : SKVQ_ERR_CUDA;
+}
+
+size_t skvq_workspace_size(const skvq_config *cfg, int32_t max_len_hint, int32_t n_splits)
+{
+    if (check_cfg(cfg) != SKVQ_OK || max_len_hint < 0 || n_splits < 0) return 0;
+    const Shape s = make_shape(cfg);
+    if (max_len_hint > s.max_tokens) max_len_hint = s.max_tokens;
+    return workspace_bytes(s, plan_splits(s, max_len_hint, n_splits));
+}
+
+int skvq_decode_attention(const skvq_config *cfg, const skvq_cache *cache, const void *q, void *out,
+                          const skvq_attn_args *args, void *cuda_stream)
+{
+    int rc = check_cfg(cfg);
+    if (rc != SKVQ_OK) return rc;
+    CachePtrs c;
+    rc = check_cache(cfg, cache, &c);
+    if (rc != SKVQ_OK) return rc;
+    if (!q || !out || !args) return SKVQ_ERR_INVALID_ARG;
+    if (misaligned(q) || misaligned(out)) return SKVQ_ERR_MISALIGNED;
+    if (args->max_len_hint < 0 || args->n_splits < 0) return SKVQ_ERR_INVALID_ARG;
+    if (args->max_len_hint > cfg->max_tokens) return SKVQ_ERR_CAPACITY;
+    const Shape s = make_shape(cfg);
+    const SplitPlan plan = plan_splits(s, args->max_len_hint, args->n_splits);
+    if (!args->workspace || args->workspace_bytes < workspace_bytes(s, plan)) return SKVQ_ERR_WORKSPACE;
+    if (misaligned(args->workspace)) return SKVQ_ERR_MISALIGNED;
+    const cudaError_t e = launch_attention(s, c, static_cast<const __half *>(q), static_cast<__half *>(out),
+                                           args->sm_scale, plan, static_cast<float *>(args->workspace),
+                                           static_cast<cudaEvent_t>(args->ev_begin),
+                                           static_cast<cudaEvent_t>(args->ev_end),
+                                           static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? SKVQ_OK : SKVQ_ERR_CUDA;
+}
+
+size_t skvq_step_staging_size(const skvq_config *cfg)
+{
+    if (check_cfg(cfg) != SKVQ_OK) return 0;
+    const size_t kv = (size_t)cfg->batch * cfg->n_kv_heads * kHeadDim * sizeof(__half);
+    const size_t qo = (size_t)cfg->batch * cfg->n_q_heads * kHeadDim * sizeof(__half);
+    return 2 * kv + 2 * qo;
+}
+
+int skvq_decode_step_host(const skvq_config *cfg, const skvq_cache *cache, const void *k_new_host,
+                          const void *v_new_host, const void *q_host, void *out_host, void *staging,
+                          const skvq_attn_args *args, void *cuda_stream)
+{
+    int rc = check_cfg(cfg);
+    if (rc != SKVQ_OK) return rc;
+    if (!k_new_host || !v_new_host || !q_host || !out_host || !staging || !args) return SKVQ_ERR_INVALID_ARG;
+    if (misaligned(staging)) return SKVQ_ERR_MISALIGNED;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t kv = (size_t)cfg->batch * cfg->n_kv_heads * kHeadDim * sizeof(__half);
+    const size_t qo = (size_t)cfg->batch * cfg->n_q_heads * kHeadDim * sizeof(__half);
+    char *base = static_cast<char *>(staging);
+    void *d_k = base, *d_v = base + kv, *d_q = base + 2 * kv, *d_out = base + 2 * kv + qo;
+    if (cudaMemcpyAsync(d_k, k_new_host, kv, cudaMemcpyHostToDevice, stream) != cudaSuccess) return SKVQ_ERR_CUDA;
+    if (cudaMemcpyAsync(d_v, v_new_host, kv, cudaMemcpyHostToDevice, stream) != cudaSuccess) return SKVQ_ERR_CUDA;
+    if (cudaMemcpyAsync(d_q, q_host, qo, cudaMemcpyHostToDevice, stream) != cudaSuccess) return SKVQ_ERR_CUDA;
+    rc = skvq_quantize_append(cfg, cache, d_k, d_v, nullptr, 1, cuda_stream);
+    if (rc != SKVQ_OK) return rc;
+    rc = skvq_decode_attention(cfg, cache, d_q, d_out, args, cuda_stream);
+    if (rc != SKVQ_OK) return rc;
+    if (cudaMemcpyAsync(out_host, d_out, qo, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return SKVQ_ERR_CUDA;
+    return SKVQ_OK;
+}
+
+}  // extern "C"

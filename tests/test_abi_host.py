@@ -1,0 +1,111 @@
+"""Host-only checks of the C ABI: the library loads without a GPU, exports every function the
+public header declares, and validates arguments before touching the device."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2405_06219_b200 import binding as B
+from paper_2405_06219_b200 import build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build_library()
+    return B.lib()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "skvq.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(skvq_[a-z_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = declared_functions()
+    assert len(names) >= 11
+    for n in names:
+        assert hasattr(lib, n), n
+    assert sorted(B.EXPORTS) == names
+
+
+def cfg(**kw):
+    base = dict(batch=2, n_q_heads=8, n_kv_heads=2, head_dim=128, k_bits=2, v_bits=2, group_size=128, window=128,
+                max_tokens=4096)
+    base.update(kw)
+    return B.SkvqConfig(**base)
+
+
+def test_version_and_strerror(lib):
+    assert B.skvq_version() >= 100
+    assert B.skvq_strerror(0) == "ok"
+    for code in range(-6, 0):
+        assert B.skvq_strerror(code) not in ("ok", "unknown error code")
+    assert B.skvq_strerror(-99) == "unknown error code"
+
+
+@pytest.mark.parametrize("kw,code", [
+    (dict(head_dim=64), B.SKVQ_ERR_UNSUPPORTED), (dict(k_bits=3), B.SKVQ_ERR_UNSUPPORTED),
+    (dict(v_bits=8), B.SKVQ_ERR_UNSUPPORTED), (dict(group_size=16), B.SKVQ_ERR_UNSUPPORTED),
+    (dict(n_q_heads=7), B.SKVQ_ERR_UNSUPPORTED), (dict(n_q_heads=32, n_kv_heads=2), B.SKVQ_ERR_UNSUPPORTED),
+    (dict(batch=0), B.SKVQ_ERR_INVALID_ARG), (dict(window=-1), B.SKVQ_ERR_INVALID_ARG),
+    (dict(max_tokens=0), B.SKVQ_ERR_INVALID_ARG), (dict(), B.SKVQ_OK), (dict(window=0, k_bits=4, group_size=32), B.SKVQ_OK),
+])
+def test_config_validation(lib, kw, code):
+    assert B.skvq_check_config(cfg(**kw)) == code
+
+
+def test_sizes_follow_the_documented_layout(lib):
+    c = cfg(max_tokens=4096 + 5, group_size=32, k_bits=4)
+    cap = B.skvq_quant_capacity(c)
+    assert cap == 4032 and cap % B.SKVQ_TOKEN_ALIGN == 0          # round_up(4101 - 128, 64)
+    sizes = B.skvq_cache_sizes(c)
+    rows = 2 * 2 * cap
+    assert sizes == [rows * 64, rows * 32, rows * 4 * 4, rows * 4 * 4, 2 * 2 * 128 * 128 * 2, 2 * 2 * 128 * 128 * 2]
+    assert B.skvq_quant_capacity(cfg(max_tokens=10)) == B.SKVQ_TOKEN_ALIGN
+    # stored bits per element of the quantized segment: 4 + 32/32 and 2 + 32/32 (N + 2*16/G)
+    assert (sizes[0] + sizes[2]) * 8 / (rows * 128) == 5.0 and (sizes[1] + sizes[3]) * 8 / (rows * 128) == 3.0
+
+
+def test_workspace_size_grows_with_splits(lib):
+    c = cfg()
+    one = B.skvq_workspace_size(c, 4096, 1)
+    four = B.skvq_workspace_size(c, 4096, 4)
+    assert one == 2 * 8 * 132 * 4 and four == 4 * one
+    assert B.skvq_workspace_size(c, 4096, 0) >= one
+    assert B.skvq_workspace_size(cfg(head_dim=64), 4096, 0) == 0
+    assert B.skvq_step_staging_size(c) == 2 * (2 * 2 * 128 * 2) + 2 * (2 * 8 * 128 * 2)
+
+
+def test_calls_reject_bad_arguments_before_any_launch(lib):
+    c = cfg()
+    empty = B.SkvqCacheStruct()
+    before = B.skvq_launch_count()
+    rc = lib.skvq_quantize_append(ctypes.byref(c), ctypes.byref(empty), None, None, None, 1, None)
+    assert rc == B.SKVQ_ERR_INVALID_ARG
+    args = B.SkvqAttnArgs(0.1, 4096, 0, None, 0, None, None)
+    assert lib.skvq_decode_attention(ctypes.byref(c), ctypes.byref(empty), None, None, ctypes.byref(args), None) \
+        == B.SKVQ_ERR_INVALID_ARG
+    # fake (never dereferenced) pointers: alignment, capacity and workspace checks are host-side
+    fake = B.SkvqCacheStruct(*([0x1000] * 11), None)
+    assert lib.skvq_quantize_append(ctypes.byref(c), ctypes.byref(fake), 0x1008, 0x1000, None, 1, None) \
+        == B.SKVQ_ERR_MISALIGNED
+    assert lib.skvq_quantize_append(ctypes.byref(c), ctypes.byref(fake), 0x1000, 0x1000, None, 5000, None) \
+        == B.SKVQ_ERR_CAPACITY
+    assert lib.skvq_quantize_append(ctypes.byref(c), ctypes.byref(fake), 0x1000, 0x1000, None, -1, None) \
+        == B.SKVQ_ERR_INVALID_ARG
+    misal = B.SkvqCacheStruct(0x1004, *([0x1000] * 10), None)
+    assert lib.skvq_quantize_append(ctypes.byref(c), ctypes.byref(misal), 0x1000, 0x1000, None, 1, None) \
+        == B.SKVQ_ERR_MISALIGNED
+    assert lib.skvq_decode_attention(ctypes.byref(c), ctypes.byref(fake), 0x1000, 0x1000, ctypes.byref(args), None) \
+        == B.SKVQ_ERR_WORKSPACE
+    small = B.SkvqAttnArgs(0.1, 4096, 4, 0x1000, 64, None, None)
+    assert lib.skvq_decode_attention(ctypes.byref(c), ctypes.byref(fake), 0x1000, 0x1000, ctypes.byref(small), None) \
+        == B.SKVQ_ERR_WORKSPACE
+    toolong = B.SkvqAttnArgs(0.1, 5000, 0, 0x1000, 1 << 30, None, None)
+    assert lib.skvq_decode_attention(ctypes.byref(c), ctypes.byref(fake), 0x1000, 0x1000, ctypes.byref(toolong), None) \
+        == B.SKVQ_ERR_CAPACITY
+    assert B.skvq_launch_count() == before

@@ -1,0 +1,204 @@
+"""GPU parity: the CUDA library against the CPU oracle through the C ABI.
+
+Quantized codes, scales/zeros, window contents and lengths must be bit-exact; the fp16 attention
+output must be within 2e-3 (max-abs) of the oracle's fp64 attention over the same cache.
+"""
+import numpy as np
+import pytest
+import torch
+
+from helpers import ATTN_TOL, assert_cache_bit_exact, oracle_cache_for
+from paper_2405_06219_b200 import binding as B
+from paper_2405_06219_b200 import build, workloads
+
+pytestmark = pytest.mark.gpu
+CF = workloads.configs()
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    build.build_library()
+    B.lib()
+
+
+def small(i, **kw):
+    return CF[i].scaled(**kw)
+
+
+def both_caches(w, max_tokens):
+    return B.SkvqCache.for_workload(w, max_tokens), oracle_cache_for(w, max_tokens)
+
+
+def dev(x):
+    return torch.from_numpy(np.ascontiguousarray(x)).cuda()
+
+
+def attention_both(gpu, ora, w, step=0, n_splits=0):
+    q = w.query(step)
+    hint = int(ora.lengths.max())
+    out = gpu.attention(dev(q), w.sm_scale, hint, n_splits=n_splits)
+    torch.cuda.synchronize()
+    want = ora.attention(q, w.sm_scale)
+    return out.cpu().numpy().astype(np.float64), want
+
+
+# ------------------------------------------------------------------ quantize_append, bit-exact
+@pytest.mark.parametrize("cfg_i,kw,n", [
+    (0, dict(context=700), 700),                      # 2-bit, g128, MHA: several tiles and a ragged tail
+    (2, dict(context=900, batch=2), 900),             # g32 GQA
+    (4, dict(context=1000, batch=3, ragged=None), 1000),   # 4-bit g64, window 256
+    (0, dict(context=100), 100),                      # shorter than the window: nothing quantized
+    (0, dict(context=128), 128),                      # exactly the window
+    (0, dict(context=129), 129),                      # one token slides out
+    (0, dict(context=300, window=0), 300),            # no window at all
+    (1, dict(context=2100, batch=2, n_kv_heads=4, n_q_heads=4, k_bits=4, v_bits=2, group_size=64), 2100),  # mixed widths
+])
+def test_prefill_quantize_bit_exact(cfg_i, kw, n):
+    w = small(cfg_i, **kw)
+    gpu, ora = both_caches(w, n + 64)
+    k, v = w.prefill("k", n), w.prefill("v", n)
+    gpu.append(dev(k), dev(v))
+    assert ora.append(k, v) == 0
+    assert_cache_bit_exact(gpu, ora)
+    assert int(gpu.status[0].item()) == 0
+
+
+def test_chunked_and_single_token_appends_bit_exact():
+    w = small(2, context=700, batch=2)
+    gpu, ora = both_caches(w, 800)
+    k, v = w.prefill("k", 700), w.prefill("v", 700)
+    t = 0
+    for step in (1, 1, 5, 130, 127, 1, 1, 300, 64, 70):
+        gpu.append(dev(k[:, t:t + step]), dev(v[:, t:t + step]))
+        ora.append(k[:, t:t + step], v[:, t:t + step])
+        t += step
+        assert_cache_bit_exact(gpu, ora)
+    assert t == 700
+    for s in range(40):                                                # decode-style single tokens
+        kn, vn = w.new_token("k", s), w.new_token("v", s)
+        gpu.append(dev(kn), dev(vn))
+        ora.append(kn, vn)
+    assert_cache_bit_exact(gpu, ora)
+    bulk = oracle_cache_for(w, 800)
+    bulk.append(np.concatenate([k] + [w.new_token("k", s) for s in range(40)], 1),
+                np.concatenate([v] + [w.new_token("v", s) for s in range(40)], 1))
+    assert_cache_bit_exact(gpu, bulk)
+
+
+def test_ragged_append_and_overflow_flag():
+    w = small(4, context=600, batch=4, ragged=None)
+    gpu, ora = both_caches(w, 640)
+    k, v = w.prefill("k", 600), w.prefill("v", 600)
+    n = np.array([600, 0, 257, 13], np.int32)
+    gpu.append(dev(k), dev(v), dev(n))
+    ora.append(k, v, n)
+    assert_cache_bit_exact(gpu, ora)
+    # second ragged round; sequence 0 would exceed max_tokens = 640 and must stay untouched
+    n2 = np.array([41, 300, 0, 41], np.int32)
+    gpu.append(dev(k[:, :300]), dev(v[:, :300]), dev(n2))
+    assert ora.append(k[:, :300], v[:, :300], n2) == -1
+    assert_cache_bit_exact(gpu, ora)
+    assert ora.lengths.tolist() == [600, 300, 257, 54]
+    assert int(gpu.status[0].item()) & B.SKVQ_STATUS_OVERFLOW
+
+
+# ------------------------------------------------------------------ decode attention, <= 2e-3
+@pytest.mark.parametrize("cfg_i,kw,n", [
+    (0, dict(), 4096),                                               # configuration 0 in full
+    (1, dict(context=3000, batch=2), 3000),
+    (2, dict(context=5000, batch=2), 5000),                          # GQA 4:1, g32
+    (3, dict(context=9000, n_q_heads=4, n_kv_heads=4), 9000),
+    (4, dict(context=1500, batch=3, ragged=None), 1500),             # 4-bit g64 W256
+    (0, dict(context=100), 100), (0, dict(context=128), 128), (0, dict(context=129), 129),
+    (0, dict(context=1), 1), (0, dict(context=500, window=0), 500),
+    (2, dict(context=777, batch=1, n_q_heads=16, n_kv_heads=2), 777),   # 8 query heads per KV head
+])
+def test_attention_matches_oracle(cfg_i, kw, n):
+    w = small(cfg_i, **kw)
+    gpu, ora = both_caches(w, n + 64)
+    k, v = w.prefill("k", n), w.prefill("v", n)
+    gpu.append(dev(k), dev(v))
+    ora.append(k, v)
+    assert_cache_bit_exact(gpu, ora)
+    got, want = attention_both(gpu, ora, w)
+    assert np.abs(got - want).max() <= ATTN_TOL
+
+
+def test_attention_ragged_batch_with_empty_sequence():
+    w = small(4, context=2000, batch=6, ragged=None)
+    gpu, ora = both_caches(w, 2048)
+    k, v = w.prefill("k", 2000), w.prefill("v", 2000)
+    n = np.array([2000, 0, 256, 257, 1024, 3], np.int32)
+    gpu.append(dev(k), dev(v), dev(n))
+    ora.append(k, v, n)
+    got, want = attention_both(gpu, ora, w)
+    assert np.abs(got - want).max() <= ATTN_TOL
+    assert not got[1].any()
+
+
+@pytest.mark.parametrize("n_splits", [1, 2, 3, 7, 64])
+def test_split_count_does_not_change_the_result(n_splits):
+    w = small(2, context=6000, batch=1)
+    gpu, ora = both_caches(w, 6016)
+    k, v = w.prefill("k", 6000), w.prefill("v", 6000)
+    gpu.append(dev(k), dev(v))
+    ora.append(k, v)
+    got, want = attention_both(gpu, ora, w, n_splits=n_splits)
+    assert np.abs(got - want).max() <= ATTN_TOL
+
+
+def test_decode_loop_append_then_attend():
+    """Steady-state decoding: each step appends one token (one slides out of the window) and attends."""
+    w = small(3, context=1000, n_q_heads=8, n_kv_heads=8)
+    gpu, ora = both_caches(w, 1100)
+    k, v = w.prefill("k", 1000), w.prefill("v", 1000)
+    gpu.append(dev(k), dev(v))
+    ora.append(k, v)
+    for s in range(20):
+        kn, vn = w.new_token("k", s), w.new_token("v", s)
+        gpu.append(dev(kn), dev(vn))
+        ora.append(kn, vn)
+        got, want = attention_both(gpu, ora, w, step=s)
+        assert np.abs(got - want).max() <= ATTN_TOL
+    assert_cache_bit_exact(gpu, ora)
+
+
+def test_host_buffer_decode_step():
+    w = small(1, context=2000, batch=2)
+    gpu, ora = both_caches(w, 2100)
+    k, v = w.prefill("k", 2000), w.prefill("v", 2000)
+    gpu.append(dev(k), dev(v))
+    ora.append(k, v)
+    kn, vn, q = w.new_token("k", 0), w.new_token("v", 0), w.query(5)
+    hk, hv, hq = (torch.from_numpy(x).pin_memory() for x in (kn, vn, q))
+    hout = torch.empty(q.shape, dtype=torch.float16).pin_memory()
+    staging = torch.empty(B.skvq_step_staging_size(gpu.cfg), dtype=torch.uint8, device="cuda")
+    before = B.skvq_launch_count()
+    B.skvq_decode_step_host(gpu.cfg, gpu.struct, hk, hv, hq, hout, staging, gpu.attn_args(w.sm_scale, 2001))
+    torch.cuda.synchronize()
+    assert B.skvq_launch_count() - before >= 3
+    ora.append(kn, vn)
+    want = ora.attention(q, w.sm_scale)
+    assert np.abs(hout.numpy().astype(np.float64) - want).max() <= ATTN_TOL
+    assert_cache_bit_exact(gpu, ora)
+
+
+def test_adversarial_values_stay_bit_exact():
+    """Constant groups (h = 0), zeros of both signs, tiny and large magnitudes, exact rounding ties."""
+    w = small(2, context=400, batch=1)
+    gpu, ora = both_caches(w, 512)
+    rng = np.random.default_rng(5)
+    k = w.prefill("k", 400).copy()
+    v = w.prefill("v", 400).copy()
+    k[0, 0:40] = np.float16(1.25)                       # constant rows
+    k[0, 40:60] = np.float16(0.0)
+    k[0, 60:80, :, ::2] = np.float16(-0.0)
+    v[0, 0:50] = (rng.integers(0, 4, (50, 8, 128)) * 0.5 - 1.0).astype(np.float16)     # exact levels
+    v[0, 50:100] = (rng.integers(0, 7, (50, 8, 128)) * 0.25 - 0.75).astype(np.float16)  # half-way ties
+    v[0, 100:120] = (rng.standard_normal((20, 8, 128)) * 1e-6).astype(np.float16)      # subnormal range
+    k[0, 100:120] = (rng.standard_normal((20, 8, 128)) * 2e4).astype(np.float16)       # near the fp16 maximum
+    gpu.append(dev(k), dev(v))
+    ora.append(k, v)
+    assert_cache_bit_exact(gpu, ora)
+    got, want = attention_both(gpu, ora, w)
+    assert np.isfinite(got).all()
