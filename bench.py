@@ -279,6 +279,10 @@ def main():
     out = torch.empty_like(q_all[0])
     ev_k = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
 
+    for a, b in ev_k:      # torch creates its events lazily: record once so the handles exist before the library re-records them
+        a.record()
+        b.record()
+    torch.cuda.synchronize()
     args_plain = cache.attn_args(w.sm_scale, hint, args.splits)
     args_timed = [cache.attn_args(w.sm_scale, hint, args.splits, a, b) for a, b in ev_k]
 
