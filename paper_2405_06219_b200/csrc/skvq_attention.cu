@@ -42,7 +42,8 @@ __device__ __forceinline__ float warp_sum(float v)
     return v;
 }
 
-// Scalar partition kernel: one thread per token for the scores, one thread per channel for P.V.
+// Scalar partition kernel (configurations the tensor-core kernel does not cover: 4-bit codes, mixed
+// widths, 8 query heads per KV head): one thread per token for the scores, one per channel for P.V.
 template <int KBITS, int VBITS>
 __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
 {
@@ -52,9 +53,10 @@ __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
     const int rep = s.rep, G = s.G, ng = s.ng, W = s.W;
     const int L = a.c.lengths[b];
     const int Lq = max(L - W, 0);
-    const int q_begin = min(split * a.plan.split_len, Lq);
-    const int q_end = min(q_begin + a.plan.split_len, Lq);
-    const bool owns_window = (split == a.plan.n_splits - 1);
+    const bool owns_window = (split == a.plan.n_splits);      // the last part is the fp16 window
+    const int q_begin = owns_window ? Lq : min(split * a.plan.split_len, Lq);
+    const int q_end = owns_window ? Lq : min(q_begin + a.plan.split_len, Lq);
+    const int n_parts = a.plan.n_splits + 1;
 
     __shared__ float sq[kMaxRep][kHeadDim];        // permuted query, times sm_scale*log2(e)
     __shared__ float sqsum[kMaxRep][4];            // per-group sums of the above
@@ -203,7 +205,7 @@ __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
 #pragma unroll
     for (int r = 0; r < kMaxRep; ++r) {
         if (r < rep) {
-            float *part = a.ws + (((size_t)b * s.Hq + hk * rep + r) * a.plan.n_splits + split) * kPartialStride;
+            float *part = a.ws + (((size_t)b * s.Hq + hk * rep + r) * n_parts + split) * kPartialStride;
             part[tid] = acc[r];
             if (tid == 0) {
                 float l = 0.f;
@@ -221,7 +223,7 @@ __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
     const int hq = blockIdx.x, b = blockIdx.y, d = threadIdx.x;
     const Shape &s = a.s;
     const int hk = hq / s.rep;
-    const int S = a.plan.n_splits;
+    const int S = a.plan.n_splits + 1;
     const float *part = a.ws + ((size_t)b * s.Hq + hq) * S * kPartialStride;
     float M = -CUDART_INF_F;
     for (int i = 0; i < S; ++i) M = fmaxf(M, part[(size_t)i * kPartialStride + kHeadDim]);
@@ -245,21 +247,22 @@ SplitPlan plan_splits(const Shape &s, int max_len, int requested_splits)
 {
     const int lq = max_len - s.W > 0 ? max_len - s.W : 0;
     SplitPlan p;
-    int split_len;
+    long split_len;
     if (requested_splits > 0) {
         split_len = (lq + requested_splits - 1) / requested_splits;
+        split_len = (split_len + SKVQ_TOKEN_ALIGN - 1) / SKVQ_TOKEN_ALIGN * SKVQ_TOKEN_ALIGN;
     } else {
-        // Enough CTAs to fill 148 SMs several times over, but at least 1024 tokens per split.
-        const long pairs = (long)s.B * s.Hkv;
-        long want = (148L * 16 + pairs - 1) / pairs;
-        if (want < 1) want = 1;
-        split_len = (int)((lq + want - 1) / want);
+        // About 8 CTAs per resident slot (148 SMs x 3 CTAs), between 1024 and 8192 tokens per split,
+        // in multiples of 256 tokens (4 warps x 64-token tiles).
+        const long total = (long)lq * s.B * s.Hkv;
+        split_len = (total + 148L * 3 * 8 - 1) / (148L * 3 * 8);
         if (split_len < 1024) split_len = 1024;
+        if (split_len > 8192) split_len = 8192;
+        split_len = (split_len + 255) / 256 * 256;
     }
-    split_len = (split_len + SKVQ_TOKEN_ALIGN - 1) / SKVQ_TOKEN_ALIGN * SKVQ_TOKEN_ALIGN;
     if (split_len < SKVQ_TOKEN_ALIGN) split_len = SKVQ_TOKEN_ALIGN;
-    p.split_len = split_len;
-    p.n_splits = (lq + split_len - 1) / split_len;
+    p.split_len = (int)split_len;
+    p.n_splits = (int)((lq + split_len - 1) / split_len);
     if (p.n_splits < 1) p.n_splits = 1;
     return p;
 }
@@ -269,9 +272,13 @@ cudaError_t launch_attention(const Shape &s, const CachePtrs &c, const __half *q
                              cudaStream_t stream)
 {
     AttnArgs a{s, c, q, out, sm_scale * 1.4426950408889634f, plan, workspace};
-    dim3 grid(plan.n_splits, s.Hkv, s.B);
+    dim3 grid(plan.n_splits + 1, s.Hkv, s.B);
     if (ev_begin) cudaEventRecord(ev_begin, stream);
-    if (s.k_bits == 2 && s.v_bits == 2) partition_kernel<2, 2><<<grid, kThreads, 0, stream>>>(a);
+    bool handled = false;
+    cudaError_t em = launch_partition_mma(s, c, q, a.scale_log2, plan, workspace, stream, &handled);
+    if (em != cudaSuccess) return em;
+    if (handled) { /* tensor-core kernel launched */ }
+    else if (s.k_bits == 2 && s.v_bits == 2) partition_kernel<2, 2><<<grid, kThreads, 0, stream>>>(a);
     else if (s.k_bits == 4 && s.v_bits == 4) partition_kernel<4, 4><<<grid, kThreads, 0, stream>>>(a);
     else if (s.k_bits == 4 && s.v_bits == 2) partition_kernel<4, 2><<<grid, kThreads, 0, stream>>>(a);
     else partition_kernel<2, 4><<<grid, kThreads, 0, stream>>>(a);

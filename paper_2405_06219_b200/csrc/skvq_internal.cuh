@@ -32,7 +32,7 @@ struct CachePtrs {
 
 struct SplitPlan {
     int split_len;   // quantized tokens per split (multiple of SKVQ_TOKEN_ALIGN)
-    int n_splits;    // grid splits per (sequence, KV head); the last one also owns the fp16 window
+    int n_splits;    // splits of the quantized prefix per (sequence, KV head); one more part holds the fp16 window
 };
 
 // Chooses the sequence partition for lengths up to max_len (host).
@@ -44,6 +44,9 @@ cudaError_t launch_append(const Shape &s, const CachePtrs &c, const __half *k, c
 cudaError_t launch_attention(const Shape &s, const CachePtrs &c, const __half *q, __half *out, float sm_scale,
                              const SplitPlan &plan, float *workspace, cudaEvent_t ev_begin, cudaEvent_t ev_end,
                              cudaStream_t stream);
+
+cudaError_t launch_partition_mma(const Shape &s, const CachePtrs &c, const __half *q, float scale_log2,
+                                 const SplitPlan &plan, float *workspace, cudaStream_t stream, bool *handled);
 
 void count_launch(int n = 1);
 
