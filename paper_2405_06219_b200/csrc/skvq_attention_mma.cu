@@ -1,15 +1,20 @@
 // Tensor-core partition kernel of skvq_decode_attention for 2-bit K and V (Eq. 1, Algorithm 1).
 //
 // Why tensor cores on an HBM-bound path: at 2 bits a cache element costs 0.28 bytes, so streaming
-// at several TB/s leaves fewer than two issue slots per element on the scalar pipes.  The 2-bit
-// codes are therefore turned into fp16 operands with ONE logic op per two codes and contracted
-// with mma.sync.m16n8k16 (fp32 accumulate); scale and zero point never touch individual elements:
-//   q'.K~_t   = sum_g h_{t,g} (sum_{j in g} q'_j c_{t,j}) + sum_g z_{t,g} (sum_{j in g} q'_j)
+// at several TB/s leaves fewer than two issue slots per element, and the logic pipe that does the
+// bit work retires half a warp instruction per clock.  The codes are therefore turned into MMA
+// operands with as few logic ops as possible and contracted on the tensor cores; scale and zero
+// point never touch individual elements:
+//   q'.K~_t            = sum_g h_{t,g} (sum_{j in g} q'_j c_{t,j}) + sum_g z_{t,g} (sum_{j in g} q'_j)
 //   sum_t p_t V~_{t,d} = sum_t (p_t h_{t,g(d)}) c_{t,d} + sum_t p_t z_{t,g(d)}
-// Unpack trick: OR-ing a 2-bit field that sits at mantissa bits [p, p+2) of an fp16 lane with an
-// exponent pattern gives the half value  base + weight*code  (base = 2^E, weight = 2^(E+p-10)).
-// The constant base contributes base * sum(B operand), which is subtracted in fp32 afterwards;
-// the weight is folded into the other operand (K side) or divided out at the end (V side).
+// Scores (integer MMA, exact): `word & (0x03030303 << 2t)` leaves four codes of a packed word as
+// bytes worth 4^t * code -- one AND per four codes, no shift -- which feed mma.m16n8k32.u8.s8.
+// The query is put on a power-of-two fixed-point grid, divided by 4^t and split into four signed
+// byte digits that sit in four B columns, so sum_j q'_j c_j is formed exactly in int32.
+// Values (fp16 MMA): OR-ing a 2-bit field that sits at mantissa bits [p, p+2) of an fp16 lane with
+// an exponent pattern gives the half value 64 + weight*code; the constant 64 contributes
+// 64 * sum(P), subtracted in fp32 at the end, and the weight is divided out per channel.
+// P = p*h is split into fp16 hi + lo pieces (two B columns) when the column budget allows.
 //
 // One CTA = 4 independent warps on one (sequence, KV head, split); each warp streams 64-token
 // tiles of codes + scale/zero through its own ring of shared-memory stages filled by
@@ -51,9 +56,24 @@ __device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t mask, uint32_t m
 __device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                          uint32_t b1)
 {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ void imma16832(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                          uint32_t b1)
+{
+    asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ float ex2_approx(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
@@ -109,11 +129,12 @@ struct Cfg {
     static constexpr int kCodeTile = kTileTok * kRowBytes;               // 2048 B
     static constexpr int kMetaTile = kTileTok * NG * 4;                  // 256 B * NG
     static constexpr int kStageBytes = 2 * kCodeTile + 2 * kMetaTile;
-    static constexpr int kStages = 3;
-    static constexpr int kScBytes = kTileTok * R * NG * 4;               // per-group raw scores
+    static constexpr int kStages = 2;
+    static constexpr int NTK = (4 * R + 7) / 8;                          // K-side n-tiles: 4 byte digits per head
+    static constexpr int kScBytes = kTileTok * R * NG * 8;               // per (token, group, head): low and high digit pairs
     static constexpr int kPBytes = 4 * NCVP * 16 * 2;                    // P operand tile
     static constexpr int kWarpBytes = kStages * kStageBytes + kScBytes + kPBytes + 64;   // + mbarriers
-    static constexpr int kQBytes = (R * kHeadDim * 4 + 2 * R * NG * 4 + 127) / 128 * 128;
+    static constexpr int kQBytes = (R * kHeadDim * 4 + R * NG * 4 + 2 * R * 4 + 64 + 127) / 128 * 128;
     static constexpr int kSmemBytes = kQBytes + kWarps * kWarpBytes;
     static_assert(kStages * kStageBytes >= NCV * kHeadDim * 4 + R * kPartialStride * 4, "stage area is reused for the final merge");
 };
@@ -254,53 +275,88 @@ __global__ void __launch_bounds__(kThreads) partition_mma_kernel(MmaArgs a)
     const int q_end = min(q_begin + a.plan.split_len, Lq);
     const int n_parts = a.plan.n_splits + 1;
 
-    // ---- CTA-wide prologue: permuted query, per-(head, group) constants
+    // ---- CTA-wide prologue: permuted query, its fixed-point grid and per-(head, group) sums
     float *qs = reinterpret_cast<float *>(smem);                       // [R][128] q' (exact fp16 values)
-    float *koff = qs + R * kHeadDim;                                   // [R][NG] scale * 16 * sum of the B operand
-    float *sqs = koff + R * NG;                                        // [R][NG] scale * sum_j q'_j
+    float *sqs = qs + R * kHeadDim;                                    // [R][NG] scale * sum_j q'_j
+    float *cF = sqs + R * NG;                                          // [R] scale / F_r, F_r = 2^kexp[r]
+    int *kexp = reinterpret_cast<int *>(cF + R);                       // [R]
+    float *redmax = reinterpret_cast<float *>(kexp + R);               // [4][R]
     uint8_t *warp_base = smem + C::kQBytes + warp * C::kWarpBytes;
     {
         const int32_t *idx_k = a.c.reorder_k + (size_t)hk * kHeadDim;
         const int src = idx_k[tid] & (kHeadDim - 1);
 #pragma unroll
-        for (int r = 0; r < R; ++r)
-            qs[r * kHeadDim + tid] = __half2float(a.q[((size_t)b * s.Hq + hk * R + r) * kHeadDim + src]);
+        for (int r = 0; r < R; ++r) {
+            const float qv = __half2float(a.q[((size_t)b * s.Hq + hk * R + r) * kHeadDim + src]);
+            qs[r * kHeadDim + tid] = qv;
+            const float wm = warp_max(fabsf(qv));
+            if (lane == 0) redmax[warp * R + r] = wm;
+        }
     }
     __syncthreads();
-    if (tid < R * NG) {
-        const int r = tid / NG, gg = tid % NG;
-        float sb = 0.f, sq = 0.f;
-        for (int j = gg * G; j < (gg + 1) * G; ++j) {
-            const float qv = qs[r * kHeadDim + j];
-            // channel j sits in field (j & 7) of its word; odd fields carry weight 4 (see the K unpack below)
-            const float bq = __half2float(__float2half_rn((j & 1) ? qv * 0.25f : qv));
-            sb += bq;
-            sq += qv;
+    if (tid < R) {
+        // F = 2^k with |q'_j| * F <= 2^30: every q'_j * F / 4^t is then an integer (or rounds at 2^-24 relative)
+        float qmax = 0.f;
+        for (int w = 0; w < kWarps; ++w) qmax = fmaxf(qmax, redmax[w * R + tid]);
+        int k = 0;
+        if (qmax > 0.f) {
+            int e;
+            const float m = frexpf(qmax, &e);          // qmax = m * 2^e, 0.5 <= m < 1
+            k = 30 - ((m == 0.5f) ? e - 1 : e);
         }
-        koff[tid] = 16.0f * sb * a.scale_log2;
-        sqs[tid] = sq * a.scale_log2;
+        kexp[tid] = k;
+        cF[tid] = ldexpf(a.scale_log2, -k);
+    }
+    if (tid >= 32 && tid < 32 + R * NG) {
+        const int r = (tid - 32) / NG, gg = (tid - 32) % NG;
+        float sq = 0.f;
+        for (int j = gg * G; j < (gg + 1) * G; ++j) sq += qs[r * kHeadDim + j];
+        sqs[r * NG + gg] = sq * a.scale_log2;
     }
     __syncthreads();
 
-    // B operand of the score MMAs: k-step s contracts the 16 channels of code word s.
-    //   b0 = (q'[16s+2t], q'[16s+8+2t])          weight 1
-    //   b1 = (q'[16s+2t+1], q'[16s+9+2t]) / 4    weight 4
-    uint32_t bq[8][2];
+    // B operand of the score MMAs (s8): k-step ks contracts the 32 channels of code words 2ks, 2ks+1;
+    // byte b of register `reg` = digit (col & 3) of round(q'[32ks + 16reg + 4b + t] * F / 4^t), column col = head*4 + digit.
+    // Thread tid owns channel tid: it writes the four digits of that channel as bytes straight into the
+    // register image bimg[head][digit][ks][reg][t] (byte b), which the lanes then load word by word.
+    uint8_t *bimg0 = smem + C::kQBytes;   // [R][4][4][2][4] words = R*512 bytes in warp 0's stage area, idle until the pipeline starts
+    {
+        const int ks = tid >> 5, reg = (tid >> 4) & 1, bb = (tid >> 2) & 3, tt = tid & 3;
 #pragma unroll
-    for (int ks = 0; ks < 8; ++ks) {
-        __half2 v0 = __floats2half2_rn(0.f, 0.f), v1 = v0;
-        if (g < R) {
-            const float *qr = qs + g * kHeadDim + 16 * ks + 2 * t;
-            v0 = __floats2half2_rn(qr[0], qr[8]);
-            v1 = __floats2half2_rn(qr[1] * 0.25f, qr[9] * 0.25f);
+        for (int r = 0; r < R; ++r) {
+            // q' * 2^(k - 2t): an exact power-of-two scaling done on the exponent field
+            int v = __float2int_rn(qs[r * kHeadDim + tid] * __int_as_float((127 + kexp[r] - 2 * tt) << 23));
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {      // balanced base-256 digits, least significant first
+                const int di = (i < 3) ? (int)(int8_t)(v & 0xFF) : v;
+                v = (v - di) >> 8;
+                bimg0[(((((r * 4 + i) * 4 + ks) * 2 + reg) * 4 + tt) << 2) + bb] = (uint8_t)(di & 0xFF);
+            }
         }
-        bq[ks][0] = *reinterpret_cast<uint32_t *>(&v0);
-        bq[ks][1] = *reinterpret_cast<uint32_t *>(&v1);
+    }
+    __syncthreads();
+    uint32_t bq[C::NTK][4][2];
+#pragma unroll
+    for (int nt = 0; nt < C::NTK; ++nt) {
+        const int col = 8 * nt + g, r = col >> 2, dig = col & 3;
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+#pragma unroll
+            for (int reg = 0; reg < 2; ++reg)
+                bq[nt][ks][reg] = (r < R) ? reinterpret_cast<const uint32_t *>(bimg0)[((((r * 4 + dig) * 4 + ks) * 2 + reg) * 4 + t)] : 0u;
+    }
+    __syncthreads();   // the image lives in the stage area: everyone has read it before any copy lands there
+    float cFr[R], sqr[R][NG];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        cFr[r] = cF[r];
+#pragma unroll
+        for (int gg = 0; gg < NG; ++gg) sqr[r][gg] = sqs[r * NG + gg];
     }
 
     // ---- per-warp pipeline state
     uint8_t *stage_base = warp_base;
-    float *Sc = reinterpret_cast<float *>(warp_base + C::kStages * C::kStageBytes);      // [64][R*NG]
+    float *Sc = reinterpret_cast<float *>(warp_base + C::kStages * C::kStageBytes);      // [64][NG][R][2]
     __half *Pt = reinterpret_cast<__half *>(warp_base + C::kStages * C::kStageBytes + C::kScBytes);
     uint64_t *bars = reinterpret_cast<uint64_t *>(warp_base + C::kStages * C::kStageBytes + C::kScBytes + C::kPBytes);
     const uint32_t bar0 = smem_u32(bars);
@@ -354,7 +410,7 @@ __global__ void __launch_bounds__(kThreads) partition_mma_kernel(MmaArgs a)
             for (int i = 0; i < 4; ++i) cv[nt][f][i] = 0.f;
 
     bool failed = false;
-    const int krot = (4 * t - 6) & 31;   // rotate right so that fields 2t, 2t+1 land on mantissa bits 6..9
+    const uint32_t kmask = 0x03030303u << (2 * t);
 
     for (int i = 0; i < n_my; ++i) {
         const int st = i % C::kStages;
@@ -366,7 +422,7 @@ __global__ void __launch_bounds__(kThreads) partition_mma_kernel(MmaArgs a)
         const __half2 *Vm = reinterpret_cast<const __half2 *>(Kc + 2 * C::kCodeTile + C::kMetaTile);
         const int tok0 = q_begin + (warp + i * kWarps) * kTileTok;
 
-        // ---------------- scores: C[token][head] per group
+        // ---------------- scores: exact integer dot products sum_j q'_j c_j per (token, head, group)
 #pragma unroll
         for (int mt = 0; mt < 4; ++mt) {
             const uint4 *r0 = reinterpret_cast<const uint4 *>(Kc + (16 * mt + g) * kRowBytes);
@@ -374,29 +430,33 @@ __global__ void __launch_bounds__(kThreads) partition_mma_kernel(MmaArgs a)
             const uint4 x0a = r0[0], x0b = r0[1], x1a = r1[0], x1b = r1[1];
             const uint32_t w0[8] = {x0a.x, x0a.y, x0a.z, x0a.w, x0b.x, x0b.y, x0b.z, x0b.w};
             const uint32_t w1[8] = {x1a.x, x1a.y, x1a.z, x1a.w, x1b.x, x1b.y, x1b.z, x1b.w};
-            float acc[NG][4];
+            int acc[C::NTK][NG][4];
 #pragma unroll
-            for (int gg = 0; gg < NG; ++gg)
+            for (int nt = 0; nt < C::NTK; ++nt)
 #pragma unroll
-                for (int e = 0; e < 4; ++e) acc[gg][e] = 0.f;
+                for (int gg = 0; gg < NG; ++gg)
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
-                constexpr uint32_t MAGIC = 0x4C004C00u, M6 = 0x00C000C0u, M8 = 0x03000300u;   // 16 + code, 16 + 4*code
-                const uint32_t rot0 = __funnelshift_r(w0[ks], w0[ks], krot);
-                const uint32_t rot1 = __funnelshift_r(w1[ks], w1[ks], krot);
-                mma16816(acc[(16 * ks) / G], and_or(rot0, M6, MAGIC), and_or(rot1, M6, MAGIC), and_or(rot0, M8, MAGIC),
-                         and_or(rot1, M8, MAGIC), bq[ks][0], bq[ks][1]);
+                    for (int e = 0; e < 4; ++e) acc[nt][gg][e] = 0;
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+                // byte b of (word & kmask) = 4^t * code(4b + t): four channels per AND, no shift
+                const uint32_t a0 = w0[2 * ks] & kmask, a1 = w1[2 * ks] & kmask;
+                const uint32_t a2 = w0[2 * ks + 1] & kmask, a3 = w1[2 * ks + 1] & kmask;
+#pragma unroll
+                for (int nt = 0; nt < C::NTK; ++nt) imma16832(acc[nt][(32 * ks) / G], a0, a1, a2, a3, bq[nt][ks][0], bq[nt][ks][1]);
             }
-            // lane (g,t) holds heads 2t, 2t+1 of tokens 16mt+g and 16mt+g+8
+            // lane (g,t) holds columns 2t, 2t+1 = two adjacent digits of one head for tokens 16mt+g and 16mt+g+8
 #pragma unroll
-            for (int gg = 0; gg < NG; ++gg) {
-                if (2 * t < R) {
-                    Sc[(16 * mt + g) * (R * NG) + (2 * t) * NG + gg] = acc[gg][0];
-                    Sc[(16 * mt + g + 8) * (R * NG) + (2 * t) * NG + gg] = acc[gg][2];
-                }
-                if (2 * t + 1 < R) {
-                    Sc[(16 * mt + g) * (R * NG) + (2 * t + 1) * NG + gg] = acc[gg][1];
-                    Sc[(16 * mt + g + 8) * (R * NG) + (2 * t + 1) * NG + gg] = acc[gg][3];
+            for (int nt = 0; nt < C::NTK; ++nt) {
+                const int r = (8 * nt + 2 * t) >> 2;
+                if (r < R) {
+#pragma unroll
+                    for (int gg = 0; gg < NG; ++gg) {
+                        const float lo = fmaf((float)acc[nt][gg][1], 256.0f, (float)acc[nt][gg][0]);
+                        const float hi = fmaf((float)acc[nt][gg][3], 256.0f, (float)acc[nt][gg][2]);
+                        Sc[(((16 * mt + g) * NG + gg) * R + r) * 2 + (t & 1)] = lo;
+                        Sc[(((16 * mt + g + 8) * NG + gg) * R + r) * 2 + (t & 1)] = hi;
+                    }
                 }
             }
         }
@@ -423,9 +483,10 @@ __global__ void __launch_bounds__(kThreads) partition_mma_kernel(MmaArgs a)
                 float sv = 0.f;
 #pragma unroll
                 for (int gg = 0; gg < NG; ++gg) {
-                    const float u = fmaf(Sc[tau * (R * NG) + r * NG + gg], a.scale_log2, -koff[r * NG + gg]);
+                    const float2 lh = *reinterpret_cast<const float2 *>(Sc + ((tau * NG + gg) * R + r) * 2);
+                    const float u = fmaf(lh.y, 65536.0f, lh.x) * cFr[r];      // scale * sum_j q'_j c_j
                     sv = fmaf(hk_[gg], u, sv);
-                    sv = fmaf(zk_[gg], sqs[r * NG + gg], sv);
+                    sv = fmaf(zk_[gg], sqr[r][gg], sv);
                 }
                 sc[hf][r] = valid[hf] ? sv : -CUDART_INF_F;
             }
@@ -437,11 +498,11 @@ __global__ void __launch_bounds__(kThreads) partition_mma_kernel(MmaArgs a)
         for (int r = 0; r < R; ++r) {
             const float tm = warp_max(fmaxf(sc[0][r], sc[1][r]));     // finite: the tile holds a valid token
             const float m_new = fmaxf(m_run[r], tm);
-            corr[r] = exp2f(m_run[r] - m_new);
+            corr[r] = ex2_approx(m_run[r] - m_new);
             rescale |= (m_new > m_run[r]);
             m_run[r] = m_new;
-            p[0][r] = valid[0] ? exp2f(sc[0][r] - m_new) : 0.f;
-            p[1][r] = valid[1] ? exp2f(sc[1][r] - m_new) : 0.f;
+            p[0][r] = valid[0] ? ex2_approx(sc[0][r] - m_new) : 0.f;
+            p[1][r] = valid[1] ? ex2_approx(sc[1][r] - m_new) : 0.f;
             l_part[r] = fmaf(l_part[r], corr[r], p[0][r] + p[1][r]);
 #pragma unroll
             for (int gg = 0; gg < NG; ++gg) { s_part[r][gg] *= corr[r]; z_part[r][gg] *= corr[r]; }
