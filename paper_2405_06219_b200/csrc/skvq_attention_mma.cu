@@ -69,6 +69,24 @@ __device__ __forceinline__ void imma16832(int (&d)[4], uint32_t a0, uint32_t a1,
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+__device__ __forceinline__ void imma16832_uu(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                             uint32_t b1)
+{
+    asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// Two 16x16 byte matrices, transposed: lanes 0-15 give the row addresses of the first, lanes 16-31 of the
+// second.  Lane (g,t) receives r0 = bytes (rows 4t..4t+3, column g), r1 = (rows 4t..4t+3, column g+8) of the
+// first matrix and r2, r3 likewise of the second: exactly the A fragment of mma.m16n8k32 with rows = byte
+// columns and k = matrix rows.
+__device__ __forceinline__ void ldmatrix_b8_trans_x2(uint32_t (&r)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m16n16.x2.trans.shared.b8 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+
 __device__ __forceinline__ float ex2_approx(float x)
 {
     float y;
@@ -122,7 +140,9 @@ __device__ __forceinline__ float warp_sum(float v)
 template <int G, int R>
 struct Cfg {
     static constexpr int NG = kHeadDim / G;
-    static constexpr int PIECES = (R * NG * 2 <= 8) ? 2 : 1;             // P split into hi+lo halves when columns allow
+    // Integer P.V path: one query head and at most two groups, so that (group, byte digit) fits the 8 MMA columns.
+    static constexpr bool VINT8 = (R == 1 && NG <= 2);
+    static constexpr int PIECES = (R * NG * 2 <= 8) ? 2 : 1;             // fp16 path: P split into hi+lo halves when columns allow
     static constexpr int NCV = R * NG * PIECES;                          // V-side columns: (head, group, piece)
     static constexpr int NTV = (NCV + 7) / 8;
     static constexpr int NCVP = NTV * 8;
@@ -132,7 +152,7 @@ struct Cfg {
     static constexpr int kStages = 2;
     static constexpr int NTK = (4 * R + 7) / 8;                          // K-side n-tiles: 4 byte digits per head
     static constexpr int kScBytes = kTileTok * R * NG * 8;               // per (token, group, head): low and high digit pairs
-    static constexpr int kPBytes = 4 * NCVP * 16 * 2;                    // P operand tile
+    static constexpr int kPBytes = VINT8 ? 2 * 8 * 32 : 4 * NCVP * 16 * 2;   // P operand tile
     static constexpr int kWarpBytes = kStages * kStageBytes + kScBytes + kPBytes + 64;   // + mbarriers
     static constexpr int kQBytes = (R * kHeadDim * 4 + R * NG * 4 + 2 * R * 4 + 64 + 127) / 128 * 128;
     static constexpr int kSmemBytes = kQBytes + kWarps * kWarpBytes;
@@ -401,16 +421,26 @@ __global__ void __launch_bounds__(kThreads) partition_mma_kernel(MmaArgs a)
 #pragma unroll
         for (int gg = 0; gg < NG; ++gg) { s_part[r][gg] = 0.f; z_part[r][gg] = 0.f; }
     }
-    float cv[C::NTV][8][4];
+    // fp16 P.V path: float accumulators cv.  Integer path: int accumulators iacc (exact while the softmax
+    // reference and the scale bound stay put) that are folded into fv whenever either one moves.
+    constexpr int NACC = C::VINT8 ? 1 : C::NTV;
+    float cv[NACC][8][4];
+    int iacc[C::VINT8 ? 8 : 1][4];
 #pragma unroll
-    for (int nt = 0; nt < C::NTV; ++nt)
+    for (int nt = 0; nt < NACC; ++nt)
 #pragma unroll
         for (int f = 0; f < 8; ++f)
 #pragma unroll
             for (int i = 0; i < 4; ++i) cv[nt][f][i] = 0.f;
+#pragma unroll
+    for (int f = 0; f < (C::VINT8 ? 8 : 1); ++f)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) iacc[f][i] = 0;
+    float h_bound = 6.103515625e-05f;   // 2^-14: every scale seen so far is below this power of two (integer path)
 
     bool failed = false;
     const uint32_t kmask = 0x03030303u << (2 * t);
+    uint8_t *Pb = reinterpret_cast<uint8_t *>(Pt);   // integer path: [2 k-blocks][8 columns][4 t][2 halves][4 tokens] bytes
 
     for (int i = 0; i < n_my; ++i) {
         const int st = i % C::kStages;
@@ -466,6 +496,7 @@ __global__ void __launch_bounds__(kThreads) partition_mma_kernel(MmaArgs a)
         float sc[2][R];
         bool valid[2];
         float hv[2][NG], zv[2][NG];
+        bool moved = false;   // does any score exceed the running maximum, or any scale the running bound?
 #pragma unroll
         for (int hf = 0; hf < 2; ++hf) {
             const int tau = lane + 32 * hf;
@@ -476,7 +507,9 @@ __global__ void __launch_bounds__(kThreads) partition_mma_kernel(MmaArgs a)
                 const float2 kz = __half22float2(Km[tau * NG + gg]);
                 const float2 vz = __half22float2(Vm[tau * NG + gg]);
                 hk_[gg] = kz.x; zk_[gg] = kz.y;
-                hv[hf][gg] = vz.x; zv[hf][gg] = vz.y;
+                hv[hf][gg] = valid[hf] ? vz.x : 0.f;      // rows past the end hold unspecified bytes
+                zv[hf][gg] = valid[hf] ? vz.y : 0.f;
+                if (C::VINT8) moved |= (hv[hf][gg] >= h_bound);
             }
 #pragma unroll
             for (int r = 0; r < R; ++r) {
@@ -489,87 +522,145 @@ __global__ void __launch_bounds__(kThreads) partition_mma_kernel(MmaArgs a)
                     sv = fmaf(zk_[gg], sqr[r][gg], sv);
                 }
                 sc[hf][r] = valid[hf] ? sv : -CUDART_INF_F;
+                moved |= (sc[hf][r] > m_run[r]);
             }
         }
-        float corr[R];
-        bool rescale = false;
+        if (__any_sync(0xffffffffu, moved)) {
+            // Rare after the first tiles: raise the references and bring every running sum onto them.
+            float corr[R];
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const float m_new = fmaxf(m_run[r], warp_max(fmaxf(sc[0][r], sc[1][r])));
+                corr[r] = ex2_approx(m_run[r] - m_new);      // 0 on the first tile (m_run = -inf)
+                m_run[r] = m_new;
+                l_part[r] *= corr[r];
+#pragma unroll
+                for (int gg = 0; gg < NG; ++gg) { s_part[r][gg] *= corr[r]; z_part[r][gg] *= corr[r]; }
+            }
+            if constexpr (C::VINT8) {
+                float hm = 0.f;
+#pragma unroll
+                for (int gg = 0; gg < NG; ++gg) hm = fmaxf(hm, fmaxf(hv[0][gg], hv[1][gg]));
+                hm = warp_max(hm);
+                // fold the integer sums into fv: value = iacc * 256^digit * h_bound * 2^-32, columns 2t, 2t+1 = digits 2(t&1), +1
+                const float f0 = h_bound * ((t & 1) ? 1.52587890625e-05f : 2.3283064365386963e-10f);   // 2^-16 : 2^-32
+                const float f1 = f0 * 256.0f;
+#pragma unroll
+                for (int f = 0; f < 8; ++f) {
+                    cv[0][f][0] = fmaf((float)iacc[f][0], f0, cv[0][f][0]) * corr[0];
+                    cv[0][f][1] = fmaf((float)iacc[f][1], f1, cv[0][f][1]) * corr[0];
+                    cv[0][f][2] = fmaf((float)iacc[f][2], f0, cv[0][f][2]) * corr[0];
+                    cv[0][f][3] = fmaf((float)iacc[f][3], f1, cv[0][f][3]) * corr[0];
+                    iacc[f][0] = 0; iacc[f][1] = 0; iacc[f][2] = 0; iacc[f][3] = 0;
+                }
+                if (hm >= h_bound) h_bound = __int_as_float(((__float_as_int(hm) >> 23) + 1) << 23);   // next power of two above hm
+            } else {
+#pragma unroll
+                for (int nt = 0; nt < C::NTV; ++nt) {
+                    // this lane's two columns and the heads they belong to
+                    const int c0 = 8 * nt + 2 * t, c1 = c0 + 1;
+                    float f0 = 1.f, f1 = 1.f;
+#pragma unroll
+                    for (int r = 0; r < R; ++r) {
+                        if (c0 / (NG * C::PIECES) == r) f0 = corr[r];
+                        if (c1 / (NG * C::PIECES) == r) f1 = corr[r];
+                    }
+#pragma unroll
+                    for (int f = 0; f < 8; ++f) {
+                        cv[nt][f][0] *= f0; cv[nt][f][2] *= f0;
+                        cv[nt][f][1] *= f1; cv[nt][f][3] *= f1;
+                    }
+                }
+            }
+        }
         float p[2][R];
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-            const float tm = warp_max(fmaxf(sc[0][r], sc[1][r]));     // finite: the tile holds a valid token
-            const float m_new = fmaxf(m_run[r], tm);
-            corr[r] = ex2_approx(m_run[r] - m_new);
-            rescale |= (m_new > m_run[r]);
-            m_run[r] = m_new;
-            p[0][r] = valid[0] ? ex2_approx(sc[0][r] - m_new) : 0.f;
-            p[1][r] = valid[1] ? ex2_approx(sc[1][r] - m_new) : 0.f;
-            l_part[r] = fmaf(l_part[r], corr[r], p[0][r] + p[1][r]);
-#pragma unroll
-            for (int gg = 0; gg < NG; ++gg) { s_part[r][gg] *= corr[r]; z_part[r][gg] *= corr[r]; }
+            p[0][r] = ex2_approx(sc[0][r] - m_run[r]);      // exp2(-inf) = 0 for tokens past the end
+            p[1][r] = ex2_approx(sc[1][r] - m_run[r]);
+            l_part[r] += p[0][r] + p[1][r];
         }
-        // P operand: value (p*h) per (head, group), split into fp16 hi (+ lo) pieces.
-        //   k index of the PV MMAs: k=2t'<->token t', 2t'+1<->t'+4, 2t'+8<->t'+8, 2t'+9<->t'+12 within a 16-token block
+        if constexpr (C::VINT8) {
+            // P operand (u8): p*h on a 32-bit fixed-point grid below h_bound; the four bytes of that integer are
+            // the four digit columns of the token.  Token tau is k index (tau & 31) of k-block tau >> 5.
+            const float hscale = 4294967296.0f / h_bound;
 #pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-            const int tau = lane + 32 * hf;
-            const int kb = tau >> 4, tt = tau & 3, ii = (tau & 15) >> 2;
-#pragma unroll
-            for (int r = 0; r < R; ++r)
+            for (int hf = 0; hf < 2; ++hf) {
+                uint8_t *dst = Pb + (hf * 8 * 4 + ((lane >> 2) & 3)) * 8 + (lane >> 4) * 4 + (lane & 3);
 #pragma unroll
                 for (int gg = 0; gg < NG; ++gg) {
-                    const float ph = valid[hf] ? p[hf][r] * hv[hf][gg] : 0.f;
-                    const float pz = valid[hf] ? p[hf][r] * zv[hf][gg] : 0.f;
-                    const __half hi = __float2half_rn(ph);
-                    float used = __half2float(hi);
-                    const int col = (r * NG + gg) * C::PIECES;
-                    Pt[((kb * C::NCVP + col) * 4 + tt) * 4 + ii] = hi;
-                    if (C::PIECES == 2) {
-                        const __half lo = __float2half_rn(ph - used);
-                        used += __half2float(lo);
-                        Pt[((kb * C::NCVP + col + 1) * 4 + tt) * 4 + ii] = lo;
+                    uint32_t fx;
+                    asm("cvt.rni.sat.u32.f32 %0, %1;" : "=r"(fx) : "f"(p[hf][0] * hv[hf][gg] * hscale));
+                    z_part[0][gg] = fmaf(p[hf][0], zv[hf][gg], z_part[0][gg]);
+#pragma unroll
+                    for (int dg = 0; dg < 4; ++dg) dst[(gg * 4 + dg) * 32] = (uint8_t)(fx >> (8 * dg));
+                }
+            }
+        } else {
+            // P operand: value (p*h) per (head, group), split into fp16 hi (+ lo) pieces.
+            //   k index of the PV MMAs: k=2t'<->token t', 2t'+1<->t'+4, 2t'+8<->t'+8, 2t'+9<->t'+12 within a 16-token block
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+                const int tau = lane + 32 * hf;
+                const int kb = tau >> 4, tt = tau & 3, ii = (tau & 15) >> 2;
+#pragma unroll
+                for (int r = 0; r < R; ++r)
+#pragma unroll
+                    for (int gg = 0; gg < NG; ++gg) {
+                        const float ph = p[hf][r] * hv[hf][gg];
+                        const __half hi = __float2half_rn(ph);
+                        float used = __half2float(hi);
+                        const int col = (r * NG + gg) * C::PIECES;
+                        Pt[((kb * C::NCVP + col) * 4 + tt) * 4 + ii] = hi;
+                        if (C::PIECES == 2) {
+                            const __half lo = __float2half_rn(ph - used);
+                            used += __half2float(lo);
+                            Pt[((kb * C::NCVP + col + 1) * 4 + tt) * 4 + ii] = lo;
+                        }
+                        s_part[r][gg] += used;
+                        z_part[r][gg] = fmaf(p[hf][r], zv[hf][gg], z_part[r][gg]);
                     }
-                    s_part[r][gg] += used;
-                    z_part[r][gg] += pz;
-                }
-        }
-        if (rescale) {   // warp-uniform
-#pragma unroll
-            for (int nt = 0; nt < C::NTV; ++nt) {
-                // this lane's two columns and the heads they belong to
-                const int c0 = 8 * nt + 2 * t, c1 = c0 + 1;
-                float f0 = 1.f, f1 = 1.f;
-#pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    if (c0 / (NG * C::PIECES) == r) f0 = corr[r];
-                    if (c1 / (NG * C::PIECES) == r) f1 = corr[r];
-                }
-#pragma unroll
-                for (int f = 0; f < 8; ++f) {
-                    cv[nt][f][0] *= f0; cv[nt][f][2] *= f0;
-                    cv[nt][f][1] *= f1; cv[nt][f][3] *= f1;
-                }
             }
         }
         __syncwarp();
 
-        // ---------------- P.V: rows = channels (lane g reads code word g), k = tokens
+        if constexpr (C::VINT8) {
+            // ---------------- P.V in int8: rows = channels 4*(byte column) + j, k = 32 tokens per MMA
+            const uint32_t vaddr = smem_u32(Vc) + lane * kRowBytes;   // lanes 0-15: tokens 0-15, lanes 16-31: tokens 16-31
 #pragma unroll
-        for (int kb = 0; kb < 4; ++kb) {
-            const uint32_t *vrow = reinterpret_cast<const uint32_t *>(Vc + (16 * kb + t) * kRowBytes) + g;
-            const uint32_t x0 = vrow[0], x1 = vrow[4 * 8], x2 = vrow[8 * 8], x3 = vrow[12 * 8];   // tokens t, t+4, t+8, t+12
-            uint32_t A0[8], A1[8], A2[8], A3[8];
-            unpack_v(__byte_perm(x0, x1, 0x5410), A0);   // low halves: channels 16g+f,   tokens (t, t+4)
-            unpack_v(__byte_perm(x0, x1, 0x7632), A1);   // high halves: channels 16g+8+f
-            unpack_v(__byte_perm(x2, x3, 0x5410), A2);   // tokens (t+8, t+12)
-            unpack_v(__byte_perm(x2, x3, 0x7632), A3);
+            for (int kk = 0; kk < 2; ++kk) {
+                const uint2 pb = *reinterpret_cast<const uint2 *>(Pb + ((kk * 8 + g) * 4 + t) * 8);
 #pragma unroll
-            for (int nt = 0; nt < C::NTV; ++nt) {
-                const uint2 pb = *reinterpret_cast<const uint2 *>(Pt + ((kb * C::NCVP + 8 * nt + g) * 4 + t) * 4);
+                for (int hh = 0; hh < 2; ++hh) {
+                    uint32_t rr[4];
+                    ldmatrix_b8_trans_x2(rr, vaddr + kk * 32 * kRowBytes + hh * 16);
 #pragma unroll
-                for (int f = 0; f < 8; ++f) mma16816(cv[nt][f], A0[f], A1[f], A2[f], A3[f], pb.x, pb.y);
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t m = 0x03030303u << (2 * j);
+                        imma16832_uu(iacc[hh * 4 + j], rr[0] & m, rr[1] & m, rr[2] & m, rr[3] & m, pb.x, pb.y);
+                    }
+                }
+            }
+        } else {
+            // ---------------- P.V in fp16: rows = channels (lane g reads code word g), k = tokens
+#pragma unroll
+            for (int kb = 0; kb < 4; ++kb) {
+                const uint32_t *vrow = reinterpret_cast<const uint32_t *>(Vc + (16 * kb + t) * kRowBytes) + g;
+                const uint32_t x0 = vrow[0], x1 = vrow[4 * 8], x2 = vrow[8 * 8], x3 = vrow[12 * 8];   // tokens t, t+4, t+8, t+12
+                uint32_t A0[8], A1[8], A2[8], A3[8];
+                unpack_v(__byte_perm(x0, x1, 0x5410), A0);   // low halves: channels 16g+f,   tokens (t, t+4)
+                unpack_v(__byte_perm(x0, x1, 0x7632), A1);   // high halves: channels 16g+8+f
+                unpack_v(__byte_perm(x2, x3, 0x5410), A2);   // tokens (t+8, t+12)
+                unpack_v(__byte_perm(x2, x3, 0x7632), A3);
+#pragma unroll
+                for (int nt = 0; nt < C::NTV; ++nt) {
+                    const uint2 pb = *reinterpret_cast<const uint2 *>(Pt + ((kb * C::NCVP + 8 * nt + g) * 4 + t) * 4);
+#pragma unroll
+                    for (int f = 0; f < 8; ++f) mma16816(cv[nt][f], A0[f], A1[f], A2[f], A3[f], pb.x, pb.y);
+                }
             }
         }
-        __syncwarp();   // every lane is done with this stage, Sc and Pt
+        __syncwarp();   // every lane is done with this stage, Sc and the P tile
         if (lane == 0 && i + C::kStages < n_my) issue(i + C::kStages);
     }
 
@@ -589,43 +680,76 @@ __global__ void __launch_bounds__(kThreads) partition_mma_kernel(MmaArgs a)
     float *Ow = Ot + C::NCV * kHeadDim;                                      // [R][132]: o', m, l
     __syncwarp();
 #pragma unroll
-    for (int nt = 0; nt < C::NTV; ++nt) {
-        const int c0 = 8 * nt + 2 * t;
-#pragma unroll
-        for (int f = 0; f < 8; ++f) {
-            if (c0 < C::NCV) {
-                Ot[c0 * kHeadDim + 16 * g + f] = cv[nt][f][0];
-                Ot[c0 * kHeadDim + 16 * g + 8 + f] = cv[nt][f][2];
-            }
-            if (c0 + 1 < C::NCV) {
-                Ot[(c0 + 1) * kHeadDim + 16 * g + f] = cv[nt][f][1];
-                Ot[(c0 + 1) * kHeadDim + 16 * g + 8 + f] = cv[nt][f][3];
-            }
-        }
-    }
-#pragma unroll
     for (int r = 0; r < R; ++r) {
         l_part[r] = warp_sum(l_part[r]);
 #pragma unroll
         for (int gg = 0; gg < NG; ++gg) { s_part[r][gg] = warp_sum(s_part[r][gg]); z_part[r][gg] = warp_sum(z_part[r][gg]); }
     }
-    __syncwarp();
+    if constexpr (C::VINT8) {
+        // last fold of the integer sums, then add the four digit columns of each group: a lane pair (t, t^1) holds them
+        const float f0 = h_bound * ((t & 1) ? 1.52587890625e-05f : 2.3283064365386963e-10f);
+        const float f1 = f0 * 256.0f;
 #pragma unroll
-    for (int q4 = 0; q4 < 4; ++q4) {
-        const int d = lane + 32 * q4;
-        const float winv = v_weight_inv(d & 7);
+        for (int f = 0; f < 8; ++f) {
+            float lo = fmaf((float)iacc[f][0], f0, cv[0][f][0]) + fmaf((float)iacc[f][1], f1, cv[0][f][1]);   // byte column (f>>2)*16+g
+            float hi = fmaf((float)iacc[f][2], f0, cv[0][f][2]) + fmaf((float)iacc[f][3], f1, cv[0][f][3]);   // byte column +8
+            lo += __shfl_xor_sync(0xffffffffu, lo, 1);
+            hi += __shfl_xor_sync(0xffffffffu, hi, 1);
+            // lanes t = 0,1 carry group 0, lanes t = 2,3 group 1; the even lane of each pair stores
+            const int gg = t >> 1;
+            if ((t & 1) == 0 && gg < NG) {
+                const int bc = (f >> 2) * 16 + g, j = f & 3;
+                Ot[gg * kHeadDim + 4 * bc + j] = lo;
+                Ot[gg * kHeadDim + 4 * (bc + 8) + j] = hi;
+            }
+        }
+        __syncwarp();
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-            float sg = 0.f, zg = 0.f;
+        for (int q4 = 0; q4 < 4; ++q4) {
+            const int d = lane + 32 * q4;
+            const int j = d & 3;                                      // channel d = 4*(byte column) + j carries weight 4^j
+            const float winv = j == 0 ? 1.0f : (j == 1 ? 0.25f : (j == 2 ? 0.0625f : 0.015625f));
+            float zg = 0.f;
 #pragma unroll
             for (int gg = 0; gg < NG; ++gg)
-                if (d / G == gg) { sg = s_part[r][gg]; zg = z_part[r][gg]; }
-            const int col = (r * NG + d / G) * C::PIECES;
-            float o = Ot[col * kHeadDim + d];
-            if (C::PIECES == 2) o += Ot[(col + 1) * kHeadDim + d];
-            // remove the constant 64 carried by every unpacked code, undo the field weight, add the zero points
-            o = (o - 64.0f * sg) * winv + zg;
-            Ow[r * kPartialStride + d] = failed ? 0.f : o;
+                if (d / G == gg) zg = z_part[0][gg];
+            const float o = Ot[(d / G) * kHeadDim + d] * winv + zg;
+            Ow[d] = failed ? 0.f : o;
+        }
+    } else {
+#pragma unroll
+        for (int nt = 0; nt < C::NTV; ++nt) {
+            const int c0 = 8 * nt + 2 * t;
+#pragma unroll
+            for (int f = 0; f < 8; ++f) {
+                if (c0 < C::NCV) {
+                    Ot[c0 * kHeadDim + 16 * g + f] = cv[nt][f][0];
+                    Ot[c0 * kHeadDim + 16 * g + 8 + f] = cv[nt][f][2];
+                }
+                if (c0 + 1 < C::NCV) {
+                    Ot[(c0 + 1) * kHeadDim + 16 * g + f] = cv[nt][f][1];
+                    Ot[(c0 + 1) * kHeadDim + 16 * g + 8 + f] = cv[nt][f][3];
+                }
+            }
+        }
+        __syncwarp();
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+            const int d = lane + 32 * q4;
+            const float winv = v_weight_inv(d & 7);
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                float sg = 0.f, zg = 0.f;
+#pragma unroll
+                for (int gg = 0; gg < NG; ++gg)
+                    if (d / G == gg) { sg = s_part[r][gg]; zg = z_part[r][gg]; }
+                const int col = (r * NG + d / G) * C::PIECES;
+                float o = Ot[col * kHeadDim + d];
+                if (C::PIECES == 2) o += Ot[(col + 1) * kHeadDim + d];
+                // remove the constant 64 carried by every unpacked code, undo the field weight, add the zero points
+                o = (o - 64.0f * sg) * winv + zg;
+                Ow[r * kPartialStride + d] = failed ? 0.f : o;
+            }
         }
     }
     if (lane < R) {
