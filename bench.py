@@ -105,8 +105,10 @@ def build_gpu_cache(w, extra_tokens, torch, binding):
     ms, moved = 0.0, 0
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     Lmax = int(lengths.max())
-    for t0 in range(0, Lmax, PREFILL_CHUNK):
-        t1 = min(t0 + PREFILL_CHUNK, Lmax)
+    # host staging of one chunk stays near 1 GiB per tensor whatever the batch size
+    chunk = max(256, min(PREFILL_CHUNK, (1 << 30) // (w.batch * w.n_kv_heads * w.head_dim * 2) // 256 * 256))
+    for t0 in range(0, Lmax, chunk):
+        t1 = min(t0 + chunk, Lmax)
         n_b = np.clip(lengths - t0, 0, t1 - t0).astype(np.int32)
         k = np.zeros((w.batch, t1 - t0, w.n_kv_heads, w.head_dim), np.float16)
         v = np.zeros_like(k)
