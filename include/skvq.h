@@ -39,6 +39,8 @@ extern "C" {
 #define SKVQ_ERR_CAPACITY (-4)    /* host-visible overflow: n_new or max_len_hint beyond max_tokens */
 #define SKVQ_ERR_WORKSPACE (-5)   /* workspace missing or smaller than skvq_workspace_size() */
 #define SKVQ_ERR_CUDA (-6)        /* the CUDA runtime reported an error at launch */
+#define SKVQ_ERR_SCRATCH_LIMIT (-7) /* skvq_decode_attention_noalloc: the split partials of this shape need more
+                                     than SKVQ_NOALLOC_SCRATCH_BYTES */
 
 #define SKVQ_STATUS_OVERFLOW 1    /* bit set in *status when a sequence would have exceeded max_tokens */
 
@@ -159,6 +161,33 @@ size_t skvq_step_staging_size(const skvq_config *cfg);
 int skvq_decode_step_host(const skvq_config *cfg, const skvq_cache *cache, const void *k_new_host,
                           const void *v_new_host, const void *q_host, void *out_host, void *staging,
                           const skvq_attn_args *args, void *cuda_stream);
+
+/*
+ * Decode attention for callers that have no device memory left to lend and must not allocate.
+ * (The paper has no counterpart: this is a packaging variant of skvq_decode_attention, same result.)
+ *
+ * Who needs it: a serving engine usually sizes its KV cache to swallow whatever HBM remains after the
+ * weights, so by the time the decode loop runs there is no spare buffer to pass as `workspace`, and a
+ * cudaMalloc inside that loop would either fail or stall every stream on the device while it runs.  The
+ * same holds for code that runs as a plug-in inside somebody else's memory pool and may not call the
+ * allocator at all.  For them the split partials go into an array that is part of the library image:
+ * SKVQ_NOALLOC_SCRATCH_BYTES of device memory on every GPU that loads the library, held until exit.
+ * The call itself allocates and frees nothing (no cudaMalloc/cudaFree, no allocating library routine).
+ *
+ * Arguments are those of skvq_decode_attention with the fields of skvq_attn_args passed directly; q, out and
+ * the cache are still the caller's.  Limits and rules:
+ *   - Shapes whose partials need more than SKVQ_NOALLOC_SCRATCH_BYTES (that is,
+ *     skvq_workspace_size(cfg, max_len_hint, n_splits) > SKVQ_NOALLOC_SCRATCH_BYTES) are refused with
+ *     SKVQ_ERR_SCRATCH_LIMIT before anything is launched; ask for fewer splits or use the workspace variant.
+ *   - The first call on each device looks up the array's device address (with that device current).  Make
+ *     that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps whatever the last call left there.  Nothing
+ *     needs clearing (a call writes every partial before it reads it), but two calls that overlap on the GPU
+ *     -- different streams, no ordering between them -- race on it.  Keep them stream-ordered.
+ */
+#define SKVQ_NOALLOC_SCRATCH_BYTES (8u << 20)
+int skvq_decode_attention_noalloc(const skvq_config *cfg, const skvq_cache *cache, const void *q, void *out,
+                                  float sm_scale, int32_t max_len_hint, int32_t n_splits, void *cuda_stream);
 
 #ifdef __cplusplus
 }

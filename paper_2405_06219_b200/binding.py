@@ -17,12 +17,14 @@ _lib = None
 SKVQ_OK = 0
 SKVQ_ERR_INVALID_ARG, SKVQ_ERR_UNSUPPORTED, SKVQ_ERR_MISALIGNED = -1, -2, -3
 SKVQ_ERR_CAPACITY, SKVQ_ERR_WORKSPACE, SKVQ_ERR_CUDA = -4, -5, -6
+SKVQ_ERR_SCRATCH_LIMIT = -7
+SKVQ_NOALLOC_SCRATCH_BYTES = 8 << 20
 SKVQ_STATUS_OVERFLOW = 1
 SKVQ_TOKEN_ALIGN = 64
 
 EXPORTS = ["skvq_version", "skvq_strerror", "skvq_launch_count", "skvq_check_config", "skvq_quant_capacity",
            "skvq_cache_sizes", "skvq_quantize_append", "skvq_workspace_size", "skvq_decode_attention",
-           "skvq_step_staging_size", "skvq_decode_step_host"]
+           "skvq_step_staging_size", "skvq_decode_step_host", "skvq_decode_attention_noalloc"]
 
 
 class SkvqConfig(ctypes.Structure):
@@ -76,6 +78,9 @@ def lib() -> ctypes.CDLL:
         L.skvq_step_staging_size.argtypes = [P(SkvqConfig)]
         L.skvq_decode_step_host.restype = c_int
         L.skvq_decode_step_host.argtypes = [P(SkvqConfig), P(SkvqCacheStruct), vp, vp, vp, vp, vp, P(SkvqAttnArgs), vp]
+        L.skvq_decode_attention_noalloc.restype = c_int
+        L.skvq_decode_attention_noalloc.argtypes = [P(SkvqConfig), P(SkvqCacheStruct), vp, vp, ctypes.c_float,
+                                                    ctypes.c_int32, ctypes.c_int32, vp]
         _lib = L
     return _lib
 
@@ -143,6 +148,14 @@ def skvq_decode_step_host(cfg, cache, k_new_host, v_new_host, q_host, out_host, 
     _check(lib().skvq_decode_step_host(ctypes.byref(cfg), ctypes.byref(cache), k_new_host.data_ptr(),
                                        v_new_host.data_ptr(), q_host.data_ptr(), out_host.data_ptr(),
                                        _dptr(staging), ctypes.byref(args), _stream(stream)), "skvq_decode_step_host")
+
+
+def skvq_decode_attention_noalloc(cfg, cache, q, out, sm_scale, max_len_hint, n_splits=0, stream=None) -> None:
+    """Decode attention whose split scratch is the library's built-in device array: for callers that cannot
+    allocate or lend a workspace.  Shapes beyond SKVQ_NOALLOC_SCRATCH_BYTES raise SkvqError(SKVQ_ERR_SCRATCH_LIMIT)."""
+    _check(lib().skvq_decode_attention_noalloc(ctypes.byref(cfg), ctypes.byref(cache), _dptr(q), _dptr(out),
+                                               float(sm_scale), int(max_len_hint), int(n_splits), _stream(stream)),
+           "skvq_decode_attention_noalloc")
 
 
 # ---------------------------------------------------------------- device-memory holder

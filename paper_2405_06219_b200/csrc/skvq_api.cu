@@ -99,6 +99,7 @@ const char *skvq_strerror(int code)
         case SKVQ_ERR_CAPACITY: return "token count exceeds the cache capacity";
         case SKVQ_ERR_WORKSPACE: return "workspace missing or too small";
         case SKVQ_ERR_CUDA: return "CUDA runtime error at launch";
+        case SKVQ_ERR_SCRATCH_LIMIT: return "split partials exceed the library's built-in scratch array";
         default: return "unknown error code";
     }
 }
@@ -211,6 +212,57 @@ int skvq_decode_step_host(const skvq_config *cfg, const skvq_cache *cache, const
     if (rc != SKVQ_OK) return rc;
     if (cudaMemcpyAsync(out_host, d_out, qo, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return SKVQ_ERR_CUDA;
     return SKVQ_OK;
+}
+
+// ---------------------------------------------------------------- decode attention without a caller workspace
+// Split partials of skvq_decode_attention_noalloc live in this array instead of caller memory.  Every GPU that
+// loads the library carries it until the process exits.  In host code the name below is only a handle for
+// cudaGetSymbolAddress; the kernels are given the device address that call returns.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[SKVQ_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::atomic<float *> g_noalloc_ptr[kMaxDevices];
+
+// Device address of the array on the current device, looked up once per device.
+int noalloc_scratch(float **out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SKVQ_ERR_CUDA;
+    float *p = g_noalloc_ptr[dev].load(std::memory_order_acquire);
+    if (!p) {
+        void *sym = nullptr;
+        if (cudaGetSymbolAddress(&sym, g_noalloc_scratch) != cudaSuccess || !sym) return SKVQ_ERR_CUDA;
+        p = static_cast<float *>(sym);
+        g_noalloc_ptr[dev].store(p, std::memory_order_release);   // racing threads store the same address
+    }
+    *out = p;
+    return SKVQ_OK;
+}
+}  // namespace
+
+int skvq_decode_attention_noalloc(const skvq_config *cfg, const skvq_cache *cache, const void *q, void *out,
+                                  float sm_scale, int32_t max_len_hint, int32_t n_splits, void *cuda_stream)
+{
+    int rc = check_cfg(cfg);
+    if (rc != SKVQ_OK) return rc;
+    CachePtrs c;
+    rc = check_cache(cfg, cache, &c);
+    if (rc != SKVQ_OK) return rc;
+    if (!q || !out) return SKVQ_ERR_INVALID_ARG;
+    if (misaligned(q) || misaligned(out)) return SKVQ_ERR_MISALIGNED;
+    if (max_len_hint < 0 || n_splits < 0) return SKVQ_ERR_INVALID_ARG;
+    if (max_len_hint > cfg->max_tokens) return SKVQ_ERR_CAPACITY;
+    const Shape s = make_shape(cfg);
+    const SplitPlan plan = plan_splits(s, max_len_hint, n_splits);
+    if (workspace_bytes(s, plan) > (size_t)SKVQ_NOALLOC_SCRATCH_BYTES) return SKVQ_ERR_SCRATCH_LIMIT;
+    float *scratch = nullptr;
+    rc = noalloc_scratch(&scratch);
+    if (rc != SKVQ_OK) return rc;
+    // Nothing in the array has to start at zero: every partial the merge reads is written by this call first.
+    const cudaError_t e = launch_attention(s, c, static_cast<const __half *>(q), static_cast<__half *>(out), sm_scale,
+                                           plan, scratch, nullptr, nullptr, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? SKVQ_OK : SKVQ_ERR_CUDA;
 }
 
 }  // extern "C"
