@@ -277,6 +277,10 @@ cudaError_t launch_attention(const Shape &s, const CachePtrs &c, const __half *q
     bool handled = false;
     cudaError_t em = launch_partition_mma(s, c, q, a.scale_log2, plan, workspace, stream, &handled);
     if (em != cudaSuccess) return em;
+    if (!handled) {
+        em = launch_partition_gqa(s, c, q, a.scale_log2, plan, workspace, stream, &handled);
+        if (em != cudaSuccess) return em;
+    }
     if (handled) { /* tensor-core kernel launched */ }
     else if (s.k_bits == 2 && s.v_bits == 2) partition_kernel<2, 2><<<grid, kThreads, 0, stream>>>(a);
     else if (s.k_bits == 4 && s.v_bits == 4) partition_kernel<4, 4><<<grid, kThreads, 0, stream>>>(a);

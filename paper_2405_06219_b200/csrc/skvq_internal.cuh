@@ -48,6 +48,9 @@ cudaError_t launch_attention(const Shape &s, const CachePtrs &c, const __half *q
 cudaError_t launch_partition_mma(const Shape &s, const CachePtrs &c, const __half *q, float scale_log2,
                                  const SplitPlan &plan, float *workspace, cudaStream_t stream, bool *handled);
 
+cudaError_t launch_partition_gqa(const Shape &s, const CachePtrs &c, const __half *q, float scale_log2,
+                                 const SplitPlan &plan, float *workspace, cudaStream_t stream, bool *handled);
+
 void count_launch(int n = 1);
 
 }  // namespace skvq

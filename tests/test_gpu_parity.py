@@ -112,6 +112,11 @@ def test_ragged_append_and_overflow_flag():
     (0, dict(context=100), 100), (0, dict(context=128), 128), (0, dict(context=129), 129),
     (0, dict(context=1), 1), (0, dict(context=500, window=0), 500),
     (2, dict(context=777, batch=1, n_q_heads=16, n_kv_heads=2), 777),   # 8 query heads per KV head
+    (2, dict(context=3000, batch=1, n_q_heads=8, n_kv_heads=4), 3000),                    # 2 heads per KV head, g32
+    (1, dict(context=3000, batch=1, n_q_heads=8, n_kv_heads=2), 3000),                    # 4 heads per KV head, g128
+    (1, dict(context=2500, batch=2, n_q_heads=4, n_kv_heads=4, group_size=32), 2500),     # MHA with fine groups
+    (1, dict(context=2500, batch=1, n_q_heads=8, n_kv_heads=4, group_size=64), 2500),     # 2 heads per KV head, g64
+    (2, dict(context=4160, batch=1, n_q_heads=4, n_kv_heads=1, group_size=64), 4160),     # 4 heads per KV head, g64, full tiles only
 ])
 def test_attention_matches_oracle(cfg_i, kw, n):
     w = small(cfg_i, **kw)
