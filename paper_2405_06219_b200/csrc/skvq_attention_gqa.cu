@@ -38,12 +38,10 @@ struct GCfg {
     static constexpr int kMetaTile = kTileTok * NG * 4;
     static constexpr int kStageBytes = 2 * kCodeTile + 2 * kMetaTile;
     static constexpr int kStages = 2;
-    static constexpr int kPStride = 68;                                  // floats per head row of the P tile (bank spread)
-    static constexpr int kPBytes = kHeadSlots * kPStride * 4;
-    static constexpr int kHBytes = kTileTok * NG * 4;                    // h_v * fixed-point scale per (token, group)
+    static constexpr int kXBytes = NG * 2 * 32 * 8;                      // digit registers on their way to the A fragments
     static constexpr int kOBytes = kHeadSlots * kHeadDim * 4;            // folded P.V sums
     static constexpr int kZBytes = kHeadSlots * 4 * 4;                   // sum p*z per (head, group)
-    static constexpr int kWarpBytes = kStages * kStageBytes + kPBytes + kHBytes + kOBytes + kZBytes + 64;
+    static constexpr int kWarpBytes = kStages * kStageBytes + kXBytes + kOBytes + kZBytes + 64;
     static constexpr int kQFloats = kHeadSlots * kHeadDim + 2 * kHeadSlots * 4 + 2 * kHeadSlots + kWarps * kHeadSlots;
     static constexpr int kQBytes = (kQFloats * 4 + 127) / 128 * 128;
     static constexpr int kSmemBytes = kQBytes + kWarps * kWarpBytes;
@@ -55,6 +53,22 @@ __device__ __forceinline__ float field_weight_inv(int f)
 {
     const int sel = (f == 0 || f == 5) ? 0 : ((f == 1 || f == 3 || f == 6) ? 1 : 2);
     return sel == 0 ? 1.0f : (sel == 1 ? 0.25f : 0.0625f);
+}
+
+// Eight half2 operands (value 64 + w_f*code, w = {1,4,16,4,16,1,4,16}) from one packed word: register f holds
+// field f of the low half (channel f of the word) and of the high half (channel f + 8).
+__device__ __forceinline__ void unpack16(uint32_t x, uint32_t (&o)[8])
+{
+    constexpr uint32_t MAGIC = 0x54005400u, M4 = 0x00300030u, M6 = 0x00C000C0u, M8 = 0x03000300u;
+    const uint32_t s0 = x << 4, s2 = x >> 6;
+    o[0] = and_or(s0, M4, MAGIC);
+    o[1] = and_or(s0, M6, MAGIC);
+    o[2] = and_or(s0, M8, MAGIC);
+    o[3] = and_or(x, M6, MAGIC);
+    o[4] = and_or(x, M8, MAGIC);
+    o[5] = and_or(s2, M4, MAGIC);
+    o[6] = and_or(s2, M6, MAGIC);
+    o[7] = and_or(s2, M8, MAGIC);
 }
 
 __device__ __forceinline__ uint32_t pack_half2(float lo, float hi)
@@ -76,6 +90,35 @@ __device__ __forceinline__ uint32_t to_fixed_u32(float x)
     asm("cvt.rni.sat.u32.f32 %0, %1;" : "=r"(r) : "f"(x));
     return r;
 }
+
+// Four 8x8 b16 matrices (rows of 16 bytes): lane (g, t) receives word t of row g of each matrix.
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+
+template <int NG>
+__device__ __forceinline__ void load_words(const uint32_t *p, uint32_t (&w)[NG])
+{
+    if constexpr (NG == 4) {
+        const uint4 x = *reinterpret_cast<const uint4 *>(p);
+        w[0] = x.x; w[1] = x.y; w[2] = x.z; w[3] = x.w;
+    } else if constexpr (NG == 2) {
+        const uint2 x = *reinterpret_cast<const uint2 *>(p);
+        w[0] = x.x; w[1] = x.y;
+    } else {
+        w[0] = p[0];
+    }
+}
+
+__device__ __forceinline__ float lo_half(uint32_t w) { return __low2float(*reinterpret_cast<const __half2 *>(&w)); }
+__device__ __forceinline__ float hi_half(uint32_t w) { return __high2float(*reinterpret_cast<const __half2 *>(&w)); }
+
+// Token ownership inside a 64-token tile.  The tile is two blocks of 32 tokens (kk), a block four octets (q);
+// lane group g owns token 32kk + 8q + ((g + q) & 7) of every octet.  The skew keeps both ldmatrix patterns
+// (8 score rows of one octet, 4 tokens of one owner for the values) at two rows per shared-memory bank group.
+__device__ __forceinline__ int owned_token(int kk, int q, int gg) { return 32 * kk + 8 * q + ((gg + q) & 7); }
 
 template <int G, int R>
 __global__ void __launch_bounds__(kThreads, 3) partition_gqa_kernel(MmaArgs a)
@@ -143,45 +186,45 @@ __global__ void __launch_bounds__(kThreads, 3) partition_gqa_kernel(MmaArgs a)
     }
     __syncthreads();
 
-    // B operand of the score MMAs, 8 k-steps of 16 channels.  Lane t = (word w1 = t >> 1, half u = t & 1) of a
-    // 32-channel word pair unpacks four registers from its word: fields {0,1,2,3} (u = 0) or {5,6,7,4} (u = 1),
-    // each with the field eight places up in the register's high half.  k-step 2p+s of pair p uses registers
-    // 2s (k = 2t, 2t+1) and 2s+1 (k = 2t+8, 2t+9).  Column n = g is query head g.
-    const int w1 = t >> 1, u = t & 1;
-    uint32_t bK[8][2];
+    // B operands of the score MMAs.  ldmatrix hands lane t words t and 4+t of a token row; all sixteen fields of a
+    // word are used, so k-step sx of channel half hf covers, in lane t, fields 2sx and 2sx+1 (+8) of word 4hf+t.
+    // The words of lanes t = 0,1 and t = 2,3 lie in different 32-channel blocks, so column n = (head n>>1,
+    // block parity n&1) carries the query only on the k rows of its own block: the two columns of a head hold the
+    // partial sums of the two blocks apart, and the lane that owns columns 2t, 2t+1 owns head t.
+    uint32_t bK[2][4][2];
+    {
+        const int hdn = g >> 1, par = g & 1;
 #pragma unroll
-    for (int p = 0; p < 4; ++p)
+        for (int hf = 0; hf < 2; ++hf)
 #pragma unroll
-        for (int sx = 0; sx < 2; ++sx)
+            for (int sx = 0; sx < 4; ++sx)
 #pragma unroll
-            for (int j = 0; j < 2; ++j) {
-                const int reg = 2 * sx + j;
-                const int fld = u ? (((reg + 1) & 3) + 4) : reg;
-                const int ch = 32 * p + 16 * w1 + fld;
-                const float wi = field_weight_inv(fld);
-                const float lo = g < kHeadSlots ? qs[g * kHeadDim + ch] * wi : 0.f;
-                const float hi = g < kHeadSlots ? qs[g * kHeadDim + ch + 8] * wi : 0.f;
-                bK[2 * p + sx][j] = pack_half2(lo, hi);
-            }
+                for (int j = 0; j < 2; ++j) {
+                    const int fld = 2 * sx + j;
+                    const int ch = 16 * (4 * hf + t) + fld;
+                    const float wi = field_weight_inv(fld);
+                    const bool on = (par == (t >> 1));
+                    const float lo = on ? qs[hdn * kHeadDim + ch] * wi : 0.f;
+                    const float hi = on ? qs[hdn * kHeadDim + ch + 8] * wi : 0.f;
+                    bK[hf][sx][j] = pack_half2(lo, hi);
+                }
+    }
     // B operand of the {h, z} MMA: k = 2t <-> h of group t, k = 2t+1 <-> z of group t; fp16 hi parts in k < 8,
-    // lo parts in k >= 8 (the A operand repeats the same words there).
+    // lo parts in k >= 8 (the A operand repeats the same words there).  Only the even column of a head is used.
     uint32_t bZ[2] = {0u, 0u};
-    if (g < kHeadSlots && t < NG) {
-        const float c0 = cst[g * 4 + t], c1 = sqs[g * 4 + t];
+    if ((g & 1) == 0 && t < NG) {
+        const float c0 = cst[(g >> 1) * 4 + t], c1 = sqs[(g >> 1) * 4 + t];
         const float c0h = __half2float(__float2half_rn(c0)), c1h = __half2float(__float2half_rn(c1));
         bZ[0] = pack_half2(c0h, c1h);
         bZ[1] = pack_half2(c0 - c0h, c1 - c1h);
     }
-    // this lane's two score columns are heads 2t and 2t+1
-    const float cs0 = (2 * t < kHeadSlots) ? csc[2 * t] : 0.f;
-    const float cs1 = (2 * t + 1 < kHeadSlots) ? csc[2 * t + 1] : 0.f;
+    const float cs = csc[t];                                     // this lane's score columns belong to head t
 
     // ---- per-warp shared memory
     uint8_t *stage_base = warp_base;
-    float *Pt = reinterpret_cast<float *>(warp_base + C::kStages * C::kStageBytes);                 // [4][68]
-    float *Hf = reinterpret_cast<float *>(warp_base + C::kStages * C::kStageBytes + C::kPBytes);    // [64][NG]
-    float *Os = reinterpret_cast<float *>(warp_base + C::kStages * C::kStageBytes + C::kPBytes + C::kHBytes);   // [4][128]
-    float *Zs = Os + kHeadSlots * kHeadDim;                                                         // [4][4]
+    uint2 *Xs = reinterpret_cast<uint2 *>(warp_base + C::kStages * C::kStageBytes);                  // [NG][2][32]
+    float *Os = reinterpret_cast<float *>(warp_base + C::kStages * C::kStageBytes + C::kXBytes);     // [4][128]
+    float *Zs = Os + kHeadSlots * kHeadDim;                                                          // [4][4]
     uint64_t *bars = reinterpret_cast<uint64_t *>(reinterpret_cast<uint8_t *>(Zs) + C::kZBytes);
     const uint32_t bar0 = smem_u32(bars);
     if (lane == 0) {
@@ -217,26 +260,39 @@ __global__ void __launch_bounds__(kThreads, 3) partition_gqa_kernel(MmaArgs a)
     if (lane == 0)
         for (int i = 0; i < C::kStages && i < n_my; ++i) issue(i);
 
-    // ---- running state
-    // softmax references of heads 2t, 2t+1 (log2 domain); lanes whose columns are no head never ask for a move
-    float m_ref0 = t < kHeadSlots / 2 ? -CUDART_INF_F : 0.f, m_ref1 = m_ref0;
-    float l0 = 0.f, l1 = 0.f;                                  // partial sums of p over this lane's token rows
-    float zacc[4] = {0.f, 0.f, 0.f, 0.f};                      // sum_t p z: rows = group g, columns = heads 2t, 2t+1
+    // ---- running state (this lane: head t, the eight tokens per tile that lane group g owns)
+    float m_ref = -CUDART_INF_F;                               // softmax reference of head t (log2 domain)
+    float l_sum = 0.f;                                         // partial sum of p over this lane's tokens
+    float zp[NG];                                              // partial sums of p * z_v per group
+#pragma unroll
+    for (int gg = 0; gg < NG; ++gg) zp[gg] = 0.f;
     int acc[16][4];                                            // P.V: rows (head g&3, digit g>>2 [+2]), columns = channels
 #pragma unroll
     for (int i = 0; i < 16; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = 0;
     float h_bound = 6.103515625e-05f;                          // power of two above every value scale seen so far
+    uint32_t h_thr = 0x0400u;                                  // the same bound as an fp16 bit pattern (2^-14)
     bool acc_live = false, failed = false;
 
-    // lane constants of the unpack and of the digit gather
-    const uint32_t rot_amt = u ? 26u : 4u;                     // rotate left: x << 4, or x >> 6
-    const uint32_t mask_x = u ? 0x03000300u : 0x00C000C0u;     // register 3 comes from the unrotated word
+    // lane constants
     const int hd = g & 3, d0 = g >> 2;                         // this lane's P.V rows: head hd, digits d0 and d0 + 2
-    const uint32_t sel_dig = d0 ? 0x7351u : 0x6240u;           // bytes d0 of two words, then bytes d0+2 of the same
+    // ldmatrix row addresses (byte offsets inside a stage).  Scores: matrices {octet 2jj, octet 2jj+1} x {bytes 0-15,
+    // 16-31}, lane supplies row lane&7 of matrix lane>>3.  Values: lanes 0-15 rows 4t'+j = token j of owner t',
+    // lanes 16-31 the same for owners t'+4.
+    uint32_t offK[2];
+#pragma unroll
+    for (int jj = 0; jj < 2; ++jj) {
+        const int mi = lane >> 3, r = lane & 7, qq = 2 * jj + (mi & 1);
+        offK[jj] = (uint32_t)(owned_token(0, qq, r) * kRowBytes + 16 * (mi >> 1));
+    }
+    const uint32_t offV = (uint32_t)(owned_token(0, lane & 3, ((lane & 15) >> 2) + 4 * (lane >> 4)) * kRowBytes);
+    int own[4];                                                // owned token of octet q inside a 32-token block
+#pragma unroll
+    for (int q = 0; q < 4; ++q) own[q] = owned_token(0, q, g);
+    const uint2 *xrd = Xs + d0 * 32;                           // digit pairs (d0, d0+2) of the owners this lane reads
 
-    // Brings the integer sums into the fp32 sums in shared memory and rescales those by 2^(old ref - new ref).
+    // Brings the integer sums into the fp32 sums in shared memory; everything there is then multiplied by corr_hd.
     auto fold = [&](float corr_hd) {
         const float sa = h_bound * (d0 ? 1.52587890625e-05f : 5.9604644775390625e-08f);   // h_bound * 2^8 * 2^-32 * 256^d0
         const float sb = sa * 65536.0f;
@@ -280,190 +336,140 @@ __global__ void __launch_bounds__(kThreads, 3) partition_gqa_kernel(MmaArgs a)
             __syncwarp();
         }
 
-        // ---------------- scores: lane (g, t) ends with tokens 16mt+g, 16mt+g+8 x heads 2t, 2t+1
-        float sraw[4][4];
+        // ---------------- scores of head t for the eight owned tokens: sraw[2kk+jj][0/1] = octets 2jj, 2jj+1
+        const uint32_t kaddr = smem_u32(Kc);
+        float sraw[4][2];
 #pragma unroll
         for (int mt = 0; mt < 4; ++mt) {
-            const uint32_t *row0 = reinterpret_cast<const uint32_t *>(Kc + (16 * mt + g) * kRowBytes) + w1;
-            const uint32_t *row1 = row0 + 8 * (kRowBytes / 4);
-            float ak[NG][4];
+            const int kk = mt >> 1, jj = mt & 1;
+            uint32_t rw[4];
+            ldmatrix_x4(rw, kaddr + kk * 32 * kRowBytes + offK[jj]);
+            float ak[2][4];
 #pragma unroll
-            for (int gg = 0; gg < NG; ++gg)
+            for (int hf = 0; hf < 2; ++hf) {
+                uint32_t u0[8], u1[8];
+                unpack16(rw[2 * hf], u0);          // row g     (octet 2jj)
+                unpack16(rw[2 * hf + 1], u1);      // row g + 8 (octet 2jj+1)
+                ak[hf][0] = 0.f; ak[hf][1] = 0.f; ak[hf][2] = 0.f; ak[hf][3] = 0.f;
 #pragma unroll
-                for (int e = 0; e < 4; ++e) ak[gg][e] = 0.f;
-#pragma unroll
-            for (int p = 0; p < 4; ++p) {
-                constexpr uint32_t MAGIC = 0x54005400u, M4 = 0x00300030u, M6 = 0x00C000C0u, M8 = 0x03000300u;
-                const uint32_t xa = row0[2 * p], xb = row1[2 * p];
-                const uint32_t ra = __funnelshift_l(xa, xa, rot_amt), rb = __funnelshift_l(xb, xb, rot_amt);
-                const uint32_t a00 = and_or(ra, M4, MAGIC), a01 = and_or(ra, M6, MAGIC);
-                const uint32_t a02 = and_or(ra, M8, MAGIC), a03 = and_or(xa, mask_x, MAGIC);
-                const uint32_t a10 = and_or(rb, M4, MAGIC), a11 = and_or(rb, M6, MAGIC);
-                const uint32_t a12 = and_or(rb, M8, MAGIC), a13 = and_or(xb, mask_x, MAGIC);
-                mma16816(ak[(32 * p) / G], a00, a10, a01, a11, bK[2 * p][0], bK[2 * p][1]);
-                mma16816(ak[(32 * p) / G], a02, a12, a03, a13, bK[2 * p + 1][0], bK[2 * p + 1][1]);
+                for (int sx = 0; sx < 4; ++sx)
+                    mma16816(ak[hf], u0[2 * sx], u1[2 * sx], u0[2 * sx + 1], u1[2 * sx + 1], bK[hf][sx][0], bK[hf][sx][1]);
             }
             // {h, z} words of the two tokens: A operand of the constant/zero-point MMA, and h for the group sums
-            const uint32_t *m0 = Km + (16 * mt + g) * NG, *m1 = m0 + 8 * NG;
+            const uint32_t *m0 = Km + (32 * kk + own[2 * jj]) * NG, *m1 = Km + (32 * kk + own[2 * jj + 1]) * NG;
             uint32_t mw0[NG], mw1[NG];
-            if constexpr (NG == 4) {
-                const uint4 x0 = *reinterpret_cast<const uint4 *>(m0), x1 = *reinterpret_cast<const uint4 *>(m1);
-                mw0[0] = x0.x; mw0[1] = x0.y; mw0[2] = x0.z; mw0[3] = x0.w;
-                mw1[0] = x1.x; mw1[1] = x1.y; mw1[2] = x1.z; mw1[3] = x1.w;
-            } else if constexpr (NG == 2) {
-                const uint2 x0 = *reinterpret_cast<const uint2 *>(m0), x1 = *reinterpret_cast<const uint2 *>(m1);
-                mw0[0] = x0.x; mw0[1] = x0.y; mw1[0] = x1.x; mw1[1] = x1.y;
-            } else {
-                mw0[0] = m0[0]; mw1[0] = m1[0];
-            }
+            load_words<NG>(m0, mw0);
+            load_words<NG>(m1, mw1);
             const uint32_t za = t < NG ? m0[t < NG ? t : 0] : 0u;
             const uint32_t zb = t < NG ? m1[t < NG ? t : 0] : 0u;
             float az[4] = {0.f, 0.f, 0.f, 0.f};
             mma16816(az, za, zb, za, zb, bZ[0], bZ[1]);
+            float s0 = az[0], s1 = az[2];
 #pragma unroll
-            for (int gg = 0; gg < NG; ++gg) {
-                const float h0 = __low2float(*reinterpret_cast<const __half2 *>(&mw0[gg]));
-                const float h1 = __low2float(*reinterpret_cast<const __half2 *>(&mw1[gg]));
-                az[0] = fmaf(h0, ak[gg][0], az[0]);
-                az[1] = fmaf(h0, ak[gg][1], az[1]);
-                az[2] = fmaf(h1, ak[gg][2], az[2]);
-                az[3] = fmaf(h1, ak[gg][3], az[3]);
-            }
-            sraw[mt][0] = az[0]; sraw[mt][1] = az[1]; sraw[mt][2] = az[2]; sraw[mt][3] = az[3];
+            for (int hf = 0; hf < 2; ++hf)
+#pragma unroll
+                for (int par = 0; par < 2; ++par) {
+                    const int gg = (64 * hf + 32 * par) / G;
+                    s0 = fmaf(lo_half(mw0[gg]), ak[hf][par], s0);
+                    s1 = fmaf(lo_half(mw1[gg]), ak[hf][2 + par], s1);
+                }
+            sraw[mt][0] = s0;
+            sraw[mt][1] = s1;
         }
 
-        // ---------------- value scales of tokens lane, lane+32; does the reference or the bound have to move?
-        float hv[2][NG];
-        bool moved = false;
-#pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-            const int tau = lane + 32 * hf;
-#pragma unroll
-            for (int gg = 0; gg < NG; ++gg) {
-                hv[hf][gg] = __low2float(*reinterpret_cast<const __half2 *>(Vm + tau * NG + gg));
-                moved |= (hv[hf][gg] >= h_bound);
-            }
-        }
-        float arg[4][4];
-#pragma unroll
-        for (int mt = 0; mt < 4; ++mt) {
-            const bool v0 = (16 * mt + g) < n_valid, v1 = (16 * mt + g + 8) < n_valid;
-            arg[mt][0] = v0 ? fmaf(sraw[mt][0], cs0, -m_ref0) : -CUDART_INF_F;
-            arg[mt][1] = v0 ? fmaf(sraw[mt][1], cs1, -m_ref1) : -CUDART_INF_F;
-            arg[mt][2] = v1 ? fmaf(sraw[mt][2], cs0, -m_ref0) : -CUDART_INF_F;
-            arg[mt][3] = v1 ? fmaf(sraw[mt][3], cs1, -m_ref1) : -CUDART_INF_F;
-            moved |= (fmaxf(fmaxf(arg[mt][0], arg[mt][1]), fmaxf(arg[mt][2], arg[mt][3])) > kRefSlack);
-        }
-        if (__any_sync(0xffffffffu, moved)) {
-            // Raise the references to the running maxima (and the bound on h), fold what was accumulated so far.
-            float tm0 = -CUDART_INF_F, tm1 = -CUDART_INF_F;
-#pragma unroll
-            for (int mt = 0; mt < 4; ++mt) {
-                const bool v0 = (16 * mt + g) < n_valid, v1 = (16 * mt + g + 8) < n_valid;
-                if (v0) { tm0 = fmaxf(tm0, sraw[mt][0] * cs0); tm1 = fmaxf(tm1, sraw[mt][1] * cs1); }
-                if (v1) { tm0 = fmaxf(tm0, sraw[mt][2] * cs0); tm1 = fmaxf(tm1, sraw[mt][3] * cs1); }
-            }
-#pragma unroll
-            for (int msk = 4; msk < 32; msk <<= 1) {
-                tm0 = fmaxf(tm0, __shfl_xor_sync(0xffffffffu, tm0, msk));
-                tm1 = fmaxf(tm1, __shfl_xor_sync(0xffffffffu, tm1, msk));
-            }
-            const float n0 = fmaxf(m_ref0, tm0), n1 = fmaxf(m_ref1, tm1);
-            const float c0 = ex2_approx(m_ref0 - n0), c1 = ex2_approx(m_ref1 - n1);   // 0 on the first tile
-            m_ref0 = n0; m_ref1 = n1;
-            l0 *= c0; l1 *= c1;
-            zacc[0] *= c0; zacc[1] *= c1; zacc[2] *= c0; zacc[3] *= c1;
-            // the correction of head hd lives in the lanes with t = hd >> 1
-            const float ca = __shfl_sync(0xffffffffu, c0, hd >> 1), cb = __shfl_sync(0xffffffffu, c1, hd >> 1);
-            const float corr_hd = (hd & 1) ? cb : ca;
-            if (acc_live) fold(corr_hd);
-            float hm = 0.f;
-#pragma unroll
-            for (int gg = 0; gg < NG; ++gg) hm = fmaxf(hm, fmaxf(hv[0][gg], hv[1][gg]));
-            hm = warp_max(hm);
-            if (hm >= h_bound) h_bound = __int_as_float(((__float_as_int(hm) >> 23) + 1) << 23);
-#pragma unroll
-            for (int mt = 0; mt < 4; ++mt) {
-                const bool v0 = (16 * mt + g) < n_valid, v1 = (16 * mt + g + 8) < n_valid;
-                arg[mt][0] = v0 ? fmaf(sraw[mt][0], cs0, -m_ref0) : -CUDART_INF_F;
-                arg[mt][1] = v0 ? fmaf(sraw[mt][1], cs1, -m_ref1) : -CUDART_INF_F;
-                arg[mt][2] = v1 ? fmaf(sraw[mt][2], cs0, -m_ref0) : -CUDART_INF_F;
-                arg[mt][3] = v1 ? fmaf(sraw[mt][3], cs1, -m_ref1) : -CUDART_INF_F;
-            }
-        }
-        // probabilities (at most 2^8) -> P tile [head][token]; value scales on the fixed-point grid -> Hf
-        if (t < kHeadSlots / 2) {
-#pragma unroll
-            for (int mt = 0; mt < 4; ++mt) {
-                const float p0 = ex2_approx(arg[mt][0]), p1 = ex2_approx(arg[mt][1]);
-                const float p2 = ex2_approx(arg[mt][2]), p3 = ex2_approx(arg[mt][3]);
-                l0 += p0 + p2;
-                l1 += p1 + p3;
-                float *pr = Pt + (2 * t) * C::kPStride + 16 * mt + g;
-                pr[0] = p0; pr[C::kPStride] = p1; pr[8] = p2; pr[C::kPStride + 8] = p3;
-            }
-        }
+        // ---------------- does the softmax reference, or the bound on the value scales, have to move?
+        uint32_t hmax_bits;
         {
-            const float hscale = 16777216.0f / h_bound;      // 2^32 / (h_bound * 2^8)
+            uint32_t wa[NG], wb[NG];
+            load_words<NG>(Vm + lane * NG, wa);
+            load_words<NG>(Vm + (lane + 32) * NG, wb);
+            uint32_t mx = __vmaxu2(wa[0], wb[0]);
 #pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-                const int tau = lane + 32 * hf;
-#pragma unroll
-                for (int gg = 0; gg < NG; ++gg) Hf[tau * NG + gg] = hv[hf][gg] * hscale;   // 0 for rows past the end
-            }
+            for (int gg = 1; gg < NG; ++gg) mx = __vmaxu2(mx, __vmaxu2(wa[gg], wb[gg]));
+            hmax_bits = mx & 0xFFFFu;                          // scales are non-negative: fp16 order = integer order
         }
-        __syncwarp();
-
-        // ---------------- sum_t p_t z_{t,g}: rows = groups, columns = heads, k = 16 tokens
+        bool moved = hmax_bits >= h_thr;
+        float arg[4][2];
+        float amax = -CUDART_INF_F;
 #pragma unroll
-        for (int kb = 0; kb < 4; ++kb) {
-            const int ta = 16 * kb + 2 * t;
-            uint32_t a0 = 0u, a2 = 0u, b0 = 0u, b1 = 0u;
-            if (g < NG) {
-                a0 = prmt(Vm[ta * NG + g], Vm[(ta + 1) * NG + g], 0x7632u);
-                a2 = prmt(Vm[(ta + 8) * NG + g], Vm[(ta + 9) * NG + g], 0x7632u);
+        for (int mt = 0; mt < 4; ++mt)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const bool valid = (32 * (mt >> 1) + own[2 * (mt & 1) + e]) < n_valid;
+                arg[mt][e] = valid ? fmaf(sraw[mt][e], cs, -m_ref) : -CUDART_INF_F;
+                amax = fmaxf(amax, arg[mt][e]);
             }
-            if (g < kHeadSlots) {
-                const float2 pa = *reinterpret_cast<const float2 *>(Pt + g * C::kPStride + ta);
-                const float2 pb = *reinterpret_cast<const float2 *>(Pt + g * C::kPStride + ta + 8);
-                b0 = pack_half2(pa.x, pa.y);
-                b1 = pack_half2(pb.x, pb.y);
+        moved |= amax > kRefSlack;
+        if (__any_sync(0xffffffffu, moved)) {
+            // Raise the reference of every head to its running maximum (and the bound on h); fold what was accumulated.
+            float tm = -CUDART_INF_F;
+#pragma unroll
+            for (int mt = 0; mt < 4; ++mt)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const bool valid = (32 * (mt >> 1) + own[2 * (mt & 1) + e]) < n_valid;
+                    if (valid) tm = fmaxf(tm, sraw[mt][e] * cs);
+                }
+#pragma unroll
+            for (int msk = 4; msk < 32; msk <<= 1) tm = fmaxf(tm, __shfl_xor_sync(0xffffffffu, tm, msk));
+            const float m_new = fmaxf(m_ref, tm);
+            const float corr = ex2_approx(m_ref - m_new);              // 0 on the first tile
+            m_ref = m_new;
+            l_sum *= corr;
+#pragma unroll
+            for (int gg = 0; gg < NG; ++gg) zp[gg] *= corr;
+            const float corr_hd = __shfl_sync(0xffffffffu, corr, hd);  // lane hd = (g 0, t hd) holds head hd
+            if (acc_live) fold(corr_hd);
+            const uint32_t hm = __reduce_max_sync(0xffffffffu, hmax_bits);
+            if (hm >= h_thr) {
+                const float hmf = __half2float(__ushort_as_half((unsigned short)hm));
+                h_bound = __int_as_float(((__float_as_int(hmf) >> 23) + 1) << 23);    // next power of two above
+                h_thr = h_bound > 32768.0f ? 0x7C00u : (uint32_t)__half_as_ushort(__float2half_rn(h_bound));
             }
-            mma16816(zacc, a0, 0u, a2, 0u, b0, b1);
+#pragma unroll
+            for (int mt = 0; mt < 4; ++mt)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const bool valid = (32 * (mt >> 1) + own[2 * (mt & 1) + e]) < n_valid;
+                    arg[mt][e] = valid ? fmaf(sraw[mt][e], cs, -m_ref) : -CUDART_INF_F;
+                }
         }
+        const float hscale = 16777216.0f / h_bound;      // 2^32 / (h_bound * 2^8)
 
-        // ---------------- P.V: A rows (head hd, digits d0 / d0+2), k = 32 tokens, columns = 8 channels of one group
-        const uint32_t vaddr = smem_u32(Vc) + lane * kRowBytes;
+        // ---------------- per 32-token block: probabilities, p*h on the fixed-point grid, digits -> A fragments, MMAs
+        const uint32_t vaddr = smem_u32(Vc) + offV;
 #pragma unroll
         for (int kk = 0; kk < 2; ++kk) {
-            uint32_t Ag[NG][4];
+            uint32_t uu[4][NG];
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                const int tk = 32 * kk + 16 * half + 4 * t;
-                const float4 p4 = *reinterpret_cast<const float4 *>(Pt + hd * C::kPStride + tk);
-                const float pv[4] = {p4.x, p4.y, p4.z, p4.w};
-                uint32_t uu[4][NG];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    float hrow[NG];
-                    if constexpr (NG == 4) {
-                        const float4 h4 = *reinterpret_cast<const float4 *>(Hf + (tk + j) * 4);
-                        hrow[0] = h4.x; hrow[1] = h4.y; hrow[2] = h4.z; hrow[3] = h4.w;
-                    } else if constexpr (NG == 2) {
-                        const float2 h2 = *reinterpret_cast<const float2 *>(Hf + (tk + j) * 2);
-                        hrow[0] = h2.x; hrow[1] = h2.y;
-                    } else {
-                        hrow[0] = Hf[tk + j];
-                    }
-#pragma unroll
-                    for (int gg = 0; gg < NG; ++gg) uu[j][gg] = to_fixed_u32(pv[j] * hrow[gg]);
-                }
+            for (int q = 0; q < 4; ++q) {
+                const float p = ex2_approx(arg[2 * kk + (q >> 1)][q & 1]);      // at most 2^8; 0 past the end
+                l_sum += p;
+                uint32_t vw[NG];
+                load_words<NG>(Vm + (32 * kk + own[q]) * NG, vw);
+                const float ps = p * hscale;
 #pragma unroll
                 for (int gg = 0; gg < NG; ++gg) {
-                    const uint32_t t01 = prmt(uu[0][gg], uu[1][gg], sel_dig), t23 = prmt(uu[2][gg], uu[3][gg], sel_dig);
-                    Ag[gg][2 * half] = prmt(t01, t23, 0x5410u);
-                    Ag[gg][2 * half + 1] = prmt(t01, t23, 0x7632u);
+                    uu[q][gg] = to_fixed_u32(ps * lo_half(vw[gg]));
+                    zp[gg] = fmaf(p, hi_half(vw[gg]), zp[gg]);
                 }
+            }
+            // byte transpose: digit d of the four owned tokens in one register; pairs (0,2) and (1,3) are what the
+            // two reader lanes of a head want
+#pragma unroll
+            for (int gg = 0; gg < NG; ++gg) {
+                const uint32_t t01 = prmt(uu[0][gg], uu[1][gg], 0x5140u), t23 = prmt(uu[2][gg], uu[3][gg], 0x5140u);
+                const uint32_t h01 = prmt(uu[0][gg], uu[1][gg], 0x7362u), h23 = prmt(uu[2][gg], uu[3][gg], 0x7362u);
+                Xs[(gg * 2 + 0) * 32 + lane] = make_uint2(prmt(t01, t23, 0x5410u), prmt(h01, h23, 0x5410u));   // digits 0, 2
+                Xs[(gg * 2 + 1) * 32 + lane] = make_uint2(prmt(t01, t23, 0x7632u), prmt(h01, h23, 0x7632u));   // digits 1, 3
+            }
+            __syncwarp();
+            // A fragments: k = 4t+j <-> token j of owner t (slot 4t + hd), k = 16+4t+j <-> owner t+4
+            uint32_t Ag[NG][4];
+#pragma unroll
+            for (int gg = 0; gg < NG; ++gg) {
+                const uint2 xa = xrd[gg * 64 + 4 * t + hd], xb = xrd[gg * 64 + 4 * (t + 4) + hd];
+                Ag[gg][0] = xa.x; Ag[gg][1] = xa.y; Ag[gg][2] = xb.x; Ag[gg][3] = xb.y;
             }
 #pragma unroll
             for (int hh = 0; hh < 2; ++hh) {
@@ -480,9 +486,9 @@ __global__ void __launch_bounds__(kThreads, 3) partition_gqa_kernel(MmaArgs a)
                     }
                 }
             }
+            __syncwarp();   // the exchange buffer is rewritten by the next block
         }
         acc_live = true;
-        __syncwarp();   // every lane is done with this stage, the P tile and Hf
         if (lane == 0 && i + C::kStages < n_my) issue(i + C::kStages);
     }
 
@@ -496,16 +502,18 @@ __global__ void __launch_bounds__(kThreads, 3) partition_gqa_kernel(MmaArgs a)
 
     // ---- per-warp result
     if (acc_live) fold(1.0f);
-    if (g < NG && t < kHeadSlots / 2) {
-        Zs[(2 * t) * 4 + g] = zacc[0];
-        Zs[(2 * t + 1) * 4 + g] = zacc[1];
-    }
 #pragma unroll
     for (int msk = 4; msk < 32; msk <<= 1) {
-        l0 += __shfl_xor_sync(0xffffffffu, l0, msk);
-        l1 += __shfl_xor_sync(0xffffffffu, l1, msk);
+        l_sum += __shfl_xor_sync(0xffffffffu, l_sum, msk);
+#pragma unroll
+        for (int gg = 0; gg < NG; ++gg) zp[gg] += __shfl_xor_sync(0xffffffffu, zp[gg], msk);
+    }
+    if (g == 0) {
+#pragma unroll
+        for (int gg = 0; gg < NG; ++gg) Zs[t * 4 + gg] = zp[gg];
     }
     __syncwarp();
+    const bool dead = failed || !acc_live;
     float *Ow = reinterpret_cast<float *>(stage_base);                       // [R][132]: o', m, l
 #pragma unroll
     for (int r = 0; r < R; ++r) {
@@ -515,18 +523,12 @@ __global__ void __launch_bounds__(kThreads, 3) partition_gqa_kernel(MmaArgs a)
             const int j = d & 3;                                             // channel d carries the weight 4^j
             const float winv = j == 0 ? 1.0f : (j == 1 ? 0.25f : (j == 2 ? 0.0625f : 0.015625f));
             const float o = Os[r * kHeadDim + d] * winv + Zs[r * 4 + d / G];
-            Ow[r * kPartialStride + d] = (failed || !acc_live) ? 0.f : o;
+            Ow[r * kPartialStride + d] = dead ? 0.f : o;
         }
     }
-    if (g == 0 && t < kHeadSlots / 2) {
-        if (2 * t < R) {
-            Ow[(2 * t) * kPartialStride + kHeadDim] = (failed || !acc_live) ? -CUDART_INF_F : m_ref0;
-            Ow[(2 * t) * kPartialStride + kHeadDim + 1] = (failed || !acc_live) ? 0.f : l0;
-        }
-        if (2 * t + 1 < R) {
-            Ow[(2 * t + 1) * kPartialStride + kHeadDim] = (failed || !acc_live) ? -CUDART_INF_F : m_ref1;
-            Ow[(2 * t + 1) * kPartialStride + kHeadDim + 1] = (failed || !acc_live) ? 0.f : l1;
-        }
+    if (g == 0 && t < R) {
+        Ow[t * kPartialStride + kHeadDim] = dead ? -CUDART_INF_F : m_ref;
+        Ow[t * kPartialStride + kHeadDim + 1] = dead ? 0.f : l_sum;
     }
     __syncthreads();
 
