@@ -6,9 +6,9 @@
 // KV head.  It never forms h*code+z per element for the scores: with q' the permuted query,
 //   q'.K~_t = sum_g h_{t,g} (sum_{j in g} q'_j c_{t,j}) + sum_g z_{t,g} (sum_{j in g} q'_j)
 // so the zero points cost one multiply-add per group.  Scores live in the log2 domain
-// (sm_scale*log2(e) folded into q').  The split that owns the tail also walks the fp16 ring.
-// Partials (o'[128], m, l) go to the caller's workspace; merge_kernel combines them, divides
-// by the softmax denominator, undoes the value permutation and writes fp16.
+// (sm_scale*log2(e) folded into q').  Partials (o'[128], m, l) of the quantized prefix go to the
+// caller's workspace; merge_kernel walks the fp16 window itself, combines everything, divides by
+// the softmax denominator, undoes the value permutation and writes fp16.
 #include <math_constants.h>
 
 #include "skvq_internal.cuh"
@@ -50,13 +50,12 @@ __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
     const Shape &s = a.s;
     const int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int rep = s.rep, G = s.G, ng = s.ng, W = s.W;
+    const int rep = s.rep, G = s.G, ng = s.ng;
     const int L = a.c.lengths[b];
-    const int Lq = max(L - W, 0);
-    const bool owns_window = (split == a.plan.n_splits);      // the last part is the fp16 window
-    const int q_begin = owns_window ? Lq : min(split * a.plan.split_len, Lq);
-    const int q_end = owns_window ? Lq : min(q_begin + a.plan.split_len, Lq);
-    const int n_parts = a.plan.n_splits + 1;
+    const int Lq = max(L - s.W, 0);
+    const int q_begin = min(split * a.plan.split_len, Lq);
+    const int q_end = min(q_begin + a.plan.split_len, Lq);
+    const int n_parts = a.plan.n_splits;
 
     __shared__ float sq[kMaxRep][kHeadDim];        // permuted query, times sm_scale*log2(e)
     __shared__ float sqsum[kMaxRep][4];            // per-group sums of the above
@@ -84,19 +83,13 @@ __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
     const uint8_t *v_codes = a.c.v_codes + bh * (size_t)s.cap * VROW;
     const __half2 *k_meta = a.c.k_meta + bh * (size_t)s.cap * ng;
     const __half2 *v_meta = a.c.v_meta + bh * (size_t)s.cap * ng;
-    const __half *k_win = a.c.k_win + bh * (size_t)W * kHeadDim;
-    const __half *v_win = a.c.v_win + bh * (size_t)W * kHeadDim;
 
     float m_run[kMaxRep], l_thread[kMaxRep], acc[kMaxRep];
 #pragma unroll
     for (int r = 0; r < kMaxRep; ++r) { m_run[r] = -CUDART_INF_F; l_thread[r] = 0.f; acc[r] = 0.f; }
 
-    // Two passes over "segments": the quantized range of this split, then (for the owner) the window.
-    for (int seg = 0; seg < 2; ++seg) {
-        const bool quant = (seg == 0);
-        if (!quant && !owns_window) break;
-        const int t_begin = quant ? q_begin : Lq;
-        const int t_end = quant ? q_end : L;
+    {
+        const int t_begin = q_begin, t_end = q_end;
         for (int tile0 = t_begin; tile0 < t_end; tile0 += kTile) {
             const int t = tile0 + tid;
             const bool valid = t < t_end;
@@ -106,7 +99,7 @@ __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
             if (valid) {
 #pragma unroll
                 for (int r = 0; r < kMaxRep; ++r) sc[r] = 0.f;
-                if (quant) {
+                {
                     const uint32_t *row = reinterpret_cast<const uint32_t *>(k_codes + (size_t)t * KROW);
                     constexpr int PER_WORD = 32 / KBITS;
                     for (int g = 0; g < ng; ++g) {
@@ -128,14 +121,6 @@ __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
 #pragma unroll
                         for (int r = 0; r < kMaxRep; ++r)
                             if (r < rep) sc[r] += hz.x * part[r] + hz.y * sqsum[r][g];
-                    }
-                } else {
-                    const __half2 *row = reinterpret_cast<const __half2 *>(k_win + (size_t)(t % W) * kHeadDim);
-                    for (int j2 = 0; j2 < kHeadDim / 2; ++j2) {
-                        const float2 kv = __half22float2(row[j2]);
-#pragma unroll
-                        for (int r = 0; r < kMaxRep; ++r)
-                            if (r < rep) sc[r] = fmaf(sq[r][2 * j2], kv.x, fmaf(sq[r][2 * j2 + 1], kv.y, sc[r]));
                     }
                 }
             }
@@ -168,7 +153,7 @@ __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
             __syncthreads();
             // P.V: this thread owns (reordered) channel tid.
             const int n_tok = min(kTile, t_end - tile0);
-            if (quant) {
+            {
                 constexpr int PER_WORD = 32 / VBITS;
                 const int g = tid / G;
                 const int w = tid / PER_WORD, sh = (tid % PER_WORD) * VBITS;
@@ -177,13 +162,6 @@ __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
                     const uint32_t word = __ldg(reinterpret_cast<const uint32_t *>(v_codes + row * VROW) + w);
                     const float2 hz = __half22float2(v_meta[row * ng + g]);
                     const float val = fmaf(hz.x, (float)((word >> sh) & VQMAX), hz.y);
-#pragma unroll
-                    for (int r = 0; r < kMaxRep; ++r)
-                        if (r < rep) acc[r] = fmaf(sp[r][tt], val, acc[r]);
-                }
-            } else {
-                for (int tt = 0; tt < n_tok; ++tt) {
-                    const float val = __half2float(v_win[(size_t)((tile0 + tt) % W) * kHeadDim + tid]);
 #pragma unroll
                     for (int r = 0; r < kMaxRep; ++r)
                         if (r < rep) acc[r] = fmaf(sp[r][tt], val, acc[r]);
@@ -217,31 +195,129 @@ __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
     }
 }
 
-// Combine the split partials of one (sequence, query head): thread d owns reordered channel d.
+// One CTA per (query head, sequence): walks the fp16 window (at most W tokens: thread = token for the scores,
+// thread = reordered channel for P.V), then combines that with the split partials of the quantized prefix.
 __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
 {
-    const int hq = blockIdx.x, b = blockIdx.y, d = threadIdx.x;
+    const int hq = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const Shape &s = a.s;
     const int hk = hq / s.rep;
-    const int S = a.plan.n_splits + 1;
+    const int W = s.W;
+    const int L = a.c.lengths[b];
+    const int Lq = max(L - W, 0);
+    __shared__ float sq[kHeadDim];
+    __shared__ float sp[kThreads];
+    __shared__ float sred[kThreads / 32];
+    const size_t bh = (size_t)b * s.Hkv + hk;
+    sq[tid] = __half2float(a.q[((size_t)b * s.Hq + hq) * kHeadDim + (a.c.reorder_k[(size_t)hk * kHeadDim + tid] & (kHeadDim - 1))]) *
+              a.scale_log2;
+    __syncthreads();
+    const __half *k_win = a.c.k_win + bh * (size_t)W * kHeadDim;
+    const __half *v_win = a.c.v_win + bh * (size_t)W * kHeadDim;
+    // P.V layout: warp w takes tokens w, w+4, ... of a tile, lane l channels 4l..4l+3 (one 8-byte load per row)
+    __shared__ float sacc[kThreads / 32][kHeadDim];
+    float m_run = -CUDART_INF_F, l_thread = 0.f;
+    float a4[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int tile0 = Lq; tile0 < L; tile0 += kThreads) {
+        const int t = tile0 + tid;
+        const bool valid = t < L;
+        float sc = valid ? 0.f : -CUDART_INF_F;
+        if (valid) {
+            const uint4 *row = reinterpret_cast<const uint4 *>(k_win + (size_t)(t % W) * kHeadDim);
+            uint4 u[kHeadDim / 8];
+#pragma unroll
+            for (int j8 = 0; j8 < kHeadDim / 8; ++j8) u[j8] = __ldg(row + j8);      // all 16 loads in flight
+#pragma unroll
+            for (int j8 = 0; j8 < kHeadDim / 8; ++j8) {
+                const __half2 *h2 = reinterpret_cast<const __half2 *>(&u[j8]);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float2 kv = __half22float2(h2[i]);
+                    sc = fmaf(sq[8 * j8 + 2 * i], kv.x, fmaf(sq[8 * j8 + 2 * i + 1], kv.y, sc));
+                }
+            }
+        }
+        const float wm = warp_max(sc);
+        if (lane == 0) sred[warp] = wm;
+        __syncthreads();
+        float tm = sred[0];
+#pragma unroll
+        for (int w = 1; w < kThreads / 32; ++w) tm = fmaxf(tm, sred[w]);
+        const float m_new = fmaxf(m_run, tm);               // finite: the tile has a valid token
+        const float corr = exp2f(m_run - m_new);            // exp2(-inf) = 0 on the first tile
+        const float p = valid ? exp2f(sc - m_new) : 0.f;
+        sp[tid] = p;
+        l_thread = l_thread * corr + p;
+        m_run = m_new;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) a4[i] *= corr;
+        __syncthreads();
+        const int n_tok = min(kThreads, L - tile0);
+#pragma unroll 8
+        for (int tt = warp; tt < n_tok; tt += kThreads / 32) {
+            const uint2 u = __ldg(reinterpret_cast<const uint2 *>(v_win + (size_t)((tile0 + tt) % W) * kHeadDim) + lane);
+            const float2 v01 = __half22float2(*reinterpret_cast<const __half2 *>(&u.x));
+            const float2 v23 = __half22float2(*reinterpret_cast<const __half2 *>(&u.y));
+            const float pt = sp[tt];
+            a4[0] = fmaf(pt, v01.x, a4[0]); a4[1] = fmaf(pt, v01.y, a4[1]);
+            a4[2] = fmaf(pt, v23.x, a4[2]); a4[3] = fmaf(pt, v23.y, a4[3]);
+        }
+        __syncthreads();   // sp and sred are rewritten by the next tile
+    }
+    *reinterpret_cast<float4 *>(&sacc[warp][4 * lane]) = make_float4(a4[0], a4[1], a4[2], a4[3]);
+    const float lw = warp_sum(l_thread);
+    if (lane == 0) sred[warp] = lw;
+    __syncthreads();
+    float l_win = 0.f, acc = 0.f;
+#pragma unroll
+    for (int w = 0; w < kThreads / 32; ++w) { l_win += sred[w]; acc += sacc[w][tid]; }
+
+    // log-sum-exp merge: the window and the S split partials; thread d owns reordered channel d
+    const int S = a.plan.n_splits;
     const float *part = a.ws + ((size_t)b * s.Hq + hq) * S * kPartialStride;
-    float M = -CUDART_INF_F;
+    float M = m_run;
     for (int i = 0; i < S; ++i) M = fmaxf(M, part[(size_t)i * kPartialStride + kHeadDim]);
     float o = 0.f, l = 0.f;
     if (M > -CUDART_INF_F) {
+        const float ww = exp2f(m_run - M);
+        o = acc * ww;
+        l = l_win * ww;
         for (int i = 0; i < S; ++i) {
             const float *p = part + (size_t)i * kPartialStride;
             const float w = exp2f(p[kHeadDim] - M);
-            o = fmaf(p[d], w, o);
+            o = fmaf(p[tid], w, o);
             l = fmaf(p[kHeadDim + 1], w, l);
         }
     }
     const float res = l > 0.f ? o / l : 0.f;
-    const int dst = a.c.reorder_v[(size_t)hk * kHeadDim + d] & (kHeadDim - 1);
+    const int dst = a.c.reorder_v[(size_t)hk * kHeadDim + tid] & (kHeadDim - 1);
     a.out[((size_t)b * s.Hq + hq) * kHeadDim + dst] = __float2half_rn(res);
 }
 
 }  // namespace
+
+// Resident CTAs per SM of the partition kernel that serves this shape (sets how many CTAs make one wave).
+static int partition_ctas_per_sm(const Shape &s)
+{
+    if (s.k_bits == 2 && s.v_bits == 2 && s.rep == 1 && s.G >= 64) return 4;   // integer kernel, 121 registers
+    if (s.k_bits == 2 && s.v_bits == 2 && s.rep <= 4) return 3;                // grouped-query kernel, 168 registers
+    return 8;                                                                  // scalar kernel
+}
+
+static int sm_count()
+{
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+            n = v;
+        else
+            n = 148;
+        (void)cudaGetLastError();
+    }
+    return n;
+}
 
 SplitPlan plan_splits(const Shape &s, int max_len, int requested_splits)
 {
@@ -252,13 +328,25 @@ SplitPlan plan_splits(const Shape &s, int max_len, int requested_splits)
         split_len = (lq + requested_splits - 1) / requested_splits;
         split_len = (split_len + SKVQ_TOKEN_ALIGN - 1) / SKVQ_TOKEN_ALIGN * SKVQ_TOKEN_ALIGN;
     } else {
-        // About 8 CTAs per resident slot (148 SMs x 3 CTAs), between 1024 and 8192 tokens per split,
-        // in multiples of 256 tokens (4 warps x 64-token tiles).
-        const long total = (long)lq * s.B * s.Hkv;
-        split_len = (total + 148L * 3 * 8 - 1) / (148L * 3 * 8);
-        if (split_len < 1024) split_len = 1024;
-        if (split_len > 8192) split_len = 8192;
-        split_len = (split_len + 255) / 256 * 256;
+        // All CTAs of a launch cost about the same, so the launch takes ceil(CTAs / resident slots) rounds of
+        // (tiles per warp + a fixed prologue/epilogue of about two tiles).  Pick the split count that minimises
+        // that product: whole waves, splits long enough to hide the fixed part.  Splits are multiples of 256
+        // tokens (4 warps x 64-token tiles).
+        const long quads = (lq + 255) / 256;                       // 256-token units per (sequence, KV head)
+        const long pairs = (long)s.B * s.Hkv;
+        const long slots = (long)sm_count() * partition_ctas_per_sm(s);
+        const long n_max = quads < 512 ? (quads > 0 ? quads : 1) : 512;
+        double best = 1e300;
+        long best_q = quads > 0 ? quads : 1;
+        for (long n = 1; n <= n_max; ++n) {
+            const long q = (quads + n - 1) / n;                    // quads per split = tiles per warp
+            if (q == 0) break;
+            const long n_eff = (quads + q - 1) / q;
+            const long waves = (n_eff * pairs + slots - 1) / slots;
+            const double cost = (double)waves * ((double)q + 2.0);
+            if (cost < best * 0.999) { best = cost; best_q = q; }
+        }
+        split_len = best_q * 256;
     }
     if (split_len < SKVQ_TOKEN_ALIGN) split_len = SKVQ_TOKEN_ALIGN;
     p.split_len = (int)split_len;
@@ -272,7 +360,7 @@ cudaError_t launch_attention(const Shape &s, const CachePtrs &c, const __half *q
                              cudaStream_t stream)
 {
     AttnArgs a{s, c, q, out, sm_scale * 1.4426950408889634f, plan, workspace};
-    dim3 grid(plan.n_splits + 1, s.Hkv, s.B);
+    dim3 grid(plan.n_splits, s.Hkv, s.B);
     if (ev_begin) cudaEventRecord(ev_begin, stream);
     bool handled = false;
     cudaError_t em = launch_partition_mma(s, c, q, a.scale_log2, plan, workspace, stream, &handled);

@@ -16,7 +16,7 @@
 // "four tokens of one byte column" registers, one AND leaves 4^j*code bytes, and p*h per group goes on a
 // 32-bit fixed-point grid whose four bytes are four A rows.  The integer accumulators are exact; they are
 // folded into fp32 (shared memory) only when the softmax reference or the bound on h moves, and the
-// reference only moves when a score exceeds it by 2^8, which after the first tile is rare.
+// reference only moves when a score exceeds it by 16 in the log2 domain, which after the first tile is rare.
 // sum_t p_t z_{t,g} is one more small fp16 MMA per 16 tokens.
 //
 // One CTA = 4 independent warps on one (sequence, KV head, split); tiles of 64 tokens arrive through a per-warp
@@ -29,7 +29,8 @@ namespace {
 using namespace mmak;
 
 constexpr int kHeadSlots = 4;           // query heads per KV head this kernel serves (rows = head x 4 digits)
-constexpr float kRefSlack = 8.0f;       // the softmax reference moves only when a score exceeds it by this (log2)
+constexpr int kRefSlackLog2 = 16;       // the softmax reference moves only when a score exceeds it by this (log2)
+constexpr float kRefSlack = (float)kRefSlackLog2;
 
 template <int G>
 struct GCfg {
@@ -129,17 +130,13 @@ __global__ void __launch_bounds__(kThreads, 3) partition_gqa_kernel(MmaArgs a)
     extern __shared__ __align__(128) uint8_t smem[];
     const Shape &s = a.s;
     const int part = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
-    if (part == a.plan.n_splits) {
-        window_part<R>(a, b, hk, smem);
-        return;
-    }
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t = lane & 3;
     const int L = a.c.lengths[b];
     const int Lq = max(L - s.W, 0);
     const int q_begin = min(part * a.plan.split_len, Lq);
     const int q_end = min(q_begin + a.plan.split_len, Lq);
-    const int n_parts = a.plan.n_splits + 1;
+    const int n_parts = a.plan.n_splits;
 
     // ---- CTA-wide prologue: permuted query on a per-head power-of-two scale, per-(head, group) constants
     float *qs = reinterpret_cast<float *>(smem);                   // [4][128] q' * F_r (exact), 0 for absent heads
@@ -294,7 +291,7 @@ __global__ void __launch_bounds__(kThreads, 3) partition_gqa_kernel(MmaArgs a)
 
     // Brings the integer sums into the fp32 sums in shared memory; everything there is then multiplied by corr_hd.
     auto fold = [&](float corr_hd) {
-        const float sa = h_bound * (d0 ? 1.52587890625e-05f : 5.9604644775390625e-08f);   // h_bound * 2^8 * 2^-32 * 256^d0
+        const float sa = h_bound * (d0 ? 256.0f : 1.0f) * (1.0f / (float)(1u << (32 - kRefSlackLog2)));   // h_bound * 2^slack * 2^-32 * 256^d0
         const float sb = sa * 65536.0f;
 #pragma unroll
         for (int nt = 0; nt < 16; ++nt) {
@@ -434,7 +431,7 @@ __global__ void __launch_bounds__(kThreads, 3) partition_gqa_kernel(MmaArgs a)
                     arg[mt][e] = valid ? fmaf(sraw[mt][e], cs, -m_ref) : -CUDART_INF_F;
                 }
         }
-        const float hscale = 16777216.0f / h_bound;      // 2^32 / (h_bound * 2^8)
+        const float hscale = (float)(1u << (32 - kRefSlackLog2)) / h_bound;      // 2^32 / (h_bound * 2^slack)
 
         // ---------------- per 32-token block: probabilities, p*h on the fixed-point grid, digits -> A fragments, MMAs
         const uint32_t vaddr = smem_u32(Vc) + offV;
@@ -443,7 +440,7 @@ __global__ void __launch_bounds__(kThreads, 3) partition_gqa_kernel(MmaArgs a)
             uint32_t uu[4][NG];
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-                const float p = ex2_approx(arg[2 * kk + (q >> 1)][q & 1]);      // at most 2^8; 0 past the end
+                const float p = ex2_approx(arg[2 * kk + (q >> 1)][q & 1]);      // at most 2^slack; 0 past the end
                 l_sum += p;
                 uint32_t vw[NG];
                 load_words<NG>(Vm + (32 * kk + own[q]) * NG, vw);
@@ -568,7 +565,7 @@ cudaError_t launch_one(const MmaArgs &a, cudaStream_t stream)
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    dim3 grid(a.plan.n_splits + 1, a.s.Hkv, a.s.B);
+    dim3 grid(a.plan.n_splits, a.s.Hkv, a.s.B);
     kern<<<grid, kThreads, C::kSmemBytes, stream>>>(a);
     return cudaGetLastError();
 }

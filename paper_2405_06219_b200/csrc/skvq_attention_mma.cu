@@ -20,7 +20,7 @@
 // tiles of codes + scale/zero through its own ring of shared-memory stages filled by
 // cp.async.bulk (mbarrier completion), keeps its own online-softmax state, and the 4 states are
 // merged in shared memory before one partial per query head is written to the workspace.
-// The fp16 window is a separate, small "part" handled by scalar code.
+// The fp16 window is handled by the merge kernel.
 #include "skvq_mma_common.cuh"
 
 namespace skvq {
@@ -82,17 +82,13 @@ __global__ void __launch_bounds__(kThreads) partition_mma_kernel(MmaArgs a)
     extern __shared__ __align__(128) uint8_t smem[];
     const Shape &s = a.s;
     const int part = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
-    if (part == a.plan.n_splits) {
-        window_part<R>(a, b, hk, smem);
-        return;
-    }
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t = lane & 3;
     const int L = a.c.lengths[b];
     const int Lq = max(L - s.W, 0);
     const int q_begin = min(part * a.plan.split_len, Lq);
     const int q_end = min(q_begin + a.plan.split_len, Lq);
-    const int n_parts = a.plan.n_splits + 1;
+    const int n_parts = a.plan.n_splits;
 
     // ---- CTA-wide prologue: permuted query, its fixed-point grid and per-(head, group) sums
     float *qs = reinterpret_cast<float *>(smem);                       // [R][128] q' (exact fp16 values)
@@ -597,7 +593,7 @@ cudaError_t launch_one(const MmaArgs &a, cudaStream_t stream)
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    dim3 grid(a.plan.n_splits + 1, a.s.Hkv, a.s.B);
+    dim3 grid(a.plan.n_splits, a.s.Hkv, a.s.B);
     kern<<<grid, kThreads, C::kSmemBytes, stream>>>(a);
     return cudaGetLastError();
 }

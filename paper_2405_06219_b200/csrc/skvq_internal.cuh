@@ -32,7 +32,7 @@ struct CachePtrs {
 
 struct SplitPlan {
     int split_len;   // quantized tokens per split (multiple of SKVQ_TOKEN_ALIGN)
-    int n_splits;    // splits of the quantized prefix per (sequence, KV head); one more part holds the fp16 window
+    int n_splits;    // splits of the quantized prefix per (sequence, KV head); the fp16 window belongs to the merge kernel
 };
 
 // Chooses the sequence partition for lengths up to max_len (host).

@@ -1,6 +1,5 @@
 // Pieces shared by the tensor-core partition kernels of skvq_decode_attention: launch arguments, PTX
-// wrappers (mma.sync, ldmatrix, cp.async.bulk + mbarrier with bounded polling) and the scalar code for
-// the fp16 window part.
+// wrappers (mma.sync, ldmatrix, cp.async.bulk + mbarrier with bounded polling).
 #pragma once
 #include <math_constants.h>
 
@@ -115,99 +114,6 @@ __device__ __forceinline__ float warp_sum(float v)
 #pragma unroll
     for (int m = 16; m > 0; m >>= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
     return v;
-}
-
-// Scalar path for the fp16 window part (at most W tokens; a few percent of the bytes).
-template <int R>
-__device__ void window_part(const MmaArgs &a, int b, int hk, uint8_t *smem_raw)
-{
-    const Shape &s = a.s;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int W = s.W;
-    const int L = a.c.lengths[b];
-    const int Lq = max(L - W, 0);
-    float (*sq)[kHeadDim] = reinterpret_cast<float (*)[kHeadDim]>(smem_raw);                 // [R][128]
-    float (*sp)[kThreads] = reinterpret_cast<float (*)[kThreads]>(smem_raw + R * kHeadDim * 4);   // [R][128]
-    float (*sred)[kWarps] = reinterpret_cast<float (*)[kWarps]>(smem_raw + 2 * R * kHeadDim * 4);  // [R][4]
-    const size_t bh = (size_t)b * s.Hkv + hk;
-    const int32_t *idx_k = a.c.reorder_k + (size_t)hk * kHeadDim;
-#pragma unroll
-    for (int r = 0; r < R; ++r)
-        sq[r][tid] = __half2float(a.q[((size_t)b * s.Hq + hk * R + r) * kHeadDim + (idx_k[tid] & (kHeadDim - 1))]) * a.scale_log2;
-    __syncthreads();
-    const __half *k_win = a.c.k_win + bh * (size_t)W * kHeadDim;
-    const __half *v_win = a.c.v_win + bh * (size_t)W * kHeadDim;
-    float m_run[R], l_thread[R], acc[R];
-#pragma unroll
-    for (int r = 0; r < R; ++r) { m_run[r] = -CUDART_INF_F; l_thread[r] = 0.f; acc[r] = 0.f; }
-    for (int tile0 = Lq; tile0 < L; tile0 += kThreads) {
-        const int t = tile0 + tid;
-        const bool valid = t < L;
-        float sc[R];
-#pragma unroll
-        for (int r = 0; r < R; ++r) sc[r] = valid ? 0.f : -CUDART_INF_F;
-        if (valid) {
-            const uint4 *row = reinterpret_cast<const uint4 *>(k_win + (size_t)(t % W) * kHeadDim);
-#pragma unroll 4
-            for (int j8 = 0; j8 < kHeadDim / 8; ++j8) {
-                const uint4 u = __ldg(row + j8);
-                const __half2 *h2 = reinterpret_cast<const __half2 *>(&u);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const float2 kv = __half22float2(h2[i]);
-#pragma unroll
-                    for (int r = 0; r < R; ++r)
-                        sc[r] = fmaf(sq[r][8 * j8 + 2 * i], kv.x, fmaf(sq[r][8 * j8 + 2 * i + 1], kv.y, sc[r]));
-                }
-            }
-        }
-#pragma unroll
-        for (int r = 0; r < R; ++r) {
-            const float wm = warp_max(sc[r]);
-            if (lane == 0) sred[r][warp] = wm;
-        }
-        __syncthreads();
-#pragma unroll
-        for (int r = 0; r < R; ++r) {
-            float tm = sred[r][0];
-#pragma unroll
-            for (int w = 1; w < kWarps; ++w) tm = fmaxf(tm, sred[r][w]);
-            const float m_new = fmaxf(m_run[r], tm);
-            const float corr = exp2f(m_run[r] - m_new);
-            const float p = valid ? exp2f(sc[r] - m_new) : 0.f;
-            sp[r][tid] = p;
-            l_thread[r] = l_thread[r] * corr + p;
-            m_run[r] = m_new;
-            acc[r] *= corr;
-        }
-        __syncthreads();
-        const int n_tok = min(kThreads, L - tile0);
-        for (int tt = 0; tt < n_tok; ++tt) {
-            const float val = __half2float(v_win[(size_t)((tile0 + tt) % W) * kHeadDim + tid]);
-#pragma unroll
-            for (int r = 0; r < R; ++r) acc[r] = fmaf(sp[r][tt], val, acc[r]);
-        }
-        __syncthreads();
-    }
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-        const float wsum = warp_sum(l_thread[r]);
-        if (lane == 0) sred[r][warp] = wsum;
-    }
-    __syncthreads();
-    const int part_idx = a.plan.n_splits;   // the window is the last part
-    const int n_parts = a.plan.n_splits + 1;
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-        float *part = a.ws + (((size_t)b * s.Hq + hk * R + r) * n_parts + part_idx) * kPartialStride;
-        part[tid] = acc[r];
-        if (tid == 0) {
-            float l = 0.f;
-            for (int w = 0; w < kWarps; ++w) l += sred[r][w];
-            part[kHeadDim] = m_run[r];
-            part[kHeadDim + 1] = l;
-        }
-    }
 }
 
 }  // namespace mmak

@@ -160,3 +160,13 @@ def algorithmic_bytes(w: Workload, lengths=None) -> int:
         total += w.n_kv_heads * (lq * per_tok + min(L, w.window) * D * 2 * 2)
     total += w.batch * w.n_q_heads * D * 2 * 2
     return int(total)
+
+
+def partition_kernel_bytes(w: Workload, lengths=None) -> int:
+    """The share of ``algorithmic_bytes`` that the partition kernel itself must move: packed codes and
+    scale/zero of the quantized prefix plus q (the fp16 window and the output belong to the merge kernel)."""
+    lengths = w.lengths() if lengths is None else np.asarray(lengths)
+    D, ng = w.head_dim, w.head_dim // w.group_size
+    per_tok = (D * w.k_bits // 8 + 4 * ng) + (D * w.v_bits // 8 + 4 * ng)
+    total = sum(w.n_kv_heads * max(L - w.window, 0) * per_tok for L in lengths.tolist())
+    return int(total + w.batch * w.n_q_heads * D * 2)

@@ -74,7 +74,7 @@ def test_workspace_size_grows_with_splits(lib):
     c = cfg()
     one = B.skvq_workspace_size(c, 4096, 1)
     four = B.skvq_workspace_size(c, 4096, 4)
-    assert one == 2 * 8 * 132 * 4 * 2 and four == 2 * 8 * 132 * 4 * 5     # splits + one window part
+    assert one == 2 * 8 * 132 * 4 * 1 and four == 2 * 8 * 132 * 4 * 4     # one partial per split and query head
     assert B.skvq_workspace_size(c, 4096, 0) >= one
     assert B.skvq_workspace_size(cfg(head_dim=64), 4096, 0) == 0
     assert B.skvq_step_staging_size(c) == 2 * (2 * 2 * 128 * 2) + 2 * (2 * 8 * 128 * 2)
