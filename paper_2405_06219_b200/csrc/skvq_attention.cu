@@ -51,6 +51,7 @@ __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
     const int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int rep = s.rep, G = s.G, ng = s.ng;
+    asm volatile("griddepcontrol.launch_dependents;");      // the merge kernel may start its window part early
     const int L = a.c.lengths[b];
     const int Lq = max(L - s.W, 0);
     const int q_begin = min(split * a.plan.split_len, Lq);
@@ -214,10 +215,11 @@ __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
     __syncthreads();
     const __half *k_win = a.c.k_win + bh * (size_t)W * kHeadDim;
     const __half *v_win = a.c.v_win + bh * (size_t)W * kHeadDim;
-    // P.V layout: warp w takes tokens w, w+4, ... of a tile, lane l channels 4l..4l+3 (one 8-byte load per row)
+    // P.V layout: a warp instruction reads two rows (16 lanes x 8 channels each); warp w takes row pairs w, w+4, ...
     __shared__ float sacc[kThreads / 32][kHeadDim];
     float m_run = -CUDART_INF_F, l_thread = 0.f;
-    float a4[4] = {0.f, 0.f, 0.f, 0.f};
+    float a8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    const int vsub = lane >> 4, vchunk = lane & 15;
     for (int tile0 = Lq; tile0 < L; tile0 += kThreads) {
         const int t = tile0 + tid;
         const bool valid = t < L;
@@ -250,21 +252,32 @@ __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
         l_thread = l_thread * corr + p;
         m_run = m_new;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) a4[i] *= corr;
+        for (int i = 0; i < 8; ++i) a8[i] *= corr;
         __syncthreads();
         const int n_tok = min(kThreads, L - tile0);
-#pragma unroll 8
-        for (int tt = warp; tt < n_tok; tt += kThreads / 32) {
-            const uint2 u = __ldg(reinterpret_cast<const uint2 *>(v_win + (size_t)((tile0 + tt) % W) * kHeadDim) + lane);
-            const float2 v01 = __half22float2(*reinterpret_cast<const __half2 *>(&u.x));
-            const float2 v23 = __half22float2(*reinterpret_cast<const __half2 *>(&u.y));
-            const float pt = sp[tt];
-            a4[0] = fmaf(pt, v01.x, a4[0]); a4[1] = fmaf(pt, v01.y, a4[1]);
-            a4[2] = fmaf(pt, v23.x, a4[2]); a4[3] = fmaf(pt, v23.y, a4[3]);
+#pragma unroll
+        for (int i = 0; i < kThreads / 8; ++i) {            // 16 independent 16-byte loads per thread
+            const int tt = 8 * i + 2 * warp + vsub;
+            if (tt < n_tok) {
+                const uint4 u = __ldg(reinterpret_cast<const uint4 *>(v_win + (size_t)((tile0 + tt) % W) * kHeadDim) + vchunk);
+                const __half2 *h2 = reinterpret_cast<const __half2 *>(&u);
+                const float pt = sp[tt];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float2 vv = __half22float2(h2[e]);
+                    a8[2 * e] = fmaf(pt, vv.x, a8[2 * e]);
+                    a8[2 * e + 1] = fmaf(pt, vv.y, a8[2 * e + 1]);
+                }
+            }
         }
         __syncthreads();   // sp and sred are rewritten by the next tile
     }
-    *reinterpret_cast<float4 *>(&sacc[warp][4 * lane]) = make_float4(a4[0], a4[1], a4[2], a4[3]);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) a8[i] += __shfl_xor_sync(0xffffffffu, a8[i], 16);
+    if (vsub == 0) {
+        *reinterpret_cast<float4 *>(&sacc[warp][8 * vchunk]) = make_float4(a8[0], a8[1], a8[2], a8[3]);
+        *reinterpret_cast<float4 *>(&sacc[warp][8 * vchunk + 4]) = make_float4(a8[4], a8[5], a8[6], a8[7]);
+    }
     const float lw = warp_sum(l_thread);
     if (lane == 0) sred[warp] = lw;
     __syncthreads();
@@ -272,6 +285,9 @@ __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
 #pragma unroll
     for (int w = 0; w < kThreads / 32; ++w) { l_win += sred[w]; acc += sacc[w][tid]; }
 
+    // The window above does not depend on the partition kernel; its partials do: wait for that grid here
+    // (a no-op unless this kernel was launched with programmatic stream serialization).
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     // log-sum-exp merge: the window and the S split partials; thread d owns reordered channel d
     const int S = a.plan.n_splits;
     const float *part = a.ws + ((size_t)b * s.Hq + hq) * S * kPartialStride;
@@ -299,7 +315,7 @@ __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
 // Resident CTAs per SM of the partition kernel that serves this shape (sets how many CTAs make one wave).
 static int partition_ctas_per_sm(const Shape &s)
 {
-    if (s.k_bits == 2 && s.v_bits == 2 && s.rep == 1 && s.G >= 64) return 4;   // integer kernel, 121 registers
+    if (s.rep == 1 && s.G >= 64) return s.k_bits == s.v_bits ? 4 : 3;           // integer kernel
     if (s.k_bits == 2 && s.v_bits == 2 && s.rep <= 4) return 3;                // grouped-query kernel, 168 registers
     return 8;                                                                  // scalar kernel
 }
@@ -377,7 +393,22 @@ cudaError_t launch_attention(const Shape &s, const CachePtrs &c, const __half *q
     if (ev_end) cudaEventRecord(ev_end, stream);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    merge_kernel<<<dim3(s.Hq, s.B), kHeadDim, 0, stream>>>(a);
+    {
+        // Programmatic dependent launch: merge CTAs may be scheduled while the last partition CTAs still run,
+        // do the window part, and wait (griddepcontrol.wait) before they read the partials.
+        cudaLaunchConfig_t lc = {};
+        lc.gridDim = dim3(s.Hq, s.B);
+        lc.blockDim = dim3(kHeadDim);
+        lc.dynamicSmemBytes = 0;
+        lc.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = ev_end ? 0 : 1;   // an event between the two kernels serialises them anyway
+        lc.attrs = attr;
+        lc.numAttrs = 1;
+        cudaError_t el = cudaLaunchKernelEx(&lc, merge_kernel, a);
+        if (el != cudaSuccess) return el;
+    }
     count_launch(2);
     return cudaGetLastError();
 }

@@ -132,6 +132,7 @@ __global__ void __launch_bounds__(kThreads, 3) partition_gqa_kernel(MmaArgs a)
     const int part = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t = lane & 3;
+    asm volatile("griddepcontrol.launch_dependents;");      // the merge kernel may start its window part early
     const int L = a.c.lengths[b];
     const int Lq = max(L - s.W, 0);
     const int q_begin = min(part * a.plan.split_len, Lq);

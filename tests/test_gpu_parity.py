@@ -117,6 +117,10 @@ def test_ragged_append_and_overflow_flag():
     (1, dict(context=2500, batch=2, n_q_heads=4, n_kv_heads=4, group_size=32), 2500),     # MHA with fine groups
     (1, dict(context=2500, batch=1, n_q_heads=8, n_kv_heads=4, group_size=64), 2500),     # 2 heads per KV head, g64
     (2, dict(context=4160, batch=1, n_q_heads=4, n_kv_heads=1, group_size=64), 4160),     # 4 heads per KV head, g64, full tiles only
+    (4, dict(context=2777, batch=2, ragged=None, n_q_heads=4, n_kv_heads=4, k_bits=4, v_bits=2), 2777),     # mixed widths
+    (4, dict(context=2777, batch=2, ragged=None, n_q_heads=4, n_kv_heads=4, k_bits=2, v_bits=4, group_size=128), 2777),
+    (4, dict(context=3100, batch=1, ragged=None, n_q_heads=4, n_kv_heads=4, group_size=128, window=128), 3100),   # 4-bit, one group
+    (4, dict(context=2000, batch=1, ragged=None, n_q_heads=8, n_kv_heads=4), 2000),      # 4-bit with 2 heads per KV head: scalar kernel
 ])
 def test_attention_matches_oracle(cfg_i, kw, n):
     w = small(cfg_i, **kw)
