@@ -8,6 +8,9 @@
 //                   the final window, so the read and the overwrite of a slot never race.
 //   "new" items     tokens t in [L0, L1): quantized straight from the input if t < L1-W, else
 //                   written to the ring unless an evict item refills that slot.
+// Bulk appends (prefill) send every whole, 64-aligned tile of tokens that goes straight from the input to the
+// quantized segment through append_bulk_kernel (rows staged in shared memory by cp.async, gathered from
+// there); append_kernel takes the rest: evictions from the ring, ring writes and the ragged ends.
 // Eight lanes own one 128-channel row (16 channels each); a warp handles two tokens at a time,
 // K rows on lanes 0-7/16-23 and V rows on lanes 8-15/24-31.  Group statistics are reduced with
 // xor-shuffles over G/16 lanes.  All quantizer arithmetic uses explicitly rounded fp32 intrinsics
@@ -26,12 +29,39 @@ struct AppendArgs {
     const __half *k, *v;
     const int32_t *n_new_per_seq;
     int n_new;
+    int use_bulk;   // append_bulk_kernel runs alongside
 };
 
 __device__ __forceinline__ int seq_new_count(const AppendArgs &a, int b)
 {
     int n = a.n_new_per_seq ? a.n_new_per_seq[b] : a.n_new;
     return min(max(n, 0), a.n_new);
+}
+
+// Tokens [f0, f1) of a sequence (multiples of 64, possibly empty) are quantized by append_bulk_kernel: they are
+// new, they end up below the window, and they form whole aligned tiles.
+__device__ __forceinline__ void bulk_range(int L0, int q_end, int &f0, int &f1)
+{
+    f0 = (L0 + 63) & ~63;
+    f1 = q_end & ~63;
+    if (f1 < f0) f1 = f0;
+}
+
+// The codes of 16 elements by the defining formula (IEEE division, rintf); kept out of line: it runs only for the
+// few row segments that have a quotient next to a rounding boundary.
+template <int BITS>
+__device__ __noinline__ void quantize16_exact(const float (&x)[16], float zf, float hf, uint32_t (&words)[2])
+{
+    constexpr int qmax = (1 << BITS) - 1;
+    words[0] = 0u;
+    words[1] = 0u;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        float c = rintf(__fdiv_rn(__fsub_rn(x[j], zf), hf));
+        c = fminf(fmaxf(c, 0.0f), (float)qmax);
+        const uint32_t code = (uint32_t)(int)c;
+        words[(j * BITS) >> 5] |= code << ((j * BITS) & 31);
+    }
 }
 
 // Quantize the 16 channels held by this lane; `lanes_per_group` lanes share the group statistics.
@@ -65,12 +95,37 @@ __device__ __forceinline__ void quantize16(const float (&x)[16], float alpha, in
     words[0] = 0u;
     words[1] = 0u;
     if (hf != 0.0f) {
+        // The code is clamp(rint(RN((x - z) / h)), 0, qmax) with IEEE division.  One division per element makes
+        // this path bound by the special-function unit, so the quotient is first formed as d * RN(1/h): that is
+        // within 3 * 2^-24 relative of the IEEE quotient, so wherever every value within 2^-18 relative of it
+        // rounds to the same integer, that integer is the code.  The test is two FMAs onto 1.5 * 2^23 (the
+        // mantissa's low bits are then the rounded integer, ties to even, like rintf) that must agree.  A lane
+        // with any element in doubt (a quotient next to k + 0.5, including exact ties) redoes its 16 elements with
+        // the division itself.  The packed word is summed modulo 2^32 with the constant bits of 1.5 * 2^23
+        // taken out at the end.
+        constexpr float MAGIC = 12582912.0f;                       // 0x4B400000
+        constexpr float UP = 1.0f + 3.814697265625e-06f, DN = 1.0f - 3.814697265625e-06f;
+        constexpr int PER_WORD = 32 / BITS;
+        uint32_t kconst = 0u;
+#pragma unroll
+        for (int j = 0; j < PER_WORD; ++j) kconst += 0x4B400000u << (j * BITS);
+        const float r = __frcp_rn(hf);
+        uint32_t doubt = 0u, w0 = 0u, w1 = 0u;
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
-            float r = rintf(__fdiv_rn(__fsub_rn(x[j], zf), hf));
-            r = fminf(fmaxf(r, 0.0f), (float)qmax);
-            const uint32_t code = (uint32_t)(int)r;
-            words[(j * BITS) >> 5] |= code << ((j * BITS) & 31);
+            const float q = __fmul_rn(__fsub_rn(x[j], zf), r);
+            const float qc = fminf(fmaxf(q, 0.0f), (float)qmax);
+            const uint32_t ta = __float_as_uint(__fmaf_rn(qc, DN, MAGIC));
+            const uint32_t tb = __float_as_uint(__fmaf_rn(qc, UP, MAGIC));
+            doubt |= ta ^ tb;
+            if ((j * BITS) < 32) w0 += ta << ((j * BITS) & 31);
+            else w1 += ta << ((j * BITS) & 31);
+        }
+        if (doubt == 0u) {
+            words[0] = w0 - kconst;
+            if (BITS == 4) words[1] = w1 - kconst;
+        } else {
+            quantize16_exact<BITS>(x, zf, hf, words);
         }
     }
 }
@@ -87,7 +142,10 @@ __global__ void __launch_bounds__(kAppendThreads) append_kernel(AppendArgs a)
     const int q_end = max(L1 - W, 0);            // tokens below this index are quantized after the call
     const int t_lo = max(L0 - W, 0);
     const int n_evict = max(min(L0, q_end) - t_lo, 0);
-    const int n_items = n_evict + n_b;
+    int f0, f1;
+    bulk_range(L0, q_end, f0, f1);
+    const int n_bulk = a.use_bulk ? f1 - f0 : 0;   // new tokens the bulk kernel takes: skipped here
+    const int n_items = n_evict + n_b - n_bulk;
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int sub = lane & 7;
@@ -138,6 +196,7 @@ __global__ void __launch_bounds__(kAppendThreads) append_kernel(AppendArgs a)
                 do_ring_write = true;
             } else {
                 t = L0 + (item - n_evict);
+                if (n_bulk > 0 && t >= f0) t += n_bulk;
                 if (t < q_end) {
                     do_quant = true;
                 } else if (W > 0) {
@@ -188,6 +247,82 @@ __global__ void __launch_bounds__(kAppendThreads) append_kernel(AppendArgs a)
     }
 }
 
+constexpr int kBulkTok = 64;
+constexpr int kBulkStride = kHeadDim + 8;   // halfs per staged row: 16 bytes of padding spread the rows over the banks
+
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc)
+                 : "memory");
+}
+
+// One CTA = one (sequence, KV head, 64-token tile) of bulk_range(): 64 K rows and 64 V rows are copied to
+// shared memory in 16-byte pieces (coalesced 256-byte rows), then gathered by the reorder index from there.
+__global__ void __launch_bounds__(kAppendThreads) append_bulk_kernel(AppendArgs a)
+{
+    const Shape &s = a.s;
+    const int b = blockIdx.z, h = blockIdx.y;
+    const int L0 = a.c.lengths[b];
+    const int n_b = seq_new_count(a, b);
+    const int L1 = L0 + n_b;
+    if (n_b == 0 || L1 > s.max_tokens) return;
+    int f0, f1;
+    bulk_range(L0, max(L1 - s.W, 0), f0, f1);
+    const int t0 = f0 + kBulkTok * blockIdx.x;
+    if (t0 >= f1) return;
+
+    __shared__ __align__(16) __half xs[2][kBulkTok][kBulkStride];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const size_t tok_stride = (size_t)s.Hkv * kHeadDim;
+    const size_t src0 = ((size_t)b * a.n_new + (t0 - L0)) * tok_stride + (size_t)h * kHeadDim;
+#pragma unroll
+    for (int c = tid; c < 2 * kBulkTok * 16; c += kAppendThreads) {
+        const int row = c >> 4, piece = c & 15, tensor = row >> 6, tok = row & (kBulkTok - 1);
+        cp_async16(&xs[tensor][tok][piece * 8], (tensor ? a.v : a.k) + src0 + (size_t)tok * tok_stride + piece * 8);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
+
+    const int sub = lane & 7, rsel = lane >> 3;
+    const size_t bh = (size_t)b * s.Hkv + h;
+    const int lanes_per_group = s.G >> 4;
+    const int g = (sub << 4) / s.G;
+#pragma unroll 1
+    for (int tensor = 0; tensor < 2; ++tensor) {
+        const int bits = tensor ? s.v_bits : s.k_bits;
+        const int row_bytes = kHeadDim * bits / 8;
+        uint8_t *codes = (tensor ? a.c.v_codes : a.c.k_codes) + bh * (size_t)s.cap * row_bytes;
+        __half2 *meta = (tensor ? a.c.v_meta : a.c.k_meta) + bh * (size_t)s.cap * s.ng;
+        const float alpha = ((tensor ? a.c.alpha_v : a.c.alpha_k) + (size_t)h * s.ng)[g];
+        int idx[16];
+        {
+            const int32_t *ip = (tensor ? a.c.reorder_v : a.c.reorder_k) + (size_t)h * kHeadDim + (sub << 4);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) idx[j] = ip[j] & (kHeadDim - 1);
+        }
+        const __half *src_j[16];      // this lane's 16 gather addresses in its first row; later rows are constant offsets
+#pragma unroll
+        for (int j = 0; j < 16; ++j) src_j[j] = &xs[tensor][warp * 4 + rsel][idx[j]];
+#pragma unroll 2
+        for (int it = 0; it < kBulkTok / 16; ++it) {
+            const int tok = it * 16 + warp * 4 + rsel;
+            float x[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) x[j] = __half2float(src_j[j][it * 16 * kBulkStride]);
+            uint32_t words[2];
+            __half2 hz;
+            if (bits == 2) quantize16<2>(x, alpha, lanes_per_group, words, hz);
+            else quantize16<4>(x, alpha, lanes_per_group, words, hz);
+            const int t = t0 + tok;
+            uint8_t *codes_row = codes + (size_t)t * row_bytes;
+            if (bits == 2) reinterpret_cast<uint32_t *>(codes_row)[sub] = words[0];
+            else reinterpret_cast<uint2 *>(codes_row)[sub] = make_uint2(words[0], words[1]);
+            if ((sub & (lanes_per_group - 1)) == 0) meta[(size_t)t * s.ng + g] = hz;
+        }
+    }
+}
+
 // lengths[b] += n_b, or flag an overflow and leave the sequence alone.
 __global__ void append_bookkeeping_kernel(AppendArgs a)
 {
@@ -208,14 +343,27 @@ cudaError_t launch_append(const Shape &s, const CachePtrs &c, const __half *k, c
                           const int32_t *n_new_per_seq, int n_new, cudaStream_t stream)
 {
     if (n_new <= 0) return cudaSuccess;
-    AppendArgs a{s, c, k, v, n_new_per_seq, n_new};
-    const int max_items = (s.W < n_new ? s.W : n_new) + n_new;
+    const bool bulk = n_new >= kBulkTok;
+    AppendArgs a{s, c, k, v, n_new_per_seq, n_new, bulk ? 1 : 0};
+    // what append_kernel keeps: evictions (at most W), and new tokens outside the bulk tiles (fewer than W + 128
+    // when there are bulk tiles, all of them otherwise)
+    const int n_evict_max = s.W < n_new ? s.W : n_new;
+    const int n_rest_max = bulk ? (n_new < s.W + 127 ? n_new : s.W + 127) : n_new;
+    const int max_items = n_evict_max + n_rest_max;
+    int launched = 0;
+    if (bulk) {
+        dim3 gridb((n_new + kBulkTok - 1) / kBulkTok, s.Hkv, s.B);
+        append_bulk_kernel<<<gridb, kAppendThreads, 0, stream>>>(a);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        ++launched;
+    }
     dim3 grid((max_items + kItemsPerCta - 1) / kItemsPerCta, s.Hkv, s.B);
     append_kernel<<<grid, kAppendThreads, 0, stream>>>(a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     append_bookkeeping_kernel<<<(s.B + 127) / 128, 128, 0, stream>>>(a);
-    count_launch(2);
+    count_launch(launched + 2);
     return cudaGetLastError();
 }
 
