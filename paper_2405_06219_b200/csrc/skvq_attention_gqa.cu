@@ -121,8 +121,13 @@ __device__ __forceinline__ float hi_half(uint32_t w) { return __high2float(*rein
 // (8 score rows of one octet, 4 tokens of one owner for the values) at two rows per shared-memory bank group.
 __device__ __forceinline__ int owned_token(int kk, int q, int gg) { return 32 * kk + 8 * q + ((gg + q) & 7); }
 
+// Two CTAs per SM (up to 255 registers per thread) measured faster than three (168 registers): the compiler needs
+// the registers to overlap the four 16-token score blocks and the two value blocks of a tile.
+#ifndef SKVQ_GQA_CTAS
+#define SKVQ_GQA_CTAS 2
+#endif
 template <int G, int R>
-__global__ void __launch_bounds__(kThreads, 3) partition_gqa_kernel(MmaArgs a)
+__global__ void __launch_bounds__(kThreads, SKVQ_GQA_CTAS) partition_gqa_kernel(MmaArgs a)
 {
     using C = GCfg<G>;
     constexpr int NG = C::NG;
