@@ -78,7 +78,7 @@ static int check_cache(const skvq_config *cfg, const skvq_cache *c, CachePtrs *o
 
 static size_t workspace_bytes(const Shape &s, const SplitPlan &p)
 {
-    return (size_t)s.B * s.Hq * p.n_splits * kPartialStride * sizeof(float);
+    return ((size_t)p.hdr_ints + (size_t)s.B * s.Hq * p.s_max * kPartialStride) * sizeof(float);
 }
 
 }  // namespace skvq

@@ -48,21 +48,28 @@ template <int KBITS, int VBITS>
 __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
 {
     const Shape &s = a.s;
-    const int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int rep = s.rep, G = s.G, ng = s.ng;
     asm volatile("griddepcontrol.launch_dependents;");      // the merge kernel may start its window part early
-    const int L = a.c.lengths[b];
-    const int Lq = max(L - s.W, 0);
-    const int q_begin = min(split * a.plan.split_len, Lq);
-    const int q_end = min(q_begin + a.plan.split_len, Lq);
-    const int n_parts = a.plan.n_splits;
+    asm volatile("griddepcontrol.wait;" ::: "memory");      // the plan kernel's header
+
+    __shared__ Segment seg_sh;
+    __shared__ int more_sh;
+    __shared__ SlotWalker walk;      // only thread 0 touches it; shared memory keeps it out of everybody's registers
+    if (tid == 0) more_sh = walk.start(reinterpret_cast<const int *>(a.ws), s.B, s.Hkv, blockIdx.x) ? 1 : 0;
+    __syncthreads();
+    if (!more_sh) return;
+    float *partials = a.ws + a.plan.hdr_ints;
 
     __shared__ float sq[kMaxRep][kHeadDim];        // permuted query, times sm_scale*log2(e)
     __shared__ float sqsum[kMaxRep][4];            // per-group sums of the above
     __shared__ float sp[kMaxRep][kTile];           // probabilities of the current tile
     __shared__ float sred[kMaxRep][kThreads / 32];
 
+    for (;;) {
+    if (tid == 0) seg_sh = walk.next(a.c.lengths, s.W, a.plan.lq_cap);
+    __syncthreads();
+    const int b = seg_sh.b, hk = seg_sh.hk, q_begin = seg_sh.tok_begin, q_end = seg_sh.tok_end, part_idx = seg_sh.part;
     const size_t bh = (size_t)b * s.Hkv + hk;
     const int32_t *idx_k = a.c.reorder_k + (size_t)hk * kHeadDim;
     for (int r = 0; r < rep; ++r) {
@@ -184,7 +191,7 @@ __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
 #pragma unroll
     for (int r = 0; r < kMaxRep; ++r) {
         if (r < rep) {
-            float *part = a.ws + (((size_t)b * s.Hq + hk * rep + r) * n_parts + split) * kPartialStride;
+            float *part = partials + (((size_t)b * s.Hq + hk * rep + r) * a.plan.s_max + part_idx) * kPartialStride;
             part[tid] = acc[r];
             if (tid == 0) {
                 float l = 0.f;
@@ -193,6 +200,58 @@ __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
                 part[kHeadDim + 1] = l;
             }
         }
+    }
+    __syncthreads();          // the segment's shared data is dead; thread 0 decides whether there is another one
+    if (tid == 0) more_sh = walk.done() ? 0 : 1;
+    __syncthreads();
+    if (!more_sh) break;
+    }
+}
+
+// Writes the workspace header of the flat partition: units (256 quantized tokens) per sequence as an exclusive
+// prefix array, their total over all KV heads, and the units per slot.  One warp; B is small next to the cache.
+__global__ void plan_kernel(AttnArgs a)
+{
+    asm volatile("griddepcontrol.launch_dependents;");      // the partition kernel may start its launch now; it waits for this grid
+    int *hdr = reinterpret_cast<int *>(a.ws);
+    int *pre = hdr + kPlanHdrInts;
+    const int lane = threadIdx.x & 31;
+    __shared__ int ups_sh;
+    if (threadIdx.x < 32) {
+    int run = 0;
+    for (int base = 0; base < a.s.B; base += 32) {
+        const int b = base + lane;
+        int nu = 0;
+        if (b < a.s.B) nu = (min(max(a.c.lengths[b] - a.s.W, 0), a.plan.lq_cap) + kUnitTok - 1) / kUnitTok;
+        int incl = nu;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += v;
+        }
+        if (b < a.s.B) pre[b] = run + incl - nu;
+        run += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    const long long total = (long long)run * a.s.Hkv;
+    const int ups = (int)max((total + a.plan.n_slots - 1) / a.plan.n_slots, 1LL);
+    if (lane == 0) {
+        pre[a.s.B] = run;
+        hdr[0] = (int)total;
+        hdr[1] = ups;
+        ups_sh = ups;
+    }
+    }
+    __syncthreads();
+    // first sequence of every slot: the largest b with Hkv * pre[b] <= w * ups (for slots past the end: unused)
+    int *slot_b = pre + a.s.B + 1;
+    for (int w = threadIdx.x; w < a.plan.n_slots; w += blockDim.x) {
+        const long long f = (long long)w * ups_sh;
+        int lo = 0, hi = a.s.B - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if ((long long)a.s.Hkv * pre[mid] <= f) lo = mid; else hi = mid - 1;
+        }
+        slot_b[w] = lo;
     }
 }
 
@@ -289,8 +348,8 @@ __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
     // (a no-op unless this kernel was launched with programmatic stream serialization).
     asm volatile("griddepcontrol.wait;" ::: "memory");
     // log-sum-exp merge: the window and the S split partials; thread d owns reordered channel d
-    const int S = a.plan.n_splits;
-    const float *part = a.ws + ((size_t)b * s.Hq + hq) * S * kPartialStride;
+    const int S = pair_partials(reinterpret_cast<const int *>(a.ws), s.Hkv, b, hk);
+    const float *part = a.ws + a.plan.hdr_ints + ((size_t)b * s.Hq + hq) * a.plan.s_max * kPartialStride;
     float M = m_run;
     for (int i = 0; i < S; ++i) M = fmaxf(M, part[(size_t)i * kPartialStride + kHeadDim]);
     float o = 0.f, l = 0.f;
@@ -337,38 +396,48 @@ static int sm_count()
 
 SplitPlan plan_splits(const Shape &s, int max_len, int requested_splits)
 {
-    const int lq = max_len - s.W > 0 ? max_len - s.W : 0;
     SplitPlan p;
-    long split_len;
+    p.lq_cap = max_len - s.W > 0 ? max_len - s.W : 0;
+    const long units = ((long)p.lq_cap + kUnitTok - 1) / kUnitTok;     // per (sequence, KV head), at most
+    const long pairs = (long)s.B * s.Hkv;
+    const long total = units * pairs > 0 ? units * pairs : 1;
+    long n;
     if (requested_splits > 0) {
-        split_len = (lq + requested_splits - 1) / requested_splits;
-        split_len = (split_len + SKVQ_TOKEN_ALIGN - 1) / SKVQ_TOKEN_ALIGN * SKVQ_TOKEN_ALIGN;
+        n = (long)requested_splits * pairs;
     } else {
-        // All CTAs of a launch cost about the same, so the launch takes ceil(CTAs / resident slots) rounds of
-        // (tiles per warp + a fixed prologue/epilogue of about two tiles).  Pick the split count that minimises
-        // that product: whole waves, splits long enough to hide the fixed part.  Splits are multiples of 256
-        // tokens (4 warps x 64-token tiles).
-        const long quads = (lq + 255) / 256;                       // 256-token units per (sequence, KV head)
-        const long pairs = (long)s.B * s.Hkv;
+        // every slot gets the same work, so one full wave is enough (a second wave costs a second prologue,
+        // pipeline fill and epilogue: about 8 us measured)
         const long slots = (long)sm_count() * partition_ctas_per_sm(s);
-        const long n_max = quads < 512 ? (quads > 0 ? quads : 1) : 512;
-        double best = 1e300;
-        long best_q = quads > 0 ? quads : 1;
-        for (long n = 1; n <= n_max; ++n) {
-            const long q = (quads + n - 1) / n;                    // quads per split = tiles per warp
-            if (q == 0) break;
-            const long n_eff = (quads + q - 1) / q;
-            const long waves = (n_eff * pairs + slots - 1) / slots;
-            const double cost = (double)waves * ((double)q + 2.0);
-            if (cost < best * 0.999) { best = cost; best_q = q; }
-        }
-        split_len = best_q * 256;
+        n = slots;
     }
-    if (split_len < SKVQ_TOKEN_ALIGN) split_len = SKVQ_TOKEN_ALIGN;
-    p.split_len = (int)split_len;
-    p.n_splits = (int)((lq + split_len - 1) / split_len);
-    if (p.n_splits < 1) p.n_splits = 1;
+    if (n > total) n = total;
+    if (n > (1L << 20)) n = 1L << 20;
+    p.n_slots = (int)n;
+    // A pair of nu units spreads over at most floor(nu / ups) + 2 slots, and ups >= total / n_slots >= Hkv * nu / n_slots.
+    long s_max = n / s.Hkv + 2;
+    if (s_max > units) s_max = units > 0 ? units : 1;
+    p.s_max = (int)s_max;
+    p.hdr_ints = (kPlanHdrInts + s.B + 1 + p.n_slots + 63) / 64 * 64;
     return p;
+}
+
+// A launch that may start before the kernel in front of it on the stream has finished; the kernel itself waits
+// (griddepcontrol.wait) where it first needs that kernel's results.
+template <typename Kern, typename Args>
+static cudaError_t launch_dependent(Kern kern, dim3 grid, dim3 block, size_t smem, cudaStream_t stream, bool overlap,
+                                    const Args &args)
+{
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = grid;
+    lc.blockDim = block;
+    lc.dynamicSmemBytes = smem;
+    lc.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = overlap ? 1 : 0;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    return cudaLaunchKernelEx(&lc, kern, args);
 }
 
 cudaError_t launch_attention(const Shape &s, const CachePtrs &c, const __half *q, __half *out, float sm_scale,
@@ -376,40 +445,31 @@ cudaError_t launch_attention(const Shape &s, const CachePtrs &c, const __half *q
                              cudaStream_t stream)
 {
     AttnArgs a{s, c, q, out, sm_scale * 1.4426950408889634f, plan, workspace};
-    dim3 grid(plan.n_splits, s.Hkv, s.B);
+    plan_kernel<<<1, 256, 0, stream>>>(a);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
     if (ev_begin) cudaEventRecord(ev_begin, stream);
+    const bool overlap = !ev_begin;      // an event between two kernels serialises them anyway
+    dim3 grid(plan.n_slots);
     bool handled = false;
-    cudaError_t em = launch_partition_mma(s, c, q, a.scale_log2, plan, workspace, stream, &handled);
+    cudaError_t em = launch_partition_mma(s, c, q, a.scale_log2, plan, workspace, stream, overlap, &handled);
     if (em != cudaSuccess) return em;
     if (!handled) {
-        em = launch_partition_gqa(s, c, q, a.scale_log2, plan, workspace, stream, &handled);
+        em = launch_partition_gqa(s, c, q, a.scale_log2, plan, workspace, stream, overlap, &handled);
         if (em != cudaSuccess) return em;
     }
     if (handled) { /* tensor-core kernel launched */ }
-    else if (s.k_bits == 2 && s.v_bits == 2) partition_kernel<2, 2><<<grid, kThreads, 0, stream>>>(a);
-    else if (s.k_bits == 4 && s.v_bits == 4) partition_kernel<4, 4><<<grid, kThreads, 0, stream>>>(a);
-    else if (s.k_bits == 4 && s.v_bits == 2) partition_kernel<4, 2><<<grid, kThreads, 0, stream>>>(a);
-    else partition_kernel<2, 4><<<grid, kThreads, 0, stream>>>(a);
+    else if (s.k_bits == 2 && s.v_bits == 2) em = launch_dependent(partition_kernel<2, 2>, grid, dim3(kThreads), 0, stream, overlap, a);
+    else if (s.k_bits == 4 && s.v_bits == 4) em = launch_dependent(partition_kernel<4, 4>, grid, dim3(kThreads), 0, stream, overlap, a);
+    else if (s.k_bits == 4 && s.v_bits == 2) em = launch_dependent(partition_kernel<4, 2>, grid, dim3(kThreads), 0, stream, overlap, a);
+    else em = launch_dependent(partition_kernel<2, 4>, grid, dim3(kThreads), 0, stream, overlap, a);
+    if (em != cudaSuccess) return em;
     if (ev_end) cudaEventRecord(ev_end, stream);
-    cudaError_t e = cudaGetLastError();
+    // merge CTAs may be scheduled while the last partition CTAs still run: they do the window part first and
+    // wait before they read the partials
+    e = launch_dependent(merge_kernel, dim3(s.Hq, s.B), dim3(kHeadDim), 0, stream, !ev_end, a);
     if (e != cudaSuccess) return e;
-    {
-        // Programmatic dependent launch: merge CTAs may be scheduled while the last partition CTAs still run,
-        // do the window part, and wait (griddepcontrol.wait) before they read the partials.
-        cudaLaunchConfig_t lc = {};
-        lc.gridDim = dim3(s.Hq, s.B);
-        lc.blockDim = dim3(kHeadDim);
-        lc.dynamicSmemBytes = 0;
-        lc.stream = stream;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = ev_end ? 0 : 1;   // an event between the two kernels serialises them anyway
-        lc.attrs = attr;
-        lc.numAttrs = 1;
-        cudaError_t el = cudaLaunchKernelEx(&lc, merge_kernel, a);
-        if (el != cudaSuccess) return el;
-    }
-    count_launch(2);
+    count_launch(3);
     return cudaGetLastError();
 }
 

@@ -134,15 +134,65 @@ __global__ void __launch_bounds__(kThreads, SKVQ_GQA_CTAS) partition_gqa_kernel(
     static_assert(R <= kHeadSlots, "rows of the P.V MMAs are 4 heads x 4 digits");
     extern __shared__ __align__(128) uint8_t smem[];
     const Shape &s = a.s;
-    const int part = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t = lane & 3;
     asm volatile("griddepcontrol.launch_dependents;");      // the merge kernel may start its window part early
-    const int L = a.c.lengths[b];
-    const int Lq = max(L - s.W, 0);
-    const int q_begin = min(part * a.plan.split_len, Lq);
-    const int q_end = min(q_begin + a.plan.split_len, Lq);
-    const int n_parts = a.plan.n_splits;
+    asm volatile("griddepcontrol.wait;" ::: "memory");      // the plan kernel's header
+
+    __shared__ Segment seg_sh;
+    __shared__ int more_sh;
+    __shared__ SlotWalker walk;      // only thread 0 touches it; shared memory keeps it out of everybody's registers
+    if (tid == 0) more_sh = walk.start(reinterpret_cast<const int *>(a.ws), s.B, s.Hkv, blockIdx.x) ? 1 : 0;
+    __syncthreads();
+    if (!more_sh) return;
+    float *partials = a.ws + a.plan.hdr_ints;
+
+    // per-warp pipeline state that outlives a segment: the stage barriers and how many tiles have gone through them
+    uint8_t *warp_base = smem + C::kQBytes + warp * C::kWarpBytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(warp_base + C::kStages * C::kStageBytes + C::kXBytes + C::kOBytes + C::kZBytes);
+    const uint32_t bar0 = smem_u32(bars);
+    if (lane == 0) {
+#pragma unroll
+        for (int i = 0; i < C::kStages; ++i) mbar_init(bar0 + 8 * i, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncwarp();
+    uint32_t tiles_done = 0;
+    bool failed = false;
+
+    for (;;) {
+    if (tid == 0) seg_sh = walk.next(a.c.lengths, s.W, a.plan.lq_cap);
+    __syncthreads();
+    const int b = seg_sh.b, hk = seg_sh.hk, q_begin = seg_sh.tok_begin, q_end = seg_sh.tok_end, part = seg_sh.part;
+    const int n_parts = a.plan.s_max;
+
+    uint8_t *stage_base = warp_base;
+    const size_t bh = (size_t)b * s.Hkv + hk;
+    const uint8_t *k_codes = a.c.k_codes + bh * (size_t)s.cap * kRowBytes;
+    const uint8_t *v_codes = a.c.v_codes + bh * (size_t)s.cap * kRowBytes;
+    const __half2 *k_meta = a.c.k_meta + bh * (size_t)s.cap * NG;
+    const __half2 *v_meta = a.c.v_meta + bh * (size_t)s.cap * NG;
+
+    const int n_tiles = (q_end - q_begin + kTileTok - 1) / kTileTok;
+    const int n_my = (n_tiles > warp && !failed) ? (n_tiles - warp + kWarps - 1) / kWarps : 0;
+
+    auto issue = [&](int i) {   // lane 0 only
+        const int st = (tiles_done + i) % C::kStages;
+        const int tok0 = q_begin + (warp + i * kWarps) * kTileTok;
+        const uint32_t dst = smem_u32(stage_base + st * C::kStageBytes);
+        const uint32_t bar = bar0 + 8 * st;
+        mbar_expect_tx(bar, C::kStageBytes);
+        bulk_g2s(dst, k_codes + (size_t)tok0 * kRowBytes, C::kCodeTile, bar);
+        bulk_g2s(dst + C::kCodeTile, v_codes + (size_t)tok0 * kRowBytes, C::kCodeTile, bar);
+        bulk_g2s(dst + 2 * C::kCodeTile, k_meta + (size_t)tok0 * NG, C::kMetaTile, bar);
+        bulk_g2s(dst + 2 * C::kCodeTile + C::kMetaTile, v_meta + (size_t)tok0 * NG, C::kMetaTile, bar);
+    };
+    if (lane == 0) {      // the first copies are in flight while the query is prepared
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the stages held the previous segment's result
+        for (int i = 0; i < C::kStages && i < n_my; ++i) issue(i);
+    }
+
 
     // ---- CTA-wide prologue: permuted query on a per-head power-of-two scale, per-(head, group) constants
     float *qs = reinterpret_cast<float *>(smem);                   // [4][128] q' * F_r (exact), 0 for absent heads
@@ -151,7 +201,6 @@ __global__ void __launch_bounds__(kThreads, SKVQ_GQA_CTAS) partition_gqa_kernel(
     float *csc = sqs + kHeadSlots * 4;                             // [4]     sm_scale*log2(e) / F_r
     int *fexp = reinterpret_cast<int *>(csc + kHeadSlots);         // [4]
     float *redmax = reinterpret_cast<float *>(fexp + kHeadSlots);  // [4 warps][4]
-    uint8_t *warp_base = smem + C::kQBytes + warp * C::kWarpBytes;
     {
         const int32_t *idx_k = a.c.reorder_k + (size_t)hk * kHeadDim;
         const int src = idx_k[tid] & (kHeadDim - 1);
@@ -224,44 +273,12 @@ __global__ void __launch_bounds__(kThreads, SKVQ_GQA_CTAS) partition_gqa_kernel(
     const float cs = csc[t];                                     // this lane's score columns belong to head t
 
     // ---- per-warp shared memory
-    uint8_t *stage_base = warp_base;
     uint2 *Xs = reinterpret_cast<uint2 *>(warp_base + C::kStages * C::kStageBytes);                  // [NG][2][32]
     float *Os = reinterpret_cast<float *>(warp_base + C::kStages * C::kStageBytes + C::kXBytes);     // [4][128]
     float *Zs = Os + kHeadSlots * kHeadDim;                                                          // [4][4]
-    uint64_t *bars = reinterpret_cast<uint64_t *>(reinterpret_cast<uint8_t *>(Zs) + C::kZBytes);
-    const uint32_t bar0 = smem_u32(bars);
-    if (lane == 0) {
-#pragma unroll
-        for (int i = 0; i < C::kStages; ++i) mbar_init(bar0 + 8 * i, 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
 #pragma unroll
     for (int i = 0; i < kHeadSlots * kHeadDim / 32; ++i) Os[lane + 32 * i] = 0.f;
     __syncwarp();
-
-    const size_t bh = (size_t)b * s.Hkv + hk;
-    const uint8_t *k_codes = a.c.k_codes + bh * (size_t)s.cap * kRowBytes;
-    const uint8_t *v_codes = a.c.v_codes + bh * (size_t)s.cap * kRowBytes;
-    const __half2 *k_meta = a.c.k_meta + bh * (size_t)s.cap * NG;
-    const __half2 *v_meta = a.c.v_meta + bh * (size_t)s.cap * NG;
-
-    const int n_tiles = (q_end - q_begin + kTileTok - 1) / kTileTok;
-    const int n_my = n_tiles > warp ? (n_tiles - warp + kWarps - 1) / kWarps : 0;
-
-    auto issue = [&](int i) {   // lane 0 only
-        const int st = i % C::kStages;
-        const int tok0 = q_begin + (warp + i * kWarps) * kTileTok;
-        const uint32_t dst = smem_u32(stage_base + st * C::kStageBytes);
-        const uint32_t bar = bar0 + 8 * st;
-        mbar_expect_tx(bar, C::kStageBytes);
-        bulk_g2s(dst, k_codes + (size_t)tok0 * kRowBytes, C::kCodeTile, bar);
-        bulk_g2s(dst + C::kCodeTile, v_codes + (size_t)tok0 * kRowBytes, C::kCodeTile, bar);
-        bulk_g2s(dst + 2 * C::kCodeTile, k_meta + (size_t)tok0 * NG, C::kMetaTile, bar);
-        bulk_g2s(dst + 2 * C::kCodeTile + C::kMetaTile, v_meta + (size_t)tok0 * NG, C::kMetaTile, bar);
-    };
-    if (lane == 0)
-        for (int i = 0; i < C::kStages && i < n_my; ++i) issue(i);
 
     // ---- running state (this lane: head t, the eight tokens per tile that lane group g owns)
     float m_ref = -CUDART_INF_F;                               // softmax reference of head t (log2 domain)
@@ -276,7 +293,7 @@ __global__ void __launch_bounds__(kThreads, SKVQ_GQA_CTAS) partition_gqa_kernel(
         for (int j = 0; j < 4; ++j) acc[i][j] = 0;
     float h_bound = 6.103515625e-05f;                          // power of two above every value scale seen so far
     uint32_t h_thr = 0x0400u;                                  // the same bound as an fp16 bit pattern (2^-14)
-    bool acc_live = false, failed = false;
+    bool acc_live = false;
 
     // lane constants
     const int hd = g & 3, d0 = g >> 2;                         // this lane's P.V rows: head hd, digits d0 and d0 + 2
@@ -317,8 +334,8 @@ __global__ void __launch_bounds__(kThreads, SKVQ_GQA_CTAS) partition_gqa_kernel(
     };
 
     for (int i = 0; i < n_my; ++i) {
-        const int st = i % C::kStages;
-        const uint32_t parity = (uint32_t)(i / C::kStages) & 1u;
+        const int st = (tiles_done + i) % C::kStages;
+        const uint32_t parity = ((tiles_done + i) / C::kStages) & 1u;
         if (!mbar_wait_bounded(bar0 + 8 * st, parity)) { failed = true; break; }
         uint8_t *Kc = stage_base + st * C::kStageBytes;
         uint8_t *Vc = Kc + C::kCodeTile;
@@ -497,8 +514,8 @@ __global__ void __launch_bounds__(kThreads, SKVQ_GQA_CTAS) partition_gqa_kernel(
 
     if (failed) {
         for (int i2 = 0; i2 < n_my; ++i2) {
-            const int st = i2 % C::kStages;
-            (void)mbar_wait_bounded(bar0 + 8 * st, (uint32_t)(i2 / C::kStages) & 1u);
+            const int st = (tiles_done + i2) % C::kStages;
+            (void)mbar_wait_bounded(bar0 + 8 * st, ((tiles_done + i2) / C::kStages) & 1u);
         }
         if (lane == 0 && a.c.status) atomicOr(a.c.status, 2);
     }
@@ -554,14 +571,20 @@ __global__ void __launch_bounds__(kThreads, SKVQ_GQA_CTAS) partition_gqa_kernel(
                 l = fmaf(ow[w][kHeadDim + 1], wgt, l);
             }
         }
-        float *dst = a.ws + (((size_t)b * s.Hq + hk * R + r) * n_parts + part) * kPartialStride;
+        float *dst = partials + (((size_t)b * s.Hq + hk * R + r) * n_parts + part) * kPartialStride;
         dst[tid] = o;
         if (tid == 0) { dst[kHeadDim] = M; dst[kHeadDim + 1] = l; }
+    }
+    tiles_done += n_my;
+    __syncthreads();          // the segment's shared data is dead; thread 0 decides whether there is another one
+    if (tid == 0) more_sh = walk.done() ? 0 : 1;
+    __syncthreads();
+    if (!more_sh) break;
     }
 }
 
 template <int G, int R>
-cudaError_t launch_one(const MmaArgs &a, cudaStream_t stream)
+cudaError_t launch_one(const MmaArgs &a, cudaStream_t stream, bool overlap)
 {
     using C = GCfg<G>;
     static bool configured = false;
@@ -571,19 +594,17 @@ cudaError_t launch_one(const MmaArgs &a, cudaStream_t stream)
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    dim3 grid(a.plan.n_splits, a.s.Hkv, a.s.B);
-    kern<<<grid, kThreads, C::kSmemBytes, stream>>>(a);
-    return cudaGetLastError();
+    return launch_dependent(kern, dim3(a.plan.n_slots), dim3(kThreads), C::kSmemBytes, stream, overlap, a);
 }
 
 template <int G>
-cudaError_t launch_g(const MmaArgs &a, cudaStream_t stream, bool *handled)
+cudaError_t launch_g(const MmaArgs &a, cudaStream_t stream, bool overlap, bool *handled)
 {
     *handled = true;
     switch (a.s.rep) {
-        case 1: return launch_one<G, 1>(a, stream);
-        case 2: return launch_one<G, 2>(a, stream);
-        case 4: return launch_one<G, 4>(a, stream);
+        case 1: return launch_one<G, 1>(a, stream, overlap);
+        case 2: return launch_one<G, 2>(a, stream, overlap);
+        case 4: return launch_one<G, 4>(a, stream, overlap);
         default: *handled = false; return cudaSuccess;
     }
 }
@@ -593,15 +614,15 @@ cudaError_t launch_g(const MmaArgs &a, cudaStream_t stream, bool *handled)
 // Launches the kernel above when the configuration is covered (2-bit K and V, 1, 2 or 4 query heads per KV
 // head); *handled tells the caller whether it did.
 cudaError_t launch_partition_gqa(const Shape &s, const CachePtrs &c, const __half *q, float scale_log2,
-                                 const SplitPlan &plan, float *workspace, cudaStream_t stream, bool *handled)
+                                 const SplitPlan &plan, float *workspace, cudaStream_t stream, bool overlap, bool *handled)
 {
     *handled = false;
     if (s.k_bits != 2 || s.v_bits != 2) return cudaSuccess;
     MmaArgs a{s, c, q, scale_log2, plan, workspace};
     switch (s.G) {
-        case 128: return launch_g<128>(a, stream, handled);
-        case 64: return launch_g<64>(a, stream, handled);
-        case 32: return launch_g<32>(a, stream, handled);
+        case 128: return launch_g<128>(a, stream, overlap, handled);
+        case 64: return launch_g<64>(a, stream, overlap, handled);
+        case 32: return launch_g<32>(a, stream, overlap, handled);
         default: return cudaSuccess;
     }
 }

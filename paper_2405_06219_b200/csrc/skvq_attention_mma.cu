@@ -43,7 +43,7 @@ struct Cfg {
     static constexpr int kScBytes = T * NG * 8;                           // per (token, group): low and high digit pairs
     static constexpr int kPBytes = (T / 32) * 8 * 32;                     // P operand tile: [k-block][8 columns][32 tokens] bytes
     static constexpr int kWarpBytes = kStages * kStageBytes + kScBytes + kPBytes + 64;   // + mbarriers
-    static constexpr int kQBytes = (kHeadDim * 4 + NG * 4 + 2 * 4 + 64 + 127) / 128 * 128;
+    static constexpr int kQBytes = (kHeadDim * 4 + NG * 4 + 2 * 4 + 64 + 127) / 128 * 128 + 512;   // + the B operand image
     static constexpr int kSmemBytes = kQBytes + kWarps * kWarpBytes;
     static constexpr int kCtasPerSm = (KB == VB) ? 4 : 3;
     static_assert(kStages * kStageBytes >= NG * kHeadDim * 4 + kPartialStride * 4, "stage area is reused for the final merge");
@@ -57,15 +57,65 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB>::kCtasPerSm) partitio
     constexpr int NG = C::NG, KROW = C::KROW, VROW = C::VROW, T = C::T;
     extern __shared__ __align__(128) uint8_t smem[];
     const Shape &s = a.s;
-    const int part = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t = lane & 3;
     asm volatile("griddepcontrol.launch_dependents;");      // the merge kernel may start its window part early
-    const int L = a.c.lengths[b];
-    const int Lq = max(L - s.W, 0);
-    const int q_begin = min(part * a.plan.split_len, Lq);
-    const int q_end = min(q_begin + a.plan.split_len, Lq);
-    const int n_parts = a.plan.n_splits;
+    asm volatile("griddepcontrol.wait;" ::: "memory");      // the plan kernel's header
+
+    __shared__ Segment seg_sh;
+    __shared__ int more_sh;
+    __shared__ SlotWalker walk;      // only thread 0 touches it; shared memory keeps it out of everybody's registers
+    if (tid == 0) more_sh = walk.start(reinterpret_cast<const int *>(a.ws), s.B, s.Hkv, blockIdx.x) ? 1 : 0;
+    __syncthreads();
+    if (!more_sh) return;
+    float *partials = a.ws + a.plan.hdr_ints;
+
+    // per-warp pipeline state that outlives a segment: the stage barriers and how many tiles have gone through them
+    uint8_t *warp_base = smem + C::kQBytes + warp * C::kWarpBytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(warp_base + C::kStages * C::kStageBytes + C::kScBytes + C::kPBytes);
+    const uint32_t bar0 = smem_u32(bars);
+    if (lane == 0) {
+#pragma unroll
+        for (int i = 0; i < C::kStages; ++i) mbar_init(bar0 + 8 * i, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncwarp();
+    uint32_t tiles_done = 0;
+    bool failed = false;
+
+    for (;;) {
+    if (tid == 0) seg_sh = walk.next(a.c.lengths, s.W, a.plan.lq_cap);
+    __syncthreads();
+    const int b = seg_sh.b, hk = seg_sh.hk, q_begin = seg_sh.tok_begin, q_end = seg_sh.tok_end, part = seg_sh.part;
+    const int n_parts = a.plan.s_max;
+
+    uint8_t *stage_base = warp_base;
+    const size_t bh = (size_t)b * s.Hkv + hk;
+    const uint8_t *k_codes = a.c.k_codes + bh * (size_t)s.cap * KROW;
+    const uint8_t *v_codes = a.c.v_codes + bh * (size_t)s.cap * VROW;
+    const __half2 *k_meta = a.c.k_meta + bh * (size_t)s.cap * NG;
+    const __half2 *v_meta = a.c.v_meta + bh * (size_t)s.cap * NG;
+
+    const int n_tiles = (q_end - q_begin + T - 1) / T;                          // tiles of this split
+    const int n_my = (n_tiles > warp && !failed) ? (n_tiles - warp + kWarps - 1) / kWarps : 0;   // tiles warp, warp+4, ...
+
+    auto issue = [&](int i) {   // lane 0 only: start the copies of this warp's i-th tile
+        const int st = (tiles_done + i) % C::kStages;
+        const int tok0 = q_begin + (warp + i * kWarps) * T;                       // multiple of 32: 16-byte aligned sources
+        const uint32_t dst = smem_u32(stage_base + st * C::kStageBytes);
+        const uint32_t bar = bar0 + 8 * st;
+        mbar_expect_tx(bar, C::kStageBytes);
+        bulk_g2s(dst, k_codes + (size_t)tok0 * KROW, C::kKTile, bar);
+        bulk_g2s(dst + C::kKTile, v_codes + (size_t)tok0 * VROW, C::kVTile, bar);
+        bulk_g2s(dst + C::kKTile + C::kVTile, k_meta + (size_t)tok0 * NG, C::kMetaTile, bar);
+        bulk_g2s(dst + C::kKTile + C::kVTile + C::kMetaTile, v_meta + (size_t)tok0 * NG, C::kMetaTile, bar);
+    };
+    if (lane == 0) {      // the first copies are in flight while the query is prepared
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the stages held the previous segment's result
+        for (int i = 0; i < C::kStages && i < n_my; ++i) issue(i);
+    }
+
 
     // ---- CTA-wide prologue: permuted query, its fixed-point grid and per-group sums
     float *qs = reinterpret_cast<float *>(smem);                       // [128] q' (exact fp16 values)
@@ -73,7 +123,6 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB>::kCtasPerSm) partitio
     float *cF = sqs + NG;                                              // scale / F, F = 2^kexp
     int *kexp = reinterpret_cast<int *>(cF + 1);
     float *redmax = reinterpret_cast<float *>(kexp + 1);               // [4]
-    uint8_t *warp_base = smem + C::kQBytes + warp * C::kWarpBytes;
     {
         const int32_t *idx_k = a.c.reorder_k + (size_t)hk * kHeadDim;
         const int src = idx_k[tid] & (kHeadDim - 1);
@@ -109,8 +158,9 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB>::kCtasPerSm) partitio
     // word (weight 4^t).  4-bit codes: register reg comes from word 4ks + 2(t>>1) + reg under mask t&1, byte bb =
     // code 2bb+(t&1) of that word (weight 16^(t&1)).  Column = byte digit of round(q' * F / weight).
     // Thread tid owns channel tid: it writes the four digits of that channel as bytes straight into the
-    // register image bimg[digit][ks][reg][t] (byte bb), which the lanes then load word by word.
-    uint8_t *bimg0 = smem + C::kQBytes;   // [4][4][2][4] words = 512 bytes in warp 0's stage area, idle until the pipeline starts
+    // register image bimg[digit][ks][reg][t] (byte bb), which the lanes then load word by word (the barrier at the
+    // end of a segment keeps the next segment's writes behind these reads).
+    uint8_t *bimg0 = smem + C::kQBytes - 512;   // [4][4][2][4] words
     {
         int ks, reg, bb, tt, wlog2;
         if constexpr (KB == 2) {
@@ -138,49 +188,14 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB>::kCtasPerSm) partitio
             for (int reg = 0; reg < 2; ++reg)
                 bq[ks][reg] = (g < 4) ? reinterpret_cast<const uint32_t *>(bimg0)[(((dig * 4 + ks) * 2 + reg) * 4 + t)] : 0u;
     }
-    __syncthreads();   // the image lives in the stage area: everyone has read it before any copy lands there
     const float cFr = cF[0];
     float sqr[NG];
 #pragma unroll
     for (int gg = 0; gg < NG; ++gg) sqr[gg] = sqs[gg];
 
-    // ---- per-warp pipeline state
-    uint8_t *stage_base = warp_base;
+    // ---- per-warp buffers
     float *Sc = reinterpret_cast<float *>(warp_base + C::kStages * C::kStageBytes);      // [T][NG][2]
     uint8_t *Pb = warp_base + C::kStages * C::kStageBytes + C::kScBytes;                 // [k-block][8 columns][4 t][2 halves][4 tokens]
-    uint64_t *bars = reinterpret_cast<uint64_t *>(warp_base + C::kStages * C::kStageBytes + C::kScBytes + C::kPBytes);
-    const uint32_t bar0 = smem_u32(bars);
-    if (lane == 0) {
-#pragma unroll
-        for (int i = 0; i < C::kStages; ++i) mbar_init(bar0 + 8 * i, 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    __syncwarp();
-
-    const size_t bh = (size_t)b * s.Hkv + hk;
-    const uint8_t *k_codes = a.c.k_codes + bh * (size_t)s.cap * KROW;
-    const uint8_t *v_codes = a.c.v_codes + bh * (size_t)s.cap * VROW;
-    const __half2 *k_meta = a.c.k_meta + bh * (size_t)s.cap * NG;
-    const __half2 *v_meta = a.c.v_meta + bh * (size_t)s.cap * NG;
-
-    const int n_tiles = (q_end - q_begin + T - 1) / T;                          // tiles of this split
-    const int n_my = n_tiles > warp ? (n_tiles - warp + kWarps - 1) / kWarps : 0;   // tiles warp, warp+4, ...
-
-    auto issue = [&](int i) {   // lane 0 only: start the copies of this warp's i-th tile
-        const int st = i % C::kStages;
-        const int tok0 = q_begin + (warp + i * kWarps) * T;                       // multiple of 32: 16-byte aligned sources
-        const uint32_t dst = smem_u32(stage_base + st * C::kStageBytes);
-        const uint32_t bar = bar0 + 8 * st;
-        mbar_expect_tx(bar, C::kStageBytes);
-        bulk_g2s(dst, k_codes + (size_t)tok0 * KROW, C::kKTile, bar);
-        bulk_g2s(dst + C::kKTile, v_codes + (size_t)tok0 * VROW, C::kVTile, bar);
-        bulk_g2s(dst + C::kKTile + C::kVTile, k_meta + (size_t)tok0 * NG, C::kMetaTile, bar);
-        bulk_g2s(dst + C::kKTile + C::kVTile + C::kMetaTile, v_meta + (size_t)tok0 * NG, C::kMetaTile, bar);
-    };
-    if (lane == 0) {
-        for (int i = 0; i < C::kStages && i < n_my; ++i) issue(i);
-    }
 
     // online-softmax state (per warp; m is warp-uniform, the sums are per-lane partials)
     float m_run = -CUDART_INF_F, l_part = 0.f, z_part[NG];
@@ -196,12 +211,11 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB>::kCtasPerSm) partitio
         for (int i = 0; i < 4; ++i) { cv[f][i] = 0.f; iacc[f][i] = 0; }
     float h_bound = 6.103515625e-05f;   // 2^-14: every scale seen so far is below this power of two
 
-    bool failed = false;
     const uint32_t kmask = KB == 2 ? (0x03030303u << (2 * t)) : (0x0F0F0F0Fu << (4 * (t & 1)));
 
     for (int i = 0; i < n_my; ++i) {
-        const int st = i % C::kStages;
-        const uint32_t parity = (uint32_t)(i / C::kStages) & 1u;
+        const int st = (tiles_done + i) % C::kStages;
+        const uint32_t parity = ((tiles_done + i) / C::kStages) & 1u;
         if (!mbar_wait_bounded(bar0 + 8 * st, parity)) { failed = true; break; }
         const uint8_t *Kc = stage_base + st * C::kStageBytes;
         const uint8_t *Vc = Kc + C::kKTile;
@@ -354,8 +368,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB>::kCtasPerSm) partitio
     if (failed) {
         // Drain (bounded) whatever copies are still in flight into this warp's stages, then report.
         for (int i2 = 0; i2 < n_my; ++i2) {
-            const int st = i2 % C::kStages;
-            (void)mbar_wait_bounded(bar0 + 8 * st, (uint32_t)(i2 / C::kStages) & 1u);
+            const int st = (tiles_done + i2) % C::kStages;
+            (void)mbar_wait_bounded(bar0 + 8 * st, ((tiles_done + i2) / C::kStages) & 1u);
         }
         if (lane == 0 && a.c.status) atomicOr(a.c.status, 2);
         m_run = -CUDART_INF_F;
@@ -425,14 +439,20 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB>::kCtasPerSm) partitio
                 l = fmaf(ow[w][kHeadDim + 1], wgt, l);
             }
         }
-        float *dst = a.ws + (((size_t)b * s.Hq + hk) * n_parts + part) * kPartialStride;
+        float *dst = partials + (((size_t)b * s.Hq + hk) * n_parts + part) * kPartialStride;
         dst[tid] = o;
         if (tid == 0) { dst[kHeadDim] = M; dst[kHeadDim + 1] = l; }
+    }
+    tiles_done += n_my;
+    __syncthreads();          // the segment's shared data is dead; thread 0 decides whether there is another one
+    if (tid == 0) more_sh = walk.done() ? 0 : 1;
+    __syncthreads();
+    if (!more_sh) break;
     }
 }
 
 template <int G, int KB, int VB>
-cudaError_t launch_one(const MmaArgs &a, cudaStream_t stream)
+cudaError_t launch_one(const MmaArgs &a, cudaStream_t stream, bool overlap)
 {
     using C = Cfg<G, KB, VB>;
     static bool configured = false;
@@ -442,16 +462,14 @@ cudaError_t launch_one(const MmaArgs &a, cudaStream_t stream)
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    dim3 grid(a.plan.n_splits, a.s.Hkv, a.s.B);
-    kern<<<grid, kThreads, C::kSmemBytes, stream>>>(a);
-    return cudaGetLastError();
+    return launch_dependent(kern, dim3(a.plan.n_slots), dim3(kThreads), C::kSmemBytes, stream, overlap, a);
 }
 
 template <int G>
-cudaError_t launch_g(const MmaArgs &a, cudaStream_t stream)
+cudaError_t launch_g(const MmaArgs &a, cudaStream_t stream, bool overlap)
 {
-    if (a.s.k_bits == 2) return a.s.v_bits == 2 ? launch_one<G, 2, 2>(a, stream) : launch_one<G, 2, 4>(a, stream);
-    return a.s.v_bits == 2 ? launch_one<G, 4, 2>(a, stream) : launch_one<G, 4, 4>(a, stream);
+    if (a.s.k_bits == 2) return a.s.v_bits == 2 ? launch_one<G, 2, 2>(a, stream, overlap) : launch_one<G, 2, 4>(a, stream, overlap);
+    return a.s.v_bits == 2 ? launch_one<G, 4, 2>(a, stream, overlap) : launch_one<G, 4, 4>(a, stream, overlap);
 }
 
 }  // namespace
@@ -459,13 +477,13 @@ cudaError_t launch_g(const MmaArgs &a, cudaStream_t stream)
 // Launches the integer kernel when the configuration is covered (one query head per KV head, G = 64 or 128);
 // *handled tells the caller whether it did.
 cudaError_t launch_partition_mma(const Shape &s, const CachePtrs &c, const __half *q, float scale_log2,
-                                 const SplitPlan &plan, float *workspace, cudaStream_t stream, bool *handled)
+                                 const SplitPlan &plan, float *workspace, cudaStream_t stream, bool overlap, bool *handled)
 {
     *handled = false;
     if (s.rep != 1 || (s.G != 64 && s.G != 128)) return cudaSuccess;
     MmaArgs a{s, c, q, scale_log2, plan, workspace};
     *handled = true;
-    return s.G == 128 ? launch_g<128>(a, stream) : launch_g<64>(a, stream);
+    return s.G == 128 ? launch_g<128>(a, stream, overlap) : launch_g<64>(a, stream, overlap);
 }
 
 }  // namespace skvq

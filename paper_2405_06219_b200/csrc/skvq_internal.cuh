@@ -30,13 +30,79 @@ struct CachePtrs {
     int32_t *status;
 };
 
+// Flat partition of the quantized prefixes.  The unit is 256 tokens of one (sequence, KV head); all units of a
+// call are laid end to end, ordered by (sequence, KV head, position), and cut into n_slots equal runs, one
+// per CTA of the partition kernel.  A run may cross into the next KV head or sequence: each piece is a segment
+// with its own partial.  Every CTA therefore does the same amount of work whatever the batch shape is.
+constexpr int kUnitTok = 256;
+constexpr int kPlanHdrInts = 4;    // workspace header: [0] total units, [1] units per slot, then the prefix array [B+1]
+                                   // and the first sequence of every slot [n_slots]
+
 struct SplitPlan {
-    int split_len;   // quantized tokens per split (multiple of SKVQ_TOKEN_ALIGN)
-    int n_splits;    // splits of the quantized prefix per (sequence, KV head); the fp16 window belongs to the merge kernel
+    int n_slots;     // CTAs of the partition kernel
+    int s_max;       // partial slots per (sequence, query head) in the workspace
+    int hdr_ints;    // ints in front of the partials: header + prefix [B+1] + first sequence per slot [n_slots], padded to 64
+    int lq_cap;      // quantized tokens per sequence the call looks at (from max_len_hint)
 };
 
-// Chooses the sequence partition for lengths up to max_len (host).
+// Chooses the partition for lengths up to max_len (host).  requested_splits > 0 asks for about that many
+// pieces per (sequence, KV head).
 SplitPlan plan_splits(const Shape &s, int max_len, int requested_splits);
+
+struct Segment {
+    int b, hk;                 // sequence, KV head
+    int tok_begin, tok_end;    // quantized tokens of that pair this segment covers
+    int part;                  // index of its partial among the pair's partials
+};
+
+#ifdef __CUDACC__
+// One thread walks the segments of slot w.  hdr is the workspace header written by the plan kernel.
+struct SlotWalker {
+    const int *pre;     // units (per KV head) of the sequences before b, [B+1]
+    int Hkv, B, ups;    // ups = units per slot
+    int f, f1, b, w;
+
+    __device__ bool start(const int *hdr, int B_, int Hkv_, int w_)
+    {
+        pre = hdr + kPlanHdrInts; Hkv = Hkv_; B = B_; w = w_;
+        const int total = hdr[0];
+        ups = hdr[1];
+        b = pre[B + 1 + w];                 // first sequence of this slot, found by the plan kernel
+        f = w * ups;
+        f1 = min(f + ups, total);
+        return f < f1;
+    }
+    __device__ bool done() const { return f >= f1; }
+    // The next segment; lq_b = quantized tokens of sequence b that the call looks at.
+    __device__ Segment next(const int32_t *lengths, int W, int lq_cap)
+    {
+        while (pre[b + 1] == pre[b]) ++b;   // sequences without quantized tokens own no unit
+        const int nu = pre[b + 1] - pre[b];
+        const int base = Hkv * pre[b];
+        const int hk = (f - base) / nu, u0 = (f - base) - hk * nu;
+        const int take = min(nu - u0, f1 - f);
+        const int lq = min(max(lengths[b] - W, 0), lq_cap);
+        Segment sg;
+        sg.b = b; sg.hk = hk;
+        sg.tok_begin = u0 * kUnitTok;
+        sg.tok_end = min((u0 + take) * kUnitTok, lq);
+        sg.part = w - (base + hk * nu) / ups;
+        f += take;
+        if (f == base + Hkv * nu) ++b;
+        return sg;
+    }
+};
+
+// Number of partials of pair (b, hk) and the slot that wrote the first one (merge kernel).
+__device__ inline int pair_partials(const int *hdr, int Hkv, int b, int hk)
+{
+    const int *pre = hdr + kPlanHdrInts;
+    const int nu = pre[b + 1] - pre[b];
+    if (nu == 0) return 0;
+    const int start = Hkv * pre[b] + hk * nu, ups = hdr[1];
+    return (start + nu - 1) / ups - start / ups + 1;
+}
+#endif
 
 // Kernel launchers (host).  Each returns a cudaError_t from the launch and bumps the launch counter.
 cudaError_t launch_append(const Shape &s, const CachePtrs &c, const __half *k, const __half *v,
@@ -46,10 +112,10 @@ cudaError_t launch_attention(const Shape &s, const CachePtrs &c, const __half *q
                              cudaStream_t stream);
 
 cudaError_t launch_partition_mma(const Shape &s, const CachePtrs &c, const __half *q, float scale_log2,
-                                 const SplitPlan &plan, float *workspace, cudaStream_t stream, bool *handled);
+                                 const SplitPlan &plan, float *workspace, cudaStream_t stream, bool overlap, bool *handled);
 
 cudaError_t launch_partition_gqa(const Shape &s, const CachePtrs &c, const __half *q, float scale_log2,
-                                 const SplitPlan &plan, float *workspace, cudaStream_t stream, bool *handled);
+                                 const SplitPlan &plan, float *workspace, cudaStream_t stream, bool overlap, bool *handled);
 
 void count_launch(int n = 1);
 

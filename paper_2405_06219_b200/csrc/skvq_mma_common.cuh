@@ -116,5 +116,24 @@ __device__ __forceinline__ float warp_sum(float v)
     return v;
 }
 
+// A launch that may start before the kernel in front of it on the stream has finished; the kernel itself waits
+// (griddepcontrol.wait) where it first needs that kernel's results.
+template <typename Kern>
+inline cudaError_t launch_dependent(Kern kern, dim3 grid, dim3 block, size_t smem_bytes, cudaStream_t stream, bool overlap,
+                                    const MmaArgs &args)
+{
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = grid;
+    lc.blockDim = block;
+    lc.dynamicSmemBytes = smem_bytes;
+    lc.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = overlap ? 1 : 0;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    return cudaLaunchKernelEx(&lc, kern, args);
+}
+
 }  // namespace mmak
 }  // namespace skvq
