@@ -132,6 +132,7 @@ __device__ __forceinline__ void quantize16(const float (&x)[16], float alpha, in
 
 __global__ void __launch_bounds__(kAppendThreads) append_kernel(AppendArgs a)
 {
+    asm volatile("griddepcontrol.launch_dependents;");      // the bookkeeping kernel may be launched; it waits for this grid
     const Shape &s = a.s;
     const int b = blockIdx.z, h = blockIdx.y;
     const int W = s.W;
@@ -326,6 +327,8 @@ __global__ void __launch_bounds__(kAppendThreads) append_bulk_kernel(AppendArgs 
 // lengths[b] += n_b, or flag an overflow and leave the sequence alone.
 __global__ void append_bookkeeping_kernel(AppendArgs a)
 {
+    asm volatile("griddepcontrol.launch_dependents;");
+    asm volatile("griddepcontrol.wait;" ::: "memory");      // every append CTA has read the old lengths
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= a.s.B) return;
     const int n_b = seq_new_count(a, b);
@@ -362,7 +365,20 @@ cudaError_t launch_append(const Shape &s, const CachePtrs &c, const __half *k, c
     append_kernel<<<grid, kAppendThreads, 0, stream>>>(a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    append_bookkeeping_kernel<<<(s.B + 127) / 128, 128, 0, stream>>>(a);
+    {
+        // launched while append_kernel still runs (it waits for that grid before it touches the lengths)
+        cudaLaunchConfig_t lc = {};
+        lc.gridDim = dim3((s.B + 127) / 128);
+        lc.blockDim = dim3(128);
+        lc.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        lc.attrs = attr;
+        lc.numAttrs = 1;
+        e = cudaLaunchKernelEx(&lc, append_bookkeeping_kernel, a);
+        if (e != cudaSuccess) return e;
+    }
     count_launch(launched + 2);
     return cudaGetLastError();
 }

@@ -51,12 +51,19 @@ __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int rep = s.rep, G = s.G, ng = s.ng;
     asm volatile("griddepcontrol.launch_dependents;");      // the merge kernel may start its window part early
-    asm volatile("griddepcontrol.wait;" ::: "memory");      // the plan kernel's header
+    asm volatile("griddepcontrol.wait;" ::: "memory");      // the lengths, and the plan kernel's header when there is one
 
-    __shared__ Segment seg_sh;
+    __shared__ __align__(16) Segment seg_sh;
     __shared__ int more_sh;
     __shared__ SlotWalker walk;      // only thread 0 touches it; shared memory keeps it out of everybody's registers
-    if (tid == 0) more_sh = walk.start(reinterpret_cast<const int *>(a.ws), s.B, s.Hkv, blockIdx.x) ? 1 : 0;
+    __shared__ __align__(16) int hdr_sh[kPlanSmemInts];
+    if (a.plan.in_kernel) {
+        if (warp == 0) plan_in_warp(a.c.lengths, s.B, s.Hkv, s.W, a.plan.lq_cap, a.plan.n_slots, hdr_sh);
+        __syncthreads();
+    }
+    if (tid == 0)
+        more_sh = walk.start(a.plan.in_kernel ? hdr_sh : reinterpret_cast<const int *>(a.ws), !a.plan.in_kernel, s.B, s.Hkv,
+                             blockIdx.x) ? 1 : 0;
     __syncthreads();
     if (!more_sh) return;
     float *partials = a.ws + a.plan.hdr_ints;
@@ -213,6 +220,7 @@ __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
 __global__ void plan_kernel(AttnArgs a)
 {
     asm volatile("griddepcontrol.launch_dependents;");      // the partition kernel may start its launch now; it waits for this grid
+    asm volatile("griddepcontrol.wait;" ::: "memory");      // whatever wrote the lengths (the append kernels, typically)
     int *hdr = reinterpret_cast<int *>(a.ws);
     int *pre = hdr + kPlanHdrInts;
     const int lane = threadIdx.x & 31;
@@ -268,6 +276,9 @@ __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
     __shared__ float sq[kHeadDim];
     __shared__ float sp[kThreads];
     __shared__ float sred[kThreads / 32];
+    __shared__ __align__(16) int hdr_sh[kPlanSmemInts];
+    if (a.plan.in_kernel && warp == 0)      // the same header the partition CTAs derived; published by the barriers below
+        plan_in_warp(a.c.lengths, s.B, s.Hkv, s.W, a.plan.lq_cap, a.plan.n_slots, hdr_sh);
     const size_t bh = (size_t)b * s.Hkv + hk;
     sq[tid] = __half2float(a.q[((size_t)b * s.Hq + hq) * kHeadDim + (a.c.reorder_k[(size_t)hk * kHeadDim + tid] & (kHeadDim - 1))]) *
               a.scale_log2;
@@ -275,7 +286,7 @@ __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
     const __half *k_win = a.c.k_win + bh * (size_t)W * kHeadDim;
     const __half *v_win = a.c.v_win + bh * (size_t)W * kHeadDim;
     // P.V layout: a warp instruction reads two rows (16 lanes x 8 channels each); warp w takes row pairs w, w+4, ...
-    __shared__ float sacc[kThreads / 32][kHeadDim];
+    __shared__ __align__(16) float sacc[kThreads / 32][kHeadDim];      // written with 16-byte stores
     float m_run = -CUDART_INF_F, l_thread = 0.f;
     float a8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
     const int vsub = lane >> 4, vchunk = lane & 15;
@@ -283,11 +294,29 @@ __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
         const int t = tile0 + tid;
         const bool valid = t < L;
         float sc = valid ? 0.f : -CUDART_INF_F;
+        uint4 vu[kThreads / 8];
+        if (!valid) {
+#pragma unroll
+            for (int i = 0; i < kThreads / 8; ++i) {
+                const int tt = 8 * i + 2 * warp + vsub;
+                vu[i] = make_uint4(0u, 0u, 0u, 0u);
+                if (tile0 + tt < L)
+                    vu[i] = __ldg(reinterpret_cast<const uint4 *>(v_win + (size_t)((tile0 + tt) % W) * kHeadDim) + vchunk);
+            }
+        }
         if (valid) {
             const uint4 *row = reinterpret_cast<const uint4 *>(k_win + (size_t)(t % W) * kHeadDim);
             uint4 u[kHeadDim / 8];
 #pragma unroll
             for (int j8 = 0; j8 < kHeadDim / 8; ++j8) u[j8] = __ldg(row + j8);      // all 16 loads in flight
+            // the value rows this thread will need do not depend on the scores: fetch them behind the key rows
+#pragma unroll
+            for (int i = 0; i < kThreads / 8; ++i) {
+                const int tt = 8 * i + 2 * warp + vsub;
+                vu[i] = make_uint4(0u, 0u, 0u, 0u);
+                if (tile0 + tt < L)
+                    vu[i] = __ldg(reinterpret_cast<const uint4 *>(v_win + (size_t)((tile0 + tt) % W) * kHeadDim) + vchunk);
+            }
 #pragma unroll
             for (int j8 = 0; j8 < kHeadDim / 8; ++j8) {
                 const __half2 *h2 = reinterpret_cast<const __half2 *>(&u[j8]);
@@ -318,8 +347,7 @@ __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
         for (int i = 0; i < kThreads / 8; ++i) {            // 16 independent 16-byte loads per thread
             const int tt = 8 * i + 2 * warp + vsub;
             if (tt < n_tok) {
-                const uint4 u = __ldg(reinterpret_cast<const uint4 *>(v_win + (size_t)((tile0 + tt) % W) * kHeadDim) + vchunk);
-                const __half2 *h2 = reinterpret_cast<const __half2 *>(&u);
+                const __half2 *h2 = reinterpret_cast<const __half2 *>(&vu[i]);
                 const float pt = sp[tt];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
@@ -348,7 +376,7 @@ __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
     // (a no-op unless this kernel was launched with programmatic stream serialization).
     asm volatile("griddepcontrol.wait;" ::: "memory");
     // log-sum-exp merge: the window and the S split partials; thread d owns reordered channel d
-    const int S = pair_partials(reinterpret_cast<const int *>(a.ws), s.Hkv, b, hk);
+    const int S = pair_partials(a.plan.in_kernel ? hdr_sh : reinterpret_cast<const int *>(a.ws), s.Hkv, b, hk);
     const float *part = a.ws + a.plan.hdr_ints + ((size_t)b * s.Hq + hq) * a.plan.s_max * kPartialStride;
     float M = m_run;
     for (int i = 0; i < S; ++i) M = fmaxf(M, part[(size_t)i * kPartialStride + kHeadDim]);
@@ -417,7 +445,8 @@ SplitPlan plan_splits(const Shape &s, int max_len, int requested_splits)
     long s_max = n / s.Hkv + 2;
     if (s_max > units) s_max = units > 0 ? units : 1;
     p.s_max = (int)s_max;
-    p.hdr_ints = (kPlanHdrInts + s.B + 1 + p.n_slots + 63) / 64 * 64;
+    p.in_kernel = s.B <= 32 ? 1 : 0;
+    p.hdr_ints = p.in_kernel ? 0 : (kPlanHdrInts + s.B + 1 + p.n_slots + 63) / 64 * 64;
     return p;
 }
 
@@ -445,9 +474,11 @@ cudaError_t launch_attention(const Shape &s, const CachePtrs &c, const __half *q
                              cudaStream_t stream)
 {
     AttnArgs a{s, c, q, out, sm_scale * 1.4426950408889634f, plan, workspace};
-    plan_kernel<<<1, 256, 0, stream>>>(a);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
+    cudaError_t e = cudaSuccess;
+    if (!plan.in_kernel) {
+        e = launch_dependent(plan_kernel, dim3(1), dim3(256), 0, stream, true, a);
+        if (e != cudaSuccess) return e;
+    }
     if (ev_begin) cudaEventRecord(ev_begin, stream);
     const bool overlap = !ev_begin;      // an event between two kernels serialises them anyway
     dim3 grid(plan.n_slots);
@@ -469,7 +500,7 @@ cudaError_t launch_attention(const Shape &s, const CachePtrs &c, const __half *q
     // wait before they read the partials
     e = launch_dependent(merge_kernel, dim3(s.Hq, s.B), dim3(kHeadDim), 0, stream, !ev_end, a);
     if (e != cudaSuccess) return e;
-    count_launch(3);
+    count_launch(plan.in_kernel ? 2 : 3);
     return cudaGetLastError();
 }
 

@@ -137,12 +137,19 @@ __global__ void __launch_bounds__(kThreads, SKVQ_GQA_CTAS) partition_gqa_kernel(
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t = lane & 3;
     asm volatile("griddepcontrol.launch_dependents;");      // the merge kernel may start its window part early
-    asm volatile("griddepcontrol.wait;" ::: "memory");      // the plan kernel's header
+    asm volatile("griddepcontrol.wait;" ::: "memory");      // the lengths, and the plan kernel's header when there is one
 
-    __shared__ Segment seg_sh;
+    __shared__ __align__(16) Segment seg_sh;
     __shared__ int more_sh;
     __shared__ SlotWalker walk;      // only thread 0 touches it; shared memory keeps it out of everybody's registers
-    if (tid == 0) more_sh = walk.start(reinterpret_cast<const int *>(a.ws), s.B, s.Hkv, blockIdx.x) ? 1 : 0;
+    __shared__ __align__(16) int hdr_sh[kPlanSmemInts];
+    if (a.plan.in_kernel) {
+        if (warp == 0) plan_in_warp(a.c.lengths, s.B, s.Hkv, s.W, a.plan.lq_cap, a.plan.n_slots, hdr_sh);
+        __syncthreads();
+    }
+    if (tid == 0)
+        more_sh = walk.start(a.plan.in_kernel ? hdr_sh : reinterpret_cast<const int *>(a.ws), !a.plan.in_kernel, s.B, s.Hkv,
+                             blockIdx.x) ? 1 : 0;
     __syncthreads();
     if (!more_sh) return;
     float *partials = a.ws + a.plan.hdr_ints;

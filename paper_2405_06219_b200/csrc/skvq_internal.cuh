@@ -43,7 +43,9 @@ struct SplitPlan {
     int s_max;       // partial slots per (sequence, query head) in the workspace
     int hdr_ints;    // ints in front of the partials: header + prefix [B+1] + first sequence per slot [n_slots], padded to 64
     int lq_cap;      // quantized tokens per sequence the call looks at (from max_len_hint)
+    int in_kernel;   // batch <= 32: every CTA derives the header itself from the lengths (one warp scan), no plan kernel
 };
+constexpr int kPlanSmemInts = 40;   // header (4) + prefix [33] of a batch of up to 32 in shared memory, padded
 
 // Chooses the partition for lengths up to max_len (host).  requested_splits > 0 asks for about that many
 // pieces per (sequence, KV head).
@@ -62,15 +64,27 @@ struct SlotWalker {
     int Hkv, B, ups;    // ups = units per slot
     int f, f1, b, w;
 
-    __device__ bool start(const int *hdr, int B_, int Hkv_, int w_)
+    // hdr: the header in the workspace (with the per-slot table behind the prefix) or a copy made by plan_in_warp
+    // (no table: the first sequence is found by bisection).
+    __device__ bool start(const int *hdr, bool has_table, int B_, int Hkv_, int w_)
     {
         pre = hdr + kPlanHdrInts; Hkv = Hkv_; B = B_; w = w_;
         const int total = hdr[0];
         ups = hdr[1];
-        b = pre[B + 1 + w];                 // first sequence of this slot, found by the plan kernel
         f = w * ups;
         f1 = min(f + ups, total);
-        return f < f1;
+        if (f >= f1) return false;
+        if (has_table) {
+            b = pre[B + 1 + w];             // found by the plan kernel
+        } else {
+            int lo = 0, hi = B - 1;         // the largest b with Hkv * pre[b] <= f
+            while (lo < hi) {
+                const int mid = (lo + hi + 1) >> 1;
+                if (Hkv * pre[mid] <= f) lo = mid; else hi = mid - 1;
+            }
+            b = lo;
+        }
+        return true;
     }
     __device__ bool done() const { return f >= f1; }
     // The next segment; lq_b = quantized tokens of sequence b that the call looks at.
@@ -92,6 +106,29 @@ struct SlotWalker {
         return sg;
     }
 };
+
+// The header for a batch of at most 32 sequences, computed by one full warp into hdr_s[kPlanSmemInts]: units per
+// sequence (256 quantized tokens each) as an exclusive prefix, their total over all KV heads, units per slot.
+__device__ inline void plan_in_warp(const int32_t *lengths, int B, int Hkv, int W, int lq_cap, int n_slots, int *hdr_s)
+{
+    const int lane = threadIdx.x & 31;
+    int nu = 0;
+    if (lane < B) nu = (min(max(lengths[lane] - W, 0), lq_cap) + kUnitTok - 1) / kUnitTok;
+    int incl = nu;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += v;
+    }
+    hdr_s[kPlanHdrInts + lane] = incl - nu;
+    const int run = __shfl_sync(0xffffffffu, incl, 31);
+    if (lane == 0) {
+        const int total = run * Hkv;
+        hdr_s[kPlanHdrInts + 32] = run;     // also pre[B] when B == 32; for B < 32 pre[B] = incl - nu of lane B = run already
+        hdr_s[0] = total;
+        hdr_s[1] = max((total + n_slots - 1) / n_slots, 1);
+    }
+}
 
 // Number of partials of pair (b, hk) and the slot that wrote the first one (merge kernel).
 __device__ inline int pair_partials(const int *hdr, int Hkv, int b, int hk)

@@ -71,23 +71,24 @@ def test_sizes_follow_the_documented_layout(lib):
 
 
 def test_workspace_size_grows_with_splits(lib):
-    """Workspace = header (4 ints + prefix [B+1] + first sequence per slot [n_slots], padded to 64 ints) +
-    [B][Hq][s_max] partials of 132 floats, where the flat partition has n_slots = n_splits * B * Hkv slots and a
-    pair can spread over at most n_slots // Hkv + 2 of them (and never over more than its 256-token units)."""
-    c = cfg()                                                 # B 2, Hq 8, Hkv 2, W 128
-
-    def expect(n_splits, hint):
+    """Workspace = [B][Hq][s_max] partials of 132 floats, where the flat partition has n_slots = n_splits * B * Hkv
+    slots and a pair can spread over at most n_slots // Hkv + 2 of them (never over more than its 256-token
+    units); batches above 32 put a header in front: 4 ints + prefix [B+1] + first sequence per slot [n_slots],
+    padded to 64 ints."""
+    def expect(batch, n_splits, hint):
         units = max(-(-(hint - 128) // 256), 1)
-        n_slots = min(n_splits * 2 * 2, units * 2 * 2)
+        n_slots = min(n_splits * batch * 2, units * batch * 2)
         s_max = min(n_slots // 2 + 2, units)
-        hdr = (4 + 2 + 1 + n_slots + 63) // 64 * 64
-        return (hdr + 2 * 8 * s_max * 132) * 4
+        hdr = 0 if batch <= 32 else (4 + batch + 1 + n_slots + 63) // 64 * 64
+        return (hdr + batch * 8 * s_max * 132) * 4
 
+    c = cfg()                                                 # B 2, Hq 8, Hkv 2, W 128
     one = B.skvq_workspace_size(c, 4096, 1)
     four = B.skvq_workspace_size(c, 4096, 4)
-    assert one == expect(1, 4096) and four == expect(4, 4096) and four > one
-    assert B.skvq_workspace_size(c, 4096, 1000) == expect(1000, 4096)      # capped by the units that exist
-    assert B.skvq_workspace_size(c, 300, 7) == expect(7, 300)
+    assert one == expect(2, 1, 4096) and four == expect(2, 4, 4096) and four > one
+    assert B.skvq_workspace_size(c, 4096, 1000) == expect(2, 1000, 4096)      # capped by the units that exist
+    assert B.skvq_workspace_size(c, 300, 7) == expect(2, 7, 300)
+    assert B.skvq_workspace_size(cfg(batch=40), 4096, 3) == expect(40, 3, 4096)
     assert B.skvq_workspace_size(c, 4096, 0) >= one
     assert B.skvq_workspace_size(cfg(head_dim=64), 4096, 0) == 0
     assert B.skvq_step_staging_size(c) == 2 * (2 * 2 * 128 * 2) + 2 * (2 * 8 * 128 * 2)
