@@ -36,9 +36,9 @@ METRIC = "decode_attention_context_tokens_per_s"
 UNIT = "tokens/s"
 PREFILL_CHUNK = 32768
 L2_BYTES = 126 * 1024 * 1024
-# DRAM bytes (read + write) per launch of the partition kernel from an ncu capture, keyed by
-# configuration; None until a capture exists for the current kernel.
-NCU_TRAFFIC_BYTES = {}
+# DRAM bytes (read + write) per launch of the partition kernel from ncu captures, keyed by configuration;
+# absent (None) where no capture exists for the current kernel.
+NCU_TRAFFIC_BYTES = {1: 617.3e6, 2: 410.1e6, 4: 2550.2e6}      # reduced-batch ncu captures scaled by tokens streamed
 
 
 def measured_peak():
@@ -171,38 +171,45 @@ def oracle_sample(w, n_seq, n_kv=None):
 
 def time_oracle(w, steps, warmup, budget_s):
     """Decode steps (append one token + attention) of the oracle, as it stands, on a bounded sample of
-    the workload: sequence 0 at full context and as many KV heads (with their query heads) as keep
-    the run within budget_s.  Tokens are pro-rated by the share of the batch's heads processed."""
+    the workload: the first sequences at full context (all KV heads), or, when one sequence alone is too
+    much, sequence 0 with its first KV heads, sized so that the timed steps take about budget_s of CPU
+    time.  Tokens are the context tokens of the (sequence, head) units actually processed, expressed in
+    whole-workload terms (a unit counts for 1 / Hkv of its sequence's tokens)."""
     from oracle import skvq_oracle as orc
     rep = w.n_q_heads // w.n_kv_heads
-    # calibrate on one KV head
+    lengths = w.lengths()
+    # calibrate on one KV head of sequence 0
     oc = oracle_sample(w, 1, 1)
     q = w.query(0)[:1, :rep]
     t0 = time.perf_counter()
     oc.attention(q, w.sm_scale)
-    per_head = max(time.perf_counter() - t0, 1e-4)
+    per_unit = max(time.perf_counter() - t0, 1e-4) * float(lengths.mean()) / float(lengths[0])
     threads = orc.num_threads()
-    per_step_budget = budget_s / max(steps + warmup, 1)
-    n_kv = int(max(1, min(w.n_kv_heads, (per_step_budget / per_head) * min(threads, w.n_kv_heads * rep) // 1)))
-    oc = oracle_sample(w, 1, n_kv)
-    share = n_kv / float(w.n_kv_heads * w.batch)
+    per_step_budget = budget_s / max(steps, 1)
+    units = max(1, int(per_step_budget / per_unit * min(threads, w.n_kv_heads * rep)))
+    if units >= w.n_kv_heads:
+        n_seq, n_kv = int(min(w.batch, units // w.n_kv_heads)), w.n_kv_heads
+    else:
+        n_seq, n_kv = 1, units
+    oc = oracle_sample(w, n_seq, n_kv)
     times, tokens = [], 0.0
     for s in range(warmup + steps):
-        kn = np.ascontiguousarray(w.new_token("k", s)[:1, :, :n_kv])
-        vn = np.ascontiguousarray(w.new_token("v", s)[:1, :, :n_kv])
-        q = np.ascontiguousarray(w.query(s)[:1, :n_kv * rep])
+        kn = np.ascontiguousarray(w.new_token("k", s)[:n_seq, :, :n_kv])
+        vn = np.ascontiguousarray(w.new_token("v", s)[:n_seq, :, :n_kv])
+        q = np.ascontiguousarray(w.query(s)[:n_seq, :n_kv * rep])
         t0 = time.perf_counter()
         oc.append(kn, vn)
         oc.attention(q, w.sm_scale)
         dt = time.perf_counter() - t0
         if s >= warmup:
             times.append(dt)
-            tokens += float(w.lengths().sum() + w.batch * (s + 1)) * share
+            tokens += float(lengths[:n_seq].sum() + n_seq * (s + 1)) * n_kv / float(w.n_kv_heads)
     total = sum(times)
     return {"value": tokens / total, "unit": UNIT, "cores": threads, "kind": "oracle",
-            "sample": f"sequence 0 of {w.batch}, full context, KV heads 0..{n_kv - 1} of {w.n_kv_heads} with their "
-                      f"query heads, {steps} decode steps (append one token + attention), {total:.2f} s of CPU "
-                      f"time; tokens pro-rated by the share of (sequence, head) units processed"}, total / len(times)
+            "sample": f"sequences 0..{n_seq - 1} of {w.batch} at full context, KV heads 0..{n_kv - 1} of {w.n_kv_heads} "
+                      f"with their query heads, {steps} decode steps (append one token + attention), {total:.2f} s "
+                      f"of CPU time; a (sequence, KV head) unit counts for 1/{w.n_kv_heads} of its sequence's tokens"}, \
+        total / len(times)
 
 
 def run_reference(args, w, rank):
@@ -424,7 +431,7 @@ def main():
                      "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
                      "frac_of_nominal_8000": achieved / 8000.0,
                      "algorithmic_bytes_per_launch": part_bytes, "kernel_ms_avg": kavg_ms,
-                     "kernel_ms_min": min(kern_ms), "traffic": NCU_TRAFFIC_BYTES.get(args.config),
+                     "kernel_ms_min": min(kern_ms), "traffic": NCU_TRAFFIC_BYTES.get(args.config) if not (args.batch or args.context) else None,
                      "whole_call": {"what": "partition + merge kernels, all algorithmic bytes (codes, scale/zero, "
                                             "fp16 window, q, out)", "algorithmic_bytes": alg_bytes, "ms_avg": cavg_ms,
                                     "achieved": alg_bytes / (cavg_ms * 1e-3) / 1e9,

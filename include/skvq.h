@@ -15,6 +15,10 @@
  *     is launched.  Conditions only the device can see (a sequence that would
  *     exceed its capacity) leave that sequence untouched and OR a bit into
  *     skvq_cache::status.
+ *   - Kernels of one call, and of consecutive calls on a stream, are chained with programmatic
+ *     dependent launches: a kernel may be scheduled while its predecessor on the stream drains
+ *     and waits on the device before it touches that predecessor's results.  Nothing changes for
+ *     the caller: stream order is kept.
  *   - Compiled for sm_100a only; there is no CPU path.
  *
  * Notation: B sequences, Hq query heads, Hkv KV heads (Hq % Hkv == 0, query head
@@ -43,6 +47,8 @@ extern "C" {
                                      than SKVQ_NOALLOC_SCRATCH_BYTES */
 
 #define SKVQ_STATUS_OVERFLOW 1    /* bit set in *status when a sequence would have exceeded max_tokens */
+#define SKVQ_STATUS_COPY_TIMEOUT 2 /* bit set when a shared-memory copy inside decode attention never completed (bounded
+                                     wait ran out); the affected tokens contribute nothing to the result */
 
 /* Rows of the quantized segment are allocated in multiples of this many tokens so
  * that a kernel may stage whole tiles; see skvq_quant_capacity(). */
@@ -90,11 +96,13 @@ typedef struct skvq_cache {
 typedef struct skvq_attn_args {
     float sm_scale;         /* softmax scale, e.g. 1/sqrt(D) */
     int32_t max_len_hint;   /* host upper bound on lengths[] (sizes the grid); <= max_tokens */
-    int32_t n_splits;       /* sequence partitions per (sequence, KV head); 0 = library chooses */
+    int32_t n_splits;       /* 0 = library chooses (one CTA per resident slot of the GPU, all with the same share of
+                               the batch's quantized tokens); n > 0 asks for about n pieces per (sequence, KV head) */
     void *workspace;        /* device scratch for the split partials, >= skvq_workspace_size() bytes */
     size_t workspace_bytes;
     void *ev_begin, *ev_end;/* optional cudaEvent_t (else NULL) recorded on the stream immediately
-                               before / after the partition kernel, for profiling */
+                               before / after the partition kernel, for profiling; events keep the merge kernel from
+                               overlapping the partition kernel's tail, so leave them NULL in production */
 } skvq_attn_args;
 
 /* Library version (major*100 + minor). */
@@ -134,7 +142,8 @@ int skvq_quantize_append(const skvq_config *cfg, const skvq_cache *cache, const 
                          const int32_t *n_new_per_seq, int32_t n_new, void *cuda_stream);
 
 /* Scratch bytes skvq_decode_attention needs for lengths up to max_len_hint and the given n_splits
- * (0 = the library's choice for that hint).  0 on a bad cfg. */
+ * (0 = the library's choice for that hint; the choice depends on the GPU's SM count, so ask on the
+ * machine that will run the call).  0 on a bad cfg. */
 size_t skvq_workspace_size(const skvq_config *cfg, int32_t max_len_hint, int32_t n_splits);
 
 /*
@@ -144,6 +153,7 @@ size_t skvq_workspace_size(const skvq_config *cfg, int32_t max_len_hint, int32_t
  *   o'_j = sum_t p_t V~[t][j],  out[reorder_v[j]] = o'_j,
  * where K~/V~ are h*code+z for t < Lq_b and the ring value for Lq_b <= t < L_b.  Dequantization
  * happens in registers; no dequantized cache is written.  A sequence of length 0 yields zeros.
+ * Tokens beyond max_len_hint (a sequence longer than the hint) are not looked at.
  *   q    half [B][Hq][D]      out  half [B][Hq][D]
  * The workspace contents are overwritten; calls sharing a workspace must be stream-ordered.
  */

@@ -20,6 +20,7 @@ SKVQ_ERR_CAPACITY, SKVQ_ERR_WORKSPACE, SKVQ_ERR_CUDA = -4, -5, -6
 SKVQ_ERR_SCRATCH_LIMIT = -7
 SKVQ_NOALLOC_SCRATCH_BYTES = 8 << 20
 SKVQ_STATUS_OVERFLOW = 1
+SKVQ_STATUS_COPY_TIMEOUT = 2
 SKVQ_TOKEN_ALIGN = 64
 
 EXPORTS = ["skvq_version", "skvq_strerror", "skvq_launch_count", "skvq_check_config", "skvq_quant_capacity",

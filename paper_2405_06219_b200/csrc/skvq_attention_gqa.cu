@@ -524,7 +524,7 @@ __global__ void __launch_bounds__(kThreads, SKVQ_GQA_CTAS) partition_gqa_kernel(
             const int st = (tiles_done + i2) % C::kStages;
             (void)mbar_wait_bounded(bar0 + 8 * st, ((tiles_done + i2) / C::kStages) & 1u);
         }
-        if (lane == 0 && a.c.status) atomicOr(a.c.status, 2);
+        if (lane == 0 && a.c.status) atomicOr(a.c.status, SKVQ_STATUS_COPY_TIMEOUT);
     }
 
     // ---- per-warp result
