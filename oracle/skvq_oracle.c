@@ -27,7 +27,9 @@
  *
  * Pins (tests/test_oracle_*.py): round-trip error bound, reduction to textbook
  * per-token min-max quantization, closed-form groups, permutation invariance,
- * single-append == bulk-append, brute-force attention, convexity, q = 0 mean.
+ * single-append == bulk-append, brute-force attention, convexity, q = 0 mean,
+ * attention sinks (exact rows, brute force over the three segments, all-sink
+ * case against a library attention).
  * End-to-end accuracy versus the paper's benchmark tables: parity unpinned (the
  * datasets and model weights those tables need are not available).
  */
@@ -187,6 +189,8 @@ typedef struct {
     int32_t *lengths;
     const int32_t *reorder_k, *reorder_v; /* [Hkv][D] */
     const float *alpha_k, *alpha_v;       /* [Hkv][D/G] */
+    int n_sink;                           /* first n_sink positions are never quantized (Sec. 3.2, filter rules) */
+    uint16_t *k_sink, *v_sink;            /* fp16 bits [B][Hkv][n_sink][D], reordered channel order */
 } orc_cache;
 
 static size_t orc_row_index(const orc_cache *c, int b, int h, int t, int rows)
@@ -199,7 +203,11 @@ static size_t orc_row_index(const orc_cache *c, int b, int h, int t, int rows)
  * new tokens of sequence b are concatenated after the L0 tokens already there;
  * every token in [processed, L1 - W) is quantized, where processed =
  * max(0, L0 - W) is what earlier calls already quantized, and the last
- * min(L1, W) tokens are left in full precision in the ring.
+ * min(L1, W) tokens are left in full precision in the ring.  Filter rule
+ * (Sec. 3.2; the mask of Algorithm 1): a token at a position below n_sink
+ * (an attention sink) is not quantized when it leaves the window; its
+ * reordered fp16 row is kept in the sink store, and its quantized row is
+ * never written.
  * k, v: fp16 bits [B][n_stride][Hkv][D] in the model's original channel order.
  * Returns 0, or -1 if a sequence would exceed its capacity (nothing is changed
  * for that sequence).
@@ -232,6 +240,12 @@ int orc_append(orc_cache *c, const uint16_t *k, const uint16_t *v, const int32_t
                     orc_reorder_row(k + s, c->reorder_k + (size_t)h * D, D, rowk);
                     orc_reorder_row(v + s, c->reorder_v + (size_t)h * D, D, rowv);
                 }
+                if (t < c->n_sink) { /* filtered: retained in full precision */
+                    size_t d = orc_row_index(c, b, h, t, c->n_sink) * (size_t)D;
+                    memcpy(c->k_sink + d, rowk, sizeof(uint16_t) * (size_t)D);
+                    memcpy(c->v_sink + d, rowv, sizeof(uint16_t) * (size_t)D);
+                    continue;
+                }
                 size_t r = orc_row_index(c, b, h, t, c->cap_q);
                 orc_quantize_reordered_row(rowk, c->alpha_k + (size_t)h * ng, D, c->G, c->k_bits,
                                            c->k_codes + r * (size_t)(D * c->k_bits / 8),
@@ -260,7 +274,8 @@ int orc_append(orc_cache *c, const uint16_t *k, const uint16_t *v, const int32_t
  * Decode attention for one query per sequence (Eq. 1 and the first lines of
  * Algorithm 1, with the softmax and its scale written out):
  *   q'      = q[reorder_k]                       (same permutation as the keys)
- *   s_t     = sm_scale * sum_j q'_j K~_{t,j}      K~ = h*c+z for t < L-W, fp16 window otherwise
+ *   s_t     = sm_scale * sum_j q'_j K~_{t,j}      K~ = h*c+z for t < L-W (the fp16 sink row where
+ *                                                t < n_sink), fp16 window otherwise
  *   p       = softmax(s) over all t < L
  *   o'_j    = sum_t p_t V~_{t,j}
  *   out[reorder_v[j]] = o'_j                      (undo the value permutation)
@@ -290,7 +305,10 @@ void orc_attention(const orc_cache *c, int Hq, const uint16_t *q, double sm_scal
                 qp[j] = (double)orc_f16_to_f32(q[((size_t)b * Hq + hq) * (size_t)D + ik[j]]);
             /* scores */
             for (int t = 0; t < L; ++t) {
-                if (t < Lq) {
+                if (t < Lq && t < c->n_sink) {
+                    size_t w = orc_row_index(c, b, hk, t, c->n_sink) * (size_t)D;
+                    for (int j = 0; j < D; ++j) row[j] = (double)orc_f16_to_f32(c->k_sink[w + j]);
+                } else if (t < Lq) {
                     size_t r = orc_row_index(c, b, hk, t, c->cap_q);
                     orc_dequant_row(c->k_codes + r * (size_t)(D * c->k_bits / 8),
                                     c->k_meta + r * (size_t)ng * 2, D, c->G, c->k_bits, row);
@@ -309,7 +327,10 @@ void orc_attention(const orc_cache *c, int Hq, const uint16_t *q, double sm_scal
             for (int t = 0; t < L; ++t) { s[t] = exp(s[t] - m); denom += s[t]; }
             /* weighted sum of values */
             for (int t = 0; t < L; ++t) {
-                if (t < Lq) {
+                if (t < Lq && t < c->n_sink) {
+                    size_t w = orc_row_index(c, b, hk, t, c->n_sink) * (size_t)D;
+                    for (int j = 0; j < D; ++j) row[j] = (double)orc_f16_to_f32(c->v_sink[w + j]);
+                } else if (t < Lq) {
                     size_t r = orc_row_index(c, b, hk, t, c->cap_q);
                     orc_dequant_row(c->v_codes + r * (size_t)(D * c->v_bits / 8),
                                     c->v_meta + r * (size_t)ng * 2, D, c->G, c->v_bits, row);

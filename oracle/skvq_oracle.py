@@ -39,6 +39,7 @@ class _Cache(ctypes.Structure):
         ("lengths", ctypes.c_void_p),
         ("reorder_k", ctypes.c_void_p), ("reorder_v", ctypes.c_void_p),
         ("alpha_k", ctypes.c_void_p), ("alpha_v", ctypes.c_void_p),
+        ("n_sink", ctypes.c_int), ("k_sink", ctypes.c_void_p), ("v_sink", ctypes.c_void_p),
     ]
 
 
@@ -117,7 +118,7 @@ class OracleCache:
     """Host-side SKVQ cache in the canonical layout, driven by the C oracle."""
 
     def __init__(self, batch, n_q_heads, n_kv_heads, head_dim, k_bits, v_bits, group_size, window,
-                 max_tokens, reorder_k, reorder_v, alpha_k, alpha_v):
+                 max_tokens, reorder_k, reorder_v, alpha_k, alpha_v, n_sink=0):
         self.B, self.Hq, self.Hkv, self.D = batch, n_q_heads, n_kv_heads, head_dim
         self.k_bits, self.v_bits, self.G, self.W = k_bits, v_bits, group_size, window
         self.ng = head_dim // group_size
@@ -129,6 +130,9 @@ class OracleCache:
         self.v_meta = np.zeros((B, H, self.cap_q, self.ng, 2), dtype=np.float16)
         self.k_win = np.zeros((B, H, W, D), dtype=np.float16)
         self.v_win = np.zeros((B, H, W, D), dtype=np.float16)
+        self.n_sink = int(n_sink)
+        self.k_sink = np.zeros((B, H, max(self.n_sink, 1), D), dtype=np.float16)
+        self.v_sink = np.zeros((B, H, max(self.n_sink, 1), D), dtype=np.float16)
         self.lengths = np.zeros((B,), dtype=np.int32)
         self.reorder_k = np.ascontiguousarray(reorder_k, dtype=np.int32).reshape(H, D)
         self.reorder_v = np.ascontiguousarray(reorder_v, dtype=np.int32).reshape(H, D)
@@ -139,7 +143,8 @@ class OracleCache:
         return _Cache(self.B, self.Hkv, self.D, self.G, self.W, self.cap_q, self.k_bits, self.v_bits,
                       _ptr(self.k_codes), _ptr(self.v_codes), _ptr(self.k_meta), _ptr(self.v_meta),
                       _ptr(self.k_win), _ptr(self.v_win), _ptr(self.lengths),
-                      _ptr(self.reorder_k), _ptr(self.reorder_v), _ptr(self.alpha_k), _ptr(self.alpha_v))
+                      _ptr(self.reorder_k), _ptr(self.reorder_v), _ptr(self.alpha_k), _ptr(self.alpha_v),
+                      self.n_sink, _ptr(self.k_sink), _ptr(self.v_sink))
 
     def append(self, k: np.ndarray, v: np.ndarray, n_new=None) -> int:
         """k, v: float16 [B, n, Hkv, D], original channel order; n_new: per-sequence counts or None."""

@@ -16,7 +16,7 @@ from test_oracle_quantizer import unpack_codes
 D = 128
 
 
-def make_cache(B, Hq, Hkv, W, cap, bits=2, group=128, alpha=0.9, seed=0, identity=False):
+def make_cache(B, Hq, Hkv, W, cap, bits=2, group=128, alpha=0.9, seed=0, identity=False, n_sink=0):
     rng = np.random.default_rng(seed)
     if identity:
         rk = rv = np.tile(np.arange(D, dtype=np.int32), (Hkv, 1))
@@ -24,7 +24,7 @@ def make_cache(B, Hq, Hkv, W, cap, bits=2, group=128, alpha=0.9, seed=0, identit
         rk = np.stack([rng.permutation(D) for _ in range(Hkv)]).astype(np.int32)
         rv = np.stack([rng.permutation(D) for _ in range(Hkv)]).astype(np.int32)
     a = np.full((Hkv, D // group), alpha, np.float32)
-    return orc.OracleCache(B, Hq, Hkv, D, bits, bits, group, W, cap, rk, rv, a, a)
+    return orc.OracleCache(B, Hq, Hkv, D, bits, bits, group, W, cap, rk, rv, a, a, n_sink=n_sink)
 
 
 def rand_kv(B, n, Hkv, seed):
@@ -46,12 +46,15 @@ def mixed_cache_dense(c, b, hk):
     L = int(c.lengths[b])
     Lq = max(L - c.W, 0)
     out = []
-    for codes, meta, win, bits in ((c.k_codes, c.k_meta, c.k_win, c.k_bits), (c.v_codes, c.v_meta, c.v_win, c.v_bits)):
+    for codes, meta, win, sink, bits in ((c.k_codes, c.k_meta, c.k_win, c.k_sink, c.k_bits),
+                                         (c.v_codes, c.v_meta, c.v_win, c.v_sink, c.v_bits)):
         code = unpack_codes(codes[b, hk, :Lq], bits).astype(np.float64)
         h = np.repeat(meta[b, hk, :Lq, :, 0].astype(np.float64), c.G, axis=1)
         z = np.repeat(meta[b, hk, :Lq, :, 1].astype(np.float64), c.G, axis=1)
         dense = np.zeros((L, D))
         dense[:Lq] = h * code + z
+        ns = min(c.n_sink, Lq)                       # attention sinks: full-precision rows, never quantized
+        dense[:ns] = sink[b, hk, :ns].astype(np.float64)
         for t in range(Lq, L):
             dense[t] = win[b, hk, t % c.W].astype(np.float64)
         out.append(dense)
@@ -212,6 +215,71 @@ def test_dominant_key_selects_its_value_row_and_score_shift_is_invisible():
     q[0, 0, 1] = 0.5
     q2[0, 0, 1] = 0.5
     assert np.abs(c2.attention(q, 1.0) - c2.attention(q2, 1.0)).max() < 1e-9
+
+
+# ------------------------------------------------------------------ attention sinks (Sec. 3.2 filter rules)
+@pytest.mark.parametrize("W,n_sink,n", [(8, 5, 40), (8, 5, 10), (8, 5, 4), (0, 3, 20), (16, 20, 30), (8, 64, 200)])
+def test_sinks_keep_exact_rows_and_leave_the_other_tokens_alone(W, n_sink, n):
+    """A position below n_sink that has left the window holds the token's exact fp16 values (reordered); every
+    other token is quantized exactly as in a cache without sinks; chunked appends give the same state."""
+    k, v = rand_kv(2, n, 3, seed=11)
+    c = make_cache(2, 3, 3, W, 256, group=32, n_sink=n_sink, seed=5)
+    ref = make_cache(2, 3, 3, W, 256, group=32, n_sink=0, seed=5)
+    c.append(k, v)
+    ref.append(k, v)
+    lq = max(n - W, 0)
+    ns = min(n_sink, lq)
+    for b in range(2):
+        for h in range(3):
+            assert np.array_equal(c.k_sink[b, h, :ns], k[b, :ns, h][:, c.reorder_k[h]])
+            assert np.array_equal(c.v_sink[b, h, :ns], v[b, :ns, h][:, c.reorder_v[h]])
+    assert np.array_equal(c.k_codes[:, :, ns:lq], ref.k_codes[:, :, ns:lq])
+    assert np.array_equal(c.v_meta.view(np.uint16)[:, :, ns:lq], ref.v_meta.view(np.uint16)[:, :, ns:lq])
+    assert np.array_equal(c.k_win.view(np.uint16), ref.k_win.view(np.uint16))
+    assert not c.k_codes[:, :, :ns].any()            # the quantized rows of the sinks are never written
+    step = make_cache(2, 3, 3, W, 256, group=32, n_sink=n_sink, seed=5)
+    t = 0
+    for m in (1, 3, 7, 2, 11, 1, 1, 64, 200):
+        m = min(m, n - t)
+        if m == 0:
+            break
+        step.append(k[:, t:t + m], v[:, t:t + m])
+        t += m
+    while t < n:
+        step.append(k[:, t:t + 1], v[:, t:t + 1])
+        t += 1
+    assert np.array_equal(step.k_sink[:, :, :ns], c.k_sink[:, :, :ns]) and np.array_equal(step.v_sink[:, :, :ns], c.v_sink[:, :, :ns])
+    assert np.array_equal(step.k_codes[:, :, ns:lq], c.k_codes[:, :, ns:lq])
+    assert np.array_equal(step.lengths, c.lengths)
+
+
+@pytest.mark.parametrize("Hq,Hkv,bits,group,W,n_sink,L", [(4, 2, 2, 32, 16, 5, 150), (2, 2, 4, 64, 8, 3, 9), (2, 1, 2, 128, 0, 4, 33),
+                                                      (2, 2, 2, 32, 16, 5, 12)])
+def test_sink_attention_matches_library_brute_force(Hq, Hkv, bits, group, W, n_sink, L):
+    k, v = rand_kv(1, L, Hkv, seed=21)
+    c = make_cache(1, Hq, Hkv, W, 256, bits=bits, group=group, n_sink=n_sink, seed=8)
+    c.append(k, v)
+    q = np.random.default_rng(3).standard_normal((1, Hq, D)).astype(np.float16)
+    got = c.attention(q, 0.088)
+    assert np.abs(got - brute_attention(c, q, 0.088)).max() < 1e-12
+
+
+def test_all_sinks_and_no_window_is_plain_attention():
+    """n_sink >= L with W = 0: nothing is quantized, so the result is softmax attention over the original K, V
+    (a library routine, fp64), whatever the reorder index."""
+    import torch
+    L, Hq, Hkv = 50, 4, 2
+    k, v = rand_kv(1, L, Hkv, seed=4)
+    c = make_cache(1, Hq, Hkv, 0, 64, group=32, n_sink=64, seed=9)
+    c.append(k, v)
+    q = np.random.default_rng(6).standard_normal((1, Hq, D)).astype(np.float16)
+    got = c.attention(q, 0.088)
+    kt = torch.from_numpy(k.astype(np.float64)).permute(0, 2, 1, 3).repeat_interleave(Hq // Hkv, dim=1)
+    vt = torch.from_numpy(v.astype(np.float64)).permute(0, 2, 1, 3).repeat_interleave(Hq // Hkv, dim=1)
+    qt = torch.from_numpy(q.astype(np.float64))[:, :, None, :]
+    want = torch.nn.functional.scaled_dot_product_attention(qt, kt, vt, scale=float(np.float32(0.088)))[:, :, 0].numpy()
+    assert np.abs(got - want).max() < 1e-12
+    assert not c.k_codes.any() and not c.v_codes.any()
 
 
 def test_empty_sequence_gives_zeros():
