@@ -38,7 +38,7 @@ PREFILL_CHUNK = 32768
 L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes (read + write) per launch of the partition kernel from ncu captures, keyed by configuration;
 # absent (None) where no capture exists for the current kernel.
-NCU_TRAFFIC_BYTES = {1: 617.3e6, 2: 410.1e6, 4: 2550.2e6}      # reduced-batch ncu captures scaled by tokens streamed
+NCU_TRAFFIC_BYTES = {}      # reduced-batch ncu captures scaled by tokens streamed; none yet for the kernels as they stand
 
 
 def measured_peak():
@@ -156,14 +156,14 @@ def oracle_sample(w, n_seq, n_kv=None):
 
     def new(batch):
         return orc.OracleCache(batch, n_kv * rep, n_kv, w.head_dim, w.k_bits, w.v_bits, w.group_size, w.window,
-                               cap, rk, rv, a, a)
+                               cap, rk, rv, a, a, n_sink=w.n_sink)
     oc = new(n_seq)
     for b in range(n_seq):
         one = new(1)
         L = int(lengths[b])
         one.append(np.ascontiguousarray(w.tokens("k", b, 0, L)[None, :, :n_kv]),
                    np.ascontiguousarray(w.tokens("v", b, 0, L)[None, :, :n_kv]))
-        for name in ("k_codes", "v_codes", "k_meta", "v_meta", "k_win", "v_win"):
+        for name in ("k_codes", "v_codes", "k_meta", "v_meta", "k_win", "v_win", "k_sink", "v_sink"):
             getattr(oc, name)[b] = getattr(one, name)[0]
         oc.lengths[b] = L
     return oc
@@ -236,6 +236,8 @@ def main():
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (small profiling cases)")
     ap.add_argument("--context", type=int, default=0, help="override the context length (small profiling cases)")
+    ap.add_argument("--sinks", type=int, default=0,
+                    help="attention sinks: first positions kept fp16 (Sec. 3.2 filter rule; the paper's experiments use 5)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-parity", action="store_true")
     args = ap.parse_args()
@@ -250,6 +252,8 @@ def main():
         w0 = w0.scaled(batch=args.batch)
     if args.context:
         w0 = w0.scaled(context=args.context, ragged=None)
+    if args.sinks:
+        w0 = w0.scaled(n_sink=args.sinks)
 
     if args.impl == "reference":
         run_reference(args, w0, rank)
@@ -282,10 +286,13 @@ def main():
     if not args.no_parity and rank == 0:
         oc = oracle_sample(w, 1)
         lq = max(int(lengths0[0]) - w.window, 0)
-        exact = bool(np.array_equal(cache.k_codes[0, :, :lq].cpu().numpy(), oc.k_codes[0, :, :lq]) and
-                     np.array_equal(cache.v_codes[0, :, :lq].cpu().numpy(), oc.v_codes[0, :, :lq]) and
-                     np.array_equal(cache.k_meta[0, :, :lq].cpu().numpy().view(np.uint16), oc.k_meta.view(np.uint16)[0, :, :lq]) and
-                     np.array_equal(cache.v_meta[0, :, :lq].cpu().numpy().view(np.uint16), oc.v_meta.view(np.uint16)[0, :, :lq]))
+        ns = min(w.n_sink, lq)      # sink rows: fp16 copies instead of codes
+        exact = bool(np.array_equal(cache.k_codes[0, :, ns:lq].cpu().numpy(), oc.k_codes[0, :, ns:lq]) and
+                     np.array_equal(cache.v_codes[0, :, ns:lq].cpu().numpy(), oc.v_codes[0, :, ns:lq]) and
+                     np.array_equal(cache.k_meta[0, :, ns:lq].cpu().numpy().view(np.uint16), oc.k_meta.view(np.uint16)[0, :, ns:lq]) and
+                     np.array_equal(cache.v_meta[0, :, ns:lq].cpu().numpy().view(np.uint16), oc.v_meta.view(np.uint16)[0, :, ns:lq]) and
+                     np.array_equal(cache.k_sink[0, :, :ns].cpu().numpy().view(np.uint16), oc.k_sink.view(np.uint16)[0, :, :ns]) and
+                     np.array_equal(cache.v_sink[0, :, :ns].cpu().numpy().view(np.uint16), oc.v_sink.view(np.uint16)[0, :, :ns]))
         q = w.query(10_000)
         out = cache.attention(torch.from_numpy(q).cuda(), w.sm_scale, hint, n_splits=args.splits)
         torch.cuda.synchronize()
@@ -419,7 +426,7 @@ def main():
         "config": {"workload": f"configs[{args.config}] {w.name}", "batch": w.batch, "n_q_heads": w.n_q_heads,
                    "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "context": int(lengths0.max()),
                    "window": w.window, "k_bits": w.k_bits, "v_bits": w.v_bits, "group_size": w.group_size,
-                   "alpha": w.alpha, "step": "append 1 token/sequence + decode attention",
+                   "alpha": w.alpha, "n_sink": w.n_sink, "step": "append 1 token/sequence + decode attention",
                    "cache_bytes": cache.nbytes(),
                    "l2": "cache larger than L2, streamed every step" if flush is None else "L2 flushed between steps",
                    "parallelism": f"replica per GPU x{world}" if world > 1 else "single GPU"},
@@ -431,7 +438,7 @@ def main():
                      "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
                      "frac_of_nominal_8000": achieved / 8000.0,
                      "algorithmic_bytes_per_launch": part_bytes, "kernel_ms_avg": kavg_ms,
-                     "kernel_ms_min": min(kern_ms), "traffic": NCU_TRAFFIC_BYTES.get(args.config) if not (args.batch or args.context) else None,
+                     "kernel_ms_min": min(kern_ms), "traffic": NCU_TRAFFIC_BYTES.get(args.config) if not (args.batch or args.context or args.sinks) else None,
                      "whole_call": {"what": "partition + merge kernels, all algorithmic bytes (codes, scale/zero, "
                                             "fp16 window, q, out)", "algorithmic_bytes": alg_bytes, "ms_avg": cavg_ms,
                                     "achieved": alg_bytes / (cavg_ms * 1e-3) / 1e9,

@@ -23,8 +23,9 @@
  *
  * Notation: B sequences, Hq query heads, Hkv KV heads (Hq % Hkv == 0, query head
  * hq reads KV head hq / (Hq/Hkv)), D = head_dim, W = window, G = group size,
- * ng = D/G groups per row, L_b = lengths[b], Lq_b = max(L_b - W, 0) quantized
- * tokens of sequence b.
+ * ng = D/G groups per row, L_b = lengths[b], Lq_b = max(L_b - W, 0) tokens of
+ * sequence b that have left the window; of those, positions below n_sink (attention
+ * sinks) stay fp16 and the rest are quantized.
  */
 #ifndef SKVQ_H_
 #define SKVQ_H_
@@ -65,6 +66,8 @@ typedef struct skvq_config {
     int32_t group_size;  /* G: 32, 64 or 128 consecutive (reordered) channels share scale/zero */
     int32_t window;      /* W >= 0 latest tokens kept in fp16 (Sec. 3.2); 0 quantizes everything */
     int32_t max_tokens;  /* per-sequence capacity (quantized segment + window) */
+    int32_t n_sink;      /* 0..64: the first n_sink positions of a sequence are never quantized (Sec. 3.2, filter
+                            rules; the paper's experiments keep 5); 0 = none */
 } skvq_config;
 
 /*
@@ -79,7 +82,9 @@ typedef struct skvq_config {
  *                                                     row must be a permutation of 0..D-1 (Eq. 1)
  *   alpha_k/_v       float   [Hkv][ng]                clip factor per group in (0,1] (Eq. 2)
  *   status           int32   [1]                      optional (may be NULL); SKVQ_STATUS_* bits are OR-ed in
- * Rows at or beyond Lq_b hold unspecified bytes.  The buffers fully describe the state:
+ *   k_sink/v_sink    half    [B][Hkv][n_sink][D]      position t < n_sink once it has left the window, reordered
+ *                                                     order; may be NULL when n_sink == 0
+ * Rows at or beyond Lq_b, and rows below n_sink, of the quantized buffers hold unspecified bytes.  The buffers fully describe the state:
  * copying them is a checkpoint.
  */
 typedef struct skvq_cache {
@@ -90,6 +95,7 @@ typedef struct skvq_cache {
     const int32_t *reorder_k, *reorder_v;
     const float *alpha_k, *alpha_v;
     int32_t *status;
+    void *k_sink, *v_sink;
 } skvq_cache;
 
 /* Options of one decode-attention call (host struct). */
@@ -124,6 +130,9 @@ int32_t skvq_quant_capacity(const skvq_config *cfg);
 /* Bytes of k_codes, v_codes, k_meta, v_meta, k_win, v_win (in that order) for cfg.  Host only. */
 int skvq_cache_sizes(const skvq_config *cfg, size_t bytes_out[6]);
 
+/* Bytes of k_sink (= v_sink) for cfg; 0 when n_sink == 0 or on a bad cfg.  Host only. */
+size_t skvq_sink_bytes(const skvq_config *cfg);
+
 /*
  * Append tokens (Sec. 3.2, Algorithm 1 body, clipping_quant; Eq. 2).
  * Sequence b receives n_b = n_new_per_seq ? n_new_per_seq[b] : n_new tokens (0 <= n_b <= n_new).
@@ -132,6 +141,8 @@ int skvq_cache_sizes(const skvq_config *cfg, size_t bytes_out[6]);
  *   lo = alpha*min, hi = alpha*max, h = fp16((hi-lo)/(2^bits-1)), z = fp16(lo),
  *   code = clamp(rint((x - z)/h), 0, 2^bits-1)   (fp32, IEEE division, ties to even; h == 0 -> code 0)
  * the last min(L1, W) tokens are kept in fp16 in the ring, and lengths[b] becomes L1.
+ * Exception (Sec. 3.2, the filter mask of Algorithm 1): a token at a position below n_sink is copied, reordered,
+ * to k_sink/v_sink when it leaves the window instead of being quantized.
  * One bulk call equals the same tokens appended one at a time.
  *   k, v           half [B][n_new][Hkv][D], original channel order (rows beyond n_b are ignored)
  *   n_new_per_seq  device int32 [B] or NULL
@@ -151,7 +162,7 @@ size_t skvq_workspace_size(const skvq_config *cfg, int32_t max_len_hint, int32_t
  * (Eq. 1 and the first lines of Algorithm 1; softmax and its scale written out):
  *   q' = q[reorder_k],  s_t = sm_scale * sum_j q'_j K~[t][j],  p = softmax_t(s),
  *   o'_j = sum_t p_t V~[t][j],  out[reorder_v[j]] = o'_j,
- * where K~/V~ are h*code+z for t < Lq_b and the ring value for Lq_b <= t < L_b.  Dequantization
+ * where K~/V~ are h*code+z for t < Lq_b (the sink row for t < n_sink) and the ring value for Lq_b <= t < L_b.  Dequantization
  * happens in registers; no dequantized cache is written.  A sequence of length 0 yields zeros.
  * Tokens beyond max_len_hint (a sequence longer than the hint) are not looked at.
  *   q    half [B][Hq][D]      out  half [B][Hq][D]

@@ -24,18 +24,19 @@ SKVQ_STATUS_COPY_TIMEOUT = 2
 SKVQ_TOKEN_ALIGN = 64
 
 EXPORTS = ["skvq_version", "skvq_strerror", "skvq_launch_count", "skvq_check_config", "skvq_quant_capacity",
-           "skvq_cache_sizes", "skvq_quantize_append", "skvq_workspace_size", "skvq_decode_attention",
+           "skvq_cache_sizes", "skvq_sink_bytes", "skvq_quantize_append", "skvq_workspace_size", "skvq_decode_attention",
            "skvq_step_staging_size", "skvq_decode_step_host", "skvq_decode_attention_noalloc"]
 
 
 class SkvqConfig(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in ("batch", "n_q_heads", "n_kv_heads", "head_dim", "k_bits", "v_bits",
-                                              "group_size", "window", "max_tokens")]
+                                              "group_size", "window", "max_tokens", "n_sink")]
 
 
 class SkvqCacheStruct(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in ("k_codes", "v_codes", "k_meta", "v_meta", "k_win", "v_win", "lengths",
-                                               "reorder_k", "reorder_v", "alpha_k", "alpha_v", "status")]
+                                               "reorder_k", "reorder_v", "alpha_k", "alpha_v", "status", "k_sink",
+                                               "v_sink")]
 
 
 class SkvqAttnArgs(ctypes.Structure):
@@ -69,6 +70,8 @@ def lib() -> ctypes.CDLL:
         L.skvq_quant_capacity.argtypes = [P(SkvqConfig)]
         L.skvq_cache_sizes.restype = c_int
         L.skvq_cache_sizes.argtypes = [P(SkvqConfig), P(c_sz)]
+        L.skvq_sink_bytes.restype = c_sz
+        L.skvq_sink_bytes.argtypes = [P(SkvqConfig)]
         L.skvq_quantize_append.restype = c_int
         L.skvq_quantize_append.argtypes = [P(SkvqConfig), P(SkvqCacheStruct), vp, vp, vp, ctypes.c_int32, vp]
         L.skvq_workspace_size.restype = c_sz
@@ -127,6 +130,10 @@ def skvq_cache_sizes(cfg: SkvqConfig) -> list[int]:
     return list(out)
 
 
+def skvq_sink_bytes(cfg: SkvqConfig) -> int:
+    return int(lib().skvq_sink_bytes(ctypes.byref(cfg)))
+
+
 def skvq_workspace_size(cfg: SkvqConfig, max_len_hint: int, n_splits: int = 0) -> int:
     return int(lib().skvq_workspace_size(ctypes.byref(cfg), max_len_hint, n_splits))
 
@@ -167,8 +174,9 @@ class SkvqCache:
     """
 
     def __init__(self, batch, n_q_heads, n_kv_heads, head_dim, k_bits, v_bits, group_size, window, max_tokens,
-                 reorder_k, reorder_v, alpha_k, alpha_v, device="cuda:0"):
-        self.cfg = SkvqConfig(batch, n_q_heads, n_kv_heads, head_dim, k_bits, v_bits, group_size, window, max_tokens)
+                 reorder_k, reorder_v, alpha_k, alpha_v, device="cuda:0", n_sink=0):
+        self.cfg = SkvqConfig(batch, n_q_heads, n_kv_heads, head_dim, k_bits, v_bits, group_size, window, max_tokens,
+                              n_sink)
         _check(skvq_check_config(self.cfg), "skvq_check_config")
         self.device = torch.device(device)
         self.cap = skvq_quant_capacity(self.cfg)
@@ -184,6 +192,9 @@ class SkvqCache:
         self.v_win = torch.zeros((B, H, max(W, 1), D), dtype=torch.float16, device=dev)
         got = [t.numel() * t.element_size() for t in (self.k_codes, self.v_codes, self.k_meta, self.v_meta)]
         assert got == sizes[:4], (got, sizes)
+        self.k_sink = torch.zeros((B, H, max(n_sink, 1), D), dtype=torch.float16, device=dev)
+        self.v_sink = torch.zeros((B, H, max(n_sink, 1), D), dtype=torch.float16, device=dev)
+        assert n_sink == 0 or self.k_sink.numel() * 2 == skvq_sink_bytes(self.cfg)
         self.lengths = torch.zeros((B,), dtype=torch.int32, device=dev)
         self.status = torch.zeros((4,), dtype=torch.int32, device=dev)
         self.reorder_k = torch.as_tensor(reorder_k, dtype=torch.int32).reshape(H, D).contiguous().to(dev)
@@ -192,7 +203,7 @@ class SkvqCache:
         self.alpha_v = torch.as_tensor(alpha_v, dtype=torch.float32).reshape(H, self.ng).contiguous().to(dev)
         self.struct = SkvqCacheStruct(*[t.data_ptr() for t in (
             self.k_codes, self.v_codes, self.k_meta, self.v_meta, self.k_win, self.v_win, self.lengths,
-            self.reorder_k, self.reorder_v, self.alpha_k, self.alpha_v, self.status)])
+            self.reorder_k, self.reorder_v, self.alpha_k, self.alpha_v, self.status, self.k_sink, self.v_sink)])
         self._workspace = None
 
     @classmethod
@@ -200,11 +211,12 @@ class SkvqCache:
         """Cache for a ``workloads.Workload`` with its reorder index and clip factors."""
         mt = w.context if max_tokens is None else max_tokens
         return cls(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.k_bits, w.v_bits, w.group_size, w.window, mt,
-                   w.reorder_index("k"), w.reorder_index("v"), w.alphas(), w.alphas(), device=device)
+                   w.reorder_index("k"), w.reorder_index("v"), w.alphas(), w.alphas(), device=device, n_sink=w.n_sink)
 
     def nbytes(self) -> int:
         return sum(t.numel() * t.element_size() for t in (self.k_codes, self.v_codes, self.k_meta, self.v_meta,
-                                                          self.k_win, self.v_win))
+                                                          self.k_win, self.v_win)) + \
+            (2 * self.k_sink.numel() * 2 if self.cfg.n_sink else 0)
 
     def append(self, k, v, n_new_per_seq=None, stream=None) -> None:
         """k, v: half [B, n, Hkv, D] CUDA tensors; n_new_per_seq: optional int32 [B] CUDA tensor."""

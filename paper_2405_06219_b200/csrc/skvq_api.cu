@@ -19,6 +19,8 @@ static int check_cfg(const skvq_config *c)
     if (c->group_size != 32 && c->group_size != 64 && c->group_size != 128) return SKVQ_ERR_UNSUPPORTED;
     if (c->n_q_heads % c->n_kv_heads != 0) return SKVQ_ERR_UNSUPPORTED;
     if (c->n_q_heads / c->n_kv_heads > kMaxRep) return SKVQ_ERR_UNSUPPORTED;
+    if (c->n_sink < 0) return SKVQ_ERR_INVALID_ARG;
+    if (c->n_sink > 64) return SKVQ_ERR_UNSUPPORTED;
     return SKVQ_OK;
 }
 
@@ -45,6 +47,7 @@ static Shape make_shape(const skvq_config *c)
     s.W = c->window;
     s.cap = quant_capacity(c);
     s.max_tokens = c->max_tokens;
+    s.n_sink = c->n_sink;
     return s;
 }
 
@@ -57,8 +60,9 @@ static int check_cache(const skvq_config *cfg, const skvq_cache *c, CachePtrs *o
         !c->alpha_k || !c->alpha_v)
         return SKVQ_ERR_INVALID_ARG;
     if (cfg->window > 0 && (!c->k_win || !c->v_win)) return SKVQ_ERR_INVALID_ARG;
+    if (cfg->n_sink > 0 && (!c->k_sink || !c->v_sink)) return SKVQ_ERR_INVALID_ARG;
     const void *ptrs[] = {c->k_codes, c->v_codes, c->k_meta, c->v_meta, c->k_win, c->v_win,
-                          c->lengths, c->reorder_k, c->reorder_v, c->alpha_k, c->alpha_v};
+                          c->lengths, c->reorder_k, c->reorder_v, c->alpha_k, c->alpha_v, c->k_sink, c->v_sink};
     for (const void *p : ptrs)
         if (p && misaligned(p)) return SKVQ_ERR_MISALIGNED;
     out->k_codes = static_cast<uint8_t *>(c->k_codes);
@@ -73,6 +77,8 @@ static int check_cache(const skvq_config *cfg, const skvq_cache *c, CachePtrs *o
     out->alpha_k = c->alpha_k;
     out->alpha_v = c->alpha_v;
     out->status = c->status;
+    out->k_sink = static_cast<__half *>(c->k_sink);
+    out->v_sink = static_cast<__half *>(c->v_sink);
     return SKVQ_OK;
 }
 
@@ -128,6 +134,12 @@ int skvq_cache_sizes(const skvq_config *cfg, size_t bytes_out[6])
     bytes_out[4] = (size_t)s.B * s.Hkv * s.W * kHeadDim * sizeof(__half);
     bytes_out[5] = bytes_out[4];
     return SKVQ_OK;
+}
+
+size_t skvq_sink_bytes(const skvq_config *cfg)
+{
+    if (check_cfg(cfg) != SKVQ_OK) return 0;
+    return (size_t)cfg->batch * cfg->n_kv_heads * cfg->n_sink * kHeadDim * sizeof(__half);
 }
 
 int skvq_quantize_append(const skvq_config *cfg, const skvq_cache *cache, const void *k, const void *v,

@@ -40,9 +40,9 @@ __device__ __forceinline__ int seq_new_count(const AppendArgs &a, int b)
 
 // Tokens [f0, f1) of a sequence (multiples of 64, possibly empty) are quantized by append_bulk_kernel: they are
 // new, they end up below the window, and they form whole aligned tiles.
-__device__ __forceinline__ void bulk_range(int L0, int q_end, int &f0, int &f1)
+__device__ __forceinline__ void bulk_range(int L0, int n_sink, int q_end, int &f0, int &f1)
 {
-    f0 = (L0 + 63) & ~63;
+    f0 = (max(L0, n_sink) + 63) & ~63;      // attention sinks are not quantized: they stay with append_kernel
     f1 = q_end & ~63;
     if (f1 < f0) f1 = f0;
 }
@@ -144,7 +144,7 @@ __global__ void __launch_bounds__(kAppendThreads) append_kernel(AppendArgs a)
     const int t_lo = max(L0 - W, 0);
     const int n_evict = max(min(L0, q_end) - t_lo, 0);
     int f0, f1;
-    bulk_range(L0, q_end, f0, f1);
+    bulk_range(L0, s.n_sink, q_end, f0, f1);
     const int n_bulk = a.use_bulk ? f1 - f0 : 0;   // new tokens the bulk kernel takes: skipped here
     const int n_items = n_evict + n_b - n_bulk;
 
@@ -230,7 +230,16 @@ __global__ void __launch_bounds__(kAppendThreads) append_kernel(AppendArgs a)
             __half2 hz;
             if (bits == 2) quantize16<2>(x, alpha, lanes_per_group, words, hz);
             else quantize16<4>(x, alpha, lanes_per_group, words, hz);
-            if (do_quant) {
+            if (do_quant && t < s.n_sink) {
+                // an attention sink (Sec. 3.2 filter rule): its reordered fp16 row is kept as it is
+                __align__(16) __half xh16[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) xh16[j] = __float2half_rn(x[j]);      // exact: x came from fp16
+                uint4 *p = reinterpret_cast<uint4 *>((is_v ? a.c.v_sink : a.c.k_sink) +
+                                                     (bh * s.n_sink + t) * (size_t)kHeadDim + (sub << 4));
+                p[0] = *reinterpret_cast<const uint4 *>(&xh16[0]);
+                p[1] = *reinterpret_cast<const uint4 *>(&xh16[8]);
+            } else if (do_quant) {
                 uint8_t *codes_row = codes + (size_t)t * row_bytes;
                 if (bits == 2) reinterpret_cast<uint32_t *>(codes_row)[sub] = words[0];
                 else reinterpret_cast<uint2 *>(codes_row)[sub] = make_uint2(words[0], words[1]);
@@ -268,7 +277,7 @@ __global__ void __launch_bounds__(kAppendThreads) append_bulk_kernel(AppendArgs 
     const int L1 = L0 + n_b;
     if (n_b == 0 || L1 > s.max_tokens) return;
     int f0, f1;
-    bulk_range(L0, max(L1 - s.W, 0), f0, f1);
+    bulk_range(L0, s.n_sink, max(L1 - s.W, 0), f0, f1);
     const int t0 = f0 + kBulkTok * blockIdx.x;
     if (t0 >= f1) return;
 

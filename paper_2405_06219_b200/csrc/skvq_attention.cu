@@ -107,7 +107,7 @@ __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
         const int t_begin = q_begin, t_end = q_end;
         for (int tile0 = t_begin; tile0 < t_end; tile0 += kTile) {
             const int t = tile0 + tid;
-            const bool valid = t < t_end;
+            const bool valid = t < t_end && t >= s.n_sink;      // sinks belong to the merge kernel
             float sc[kMaxRep];
 #pragma unroll
             for (int r = 0; r < kMaxRep; ++r) sc[r] = -CUDART_INF_F;
@@ -157,7 +157,7 @@ __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
 #pragma unroll
                     for (int w = 1; w < kThreads / 32; ++w) tm = fmaxf(tm, sred[r][w]);
                     const float m_new = fmaxf(m_run[r], tm);    // finite: the tile has a valid token
-                    corr[r] = exp2f(m_run[r] - m_new);          // exp2(-inf) = 0 on the first tile
+                    corr[r] = m_new == -CUDART_INF_F ? 1.f : exp2f(m_run[r] - m_new);   // 0 on the first tile with a token
                     const float p = valid ? exp2f(sc[r] - m_new) : 0.f;
                     sp[r][tid] = p;
                     l_thread[r] = l_thread[r] * corr[r] + p;
@@ -172,7 +172,7 @@ __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
                 constexpr int PER_WORD = 32 / VBITS;
                 const int g = tid / G;
                 const int w = tid / PER_WORD, sh = (tid % PER_WORD) * VBITS;
-                for (int tt = 0; tt < n_tok; ++tt) {
+                for (int tt = max(s.n_sink - tile0, 0); tt < n_tok; ++tt) {      // rows of sinks hold unspecified bytes
                     const size_t row = (size_t)(tile0 + tt);
                     const uint32_t word = __ldg(reinterpret_cast<const uint32_t *>(v_codes + row * VROW) + w);
                     const float2 hz = __half22float2(v_meta[row * ng + g]);
@@ -263,8 +263,9 @@ __global__ void plan_kernel(AttnArgs a)
     }
 }
 
-// One CTA per (query head, sequence): walks the fp16 window (at most W tokens: thread = token for the scores,
-// thread = reordered channel for P.V), then combines that with the split partials of the quantized prefix.
+// One CTA per (query head, sequence): walks the fp16 rows -- the attention sinks that have left the window, then
+// the window (thread = token for the scores, 16 lanes per row for P.V) -- then combines that with the split
+// partials of the quantized prefix.
 __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
 {
     const int hq = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -283,16 +284,16 @@ __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
     sq[tid] = __half2float(a.q[((size_t)b * s.Hq + hq) * kHeadDim + (a.c.reorder_k[(size_t)hk * kHeadDim + tid] & (kHeadDim - 1))]) *
               a.scale_log2;
     __syncthreads();
-    const __half *k_win = a.c.k_win + bh * (size_t)W * kHeadDim;
-    const __half *v_win = a.c.v_win + bh * (size_t)W * kHeadDim;
     // P.V layout: a warp instruction reads two rows (16 lanes x 8 channels each); warp w takes row pairs w, w+4, ...
     __shared__ __align__(16) float sacc[kThreads / 32][kHeadDim];      // written with 16-byte stores
     float m_run = -CUDART_INF_F, l_thread = 0.f;
     float a8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
     const int vsub = lane >> 4, vchunk = lane & 15;
-    for (int tile0 = Lq; tile0 < L; tile0 += kThreads) {
+    // Online softmax over the fp16 rows of tokens [t_begin, t_end): row of token t = t % ring (ring > 0) or t.
+    auto walk = [&](const __half *k_rows, const __half *v_rows, int t_begin, int t_end, int ring) {
+    for (int tile0 = t_begin; tile0 < t_end; tile0 += kThreads) {
         const int t = tile0 + tid;
-        const bool valid = t < L;
+        const bool valid = t < t_end;
         float sc = valid ? 0.f : -CUDART_INF_F;
         uint4 vu[kThreads / 8];
         if (!valid) {
@@ -300,12 +301,12 @@ __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
             for (int i = 0; i < kThreads / 8; ++i) {
                 const int tt = 8 * i + 2 * warp + vsub;
                 vu[i] = make_uint4(0u, 0u, 0u, 0u);
-                if (tile0 + tt < L)
-                    vu[i] = __ldg(reinterpret_cast<const uint4 *>(v_win + (size_t)((tile0 + tt) % W) * kHeadDim) + vchunk);
+                if (tile0 + tt < t_end)
+                    vu[i] = __ldg(reinterpret_cast<const uint4 *>(v_rows + (size_t)(ring ? (tile0 + tt) % ring : (tile0 + tt)) * kHeadDim) + vchunk);
             }
         }
         if (valid) {
-            const uint4 *row = reinterpret_cast<const uint4 *>(k_win + (size_t)(t % W) * kHeadDim);
+            const uint4 *row = reinterpret_cast<const uint4 *>(k_rows + (size_t)(ring ? t % ring : t) * kHeadDim);
             uint4 u[kHeadDim / 8];
 #pragma unroll
             for (int j8 = 0; j8 < kHeadDim / 8; ++j8) u[j8] = __ldg(row + j8);      // all 16 loads in flight
@@ -314,8 +315,8 @@ __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
             for (int i = 0; i < kThreads / 8; ++i) {
                 const int tt = 8 * i + 2 * warp + vsub;
                 vu[i] = make_uint4(0u, 0u, 0u, 0u);
-                if (tile0 + tt < L)
-                    vu[i] = __ldg(reinterpret_cast<const uint4 *>(v_win + (size_t)((tile0 + tt) % W) * kHeadDim) + vchunk);
+                if (tile0 + tt < t_end)
+                    vu[i] = __ldg(reinterpret_cast<const uint4 *>(v_rows + (size_t)(ring ? (tile0 + tt) % ring : (tile0 + tt)) * kHeadDim) + vchunk);
             }
 #pragma unroll
             for (int j8 = 0; j8 < kHeadDim / 8; ++j8) {
@@ -342,7 +343,7 @@ __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
 #pragma unroll
         for (int i = 0; i < 8; ++i) a8[i] *= corr;
         __syncthreads();
-        const int n_tok = min(kThreads, L - tile0);
+        const int n_tok = min(kThreads, t_end - tile0);
 #pragma unroll
         for (int i = 0; i < kThreads / 8; ++i) {            // 16 independent 16-byte loads per thread
             const int tt = 8 * i + 2 * warp + vsub;
@@ -359,6 +360,11 @@ __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
         }
         __syncthreads();   // sp and sred are rewritten by the next tile
     }
+    };
+    // attention sinks that have left the window (fp16 copies), then the window itself
+    const int n_s = min(s.n_sink, Lq);
+    if (n_s > 0) walk(a.c.k_sink + bh * (size_t)s.n_sink * kHeadDim, a.c.v_sink + bh * (size_t)s.n_sink * kHeadDim, 0, n_s, 0);
+    if (W > 0) walk(a.c.k_win + bh * (size_t)W * kHeadDim, a.c.v_win + bh * (size_t)W * kHeadDim, Lq, L, W);
 #pragma unroll
     for (int i = 0; i < 8; ++i) a8[i] += __shfl_xor_sync(0xffffffffu, a8[i], 16);
     if (vsub == 0) {

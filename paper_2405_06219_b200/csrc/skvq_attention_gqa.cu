@@ -350,12 +350,13 @@ __global__ void __launch_bounds__(kThreads, SKVQ_GQA_CTAS) partition_gqa_kernel(
         uint32_t *Vm = reinterpret_cast<uint32_t *>(Kc + 2 * C::kCodeTile + C::kMetaTile);
         const int tok0 = q_begin + (warp + i * kWarps) * kTileTok;
         const int n_valid = min(kTileTok, q_end - tok0);
-        if (n_valid < kTileTok) {
-            // rows past the end hold unspecified bytes: give their scale/zero words a defined value
+        const int n_skip = max(s.n_sink - tok0, 0);      // rows of attention sinks: the merge kernel reads their fp16 copies
+        if (n_valid < kTileTok || n_skip > 0) {
+            // rows past the end (and rows of sinks) hold unspecified bytes: give their scale/zero words a defined value
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf) {
                 const int tau = lane + 32 * hf;
-                if (tau >= n_valid) {
+                if (tau >= n_valid || tau < n_skip) {
 #pragma unroll
                     for (int gg = 0; gg < NG; ++gg) { Km[tau * NG + gg] = 0u; Vm[tau * NG + gg] = 0u; }
                 }
@@ -422,7 +423,8 @@ __global__ void __launch_bounds__(kThreads, SKVQ_GQA_CTAS) partition_gqa_kernel(
         for (int mt = 0; mt < 4; ++mt)
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
-                const bool valid = (32 * (mt >> 1) + own[2 * (mt & 1) + e]) < n_valid;
+                const int tok_in = 32 * (mt >> 1) + own[2 * (mt & 1) + e];
+                const bool valid = tok_in < n_valid && tok_in >= n_skip;
                 arg[mt][e] = valid ? fmaf(sraw[mt][e], cs, -m_ref) : -CUDART_INF_F;
                 amax = fmaxf(amax, arg[mt][e]);
             }
@@ -434,13 +436,14 @@ __global__ void __launch_bounds__(kThreads, SKVQ_GQA_CTAS) partition_gqa_kernel(
             for (int mt = 0; mt < 4; ++mt)
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
-                    const bool valid = (32 * (mt >> 1) + own[2 * (mt & 1) + e]) < n_valid;
+                    const int tok_in = 32 * (mt >> 1) + own[2 * (mt & 1) + e];
+                    const bool valid = tok_in < n_valid && tok_in >= n_skip;
                     if (valid) tm = fmaxf(tm, sraw[mt][e] * cs);
                 }
 #pragma unroll
             for (int msk = 4; msk < 32; msk <<= 1) tm = fmaxf(tm, __shfl_xor_sync(0xffffffffu, tm, msk));
             const float m_new = fmaxf(m_ref, tm);
-            const float corr = ex2_approx(m_ref - m_new);              // 0 on the first tile
+            const float corr = m_new == -CUDART_INF_F ? 1.f : ex2_approx(m_ref - m_new);      // 0 on the first tile with a token
             m_ref = m_new;
             l_sum *= corr;
 #pragma unroll
@@ -457,7 +460,8 @@ __global__ void __launch_bounds__(kThreads, SKVQ_GQA_CTAS) partition_gqa_kernel(
             for (int mt = 0; mt < 4; ++mt)
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
-                    const bool valid = (32 * (mt >> 1) + own[2 * (mt & 1) + e]) < n_valid;
+                    const int tok_in = 32 * (mt >> 1) + own[2 * (mt & 1) + e];
+                    const bool valid = tok_in < n_valid && tok_in >= n_skip;
                     arg[mt][e] = valid ? fmaf(sraw[mt][e], cs, -m_ref) : -CUDART_INF_F;
                 }
         }

@@ -283,7 +283,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB>::kCtasPerSm) partitio
 #pragma unroll
         for (int hf = 0; hf < T / 32; ++hf) {
             const int tau = lane + 32 * hf;
-            const bool valid = (tok0 + tau) < q_end;
+            const bool valid = (tok0 + tau) < q_end && (tok0 + tau) >= s.n_sink;      // sinks belong to the merge kernel
             float sv = 0.f;
 #pragma unroll
             for (int gg = 0; gg < NG; ++gg) {
@@ -310,7 +310,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB>::kCtasPerSm) partitio
                 for (int gg = 0; gg < NG; ++gg) hm = fmaxf(hm, hv[hf][gg]);
             }
             const float m_new = fmaxf(m_run, warp_max(tmx));
-            const float corr = ex2_approx(m_run - m_new);      // 0 on the first tile (m_run = -inf)
+            // 0 on the first tile (m_run = -inf); nothing to rescale while every token so far was masked
+            const float corr = m_new == -CUDART_INF_F ? 1.f : ex2_approx(m_run - m_new);
             m_run = m_new;
             l_part *= corr;
 #pragma unroll
@@ -335,7 +336,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB>::kCtasPerSm) partitio
             const float hscale = 4294967296.0f / h_bound;
 #pragma unroll
             for (int hf = 0; hf < T / 32; ++hf) {
-                const float p = ex2_approx(sc[hf] - m_run);      // exp2(-inf) = 0 for tokens past the end
+                // 0 for tokens past the end and for attention sinks (also while m_run is still -inf)
+                const float p = sc[hf] == -CUDART_INF_F ? 0.f : ex2_approx(sc[hf] - m_run);
                 l_part += p;
                 uint8_t *dst = Pb + (hf * 8 * 4 + ((lane >> 2) & 3)) * 8 + (lane >> 4) * 4 + (lane & 3);
 #pragma unroll

@@ -18,6 +18,7 @@ struct Shape {
     int B, Hq, Hkv, rep;   // rep = Hq / Hkv
     int k_bits, v_bits, G, ng;
     int W, cap, max_tokens;
+    int n_sink;            // positions below this are kept fp16 in the sink store when they leave the window
 };
 
 struct CachePtrs {
@@ -28,6 +29,7 @@ struct CachePtrs {
     const int32_t *reorder_k, *reorder_v;
     const float *alpha_k, *alpha_v;
     int32_t *status;
+    __half *k_sink, *v_sink;
 };
 
 // Flat partition of the quantized prefixes.  The unit is 256 tokens of one (sequence, KV head); all units of a

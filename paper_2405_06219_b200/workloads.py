@@ -45,6 +45,7 @@ class Workload:
     seed: int
     ragged: tuple | None = None  # (lo, hi) inclusive per-sequence length range
     calib_tokens: int = 512
+    n_sink: int = 0              # first positions kept fp16 for good (attention sinks; the paper's experiments use 5)
 
     @property
     def sm_scale(self) -> float:
@@ -150,14 +151,15 @@ def configs() -> list[Workload]:
 
 def algorithmic_bytes(w: Workload, lengths=None) -> int:
     """Bytes one decode-attention call must move: packed codes + scale/zero of the quantized
-    prefix, the fp16 window, and q/out.  Split scratch is not counted."""
+    prefix, the fp16 window and sinks, and q/out.  Split scratch is not counted."""
     lengths = w.lengths() if lengths is None else np.asarray(lengths)
     D, ng = w.head_dim, w.head_dim // w.group_size
     per_tok = (D * w.k_bits // 8 + 4 * ng) + (D * w.v_bits // 8 + 4 * ng)
     total = 0
     for L in lengths.tolist():
         lq = max(L - w.window, 0)
-        total += w.n_kv_heads * (lq * per_tok + min(L, w.window) * D * 2 * 2)
+        ns = min(w.n_sink, lq)
+        total += w.n_kv_heads * ((lq - ns) * per_tok + (ns + min(L, w.window)) * D * 2 * 2)
     total += w.batch * w.n_q_heads * D * 2 * 2
     return int(total)
 
@@ -168,5 +170,5 @@ def partition_kernel_bytes(w: Workload, lengths=None) -> int:
     lengths = w.lengths() if lengths is None else np.asarray(lengths)
     D, ng = w.head_dim, w.head_dim // w.group_size
     per_tok = (D * w.k_bits // 8 + 4 * ng) + (D * w.v_bits // 8 + 4 * ng)
-    total = sum(w.n_kv_heads * max(L - w.window, 0) * per_tok for L in lengths.tolist())
+    total = sum(w.n_kv_heads * max(L - w.window - w.n_sink, 0) * per_tok for L in lengths.tolist())
     return int(total + w.batch * w.n_q_heads * D * 2)

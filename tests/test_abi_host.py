@@ -52,7 +52,8 @@ def test_version_and_strerror(lib):
     (dict(v_bits=8), B.SKVQ_ERR_UNSUPPORTED), (dict(group_size=16), B.SKVQ_ERR_UNSUPPORTED),
     (dict(n_q_heads=7), B.SKVQ_ERR_UNSUPPORTED), (dict(n_q_heads=32, n_kv_heads=2), B.SKVQ_ERR_UNSUPPORTED),
     (dict(batch=0), B.SKVQ_ERR_INVALID_ARG), (dict(window=-1), B.SKVQ_ERR_INVALID_ARG),
-    (dict(max_tokens=0), B.SKVQ_ERR_INVALID_ARG), (dict(), B.SKVQ_OK), (dict(window=0, k_bits=4, group_size=32), B.SKVQ_OK),
+    (dict(max_tokens=0), B.SKVQ_ERR_INVALID_ARG), (dict(), B.SKVQ_OK), (dict(n_sink=5), B.SKVQ_OK),
+    (dict(n_sink=-1), B.SKVQ_ERR_INVALID_ARG), (dict(n_sink=65), B.SKVQ_ERR_UNSUPPORTED), (dict(window=0, k_bits=4, group_size=32), B.SKVQ_OK),
 ])
 def test_config_validation(lib, kw, code):
     assert B.skvq_check_config(cfg(**kw)) == code
@@ -104,14 +105,18 @@ def test_calls_reject_bad_arguments_before_any_launch(lib):
     assert lib.skvq_decode_attention(ctypes.byref(c), ctypes.byref(empty), None, None, ctypes.byref(args), None) \
         == B.SKVQ_ERR_INVALID_ARG
     # fake (never dereferenced) pointers: alignment, capacity and workspace checks are host-side
-    fake = B.SkvqCacheStruct(*([0x1000] * 11), None)
+    fake = B.SkvqCacheStruct(*([0x1000] * 11), None, None, None)
     assert lib.skvq_quantize_append(ctypes.byref(c), ctypes.byref(fake), 0x1008, 0x1000, None, 1, None) \
         == B.SKVQ_ERR_MISALIGNED
     assert lib.skvq_quantize_append(ctypes.byref(c), ctypes.byref(fake), 0x1000, 0x1000, None, 5000, None) \
         == B.SKVQ_ERR_CAPACITY
     assert lib.skvq_quantize_append(ctypes.byref(c), ctypes.byref(fake), 0x1000, 0x1000, None, -1, None) \
         == B.SKVQ_ERR_INVALID_ARG
-    misal = B.SkvqCacheStruct(0x1004, *([0x1000] * 10), None)
+    misal = B.SkvqCacheStruct(0x1004, *([0x1000] * 10), None, None, None)
+    nosink = cfg(n_sink=4)
+    assert lib.skvq_quantize_append(ctypes.byref(nosink), ctypes.byref(fake), 0x1000, 0x1000, None, 1, None) \
+        == B.SKVQ_ERR_INVALID_ARG                                  # sinks asked for, no sink buffers
+    assert B.skvq_sink_bytes(nosink) == 2 * 2 * 4 * 128 * 2 and B.skvq_sink_bytes(cfg()) == 0
     assert lib.skvq_quantize_append(ctypes.byref(c), ctypes.byref(misal), 0x1000, 0x1000, None, 1, None) \
         == B.SKVQ_ERR_MISALIGNED
     assert lib.skvq_decode_attention(ctypes.byref(c), ctypes.byref(fake), 0x1000, 0x1000, ctypes.byref(args), None) \

@@ -133,6 +133,37 @@ def test_attention_matches_oracle(cfg_i, kw, n):
     assert np.abs(got - want).max() <= ATTN_TOL
 
 
+# ------------------------------------------------------------------ attention sinks (Sec. 3.2 filter rules)
+@pytest.mark.parametrize("cfg_i,kw,n", [
+    (1, dict(context=3000, batch=2, n_kv_heads=4, n_q_heads=4, n_sink=5), 3000),              # integer kernel, 5 sinks as in the paper
+    (2, dict(context=2900, batch=1, n_sink=5), 2900),                                         # grouped-query kernel
+    (4, dict(context=1400, batch=2, ragged=None, n_kv_heads=4, n_q_heads=4, n_sink=64), 1400),   # 4-bit, a whole tile of sinks
+    (2, dict(context=800, batch=1, n_q_heads=16, n_kv_heads=2, n_sink=7), 800),               # scalar kernel
+    (2, dict(context=900, batch=2, ragged=None, n_sink=64), 900),                             # grouped-query kernel, first tile all sinks
+    (2, dict(context=700, batch=1, n_q_heads=16, n_kv_heads=2, n_sink=64), 700),              # scalar kernel, first tile all sinks
+    (0, dict(context=130, n_sink=5), 130),                                                    # fewer tokens out of the window than sinks
+    (0, dict(context=300, window=0, n_sink=3), 300),
+])
+def test_sinks_stay_fp16_and_attention_matches_oracle(cfg_i, kw, n):
+    w = small(cfg_i, **kw)
+    gpu, ora = both_caches(w, n + 64)
+    k, v = w.prefill("k", n), w.prefill("v", n)
+    cut = n // 3
+    gpu.append(dev(k[:, :cut]), dev(v[:, :cut]))                      # in two pieces: sinks leave the window in either call
+    gpu.append(dev(k[:, cut:]), dev(v[:, cut:]))
+    ora.append(k, v)
+    assert_cache_bit_exact(gpu, ora)
+    got, want = attention_both(gpu, ora, w)
+    assert np.abs(got - want).max() <= ATTN_TOL
+    for s in range(6):                                                # decode steps: single-token appends
+        kn, vn = w.new_token("k", s), w.new_token("v", s)
+        gpu.append(dev(kn), dev(vn))
+        ora.append(kn, vn)
+    assert_cache_bit_exact(gpu, ora)
+    got, want = attention_both(gpu, ora, w, step=1)
+    assert np.abs(got - want).max() <= ATTN_TOL
+
+
 def test_attention_ragged_batch_with_empty_sequence():
     w = small(4, context=2000, batch=6, ragged=None)
     gpu, ora = both_caches(w, 2048)

@@ -27,7 +27,7 @@ def test_shapes_beyond_the_builtin_array_are_refused_before_any_launch(lib):
     """Host-side check (no GPU needed): 4 x 32 heads x 4001 parts x 528 B is far beyond 8 MiB."""
     c = B.SkvqConfig(4, 32, 8, 128, 2, 2, 32, 128, 1 << 20)
     assert B.skvq_workspace_size(c, 1 << 20, 4000) > B.SKVQ_NOALLOC_SCRATCH_BYTES
-    fake = B.SkvqCacheStruct(*([0x1000] * 11), None)
+    fake = B.SkvqCacheStruct(*([0x1000] * 11), None, None, None)
     before = B.skvq_launch_count()
     rc = lib.skvq_decode_attention_noalloc(ctypes.byref(c), ctypes.byref(fake), 0x1000, 0x1000, 0.1, 1 << 20, 4000,
                                            None)
