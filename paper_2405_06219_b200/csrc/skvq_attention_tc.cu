@@ -1,0 +1,568 @@
+// Partition kernel of skvq_decode_attention on the fifth-generation tensor cores (tcgen05.mma, accumulators in
+// tensor memory) for 2-bit K and V with up to 4 query heads per KV head and any group size (Eq. 1, Algorithm 1).
+//
+//   q'.K~_t            = sum_g h_{t,g} (sum_{j in g} q'_j c_{t,j}) + sum_g z_{t,g} (sum_{j in g} q'_j)
+//   sum_t p_t V~_{t,d} = sum_t (p_t h_{t,g(d)}) c_{t,d} + sum_t p_t z_{t,g(d)}
+//
+// One CTA = 128 threads = one tile of 128 tokens at a time, one thread per token.  The warps only unpack and do the
+// per-(token, head, group) arithmetic; both contractions run asynchronously on the tensor core:
+//   * a thread turns its token's 32 packed bytes into 128 bytes "4^j * code" (one AND per four codes) and stores them
+//     as a row of the A operand of the score MMA (u8, K-major).  The B operand holds the permuted query of every head
+//     as four signed byte digits of a 31-bit fixed-point number with the weight 4^j divided out, so the int32
+//     accumulators are the exact group dot products: one MMA k-step (32 channels) per 32 channels, a fresh set of
+//     16 columns (head, digit) per quantization group.
+//   * the thread reads its row of accumulators from tensor memory, combines digits and groups with h and z (fp32),
+//     and takes part in a lazy online softmax: the reference of a head moves only when a score exceeds it by 16 in
+//     the log2 domain (or the bound on the value scales has to grow), which after the first tile is rare.
+//   * p*h per (head, group) goes onto a 32-bit fixed-point grid; the four bytes of that integer are four rows
+//     (head, digit) of the A operand of the value MMA (u8, MN-major: one 16-byte store per group), whose B operand
+//     is the unpacked V tile exactly as the thread stored it (u8, MN-major).  Rows are (group, head, digit): 64 rows
+//     x 128 channels of exact int32 sums in tensor memory, of which the (group, channels of that group) blocks are
+//     read when the reference moves, every 256 tiles, and at the end of a segment.
+// Tiles arrive through a ring of shared-memory stages filled by cp.async.bulk (mbarrier completion); every wait is
+// bounded and reports through the cache's status word.
+#include "skvq_mma_common.cuh"
+
+namespace skvq {
+namespace {
+
+using namespace mmak;
+
+constexpr int kTile = 128;              // tokens per tile = rows of the score MMA = threads per CTA
+constexpr int kHeads = 4;               // query heads per KV head served (absent heads carry a zero query)
+constexpr int kSlackLog2 = 16;          // the softmax reference moves only when a score exceeds it by this (log2)
+constexpr int kStages = 3;
+constexpr int kTmemCols = 256;          // allocation: scores in columns [0, 64), value sums in [128, 256)
+constexpr int kScoreCol = 0, kPvCol = 128;
+constexpr int kFoldTiles = 256;         // 255 * 192 * 128 * 256 < 2^31: the int32 value sums are folded at least this often
+constexpr uint32_t kLbo = 128;          // bytes between core matrices along K (all operands)
+constexpr uint32_t kSboK = 1024;        // K-major operands: bytes between groups of 8 rows
+constexpr uint32_t kSboMN = 2048;       // MN-major operands: bytes between 16-byte chunks of the M/N extent (128 tokens)
+
+template <int G>
+struct TCfg {
+    static constexpr int NG = kHeadDim / G;
+    static constexpr int kCodeTile = kTile * kRowBytes;                  // 4096
+    static constexpr int kMetaTile = kTile * NG * 4;
+    static constexpr int kStageBytes = 2 * kCodeTile + 2 * kMetaTile;
+    static constexpr int kOffKA = kStages * kStageBytes;                 // A of the score MMA: [128 tokens][128 bytes]
+    static constexpr int kOffQB = kOffKA + kTile * 128;                  // B of the score MMA: [16 (head, digit)][128 bytes]
+    static constexpr int kOffVB = kOffQB + 16 * 128;                     // B of the value MMA, two buffers
+    static constexpr int kOffPA = kOffVB + 2 * kTile * 128;              // A of the value MMA, two buffers of [128 tokens][64 rows]
+    static constexpr int kOffOs = kOffPA + 2 * kTile * 64;               // folded value sums [4][128] fp32, by MMA column
+    static constexpr int kOffQs = kOffOs + kHeads * kHeadDim * 4;        // prologue scratch [4][128] fp32
+    static constexpr int kOffMisc = kOffQs + kHeads * kHeadDim * 4;      // small arrays, see the kernel
+    static constexpr int kSmemBytes = kOffMisc + 1024;
+};
+
+// ---------------------------------------------------------------- tcgen05 wrappers
+// Shared-memory matrix descriptor, no swizzle: start address, leading (K direction) and stride (M/N direction) byte
+// offsets between 8 x 16-byte core matrices, all in units of 16 bytes; descriptor version 1.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo)
+{
+    return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo >> 4) & 0x3FFFu) << 16) |
+           ((uint64_t)((sbo >> 4) & 0x3FFFu) << 32) | (1ull << 46);
+}
+// Instruction descriptor of kind::i8: int32 accumulators, operand signedness, operand majorness, N and M.
+__host__ __device__ constexpr uint32_t idesc_i8(int M, int N, bool a_signed, bool b_signed, bool a_mn, bool b_mn)
+{
+    return (2u << 4) | ((a_signed ? 1u : 0u) << 7) | ((b_signed ? 1u : 0u) << 10) | ((a_mn ? 1u : 0u) << 15) |
+           ((b_mn ? 1u : 0u) << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+                 " tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}"
+                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// The mbarrier gets one arrival when every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void proxy_fence() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// Lane i of the warp receives 16 consecutive 32-bit columns of tensor-memory lane (lane field of addr) + i.
+__device__ __forceinline__ void tmem_ld16(uint32_t addr, int (&r)[16])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+                 : "r"(addr));
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ uint32_t to_fixed_u32(float x)
+{
+    uint32_t r;
+    asm("cvt.rni.sat.u32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return r;
+}
+__device__ __forceinline__ float lo_half(uint32_t w) { return __low2float(*reinterpret_cast<const __half2 *>(&w)); }
+__device__ __forceinline__ float hi_half(uint32_t w) { return __high2float(*reinterpret_cast<const __half2 *>(&w)); }
+
+template <int NG>
+__device__ __forceinline__ void load_words(const uint32_t *p, uint32_t (&w)[NG])
+{
+    if constexpr (NG == 4) {
+        const uint4 x = *reinterpret_cast<const uint4 *>(p);
+        w[0] = x.x; w[1] = x.y; w[2] = x.z; w[3] = x.w;
+    } else if constexpr (NG == 2) {
+        const uint2 x = *reinterpret_cast<const uint2 *>(p);
+        w[0] = x.x; w[1] = x.y;
+    } else {
+        w[0] = p[0];
+    }
+}
+
+// One token's 32 packed bytes -> 128 bytes 4^j * code.  Byte 16w + 4j + b of the row is code j + 4b of word w (channel
+// 16w + j + 4b) times 4^j; chunk w (16 bytes) goes to dst + w * chunk_stride.
+__device__ __forceinline__ void unpack_row(const uint8_t *packed, uint8_t *dst, uint32_t chunk_stride)
+{
+    const uint4 x0 = *reinterpret_cast<const uint4 *>(packed), x1 = *reinterpret_cast<const uint4 *>(packed + 16);
+    const uint32_t w[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+        *reinterpret_cast<uint4 *>(dst + i * chunk_stride) =
+            make_uint4(w[i] & 0x03030303u, w[i] & 0x0C0C0C0Cu, w[i] & 0x30303030u, w[i] & 0xC0C0C0C0u);
+}
+
+// Channel and weight exponent of byte column n of an unpacked row (the K index of the score MMA, the N index of the
+// value MMA).
+__device__ __forceinline__ int column_channel(int n) { return 16 * (n >> 4) + ((n >> 2) & 3) + 4 * (n & 3); }
+__device__ __forceinline__ int column_shift(int n) { return 2 * ((n >> 2) & 3); }
+
+template <int G>
+__global__ void __launch_bounds__(kTile, 2) partition_tc_kernel(MmaArgs a)
+{
+    using C = TCfg<G>;
+    constexpr int NG = C::NG;
+    extern __shared__ __align__(128) uint8_t smem[];
+    const Shape &s = a.s;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int R = s.rep;
+    asm volatile("griddepcontrol.launch_dependents;");      // the merge kernel may start its window part early
+    asm volatile("griddepcontrol.wait;" ::: "memory");      // the lengths, and the plan kernel's header when there is one
+
+    __shared__ __align__(16) Segment seg_sh;
+    __shared__ int more_sh;
+    __shared__ int fail_sh;
+    __shared__ uint32_t tmem_sh;
+    __shared__ SlotWalker walk;      // only thread 0 touches it
+    __shared__ __align__(16) int hdr_sh[kPlanSmemInts];
+    if (a.plan.in_kernel) {
+        if (warp == 0) plan_in_warp(a.c.lengths, s.B, s.Hkv, s.W, a.plan.lq_cap, a.plan.n_slots, hdr_sh);
+        __syncthreads();
+    }
+    if (tid == 0) {
+        more_sh = walk.start(a.plan.in_kernel ? hdr_sh : reinterpret_cast<const int *>(a.ws), !a.plan.in_kernel, s.B, s.Hkv,
+                             blockIdx.x) ? 1 : 0;
+        fail_sh = 0;
+    }
+    __syncthreads();
+    if (!more_sh) return;
+    float *partials = a.ws + a.plan.hdr_ints;
+
+    // ---- shared memory
+    uint8_t *KA = smem + C::kOffKA, *QB = smem + C::kOffQB;
+    float *Os = reinterpret_cast<float *>(smem + C::kOffOs);         // [4][128] by MMA column
+    float *qs = reinterpret_cast<float *>(smem + C::kOffQs);         // [4][128] permuted query (prologue)
+    float *sqs = reinterpret_cast<float *>(smem + C::kOffMisc);      // [4][4]  sm_scale*log2(e) * sum_{j in g} q'_j
+    float *csc = sqs + 16;                                           // [4]     sm_scale*log2(e) * 2^(e_r - 30)
+    int *fexp = reinterpret_cast<int *>(csc + 4);                    // [4]
+    float *red = reinterpret_cast<float *>(fexp + 4);                // [4 warps][24] reductions
+    uint64_t *bars = reinterpret_cast<uint64_t *>(red + kWarps * 24);   // [kStages] tiles, [1] scores, [2] value MMAs
+    const uint32_t bar_tile = smem_u32(bars), bar_s = bar_tile + 8 * kStages, bar_pv = bar_s + 8;
+
+    // ---- tensor memory and barriers (once per CTA)
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_sh)), "r"(kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (tid == 0) {
+#pragma unroll
+        for (int i = 0; i < kStages + 3; ++i) mbar_init(bar_tile + 8 * i, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        proxy_fence();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_sh;
+    const uint32_t tmem_row = tmem + ((uint32_t)(warp * 32) << 16);      // this warp's 32 lanes
+
+    constexpr uint32_t kIdescS = idesc_i8(128, 16, false, true, false, false);
+    constexpr uint32_t kIdescPV = idesc_i8(64, 128, false, false, true, true);
+
+    // kernel-lifetime pipeline counters (uniform across the CTA)
+    uint32_t tiles_done = 0;           // tiles that went through the stage ring
+    uint32_t s_done = 0;               // completions of the score barrier consumed
+    uint32_t pv_issued0 = 0, pv_issued1 = 0, pv_waited0 = 0, pv_waited1 = 0;      // value MMAs per operand buffer
+    bool failed = false;
+
+    auto wait_pv = [&](int buf) {
+        const uint32_t issued = buf ? pv_issued1 : pv_issued0, waited = buf ? pv_waited1 : pv_waited0;
+        if (waited < issued) {
+            if (!mbar_wait_bounded(bar_pv + 8 * buf, (issued - 1) & 1u)) fail_sh = 1;
+            if (buf) pv_waited1 = issued; else pv_waited0 = issued;
+        }
+    };
+
+    for (;;) {
+    if (tid == 0) seg_sh = walk.next(a.c.lengths, s.W, a.plan.lq_cap);
+    __syncthreads();
+    const int b = seg_sh.b, hk = seg_sh.hk, q_begin = seg_sh.tok_begin, q_end = seg_sh.tok_end, part = seg_sh.part;
+    const int n_parts = a.plan.s_max;
+    const size_t bh = (size_t)b * s.Hkv + hk;
+    const uint8_t *k_codes = a.c.k_codes + bh * (size_t)s.cap * kRowBytes;
+    const uint8_t *v_codes = a.c.v_codes + bh * (size_t)s.cap * kRowBytes;
+    const __half2 *k_meta = a.c.k_meta + bh * (size_t)s.cap * NG;
+    const __half2 *v_meta = a.c.v_meta + bh * (size_t)s.cap * NG;
+    const int n_tiles = failed ? 0 : (q_end - q_begin + kTile - 1) / kTile;
+
+    auto issue_tile = [&](int i) {      // thread 0 only: tile i of this segment into its stage
+        const uint32_t st = (tiles_done + i) % kStages;
+        const int tok0 = q_begin + i * kTile;
+        const uint32_t rows = (uint32_t)min(kTile, (q_end - tok0 + 63) & ~63);      // the cache's capacity is a multiple of 64
+        const uint32_t dst = smem_u32(smem + st * C::kStageBytes);
+        const uint32_t bar = bar_tile + 8 * st;
+        mbar_expect_tx(bar, rows * (2 * kRowBytes + 2 * NG * 4));
+        bulk_g2s(dst, k_codes + (size_t)tok0 * kRowBytes, rows * kRowBytes, bar);
+        bulk_g2s(dst + C::kCodeTile, v_codes + (size_t)tok0 * kRowBytes, rows * kRowBytes, bar);
+        bulk_g2s(dst + 2 * C::kCodeTile, k_meta + (size_t)tok0 * NG, rows * NG * 4, bar);
+        bulk_g2s(dst + 2 * C::kCodeTile + C::kMetaTile, v_meta + (size_t)tok0 * NG, rows * NG * 4, bar);
+    };
+    auto wait_tile = [&](int i) {
+        const uint32_t t = tiles_done + i;
+        if (!mbar_wait_bounded(bar_tile + 8 * (t % kStages), (t / kStages) & 1u)) fail_sh = 1;
+    };
+    auto stage_of = [&](int i) { return smem + ((tiles_done + i) % kStages) * C::kStageBytes; };
+    auto issue_scores = [&]() {         // thread 0 only
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+            umma_i8(tmem + kScoreCol + 16 * ((32 * ks) / G), smem_desc(smem_u32(KA) + ks * 2 * kLbo, kLbo, kSboK),
+                    smem_desc(smem_u32(QB) + ks * 2 * kLbo, kLbo, kSboK), kIdescS, ((32 * ks) % G) != 0 ? 1u : 0u);
+        umma_commit(bar_s);
+    };
+
+    if (tid == 0) {      // the first copies are in flight while the query is prepared
+        proxy_fence();   // the stages were read through the generic proxy by the previous segment
+        for (int i = 0; i < kStages && i < n_tiles; ++i) issue_tile(i);
+    }
+
+    // ---- CTA-wide prologue: permuted query per head on a power-of-two scale -> byte digits, group constants
+    {
+        const int32_t *idx_k = a.c.reorder_k + (size_t)hk * kHeadDim;
+        const int src = idx_k[tid] & (kHeadDim - 1);
+#pragma unroll
+        for (int r = 0; r < kHeads; ++r) {
+            const float qv = r < R ? __half2float(a.q[((size_t)b * s.Hq + hk * R + r) * kHeadDim + src]) : 0.f;
+            qs[r * kHeadDim + tid] = qv;
+            const float wm = warp_max(fabsf(qv));
+            if (lane == 0) red[warp * 24 + r] = wm;
+        }
+        Os[tid] = 0.f; Os[kHeadDim + tid] = 0.f; Os[2 * kHeadDim + tid] = 0.f; Os[3 * kHeadDim + tid] = 0.f;
+    }
+    __syncthreads();
+    if (tid < kHeads) {
+        float qmax = 0.f;
+        for (int w = 0; w < kWarps; ++w) qmax = fmaxf(qmax, red[w * 24 + tid]);
+        int e = 0;
+        if (qmax > 0.f) (void)frexpf(qmax, &e);            // qmax = m * 2^e, 0.5 <= m < 1: |q' * 2^-e| < 1
+        fexp[tid] = e;
+        csc[tid] = ldexpf(a.scale_log2, e - 30);
+    }
+    if (tid >= 32 && tid < 32 + kHeads * NG) {
+        const int r = (tid - 32) / NG, gg = (tid - 32) % NG;
+        float sq = 0.f;
+        for (int j = gg * G; j < (gg + 1) * G; ++j) sq += qs[r * kHeadDim + j];
+        sqs[r * 4 + gg] = sq * a.scale_log2;
+    }
+    __syncthreads();
+    {
+        // thread = byte column k of the operand: channel column_channel(k), weight 4^j divided out of the query
+        const int ch = column_channel(tid), sh = column_shift(tid);
+        uint8_t *col = QB + (tid >> 4) * kLbo + (tid & 15);
+#pragma unroll
+        for (int r = 0; r < kHeads; ++r) {
+            int qi = __float2int_rn(ldexpf(qs[r * kHeadDim + ch], 30 - fexp[r] - sh));      // |qi| < 2^30
+#pragma unroll
+            for (int d = 0; d < 4; ++d) {
+                const int dg = d < 3 ? ((qi + 128) & 255) - 128 : qi;      // balanced digits: qi = sum dg * 256^d
+                qi = (qi - dg) >> 8;
+                const int n = 4 * r + d;
+                col[(n >> 3) * kSboK + (n & 7) * 16] = (uint8_t)(dg & 255);
+            }
+        }
+    }
+
+    // ---- running state: this thread's token of every tile, all four heads
+    float m_ref[kHeads], l_sum[kHeads], zp[kHeads][NG];
+#pragma unroll
+    for (int r = 0; r < kHeads; ++r) {
+        m_ref[r] = -CUDART_INF_F;
+        l_sum[r] = 0.f;
+#pragma unroll
+        for (int gg = 0; gg < NG; ++gg) zp[r][gg] = 0.f;
+    }
+    float h_bound = 6.103515625e-05f;      // power of two above every value scale seen so far (2^-14 to start with)
+    bool pv_fresh = true;                  // the next value MMA overwrites the accumulators
+    int tiles_since_fold = 0;
+
+    // Brings the int32 value sums into the fp32 sums in shared memory (relative to the old references and bound).
+    auto fold_pv = [&]() {
+        wait_pv(0);
+        wait_pv(1);
+        tc_fence_after();
+        if (!pv_fresh && warp < NG) {
+            // lanes 0-15 of this warp's tensor-memory lanes hold rows (group = warp, head = lane / 4, digit = lane % 4)
+            const float sa = h_bound * (1.0f / (float)(1u << (32 - kSlackLog2))) * (float)(1u << (8 * (lane & 3)));
+#pragma unroll 1
+            for (int c0 = 0; c0 < G; c0 += 16) {
+                int v[16];
+                tmem_ld16(tmem_row + kPvCol + warp * G + c0, v);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    float x = (float)v[j] * sa;
+                    x += __shfl_xor_sync(0xffffffffu, x, 1);
+                    x += __shfl_xor_sync(0xffffffffu, x, 2);
+                    if (lane < 16 && (lane & 3) == 0) Os[(lane >> 2) * kHeadDim + warp * G + c0 + j] += x;
+                }
+            }
+        }
+        tc_fence_before();
+        pv_fresh = true;
+        tiles_since_fold = 0;
+    };
+
+    // ---- first tile: unpack K and start its score MMA
+    if (n_tiles > 0) {
+        wait_tile(0);
+        unpack_row(stage_of(0) + tid * kRowBytes, KA + (tid >> 3) * kSboK + (tid & 7) * 16, kLbo);
+    }
+    proxy_fence();
+    __syncthreads();
+    if (fail_sh) failed = true;
+    if (tid == 0 && n_tiles > 0 && !failed) issue_scores();
+
+    for (int i = 0; i < n_tiles && !failed; ++i) {
+        const int buf = i & 1;
+        uint8_t *stg = stage_of(i);
+        const uint32_t *Km = reinterpret_cast<const uint32_t *>(stg + 2 * C::kCodeTile);       // [128][NG] words {h, z}
+        const uint32_t *Vm = reinterpret_cast<const uint32_t *>(stg + 2 * C::kCodeTile + C::kMetaTile);
+        uint8_t *VB = smem + C::kOffVB + buf * (kTile * 128);
+        uint8_t *PA = smem + C::kOffPA + buf * (kTile * 64);
+        const int tok = q_begin + i * kTile + tid;
+        const bool valid = tok < q_end && tok >= s.n_sink;      // sinks belong to the merge kernel
+
+        // ---------------- V tile -> B operand of the value MMA (its buffer was last read by the MMA two tiles ago)
+        wait_pv(buf);
+        unpack_row(stg + C::kCodeTile + tid * kRowBytes, VB + (tid >> 3) * kLbo + (tid & 7) * 16, kSboMN);
+
+        // ---------------- scores of this thread's token
+        if (!mbar_wait_bounded(bar_s, s_done & 1u)) fail_sh = 1;
+        ++s_done;
+        tc_fence_after();
+        uint32_t kw[NG], vw[NG];
+        load_words<NG>(Km + tid * NG, kw);
+        load_words<NG>(Vm + tid * NG, vw);
+        float sc[kHeads];
+#pragma unroll
+        for (int r = 0; r < kHeads; ++r) sc[r] = 0.f;
+        float zt[kHeads] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int gg = 0; gg < NG; ++gg) {
+            int v[16];
+            tmem_ld16(tmem_row + kScoreCol + 16 * gg, v);
+            tmem_wait_ld();
+            const float hk_ = lo_half(kw[gg]), zk_ = hi_half(kw[gg]);
+#pragma unroll
+            for (int r = 0; r < kHeads; ++r) {
+                const int lo = v[4 * r] + (v[4 * r + 1] << 8), hi = v[4 * r + 2] + (v[4 * r + 3] << 8);
+                const float u = fmaf((float)hi, 65536.0f, (float)lo);      // 2^30 * sum_j q'_j 2^-e c_j over the group
+                sc[r] = fmaf(hk_, u, sc[r]);
+                zt[r] = fmaf(zk_, sqs[r * 4 + gg], zt[r]);
+            }
+        }
+        float hmax = 0.f;
+        float hv[NG], zv[NG];
+#pragma unroll
+        for (int gg = 0; gg < NG; ++gg) {
+            hv[gg] = valid ? lo_half(vw[gg]) : 0.f;      // rows past the end and rows of sinks hold unspecified bytes
+            zv[gg] = valid ? hi_half(vw[gg]) : 0.f;
+            hmax = fmaxf(hmax, hv[gg]);
+        }
+        float arg[kHeads];
+        bool need = hmax >= h_bound;
+#pragma unroll
+        for (int r = 0; r < kHeads; ++r) {
+            sc[r] = valid ? fmaf(sc[r], csc[r], zt[r]) : -CUDART_INF_F;      // log2 domain
+            arg[r] = sc[r] - m_ref[r];
+            need |= valid && (arg[r] > (float)kSlackLog2 || m_ref[r] == -CUDART_INF_F);
+        }
+        need |= tiles_since_fold >= kFoldTiles;
+        tc_fence_before();
+        const int moved = __syncthreads_or(need ? 1 : 0);
+        if (fail_sh) { failed = true; break; }
+        if (moved) {
+            // Rare after the first tile: raise every head's reference to its running maximum (and the bound on h),
+            // fold what was accumulated and bring it onto the new references.
+            float hm = warp_max(hmax);
+            if (lane == 0) red[warp * 24 + 4] = hm;
+#pragma unroll
+            for (int r = 0; r < kHeads; ++r) {
+                const float wm = warp_max(sc[r]);
+                if (lane == 0) red[warp * 24 + r] = wm;
+            }
+            fold_pv();
+            __syncthreads();
+            if (fail_sh) { failed = true; break; }
+            float corr[kHeads];
+#pragma unroll
+            for (int r = 0; r < kHeads; ++r) {
+                float mx = m_ref[r];
+                for (int w = 0; w < kWarps; ++w) mx = fmaxf(mx, red[w * 24 + r]);
+                corr[r] = mx == -CUDART_INF_F ? 1.f : ex2_approx(m_ref[r] - mx);      // 0 on the first tile with a token
+                m_ref[r] = mx;
+                l_sum[r] *= corr[r];
+#pragma unroll
+                for (int gg = 0; gg < NG; ++gg) zp[r][gg] *= corr[r];
+                Os[r * kHeadDim + tid] *= corr[r];
+                arg[r] = sc[r] - m_ref[r];
+            }
+            hm = 0.f;
+            for (int w = 0; w < kWarps; ++w) hm = fmaxf(hm, red[w * 24 + 4]);
+            if (hm >= h_bound) h_bound = __int_as_float(((__float_as_int(hm) >> 23) + 1) << 23);   // next power of two above
+            __syncthreads();      // red is rewritten by the next move
+        }
+
+        // ---------------- p and the digits of p*h -> A operand of the value MMA
+        {
+            const float hscale = (float)(1u << (32 - kSlackLog2)) / h_bound;
+            float ps[kHeads];
+#pragma unroll
+            for (int r = 0; r < kHeads; ++r) {
+                const float p = sc[r] == -CUDART_INF_F ? 0.f : ex2_approx(arg[r]);      // at most 2^slack
+                l_sum[r] += p;
+                ps[r] = p * hscale;
+#pragma unroll
+                for (int gg = 0; gg < NG; ++gg) zp[r][gg] = fmaf(p, zv[gg], zp[r][gg]);
+            }
+#pragma unroll
+            for (int gg = 0; gg < NG; ++gg)
+                *reinterpret_cast<uint4 *>(PA + gg * kSboMN + (tid >> 3) * kLbo + (tid & 7) * 16) =
+                    make_uint4(to_fixed_u32(ps[0] * hv[gg]), to_fixed_u32(ps[1] * hv[gg]), to_fixed_u32(ps[2] * hv[gg]),
+                               to_fixed_u32(ps[3] * hv[gg]));
+        }
+
+        // ---------------- next tile's K -> A operand of the score MMA (this tile's score MMA has completed)
+        if (i + 1 < n_tiles) {
+            wait_tile(i + 1);
+            unpack_row(stage_of(i + 1) + tid * kRowBytes, KA + (tid >> 3) * kSboK + (tid & 7) * 16, kLbo);
+        }
+        proxy_fence();
+        __syncthreads();
+        if (fail_sh) { failed = true; break; }
+        if (tid == 0) {
+            tc_fence_after();
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+                umma_i8(tmem + kPvCol, smem_desc(smem_u32(PA) + ks * 4 * kLbo, kLbo, kSboMN),
+                        smem_desc(smem_u32(VB) + ks * 4 * kLbo, kLbo, kSboMN), kIdescPV, (pv_fresh && ks == 0) ? 0u : 1u);
+            umma_commit(bar_pv + 8 * buf);
+            if (i + 1 < n_tiles) issue_scores();
+            if (i + kStages < n_tiles) {
+                proxy_fence();      // the stage was read through the generic proxy
+                issue_tile(i + kStages);
+            }
+        }
+        if (buf) ++pv_issued1; else ++pv_issued0;
+        pv_fresh = false;
+        ++tiles_since_fold;
+    }
+
+    // ---- end of the segment: last fold, CTA-wide sums, one partial per query head
+    if (failed) {
+        // let whatever is still in flight land (bounded), then report
+        for (int i = 0; i < n_tiles; ++i) wait_tile(i);
+        if (tid == 0 && a.c.status) atomicOr(a.c.status, SKVQ_STATUS_COPY_TIMEOUT);
+    }
+    fold_pv();
+#pragma unroll
+    for (int r = 0; r < kHeads; ++r) {
+        const float ls = warp_sum(l_sum[r]);
+        if (lane == 0) red[warp * 24 + r] = ls;
+#pragma unroll
+        for (int gg = 0; gg < NG; ++gg) {
+            const float zs = warp_sum(zp[r][gg]);
+            if (lane == 0) red[warp * 24 + 8 + r * 4 + gg] = zs;
+        }
+    }
+    __syncthreads();
+    {
+        const int ch = column_channel(tid);
+        const float winv = __int_as_float((127 - column_shift(tid)) << 23);      // 4^-j
+#pragma unroll
+        for (int r = 0; r < kHeads; ++r) {
+            if (r >= R) break;
+            float l = 0.f, z = 0.f;
+            for (int w = 0; w < kWarps; ++w) {
+                l += red[w * 24 + r];
+                z += red[w * 24 + 8 + r * 4 + ch / G];
+            }
+            const bool dead = failed || m_ref[r] == -CUDART_INF_F;
+            float *dst = partials + (((size_t)b * s.Hq + hk * R + r) * n_parts + part) * kPartialStride;
+            dst[ch] = dead ? 0.f : fmaf(Os[r * kHeadDim + tid], winv, z);
+            if (tid == 0) { dst[kHeadDim] = dead ? -CUDART_INF_F : m_ref[r]; dst[kHeadDim + 1] = dead ? 0.f : l; }
+        }
+    }
+    tiles_done += (uint32_t)n_tiles;
+    __syncthreads();          // the segment's shared data is dead; thread 0 decides whether there is another one
+    if (tid == 0) more_sh = walk.done() ? 0 : 1;
+    __syncthreads();
+    if (!more_sh) break;
+    }
+
+    // ---- give the tensor memory back (every tensor-memory read of this CTA is behind the barriers above)
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+}
+
+template <int G>
+cudaError_t launch_g(const MmaArgs &a, cudaStream_t stream, bool overlap)
+{
+    using C = TCfg<G>;
+    static bool configured = false;
+    auto kern = partition_tc_kernel<G>;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    return launch_dependent(kern, dim3(a.plan.n_slots), dim3(kTile), C::kSmemBytes, stream, overlap, a);
+}
+
+}  // namespace
+
+// Launches the kernel above when the configuration is covered (2-bit K and V, 1, 2 or 4 query heads per KV
+// head); *handled tells the caller whether it did.
+cudaError_t launch_partition_tc(const Shape &s, const CachePtrs &c, const __half *q, float scale_log2, const SplitPlan &plan,
+                                float *workspace, cudaStream_t stream, bool overlap, bool *handled)
+{
+    *handled = false;
+    if (s.k_bits != 2 || s.v_bits != 2 || s.rep > kHeads) return cudaSuccess;
+    MmaArgs a{s, c, q, scale_log2, plan, workspace};
+    *handled = true;
+    switch (s.G) {
+        case 128: return launch_g<128>(a, stream, overlap);
+        case 64: return launch_g<64>(a, stream, overlap);
+        case 32: return launch_g<32>(a, stream, overlap);
+        default: *handled = false; return cudaSuccess;
+    }
+}
+
+}  // namespace skvq

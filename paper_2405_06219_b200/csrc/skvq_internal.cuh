@@ -156,6 +156,9 @@ cudaError_t launch_partition_mma(const Shape &s, const CachePtrs &c, const __hal
 cudaError_t launch_partition_gqa(const Shape &s, const CachePtrs &c, const __half *q, float scale_log2,
                                  const SplitPlan &plan, float *workspace, cudaStream_t stream, bool overlap, bool *handled);
 
+cudaError_t launch_partition_tc(const Shape &s, const CachePtrs &c, const __half *q, float scale_log2,
+                                const SplitPlan &plan, float *workspace, cudaStream_t stream, bool overlap, bool *handled);
+
 void count_launch(int n = 1);
 
 }  // namespace skvq
