@@ -492,11 +492,11 @@ cudaError_t launch_attention(const Shape &s, const CachePtrs &c, const __half *q
     cudaError_t em = launch_partition_mma(s, c, q, a.scale_log2, plan, workspace, stream, overlap, &handled);
     if (em != cudaSuccess) return em;
     if (!handled) {
-        em = launch_partition_tc(s, c, q, a.scale_log2, plan, workspace, stream, overlap, &handled);
+        em = launch_partition_gqa(s, c, q, a.scale_log2, plan, workspace, stream, overlap, &handled);
         if (em != cudaSuccess) return em;
     }
     if (!handled) {
-        em = launch_partition_gqa(s, c, q, a.scale_log2, plan, workspace, stream, overlap, &handled);
+        em = launch_partition_tc(s, c, q, a.scale_log2, plan, workspace, stream, overlap, &handled);
         if (em != cudaSuccess) return em;
     }
     if (handled) { /* tensor-core kernel launched */ }

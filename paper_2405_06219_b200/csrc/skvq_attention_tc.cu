@@ -31,28 +31,31 @@ using namespace mmak;
 constexpr int kTile = 128;              // tokens per tile = rows of the score MMA = threads per CTA
 constexpr int kHeads = 4;               // query heads per KV head served (absent heads carry a zero query)
 constexpr int kSlackLog2 = 16;          // the softmax reference moves only when a score exceeds it by this (log2)
-constexpr int kStages = 3;
-constexpr int kTmemCols = 256;          // allocation: scores in columns [0, 64), value sums in [128, 256)
+constexpr int kRing = 3;                // slots of each of the two copy rings
+constexpr int kTmemCols = 256;          // allocation: two score buffers in columns [0, 128), value sums in [128, 256)
 constexpr int kScoreCol = 0, kPvCol = 128;
 constexpr int kFoldTiles = 256;         // 255 * 192 * 128 * 256 < 2^31: the int32 value sums are folded at least this often
 constexpr uint32_t kLbo = 128;          // bytes between core matrices along K (all operands)
 constexpr uint32_t kSboK = 1024;        // K-major operands: bytes between groups of 8 rows
 constexpr uint32_t kSboMN = 2048;       // MN-major operands: bytes between 16-byte chunks of the M/N extent (128 tokens)
 
+// Shared memory.  The K codes of a tile are needed two tiles before everything else of it (its score MMA is issued
+// that far ahead), so they travel in a ring of their own.
 template <int G>
 struct TCfg {
     static constexpr int NG = kHeadDim / G;
     static constexpr int kCodeTile = kTile * kRowBytes;                  // 4096
     static constexpr int kMetaTile = kTile * NG * 4;
-    static constexpr int kStageBytes = 2 * kCodeTile + 2 * kMetaTile;
-    static constexpr int kOffKA = kStages * kStageBytes;                 // A of the score MMA: [128 tokens][128 bytes]
-    static constexpr int kOffQB = kOffKA + kTile * 128;                  // B of the score MMA: [16 (head, digit)][128 bytes]
-    static constexpr int kOffVB = kOffQB + 16 * 128;                     // B of the value MMA, two buffers
-    static constexpr int kOffPA = kOffVB + 2 * kTile * 128;              // A of the value MMA, two buffers of [128 tokens][64 rows]
+    static constexpr int kVmBytes = kCodeTile + 2 * kMetaTile;           // V codes, K scale/zero, V scale/zero
+    static constexpr int kOffVm = kRing * kCodeTile;
+    static constexpr int kOffKA = kOffVm + kRing * kVmBytes;             // A of the score MMA, two buffers of [128 tokens][128 bytes]
+    static constexpr int kOffQB = kOffKA + 2 * kTile * 128;              // B of the score MMA: [16 (head, digit)][128 bytes]
+    static constexpr int kOffVB = kOffQB + 16 * 128;                     // B of the value MMA: [128 tokens][128 bytes]
+    static constexpr int kOffPA = kOffVB + kTile * 128;                  // A of the value MMA, two buffers of [128 tokens][64 rows]
     static constexpr int kOffOs = kOffPA + 2 * kTile * 64;               // folded value sums [4][128] fp32, by MMA column
-    static constexpr int kOffQs = kOffOs + kHeads * kHeadDim * 4;        // prologue scratch [4][128] fp32
-    static constexpr int kOffMisc = kOffQs + kHeads * kHeadDim * 4;      // small arrays, see the kernel
+    static constexpr int kOffMisc = kOffOs + kHeads * kHeadDim * 4;      // small arrays, see the kernel
     static constexpr int kSmemBytes = kOffMisc + 1024;
+    static_assert(kTile * 128 >= kHeads * kHeadDim * 4, "the V operand buffer doubles as query scratch in the prologue");
 };
 
 // ---------------------------------------------------------------- tcgen05 wrappers
@@ -83,8 +86,8 @@ __device__ __forceinline__ void umma_commit(uint32_t bar)
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void proxy_fence() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-// Lane i of the warp receives 16 consecutive 32-bit columns of tensor-memory lane (lane field of addr) + i.
-__device__ __forceinline__ void tmem_ld16(uint32_t addr, int (&r)[16])
+// Lane i of the warp receives N consecutive 32-bit columns of tensor-memory lane (lane field of addr) + i.
+__device__ __forceinline__ void tmem_ld16(uint32_t addr, int *r)
 {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
@@ -165,15 +168,15 @@ __global__ void __launch_bounds__(kTile, 2) partition_tc_kernel(MmaArgs a)
     float *partials = a.ws + a.plan.hdr_ints;
 
     // ---- shared memory
-    uint8_t *KA = smem + C::kOffKA, *QB = smem + C::kOffQB;
+    uint8_t *QB = smem + C::kOffQB, *VB = smem + C::kOffVB;
     float *Os = reinterpret_cast<float *>(smem + C::kOffOs);         // [4][128] by MMA column
-    float *qs = reinterpret_cast<float *>(smem + C::kOffQs);         // [4][128] permuted query (prologue)
-    float *sqs = reinterpret_cast<float *>(smem + C::kOffMisc);      // [4][4]  sm_scale*log2(e) * sum_{j in g} q'_j
-    float *csc = sqs + 16;                                           // [4]     sm_scale*log2(e) * 2^(e_r - 30)
-    int *fexp = reinterpret_cast<int *>(csc + 4);                    // [4]
+    float *qs = reinterpret_cast<float *>(VB);                       // [4][128] permuted query (prologue only)
+    float *sqs_sh = reinterpret_cast<float *>(smem + C::kOffMisc);   // [4][4]  sm_scale*log2(e) * sum_{j in g} q'_j
+    float *csc_sh = sqs_sh + 16;                                     // [4]     sm_scale*log2(e) * 2^(e_r - 30)
+    int *fexp = reinterpret_cast<int *>(csc_sh + 4);                 // [4]
     float *red = reinterpret_cast<float *>(fexp + 4);                // [4 warps][24] reductions
-    uint64_t *bars = reinterpret_cast<uint64_t *>(red + kWarps * 24);   // [kStages] tiles, [1] scores, [2] value MMAs
-    const uint32_t bar_tile = smem_u32(bars), bar_s = bar_tile + 8 * kStages, bar_pv = bar_s + 8;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(red + kWarps * 24);   // K ring, V ring, two score buffers, value MMA
+    const uint32_t bar_k = smem_u32(bars), bar_v = bar_k + 8 * kRing, bar_s = bar_v + 8 * kRing, bar_pv = bar_s + 16;
 
     // ---- tensor memory and barriers (once per CTA)
     if (warp == 0) {
@@ -183,7 +186,7 @@ __global__ void __launch_bounds__(kTile, 2) partition_tc_kernel(MmaArgs a)
     }
     if (tid == 0) {
 #pragma unroll
-        for (int i = 0; i < kStages + 3; ++i) mbar_init(bar_tile + 8 * i, 1);
+        for (int i = 0; i < 2 * kRing + 3; ++i) mbar_init(bar_k + 8 * i, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         proxy_fence();
     }
@@ -195,18 +198,21 @@ __global__ void __launch_bounds__(kTile, 2) partition_tc_kernel(MmaArgs a)
 
     constexpr uint32_t kIdescS = idesc_i8(128, 16, false, true, false, false);
     constexpr uint32_t kIdescPV = idesc_i8(64, 128, false, false, true, true);
+    // operand descriptors (thread 0 issues every MMA); a k-step moves the start address, i.e. the low word
+    const uint64_t dKA = smem_desc(smem_u32(smem + C::kOffKA), kLbo, kSboK), dQB = smem_desc(smem_u32(QB), kLbo, kSboK);
+    const uint64_t dVB = smem_desc(smem_u32(VB), kLbo, kSboMN), dPA = smem_desc(smem_u32(smem + C::kOffPA), kLbo, kSboMN);
 
     // kernel-lifetime pipeline counters (uniform across the CTA)
-    uint32_t tiles_done = 0;           // tiles that went through the stage ring
-    uint32_t s_done = 0;               // completions of the score barrier consumed
-    uint32_t pv_issued0 = 0, pv_issued1 = 0, pv_waited0 = 0, pv_waited1 = 0;      // value MMAs per operand buffer
+    uint32_t tiles_done = 0;           // tiles that went through the rings
+    uint32_t s_issued = 0;             // score MMAs issued = tiles whose K operand was built (buffer = index & 1)
+    uint32_t s_taken = 0;              // score results consumed
+    uint32_t pv_issued = 0, pv_waited = 0;
     bool failed = false;
 
-    auto wait_pv = [&](int buf) {
-        const uint32_t issued = buf ? pv_issued1 : pv_issued0, waited = buf ? pv_waited1 : pv_waited0;
-        if (waited < issued) {
-            if (!mbar_wait_bounded(bar_pv + 8 * buf, (issued - 1) & 1u)) fail_sh = 1;
-            if (buf) pv_waited1 = issued; else pv_waited0 = issued;
+    auto wait_pv = [&]() {             // at most one value MMA is outstanding
+        if (pv_waited < pv_issued) {
+            if (!mbar_wait_bounded(bar_pv, (pv_issued - 1) & 1u)) fail_sh = 1;
+            pv_waited = pv_issued;
         }
     };
 
@@ -222,34 +228,44 @@ __global__ void __launch_bounds__(kTile, 2) partition_tc_kernel(MmaArgs a)
     const __half2 *v_meta = a.c.v_meta + bh * (size_t)s.cap * NG;
     const int n_tiles = failed ? 0 : (q_end - q_begin + kTile - 1) / kTile;
 
-    auto issue_tile = [&](int i) {      // thread 0 only: tile i of this segment into its stage
-        const uint32_t st = (tiles_done + i) % kStages;
+    // thread 0 only: the copies of tile i of this segment (the cache's capacity is a multiple of 64 rows)
+    auto rows_of = [&](int i) { return (uint32_t)min(kTile, (q_end - (q_begin + i * kTile) + 63) & ~63); };
+    auto issue_k = [&](int i) {
+        const uint32_t slot = (tiles_done + i) % kRing, rows = rows_of(i);
+        mbar_expect_tx(bar_k + 8 * slot, rows * kRowBytes);
+        bulk_g2s(smem_u32(smem + slot * C::kCodeTile), k_codes + (size_t)(q_begin + i * kTile) * kRowBytes, rows * kRowBytes,
+                 bar_k + 8 * slot);
+    };
+    auto issue_v = [&](int i) {
+        const uint32_t slot = (tiles_done + i) % kRing, rows = rows_of(i);
         const int tok0 = q_begin + i * kTile;
-        const uint32_t rows = (uint32_t)min(kTile, (q_end - tok0 + 63) & ~63);      // the cache's capacity is a multiple of 64
-        const uint32_t dst = smem_u32(smem + st * C::kStageBytes);
-        const uint32_t bar = bar_tile + 8 * st;
-        mbar_expect_tx(bar, rows * (2 * kRowBytes + 2 * NG * 4));
-        bulk_g2s(dst, k_codes + (size_t)tok0 * kRowBytes, rows * kRowBytes, bar);
-        bulk_g2s(dst + C::kCodeTile, v_codes + (size_t)tok0 * kRowBytes, rows * kRowBytes, bar);
-        bulk_g2s(dst + 2 * C::kCodeTile, k_meta + (size_t)tok0 * NG, rows * NG * 4, bar);
-        bulk_g2s(dst + 2 * C::kCodeTile + C::kMetaTile, v_meta + (size_t)tok0 * NG, rows * NG * 4, bar);
+        const uint32_t dst = smem_u32(smem + C::kOffVm + slot * C::kVmBytes), bar = bar_v + 8 * slot;
+        mbar_expect_tx(bar, rows * (kRowBytes + 2 * NG * 4));
+        bulk_g2s(dst, v_codes + (size_t)tok0 * kRowBytes, rows * kRowBytes, bar);
+        bulk_g2s(dst + C::kCodeTile, k_meta + (size_t)tok0 * NG, rows * NG * 4, bar);
+        bulk_g2s(dst + C::kCodeTile + C::kMetaTile, v_meta + (size_t)tok0 * NG, rows * NG * 4, bar);
     };
-    auto wait_tile = [&](int i) {
+    auto wait_ring = [&](uint32_t bar0, int i) {
         const uint32_t t = tiles_done + i;
-        if (!mbar_wait_bounded(bar_tile + 8 * (t % kStages), (t / kStages) & 1u)) fail_sh = 1;
+        if (!mbar_wait_bounded(bar0 + 8 * (t % kRing), (t / kRing) & 1u)) fail_sh = 1;
     };
-    auto stage_of = [&](int i) { return smem + ((tiles_done + i) % kStages) * C::kStageBytes; };
-    auto issue_scores = [&]() {         // thread 0 only
+    // every thread: its token's row of tile i -> A operand of the score MMA (buffer = parity of the score MMA count)
+    auto build_k = [&](int i, uint32_t sbuf) {
+        wait_ring(bar_k, i);
+        unpack_row(smem + ((tiles_done + i) % kRing) * C::kCodeTile + tid * kRowBytes,
+                   smem + C::kOffKA + sbuf * (kTile * 128) + (tid >> 3) * kSboK + (tid & 7) * 16, kLbo);
+    };
+    auto issue_scores = [&](uint32_t sbuf) {         // thread 0 only
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks)
-            umma_i8(tmem + kScoreCol + 16 * ((32 * ks) / G), smem_desc(smem_u32(KA) + ks * 2 * kLbo, kLbo, kSboK),
-                    smem_desc(smem_u32(QB) + ks * 2 * kLbo, kLbo, kSboK), kIdescS, ((32 * ks) % G) != 0 ? 1u : 0u);
-        umma_commit(bar_s);
+            umma_i8(tmem + kScoreCol + 64 * sbuf + 16 * ((32 * ks) / G), dKA + ((sbuf * (kTile * 128) + ks * 2 * kLbo) >> 4),
+                    dQB + ((ks * 2 * kLbo) >> 4), kIdescS, ((32 * ks) % G) != 0 ? 1u : 0u);
+        umma_commit(bar_s + 8 * sbuf);
     };
 
     if (tid == 0) {      // the first copies are in flight while the query is prepared
-        proxy_fence();   // the stages were read through the generic proxy by the previous segment
-        for (int i = 0; i < kStages && i < n_tiles; ++i) issue_tile(i);
+        proxy_fence();   // the slots were read through the generic proxy by the previous segment
+        for (int i = 0; i < kRing && i < n_tiles; ++i) { issue_k(i); issue_v(i); }
     }
 
     // ---- CTA-wide prologue: permuted query per head on a power-of-two scale -> byte digits, group constants
@@ -272,13 +288,13 @@ __global__ void __launch_bounds__(kTile, 2) partition_tc_kernel(MmaArgs a)
         int e = 0;
         if (qmax > 0.f) (void)frexpf(qmax, &e);            // qmax = m * 2^e, 0.5 <= m < 1: |q' * 2^-e| < 1
         fexp[tid] = e;
-        csc[tid] = ldexpf(a.scale_log2, e - 30);
+        csc_sh[tid] = ldexpf(a.scale_log2, e - 30);
     }
     if (tid >= 32 && tid < 32 + kHeads * NG) {
         const int r = (tid - 32) / NG, gg = (tid - 32) % NG;
         float sq = 0.f;
         for (int j = gg * G; j < (gg + 1) * G; ++j) sq += qs[r * kHeadDim + j];
-        sqs[r * 4 + gg] = sq * a.scale_log2;
+        sqs_sh[r * 4 + gg] = sq * a.scale_log2;
     }
     __syncthreads();
     {
@@ -297,6 +313,13 @@ __global__ void __launch_bounds__(kTile, 2) partition_tc_kernel(MmaArgs a)
             }
         }
     }
+    float csc[kHeads], sqs[kHeads][NG];
+#pragma unroll
+    for (int r = 0; r < kHeads; ++r) {
+        csc[r] = csc_sh[r];
+#pragma unroll
+        for (int gg = 0; gg < NG; ++gg) sqs[r][gg] = sqs_sh[r * 4 + gg];
+    }
 
     // ---- running state: this thread's token of every tile, all four heads
     float m_ref[kHeads], l_sum[kHeads], zp[kHeads][NG];
@@ -308,13 +331,13 @@ __global__ void __launch_bounds__(kTile, 2) partition_tc_kernel(MmaArgs a)
         for (int gg = 0; gg < NG; ++gg) zp[r][gg] = 0.f;
     }
     float h_bound = 6.103515625e-05f;      // power of two above every value scale seen so far (2^-14 to start with)
+    float hscale = (float)(1u << (32 - kSlackLog2)) / h_bound;
     bool pv_fresh = true;                  // the next value MMA overwrites the accumulators
     int tiles_since_fold = 0;
 
     // Brings the int32 value sums into the fp32 sums in shared memory (relative to the old references and bound).
     auto fold_pv = [&]() {
-        wait_pv(0);
-        wait_pv(1);
+        wait_pv();
         tc_fence_after();
         if (!pv_fresh && warp < NG) {
             // lanes 0-15 of this warp's tensor-memory lanes hold rows (group = warp, head = lane / 4, digit = lane % 4)
@@ -338,53 +361,55 @@ __global__ void __launch_bounds__(kTile, 2) partition_tc_kernel(MmaArgs a)
         tiles_since_fold = 0;
     };
 
-    // ---- first tile: unpack K and start its score MMA
-    if (n_tiles > 0) {
-        wait_tile(0);
-        unpack_row(stage_of(0) + tid * kRowBytes, KA + (tid >> 3) * kSboK + (tid & 7) * 16, kLbo);
-    }
+    // ---- the first two tiles' K operands and score MMAs (the query scratch in the V buffer is dead after the barrier)
+    const uint32_t s_base = s_issued;      // score MMA index of tile 0 of this segment
+    if (n_tiles > 0) build_k(0, s_base & 1u);
+    if (n_tiles > 1) build_k(1, (s_base + 1) & 1u);
     proxy_fence();
     __syncthreads();
     if (fail_sh) failed = true;
-    if (tid == 0 && n_tiles > 0 && !failed) issue_scores();
+    if (tid == 0 && !failed) {
+        if (n_tiles > 0) issue_scores(s_base & 1u);
+        if (n_tiles > 1) issue_scores((s_base + 1) & 1u);
+        proxy_fence();
+        if (n_tiles > kRing) issue_k(kRing);
+        if (n_tiles > kRing + 1) issue_k(kRing + 1);
+    }
+    s_issued += (uint32_t)min(n_tiles, 2);
 
+    int i_stop = 0;      // first tile that was not completed (for the bounded drain after a failure)
     for (int i = 0; i < n_tiles && !failed; ++i) {
-        const int buf = i & 1;
-        uint8_t *stg = stage_of(i);
-        const uint32_t *Km = reinterpret_cast<const uint32_t *>(stg + 2 * C::kCodeTile);       // [128][NG] words {h, z}
-        const uint32_t *Vm = reinterpret_cast<const uint32_t *>(stg + 2 * C::kCodeTile + C::kMetaTile);
-        uint8_t *VB = smem + C::kOffVB + buf * (kTile * 128);
-        uint8_t *PA = smem + C::kOffPA + buf * (kTile * 64);
+        i_stop = i;
+        const uint32_t sbuf = (s_base + i) & 1u;
+        const uint8_t *vm = smem + C::kOffVm + ((tiles_done + i) % kRing) * C::kVmBytes;
+        const uint32_t *Km = reinterpret_cast<const uint32_t *>(vm + C::kCodeTile);                      // [128][NG] words {h, z}
+        const uint32_t *Vm = reinterpret_cast<const uint32_t *>(vm + C::kCodeTile + C::kMetaTile);
+        uint8_t *PA = smem + C::kOffPA + (i & 1) * (kTile * 64);
         const int tok = q_begin + i * kTile + tid;
         const bool valid = tok < q_end && tok >= s.n_sink;      // sinks belong to the merge kernel
 
-        // ---------------- V tile -> B operand of the value MMA (its buffer was last read by the MMA two tiles ago)
-        wait_pv(buf);
-        unpack_row(stg + C::kCodeTile + tid * kRowBytes, VB + (tid >> 3) * kLbo + (tid & 7) * 16, kSboMN);
-
-        // ---------------- scores of this thread's token
-        if (!mbar_wait_bounded(bar_s, s_done & 1u)) fail_sh = 1;
-        ++s_done;
+        // ---------------- scores of this thread's token (the MMA was issued two tiles ago)
+        if (!mbar_wait_bounded(bar_s + 8 * sbuf, (s_taken >> 1) & 1u)) fail_sh = 1;
+        ++s_taken;
         tc_fence_after();
+        int v[NG][16];
+#pragma unroll
+        for (int gg = 0; gg < NG; ++gg) tmem_ld16(tmem_row + kScoreCol + 64 * sbuf + 16 * gg, v[gg]);
+        wait_ring(bar_v, i);
         uint32_t kw[NG], vw[NG];
         load_words<NG>(Km + tid * NG, kw);
         load_words<NG>(Vm + tid * NG, vw);
-        float sc[kHeads];
-#pragma unroll
-        for (int r = 0; r < kHeads; ++r) sc[r] = 0.f;
-        float zt[kHeads] = {0.f, 0.f, 0.f, 0.f};
+        tmem_wait_ld();
+        float sc[kHeads] = {0.f, 0.f, 0.f, 0.f}, zt[kHeads] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int gg = 0; gg < NG; ++gg) {
-            int v[16];
-            tmem_ld16(tmem_row + kScoreCol + 16 * gg, v);
-            tmem_wait_ld();
             const float hk_ = lo_half(kw[gg]), zk_ = hi_half(kw[gg]);
 #pragma unroll
             for (int r = 0; r < kHeads; ++r) {
-                const int lo = v[4 * r] + (v[4 * r + 1] << 8), hi = v[4 * r + 2] + (v[4 * r + 3] << 8);
+                const int lo = v[gg][4 * r] + (v[gg][4 * r + 1] << 8), hi = v[gg][4 * r + 2] + (v[gg][4 * r + 3] << 8);
                 const float u = fmaf((float)hi, 65536.0f, (float)lo);      // 2^30 * sum_j q'_j 2^-e c_j over the group
                 sc[r] = fmaf(hk_, u, sc[r]);
-                zt[r] = fmaf(zk_, sqs[r * 4 + gg], zt[r]);
+                zt[r] = fmaf(zk_, sqs[r][gg], zt[r]);
             }
         }
         float hmax = 0.f;
@@ -396,14 +421,13 @@ __global__ void __launch_bounds__(kTile, 2) partition_tc_kernel(MmaArgs a)
             hmax = fmaxf(hmax, hv[gg]);
         }
         float arg[kHeads];
-        bool need = hmax >= h_bound;
+        bool need = hmax >= h_bound || tiles_since_fold >= kFoldTiles;
 #pragma unroll
         for (int r = 0; r < kHeads; ++r) {
             sc[r] = valid ? fmaf(sc[r], csc[r], zt[r]) : -CUDART_INF_F;      // log2 domain
-            arg[r] = sc[r] - m_ref[r];
-            need |= valid && (arg[r] > (float)kSlackLog2 || m_ref[r] == -CUDART_INF_F);
+            arg[r] = sc[r] - m_ref[r];                                      // +inf while the head has no reference yet
+            need |= valid && arg[r] > (float)kSlackLog2;
         }
-        need |= tiles_since_fold >= kFoldTiles;
         tc_fence_before();
         const int moved = __syncthreads_or(need ? 1 : 0);
         if (fail_sh) { failed = true; break; }
@@ -420,28 +444,29 @@ __global__ void __launch_bounds__(kTile, 2) partition_tc_kernel(MmaArgs a)
             fold_pv();
             __syncthreads();
             if (fail_sh) { failed = true; break; }
-            float corr[kHeads];
 #pragma unroll
             for (int r = 0; r < kHeads; ++r) {
                 float mx = m_ref[r];
                 for (int w = 0; w < kWarps; ++w) mx = fmaxf(mx, red[w * 24 + r]);
-                corr[r] = mx == -CUDART_INF_F ? 1.f : ex2_approx(m_ref[r] - mx);      // 0 on the first tile with a token
+                const float corr = mx == -CUDART_INF_F ? 1.f : ex2_approx(m_ref[r] - mx);      // 0 on the first tile with a token
                 m_ref[r] = mx;
-                l_sum[r] *= corr[r];
+                l_sum[r] *= corr;
 #pragma unroll
-                for (int gg = 0; gg < NG; ++gg) zp[r][gg] *= corr[r];
-                Os[r * kHeadDim + tid] *= corr[r];
+                for (int gg = 0; gg < NG; ++gg) zp[r][gg] *= corr;
+                Os[r * kHeadDim + tid] *= corr;
                 arg[r] = sc[r] - m_ref[r];
             }
             hm = 0.f;
             for (int w = 0; w < kWarps; ++w) hm = fmaxf(hm, red[w * 24 + 4]);
-            if (hm >= h_bound) h_bound = __int_as_float(((__float_as_int(hm) >> 23) + 1) << 23);   // next power of two above
+            if (hm >= h_bound) {
+                h_bound = __int_as_float(((__float_as_int(hm) >> 23) + 1) << 23);   // next power of two above
+                hscale = (float)(1u << (32 - kSlackLog2)) / h_bound;
+            }
             __syncthreads();      // red is rewritten by the next move
         }
 
-        // ---------------- p and the digits of p*h -> A operand of the value MMA
+        // ---------------- p and the digits of p*h -> A operand of the value MMA (buffer last read two tiles ago)
         {
-            const float hscale = (float)(1u << (32 - kSlackLog2)) / h_bound;
             float ps[kHeads];
 #pragma unroll
             for (int r = 0; r < kHeads; ++r) {
@@ -458,11 +483,13 @@ __global__ void __launch_bounds__(kTile, 2) partition_tc_kernel(MmaArgs a)
                                to_fixed_u32(ps[3] * hv[gg]));
         }
 
-        // ---------------- next tile's K -> A operand of the score MMA (this tile's score MMA has completed)
-        if (i + 1 < n_tiles) {
-            wait_tile(i + 1);
-            unpack_row(stage_of(i + 1) + tid * kRowBytes, KA + (tid >> 3) * kSboK + (tid & 7) * 16, kLbo);
-        }
+        // ---------------- K of the tile after next -> the A operand buffer this tile's score MMA has just released
+        if (i + 2 < n_tiles) build_k(i + 2, sbuf);
+
+        // ---------------- V tile -> B operand of the value MMA, once the previous value MMA has read the buffer
+        wait_pv();
+        unpack_row(vm + tid * kRowBytes, VB + (tid >> 3) * kLbo + (tid & 7) * 16, kSboMN);
+
         proxy_fence();
         __syncthreads();
         if (fail_sh) { failed = true; break; }
@@ -470,16 +497,16 @@ __global__ void __launch_bounds__(kTile, 2) partition_tc_kernel(MmaArgs a)
             tc_fence_after();
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks)
-                umma_i8(tmem + kPvCol, smem_desc(smem_u32(PA) + ks * 4 * kLbo, kLbo, kSboMN),
-                        smem_desc(smem_u32(VB) + ks * 4 * kLbo, kLbo, kSboMN), kIdescPV, (pv_fresh && ks == 0) ? 0u : 1u);
-            umma_commit(bar_pv + 8 * buf);
-            if (i + 1 < n_tiles) issue_scores();
-            if (i + kStages < n_tiles) {
-                proxy_fence();      // the stage was read through the generic proxy
-                issue_tile(i + kStages);
-            }
+                umma_i8(tmem + kPvCol, dPA + (((i & 1) * (kTile * 64) + ks * 4 * kLbo) >> 4), dVB + ((ks * 4 * kLbo) >> 4), kIdescPV,
+                        (pv_fresh && ks == 0) ? 0u : 1u);
+            umma_commit(bar_pv);
+            if (i + 2 < n_tiles) issue_scores(sbuf);
+            proxy_fence();      // the slots were read through the generic proxy
+            if (i + kRing < n_tiles) issue_v(i + kRing);
+            if (i + 2 + kRing < n_tiles) issue_k(i + 2 + kRing);
         }
-        if (buf) ++pv_issued1; else ++pv_issued0;
+        ++pv_issued;
+        if (i + 2 < n_tiles) ++s_issued;
         pv_fresh = false;
         ++tiles_since_fold;
     }
@@ -487,7 +514,7 @@ __global__ void __launch_bounds__(kTile, 2) partition_tc_kernel(MmaArgs a)
     // ---- end of the segment: last fold, CTA-wide sums, one partial per query head
     if (failed) {
         // let whatever is still in flight land (bounded), then report
-        for (int i = 0; i < n_tiles; ++i) wait_tile(i);
+        for (int i = i_stop; i < n_tiles && i < i_stop + kRing + 3; ++i) { wait_ring(bar_k, i); wait_ring(bar_v, i); }
         if (tid == 0 && a.c.status) atomicOr(a.c.status, SKVQ_STATUS_COPY_TIMEOUT);
     }
     fold_pv();

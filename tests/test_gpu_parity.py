@@ -121,6 +121,9 @@ def test_ragged_append_and_overflow_flag():
     (4, dict(context=2777, batch=2, ragged=None, n_q_heads=4, n_kv_heads=4, k_bits=2, v_bits=4, group_size=128), 2777),
     (4, dict(context=3100, batch=1, ragged=None, n_q_heads=4, n_kv_heads=4, group_size=128, window=128), 3100),   # 4-bit, one group
     (4, dict(context=2000, batch=1, ragged=None, n_q_heads=8, n_kv_heads=4), 2000),      # 4-bit with 2 heads per KV head: scalar kernel
+    (2, dict(context=5300, batch=2, ragged=None, n_q_heads=12, n_kv_heads=4), 5300),     # 3 heads per KV head, g32: tcgen05 kernel
+    (1, dict(context=70000, batch=1, n_q_heads=6, n_kv_heads=2), 70000),                 # 3 heads per KV head, g128, many tiles per CTA
+    (2, dict(context=1000, batch=33, ragged=(1, 1000), n_q_heads=3, n_kv_heads=1, group_size=64), 1000),   # 3 heads, g64, plan kernel, short and empty prefixes
 ])
 def test_attention_matches_oracle(cfg_i, kw, n):
     w = small(cfg_i, **kw)
@@ -141,6 +144,7 @@ def test_attention_matches_oracle(cfg_i, kw, n):
     (2, dict(context=800, batch=1, n_q_heads=16, n_kv_heads=2, n_sink=7), 800),               # scalar kernel
     (2, dict(context=900, batch=2, ragged=None, n_sink=64), 900),                             # grouped-query kernel, first tile all sinks
     (2, dict(context=700, batch=1, n_q_heads=16, n_kv_heads=2, n_sink=64), 700),              # scalar kernel, first tile all sinks
+    (2, dict(context=1900, batch=1, n_q_heads=6, n_kv_heads=2, n_sink=9), 1900),              # tcgen05 kernel (3 heads per KV head)
     (0, dict(context=130, n_sink=5), 130),                                                    # fewer tokens out of the window than sinks
     (0, dict(context=300, window=0, n_sink=3), 300),
 ])
