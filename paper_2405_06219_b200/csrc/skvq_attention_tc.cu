@@ -136,14 +136,29 @@ __device__ __forceinline__ void unpack_row(const uint8_t *packed, uint8_t *dst, 
 __device__ __forceinline__ int column_channel(int n) { return 16 * (n >> 4) + ((n >> 2) & 3) + 4 * (n & 3); }
 __device__ __forceinline__ int column_shift(int n) { return 2 * ((n >> 2) & 3); }
 
+// Barrier 1: the 128 token threads only (the control warp never joins it).
+__device__ __forceinline__ void token_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ int token_sync_or(int pred)
+{
+    int out;
+    asm volatile("{\n .reg .pred p, q;\n setp.ne.u32 q, %1, 0;\n bar.red.or.pred p, 1, 128, q;\n selp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(out) : "r"(pred) : "memory");
+    return out;
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
 template <int G>
-__global__ void __launch_bounds__(kTile, 2) partition_tc_kernel(MmaArgs a)
+__global__ void __launch_bounds__(kTile + 32, 2) partition_tc_kernel(MmaArgs a)
 {
     using C = TCfg<G>;
     constexpr int NG = C::NG;
     extern __shared__ __align__(128) uint8_t smem[];
     const Shape &s = a.s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const bool control = warp == kWarps;      // warp 4 issues every copy and MMA; warps 0-3 own one token each
     const int R = s.rep;
     asm volatile("griddepcontrol.launch_dependents;");      // the merge kernel may start its window part early
     asm volatile("griddepcontrol.wait;" ::: "memory");      // the lengths, and the plan kernel's header when there is one
@@ -151,6 +166,7 @@ __global__ void __launch_bounds__(kTile, 2) partition_tc_kernel(MmaArgs a)
     __shared__ __align__(16) Segment seg_sh;
     __shared__ int more_sh;
     __shared__ int fail_sh;
+    __shared__ int fresh_sh[2];      // does the value MMA of an even / odd tile overwrite the accumulators?
     __shared__ uint32_t tmem_sh;
     __shared__ SlotWalker walk;      // only thread 0 touches it
     __shared__ __align__(16) int hdr_sh[kPlanSmemInts];
@@ -175,46 +191,42 @@ __global__ void __launch_bounds__(kTile, 2) partition_tc_kernel(MmaArgs a)
     float *csc_sh = sqs_sh + 16;                                     // [4]     sm_scale*log2(e) * 2^(e_r - 30)
     int *fexp = reinterpret_cast<int *>(csc_sh + 4);                 // [4]
     float *red = reinterpret_cast<float *>(fexp + 4);                // [4 warps][24] reductions
-    uint64_t *bars = reinterpret_cast<uint64_t *>(red + kWarps * 24);   // K ring, V ring, two score buffers, value MMA
-    const uint32_t bar_k = smem_u32(bars), bar_v = bar_k + 8 * kRing, bar_s = bar_v + 8 * kRing, bar_pv = bar_s + 16;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(red + kWarps * 24);
+    const uint32_t bar_k = smem_u32(bars);            // [kRing] K codes landed (copy)
+    const uint32_t bar_v = bar_k + 8 * kRing;         // [kRing] V codes and scale/zero landed (copy)
+    const uint32_t bar_s = bar_v + 8 * kRing;         // [2] score MMA done (tcgen05.commit)
+    const uint32_t bar_pv = bar_s + 16;               // [1] value MMA done (tcgen05.commit)
+    const uint32_t bar_ka = bar_pv + 8;               // [2] A operand of a score MMA built (128 token threads)
+    const uint32_t bar_pa = bar_ka + 16;              // [1] operands of a value MMA built (128 token threads)
 
     // ---- tensor memory and barriers (once per CTA)
-    if (warp == 0) {
+    if (control) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_sh)), "r"(kTmemCols)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    if (tid == 0) {
+        if (lane == 0) {
 #pragma unroll
-        for (int i = 0; i < 2 * kRing + 3; ++i) mbar_init(bar_k + 8 * i, 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        proxy_fence();
+            for (int i = 0; i < 2 * kRing + 3; ++i) mbar_init(bar_k + 8 * i, 1);
+#pragma unroll
+            for (int i = 0; i < 3; ++i) mbar_init(bar_ka + 8 * i, kTile);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            proxy_fence();
+        }
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = tmem_sh;
-    const uint32_t tmem_row = tmem + ((uint32_t)(warp * 32) << 16);      // this warp's 32 lanes
+    const uint32_t tmem_row = tmem + ((uint32_t)((warp & 3) * 32) << 16);      // this warp's 32 lanes
 
     constexpr uint32_t kIdescS = idesc_i8(128, 16, false, true, false, false);
     constexpr uint32_t kIdescPV = idesc_i8(64, 128, false, false, true, true);
-    // operand descriptors (thread 0 issues every MMA); a k-step moves the start address, i.e. the low word
-    const uint64_t dKA = smem_desc(smem_u32(smem + C::kOffKA), kLbo, kSboK), dQB = smem_desc(smem_u32(QB), kLbo, kSboK);
-    const uint64_t dVB = smem_desc(smem_u32(VB), kLbo, kSboMN), dPA = smem_desc(smem_u32(smem + C::kOffPA), kLbo, kSboMN);
 
-    // kernel-lifetime pipeline counters (uniform across the CTA)
+    // kernel-lifetime pipeline counters (every thread counts alike)
     uint32_t tiles_done = 0;           // tiles that went through the rings
-    uint32_t s_issued = 0;             // score MMAs issued = tiles whose K operand was built (buffer = index & 1)
-    uint32_t s_taken = 0;              // score results consumed
-    uint32_t pv_issued = 0, pv_waited = 0;
+    uint32_t s_count = 0;              // score MMAs of finished segments (buffer and barrier phase follow from the index)
+    uint32_t pv_count = 0;             // value MMAs of finished segments
     bool failed = false;
-
-    auto wait_pv = [&]() {             // at most one value MMA is outstanding
-        if (pv_waited < pv_issued) {
-            if (!mbar_wait_bounded(bar_pv, (pv_issued - 1) & 1u)) fail_sh = 1;
-            pv_waited = pv_issued;
-        }
-    };
 
     for (;;) {
     if (tid == 0) seg_sh = walk.next(a.c.lengths, s.W, a.plan.lq_cap);
@@ -222,21 +234,22 @@ __global__ void __launch_bounds__(kTile, 2) partition_tc_kernel(MmaArgs a)
     const int b = seg_sh.b, hk = seg_sh.hk, q_begin = seg_sh.tok_begin, q_end = seg_sh.tok_end, part = seg_sh.part;
     const int n_parts = a.plan.s_max;
     const size_t bh = (size_t)b * s.Hkv + hk;
-    const uint8_t *k_codes = a.c.k_codes + bh * (size_t)s.cap * kRowBytes;
-    const uint8_t *v_codes = a.c.v_codes + bh * (size_t)s.cap * kRowBytes;
-    const __half2 *k_meta = a.c.k_meta + bh * (size_t)s.cap * NG;
-    const __half2 *v_meta = a.c.v_meta + bh * (size_t)s.cap * NG;
     const int n_tiles = failed ? 0 : (q_end - q_begin + kTile - 1) / kTile;
 
-    // thread 0 only: the copies of tile i of this segment (the cache's capacity is a multiple of 64 rows)
+    // ---- CTA-wide prologue: permuted query per head on a power-of-two scale -> byte digits, group constants.
+    // The control warp starts the first copies meanwhile.
     auto rows_of = [&](int i) { return (uint32_t)min(kTile, (q_end - (q_begin + i * kTile) + 63) & ~63); };
-    auto issue_k = [&](int i) {
+    auto issue_k = [&](int i) {       // control lane only (the cache's capacity is a multiple of 64 rows)
+        const uint8_t *k_codes = a.c.k_codes + bh * (size_t)s.cap * kRowBytes;
         const uint32_t slot = (tiles_done + i) % kRing, rows = rows_of(i);
         mbar_expect_tx(bar_k + 8 * slot, rows * kRowBytes);
         bulk_g2s(smem_u32(smem + slot * C::kCodeTile), k_codes + (size_t)(q_begin + i * kTile) * kRowBytes, rows * kRowBytes,
                  bar_k + 8 * slot);
     };
-    auto issue_v = [&](int i) {
+    auto issue_v = [&](int i) {       // control lane only
+        const uint8_t *v_codes = a.c.v_codes + bh * (size_t)s.cap * kRowBytes;
+        const __half2 *k_meta = a.c.k_meta + bh * (size_t)s.cap * NG;
+        const __half2 *v_meta = a.c.v_meta + bh * (size_t)s.cap * NG;
         const uint32_t slot = (tiles_done + i) % kRing, rows = rows_of(i);
         const int tok0 = q_begin + i * kTile;
         const uint32_t dst = smem_u32(smem + C::kOffVm + slot * C::kVmBytes), bar = bar_v + 8 * slot;
@@ -249,27 +262,12 @@ __global__ void __launch_bounds__(kTile, 2) partition_tc_kernel(MmaArgs a)
         const uint32_t t = tiles_done + i;
         if (!mbar_wait_bounded(bar0 + 8 * (t % kRing), (t / kRing) & 1u)) fail_sh = 1;
     };
-    // every thread: its token's row of tile i -> A operand of the score MMA (buffer = parity of the score MMA count)
-    auto build_k = [&](int i, uint32_t sbuf) {
-        wait_ring(bar_k, i);
-        unpack_row(smem + ((tiles_done + i) % kRing) * C::kCodeTile + tid * kRowBytes,
-                   smem + C::kOffKA + sbuf * (kTile * 128) + (tid >> 3) * kSboK + (tid & 7) * 16, kLbo);
-    };
-    auto issue_scores = [&](uint32_t sbuf) {         // thread 0 only
-#pragma unroll
-        for (int ks = 0; ks < 4; ++ks)
-            umma_i8(tmem + kScoreCol + 64 * sbuf + 16 * ((32 * ks) / G), dKA + ((sbuf * (kTile * 128) + ks * 2 * kLbo) >> 4),
-                    dQB + ((ks * 2 * kLbo) >> 4), kIdescS, ((32 * ks) % G) != 0 ? 1u : 0u);
-        umma_commit(bar_s + 8 * sbuf);
-    };
-
-    if (tid == 0) {      // the first copies are in flight while the query is prepared
-        proxy_fence();   // the slots were read through the generic proxy by the previous segment
-        for (int i = 0; i < kRing && i < n_tiles; ++i) { issue_k(i); issue_v(i); }
-    }
-
-    // ---- CTA-wide prologue: permuted query per head on a power-of-two scale -> byte digits, group constants
-    {
+    if (control) {
+        if (lane == 0) {
+            proxy_fence();   // the slots were read through the generic proxy by the previous segment
+            for (int i = 0; i < kRing && i < n_tiles; ++i) { issue_k(i); issue_v(i); }
+        }
+    } else {
         const int32_t *idx_k = a.c.reorder_k + (size_t)hk * kHeadDim;
         const int src = idx_k[tid] & (kHeadDim - 1);
 #pragma unroll
@@ -297,266 +295,301 @@ __global__ void __launch_bounds__(kTile, 2) partition_tc_kernel(MmaArgs a)
         sqs_sh[r * 4 + gg] = sq * a.scale_log2;
     }
     __syncthreads();
-    {
-        // thread = byte column k of the operand: channel column_channel(k), weight 4^j divided out of the query
-        const int ch = column_channel(tid), sh = column_shift(tid);
-        uint8_t *col = QB + (tid >> 4) * kLbo + (tid & 15);
+
+    if (control) {
+        // ================================================================ control warp: one lane issues, in the order
+        // in which the token threads finish the operands
+        if (lane == 0 && n_tiles > 0) {
+            const uint64_t dKA = smem_desc(smem_u32(smem + C::kOffKA), kLbo, kSboK), dQB = smem_desc(smem_u32(QB), kLbo, kSboK);
+            const uint64_t dVB = smem_desc(smem_u32(VB), kLbo, kSboMN), dPA = smem_desc(smem_u32(smem + C::kOffPA), kLbo, kSboMN);
+            bool ok = true;
+            auto scores = [&](int j) {      // score MMA of tile j, once its A operand is complete
+                const uint32_t n = s_count + j, sbuf = n & 1u;
+                if (!mbar_wait_bounded(bar_ka + 8 * sbuf, (n >> 1) & 1u)) { ok = false; return; }
+                tc_fence_after();
 #pragma unroll
-        for (int r = 0; r < kHeads; ++r) {
-            int qi = __float2int_rn(ldexpf(qs[r * kHeadDim + ch], 30 - fexp[r] - sh));      // |qi| < 2^30
+                for (int ks = 0; ks < 4; ++ks)
+                    umma_i8(tmem + kScoreCol + 64 * sbuf + 16 * ((32 * ks) / G), dKA + ((sbuf * (kTile * 128) + ks * 2 * kLbo) >> 4),
+                            dQB + ((ks * 2 * kLbo) >> 4), kIdescS, ((32 * ks) % G) != 0 ? 1u : 0u);
+                umma_commit(bar_s + 8 * sbuf);
+                if (j + kRing < n_tiles) { proxy_fence(); issue_k(j + kRing); }      // the token threads are done with that slot
+            };
+            scores(0);
+            if (ok && n_tiles > 1) scores(1);
+            for (int i = 0; i < n_tiles && ok; ++i) {
+                if (i + 2 < n_tiles) scores(i + 2);
+                if (!ok) break;
+                const uint32_t n = pv_count + i;
+                if (!mbar_wait_bounded(bar_pa, n & 1u)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t fresh = (uint32_t)fresh_sh[i & 1];
 #pragma unroll
-            for (int d = 0; d < 4; ++d) {
-                const int dg = d < 3 ? ((qi + 128) & 255) - 128 : qi;      // balanced digits: qi = sum dg * 256^d
-                qi = (qi - dg) >> 8;
-                const int n = 4 * r + d;
-                col[(n >> 3) * kSboK + (n & 7) * 16] = (uint8_t)(dg & 255);
+                for (int ks = 0; ks < 4; ++ks)
+                    umma_i8(tmem + kPvCol, dPA + (((i & 1) * (kTile * 64) + ks * 4 * kLbo) >> 4), dVB + ((ks * 4 * kLbo) >> 4), kIdescPV,
+                            (fresh && ks == 0) ? 0u : 1u);
+                umma_commit(bar_pv);
+                if (i + kRing < n_tiles) { proxy_fence(); issue_v(i + kRing); }
             }
+            if (!ok) fail_sh = 1;
         }
-    }
-    float csc[kHeads], sqs[kHeads][NG];
+        __syncwarp();
+    } else {
+        // ================================================================ token threads
+        {
+            // thread = byte column k of the operand: channel column_channel(k), weight 4^j divided out of the query
+            const int ch = column_channel(tid), sh = column_shift(tid);
+            uint8_t *col = QB + (tid >> 4) * kLbo + (tid & 15);
 #pragma unroll
-    for (int r = 0; r < kHeads; ++r) {
-        csc[r] = csc_sh[r];
+            for (int r = 0; r < kHeads; ++r) {
+                int qi = __float2int_rn(ldexpf(qs[r * kHeadDim + ch], 30 - fexp[r] - sh));      // |qi| < 2^30
 #pragma unroll
-        for (int gg = 0; gg < NG; ++gg) sqs[r][gg] = sqs_sh[r * 4 + gg];
-    }
-
-    // ---- running state: this thread's token of every tile, all four heads
-    float m_ref[kHeads], l_sum[kHeads], zp[kHeads][NG];
-#pragma unroll
-    for (int r = 0; r < kHeads; ++r) {
-        m_ref[r] = -CUDART_INF_F;
-        l_sum[r] = 0.f;
-#pragma unroll
-        for (int gg = 0; gg < NG; ++gg) zp[r][gg] = 0.f;
-    }
-    float h_bound = 6.103515625e-05f;      // power of two above every value scale seen so far (2^-14 to start with)
-    float hscale = (float)(1u << (32 - kSlackLog2)) / h_bound;
-    bool pv_fresh = true;                  // the next value MMA overwrites the accumulators
-    int tiles_since_fold = 0;
-
-    // Brings the int32 value sums into the fp32 sums in shared memory (relative to the old references and bound).
-    auto fold_pv = [&]() {
-        wait_pv();
-        tc_fence_after();
-        if (!pv_fresh && warp < NG) {
-            // lanes 0-15 of this warp's tensor-memory lanes hold rows (group = warp, head = lane / 4, digit = lane % 4)
-            const float sa = h_bound * (1.0f / (float)(1u << (32 - kSlackLog2))) * (float)(1u << (8 * (lane & 3)));
-#pragma unroll 1
-            for (int c0 = 0; c0 < G; c0 += 16) {
-                int v[16];
-                tmem_ld16(tmem_row + kPvCol + warp * G + c0, v);
-                tmem_wait_ld();
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    float x = (float)v[j] * sa;
-                    x += __shfl_xor_sync(0xffffffffu, x, 1);
-                    x += __shfl_xor_sync(0xffffffffu, x, 2);
-                    if (lane < 16 && (lane & 3) == 0) Os[(lane >> 2) * kHeadDim + warp * G + c0 + j] += x;
+                for (int d = 0; d < 4; ++d) {
+                    const int dg = d < 3 ? ((qi + 128) & 255) - 128 : qi;      // balanced digits: qi = sum dg * 256^d
+                    qi = (qi - dg) >> 8;
+                    const int n = 4 * r + d;
+                    col[(n >> 3) * kSboK + (n & 7) * 16] = (uint8_t)(dg & 255);
                 }
             }
         }
-        tc_fence_before();
-        pv_fresh = true;
-        tiles_since_fold = 0;
-    };
-
-    // ---- the first two tiles' K operands and score MMAs (the query scratch in the V buffer is dead after the barrier)
-    const uint32_t s_base = s_issued;      // score MMA index of tile 0 of this segment
-    if (n_tiles > 0) build_k(0, s_base & 1u);
-    if (n_tiles > 1) build_k(1, (s_base + 1) & 1u);
-    proxy_fence();
-    __syncthreads();
-    if (fail_sh) failed = true;
-    if (tid == 0 && !failed) {
-        if (n_tiles > 0) issue_scores(s_base & 1u);
-        if (n_tiles > 1) issue_scores((s_base + 1) & 1u);
-        proxy_fence();
-        if (n_tiles > kRing) issue_k(kRing);
-        if (n_tiles > kRing + 1) issue_k(kRing + 1);
-    }
-    s_issued += (uint32_t)min(n_tiles, 2);
-
-    int i_stop = 0;      // first tile that was not completed (for the bounded drain after a failure)
-    for (int i = 0; i < n_tiles && !failed; ++i) {
-        i_stop = i;
-        const uint32_t sbuf = (s_base + i) & 1u;
-        const uint8_t *vm = smem + C::kOffVm + ((tiles_done + i) % kRing) * C::kVmBytes;
-        const uint32_t *Km = reinterpret_cast<const uint32_t *>(vm + C::kCodeTile);                      // [128][NG] words {h, z}
-        const uint32_t *Vm = reinterpret_cast<const uint32_t *>(vm + C::kCodeTile + C::kMetaTile);
-        uint8_t *PA = smem + C::kOffPA + (i & 1) * (kTile * 64);
-        const int tok = q_begin + i * kTile + tid;
-        const bool valid = tok < q_end && tok >= s.n_sink;      // sinks belong to the merge kernel
-
-        // ---------------- scores of this thread's token (the MMA was issued two tiles ago)
-        if (!mbar_wait_bounded(bar_s + 8 * sbuf, (s_taken >> 1) & 1u)) fail_sh = 1;
-        ++s_taken;
-        tc_fence_after();
-        int v[NG][16];
-#pragma unroll
-        for (int gg = 0; gg < NG; ++gg) tmem_ld16(tmem_row + kScoreCol + 64 * sbuf + 16 * gg, v[gg]);
-        wait_ring(bar_v, i);
-        uint32_t kw[NG], vw[NG];
-        load_words<NG>(Km + tid * NG, kw);
-        load_words<NG>(Vm + tid * NG, vw);
-        tmem_wait_ld();
-        float sc[kHeads] = {0.f, 0.f, 0.f, 0.f}, zt[kHeads] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int gg = 0; gg < NG; ++gg) {
-            const float hk_ = lo_half(kw[gg]), zk_ = hi_half(kw[gg]);
-#pragma unroll
-            for (int r = 0; r < kHeads; ++r) {
-                const int lo = v[gg][4 * r] + (v[gg][4 * r + 1] << 8), hi = v[gg][4 * r + 2] + (v[gg][4 * r + 3] << 8);
-                const float u = fmaf((float)hi, 65536.0f, (float)lo);      // 2^30 * sum_j q'_j 2^-e c_j over the group
-                sc[r] = fmaf(hk_, u, sc[r]);
-                zt[r] = fmaf(zk_, sqs[r][gg], zt[r]);
-            }
-        }
-        float hmax = 0.f;
-        float hv[NG], zv[NG];
-#pragma unroll
-        for (int gg = 0; gg < NG; ++gg) {
-            hv[gg] = valid ? lo_half(vw[gg]) : 0.f;      // rows past the end and rows of sinks hold unspecified bytes
-            zv[gg] = valid ? hi_half(vw[gg]) : 0.f;
-            hmax = fmaxf(hmax, hv[gg]);
-        }
-        float arg[kHeads];
-        bool need = hmax >= h_bound || tiles_since_fold >= kFoldTiles;
+        float csc[kHeads], sqs[kHeads][NG];
 #pragma unroll
         for (int r = 0; r < kHeads; ++r) {
-            sc[r] = valid ? fmaf(sc[r], csc[r], zt[r]) : -CUDART_INF_F;      // log2 domain
-            arg[r] = sc[r] - m_ref[r];                                      // +inf while the head has no reference yet
-            need |= valid && arg[r] > (float)kSlackLog2;
+            csc[r] = csc_sh[r];
+#pragma unroll
+            for (int gg = 0; gg < NG; ++gg) sqs[r][gg] = sqs_sh[r * 4 + gg];
         }
-        tc_fence_before();
-        const int moved = __syncthreads_or(need ? 1 : 0);
-        if (fail_sh) { failed = true; break; }
-        if (moved) {
-            // Rare after the first tile: raise every head's reference to its running maximum (and the bound on h),
-            // fold what was accumulated and bring it onto the new references.
-            float hm = warp_max(hmax);
-            if (lane == 0) red[warp * 24 + 4] = hm;
+        token_sync();      // the query scratch (in the V operand buffer) is dead from here on
+
+        // running state: this thread's token of every tile, all four heads
+        float m_ref[kHeads], l_sum[kHeads], zp[kHeads][NG];
 #pragma unroll
-            for (int r = 0; r < kHeads; ++r) {
-                const float wm = warp_max(sc[r]);
-                if (lane == 0) red[warp * 24 + r] = wm;
-            }
-            fold_pv();
-            __syncthreads();
-            if (fail_sh) { failed = true; break; }
+        for (int r = 0; r < kHeads; ++r) {
+            m_ref[r] = -CUDART_INF_F;
+            l_sum[r] = 0.f;
 #pragma unroll
-            for (int r = 0; r < kHeads; ++r) {
-                float mx = m_ref[r];
-                for (int w = 0; w < kWarps; ++w) mx = fmaxf(mx, red[w * 24 + r]);
-                const float corr = mx == -CUDART_INF_F ? 1.f : ex2_approx(m_ref[r] - mx);      // 0 on the first tile with a token
-                m_ref[r] = mx;
-                l_sum[r] *= corr;
-#pragma unroll
-                for (int gg = 0; gg < NG; ++gg) zp[r][gg] *= corr;
-                Os[r * kHeadDim + tid] *= corr;
-                arg[r] = sc[r] - m_ref[r];
-            }
-            hm = 0.f;
-            for (int w = 0; w < kWarps; ++w) hm = fmaxf(hm, red[w * 24 + 4]);
-            if (hm >= h_bound) {
-                h_bound = __int_as_float(((__float_as_int(hm) >> 23) + 1) << 23);   // next power of two above
-                hscale = (float)(1u << (32 - kSlackLog2)) / h_bound;
-            }
-            __syncthreads();      // red is rewritten by the next move
+            for (int gg = 0; gg < NG; ++gg) zp[r][gg] = 0.f;
         }
+        float h_bound = 6.103515625e-05f;      // power of two above every value scale seen so far (2^-14 to start with)
+        float hscale = (float)(1u << (32 - kSlackLog2)) / h_bound;
+        bool pv_fresh = true;                  // the next value MMA overwrites the accumulators
+        int tiles_since_fold = 0;
+        uint32_t pv_local = 0;                 // value MMAs of this segment handed to the control warp
+        uint32_t pv_waited = 0;
 
-        // ---------------- p and the digits of p*h -> A operand of the value MMA (buffer last read two tiles ago)
-        {
-            float ps[kHeads];
-#pragma unroll
-            for (int r = 0; r < kHeads; ++r) {
-                const float p = sc[r] == -CUDART_INF_F ? 0.f : ex2_approx(arg[r]);      // at most 2^slack
-                l_sum[r] += p;
-                ps[r] = p * hscale;
-#pragma unroll
-                for (int gg = 0; gg < NG; ++gg) zp[r][gg] = fmaf(p, zv[gg], zp[r][gg]);
+        auto wait_pv = [&]() {                 // every value MMA handed over so far has completed
+            if (pv_waited < pv_local) {
+                if (!mbar_wait_bounded(bar_pv, (pv_count + pv_local - 1) & 1u)) fail_sh = 1;
+                pv_waited = pv_local;
             }
-#pragma unroll
-            for (int gg = 0; gg < NG; ++gg)
-                *reinterpret_cast<uint4 *>(PA + gg * kSboMN + (tid >> 3) * kLbo + (tid & 7) * 16) =
-                    make_uint4(to_fixed_u32(ps[0] * hv[gg]), to_fixed_u32(ps[1] * hv[gg]), to_fixed_u32(ps[2] * hv[gg]),
-                               to_fixed_u32(ps[3] * hv[gg]));
-        }
-
-        // ---------------- K of the tile after next -> the A operand buffer this tile's score MMA has just released
-        if (i + 2 < n_tiles) build_k(i + 2, sbuf);
-
-        // ---------------- V tile -> B operand of the value MMA, once the previous value MMA has read the buffer
-        wait_pv();
-        unpack_row(vm + tid * kRowBytes, VB + (tid >> 3) * kLbo + (tid & 7) * 16, kSboMN);
-
-        proxy_fence();
-        __syncthreads();
-        if (fail_sh) { failed = true; break; }
-        if (tid == 0) {
+        };
+        // every thread: its token's row of tile i -> A operand of the score MMA, then tell the control warp
+        auto build_k = [&](int i) {
+            const uint32_t sbuf = (s_count + i) & 1u;
+            wait_ring(bar_k, i);
+            unpack_row(smem + ((tiles_done + i) % kRing) * C::kCodeTile + tid * kRowBytes,
+                       smem + C::kOffKA + sbuf * (kTile * 128) + (tid >> 3) * kSboK + (tid & 7) * 16, kLbo);
+            proxy_fence();
+            mbar_arrive(bar_ka + 8 * sbuf);
+        };
+        // Brings the int32 value sums into the fp32 sums in shared memory (relative to the old references and bound).
+        auto fold_pv = [&]() {
+            wait_pv();
             tc_fence_after();
+            if (!pv_fresh && warp < NG) {
+                // lanes 0-15 of this warp's tensor-memory lanes hold rows (group = warp, head = lane / 4, digit = lane % 4)
+                const float sa = h_bound * (1.0f / (float)(1u << (32 - kSlackLog2))) * (float)(1u << (8 * (lane & 3)));
+#pragma unroll 1
+                for (int c0 = 0; c0 < G; c0 += 16) {
+                    int v[16];
+                    tmem_ld16(tmem_row + kPvCol + warp * G + c0, v);
+                    tmem_wait_ld();
 #pragma unroll
-            for (int ks = 0; ks < 4; ++ks)
-                umma_i8(tmem + kPvCol, dPA + (((i & 1) * (kTile * 64) + ks * 4 * kLbo) >> 4), dVB + ((ks * 4 * kLbo) >> 4), kIdescPV,
-                        (pv_fresh && ks == 0) ? 0u : 1u);
-            umma_commit(bar_pv);
-            if (i + 2 < n_tiles) issue_scores(sbuf);
-            proxy_fence();      // the slots were read through the generic proxy
-            if (i + kRing < n_tiles) issue_v(i + kRing);
-            if (i + 2 + kRing < n_tiles) issue_k(i + 2 + kRing);
-        }
-        ++pv_issued;
-        if (i + 2 < n_tiles) ++s_issued;
-        pv_fresh = false;
-        ++tiles_since_fold;
-    }
+                    for (int j = 0; j < 16; ++j) {
+                        float x = (float)v[j] * sa;
+                        x += __shfl_xor_sync(0xffffffffu, x, 1);
+                        x += __shfl_xor_sync(0xffffffffu, x, 2);
+                        if (lane < 16 && (lane & 3) == 0) Os[(lane >> 2) * kHeadDim + warp * G + c0 + j] += x;
+                    }
+                }
+            }
+            tc_fence_before();
+            pv_fresh = true;
+            tiles_since_fold = 0;
+        };
 
-    // ---- end of the segment: last fold, CTA-wide sums, one partial per query head
-    if (failed) {
-        // let whatever is still in flight land (bounded), then report
-        for (int i = i_stop; i < n_tiles && i < i_stop + kRing + 3; ++i) { wait_ring(bar_k, i); wait_ring(bar_v, i); }
-        if (tid == 0 && a.c.status) atomicOr(a.c.status, SKVQ_STATUS_COPY_TIMEOUT);
-    }
-    fold_pv();
+        // the first two tiles' K operands
+        if (n_tiles > 0) build_k(0);
+        if (n_tiles > 1) build_k(1);
+
+        for (int i = 0; i < n_tiles; ++i) {
+            const uint32_t n = s_count + i, sbuf = n & 1u;
+            const uint8_t *vm = smem + C::kOffVm + ((tiles_done + i) % kRing) * C::kVmBytes;
+            const uint32_t *Km = reinterpret_cast<const uint32_t *>(vm + C::kCodeTile);                      // [128][NG] words {h, z}
+            const uint32_t *Vm = reinterpret_cast<const uint32_t *>(vm + C::kCodeTile + C::kMetaTile);
+            uint8_t *PA = smem + C::kOffPA + (i & 1) * (kTile * 64);
+            const int tok = q_begin + i * kTile + tid;
+            const bool valid = tok < q_end && tok >= s.n_sink;      // sinks belong to the merge kernel
+
+            // ---------------- scores of this thread's token (the MMA was issued two tiles ago)
+            if (!mbar_wait_bounded(bar_s + 8 * sbuf, (n >> 1) & 1u)) fail_sh = 1;
+            tc_fence_after();
+            int v[NG][16];
 #pragma unroll
-    for (int r = 0; r < kHeads; ++r) {
-        const float ls = warp_sum(l_sum[r]);
-        if (lane == 0) red[warp * 24 + r] = ls;
+            for (int gg = 0; gg < NG; ++gg) tmem_ld16(tmem_row + kScoreCol + 64 * sbuf + 16 * gg, v[gg]);
+            wait_ring(bar_v, i);
+            uint32_t kw[NG], vw[NG];
+            load_words<NG>(Km + tid * NG, kw);
+            load_words<NG>(Vm + tid * NG, vw);
+            tmem_wait_ld();
+            float sc[kHeads] = {0.f, 0.f, 0.f, 0.f}, zt[kHeads] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int gg = 0; gg < NG; ++gg) {
-            const float zs = warp_sum(zp[r][gg]);
-            if (lane == 0) red[warp * 24 + 8 + r * 4 + gg] = zs;
+            for (int gg = 0; gg < NG; ++gg) {
+                const float hk_ = lo_half(kw[gg]), zk_ = hi_half(kw[gg]);
+#pragma unroll
+                for (int r = 0; r < kHeads; ++r) {
+                    const int lo = v[gg][4 * r] + (v[gg][4 * r + 1] << 8), hi = v[gg][4 * r + 2] + (v[gg][4 * r + 3] << 8);
+                    const float u = fmaf((float)hi, 65536.0f, (float)lo);      // 2^30 * sum_j q'_j 2^-e c_j over the group
+                    sc[r] = fmaf(hk_, u, sc[r]);
+                    zt[r] = fmaf(zk_, sqs[r][gg], zt[r]);
+                }
+            }
+            float hmax = 0.f;
+            float hv[NG], zv[NG];
+#pragma unroll
+            for (int gg = 0; gg < NG; ++gg) {
+                hv[gg] = valid ? lo_half(vw[gg]) : 0.f;      // rows past the end and rows of sinks hold unspecified bytes
+                zv[gg] = valid ? hi_half(vw[gg]) : 0.f;
+                hmax = fmaxf(hmax, hv[gg]);
+            }
+            float arg[kHeads];
+            bool need = hmax >= h_bound || tiles_since_fold >= kFoldTiles;
+#pragma unroll
+            for (int r = 0; r < kHeads; ++r) {
+                sc[r] = valid ? fmaf(sc[r], csc[r], zt[r]) : -CUDART_INF_F;      // log2 domain
+                arg[r] = sc[r] - m_ref[r];                                      // +inf while the head has no reference yet
+                need |= valid && arg[r] > (float)kSlackLog2;
+            }
+            tc_fence_before();
+            const int moved = token_sync_or((need ? 1 : 0) | fail_sh);
+            if (moved) {
+                if (token_sync_or(fail_sh)) { failed = true; break; }      // a uniform decision: every thread leaves, or none
+                // Rare after the first tile: raise every head's reference to its running maximum (and the bound on h),
+                // fold what was accumulated and bring it onto the new references.
+                float hm = warp_max(hmax);
+                if (lane == 0) red[warp * 24 + 4] = hm;
+#pragma unroll
+                for (int r = 0; r < kHeads; ++r) {
+                    const float wm = warp_max(sc[r]);
+                    if (lane == 0) red[warp * 24 + r] = wm;
+                }
+                fold_pv();
+                token_sync();
+#pragma unroll
+                for (int r = 0; r < kHeads; ++r) {
+                    float mx = m_ref[r];
+                    for (int w = 0; w < kWarps; ++w) mx = fmaxf(mx, red[w * 24 + r]);
+                    const float corr = mx == -CUDART_INF_F ? 1.f : ex2_approx(m_ref[r] - mx);      // 0 on the first tile with a token
+                    m_ref[r] = mx;
+                    l_sum[r] *= corr;
+#pragma unroll
+                    for (int gg = 0; gg < NG; ++gg) zp[r][gg] *= corr;
+                    Os[r * kHeadDim + tid] *= corr;
+                    arg[r] = sc[r] - m_ref[r];
+                }
+                hm = 0.f;
+                for (int w = 0; w < kWarps; ++w) hm = fmaxf(hm, red[w * 24 + 4]);
+                if (hm >= h_bound) {
+                    h_bound = __int_as_float(((__float_as_int(hm) >> 23) + 1) << 23);   // next power of two above
+                    hscale = (float)(1u << (32 - kSlackLog2)) / h_bound;
+                }
+                token_sync();      // red is rewritten by the next move
+            }
+
+            // ---------------- p and the digits of p*h -> A operand of the value MMA (buffer last read two tiles ago)
+            {
+                float ps[kHeads];
+#pragma unroll
+                for (int r = 0; r < kHeads; ++r) {
+                    const float p = sc[r] == -CUDART_INF_F ? 0.f : ex2_approx(arg[r]);      // at most 2^slack
+                    l_sum[r] += p;
+                    ps[r] = p * hscale;
+#pragma unroll
+                    for (int gg = 0; gg < NG; ++gg) zp[r][gg] = fmaf(p, zv[gg], zp[r][gg]);
+                }
+#pragma unroll
+                for (int gg = 0; gg < NG; ++gg)
+                    *reinterpret_cast<uint4 *>(PA + gg * kSboMN + (tid >> 3) * kLbo + (tid & 7) * 16) =
+                        make_uint4(to_fixed_u32(ps[0] * hv[gg]), to_fixed_u32(ps[1] * hv[gg]), to_fixed_u32(ps[2] * hv[gg]),
+                                   to_fixed_u32(ps[3] * hv[gg]));
+            }
+
+            // ---------------- K of the tile after next -> the A operand buffer this tile's score MMA has just released
+            if (i + 2 < n_tiles) build_k(i + 2);
+
+            // ---------------- V tile -> B operand of the value MMA, once the previous value MMA has read the buffer
+            wait_pv();
+            unpack_row(vm + tid * kRowBytes, VB + (tid >> 3) * kLbo + (tid & 7) * 16, kSboMN);
+            fresh_sh[i & 1] = pv_fresh ? 1 : 0;      // every thread writes the same value
+            proxy_fence();
+            mbar_arrive(bar_pa);
+            ++pv_local;
+            pv_fresh = false;
+            ++tiles_since_fold;
         }
-    }
-    __syncthreads();
-    {
-        const int ch = column_channel(tid);
-        const float winv = __int_as_float((127 - column_shift(tid)) << 23);      // 4^-j
+
+        // ---- end of the segment: last fold, CTA-wide sums
+        if (failed) {
+            if (tid == 0 && a.c.status) atomicOr(a.c.status, SKVQ_STATUS_COPY_TIMEOUT);
+            pv_waited = pv_local;      // nothing more is waited for
+        }
+        fold_pv();
 #pragma unroll
         for (int r = 0; r < kHeads; ++r) {
-            if (r >= R) break;
-            float l = 0.f, z = 0.f;
-            for (int w = 0; w < kWarps; ++w) {
-                l += red[w * 24 + r];
-                z += red[w * 24 + 8 + r * 4 + ch / G];
+            const float ls = warp_sum(l_sum[r]);
+            if (lane == 0) red[warp * 24 + r] = ls;
+#pragma unroll
+            for (int gg = 0; gg < NG; ++gg) {
+                const float zs = warp_sum(zp[r][gg]);
+                if (lane == 0) red[warp * 24 + 8 + r * 4 + gg] = zs;
             }
-            const bool dead = failed || m_ref[r] == -CUDART_INF_F;
-            float *dst = partials + (((size_t)b * s.Hq + hk * R + r) * n_parts + part) * kPartialStride;
-            dst[ch] = dead ? 0.f : fmaf(Os[r * kHeadDim + tid], winv, z);
-            if (tid == 0) { dst[kHeadDim] = dead ? -CUDART_INF_F : m_ref[r]; dst[kHeadDim + 1] = dead ? 0.f : l; }
         }
+        token_sync();
+        {
+            const int ch = column_channel(tid);
+            const float winv = __int_as_float((127 - column_shift(tid)) << 23);      // 4^-j
+#pragma unroll
+            for (int r = 0; r < kHeads; ++r) {
+                if (r >= R) break;
+                float l = 0.f, z = 0.f;
+                for (int w = 0; w < kWarps; ++w) {
+                    l += red[w * 24 + r];
+                    z += red[w * 24 + 8 + r * 4 + ch / G];
+                }
+                const bool dead = failed || m_ref[r] == -CUDART_INF_F;
+                float *dst = partials + (((size_t)b * s.Hq + hk * R + r) * n_parts + part) * kPartialStride;
+                dst[ch] = dead ? 0.f : fmaf(Os[r * kHeadDim + tid], winv, z);
+                if (tid == 0) { dst[kHeadDim] = dead ? -CUDART_INF_F : m_ref[r]; dst[kHeadDim + 1] = dead ? 0.f : l; }
+            }
+        }
+    }
+    __syncthreads();          // the segment's shared data is dead; thread 0 decides whether there is another one
+    if (fail_sh) {
+        // bounded drain of whatever copies are still in flight before the slots are reused or the CTA leaves
+        if (!failed && tid == 0) for (int i = 0; i < n_tiles; ++i) { wait_ring(bar_k, i); wait_ring(bar_v, i); }
+        failed = true;
     }
     tiles_done += (uint32_t)n_tiles;
-    __syncthreads();          // the segment's shared data is dead; thread 0 decides whether there is another one
+    s_count += (uint32_t)n_tiles;
+    pv_count += (uint32_t)n_tiles;
     if (tid == 0) more_sh = walk.done() ? 0 : 1;
     __syncthreads();
     if (!more_sh) break;
     }
 
-    // ---- give the tensor memory back (every tensor-memory read of this CTA is behind the barriers above)
+    // ---- give the tensor memory back (every tensor-memory access of this CTA is behind the barriers above)
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    if (control) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
 }
 
 template <int G>
@@ -570,7 +603,7 @@ cudaError_t launch_g(const MmaArgs &a, cudaStream_t stream, bool overlap)
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    return launch_dependent(kern, dim3(a.plan.n_slots), dim3(kTile), C::kSmemBytes, stream, overlap, a);
+    return launch_dependent(kern, dim3(a.plan.n_slots), dim3(kTile + 32), C::kSmemBytes, stream, overlap, a);
 }
 
 }  // namespace
