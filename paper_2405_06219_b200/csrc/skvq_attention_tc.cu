@@ -31,15 +31,16 @@ using namespace mmak;
 constexpr int kTile = 128;              // tokens per tile = rows of the score MMA = threads per CTA
 constexpr int kHeads = 4;               // query heads per KV head served (absent heads carry a zero query)
 constexpr int kSlackLog2 = 16;          // the softmax reference moves only when a score exceeds it by this (log2)
-constexpr int kRing = 3;                // slots of each of the two copy rings
-constexpr int kTmemCols = 256;          // allocation: two score buffers in columns [0, 128), value sums in [128, 256)
-constexpr int kScoreCol = 0, kPvCol = 128;
+constexpr int kRing = 2;                // slots of each of the two copy rings
+constexpr int kTmemCols = 128;          // allocation: scores in columns [0, 64), value sums in [64, 128)
+constexpr int kScoreCol = 0, kPvCol = 64;
+constexpr int kCtasPerSm = 3;           // by tensor memory (512 columns), shared memory and registers
 constexpr int kFoldTiles = 256;         // 255 * 192 * 128 * 256 < 2^31: the int32 value sums are folded at least this often
 constexpr uint32_t kLbo = 128;          // bytes between core matrices along K (all operands)
 constexpr uint32_t kSboK = 1024;        // K-major operands: bytes between groups of 8 rows
 constexpr uint32_t kSboMN = 2048;       // MN-major operands: bytes between 16-byte chunks of the M/N extent (128 tokens)
 
-// Shared memory.  The K codes of a tile are needed two tiles before everything else of it (its score MMA is issued
+// Shared memory.  The K codes of a tile are needed one tile before everything else of it (its score MMA is issued
 // that far ahead), so they travel in a ring of their own.
 template <int G>
 struct TCfg {
@@ -48,11 +49,11 @@ struct TCfg {
     static constexpr int kMetaTile = kTile * NG * 4;
     static constexpr int kVmBytes = kCodeTile + 2 * kMetaTile;           // V codes, K scale/zero, V scale/zero
     static constexpr int kOffVm = kRing * kCodeTile;
-    static constexpr int kOffKA = kOffVm + kRing * kVmBytes;             // A of the score MMA, two buffers of [128 tokens][128 bytes]
-    static constexpr int kOffQB = kOffKA + 2 * kTile * 128;              // B of the score MMA: [16 (head, digit)][128 bytes]
-    static constexpr int kOffVB = kOffQB + 16 * 128;                     // B of the value MMA: [128 tokens][128 bytes]
-    static constexpr int kOffPA = kOffVB + kTile * 128;                  // A of the value MMA, two buffers of [128 tokens][64 rows]
-    static constexpr int kOffOs = kOffPA + 2 * kTile * 64;               // folded value sums [4][128] fp32, by MMA column
+    static constexpr int kOffKA = kOffVm + kRing * kVmBytes;             // A of the score MMA: [128 tokens][128 bytes]
+    static constexpr int kOffQB = kOffKA + kTile * 128;                  // B of the score MMA: [16 (head, digit)][128 bytes]
+    static constexpr int kOffVB = kOffQB + 16 * 128;                     // A of the value MMA: [128 tokens][128 byte columns]
+    static constexpr int kOffPA = kOffVB + kTile * 128;                  // B of the value MMA: [128 tokens][64 (group, head, digit)]
+    static constexpr int kOffOs = kOffPA + kTile * 64;                   // folded value sums [4][128] fp32, by byte column
     static constexpr int kOffMisc = kOffOs + kHeads * kHeadDim * 4;      // small arrays, see the kernel
     static constexpr int kSmemBytes = kOffMisc + 1024;
     static_assert(kTile * 128 >= kHeads * kHeadDim * 4, "the V operand buffer doubles as query scratch in the prologue");
@@ -151,7 +152,7 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 }
 
 template <int G>
-__global__ void __launch_bounds__(kTile + 32, 2) partition_tc_kernel(MmaArgs a)
+__global__ void __launch_bounds__(kTile + 32, kCtasPerSm) partition_tc_kernel(MmaArgs a)
 {
     using C = TCfg<G>;
     constexpr int NG = C::NG;
@@ -166,7 +167,7 @@ __global__ void __launch_bounds__(kTile + 32, 2) partition_tc_kernel(MmaArgs a)
     __shared__ __align__(16) Segment seg_sh;
     __shared__ int more_sh;
     __shared__ int fail_sh;
-    __shared__ int fresh_sh[2];      // does the value MMA of an even / odd tile overwrite the accumulators?
+    __shared__ int fresh_sh;         // does the next value MMA overwrite the accumulators?
     __shared__ uint32_t tmem_sh;
     __shared__ SlotWalker walk;      // only thread 0 touches it
     __shared__ __align__(16) int hdr_sh[kPlanSmemInts];
@@ -194,10 +195,10 @@ __global__ void __launch_bounds__(kTile + 32, 2) partition_tc_kernel(MmaArgs a)
     uint64_t *bars = reinterpret_cast<uint64_t *>(red + kWarps * 24);
     const uint32_t bar_k = smem_u32(bars);            // [kRing] K codes landed (copy)
     const uint32_t bar_v = bar_k + 8 * kRing;         // [kRing] V codes and scale/zero landed (copy)
-    const uint32_t bar_s = bar_v + 8 * kRing;         // [2] score MMA done (tcgen05.commit)
-    const uint32_t bar_pv = bar_s + 16;               // [1] value MMA done (tcgen05.commit)
-    const uint32_t bar_ka = bar_pv + 8;               // [2] A operand of a score MMA built (128 token threads)
-    const uint32_t bar_pa = bar_ka + 16;              // [1] operands of a value MMA built (128 token threads)
+    const uint32_t bar_s = bar_v + 8 * kRing;         // score MMA done (tcgen05.commit)
+    const uint32_t bar_pv = bar_s + 8;                // value MMA done (tcgen05.commit)
+    const uint32_t bar_ka = bar_pv + 8;               // A operand of a score MMA built (128 token threads)
+    const uint32_t bar_pa = bar_ka + 8;               // operands of a value MMA built (128 token threads)
 
     // ---- tensor memory and barriers (once per CTA)
     if (control) {
@@ -206,9 +207,9 @@ __global__ void __launch_bounds__(kTile + 32, 2) partition_tc_kernel(MmaArgs a)
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
         if (lane == 0) {
 #pragma unroll
-            for (int i = 0; i < 2 * kRing + 3; ++i) mbar_init(bar_k + 8 * i, 1);
-#pragma unroll
-            for (int i = 0; i < 3; ++i) mbar_init(bar_ka + 8 * i, kTile);
+            for (int i = 0; i < 2 * kRing + 2; ++i) mbar_init(bar_k + 8 * i, 1);
+            mbar_init(bar_ka, kTile);
+            mbar_init(bar_pa, kTile);
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
             proxy_fence();
         }
@@ -220,7 +221,7 @@ __global__ void __launch_bounds__(kTile + 32, 2) partition_tc_kernel(MmaArgs a)
     const uint32_t tmem_row = tmem + ((uint32_t)((warp & 3) * 32) << 16);      // this warp's 32 lanes
 
     constexpr uint32_t kIdescS = idesc_i8(128, 16, false, true, false, false);
-    constexpr uint32_t kIdescPV = idesc_i8(64, 128, false, false, true, true);
+    constexpr uint32_t kIdescPV = idesc_i8(128, 64, false, false, true, true);
 
     // kernel-lifetime pipeline counters (every thread counts alike)
     uint32_t tiles_done = 0;           // tiles that went through the rings
@@ -303,29 +304,29 @@ __global__ void __launch_bounds__(kTile + 32, 2) partition_tc_kernel(MmaArgs a)
             const uint64_t dKA = smem_desc(smem_u32(smem + C::kOffKA), kLbo, kSboK), dQB = smem_desc(smem_u32(QB), kLbo, kSboK);
             const uint64_t dVB = smem_desc(smem_u32(VB), kLbo, kSboMN), dPA = smem_desc(smem_u32(smem + C::kOffPA), kLbo, kSboMN);
             bool ok = true;
-            auto scores = [&](int j) {      // score MMA of tile j, once its A operand is complete
-                const uint32_t n = s_count + j, sbuf = n & 1u;
-                if (!mbar_wait_bounded(bar_ka + 8 * sbuf, (n >> 1) & 1u)) { ok = false; return; }
+            auto scores = [&](int j) {      // score MMA of tile j, once its A operand is complete and the old scores are read
+                const uint32_t n = s_count + j;
+                if (!mbar_wait_bounded(bar_ka, n & 1u)) { ok = false; return; }
                 tc_fence_after();
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks)
-                    umma_i8(tmem + kScoreCol + 64 * sbuf + 16 * ((32 * ks) / G), dKA + ((sbuf * (kTile * 128) + ks * 2 * kLbo) >> 4),
-                            dQB + ((ks * 2 * kLbo) >> 4), kIdescS, ((32 * ks) % G) != 0 ? 1u : 0u);
-                umma_commit(bar_s + 8 * sbuf);
+                    umma_i8(tmem + kScoreCol + 16 * ((32 * ks) / G), dKA + ((ks * 2 * kLbo) >> 4), dQB + ((ks * 2 * kLbo) >> 4), kIdescS,
+                            ((32 * ks) % G) != 0 ? 1u : 0u);
+                umma_commit(bar_s);
                 if (j + kRing < n_tiles) { proxy_fence(); issue_k(j + kRing); }      // the token threads are done with that slot
             };
             scores(0);
-            if (ok && n_tiles > 1) scores(1);
             for (int i = 0; i < n_tiles && ok; ++i) {
-                if (i + 2 < n_tiles) scores(i + 2);
+                if (i + 1 < n_tiles) scores(i + 1);
                 if (!ok) break;
                 const uint32_t n = pv_count + i;
                 if (!mbar_wait_bounded(bar_pa, n & 1u)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t fresh = (uint32_t)fresh_sh[i & 1];
+                const uint32_t fresh = (uint32_t)fresh_sh;
+                // channels on the M rows (the V tile as stored is the A operand), (group, head, digit) on the N columns
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks)
-                    umma_i8(tmem + kPvCol, dPA + (((i & 1) * (kTile * 64) + ks * 4 * kLbo) >> 4), dVB + ((ks * 4 * kLbo) >> 4), kIdescPV,
+                    umma_i8(tmem + kPvCol, dVB + ((ks * 4 * kLbo) >> 4), dPA + ((ks * 4 * kLbo) >> 4), kIdescPV,
                             (fresh && ks == 0) ? 0u : 1u);
                 umma_commit(bar_pv);
                 if (i + kRing < n_tiles) { proxy_fence(); issue_v(i + kRing); }
@@ -384,32 +385,28 @@ __global__ void __launch_bounds__(kTile + 32, 2) partition_tc_kernel(MmaArgs a)
         };
         // every thread: its token's row of tile i -> A operand of the score MMA, then tell the control warp
         auto build_k = [&](int i) {
-            const uint32_t sbuf = (s_count + i) & 1u;
             wait_ring(bar_k, i);
             unpack_row(smem + ((tiles_done + i) % kRing) * C::kCodeTile + tid * kRowBytes,
-                       smem + C::kOffKA + sbuf * (kTile * 128) + (tid >> 3) * kSboK + (tid & 7) * 16, kLbo);
+                       smem + C::kOffKA + (tid >> 3) * kSboK + (tid & 7) * 16, kLbo);
             proxy_fence();
-            mbar_arrive(bar_ka + 8 * sbuf);
+            mbar_arrive(bar_ka);
         };
         // Brings the int32 value sums into the fp32 sums in shared memory (relative to the old references and bound).
+        // Only this thread touches column tid of Os.
         auto fold_pv = [&]() {
             wait_pv();
             tc_fence_after();
-            if (!pv_fresh && warp < NG) {
-                // lanes 0-15 of this warp's tensor-memory lanes hold rows (group = warp, head = lane / 4, digit = lane % 4)
-                const float sa = h_bound * (1.0f / (float)(1u << (32 - kSlackLog2))) * (float)(1u << (8 * (lane & 3)));
-#pragma unroll 1
-                for (int c0 = 0; c0 < G; c0 += 16) {
-                    int v[16];
-                    tmem_ld16(tmem_row + kPvCol + warp * G + c0, v);
-                    tmem_wait_ld();
+            if (!pv_fresh) {
+                // tensor-memory lane tid = byte column tid of the V rows; its group's 16 columns are (head, digit)
+                int v[16];
+                tmem_ld16(tmem_row + kPvCol + 16 * ((warp * 32) / G), v);
+                tmem_wait_ld();
+                const float sa = h_bound * (1.0f / (float)(1u << (32 - kSlackLog2)));
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        float x = (float)v[j] * sa;
-                        x += __shfl_xor_sync(0xffffffffu, x, 1);
-                        x += __shfl_xor_sync(0xffffffffu, x, 2);
-                        if (lane < 16 && (lane & 3) == 0) Os[(lane >> 2) * kHeadDim + warp * G + c0 + j] += x;
-                    }
+                for (int r = 0; r < kHeads; ++r) {
+                    const float lo = fmaf((float)v[4 * r + 1], 256.0f, (float)v[4 * r]);
+                    const float hi = fmaf((float)v[4 * r + 3], 256.0f, (float)v[4 * r + 2]);
+                    Os[r * kHeadDim + tid] += fmaf(hi, 65536.0f, lo) * sa;
                 }
             }
             tc_fence_before();
@@ -417,30 +414,29 @@ __global__ void __launch_bounds__(kTile + 32, 2) partition_tc_kernel(MmaArgs a)
             tiles_since_fold = 0;
         };
 
-        // the first two tiles' K operands
-        if (n_tiles > 0) build_k(0);
-        if (n_tiles > 1) build_k(1);
+        if (n_tiles > 0) build_k(0);      // the first tile's K operand
 
         for (int i = 0; i < n_tiles; ++i) {
-            const uint32_t n = s_count + i, sbuf = n & 1u;
+            const uint32_t n = s_count + i;
             const uint8_t *vm = smem + C::kOffVm + ((tiles_done + i) % kRing) * C::kVmBytes;
             const uint32_t *Km = reinterpret_cast<const uint32_t *>(vm + C::kCodeTile);                      // [128][NG] words {h, z}
             const uint32_t *Vm = reinterpret_cast<const uint32_t *>(vm + C::kCodeTile + C::kMetaTile);
-            uint8_t *PA = smem + C::kOffPA + (i & 1) * (kTile * 64);
+            uint8_t *PA = smem + C::kOffPA;
             const int tok = q_begin + i * kTile + tid;
             const bool valid = tok < q_end && tok >= s.n_sink;      // sinks belong to the merge kernel
 
-            // ---------------- scores of this thread's token (the MMA was issued two tiles ago)
-            if (!mbar_wait_bounded(bar_s + 8 * sbuf, (n >> 1) & 1u)) fail_sh = 1;
+            // ---------------- scores of this thread's token (the MMA was issued one tile ago)
+            if (!mbar_wait_bounded(bar_s, n & 1u)) fail_sh = 1;
             tc_fence_after();
             int v[NG][16];
 #pragma unroll
-            for (int gg = 0; gg < NG; ++gg) tmem_ld16(tmem_row + kScoreCol + 64 * sbuf + 16 * gg, v[gg]);
+            for (int gg = 0; gg < NG; ++gg) tmem_ld16(tmem_row + kScoreCol + 16 * gg, v[gg]);
             wait_ring(bar_v, i);
             uint32_t kw[NG], vw[NG];
             load_words<NG>(Km + tid * NG, kw);
             load_words<NG>(Vm + tid * NG, vw);
             tmem_wait_ld();
+            tc_fence_before();
             float sc[kHeads] = {0.f, 0.f, 0.f, 0.f}, zt[kHeads] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int gg = 0; gg < NG; ++gg) {
@@ -453,6 +449,8 @@ __global__ void __launch_bounds__(kTile + 32, 2) partition_tc_kernel(MmaArgs a)
                     zt[r] = fmaf(zk_, sqs[r][gg], zt[r]);
                 }
             }
+            // the next tile's K -> the A operand the score MMA of this tile has released; its MMA runs under the rest
+            if (i + 1 < n_tiles) build_k(i + 1);
             float hmax = 0.f;
             float hv[NG], zv[NG];
 #pragma unroll
@@ -483,7 +481,7 @@ __global__ void __launch_bounds__(kTile + 32, 2) partition_tc_kernel(MmaArgs a)
                     if (lane == 0) red[warp * 24 + r] = wm;
                 }
                 fold_pv();
-                token_sync();
+                token_sync();      // red is complete
 #pragma unroll
                 for (int r = 0; r < kHeads; ++r) {
                     float mx = m_ref[r];
@@ -505,7 +503,8 @@ __global__ void __launch_bounds__(kTile + 32, 2) partition_tc_kernel(MmaArgs a)
                 token_sync();      // red is rewritten by the next move
             }
 
-            // ---------------- p and the digits of p*h -> A operand of the value MMA (buffer last read two tiles ago)
+            // ---------------- p and the digits of p*h -> B operand of the value MMA, once the previous one has read it
+            wait_pv();
             {
                 float ps[kHeads];
 #pragma unroll
@@ -523,13 +522,9 @@ __global__ void __launch_bounds__(kTile + 32, 2) partition_tc_kernel(MmaArgs a)
                                    to_fixed_u32(ps[3] * hv[gg]));
             }
 
-            // ---------------- K of the tile after next -> the A operand buffer this tile's score MMA has just released
-            if (i + 2 < n_tiles) build_k(i + 2);
-
-            // ---------------- V tile -> B operand of the value MMA, once the previous value MMA has read the buffer
-            wait_pv();
+            // ---------------- V tile -> A operand of the value MMA
             unpack_row(vm + tid * kRowBytes, VB + (tid >> 3) * kLbo + (tid & 7) * 16, kSboMN);
-            fresh_sh[i & 1] = pv_fresh ? 1 : 0;      // every thread writes the same value
+            fresh_sh = pv_fresh ? 1 : 0;      // every thread writes the same value
             proxy_fence();
             mbar_arrive(bar_pa);
             ++pv_local;
