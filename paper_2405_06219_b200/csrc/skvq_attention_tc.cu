@@ -428,29 +428,38 @@ __global__ void __launch_bounds__(kTile + 32, kCtasPerSm) partition_tc_kernel(Mm
             // ---------------- scores of this thread's token (the MMA was issued one tile ago)
             if (!mbar_wait_bounded(bar_s, n & 1u)) fail_sh = 1;
             tc_fence_after();
-            int v[NG][16];
+            // The accumulators are read in two halves: the second half is in flight while the first is combined, and
+            // the next tile's K operand is built as soon as the last read has landed, so that its MMA runs under the rest.
+            constexpr int H0 = NG > 1 ? NG / 2 : 1;      // groups in the first half
+            int va[H0][16];
 #pragma unroll
-            for (int gg = 0; gg < NG; ++gg) tmem_ld16(tmem_row + kScoreCol + 16 * gg, v[gg]);
+            for (int gg = 0; gg < H0; ++gg) tmem_ld16(tmem_row + kScoreCol + 16 * gg, va[gg]);
             wait_ring(bar_v, i);
             uint32_t kw[NG], vw[NG];
             load_words<NG>(Km + tid * NG, kw);
             load_words<NG>(Vm + tid * NG, vw);
             tmem_wait_ld();
-            tc_fence_before();
-            float sc[kHeads] = {0.f, 0.f, 0.f, 0.f}, zt[kHeads] = {0.f, 0.f, 0.f, 0.f};
+            int vb[NG - H0 > 0 ? NG - H0 : 1][16];
 #pragma unroll
-            for (int gg = 0; gg < NG; ++gg) {
+            for (int gg = H0; gg < NG; ++gg) tmem_ld16(tmem_row + kScoreCol + 16 * gg, vb[gg - H0]);
+            float sc[kHeads] = {0.f, 0.f, 0.f, 0.f}, zt[kHeads] = {0.f, 0.f, 0.f, 0.f};
+            auto combine = [&](const int (&v)[16], int gg) {
                 const float hk_ = lo_half(kw[gg]), zk_ = hi_half(kw[gg]);
 #pragma unroll
                 for (int r = 0; r < kHeads; ++r) {
-                    const int lo = v[gg][4 * r] + (v[gg][4 * r + 1] << 8), hi = v[gg][4 * r + 2] + (v[gg][4 * r + 3] << 8);
+                    const int lo = v[4 * r] + (v[4 * r + 1] << 8), hi = v[4 * r + 2] + (v[4 * r + 3] << 8);
                     const float u = fmaf((float)hi, 65536.0f, (float)lo);      // 2^30 * sum_j q'_j 2^-e c_j over the group
                     sc[r] = fmaf(hk_, u, sc[r]);
                     zt[r] = fmaf(zk_, sqs[r][gg], zt[r]);
                 }
-            }
-            // the next tile's K -> the A operand the score MMA of this tile has released; its MMA runs under the rest
-            if (i + 1 < n_tiles) build_k(i + 1);
+            };
+#pragma unroll
+            for (int gg = 0; gg < H0; ++gg) combine(va[gg], gg);
+            tmem_wait_ld();
+            tc_fence_before();
+            if (i + 1 < n_tiles) build_k(i + 1);      // the score MMA of this tile has released the A operand and the columns
+#pragma unroll
+            for (int gg = H0; gg < NG; ++gg) combine(vb[gg - H0], gg);
             float hmax = 0.f;
             float hv[NG], zv[NG];
 #pragma unroll
