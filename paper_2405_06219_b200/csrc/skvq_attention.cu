@@ -409,7 +409,8 @@ __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
 static int partition_ctas_per_sm(const Shape &s)
 {
     if (s.rep == 1 && s.G >= 64) return s.k_bits == s.v_bits ? 4 : 3;           // integer kernel
-    if (s.k_bits == 2 && s.v_bits == 2 && s.rep == 3) return 3;                // tcgen05 kernel: 128 tensor-memory columns, 69 KB
+    if (s.k_bits == 2 && s.v_bits == 2 && (s.rep == 3 || (s.rep > 4 && s.rep <= 8)) && (s.G == 128 || s.G == 64 || s.G == 32))
+        return 3;                                                              // tcgen05 kernel: 128 tensor-memory columns, 69 KB
     if (s.k_bits == 2 && s.v_bits == 2 && s.rep <= 4) return 2;                // grouped-query kernel, 244 registers
     return 8;                                                                  // scalar kernel
 }

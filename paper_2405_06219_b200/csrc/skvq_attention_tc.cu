@@ -160,7 +160,7 @@ __global__ void __launch_bounds__(kTile + 32, kCtasPerSm) partition_tc_kernel(Mm
     const Shape &s = a.s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool control = warp == kWarps;      // warp 4 issues every copy and MMA; warps 0-3 own one token each
-    const int R = s.rep;
+    const int R = min(kHeads, s.rep - a.head0);      // query heads of every KV head served by this launch
     asm volatile("griddepcontrol.launch_dependents;");      // the merge kernel may start its window part early
     asm volatile("griddepcontrol.wait;" ::: "memory");      // the lengths, and the plan kernel's header when there is one
 
@@ -273,7 +273,7 @@ __global__ void __launch_bounds__(kTile + 32, kCtasPerSm) partition_tc_kernel(Mm
         const int src = idx_k[tid] & (kHeadDim - 1);
 #pragma unroll
         for (int r = 0; r < kHeads; ++r) {
-            const float qv = r < R ? __half2float(a.q[((size_t)b * s.Hq + hk * R + r) * kHeadDim + src]) : 0.f;
+            const float qv = r < R ? __half2float(a.q[((size_t)b * s.Hq + hk * s.rep + a.head0 + r) * kHeadDim + src]) : 0.f;
             qs[r * kHeadDim + tid] = qv;
             const float wm = warp_max(fabsf(qv));
             if (lane == 0) red[warp * 24 + r] = wm;
@@ -570,7 +570,7 @@ __global__ void __launch_bounds__(kTile + 32, kCtasPerSm) partition_tc_kernel(Mm
                     z += red[w * 24 + 8 + r * 4 + ch / G];
                 }
                 const bool dead = failed || m_ref[r] == -CUDART_INF_F;
-                float *dst = partials + (((size_t)b * s.Hq + hk * R + r) * n_parts + part) * kPartialStride;
+                float *dst = partials + (((size_t)b * s.Hq + hk * s.rep + a.head0 + r) * n_parts + part) * kPartialStride;
                 dst[ch] = dead ? 0.f : fmaf(Os[r * kHeadDim + tid], winv, z);
                 if (tid == 0) { dst[kHeadDim] = dead ? -CUDART_INF_F : m_ref[r]; dst[kHeadDim + 1] = dead ? 0.f : l; }
             }
@@ -612,21 +612,24 @@ cudaError_t launch_g(const MmaArgs &a, cudaStream_t stream, bool overlap)
 
 }  // namespace
 
-// Launches the kernel above when the configuration is covered (2-bit K and V, 1, 2 or 4 query heads per KV
-// head); *handled tells the caller whether it did.
+// Launches the kernel above when the configuration is covered (2-bit K and V, up to 8 query heads per KV head: one
+// launch per four heads); *handled tells the caller whether it did.
 cudaError_t launch_partition_tc(const Shape &s, const CachePtrs &c, const __half *q, float scale_log2, const SplitPlan &plan,
                                 float *workspace, cudaStream_t stream, bool overlap, bool *handled)
 {
     *handled = false;
-    if (s.k_bits != 2 || s.v_bits != 2 || s.rep > kHeads) return cudaSuccess;
-    MmaArgs a{s, c, q, scale_log2, plan, workspace};
+    if (s.k_bits != 2 || s.v_bits != 2 || s.rep > 2 * kHeads || (s.G != 128 && s.G != 64 && s.G != 32)) return cudaSuccess;
     *handled = true;
-    switch (s.G) {
-        case 128: return launch_g<128>(a, stream, overlap);
-        case 64: return launch_g<64>(a, stream, overlap);
-        case 32: return launch_g<32>(a, stream, overlap);
-        default: *handled = false; return cudaSuccess;
+    for (int head0 = 0; head0 < s.rep; head0 += kHeads) {
+        MmaArgs a{s, c, q, scale_log2, plan, workspace};
+        a.head0 = head0;
+        // a second launch reads the same cache again for the next four heads; it starts when the first has finished
+        const bool ov = overlap && head0 == 0;
+        const cudaError_t e = s.G == 128 ? launch_g<128>(a, stream, ov) : s.G == 64 ? launch_g<64>(a, stream, ov) : launch_g<32>(a, stream, ov);
+        if (e != cudaSuccess) return e;
+        if (head0 > 0) count_launch(1);
     }
+    return cudaSuccess;
 }
 
 }  // namespace skvq

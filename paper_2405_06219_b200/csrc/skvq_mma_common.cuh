@@ -21,6 +21,7 @@ struct MmaArgs {
     float scale_log2;
     SplitPlan plan;
     float *ws;
+    int head0 = 0;      // first query head (of every KV head's group) this launch serves
 };
 
 // ---------------------------------------------------------------- small PTX helpers

@@ -124,6 +124,8 @@ def test_ragged_append_and_overflow_flag():
     (2, dict(context=5300, batch=2, ragged=None, n_q_heads=12, n_kv_heads=4), 5300),     # 3 heads per KV head, g32: tcgen05 kernel
     (1, dict(context=70000, batch=1, n_q_heads=6, n_kv_heads=2), 70000),                 # 3 heads per KV head, g128, many tiles per CTA
     (2, dict(context=1000, batch=33, ragged=(1, 1000), n_q_heads=3, n_kv_heads=1, group_size=64), 1000),   # 3 heads, g64, plan kernel, short and empty prefixes
+    (2, dict(context=6000, batch=1, n_q_heads=64, n_kv_heads=8), 6000),                  # 8 heads per KV head: two tcgen05 launches
+    (1, dict(context=3500, batch=2, n_q_heads=10, n_kv_heads=2), 3500),                  # 5 heads per KV head, g128: 4 + 1
 ])
 def test_attention_matches_oracle(cfg_i, kw, n):
     w = small(cfg_i, **kw)
