@@ -13,14 +13,17 @@
  * Precision contract
  *   - quantizer: IEEE fp32, one rounding per operation (build with
  *     -ffp-contract=off, never -ffast-math), round-half-to-even via rintf();
- *     scale and zero point are stored in fp16 (round-to-nearest-even) and the
- *     codes are computed against the *stored* (rounded) parameters.
+ *     scale and zero point are stored in fp16 (round-to-nearest-even), or, in
+ *     FP8 mode (Sec. 4.1 "Quantization"; the FP8 row of the component
+ *     breakdown), in FP8 E4M3 (round-to-nearest-even, saturating at +-448),
+ *     and the codes are computed against the *stored* (rounded) parameters.
  *   - attention: fp64 everywhere; dequantized values are never rounded.
  *
  * Layout (all row-major, host memory)
  *   codes  uint8  [B][Hkv][cap_q][D*bits/8]   code j of a row sits in bits
  *                                             [(j*bits) mod 8, +bits) of byte (j*bits)/8
- *   meta   uint16 [B][Hkv][cap_q][D/G][2]     {h, z} as fp16 bit patterns
+ *   meta   uint16 [B][Hkv][cap_q][D/G][2]     {h, z} as fp16 bit patterns; in FP8 mode the
+ *                                             E4M3 byte of each in the low 8 bits
  *   win    uint16 [B][Hkv][W][D]              ring: token t lives in slot t mod W,
  *                                             channels already in reordered order
  *   lengths int32 [B]                         tokens appended so far
@@ -29,7 +32,8 @@
  * per-token min-max quantization, closed-form groups, permutation invariance,
  * single-append == bulk-append, brute-force attention, convexity, q = 0 mean,
  * attention sinks (exact rows, brute force over the three segments, all-sink
- * case against a library attention).
+ * case against a library attention), FP8 E4M3 conversions against a library's
+ * (all 256 bytes, random and midpoint inputs) and the paper's 2.5-bit average.
  * End-to-end accuracy versus the paper's benchmark tables: parity unpinned (the
  * datasets and model weights those tables need are not available).
  */
@@ -97,18 +101,53 @@ void orc_reorder_row(const uint16_t *src, const int32_t *idx, int D, uint16_t *d
     for (int j = 0; j < D; ++j) dst[j] = src[idx[j]];
 }
 
+/* ---------------------------------------------------------------- FP8 E4M3 <-> fp32 */
+
+/*
+ * FP8 E4M3 as used for quantization parameters (Sec. 4.1): 1 sign bit, 4
+ * exponent bits with bias 7, 3 mantissa bits, subnormals m * 2^-9, no
+ * infinities, S.1111.111 is NaN, largest finite value 1.75 * 2^8 = 448.
+ */
+float orc_e4m3_to_f32(uint8_t b)
+{
+    const int e = (b >> 3) & 15, m = b & 7;
+    if (e == 15 && m == 7) return NAN;
+    const float v = e == 0 ? ldexpf((float)m, -9) : ldexpf((float)(8 + m), e - 10);
+    return (b & 0x80) ? -v : v;
+}
+
+/* fp32 -> E4M3, round to nearest even; anything beyond the largest finite value becomes +-448. */
+uint8_t orc_f32_to_e4m3(float f)
+{
+    if (isnan(f)) return 0x7F;
+    const uint8_t sign = signbit(f) ? 0x80 : 0x00;
+    const float a = fabsf(f);
+    if (a == 0.0f) return sign;
+    if (isinf(a)) return sign | 0x7E;
+    int e;
+    (void)frexpf(a, &e);        /* a = m * 2^e, 0.5 <= m < 1: the leading bit has weight 2^(e-1) */
+    int E = e - 1;
+    if (E < -6) E = -6;         /* subnormal range: the grid stays 2^-9 */
+    if (E > 9) return sign | 0x7E;
+    int n = (int)rintf(a / ldexpf(1.0f, E - 3));   /* multiples of the grid step; exact division, ties to even */
+    if (n == 16) { E += 1; n = 8; }
+    if (E > 8 || (E == 8 && n > 14)) return sign | 0x7E;
+    if (n < 8) return sign | (uint8_t)n;           /* subnormal (E == -6) */
+    return sign | (uint8_t)(((E + 7) << 3) | (n - 8));
+}
+
 /*
  * Clipped dynamic asymmetric quantization of one already-reordered row
  * (Sec. 3.1 uniform quantizer, Eq. 2, and clipping_quant of Algorithm 1):
  * per group of G consecutive channels take min and max, multiply both by the
- * group's clip factor, derive scale h and zero point z, round both to fp16,
- * then code = clamp(rint((x - z) / h), 0, 2^bits - 1).
+ * group's clip factor, derive scale h and zero point z, round both to fp16
+ * (to FP8 E4M3 if meta_fp8), then code = clamp(rint((x - z) / h), 0, 2^bits - 1).
  * A zero is canonicalised to +0 before it is used so that the sign of a zero
  * minimum or maximum (which depends on the order elements are visited) cannot
  * leak into the stored parameters.
  */
 void orc_quantize_reordered_row(const uint16_t *xr, const float *alpha, int D, int G, int bits,
-                                uint8_t *codes, uint16_t *meta)
+                                uint8_t *codes, uint16_t *meta, int meta_fp8)
 {
     const int qmax = (1 << bits) - 1;
     const int ng = D / G;
@@ -125,12 +164,20 @@ void orc_quantize_reordered_row(const uint16_t *xr, const float *alpha, int D, i
         lo = lo + 0.0f;
         hi = hi + 0.0f;
         float h32 = (hi - lo) / (float)qmax;
-        uint16_t h16 = orc_f32_to_f16(h32);
-        uint16_t z16 = orc_f32_to_f16(lo);
-        float hf = orc_f16_to_f32(h16);
-        float zf = orc_f16_to_f32(z16);
-        meta[2 * g + 0] = h16;
-        meta[2 * g + 1] = z16;
+        float hf, zf;
+        if (meta_fp8) {
+            const uint8_t h8 = orc_f32_to_e4m3(h32), z8 = orc_f32_to_e4m3(lo);
+            hf = orc_e4m3_to_f32(h8);
+            zf = orc_e4m3_to_f32(z8);
+            meta[2 * g + 0] = h8;
+            meta[2 * g + 1] = z8;
+        } else {
+            const uint16_t h16 = orc_f32_to_f16(h32), z16 = orc_f32_to_f16(lo);
+            hf = orc_f16_to_f32(h16);
+            zf = orc_f16_to_f32(z16);
+            meta[2 * g + 0] = h16;
+            meta[2 * g + 1] = z16;
+        }
         for (int j = g * G; j < (g + 1) * G; ++j) {
             int c = 0;
             if (hf != 0.0f) {
@@ -155,25 +202,25 @@ static int orc_code_at(const uint8_t *codes, int j, int bits)
 }
 
 /* Dequantize one row to fp64 without rounding: x^ = h*c + z. */
-void orc_dequant_row(const uint8_t *codes, const uint16_t *meta, int D, int G, int bits, double *out)
+void orc_dequant_row(const uint8_t *codes, const uint16_t *meta, int D, int G, int bits, int meta_fp8, double *out)
 {
     for (int j = 0; j < D; ++j) {
         int g = j / G;
-        double h = (double)orc_f16_to_f32(meta[2 * g + 0]);
-        double z = (double)orc_f16_to_f32(meta[2 * g + 1]);
+        double h = (double)(meta_fp8 ? orc_e4m3_to_f32((uint8_t)meta[2 * g + 0]) : orc_f16_to_f32(meta[2 * g + 0]));
+        double z = (double)(meta_fp8 ? orc_e4m3_to_f32((uint8_t)meta[2 * g + 1]) : orc_f16_to_f32(meta[2 * g + 1]));
         out[j] = h * (double)orc_code_at(codes, j, bits) + z;
     }
 }
 
 /* Reorder then quantize n independent rows (no cache state); for unit tests. */
 void orc_quantize_rows(const uint16_t *x, int n, const int32_t *idx, const float *alpha, int D, int G,
-                       int bits, uint8_t *codes, uint16_t *meta)
+                       int bits, int meta_fp8, uint8_t *codes, uint16_t *meta)
 {
     uint16_t *tmp = (uint16_t *)malloc(sizeof(uint16_t) * (size_t)D);
     for (int r = 0; r < n; ++r) {
         orc_reorder_row(x + (size_t)r * D, idx, D, tmp);
         orc_quantize_reordered_row(tmp, alpha, D, G, bits, codes + (size_t)r * (D * bits / 8),
-                                   meta + (size_t)r * (D / G) * 2);
+                                   meta + (size_t)r * (D / G) * 2, meta_fp8);
     }
     free(tmp);
 }
@@ -191,6 +238,7 @@ typedef struct {
     const float *alpha_k, *alpha_v;       /* [Hkv][D/G] */
     int n_sink;                           /* first n_sink positions are never quantized (Sec. 3.2, filter rules) */
     uint16_t *k_sink, *v_sink;            /* fp16 bits [B][Hkv][n_sink][D], reordered channel order */
+    int meta_fp8;                         /* scale and zero point stored as FP8 E4M3 instead of fp16 */
 } orc_cache;
 
 static size_t orc_row_index(const orc_cache *c, int b, int h, int t, int rows)
@@ -249,10 +297,10 @@ int orc_append(orc_cache *c, const uint16_t *k, const uint16_t *v, const int32_t
                 size_t r = orc_row_index(c, b, h, t, c->cap_q);
                 orc_quantize_reordered_row(rowk, c->alpha_k + (size_t)h * ng, D, c->G, c->k_bits,
                                            c->k_codes + r * (size_t)(D * c->k_bits / 8),
-                                           c->k_meta + r * (size_t)ng * 2);
+                                           c->k_meta + r * (size_t)ng * 2, c->meta_fp8);
                 orc_quantize_reordered_row(rowv, c->alpha_v + (size_t)h * ng, D, c->G, c->v_bits,
                                            c->v_codes + r * (size_t)(D * c->v_bits / 8),
-                                           c->v_meta + r * (size_t)ng * 2);
+                                           c->v_meta + r * (size_t)ng * 2, c->meta_fp8);
             }
             /* 2. the new tokens that remain inside the window go to the ring */
             int first_kept = q_end > L0 ? q_end : L0;
@@ -311,7 +359,7 @@ void orc_attention(const orc_cache *c, int Hq, const uint16_t *q, double sm_scal
                 } else if (t < Lq) {
                     size_t r = orc_row_index(c, b, hk, t, c->cap_q);
                     orc_dequant_row(c->k_codes + r * (size_t)(D * c->k_bits / 8),
-                                    c->k_meta + r * (size_t)ng * 2, D, c->G, c->k_bits, row);
+                                    c->k_meta + r * (size_t)ng * 2, D, c->G, c->k_bits, c->meta_fp8, row);
                 } else {
                     size_t w = orc_row_index(c, b, hk, t % W, W) * (size_t)D;
                     for (int j = 0; j < D; ++j) row[j] = (double)orc_f16_to_f32(c->k_win[w + j]);
@@ -333,7 +381,7 @@ void orc_attention(const orc_cache *c, int Hq, const uint16_t *q, double sm_scal
                 } else if (t < Lq) {
                     size_t r = orc_row_index(c, b, hk, t, c->cap_q);
                     orc_dequant_row(c->v_codes + r * (size_t)(D * c->v_bits / 8),
-                                    c->v_meta + r * (size_t)ng * 2, D, c->G, c->v_bits, row);
+                                    c->v_meta + r * (size_t)ng * 2, D, c->G, c->v_bits, c->meta_fp8, row);
                 } else {
                     size_t w = orc_row_index(c, b, hk, t % W, W) * (size_t)D;
                     for (int j = 0; j < D; ++j) row[j] = (double)orc_f16_to_f32(c->v_win[w + j]);

@@ -40,6 +40,7 @@ class _Cache(ctypes.Structure):
         ("reorder_k", ctypes.c_void_p), ("reorder_v", ctypes.c_void_p),
         ("alpha_k", ctypes.c_void_p), ("alpha_v", ctypes.c_void_p),
         ("n_sink", ctypes.c_int), ("k_sink", ctypes.c_void_p), ("v_sink", ctypes.c_void_p),
+        ("meta_fp8", ctypes.c_int),
     ]
 
 
@@ -53,11 +54,15 @@ def lib():
         _lib.orc_f32_to_f16.argtypes = [ctypes.c_float]
         _lib.orc_quantize_rows.restype = None
         _lib.orc_quantize_rows.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p,
-                                           ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_void_p,
+                                           ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_void_p,
                                            ctypes.c_void_p]
         _lib.orc_dequant_row.restype = None
         _lib.orc_dequant_row.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
-                                         ctypes.c_int, ctypes.c_void_p]
+                                         ctypes.c_int, ctypes.c_int, ctypes.c_void_p]
+        _lib.orc_e4m3_to_f32.restype = ctypes.c_float
+        _lib.orc_e4m3_to_f32.argtypes = [ctypes.c_uint8]
+        _lib.orc_f32_to_e4m3.restype = ctypes.c_uint8
+        _lib.orc_f32_to_e4m3.argtypes = [ctypes.c_float]
         _lib.orc_append.restype = ctypes.c_int
         _lib.orc_append.argtypes = [ctypes.POINTER(_Cache), ctypes.c_void_p, ctypes.c_void_p,
                                     ctypes.c_void_p, ctypes.c_int]
@@ -85,11 +90,20 @@ def f16_bits_to_f32(b: int) -> float:
     return float(lib().orc_f16_to_f32(ctypes.c_uint16(b)))
 
 
-def quantize_rows(x: np.ndarray, idx: np.ndarray, alpha: np.ndarray, bits: int, group: int):
+def f32_to_e4m3_bits(x: float) -> int:
+    return int(lib().orc_f32_to_e4m3(ctypes.c_float(x)))
+
+
+def e4m3_bits_to_f32(b: int) -> float:
+    return float(lib().orc_e4m3_to_f32(ctypes.c_uint8(b)))
+
+
+def quantize_rows(x: np.ndarray, idx: np.ndarray, alpha: np.ndarray, bits: int, group: int, meta_fp8: bool = False):
     """Reorder + clipped group quantization of independent rows.
 
     x: float16 [n, D] in original channel order; idx: int32 [D]; alpha: float32 [D/group].
-    Returns (codes uint8 [n, D*bits/8], meta float16 [n, D/group, 2] = {h, z}).
+    Returns (codes uint8 [n, D*bits/8], meta float16 [n, D/group, 2] = {h, z}); with meta_fp8 the
+    meta array holds the E4M3 byte of h and z as uint16 [n, D/group, 2].
     """
     x = np.ascontiguousarray(x, dtype=np.float16)
     n, D = x.shape
@@ -97,20 +111,20 @@ def quantize_rows(x: np.ndarray, idx: np.ndarray, alpha: np.ndarray, bits: int, 
     alpha = np.ascontiguousarray(alpha, dtype=np.float32)
     assert idx.shape == (D,) and alpha.shape == (D // group,)
     codes = np.zeros((n, D * bits // 8), dtype=np.uint8)
-    meta = np.zeros((n, D // group, 2), dtype=np.float16)
-    lib().orc_quantize_rows(_ptr(x), n, _ptr(idx), _ptr(alpha), D, group, bits, _ptr(codes), _ptr(meta))
+    meta = np.zeros((n, D // group, 2), dtype=np.uint16 if meta_fp8 else np.float16)
+    lib().orc_quantize_rows(_ptr(x), n, _ptr(idx), _ptr(alpha), D, group, bits, int(meta_fp8), _ptr(codes), _ptr(meta))
     return codes, meta
 
 
-def dequant_rows(codes: np.ndarray, meta: np.ndarray, bits: int, group: int) -> np.ndarray:
+def dequant_rows(codes: np.ndarray, meta: np.ndarray, bits: int, group: int, meta_fp8: bool = False) -> np.ndarray:
     """fp64 dequantization x^ = h*c + z of packed rows (no rounding)."""
     codes = np.ascontiguousarray(codes, dtype=np.uint8)
-    meta = np.ascontiguousarray(meta, dtype=np.float16)
+    meta = np.ascontiguousarray(meta, dtype=np.uint16 if meta_fp8 else np.float16)
     n = codes.shape[0]
     D = codes.shape[1] * 8 // bits
     out = np.zeros((n, D), dtype=np.float64)
     for r in range(n):
-        lib().orc_dequant_row(_ptr(codes[r]), _ptr(meta[r]), D, group, bits, _ptr(out[r]))
+        lib().orc_dequant_row(_ptr(codes[r]), _ptr(meta[r]), D, group, bits, int(meta_fp8), _ptr(out[r]))
     return out
 
 
@@ -118,7 +132,7 @@ class OracleCache:
     """Host-side SKVQ cache in the canonical layout, driven by the C oracle."""
 
     def __init__(self, batch, n_q_heads, n_kv_heads, head_dim, k_bits, v_bits, group_size, window,
-                 max_tokens, reorder_k, reorder_v, alpha_k, alpha_v, n_sink=0):
+                 max_tokens, reorder_k, reorder_v, alpha_k, alpha_v, n_sink=0, meta_fp8=False):
         self.B, self.Hq, self.Hkv, self.D = batch, n_q_heads, n_kv_heads, head_dim
         self.k_bits, self.v_bits, self.G, self.W = k_bits, v_bits, group_size, window
         self.ng = head_dim // group_size
@@ -126,8 +140,10 @@ class OracleCache:
         B, H, D, W = batch, n_kv_heads, head_dim, window
         self.k_codes = np.zeros((B, H, self.cap_q, D * k_bits // 8), dtype=np.uint8)
         self.v_codes = np.zeros((B, H, self.cap_q, D * v_bits // 8), dtype=np.uint8)
-        self.k_meta = np.zeros((B, H, self.cap_q, self.ng, 2), dtype=np.float16)
-        self.v_meta = np.zeros((B, H, self.cap_q, self.ng, 2), dtype=np.float16)
+        self.meta_fp8 = bool(meta_fp8)      # scale/zero as FP8 E4M3: the arrays then hold the byte of each as uint16
+        meta_t = np.uint16 if self.meta_fp8 else np.float16
+        self.k_meta = np.zeros((B, H, self.cap_q, self.ng, 2), dtype=meta_t)
+        self.v_meta = np.zeros((B, H, self.cap_q, self.ng, 2), dtype=meta_t)
         self.k_win = np.zeros((B, H, W, D), dtype=np.float16)
         self.v_win = np.zeros((B, H, W, D), dtype=np.float16)
         self.n_sink = int(n_sink)
@@ -144,7 +160,7 @@ class OracleCache:
                       _ptr(self.k_codes), _ptr(self.v_codes), _ptr(self.k_meta), _ptr(self.v_meta),
                       _ptr(self.k_win), _ptr(self.v_win), _ptr(self.lengths),
                       _ptr(self.reorder_k), _ptr(self.reorder_v), _ptr(self.alpha_k), _ptr(self.alpha_v),
-                      self.n_sink, _ptr(self.k_sink), _ptr(self.v_sink))
+                      self.n_sink, _ptr(self.k_sink), _ptr(self.v_sink), int(self.meta_fp8))
 
     def append(self, k: np.ndarray, v: np.ndarray, n_new=None) -> int:
         """k, v: float16 [B, n, Hkv, D], original channel order; n_new: per-sequence counts or None."""

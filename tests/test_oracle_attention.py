@@ -16,7 +16,7 @@ from test_oracle_quantizer import unpack_codes
 D = 128
 
 
-def make_cache(B, Hq, Hkv, W, cap, bits=2, group=128, alpha=0.9, seed=0, identity=False, n_sink=0):
+def make_cache(B, Hq, Hkv, W, cap, bits=2, group=128, alpha=0.9, seed=0, identity=False, n_sink=0, meta_fp8=False):
     rng = np.random.default_rng(seed)
     if identity:
         rk = rv = np.tile(np.arange(D, dtype=np.int32), (Hkv, 1))
@@ -24,7 +24,7 @@ def make_cache(B, Hq, Hkv, W, cap, bits=2, group=128, alpha=0.9, seed=0, identit
         rk = np.stack([rng.permutation(D) for _ in range(Hkv)]).astype(np.int32)
         rv = np.stack([rng.permutation(D) for _ in range(Hkv)]).astype(np.int32)
     a = np.full((Hkv, D // group), alpha, np.float32)
-    return orc.OracleCache(B, Hq, Hkv, D, bits, bits, group, W, cap, rk, rv, a, a, n_sink=n_sink)
+    return orc.OracleCache(B, Hq, Hkv, D, bits, bits, group, W, cap, rk, rv, a, a, n_sink=n_sink, meta_fp8=meta_fp8)
 
 
 def rand_kv(B, n, Hkv, seed):
@@ -49,8 +49,13 @@ def mixed_cache_dense(c, b, hk):
     for codes, meta, win, sink, bits in ((c.k_codes, c.k_meta, c.k_win, c.k_sink, c.k_bits),
                                          (c.v_codes, c.v_meta, c.v_win, c.v_sink, c.v_bits)):
         code = unpack_codes(codes[b, hk, :Lq], bits).astype(np.float64)
-        h = np.repeat(meta[b, hk, :Lq, :, 0].astype(np.float64), c.G, axis=1)
-        z = np.repeat(meta[b, hk, :Lq, :, 1].astype(np.float64), c.G, axis=1)
+        if c.meta_fp8:                               # E4M3 bytes: decoded by a library, not by the oracle
+            import torch
+            meta = torch.from_numpy(meta[b, hk, :Lq].astype(np.uint8)).view(torch.float8_e4m3fn).to(torch.float64).numpy()
+        else:
+            meta = meta[b, hk, :Lq]
+        h = np.repeat(meta[:, :, 0].astype(np.float64), c.G, axis=1)
+        z = np.repeat(meta[:, :, 1].astype(np.float64), c.G, axis=1)
         dense = np.zeros((L, D))
         dense[:Lq] = h * code + z
         ns = min(c.n_sink, Lq)                       # attention sinks: full-precision rows, never quantized
@@ -262,6 +267,23 @@ def test_sink_attention_matches_library_brute_force(Hq, Hkv, bits, group, W, n_s
     q = np.random.default_rng(3).standard_normal((1, Hq, D)).astype(np.float16)
     got = c.attention(q, 0.088)
     assert np.abs(got - brute_attention(c, q, 0.088)).max() < 1e-12
+
+
+@pytest.mark.parametrize("Hq,Hkv,bits,group,W,n_sink,L", [(4, 2, 2, 32, 16, 0, 150), (4, 4, 4, 64, 8, 3, 90), (8, 2, 2, 128, 0, 0, 77)])
+def test_fp8_parameter_attention_matches_library_brute_force(Hq, Hkv, bits, group, W, n_sink, L):
+    """Scale and zero point stored in E4M3: the oracle against numpy/scipy over a cache dequantized with a library's
+    E4M3 decoding; and single appends equal one bulk append."""
+    k, v = rand_kv(1, L, Hkv, seed=23)
+    c = make_cache(1, Hq, Hkv, W, 256, bits=bits, group=group, n_sink=n_sink, seed=12, meta_fp8=True)
+    c.append(k, v)
+    assert c.k_meta.max() <= 255 and c.k_meta[0, :, n_sink:max(L - W, 0)].any()
+    q = np.random.default_rng(4).standard_normal((1, Hq, D)).astype(np.float16)
+    got = c.attention(q, 0.088)
+    assert np.abs(got - brute_attention(c, q, 0.088)).max() < 1e-12
+    c1 = make_cache(1, Hq, Hkv, W, 256, bits=bits, group=group, n_sink=n_sink, seed=12, meta_fp8=True)
+    for t in range(L):
+        c1.append(k[:, t:t + 1], v[:, t:t + 1])
+    assert np.array_equal(c1.k_codes, c.k_codes) and np.array_equal(c1.v_meta, c.v_meta)
 
 
 def test_all_sinks_and_no_window_is_plain_attention():

@@ -266,3 +266,80 @@ def test_average_bits_match_paper():
         assert stored_bits / D == pytest.approx(want, abs=1e-12)
         if param_bits == 16:                                              # what the oracle really stores
             assert (codes[0].nbytes + meta[0].nbytes) * 8 / D == pytest.approx(want, abs=1e-12)
+        else:                                                             # FP8 mode: one byte per parameter
+            codes8, meta8 = orc.quantize_rows(x, ident(), np.ones(D // group, np.float32), bits, group, meta_fp8=True)
+            assert meta8.max() <= 255
+            assert (codes8[0].nbytes + meta8[0].size) * 8 / D == pytest.approx(want, abs=1e-12)
+
+
+# ------------------------------------------------------------------ FP8 E4M3 parameters (Sec. 4.1, component breakdown)
+def _torch_e4m3():
+    import torch
+    if not hasattr(torch, "float8_e4m3fn"):
+        pytest.skip("this torch has no float8_e4m3fn")
+    return torch
+
+
+def test_e4m3_decode_all_bytes_match_library():
+    torch = _torch_e4m3()
+    want = torch.arange(256, dtype=torch.uint8).view(torch.float8_e4m3fn).to(torch.float32).numpy()
+    got = np.array([orc.e4m3_bits_to_f32(b) for b in range(256)], np.float32)
+    assert np.array_equal(np.isnan(got), np.isnan(want)) and np.isnan(got).sum() == 2       # S.1111.111 only
+    ok = ~np.isnan(want)
+    assert np.array_equal(got[ok].view(np.uint32), want[ok].view(np.uint32))
+    assert got[0x7E] == 448.0 and got[0x01] == 2.0 ** -9 and got[0x08] == 2.0 ** -6 and got[0x38] == 1.0
+
+
+def test_e4m3_encode_matches_library_round_to_nearest_even():
+    """Random values over the whole finite range, every representable value, and every midpoint between two
+    neighbours (ties must go to the even mantissa)."""
+    torch = _torch_e4m3()
+    rng = np.random.default_rng(5)
+    grid = np.array([orc.e4m3_bits_to_f32(b) for b in range(0x7F)], np.float64)              # 0 .. 448, ascending
+    mids = (grid[:-1] + grid[1:]) / 2
+    x = np.concatenate([grid, mids, np.nextafter(mids.astype(np.float32), np.float32(0)).astype(np.float64),
+                        np.nextafter(mids.astype(np.float32), np.float32(1e9)).astype(np.float64),
+                        rng.uniform(-448, 448, 4000), np.ldexp(rng.uniform(-1, 1, 4000), rng.integers(-14, 9, 4000))])
+    x = np.concatenate([x, -x]).astype(np.float32)
+    x = x[np.abs(x) <= 448]
+    want = torch.from_numpy(x).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    got = np.array([orc.f32_to_e4m3_bits(float(v)) for v in x], np.uint8)
+    assert np.array_equal(got, want)
+
+
+def test_e4m3_encode_saturates_and_keeps_the_grid():
+    for v in (448.5, 463.9, 464.0, 480.0, 1e4, 6.5e4, float("inf")):
+        assert orc.f32_to_e4m3_bits(v) == 0x7E and orc.f32_to_e4m3_bits(-v) == 0xFE
+    for b in range(0x7F):                                                   # encoding a representable value is the identity
+        assert orc.f32_to_e4m3_bits(orc.e4m3_bits_to_f32(b)) == b
+    assert orc.f32_to_e4m3_bits(2.0 ** -10) == 0x00 and orc.f32_to_e4m3_bits(3 * 2.0 ** -10) == 0x02    # ties to even
+
+
+@pytest.mark.parametrize("bits,group", [(2, 32), (2, 128), (4, 64)])
+def test_fp8_parameters_are_the_rounded_fp32_ones_and_codes_use_them(bits, group):
+    """Eq. 2 with the parameters stored in E4M3: h8 = e4m3(alpha (max - min) / qmax), z8 = e4m3(alpha min), and the
+    codes are the nearest levels of the grid those stored values define (brute force in fp64)."""
+    qmax = 2 ** bits - 1
+    x = random_rows(40, 31)
+    alpha = np.full(D // group, 0.9, np.float32)
+    codes, meta = orc.quantize_rows(x, ident(), alpha, bits, group, meta_fp8=True)
+    c = unpack_codes(codes, bits)
+    for r in range(x.shape[0]):
+        for g in range(D // group):
+            seg = x[r, g * group:(g + 1) * group].astype(np.float32)
+            lo, hi = np.float32(0.9) * seg.min(), np.float32(0.9) * seg.max()
+            h8, z8 = orc.f32_to_e4m3_bits(float((hi - lo) / np.float32(qmax))), orc.f32_to_e4m3_bits(float(lo))
+            assert (int(meta[r, g, 0]), int(meta[r, g, 1])) == (h8, z8)
+            h, z = orc.e4m3_bits_to_f32(h8), orc.e4m3_bits_to_f32(z8)
+            levels = z + h * np.arange(qmax + 1)
+            want = np.abs(seg.astype(np.float64)[:, None] - levels[None, :]).argmin(axis=1)
+            got = c[r, g * group:(g + 1) * group]
+            # an element may sit within rounding distance of the midpoint between two levels: accept either there
+            d = np.abs(seg.astype(np.float64) - levels[got]) - np.abs(seg.astype(np.float64) - levels[want])
+            assert np.all(d <= 1e-6 * max(h, 1e-30) + 1e-12)
+    xhat = orc.dequant_rows(codes, meta, bits, group, meta_fp8=True)
+    h_all = np.repeat(np.vectorize(orc.e4m3_bits_to_f32)(meta[:, :, 0].astype(np.uint8)), group, axis=1)
+    z_all = np.repeat(np.vectorize(orc.e4m3_bits_to_f32)(meta[:, :, 1].astype(np.uint8)), group, axis=1)
+    assert np.array_equal(xhat, h_all.astype(np.float64) * c + z_all.astype(np.float64))
+    inside = (x >= z_all) & (x <= z_all + qmax * h_all)                    # inside the stored grid the error is half a step
+    assert np.all(np.abs(x.astype(np.float64) - xhat)[inside] <= 0.5 * h_all[inside] * (1 + 1e-6))
