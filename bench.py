@@ -156,7 +156,7 @@ def oracle_sample(w, n_seq, n_kv=None):
 
     def new(batch):
         return orc.OracleCache(batch, n_kv * rep, n_kv, w.head_dim, w.k_bits, w.v_bits, w.group_size, w.window,
-                               cap, rk, rv, a, a, n_sink=w.n_sink)
+                               cap, rk, rv, a, a, n_sink=w.n_sink, meta_fp8=w.meta_fp8)
     oc = new(n_seq)
     for b in range(n_seq):
         one = new(1)
@@ -237,6 +237,8 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (small profiling cases)")
     ap.add_argument("--context", type=int, default=0, help="override the context length (small profiling cases)")
     ap.add_argument("--q-heads", type=int, default=0, help="override the number of query heads (other grouped-query ratios)")
+    ap.add_argument("--meta-fp8", action="store_true",
+                    help="scale and zero point stored in FP8 E4M3 instead of fp16 (Sec. 4.1; 2.5 bits per element at g32)")
     ap.add_argument("--sinks", type=int, default=0,
                     help="attention sinks: first positions kept fp16 (Sec. 3.2 filter rule; the paper's experiments use 5)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -257,6 +259,8 @@ def main():
         w0 = w0.scaled(n_sink=args.sinks)
     if args.q_heads:
         w0 = w0.scaled(n_q_heads=args.q_heads)
+    if args.meta_fp8:
+        w0 = w0.scaled(meta_fp8=True)
 
     if args.impl == "reference":
         run_reference(args, w0, rank)
@@ -290,10 +294,14 @@ def main():
         oc = oracle_sample(w, 1)
         lq = max(int(lengths0[0]) - w.window, 0)
         ns = min(w.n_sink, lq)      # sink rows: fp16 copies instead of codes
+
+        def meta_bits(t):           # fp16 bit patterns, or one E4M3 byte per parameter (the oracle keeps each in a uint16)
+            a = t[0, :, ns:lq].cpu().numpy()
+            return a.astype(np.uint16) if w.meta_fp8 else a.view(np.uint16)
         exact = bool(np.array_equal(cache.k_codes[0, :, ns:lq].cpu().numpy(), oc.k_codes[0, :, ns:lq]) and
                      np.array_equal(cache.v_codes[0, :, ns:lq].cpu().numpy(), oc.v_codes[0, :, ns:lq]) and
-                     np.array_equal(cache.k_meta[0, :, ns:lq].cpu().numpy().view(np.uint16), oc.k_meta.view(np.uint16)[0, :, ns:lq]) and
-                     np.array_equal(cache.v_meta[0, :, ns:lq].cpu().numpy().view(np.uint16), oc.v_meta.view(np.uint16)[0, :, ns:lq]) and
+                     np.array_equal(meta_bits(cache.k_meta), oc.k_meta.view(np.uint16)[0, :, ns:lq]) and
+                     np.array_equal(meta_bits(cache.v_meta), oc.v_meta.view(np.uint16)[0, :, ns:lq]) and
                      np.array_equal(cache.k_sink[0, :, :ns].cpu().numpy().view(np.uint16), oc.k_sink.view(np.uint16)[0, :, :ns]) and
                      np.array_equal(cache.v_sink[0, :, :ns].cpu().numpy().view(np.uint16), oc.v_sink.view(np.uint16)[0, :, :ns]))
         q = w.query(10_000)
@@ -429,7 +437,7 @@ def main():
         "config": {"workload": f"configs[{args.config}] {w.name}", "batch": w.batch, "n_q_heads": w.n_q_heads,
                    "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "context": int(lengths0.max()),
                    "window": w.window, "k_bits": w.k_bits, "v_bits": w.v_bits, "group_size": w.group_size,
-                   "alpha": w.alpha, "n_sink": w.n_sink, "step": "append 1 token/sequence + decode attention",
+                   "alpha": w.alpha, "n_sink": w.n_sink, "meta_fp8": bool(w.meta_fp8), "step": "append 1 token/sequence + decode attention",
                    "cache_bytes": cache.nbytes(),
                    "l2": "cache larger than L2, streamed every step" if flush is None else "L2 flushed between steps",
                    "parallelism": f"replica per GPU x{world}" if world > 1 else "single GPU"},
@@ -441,7 +449,7 @@ def main():
                      "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
                      "frac_of_nominal_8000": achieved / 8000.0,
                      "algorithmic_bytes_per_launch": part_bytes, "kernel_ms_avg": kavg_ms,
-                     "kernel_ms_min": min(kern_ms), "traffic": NCU_TRAFFIC_BYTES.get(args.config) if not (args.batch or args.context or args.sinks or args.q_heads) else None,
+                     "kernel_ms_min": min(kern_ms), "traffic": NCU_TRAFFIC_BYTES.get(args.config) if not (args.batch or args.context or args.sinks or args.q_heads or args.meta_fp8) else None,
                      "whole_call": {"what": "partition + merge kernels, all algorithmic bytes (codes, scale/zero, "
                                             "fp16 window, q, out)", "algorithmic_bytes": alg_bytes, "ms_avg": cavg_ms,
                                     "achieved": alg_bytes / (cavg_ms * 1e-3) / 1e9,

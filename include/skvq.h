@@ -68,6 +68,9 @@ typedef struct skvq_config {
     int32_t max_tokens;  /* per-sequence capacity (quantized segment + window) */
     int32_t n_sink;      /* 0..64: the first n_sink positions of a sequence are never quantized (Sec. 3.2, filter
                             rules; the paper's experiments keep 5); 0 = none */
+    int32_t meta_fp8;    /* 0: scale and zero point stored in fp16; 1: in FP8 E4M3 (Sec. 4.1 "Quantization"; 2.5
+                            instead of 3 bits per element at 2 bits and group 32).  The codes are computed
+                            against the stored, rounded parameters either way. */
 } skvq_config;
 
 /*
@@ -75,7 +78,10 @@ typedef struct skvq_config {
  * Layouts are row-major:
  *   k_codes/v_codes  uint8   [B][Hkv][cap][D*bits/8]  code j of a row = bits [(j*bits)%8, +bits) of
  *                                                     byte (j*bits)/8, j counted in reordered order
- *   k_meta/v_meta    half2   [B][Hkv][cap][ng]        {scale h, zero z}; dequantized x^ = h*code + z
+ *   k_meta/v_meta    half2   [B][Hkv][cap][ng]        {scale h, zero z}; dequantized x^ = h*code + z.  With meta_fp8:
+ *                    uint8   [B][Hkv][cap][ng][2]     {E4M3 byte of h, E4M3 byte of z} (1 sign, 4 exponent bits with
+ *                                                     bias 7, 3 mantissa bits, no infinities, largest finite 448;
+ *                                                     rounded to nearest even from fp32, saturating)
  *   k_win/v_win      half    [B][Hkv][W][D]           ring; token t sits in slot t % W, reordered order
  *   lengths          int32   [B]                      tokens appended so far (start at 0)
  *   reorder_k/_v     int32   [Hkv][D]                 gather index: stored[j] = source[idx[j]]; each

@@ -30,7 +30,7 @@ EXPORTS = ["skvq_version", "skvq_strerror", "skvq_launch_count", "skvq_check_con
 
 class SkvqConfig(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in ("batch", "n_q_heads", "n_kv_heads", "head_dim", "k_bits", "v_bits",
-                                              "group_size", "window", "max_tokens", "n_sink")]
+                                              "group_size", "window", "max_tokens", "n_sink", "meta_fp8")]
 
 
 class SkvqCacheStruct(ctypes.Structure):
@@ -174,9 +174,9 @@ class SkvqCache:
     """
 
     def __init__(self, batch, n_q_heads, n_kv_heads, head_dim, k_bits, v_bits, group_size, window, max_tokens,
-                 reorder_k, reorder_v, alpha_k, alpha_v, device="cuda:0", n_sink=0):
+                 reorder_k, reorder_v, alpha_k, alpha_v, device="cuda:0", n_sink=0, meta_fp8=False):
         self.cfg = SkvqConfig(batch, n_q_heads, n_kv_heads, head_dim, k_bits, v_bits, group_size, window, max_tokens,
-                              n_sink)
+                              n_sink, 1 if meta_fp8 else 0)
         _check(skvq_check_config(self.cfg), "skvq_check_config")
         self.device = torch.device(device)
         self.cap = skvq_quant_capacity(self.cfg)
@@ -186,8 +186,9 @@ class SkvqCache:
         dev = self.device
         self.k_codes = torch.zeros((B, H, self.cap, D * k_bits // 8), dtype=torch.uint8, device=dev)
         self.v_codes = torch.zeros((B, H, self.cap, D * v_bits // 8), dtype=torch.uint8, device=dev)
-        self.k_meta = torch.zeros((B, H, self.cap, self.ng, 2), dtype=torch.float16, device=dev)
-        self.v_meta = torch.zeros((B, H, self.cap, self.ng, 2), dtype=torch.float16, device=dev)
+        meta_t = torch.uint8 if meta_fp8 else torch.float16      # {h, z} per (token, group): E4M3 bytes or fp16
+        self.k_meta = torch.zeros((B, H, self.cap, self.ng, 2), dtype=meta_t, device=dev)
+        self.v_meta = torch.zeros((B, H, self.cap, self.ng, 2), dtype=meta_t, device=dev)
         self.k_win = torch.zeros((B, H, max(W, 1), D), dtype=torch.float16, device=dev)
         self.v_win = torch.zeros((B, H, max(W, 1), D), dtype=torch.float16, device=dev)
         got = [t.numel() * t.element_size() for t in (self.k_codes, self.v_codes, self.k_meta, self.v_meta)]
@@ -211,7 +212,8 @@ class SkvqCache:
         """Cache for a ``workloads.Workload`` with its reorder index and clip factors."""
         mt = w.context if max_tokens is None else max_tokens
         return cls(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.k_bits, w.v_bits, w.group_size, w.window, mt,
-                   w.reorder_index("k"), w.reorder_index("v"), w.alphas(), w.alphas(), device=device, n_sink=w.n_sink)
+                   w.reorder_index("k"), w.reorder_index("v"), w.alphas(), w.alphas(), device=device, n_sink=w.n_sink,
+                   meta_fp8=w.meta_fp8)
 
     def nbytes(self) -> int:
         return sum(t.numel() * t.element_size() for t in (self.k_codes, self.v_codes, self.k_meta, self.v_meta,

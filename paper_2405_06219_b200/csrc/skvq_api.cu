@@ -21,6 +21,7 @@ static int check_cfg(const skvq_config *c)
     if (c->n_q_heads / c->n_kv_heads > kMaxRep) return SKVQ_ERR_UNSUPPORTED;
     if (c->n_sink < 0) return SKVQ_ERR_INVALID_ARG;
     if (c->n_sink > 64) return SKVQ_ERR_UNSUPPORTED;
+    if (c->meta_fp8 != 0 && c->meta_fp8 != 1) return SKVQ_ERR_INVALID_ARG;
     return SKVQ_OK;
 }
 
@@ -48,6 +49,7 @@ static Shape make_shape(const skvq_config *c)
     s.cap = quant_capacity(c);
     s.max_tokens = c->max_tokens;
     s.n_sink = c->n_sink;
+    s.meta_fp8 = c->meta_fp8;
     return s;
 }
 
@@ -129,8 +131,8 @@ int skvq_cache_sizes(const skvq_config *cfg, size_t bytes_out[6])
     const size_t rows = (size_t)s.B * s.Hkv * s.cap;
     bytes_out[0] = rows * (kHeadDim * s.k_bits / 8);
     bytes_out[1] = rows * (kHeadDim * s.v_bits / 8);
-    bytes_out[2] = rows * s.ng * sizeof(__half2);
-    bytes_out[3] = rows * s.ng * sizeof(__half2);
+    bytes_out[2] = rows * s.ng * (s.meta_fp8 ? 2 : sizeof(__half2));
+    bytes_out[3] = bytes_out[2];
     bytes_out[4] = (size_t)s.B * s.Hkv * s.W * kHeadDim * sizeof(__half);
     bytes_out[5] = bytes_out[4];
     return SKVQ_OK;

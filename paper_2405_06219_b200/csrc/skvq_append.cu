@@ -65,9 +65,25 @@ __device__ __noinline__ void quantize16_exact(const float (&x)[16], float zf, fl
 }
 
 // Quantize the 16 channels held by this lane; `lanes_per_group` lanes share the group statistics.
+// fp32 scale and zero point -> the two E4M3 bytes {h, z} (round to nearest even, saturating at 448) ...
+__device__ __forceinline__ uint16_t to_e4m3x2(float h, float z)
+{
+    uint16_t r;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(z), "f"(h));      // first operand -> upper byte
+    return r;
+}
+// ... and back: {h, z} as a half2 (every E4M3 value is an fp16 value)
+__device__ __forceinline__ __half2 from_e4m3x2(uint16_t b)
+{
+    uint32_t r;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(r) : "h"(b));
+    return *reinterpret_cast<const __half2 *>(&r);
+}
+
+// Writes what is stored per (token, group): a half2 {h, z}, or its two E4M3 bytes in the low 16 bits of hz_bits.
 template <int BITS>
-__device__ __forceinline__ void quantize16(const float (&x)[16], float alpha, int lanes_per_group, uint32_t (&words)[2],
-                                           __half2 &hz)
+__device__ __forceinline__ void quantize16(const float (&x)[16], float alpha, int lanes_per_group, bool meta_fp8,
+                                           uint32_t (&words)[2], uint32_t &hz_bits)
 {
     // The 8 lanes that own one row always take the same path, so they are the shuffle's member set
     // (K and V rows may use different bit widths and therefore different instantiations).
@@ -87,11 +103,17 @@ __device__ __forceinline__ void quantize16(const float (&x)[16], float alpha, in
     const float lo = __fadd_rn(__fmul_rn(alpha, mn), 0.0f);
     const float hi = __fadd_rn(__fmul_rn(alpha, mx), 0.0f);
     const float h32 = __fdiv_rn(__fsub_rn(hi, lo), (float)qmax);
-    const __half h16 = __float2half_rn(h32);
-    const __half z16 = __float2half_rn(lo);
-    const float hf = __half2float(h16);
-    const float zf = __half2float(z16);
-    hz = __halves2half2(h16, z16);
+    __half2 hz;      // the stored parameters: the codes are computed against these
+    if (meta_fp8) {
+        const uint16_t b = to_e4m3x2(h32, lo);
+        hz = from_e4m3x2(b);
+        hz_bits = b;
+    } else {
+        hz = __halves2half2(__float2half_rn(h32), __float2half_rn(lo));
+        hz_bits = *reinterpret_cast<const uint32_t *>(&hz);
+    }
+    const float hf = __low2float(hz);
+    const float zf = __high2float(hz);
     words[0] = 0u;
     words[1] = 0u;
     if (hf != 0.0f) {
@@ -157,7 +179,9 @@ __global__ void __launch_bounds__(kAppendThreads) append_kernel(AppendArgs a)
     const int row_bytes = kHeadDim * bits / 8;
     const size_t bh = (size_t)b * s.Hkv + h;
     uint8_t *codes = (is_v ? a.c.v_codes : a.c.k_codes) + bh * (size_t)s.cap * row_bytes;
-    __half2 *meta = (is_v ? a.c.v_meta : a.c.k_meta) + bh * (size_t)s.cap * s.ng;
+    __half2 *meta = (is_v ? a.c.v_meta : a.c.k_meta);      // two bytes per (token, group) with FP8 parameters
+    const size_t meta0 = bh * (size_t)s.cap * s.ng;
+    const bool f8 = s.meta_fp8 != 0;
     __half *win = (is_v ? a.c.v_win : a.c.k_win) + bh * (size_t)W * kHeadDim;
     const __half *src = (is_v ? a.v : a.k) + ((size_t)b * a.n_new * s.Hkv + h) * kHeadDim;   // token stride Hkv*D
     const size_t src_tok_stride = (size_t)s.Hkv * kHeadDim;
@@ -227,9 +251,9 @@ __global__ void __launch_bounds__(kAppendThreads) append_kernel(AppendArgs a)
             const int g = (sub << 4) / s.G;
             const float alpha = alpha_head[g];
             uint32_t words[2];
-            __half2 hz;
-            if (bits == 2) quantize16<2>(x, alpha, lanes_per_group, words, hz);
-            else quantize16<4>(x, alpha, lanes_per_group, words, hz);
+            uint32_t hz;
+            if (bits == 2) quantize16<2>(x, alpha, lanes_per_group, f8, words, hz);
+            else quantize16<4>(x, alpha, lanes_per_group, f8, words, hz);
             if (do_quant && t < s.n_sink) {
                 // an attention sink (Sec. 3.2 filter rule): its reordered fp16 row is kept as it is
                 __align__(16) __half xh16[16];
@@ -243,7 +267,11 @@ __global__ void __launch_bounds__(kAppendThreads) append_kernel(AppendArgs a)
                 uint8_t *codes_row = codes + (size_t)t * row_bytes;
                 if (bits == 2) reinterpret_cast<uint32_t *>(codes_row)[sub] = words[0];
                 else reinterpret_cast<uint2 *>(codes_row)[sub] = make_uint2(words[0], words[1]);
-                if ((sub & (lanes_per_group - 1)) == 0) meta[(size_t)t * s.ng + g] = hz;
+                if ((sub & (lanes_per_group - 1)) == 0) {
+                    const size_t mi = meta0 + (size_t)t * s.ng + g;
+                    if (f8) reinterpret_cast<uint16_t *>(meta)[mi] = (uint16_t)hz;
+                    else reinterpret_cast<uint32_t *>(meta)[mi] = hz;
+                }
             }
         }
         if (do_ring_write) {
@@ -303,7 +331,9 @@ __global__ void __launch_bounds__(kAppendThreads) append_bulk_kernel(AppendArgs 
         const int bits = tensor ? s.v_bits : s.k_bits;
         const int row_bytes = kHeadDim * bits / 8;
         uint8_t *codes = (tensor ? a.c.v_codes : a.c.k_codes) + bh * (size_t)s.cap * row_bytes;
-        __half2 *meta = (tensor ? a.c.v_meta : a.c.k_meta) + bh * (size_t)s.cap * s.ng;
+        __half2 *meta = (tensor ? a.c.v_meta : a.c.k_meta);      // two bytes per (token, group) with FP8 parameters
+        const size_t meta0 = bh * (size_t)s.cap * s.ng;
+        const bool f8 = s.meta_fp8 != 0;
         const float alpha = ((tensor ? a.c.alpha_v : a.c.alpha_k) + (size_t)h * s.ng)[g];
         int idx[16];
         {
@@ -321,14 +351,18 @@ __global__ void __launch_bounds__(kAppendThreads) append_bulk_kernel(AppendArgs 
 #pragma unroll
             for (int j = 0; j < 16; ++j) x[j] = __half2float(src_j[j][it * 16 * kBulkStride]);
             uint32_t words[2];
-            __half2 hz;
-            if (bits == 2) quantize16<2>(x, alpha, lanes_per_group, words, hz);
-            else quantize16<4>(x, alpha, lanes_per_group, words, hz);
+            uint32_t hz;
+            if (bits == 2) quantize16<2>(x, alpha, lanes_per_group, f8, words, hz);
+            else quantize16<4>(x, alpha, lanes_per_group, f8, words, hz);
             const int t = t0 + tok;
             uint8_t *codes_row = codes + (size_t)t * row_bytes;
             if (bits == 2) reinterpret_cast<uint32_t *>(codes_row)[sub] = words[0];
             else reinterpret_cast<uint2 *>(codes_row)[sub] = make_uint2(words[0], words[1]);
-            if ((sub & (lanes_per_group - 1)) == 0) meta[(size_t)t * s.ng + g] = hz;
+            if ((sub & (lanes_per_group - 1)) == 0) {
+                const size_t mi = meta0 + (size_t)t * s.ng + g;
+                if (f8) reinterpret_cast<uint16_t *>(meta)[mi] = (uint16_t)hz;
+                else reinterpret_cast<uint32_t *>(meta)[mi] = hz;
+            }
         }
     }
 }

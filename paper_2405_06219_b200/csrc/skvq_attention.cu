@@ -96,8 +96,17 @@ __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
     constexpr int KQMAX = (1 << KBITS) - 1, VQMAX = (1 << VBITS) - 1;
     const uint8_t *k_codes = a.c.k_codes + bh * (size_t)s.cap * KROW;
     const uint8_t *v_codes = a.c.v_codes + bh * (size_t)s.cap * VROW;
-    const __half2 *k_meta = a.c.k_meta + bh * (size_t)s.cap * ng;
-    const __half2 *v_meta = a.c.v_meta + bh * (size_t)s.cap * ng;
+    // {h, z} of row r, group g: a half2, or two E4M3 bytes (every E4M3 value is an fp16 value)
+    const bool f8 = s.meta_fp8 != 0;
+    auto load_hz = [&](const __half2 *base, size_t idx) -> float2 {
+        if (!f8) return __half22float2(base[idx]);
+        const uint16_t b = reinterpret_cast<const uint16_t *>(base)[idx];
+        uint32_t r;
+        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(r) : "h"(b));
+        return __half22float2(*reinterpret_cast<const __half2 *>(&r));
+    };
+    const size_t meta0 = bh * (size_t)s.cap * ng;
+    const __half2 *k_meta = a.c.k_meta, *v_meta = a.c.v_meta;
 
     float m_run[kMaxRep], l_thread[kMaxRep], acc[kMaxRep];
 #pragma unroll
@@ -132,7 +141,7 @@ __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
                                     if (r < rep) part[r] = fmaf(sq[r][j], code, part[r]);
                             }
                         }
-                        const float2 hz = __half22float2(k_meta[(size_t)t * ng + g]);
+                        const float2 hz = load_hz(k_meta, meta0 + (size_t)t * ng + g);
 #pragma unroll
                         for (int r = 0; r < kMaxRep; ++r)
                             if (r < rep) sc[r] += hz.x * part[r] + hz.y * sqsum[r][g];
@@ -175,7 +184,7 @@ __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
                 for (int tt = max(s.n_sink - tile0, 0); tt < n_tok; ++tt) {      // rows of sinks hold unspecified bytes
                     const size_t row = (size_t)(tile0 + tt);
                     const uint32_t word = __ldg(reinterpret_cast<const uint32_t *>(v_codes + row * VROW) + w);
-                    const float2 hz = __half22float2(v_meta[row * ng + g]);
+                    const float2 hz = load_hz(v_meta, meta0 + row * ng + g);
                     const float val = fmaf(hz.x, (float)((word >> sh) & VQMAX), hz.y);
 #pragma unroll
                     for (int r = 0; r < kMaxRep; ++r)
@@ -408,6 +417,8 @@ __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
 // Resident CTAs per SM of the partition kernel that serves this shape (sets how many CTAs make one wave).
 static int partition_ctas_per_sm(const Shape &s)
 {
+    if (s.meta_fp8)      // FP8 parameters: the tcgen05 kernel where it applies, else the scalar kernel
+        return (s.k_bits == 2 && s.v_bits == 2 && s.rep <= 8 && (s.G == 128 || s.G == 64 || s.G == 32)) ? 3 : 8;
     if (s.rep == 1 && s.G >= 64) return s.k_bits == s.v_bits ? 4 : 3;           // integer kernel
     if (s.k_bits == 2 && s.v_bits == 2 && (s.rep == 3 || (s.rep > 4 && s.rep <= 8)) && (s.G == 128 || s.G == 64 || s.G == 32))
         return 3;                                                              // tcgen05 kernel: 128 tensor-memory columns, 69 KB

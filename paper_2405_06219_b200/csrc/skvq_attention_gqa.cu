@@ -16,7 +16,8 @@
 // "four tokens of one byte column" registers, one AND leaves 4^j*code bytes, and p*h per group goes on a
 // 32-bit fixed-point grid whose four bytes are four A rows.  The integer accumulators are exact; they are
 // folded into fp32 (shared memory) only when the softmax reference or the bound on h moves, and the
-// reference only moves when a score exceeds it by 16 in the log2 domain, which after the first tile is rare.
+// reference only moves when a score exceeds it by 12 in the log2 domain (a factor 4096: the 32-bit grid then still
+// resolves 2^-20 of the largest p*h), which after the first tiles is rare.
 // sum_t p_t z_{t,g} is one more small fp16 MMA per 16 tokens.
 //
 // One CTA = 4 independent warps on one (sequence, KV head, split); tiles of 64 tokens arrive through a per-warp
@@ -29,7 +30,7 @@ namespace {
 using namespace mmak;
 
 constexpr int kHeadSlots = 4;           // query heads per KV head this kernel serves (rows = head x 4 digits)
-constexpr int kRefSlackLog2 = 16;       // the softmax reference moves only when a score exceeds it by this (log2)
+constexpr int kRefSlackLog2 = 12;       // the softmax reference moves only when a score exceeds it by this (log2)
 constexpr float kRefSlack = (float)kRefSlackLog2;
 
 template <int G>
@@ -628,7 +629,7 @@ cudaError_t launch_partition_gqa(const Shape &s, const CachePtrs &c, const __hal
                                  const SplitPlan &plan, float *workspace, cudaStream_t stream, bool overlap, bool *handled)
 {
     *handled = false;
-    if (s.k_bits != 2 || s.v_bits != 2) return cudaSuccess;
+    if (s.k_bits != 2 || s.v_bits != 2 || s.meta_fp8) return cudaSuccess;      // this kernel reads fp16 scale/zero pairs
     MmaArgs a{s, c, q, scale_log2, plan, workspace};
     switch (s.G) {
         case 128: return launch_g<128>(a, stream, overlap, handled);

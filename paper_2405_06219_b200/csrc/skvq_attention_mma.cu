@@ -489,6 +489,7 @@ cudaError_t launch_partition_mma(const Shape &s, const CachePtrs &c, const __hal
                                  const SplitPlan &plan, float *workspace, cudaStream_t stream, bool overlap, bool *handled)
 {
     *handled = false;
+    if (s.meta_fp8) return cudaSuccess;      // this kernel reads fp16 scale/zero pairs
     if (s.rep != 1 || (s.G != 64 && s.G != 128)) return cudaSuccess;
     MmaArgs a{s, c, q, scale_log2, plan, workspace};
     *handled = true;

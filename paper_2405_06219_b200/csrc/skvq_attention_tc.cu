@@ -12,7 +12,7 @@
 //     accumulators are the exact group dot products: one MMA k-step (32 channels) per 32 channels, a fresh set of
 //     16 columns (head, digit) per quantization group.
 //   * the thread reads its row of accumulators from tensor memory, combines digits and groups with h and z (fp32),
-//     and takes part in a lazy online softmax: the reference of a head moves only when a score exceeds it by 16 in
+//     and takes part in a lazy online softmax: the reference of a head moves only when a score exceeds it by 8 in
 //     the log2 domain (or the bound on the value scales has to grow), which after the first tile is rare.
 //   * p*h per (head, group) goes onto a 32-bit fixed-point grid; the four bytes of that integer are four rows
 //     (head, digit) of the A operand of the value MMA (u8, MN-major: one 16-byte store per group), whose B operand
@@ -30,7 +30,7 @@ using namespace mmak;
 
 constexpr int kTile = 128;              // tokens per tile = rows of the score MMA = threads per CTA
 constexpr int kHeads = 4;               // query heads per KV head served (absent heads carry a zero query)
-constexpr int kSlackLog2 = 16;          // the softmax reference moves only when a score exceeds it by this (log2)
+constexpr int kSlackLog2 = 8;           // the softmax reference moves only when a score exceeds it by this (log2)
 constexpr int kRing = 2;                // slots of each of the two copy rings
 constexpr int kTmemCols = 128;          // allocation: scores in columns [0, 64), value sums in [64, 128)
 constexpr int kScoreCol = 0, kPvCol = 64;
@@ -42,11 +42,12 @@ constexpr uint32_t kSboMN = 2048;       // MN-major operands: bytes between 16-b
 
 // Shared memory.  The K codes of a tile are needed one tile before everything else of it (its score MMA is issued
 // that far ahead), so they travel in a ring of their own.
-template <int G>
+template <int G, bool F8>
 struct TCfg {
     static constexpr int NG = kHeadDim / G;
+    static constexpr int kMetaBytes = F8 ? 2 : 4;                        // {scale, zero} per (token, group): E4M3 bytes or a half2
     static constexpr int kCodeTile = kTile * kRowBytes;                  // 4096
-    static constexpr int kMetaTile = kTile * NG * 4;
+    static constexpr int kMetaTile = kTile * NG * kMetaBytes;
     static constexpr int kVmBytes = kCodeTile + 2 * kMetaTile;           // V codes, K scale/zero, V scale/zero
     static constexpr int kOffVm = kRing * kCodeTile;
     static constexpr int kOffKA = kOffVm + kRing * kVmBytes;             // A of the score MMA: [128 tokens][128 bytes]
@@ -107,7 +108,7 @@ __device__ __forceinline__ float lo_half(uint32_t w) { return __low2float(*reint
 __device__ __forceinline__ float hi_half(uint32_t w) { return __high2float(*reinterpret_cast<const __half2 *>(&w)); }
 
 template <int NG>
-__device__ __forceinline__ void load_words(const uint32_t *p, uint32_t (&w)[NG])
+__device__ __forceinline__ void load_words32(const uint32_t *p, uint32_t (&w)[NG])
 {
     if constexpr (NG == 4) {
         const uint4 x = *reinterpret_cast<const uint4 *>(p);
@@ -117,6 +118,28 @@ __device__ __forceinline__ void load_words(const uint32_t *p, uint32_t (&w)[NG])
         w[0] = x.x; w[1] = x.y;
     } else {
         w[0] = p[0];
+    }
+}
+
+// The {h, z} words of one token as fp16 pairs, from fp16 pairs or from E4M3 byte pairs.
+template <int NG, bool F8>
+__device__ __forceinline__ void load_words(const uint8_t *p, uint32_t (&w)[NG])
+{
+    if constexpr (F8) {
+        uint16_t b[NG];
+        if constexpr (NG == 4) {
+            const uint2 x = *reinterpret_cast<const uint2 *>(p);
+            b[0] = (uint16_t)x.x; b[1] = (uint16_t)(x.x >> 16); b[2] = (uint16_t)x.y; b[3] = (uint16_t)(x.y >> 16);
+        } else if constexpr (NG == 2) {
+            const uint32_t x = *reinterpret_cast<const uint32_t *>(p);
+            b[0] = (uint16_t)x; b[1] = (uint16_t)(x >> 16);
+        } else {
+            b[0] = *reinterpret_cast<const uint16_t *>(p);
+        }
+#pragma unroll
+        for (int i = 0; i < NG; ++i) asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(w[i]) : "h"(b[i]));
+    } else {
+        load_words32<NG>(reinterpret_cast<const uint32_t *>(p), w);
     }
 }
 
@@ -151,10 +174,10 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
-template <int G>
+template <int G, bool F8>
 __global__ void __launch_bounds__(kTile + 32, kCtasPerSm) partition_tc_kernel(MmaArgs a)
 {
-    using C = TCfg<G>;
+    using C = TCfg<G, F8>;
     constexpr int NG = C::NG;
     extern __shared__ __align__(128) uint8_t smem[];
     const Shape &s = a.s;
@@ -249,15 +272,16 @@ __global__ void __launch_bounds__(kTile + 32, kCtasPerSm) partition_tc_kernel(Mm
     };
     auto issue_v = [&](int i) {       // control lane only
         const uint8_t *v_codes = a.c.v_codes + bh * (size_t)s.cap * kRowBytes;
-        const __half2 *k_meta = a.c.k_meta + bh * (size_t)s.cap * NG;
-        const __half2 *v_meta = a.c.v_meta + bh * (size_t)s.cap * NG;
+        constexpr uint32_t kRowMeta = NG * C::kMetaBytes;
+        const uint8_t *k_meta = reinterpret_cast<const uint8_t *>(a.c.k_meta) + bh * (size_t)s.cap * kRowMeta;
+        const uint8_t *v_meta = reinterpret_cast<const uint8_t *>(a.c.v_meta) + bh * (size_t)s.cap * kRowMeta;
         const uint32_t slot = (tiles_done + i) % kRing, rows = rows_of(i);
         const int tok0 = q_begin + i * kTile;
         const uint32_t dst = smem_u32(smem + C::kOffVm + slot * C::kVmBytes), bar = bar_v + 8 * slot;
-        mbar_expect_tx(bar, rows * (kRowBytes + 2 * NG * 4));
+        mbar_expect_tx(bar, rows * (kRowBytes + 2 * kRowMeta));
         bulk_g2s(dst, v_codes + (size_t)tok0 * kRowBytes, rows * kRowBytes, bar);
-        bulk_g2s(dst + C::kCodeTile, k_meta + (size_t)tok0 * NG, rows * NG * 4, bar);
-        bulk_g2s(dst + C::kCodeTile + C::kMetaTile, v_meta + (size_t)tok0 * NG, rows * NG * 4, bar);
+        bulk_g2s(dst + C::kCodeTile, k_meta + (size_t)tok0 * kRowMeta, rows * kRowMeta, bar);
+        bulk_g2s(dst + C::kCodeTile + C::kMetaTile, v_meta + (size_t)tok0 * kRowMeta, rows * kRowMeta, bar);
     };
     auto wait_ring = [&](uint32_t bar0, int i) {
         const uint32_t t = tiles_done + i;
@@ -419,8 +443,8 @@ __global__ void __launch_bounds__(kTile + 32, kCtasPerSm) partition_tc_kernel(Mm
         for (int i = 0; i < n_tiles; ++i) {
             const uint32_t n = s_count + i;
             const uint8_t *vm = smem + C::kOffVm + ((tiles_done + i) % kRing) * C::kVmBytes;
-            const uint32_t *Km = reinterpret_cast<const uint32_t *>(vm + C::kCodeTile);                      // [128][NG] words {h, z}
-            const uint32_t *Vm = reinterpret_cast<const uint32_t *>(vm + C::kCodeTile + C::kMetaTile);
+            const uint8_t *Km = vm + C::kCodeTile;                      // [128][NG] {h, z}
+            const uint8_t *Vm = vm + C::kCodeTile + C::kMetaTile;
             uint8_t *PA = smem + C::kOffPA;
             const int tok = q_begin + i * kTile + tid;
             const bool valid = tok < q_end && tok >= s.n_sink;      // sinks belong to the merge kernel
@@ -436,8 +460,8 @@ __global__ void __launch_bounds__(kTile + 32, kCtasPerSm) partition_tc_kernel(Mm
             for (int gg = 0; gg < H0; ++gg) tmem_ld16(tmem_row + kScoreCol + 16 * gg, va[gg]);
             wait_ring(bar_v, i);
             uint32_t kw[NG], vw[NG];
-            load_words<NG>(Km + tid * NG, kw);
-            load_words<NG>(Vm + tid * NG, vw);
+            load_words<NG, F8>(Km + tid * NG * C::kMetaBytes, kw);
+            load_words<NG, F8>(Vm + tid * NG * C::kMetaBytes, vw);
             tmem_wait_ld();
             int vb[NG - H0 > 0 ? NG - H0 : 1][16];
 #pragma unroll
@@ -596,12 +620,12 @@ __global__ void __launch_bounds__(kTile + 32, kCtasPerSm) partition_tc_kernel(Mm
     if (control) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
 }
 
-template <int G>
+template <int G, bool F8>
 cudaError_t launch_g(const MmaArgs &a, cudaStream_t stream, bool overlap)
 {
-    using C = TCfg<G>;
+    using C = TCfg<G, F8>;
     static bool configured = false;
-    auto kern = partition_tc_kernel<G>;
+    auto kern = partition_tc_kernel<G, F8>;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
         if (e != cudaSuccess) return e;
@@ -625,7 +649,9 @@ cudaError_t launch_partition_tc(const Shape &s, const CachePtrs &c, const __half
         a.head0 = head0;
         // a second launch reads the same cache again for the next four heads; it starts when the first has finished
         const bool ov = overlap && head0 == 0;
-        const cudaError_t e = s.G == 128 ? launch_g<128>(a, stream, ov) : s.G == 64 ? launch_g<64>(a, stream, ov) : launch_g<32>(a, stream, ov);
+        cudaError_t e;
+        if (s.meta_fp8) e = s.G == 128 ? launch_g<128, true>(a, stream, ov) : s.G == 64 ? launch_g<64, true>(a, stream, ov) : launch_g<32, true>(a, stream, ov);
+        else e = s.G == 128 ? launch_g<128, false>(a, stream, ov) : s.G == 64 ? launch_g<64, false>(a, stream, ov) : launch_g<32, false>(a, stream, ov);
         if (e != cudaSuccess) return e;
         if (head0 > 0) count_launch(1);
     }

@@ -19,6 +19,7 @@ struct Shape {
     int k_bits, v_bits, G, ng;
     int W, cap, max_tokens;
     int n_sink;            // positions below this are kept fp16 in the sink store when they leave the window
+    int meta_fp8;          // scale/zero stored as two E4M3 bytes per (token, group) instead of a half2
 };
 
 struct CachePtrs {

@@ -46,6 +46,7 @@ class Workload:
     ragged: tuple | None = None  # (lo, hi) inclusive per-sequence length range
     calib_tokens: int = 512
     n_sink: int = 0              # first positions kept fp16 for good (attention sinks; the paper's experiments use 5)
+    meta_fp8: bool = False       # scale and zero point stored in FP8 E4M3 instead of fp16
 
     @property
     def sm_scale(self) -> float:
@@ -154,7 +155,8 @@ def algorithmic_bytes(w: Workload, lengths=None) -> int:
     prefix, the fp16 window and sinks, and q/out.  Split scratch is not counted."""
     lengths = w.lengths() if lengths is None else np.asarray(lengths)
     D, ng = w.head_dim, w.head_dim // w.group_size
-    per_tok = (D * w.k_bits // 8 + 4 * ng) + (D * w.v_bits // 8 + 4 * ng)
+    mb = 2 if w.meta_fp8 else 4      # bytes of {scale, zero} per (token, group)
+    per_tok = (D * w.k_bits // 8 + mb * ng) + (D * w.v_bits // 8 + mb * ng)
     total = 0
     for L in lengths.tolist():
         lq = max(L - w.window, 0)
@@ -169,6 +171,7 @@ def partition_kernel_bytes(w: Workload, lengths=None) -> int:
     scale/zero of the quantized prefix plus q (the fp16 window and the output belong to the merge kernel)."""
     lengths = w.lengths() if lengths is None else np.asarray(lengths)
     D, ng = w.head_dim, w.head_dim // w.group_size
-    per_tok = (D * w.k_bits // 8 + 4 * ng) + (D * w.v_bits // 8 + 4 * ng)
+    mb = 2 if w.meta_fp8 else 4      # bytes of {scale, zero} per (token, group)
+    per_tok = (D * w.k_bits // 8 + mb * ng) + (D * w.v_bits // 8 + mb * ng)
     total = sum(w.n_kv_heads * max(L - w.window - w.n_sink, 0) * per_tok for L in lengths.tolist())
     return int(total + w.batch * w.n_q_heads * D * 2)

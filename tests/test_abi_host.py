@@ -52,7 +52,7 @@ def test_version_and_strerror(lib):
     (dict(v_bits=8), B.SKVQ_ERR_UNSUPPORTED), (dict(group_size=16), B.SKVQ_ERR_UNSUPPORTED),
     (dict(n_q_heads=7), B.SKVQ_ERR_UNSUPPORTED), (dict(n_q_heads=32, n_kv_heads=2), B.SKVQ_ERR_UNSUPPORTED),
     (dict(batch=0), B.SKVQ_ERR_INVALID_ARG), (dict(window=-1), B.SKVQ_ERR_INVALID_ARG),
-    (dict(max_tokens=0), B.SKVQ_ERR_INVALID_ARG), (dict(), B.SKVQ_OK), (dict(n_sink=5), B.SKVQ_OK),
+    (dict(max_tokens=0), B.SKVQ_ERR_INVALID_ARG), (dict(), B.SKVQ_OK), (dict(n_sink=5), B.SKVQ_OK), (dict(meta_fp8=1), B.SKVQ_OK), (dict(meta_fp8=2), B.SKVQ_ERR_INVALID_ARG),
     (dict(n_sink=-1), B.SKVQ_ERR_INVALID_ARG), (dict(n_sink=65), B.SKVQ_ERR_UNSUPPORTED), (dict(window=0, k_bits=4, group_size=32), B.SKVQ_OK),
 ])
 def test_config_validation(lib, kw, code):

@@ -170,6 +170,35 @@ def test_sinks_stay_fp16_and_attention_matches_oracle(cfg_i, kw, n):
     assert np.abs(got - want).max() <= ATTN_TOL
 
 
+# ------------------------------------------------------------------ FP8 E4M3 scale and zero point (Sec. 4.1)
+@pytest.mark.parametrize("cfg_i,kw,n", [
+    (2, dict(context=3000, batch=2, meta_fp8=True), 3000),                                     # 2-bit g32, 4 heads per KV head: 2.5 bits
+    (1, dict(context=2500, batch=2, n_q_heads=4, n_kv_heads=4, meta_fp8=True), 2500),          # one head per KV head, g128
+    (1, dict(context=2100, batch=1, n_q_heads=16, n_kv_heads=2, group_size=64, meta_fp8=True, n_sink=5), 2100),   # 8 heads, g64, sinks
+    (4, dict(context=1300, batch=2, ragged=None, n_q_heads=4, n_kv_heads=4, meta_fp8=True), 1300),   # 4-bit g64: scalar kernel
+    (0, dict(context=200, meta_fp8=True), 200),
+])
+def test_fp8_parameters_bit_exact_cache_and_attention(cfg_i, kw, n):
+    w = small(cfg_i, **kw)
+    gpu, ora = both_caches(w, n + 64)
+    assert gpu.k_meta.dtype == torch.uint8 and gpu.k_meta.shape[-2:] == (128 // w.group_size, 2)      # two bytes per (token, group)
+    k, v = w.prefill("k", n), w.prefill("v", n)
+    cut = (n * 2) // 3
+    gpu.append(dev(k[:, :cut]), dev(v[:, :cut]))                      # bulk tiles, ragged ends, evictions from the ring
+    gpu.append(dev(k[:, cut:]), dev(v[:, cut:]))
+    ora.append(k, v)
+    assert_cache_bit_exact(gpu, ora)
+    got, want = attention_both(gpu, ora, w)
+    assert np.abs(got - want).max() <= ATTN_TOL
+    for s in range(5):                                                # decode steps: single-token appends
+        kn, vn = w.new_token("k", s), w.new_token("v", s)
+        gpu.append(dev(kn), dev(vn))
+        ora.append(kn, vn)
+    assert_cache_bit_exact(gpu, ora)
+    got, want = attention_both(gpu, ora, w, step=1)
+    assert np.abs(got - want).max() <= ATTN_TOL
+
+
 def test_attention_ragged_batch_with_empty_sequence():
     w = small(4, context=2000, batch=6, ragged=None)
     gpu, ora = both_caches(w, 2048)
