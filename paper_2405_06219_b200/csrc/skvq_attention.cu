@@ -417,8 +417,6 @@ __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
 // Resident CTAs per SM of the partition kernel that serves this shape (sets how many CTAs make one wave).
 static int partition_ctas_per_sm(const Shape &s)
 {
-    if (s.meta_fp8)      // FP8 parameters: the tcgen05 kernel where it applies, else the scalar kernel
-        return (s.k_bits == 2 && s.v_bits == 2 && s.rep <= 8 && (s.G == 128 || s.G == 64 || s.G == 32)) ? 3 : 8;
     if (s.rep == 1 && s.G >= 64) return s.k_bits == s.v_bits ? 4 : 3;           // integer kernel
     if (s.k_bits == 2 && s.v_bits == 2 && (s.rep == 3 || (s.rep > 4 && s.rep <= 8)) && (s.G == 128 || s.G == 64 || s.G == 32))
         return 3;                                                              // tcgen05 kernel: 128 tensor-memory columns, 69 KB

@@ -33,11 +33,12 @@ constexpr int kHeadSlots = 4;           // query heads per KV head this kernel s
 constexpr int kRefSlackLog2 = 12;       // the softmax reference moves only when a score exceeds it by this (log2)
 constexpr float kRefSlack = (float)kRefSlackLog2;
 
-template <int G>
+template <int G, bool F8>
 struct GCfg {
     static constexpr int NG = kHeadDim / G;
     static constexpr int kCodeTile = kTileTok * kRowBytes;               // 2048 B
-    static constexpr int kMetaTile = kTileTok * NG * 4;
+    static constexpr int kMetaBytes = F8 ? 2 : 4;                        // {scale, zero} per (token, group): two E4M3 bytes or a half2
+    static constexpr int kMetaTile = kTileTok * NG * kMetaBytes;
     static constexpr int kStageBytes = 2 * kCodeTile + 2 * kMetaTile;
     static constexpr int kStages = 2;
     static constexpr int kXBytes = NG * 2 * 32 * 8;                      // digit registers on their way to the A fragments
@@ -114,6 +115,42 @@ __device__ __forceinline__ void load_words(const uint32_t *p, uint32_t (&w)[NG])
     }
 }
 
+// One E4M3 byte pair {h, z} -> the same pair as fp16 (every E4M3 value is an fp16 value).
+__device__ __forceinline__ uint32_t e4m3x2_to_half2(uint16_t b)
+{
+    uint32_t r;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(r) : "h"(b));
+    return r;
+}
+// The NG {h, z} words of token tok of a scale/zero tile, as fp16 pairs.
+template <int NG, bool F8>
+__device__ __forceinline__ void load_meta(const uint8_t *tile, int tok, uint32_t (&w)[NG])
+{
+    if constexpr (F8) {
+        uint16_t b[NG];
+        if constexpr (NG == 4) {
+            const uint2 x = *reinterpret_cast<const uint2 *>(tile + tok * 8);
+            b[0] = (uint16_t)x.x; b[1] = (uint16_t)(x.x >> 16); b[2] = (uint16_t)x.y; b[3] = (uint16_t)(x.y >> 16);
+        } else if constexpr (NG == 2) {
+            const uint32_t x = *reinterpret_cast<const uint32_t *>(tile + tok * 4);
+            b[0] = (uint16_t)x; b[1] = (uint16_t)(x >> 16);
+        } else {
+            b[0] = *reinterpret_cast<const uint16_t *>(tile + tok * 2);
+        }
+#pragma unroll
+        for (int i = 0; i < NG; ++i) w[i] = e4m3x2_to_half2(b[i]);
+    } else {
+        load_words<NG>(reinterpret_cast<const uint32_t *>(tile) + tok * NG, w);
+    }
+}
+// Word g (not a compile-time index) of the same.
+template <int NG, bool F8>
+__device__ __forceinline__ uint32_t load_meta_word(const uint8_t *tile, int tok, int g)
+{
+    if constexpr (F8) return e4m3x2_to_half2(reinterpret_cast<const uint16_t *>(tile)[tok * NG + g]);
+    else return reinterpret_cast<const uint32_t *>(tile)[tok * NG + g];
+}
+
 __device__ __forceinline__ float lo_half(uint32_t w) { return __low2float(*reinterpret_cast<const __half2 *>(&w)); }
 __device__ __forceinline__ float hi_half(uint32_t w) { return __high2float(*reinterpret_cast<const __half2 *>(&w)); }
 
@@ -127,10 +164,10 @@ __device__ __forceinline__ int owned_token(int kk, int q, int gg) { return 32 * 
 #ifndef SKVQ_GQA_CTAS
 #define SKVQ_GQA_CTAS 2
 #endif
-template <int G, int R>
+template <int G, int R, bool F8>
 __global__ void __launch_bounds__(kThreads, SKVQ_GQA_CTAS) partition_gqa_kernel(MmaArgs a)
 {
-    using C = GCfg<G>;
+    using C = GCfg<G, F8>;
     constexpr int NG = C::NG;
     static_assert(R <= kHeadSlots, "rows of the P.V MMAs are 4 heads x 4 digits");
     extern __shared__ __align__(128) uint8_t smem[];
@@ -179,8 +216,8 @@ __global__ void __launch_bounds__(kThreads, SKVQ_GQA_CTAS) partition_gqa_kernel(
     const size_t bh = (size_t)b * s.Hkv + hk;
     const uint8_t *k_codes = a.c.k_codes + bh * (size_t)s.cap * kRowBytes;
     const uint8_t *v_codes = a.c.v_codes + bh * (size_t)s.cap * kRowBytes;
-    const __half2 *k_meta = a.c.k_meta + bh * (size_t)s.cap * NG;
-    const __half2 *v_meta = a.c.v_meta + bh * (size_t)s.cap * NG;
+    const uint8_t *k_meta = reinterpret_cast<const uint8_t *>(a.c.k_meta) + bh * (size_t)s.cap * NG * C::kMetaBytes;
+    const uint8_t *v_meta = reinterpret_cast<const uint8_t *>(a.c.v_meta) + bh * (size_t)s.cap * NG * C::kMetaBytes;
 
     const int n_tiles = (q_end - q_begin + kTileTok - 1) / kTileTok;
     const int n_my = (n_tiles > warp && !failed) ? (n_tiles - warp + kWarps - 1) / kWarps : 0;
@@ -193,8 +230,8 @@ __global__ void __launch_bounds__(kThreads, SKVQ_GQA_CTAS) partition_gqa_kernel(
         mbar_expect_tx(bar, C::kStageBytes);
         bulk_g2s(dst, k_codes + (size_t)tok0 * kRowBytes, C::kCodeTile, bar);
         bulk_g2s(dst + C::kCodeTile, v_codes + (size_t)tok0 * kRowBytes, C::kCodeTile, bar);
-        bulk_g2s(dst + 2 * C::kCodeTile, k_meta + (size_t)tok0 * NG, C::kMetaTile, bar);
-        bulk_g2s(dst + 2 * C::kCodeTile + C::kMetaTile, v_meta + (size_t)tok0 * NG, C::kMetaTile, bar);
+        bulk_g2s(dst + 2 * C::kCodeTile, k_meta + (size_t)tok0 * NG * C::kMetaBytes, C::kMetaTile, bar);
+        bulk_g2s(dst + 2 * C::kCodeTile + C::kMetaTile, v_meta + (size_t)tok0 * NG * C::kMetaBytes, C::kMetaTile, bar);
     };
     if (lane == 0) {      // the first copies are in flight while the query is prepared
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the stages held the previous segment's result
@@ -347,8 +384,8 @@ __global__ void __launch_bounds__(kThreads, SKVQ_GQA_CTAS) partition_gqa_kernel(
         if (!mbar_wait_bounded(bar0 + 8 * st, parity)) { failed = true; break; }
         uint8_t *Kc = stage_base + st * C::kStageBytes;
         uint8_t *Vc = Kc + C::kCodeTile;
-        uint32_t *Km = reinterpret_cast<uint32_t *>(Kc + 2 * C::kCodeTile);       // [64][NG] words {h, z}
-        uint32_t *Vm = reinterpret_cast<uint32_t *>(Kc + 2 * C::kCodeTile + C::kMetaTile);
+        uint8_t *Km = Kc + 2 * C::kCodeTile;                        // [64][NG] {h, z}
+        uint8_t *Vm = Kc + 2 * C::kCodeTile + C::kMetaTile;
         const int tok0 = q_begin + (warp + i * kWarps) * kTileTok;
         const int n_valid = min(kTileTok, q_end - tok0);
         const int n_skip = max(s.n_sink - tok0, 0);      // rows of attention sinks: the merge kernel reads their fp16 copies
@@ -359,7 +396,15 @@ __global__ void __launch_bounds__(kThreads, SKVQ_GQA_CTAS) partition_gqa_kernel(
                 const int tau = lane + 32 * hf;
                 if (tau >= n_valid || tau < n_skip) {
 #pragma unroll
-                    for (int gg = 0; gg < NG; ++gg) { Km[tau * NG + gg] = 0u; Vm[tau * NG + gg] = 0u; }
+                    for (int gg = 0; gg < NG; ++gg) {
+                        if constexpr (F8) {
+                            reinterpret_cast<uint16_t *>(Km)[tau * NG + gg] = 0;
+                            reinterpret_cast<uint16_t *>(Vm)[tau * NG + gg] = 0;
+                        } else {
+                            reinterpret_cast<uint32_t *>(Km)[tau * NG + gg] = 0u;
+                            reinterpret_cast<uint32_t *>(Vm)[tau * NG + gg] = 0u;
+                        }
+                    }
                 }
             }
             __syncwarp();
@@ -385,12 +430,12 @@ __global__ void __launch_bounds__(kThreads, SKVQ_GQA_CTAS) partition_gqa_kernel(
                     mma16816(ak[hf], u0[2 * sx], u1[2 * sx], u0[2 * sx + 1], u1[2 * sx + 1], bK[hf][sx][0], bK[hf][sx][1]);
             }
             // {h, z} words of the two tokens: A operand of the constant/zero-point MMA, and h for the group sums
-            const uint32_t *m0 = Km + (32 * kk + own[2 * jj]) * NG, *m1 = Km + (32 * kk + own[2 * jj + 1]) * NG;
+            const int tk0 = 32 * kk + own[2 * jj], tk1 = 32 * kk + own[2 * jj + 1];
             uint32_t mw0[NG], mw1[NG];
-            load_words<NG>(m0, mw0);
-            load_words<NG>(m1, mw1);
-            const uint32_t za = t < NG ? m0[t < NG ? t : 0] : 0u;
-            const uint32_t zb = t < NG ? m1[t < NG ? t : 0] : 0u;
+            load_meta<NG, F8>(Km, tk0, mw0);
+            load_meta<NG, F8>(Km, tk1, mw1);
+            const uint32_t za = t < NG ? load_meta_word<NG, F8>(Km, tk0, t < NG ? t : 0) : 0u;
+            const uint32_t zb = t < NG ? load_meta_word<NG, F8>(Km, tk1, t < NG ? t : 0) : 0u;
             float az[4] = {0.f, 0.f, 0.f, 0.f};
             mma16816(az, za, zb, za, zb, bZ[0], bZ[1]);
             float s0 = az[0], s1 = az[2];
@@ -410,8 +455,8 @@ __global__ void __launch_bounds__(kThreads, SKVQ_GQA_CTAS) partition_gqa_kernel(
         uint32_t hmax_bits;
         {
             uint32_t wa[NG], wb[NG];
-            load_words<NG>(Vm + lane * NG, wa);
-            load_words<NG>(Vm + (lane + 32) * NG, wb);
+            load_meta<NG, F8>(Vm, lane, wa);
+            load_meta<NG, F8>(Vm, lane + 32, wb);
             uint32_t mx = __vmaxu2(wa[0], wb[0]);
 #pragma unroll
             for (int gg = 1; gg < NG; ++gg) mx = __vmaxu2(mx, __vmaxu2(wa[gg], wb[gg]));
@@ -478,7 +523,7 @@ __global__ void __launch_bounds__(kThreads, SKVQ_GQA_CTAS) partition_gqa_kernel(
                 const float p = ex2_approx(arg[2 * kk + (q >> 1)][q & 1]);      // at most 2^slack; 0 past the end
                 l_sum += p;
                 uint32_t vw[NG];
-                load_words<NG>(Vm + (32 * kk + own[q]) * NG, vw);
+                load_meta<NG, F8>(Vm, 32 * kk + own[q], vw);
                 const float ps = p * hscale;
 #pragma unroll
                 for (int gg = 0; gg < NG; ++gg) {
@@ -595,12 +640,12 @@ __global__ void __launch_bounds__(kThreads, SKVQ_GQA_CTAS) partition_gqa_kernel(
     }
 }
 
-template <int G, int R>
+template <int G, int R, bool F8>
 cudaError_t launch_one(const MmaArgs &a, cudaStream_t stream, bool overlap)
 {
-    using C = GCfg<G>;
+    using C = GCfg<G, F8>;
     static bool configured = false;
-    auto kern = partition_gqa_kernel<G, R>;
+    auto kern = partition_gqa_kernel<G, R, F8>;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
         if (e != cudaSuccess) return e;
@@ -609,14 +654,14 @@ cudaError_t launch_one(const MmaArgs &a, cudaStream_t stream, bool overlap)
     return launch_dependent(kern, dim3(a.plan.n_slots), dim3(kThreads), C::kSmemBytes, stream, overlap, a);
 }
 
-template <int G>
+template <int G, bool F8>
 cudaError_t launch_g(const MmaArgs &a, cudaStream_t stream, bool overlap, bool *handled)
 {
     *handled = true;
     switch (a.s.rep) {
-        case 1: return launch_one<G, 1>(a, stream, overlap);
-        case 2: return launch_one<G, 2>(a, stream, overlap);
-        case 4: return launch_one<G, 4>(a, stream, overlap);
+        case 1: return launch_one<G, 1, F8>(a, stream, overlap);
+        case 2: return launch_one<G, 2, F8>(a, stream, overlap);
+        case 4: return launch_one<G, 4, F8>(a, stream, overlap);
         default: *handled = false; return cudaSuccess;
     }
 }
@@ -629,12 +674,20 @@ cudaError_t launch_partition_gqa(const Shape &s, const CachePtrs &c, const __hal
                                  const SplitPlan &plan, float *workspace, cudaStream_t stream, bool overlap, bool *handled)
 {
     *handled = false;
-    if (s.k_bits != 2 || s.v_bits != 2 || s.meta_fp8) return cudaSuccess;      // this kernel reads fp16 scale/zero pairs
+    if (s.k_bits != 2 || s.v_bits != 2) return cudaSuccess;
     MmaArgs a{s, c, q, scale_log2, plan, workspace};
+    if (s.meta_fp8) {
+        switch (s.G) {
+            case 128: return launch_g<128, true>(a, stream, overlap, handled);
+            case 64: return launch_g<64, true>(a, stream, overlap, handled);
+            case 32: return launch_g<32, true>(a, stream, overlap, handled);
+            default: return cudaSuccess;
+        }
+    }
     switch (s.G) {
-        case 128: return launch_g<128>(a, stream, overlap, handled);
-        case 64: return launch_g<64>(a, stream, overlap, handled);
-        case 32: return launch_g<32>(a, stream, overlap, handled);
+        case 128: return launch_g<128, false>(a, stream, overlap, handled);
+        case 64: return launch_g<64, false>(a, stream, overlap, handled);
+        case 32: return launch_g<32, false>(a, stream, overlap, handled);
         default: return cudaSuccess;
     }
 }

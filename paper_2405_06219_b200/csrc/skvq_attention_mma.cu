@@ -29,7 +29,7 @@ namespace {
 using namespace mmak;
 
 // ---------------------------------------------------------------- compile-time layout
-template <int G, int KB, int VB>
+template <int G, int KB, int VB, bool F8>
 struct Cfg {
     static constexpr int NG = kHeadDim / G;
     static_assert(NG <= 2, "(group, byte digit) has to fit the 8 MMA columns");
@@ -37,7 +37,8 @@ struct Cfg {
     static constexpr int KROW = kHeadDim * KB / 8, VROW = kHeadDim * VB / 8;   // bytes per token row
     static constexpr int VCPB = 8 / VB;                                   // codes per byte = masks per register
     static constexpr int kKTile = T * KROW, kVTile = T * VROW;
-    static constexpr int kMetaTile = T * NG * 4;
+    static constexpr int kMetaBytes = F8 ? 2 : 4;      // {scale, zero} per (token, group): two E4M3 bytes or a half2
+    static constexpr int kMetaTile = T * NG * kMetaBytes;
     static constexpr int kStageBytes = kKTile + kVTile + 2 * kMetaTile;
     static constexpr int kStages = 2;
     static constexpr int kScBytes = T * NG * 8;                           // per (token, group): low and high digit pairs
@@ -50,10 +51,10 @@ struct Cfg {
     static_assert(kKTile % 16 == 0 && kVTile % 16 == 0 && kMetaTile % 16 == 0, "bulk copies move multiples of 16 bytes");
 };
 
-template <int G, int KB, int VB>
-__global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB>::kCtasPerSm) partition_mma_kernel(MmaArgs a)
+template <int G, int KB, int VB, bool F8>
+__global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB, F8>::kCtasPerSm) partition_mma_kernel(MmaArgs a)
 {
-    using C = Cfg<G, KB, VB>;
+    using C = Cfg<G, KB, VB, F8>;
     constexpr int NG = C::NG, KROW = C::KROW, VROW = C::VROW, T = C::T;
     extern __shared__ __align__(128) uint8_t smem[];
     const Shape &s = a.s;
@@ -101,8 +102,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB>::kCtasPerSm) partitio
     const size_t bh = (size_t)b * s.Hkv + hk;
     const uint8_t *k_codes = a.c.k_codes + bh * (size_t)s.cap * KROW;
     const uint8_t *v_codes = a.c.v_codes + bh * (size_t)s.cap * VROW;
-    const __half2 *k_meta = a.c.k_meta + bh * (size_t)s.cap * NG;
-    const __half2 *v_meta = a.c.v_meta + bh * (size_t)s.cap * NG;
+    const uint8_t *k_meta = reinterpret_cast<const uint8_t *>(a.c.k_meta) + bh * (size_t)s.cap * NG * C::kMetaBytes;
+    const uint8_t *v_meta = reinterpret_cast<const uint8_t *>(a.c.v_meta) + bh * (size_t)s.cap * NG * C::kMetaBytes;
 
     const int n_tiles = (q_end - q_begin + T - 1) / T;                          // tiles of this split
     const int n_my = (n_tiles > warp && !failed) ? (n_tiles - warp + kWarps - 1) / kWarps : 0;   // tiles warp, warp+4, ...
@@ -115,8 +116,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB>::kCtasPerSm) partitio
         mbar_expect_tx(bar, C::kStageBytes);
         bulk_g2s(dst, k_codes + (size_t)tok0 * KROW, C::kKTile, bar);
         bulk_g2s(dst + C::kKTile, v_codes + (size_t)tok0 * VROW, C::kVTile, bar);
-        bulk_g2s(dst + C::kKTile + C::kVTile, k_meta + (size_t)tok0 * NG, C::kMetaTile, bar);
-        bulk_g2s(dst + C::kKTile + C::kVTile + C::kMetaTile, v_meta + (size_t)tok0 * NG, C::kMetaTile, bar);
+        bulk_g2s(dst + C::kKTile + C::kVTile, k_meta + (size_t)tok0 * NG * C::kMetaBytes, C::kMetaTile, bar);
+        bulk_g2s(dst + C::kKTile + C::kVTile + C::kMetaTile, v_meta + (size_t)tok0 * NG * C::kMetaBytes, C::kMetaTile, bar);
     };
     if (lane == 0) {      // the first copies are in flight while the query is prepared
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the stages held the previous segment's result
@@ -226,8 +227,18 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB>::kCtasPerSm) partitio
         if (!mbar_wait_bounded(bar0 + 8 * st, parity)) { failed = true; break; }
         const uint8_t *Kc = stage_base + st * C::kStageBytes;
         const uint8_t *Vc = Kc + C::kKTile;
-        const __half2 *Km = reinterpret_cast<const __half2 *>(Kc + C::kKTile + C::kVTile);
-        const __half2 *Vm = reinterpret_cast<const __half2 *>(Kc + C::kKTile + C::kVTile + C::kMetaTile);
+        const uint8_t *Km = Kc + C::kKTile + C::kVTile;                      // [T][NG] {h, z}
+        const uint8_t *Vm = Kc + C::kKTile + C::kVTile + C::kMetaTile;
+        // {h, z} of (token, group) as floats: a half2, or two E4M3 bytes (every E4M3 value is an fp16 value)
+        auto load_hz = [&](const uint8_t *base, int idx) -> float2 {
+            if constexpr (F8) {
+                uint32_t r;
+                asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(r) : "h"(reinterpret_cast<const uint16_t *>(base)[idx]));
+                return __half22float2(*reinterpret_cast<const __half2 *>(&r));
+            } else {
+                return __half22float2(reinterpret_cast<const __half2 *>(base)[idx]);
+            }
+        };
         const int tok0 = q_begin + (warp + i * kWarps) * T;
 
         // ---------------- scores: exact integer dot products sum_j q'_j c_j per (token, group)
@@ -287,8 +298,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB>::kCtasPerSm) partitio
             float sv = 0.f;
 #pragma unroll
             for (int gg = 0; gg < NG; ++gg) {
-                const float2 kz = __half22float2(Km[tau * NG + gg]);
-                const float2 vz = __half22float2(Vm[tau * NG + gg]);
+                const float2 kz = load_hz(Km, tau * NG + gg);
+                const float2 vz = load_hz(Vm, tau * NG + gg);
                 hv[hf][gg] = valid ? vz.x : 0.f;      // rows past the end hold unspecified bytes
                 zv[hf][gg] = valid ? vz.y : 0.f;
                 moved |= (hv[hf][gg] >= h_bound);
@@ -460,12 +471,12 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB>::kCtasPerSm) partitio
     }
 }
 
-template <int G, int KB, int VB>
+template <int G, int KB, int VB, bool F8>
 cudaError_t launch_one(const MmaArgs &a, cudaStream_t stream, bool overlap)
 {
-    using C = Cfg<G, KB, VB>;
+    using C = Cfg<G, KB, VB, F8>;
     static bool configured = false;
-    auto kern = partition_mma_kernel<G, KB, VB>;
+    auto kern = partition_mma_kernel<G, KB, VB, F8>;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
         if (e != cudaSuccess) return e;
@@ -474,11 +485,12 @@ cudaError_t launch_one(const MmaArgs &a, cudaStream_t stream, bool overlap)
     return launch_dependent(kern, dim3(a.plan.n_slots), dim3(kThreads), C::kSmemBytes, stream, overlap, a);
 }
 
-template <int G>
+template <int G, bool F8>
 cudaError_t launch_g(const MmaArgs &a, cudaStream_t stream, bool overlap)
 {
-    if (a.s.k_bits == 2) return a.s.v_bits == 2 ? launch_one<G, 2, 2>(a, stream, overlap) : launch_one<G, 2, 4>(a, stream, overlap);
-    return a.s.v_bits == 2 ? launch_one<G, 4, 2>(a, stream, overlap) : launch_one<G, 4, 4>(a, stream, overlap);
+    if (a.s.k_bits == 2)
+        return a.s.v_bits == 2 ? launch_one<G, 2, 2, F8>(a, stream, overlap) : launch_one<G, 2, 4, F8>(a, stream, overlap);
+    return a.s.v_bits == 2 ? launch_one<G, 4, 2, F8>(a, stream, overlap) : launch_one<G, 4, 4, F8>(a, stream, overlap);
 }
 
 }  // namespace
@@ -489,11 +501,11 @@ cudaError_t launch_partition_mma(const Shape &s, const CachePtrs &c, const __hal
                                  const SplitPlan &plan, float *workspace, cudaStream_t stream, bool overlap, bool *handled)
 {
     *handled = false;
-    if (s.meta_fp8) return cudaSuccess;      // this kernel reads fp16 scale/zero pairs
     if (s.rep != 1 || (s.G != 64 && s.G != 128)) return cudaSuccess;
     MmaArgs a{s, c, q, scale_log2, plan, workspace};
     *handled = true;
-    return s.G == 128 ? launch_g<128>(a, stream, overlap) : launch_g<64>(a, stream, overlap);
+    if (s.meta_fp8) return s.G == 128 ? launch_g<128, true>(a, stream, overlap) : launch_g<64, true>(a, stream, overlap);
+    return s.G == 128 ? launch_g<128, false>(a, stream, overlap) : launch_g<64, false>(a, stream, overlap);
 }
 
 }  // namespace skvq

@@ -175,7 +175,10 @@ def test_sinks_stay_fp16_and_attention_matches_oracle(cfg_i, kw, n):
     (2, dict(context=3000, batch=2, meta_fp8=True), 3000),                                     # 2-bit g32, 4 heads per KV head: 2.5 bits
     (1, dict(context=2500, batch=2, n_q_heads=4, n_kv_heads=4, meta_fp8=True), 2500),          # one head per KV head, g128
     (1, dict(context=2100, batch=1, n_q_heads=16, n_kv_heads=2, group_size=64, meta_fp8=True, n_sink=5), 2100),   # 8 heads, g64, sinks
-    (4, dict(context=1300, batch=2, ragged=None, n_q_heads=4, n_kv_heads=4, meta_fp8=True), 1300),   # 4-bit g64: scalar kernel
+    (4, dict(context=1300, batch=2, ragged=None, n_q_heads=4, n_kv_heads=4, meta_fp8=True), 1300),   # 4-bit g64, integer kernel
+    (4, dict(context=1100, batch=1, ragged=None, n_q_heads=8, n_kv_heads=4, meta_fp8=True), 1100),   # 4-bit, 2 heads per KV head: scalar kernel
+    (2, dict(context=1500, batch=1, n_q_heads=24, meta_fp8=True), 1500),                             # 3 heads per KV head: tcgen05 kernel
+    (4, dict(context=1500, batch=1, ragged=None, n_q_heads=4, n_kv_heads=4, k_bits=4, v_bits=2, group_size=128, meta_fp8=True), 1500),   # mixed widths
     (0, dict(context=200, meta_fp8=True), 200),
 ])
 def test_fp8_parameters_bit_exact_cache_and_attention(cfg_i, kw, n):
