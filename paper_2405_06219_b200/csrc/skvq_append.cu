@@ -15,6 +15,8 @@
 // K rows on lanes 0-7/16-23 and V rows on lanes 8-15/24-31.  Group statistics are reduced with
 // xor-shuffles over G/16 lanes.  All quantizer arithmetic uses explicitly rounded fp32 intrinsics
 // so the codes, scales and zeros do not depend on compiler contraction.
+#include <type_traits>
+
 #include "skvq_internal.cuh"
 
 namespace skvq {
@@ -326,44 +328,50 @@ __global__ void __launch_bounds__(kAppendThreads) append_bulk_kernel(AppendArgs 
     const size_t bh = (size_t)b * s.Hkv + h;
     const int lanes_per_group = s.G >> 4;
     const int g = (sub << 4) / s.G;
-#pragma unroll 1
-    for (int tensor = 0; tensor < 2; ++tensor) {
-        const int bits = tensor ? s.v_bits : s.k_bits;
-        const int row_bytes = kHeadDim * bits / 8;
-        uint8_t *codes = (tensor ? a.c.v_codes : a.c.k_codes) + bh * (size_t)s.cap * row_bytes;
+    const bool f8 = s.meta_fp8 != 0;
+    // One tensor's 64 rows; the code width is a template parameter so that nothing inside branches on it.
+    auto quantize_tile = [&](auto bits_tag, int tensor) {
+        constexpr int BITS = decltype(bits_tag)::value;
+        constexpr int row_bytes = kHeadDim * BITS / 8;
+        uint8_t *codes = (tensor ? a.c.v_codes : a.c.k_codes) + (bh * (size_t)s.cap + t0) * row_bytes;
         __half2 *meta = (tensor ? a.c.v_meta : a.c.k_meta);      // two bytes per (token, group) with FP8 parameters
-        const size_t meta0 = bh * (size_t)s.cap * s.ng;
-        const bool f8 = s.meta_fp8 != 0;
+        const size_t meta0 = (bh * (size_t)s.cap + t0) * s.ng + g;
         const float alpha = ((tensor ? a.c.alpha_v : a.c.alpha_k) + (size_t)h * s.ng)[g];
-        int idx[16];
+        // this lane's 16 gather addresses (shared-memory window) in its first row; later rows are constant offsets
+        uint32_t src_j[16];
         {
             const int32_t *ip = (tensor ? a.c.reorder_v : a.c.reorder_k) + (size_t)h * kHeadDim + (sub << 4);
+            const uint32_t row0 = (uint32_t)__cvta_generic_to_shared(&xs[tensor][warp * 4 + rsel][0]);
 #pragma unroll
-            for (int j = 0; j < 16; ++j) idx[j] = ip[j] & (kHeadDim - 1);
+            for (int j = 0; j < 16; ++j) src_j[j] = row0 + 2u * (uint32_t)(ip[j] & (kHeadDim - 1));
         }
-        const __half *src_j[16];      // this lane's 16 gather addresses in its first row; later rows are constant offsets
 #pragma unroll
-        for (int j = 0; j < 16; ++j) src_j[j] = &xs[tensor][warp * 4 + rsel][idx[j]];
-#pragma unroll 2
         for (int it = 0; it < kBulkTok / 16; ++it) {
             const int tok = it * 16 + warp * 4 + rsel;
             float x[16];
 #pragma unroll
-            for (int j = 0; j < 16; ++j) x[j] = __half2float(src_j[j][it * 16 * kBulkStride]);
+            for (int j = 0; j < 16; ++j) {
+                unsigned short v;
+                asm("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(src_j[j] + (uint32_t)(it * 16 * kBulkStride * 2)));
+                x[j] = __half2float(__ushort_as_half(v));
+            }
             uint32_t words[2];
             uint32_t hz;
-            if (bits == 2) quantize16<2>(x, alpha, lanes_per_group, f8, words, hz);
-            else quantize16<4>(x, alpha, lanes_per_group, f8, words, hz);
-            const int t = t0 + tok;
-            uint8_t *codes_row = codes + (size_t)t * row_bytes;
-            if (bits == 2) reinterpret_cast<uint32_t *>(codes_row)[sub] = words[0];
+            quantize16<BITS>(x, alpha, lanes_per_group, f8, words, hz);
+            uint8_t *codes_row = codes + (size_t)tok * row_bytes;
+            if constexpr (BITS == 2) reinterpret_cast<uint32_t *>(codes_row)[sub] = words[0];
             else reinterpret_cast<uint2 *>(codes_row)[sub] = make_uint2(words[0], words[1]);
             if ((sub & (lanes_per_group - 1)) == 0) {
-                const size_t mi = meta0 + (size_t)t * s.ng + g;
+                const size_t mi = meta0 + (size_t)tok * s.ng;
                 if (f8) reinterpret_cast<uint16_t *>(meta)[mi] = (uint16_t)hz;
                 else reinterpret_cast<uint32_t *>(meta)[mi] = hz;
             }
         }
+    };
+#pragma unroll 1
+    for (int tensor = 0; tensor < 2; ++tensor) {
+        if ((tensor ? s.v_bits : s.k_bits) == 2) quantize_tile(std::integral_constant<int, 2>{}, tensor);
+        else quantize_tile(std::integral_constant<int, 4>{}, tensor);
     }
 }
 
