@@ -395,9 +395,14 @@ def main():
     value = job_tokens / (job_ms * 1e-3)
 
     # -- end to end through the host-buffer entry point
-    hk = torch.from_numpy(np.stack([w.new_token("k", 5000 + s) for s in range(n_in)])).pin_memory()
-    hv = torch.from_numpy(np.stack([w.new_token("v", 5000 + s) for s in range(n_in)])).pin_memory()
-    hq = torch.from_numpy(np.stack([w.query(5000 + s) for s in range(n_in)])).pin_memory()
+    # a step's k, v and q lie back to back in one pinned buffer, as a serving loop would stage them: one copy per step
+    kv_el, q_el = w.batch * w.n_kv_heads * w.head_dim, w.batch * w.n_q_heads * w.head_dim
+    hin = torch.empty((n_in, 2 * kv_el + q_el), dtype=torch.float16).pin_memory()
+    for s in range(n_in):
+        hin[s, :kv_el] = torch.from_numpy(w.new_token("k", 5000 + s).reshape(-1))
+        hin[s, kv_el:2 * kv_el] = torch.from_numpy(w.new_token("v", 5000 + s).reshape(-1))
+        hin[s, 2 * kv_el:] = torch.from_numpy(w.query(5000 + s).reshape(-1))
+    hk, hv, hq = hin[:, :kv_el], hin[:, kv_el:2 * kv_el], hin[:, 2 * kv_el:]
     hout = torch.empty(tuple(q_all[0].shape), dtype=torch.float16).pin_memory()
     staging = torch.empty(binding.skvq_step_staging_size(cache.cfg), dtype=torch.uint8, device="cuda")
     a = cache.attn_args(w.sm_scale, hint, args.splits)

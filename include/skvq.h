@@ -181,7 +181,8 @@ int skvq_decode_attention(const skvq_config *cfg, const skvq_cache *cache, const
  * One decode step driven from HOST buffers: copies k_new, v_new (half [B][1][Hkv][D]) and q
  * (half [B][Hq][D]) from host memory into `staging`, appends the token, runs decode attention and
  * copies out (half [B][Hq][D]) back to host memory, all enqueued on the stream (the caller
- * synchronises before reading out_host).  Pinned host memory keeps the copies asynchronous.
+ * synchronises before reading out_host).  Pinned host memory keeps the copies asynchronous; when k_new, v_new
+ * and q lie back to back in host memory in that order they travel in one copy instead of three.
  *   staging  device scratch of at least skvq_step_staging_size(cfg) bytes
  */
 size_t skvq_step_staging_size(const skvq_config *cfg);

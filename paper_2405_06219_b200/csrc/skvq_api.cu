@@ -217,9 +217,15 @@ int skvq_decode_step_host(const skvq_config *cfg, const skvq_cache *cache, const
     const size_t qo = (size_t)cfg->batch * cfg->n_q_heads * kHeadDim * sizeof(__half);
     char *base = static_cast<char *>(staging);
     void *d_k = base, *d_v = base + kv, *d_q = base + 2 * kv, *d_out = base + 2 * kv + qo;
-    if (cudaMemcpyAsync(d_k, k_new_host, kv, cudaMemcpyHostToDevice, stream) != cudaSuccess) return SKVQ_ERR_CUDA;
-    if (cudaMemcpyAsync(d_v, v_new_host, kv, cudaMemcpyHostToDevice, stream) != cudaSuccess) return SKVQ_ERR_CUDA;
-    if (cudaMemcpyAsync(d_q, q_host, qo, cudaMemcpyHostToDevice, stream) != cudaSuccess) return SKVQ_ERR_CUDA;
+    const char *hk = static_cast<const char *>(k_new_host);
+    if (static_cast<const char *>(v_new_host) == hk + kv && static_cast<const char *>(q_host) == hk + 2 * kv) {
+        // the three inputs lie back to back in host memory, in the order they have in `staging`: one copy
+        if (cudaMemcpyAsync(d_k, k_new_host, 2 * kv + qo, cudaMemcpyHostToDevice, stream) != cudaSuccess) return SKVQ_ERR_CUDA;
+    } else {
+        if (cudaMemcpyAsync(d_k, k_new_host, kv, cudaMemcpyHostToDevice, stream) != cudaSuccess) return SKVQ_ERR_CUDA;
+        if (cudaMemcpyAsync(d_v, v_new_host, kv, cudaMemcpyHostToDevice, stream) != cudaSuccess) return SKVQ_ERR_CUDA;
+        if (cudaMemcpyAsync(d_q, q_host, qo, cudaMemcpyHostToDevice, stream) != cudaSuccess) return SKVQ_ERR_CUDA;
+    }
     rc = skvq_quantize_append(cfg, cache, d_k, d_v, nullptr, 1, cuda_stream);
     if (rc != SKVQ_OK) return rc;
     rc = skvq_decode_attention(cfg, cache, d_q, d_out, args, cuda_stream);

@@ -241,15 +241,21 @@ def test_decode_loop_append_then_attend():
     assert_cache_bit_exact(gpu, ora)
 
 
-def test_host_buffer_decode_step():
+@pytest.mark.parametrize("pinned", [True, False])
+def test_host_buffer_decode_step(pinned):
+    """Page-locked and pageable host buffers alike."""
     w = small(1, context=2000, batch=2)
     gpu, ora = both_caches(w, 2100)
     k, v = w.prefill("k", 2000), w.prefill("v", 2000)
     gpu.append(dev(k), dev(v))
     ora.append(k, v)
     kn, vn, q = w.new_token("k", 0), w.new_token("v", 0), w.query(5)
-    hk, hv, hq = (torch.from_numpy(x).pin_memory() for x in (kn, vn, q))
-    hout = torch.empty(q.shape, dtype=torch.float16).pin_memory()
+    hk, hv, hq = (torch.from_numpy(np.ascontiguousarray(x)) for x in (kn, vn, q))
+    hout = torch.zeros(q.shape, dtype=torch.float16)
+    if pinned:      # one pinned buffer, k, v and q back to back: a single copy
+        hin = torch.cat([hk.reshape(-1), hv.reshape(-1), hq.reshape(-1)]).pin_memory()
+        hk, hv, hq = hin[:hk.numel()], hin[hk.numel():2 * hk.numel()], hin[2 * hk.numel():]
+        hout = hout.pin_memory()
     staging = torch.empty(B.skvq_step_staging_size(gpu.cfg), dtype=torch.uint8, device="cuda")
     before = B.skvq_launch_count()
     B.skvq_decode_step_host(gpu.cfg, gpu.struct, hk, hv, hq, hout, staging, gpu.attn_args(w.sm_scale, 2001))
