@@ -1,10 +1,12 @@
 // Partition kernel of skvq_decode_attention on the fifth-generation tensor cores (tcgen05.mma, accumulators in
-// tensor memory) for 2-bit K and V with up to 4 query heads per KV head and any group size (Eq. 1, Algorithm 1).
+// tensor memory) for 2-bit K and V with up to 4 query heads per KV head per launch and any group size (Eq. 1,
+// Algorithm 1); scale and zero point stored as fp16 pairs or as E4M3 byte pairs.
 //
 //   q'.K~_t            = sum_g h_{t,g} (sum_{j in g} q'_j c_{t,j}) + sum_g z_{t,g} (sum_{j in g} q'_j)
 //   sum_t p_t V~_{t,d} = sum_t (p_t h_{t,g(d)}) c_{t,d} + sum_t p_t z_{t,g(d)}
 //
-// One CTA = 128 threads = one tile of 128 tokens at a time, one thread per token.  The warps only unpack and do the
+// One CTA = 128 token threads (one tile of 128 tokens at a time, one thread per token) and one control warp; three
+// CTAs per SM (128 tensor-memory columns and 69 KB of shared memory each).  The token threads only unpack and do the
 // per-(token, head, group) arithmetic; both contractions run asynchronously on the tensor core:
 //   * a thread turns its token's 32 packed bytes into 128 bytes "4^j * code" (one AND per four codes) and stores them
 //     as a row of the A operand of the score MMA (u8, K-major).  The B operand holds the permuted query of every head
@@ -13,14 +15,18 @@
 //     16 columns (head, digit) per quantization group.
 //   * the thread reads its row of accumulators from tensor memory, combines digits and groups with h and z (fp32),
 //     and takes part in a lazy online softmax: the reference of a head moves only when a score exceeds it by 8 in
-//     the log2 domain (or the bound on the value scales has to grow), which after the first tile is rare.
-//   * p*h per (head, group) goes onto a 32-bit fixed-point grid; the four bytes of that integer are four rows
-//     (head, digit) of the A operand of the value MMA (u8, MN-major: one 16-byte store per group), whose B operand
-//     is the unpacked V tile exactly as the thread stored it (u8, MN-major).  Rows are (group, head, digit): 64 rows
-//     x 128 channels of exact int32 sums in tensor memory, of which the (group, channels of that group) blocks are
-//     read when the reference moves, every 256 tiles, and at the end of a segment.
-// Tiles arrive through a ring of shared-memory stages filled by cp.async.bulk (mbarrier completion); every wait is
-// bounded and reports through the cache's status word.
+//     the log2 domain (or the bound on the value scales has to grow), which after the first tiles is rare.
+//   * p*h per (head, group) goes onto a 32-bit fixed-point grid; the four bytes of that integer are four columns
+//     (group, head, digit) of the B operand of the value MMA (u8, MN-major: one 16-byte store per group and token),
+//     whose A operand is the V tile unpacked like K (u8, MN-major): 128 byte columns of V on the M rows x 64 columns
+//     of exact int32 sums in tensor memory.  The thread that owns tensor-memory lane c folds the 16 columns of
+//     channel c's group into fp32 when the reference moves, every 256 tiles, and at the end of a segment.
+//   * the control warp issues every copy and every MMA in the order in which the token threads finish the operands:
+//     they arrive on an mbarrier (behind fence.proxy.async), the control lane waits, issues, and commits the MMAs to
+//     the mbarrier the token threads wait on.
+// K codes are needed one tile before the rest of a tile, so they have a copy ring of their own (cp.async.bulk,
+// mbarrier completion); every wait is bounded and reports through the cache's status word; the tensor memory is
+// given back on every exit path.
 #include "skvq_mma_common.cuh"
 
 namespace skvq {
