@@ -83,7 +83,8 @@ __device__ __forceinline__ __half2 from_e4m3x2(uint16_t b)
 }
 
 // Writes what is stored per (token, group): a half2 {h, z}, or its two E4M3 bytes in the low 16 bits of hz_bits.
-template <int BITS>
+// LPG > 0: lanes per group known at compile time (the shuffle rounds unroll); 0: taken from lanes_per_group.
+template <int BITS, int LPG = 0>
 __device__ __forceinline__ void quantize16(const float (&x)[16], float alpha, int lanes_per_group, bool meta_fp8,
                                            uint32_t (&words)[2], uint32_t &hz_bits)
 {
@@ -97,9 +98,17 @@ __device__ __forceinline__ void quantize16(const float (&x)[16], float alpha, in
         mn = fminf(mn, x[j]);
         mx = fmaxf(mx, x[j]);
     }
-    for (int m = 1; m < lanes_per_group; m <<= 1) {
-        mn = fminf(mn, __shfl_xor_sync(seg_mask, mn, m));
-        mx = fmaxf(mx, __shfl_xor_sync(seg_mask, mx, m));
+    if constexpr (LPG > 0) {
+#pragma unroll
+        for (int m = 1; m < LPG; m <<= 1) {
+            mn = fminf(mn, __shfl_xor_sync(seg_mask, mn, m));
+            mx = fmaxf(mx, __shfl_xor_sync(seg_mask, mx, m));
+        }
+    } else {
+        for (int m = 1; m < lanes_per_group; m <<= 1) {
+            mn = fminf(mn, __shfl_xor_sync(seg_mask, mn, m));
+            mx = fmaxf(mx, __shfl_xor_sync(seg_mask, mx, m));
+        }
     }
     // Clip both ends (Eq. 2 / clipping_quant); "+ 0" turns a negative zero into +0.
     const float lo = __fadd_rn(__fmul_rn(alpha, mn), 0.0f);
@@ -298,6 +307,7 @@ __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc)
 
 // One CTA = one (sequence, KV head, 64-token tile) of bulk_range(): 64 K rows and 64 V rows are copied to
 // shared memory in 16-byte pieces (coalesced 256-byte rows), then gathered by the reorder index from there.
+template <int G>
 __global__ void __launch_bounds__(kAppendThreads) append_bulk_kernel(AppendArgs a)
 {
     const Shape &s = a.s;
@@ -326,8 +336,8 @@ __global__ void __launch_bounds__(kAppendThreads) append_bulk_kernel(AppendArgs 
 
     const int sub = lane & 7, rsel = lane >> 3;
     const size_t bh = (size_t)b * s.Hkv + h;
-    const int lanes_per_group = s.G >> 4;
-    const int g = (sub << 4) / s.G;
+    constexpr int lanes_per_group = G >> 4;
+    const int g = (sub << 4) / G;
     const bool f8 = s.meta_fp8 != 0;
     // One tensor's 64 rows; the code width is a template parameter so that nothing inside branches on it.
     auto quantize_tile = [&](auto bits_tag, int tensor) {
@@ -357,7 +367,7 @@ __global__ void __launch_bounds__(kAppendThreads) append_bulk_kernel(AppendArgs 
             }
             uint32_t words[2];
             uint32_t hz;
-            quantize16<BITS>(x, alpha, lanes_per_group, f8, words, hz);
+            quantize16<BITS, lanes_per_group>(x, alpha, lanes_per_group, f8, words, hz);
             uint8_t *codes_row = codes + (size_t)tok * row_bytes;
             if constexpr (BITS == 2) reinterpret_cast<uint32_t *>(codes_row)[sub] = words[0];
             else reinterpret_cast<uint2 *>(codes_row)[sub] = make_uint2(words[0], words[1]);
@@ -407,7 +417,9 @@ cudaError_t launch_append(const Shape &s, const CachePtrs &c, const __half *k, c
     int launched = 0;
     if (bulk) {
         dim3 gridb((n_new + kBulkTok - 1) / kBulkTok, s.Hkv, s.B);
-        append_bulk_kernel<<<gridb, kAppendThreads, 0, stream>>>(a);
+        if (s.G == 128) append_bulk_kernel<128><<<gridb, kAppendThreads, 0, stream>>>(a);
+        else if (s.G == 64) append_bulk_kernel<64><<<gridb, kAppendThreads, 0, stream>>>(a);
+        else append_bulk_kernel<32><<<gridb, kAppendThreads, 0, stream>>>(a);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         ++launched;
