@@ -241,6 +241,44 @@ def test_decode_loop_append_then_attend():
     assert_cache_bit_exact(gpu, ora)
 
 
+@pytest.mark.parametrize("cfg_i,kw", [(1, dict(context=3000, batch=2, n_q_heads=4, n_kv_heads=4)),       # integer kernel
+                                       (2, dict(context=2500, batch=2)),                                 # grouped-query kernel
+                                       (2, dict(context=2500, batch=1, n_q_heads=24))])                  # tcgen05 kernel
+def test_decode_step_replays_from_a_cuda_graph(cfg_i, kw):
+    """The calls only enqueue work and read the lengths on the device, so one captured decode step (append one
+    token, attend) can be replayed with new inputs in the same buffers."""
+    w = small(cfg_i, **kw)
+    n = w.context
+    gpu, ora = both_caches(w, n + 64)
+    k, v = w.prefill("k", n), w.prefill("v", n)
+    gpu.append(dev(k), dev(v))
+    ora.append(k, v)
+    k_in, v_in, q_in = dev(w.new_token("k", 0)), dev(w.new_token("v", 0)), dev(w.query(0))
+    out = torch.empty_like(q_in)
+    args = gpu.attn_args(w.sm_scale, n + 64)                          # workspace allocated before the capture
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):                                     # one eager step first: kernels get configured
+        gpu.append(k_in, v_in)
+        B.skvq_decode_attention(gpu.cfg, gpu.struct, q_in, out, args)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    ora.append(w.new_token("k", 0), w.new_token("v", 0))
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        gpu.append(k_in, v_in)
+        B.skvq_decode_attention(gpu.cfg, gpu.struct, q_in, out, args)
+    for s in range(1, 6):
+        kn, vn, q = w.new_token("k", s), w.new_token("v", s), w.query(s)
+        k_in.copy_(dev(kn)); v_in.copy_(dev(vn)); q_in.copy_(dev(q))
+        graph.replay()
+        torch.cuda.synchronize()
+        ora.append(kn, vn)
+        want = ora.attention(q, w.sm_scale)
+        assert np.abs(out.cpu().numpy().astype(np.float64) - want).max() <= ATTN_TOL
+    assert_cache_bit_exact(gpu, ora)
+
+
 @pytest.mark.parametrize("pinned", [True, False])
 def test_host_buffer_decode_step(pinned):
     """Page-locked and pageable host buffers alike."""
