@@ -337,6 +337,7 @@ __global__ void __launch_bounds__(kThreads, SKVQ_GQA_CTAS) partition_gqa_kernel(
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = 0;
     float h_bound = 6.103515625e-05f;                          // power of two above every value scale seen so far
+    int tiles_since_fold = 0;                                  // a token adds at most 255 * 192 to an int32 sum: fold at least every 32768 tokens
     uint32_t h_thr = 0x0400u;                                  // the same bound as an fp16 bit pattern (2^-14)
     bool acc_live = false;
 
@@ -375,6 +376,7 @@ __global__ void __launch_bounds__(kThreads, SKVQ_GQA_CTAS) partition_gqa_kernel(
                 o[4] = (o[4] + x1) * corr_hd;
             }
             acc[nt][0] = 0; acc[nt][1] = 0; acc[nt][2] = 0; acc[nt][3] = 0;
+            tiles_since_fold = 0;
         }
     };
 
@@ -462,7 +464,7 @@ __global__ void __launch_bounds__(kThreads, SKVQ_GQA_CTAS) partition_gqa_kernel(
             for (int gg = 1; gg < NG; ++gg) mx = __vmaxu2(mx, __vmaxu2(wa[gg], wb[gg]));
             hmax_bits = mx & 0xFFFFu;                          // scales are non-negative: fp16 order = integer order
         }
-        bool moved = hmax_bits >= h_thr;
+        bool moved = hmax_bits >= h_thr || ++tiles_since_fold * kTileTok >= 32768;
         float arg[4][2];
         float amax = -CUDART_INF_F;
 #pragma unroll

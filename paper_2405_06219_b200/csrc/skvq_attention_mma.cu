@@ -218,6 +218,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB, F8>::kCtasPerSm) part
 #pragma unroll
         for (int i = 0; i < 4; ++i) { cv[f][i] = 0.f; iacc[f][i] = 0; }
     float h_bound = 6.103515625e-05f;   // 2^-14: every scale seen so far is below this power of two
+    int tiles_since_fold = 0;           // a token adds at most 255 * 240 to an int32 sum: fold at least every 32768 tokens
 
     const uint32_t kmask = KB == 2 ? (0x03030303u << (2 * t)) : (0x0F0F0F0Fu << (4 * (t & 1)));
 
@@ -290,7 +291,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB, F8>::kCtasPerSm) part
         // ---------------- softmax bookkeeping: lane owns tokens lane (and lane+32) of the tile
         float sc[T / 32];
         float hv[T / 32][NG], zv[T / 32][NG];
-        bool moved = false;   // does any score exceed the running maximum, or any scale the running bound?
+        // does any score exceed the running maximum, or any scale the running bound (or are the int32 sums getting full)?
+        bool moved = ++tiles_since_fold * T >= 32768;
 #pragma unroll
         for (int hf = 0; hf < T / 32; ++hf) {
             const int tau = lane + 32 * hf;
@@ -338,6 +340,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB, F8>::kCtasPerSm) part
                 cv[f][2] = fmaf((float)iacc[f][2], f0, cv[f][2]) * corr;
                 cv[f][3] = fmaf((float)iacc[f][3], f1, cv[f][3]) * corr;
                 iacc[f][0] = 0; iacc[f][1] = 0; iacc[f][2] = 0; iacc[f][3] = 0;
+                tiles_since_fold = 0;
             }
             if (hm >= h_bound) h_bound = __int_as_float(((__float_as_int(hm) >> 23) + 1) << 23);   // next power of two above hm
         }

@@ -99,3 +99,24 @@ def test_full_size_sampled_pairs_match_oracle(cfg_i, kw, b, kv_heads):
     assert np.isfinite(out.cpu().numpy()).all()
     assert np.abs(got - want).max() <= ATTN_TOL
     assert int(gpu.status[0]) == 0
+
+
+@pytest.mark.parametrize("kw", [
+    dict(n_q_heads=1, n_kv_heads=1),                       # integer kernel, one head
+    dict(n_q_heads=4, n_kv_heads=1, group_size=32),        # grouped-query kernel
+    dict(n_q_heads=3, n_kv_heads=1, group_size=64),        # tcgen05 kernel
+])
+def test_one_cta_streams_a_whole_long_sequence(kw):
+    """n_splits = 1 gives the whole sequence to one CTA: each warp then accumulates several hundred thousand tokens,
+    far more than the int32 value sums hold between two folds unless the kernels fold on their own."""
+    from paper_2405_06219_b200 import binding as B
+    w = workloads.configs()[1].scaled(batch=1, context=900_000, **kw)
+    gpu = B.SkvqCache.for_workload(w, w.context + 64)
+    prefill_like_the_benchmark(w, gpu, chunk=1 << 17)
+    oc = oracle_for_pairs(w, 0, [0], 0)
+    q = w.query(3)
+    out = gpu.attention(torch.from_numpy(q).cuda(), w.sm_scale, w.context + 64, n_splits=1)
+    torch.cuda.synchronize()
+    want = oc.attention(q, w.sm_scale)
+    assert np.abs(out.cpu().numpy().astype(np.float64) - want).max() <= ATTN_TOL
+    assert int(gpu.status[0]) == 0
