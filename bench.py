@@ -38,7 +38,7 @@ PREFILL_CHUNK = 32768
 L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes (read + write) per launch of the partition kernel from ncu captures, keyed by configuration;
 # absent (None) where no capture exists for the current kernel.
-NCU_TRAFFIC_BYTES = {1: 618.3e6, 2: 411.5e6, 4: 2553.3e6}      # reduced-batch ncu captures scaled by tokens streamed
+NCU_TRAFFIC_BYTES = {1: 632.6e6, 2: 412.8e6, 4: 2551.9e6}      # reduced-batch ncu captures scaled by tokens streamed
 
 
 def measured_peak():
