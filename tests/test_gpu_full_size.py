@@ -119,4 +119,10 @@ def test_one_cta_streams_a_whole_long_sequence(kw):
     torch.cuda.synchronize()
     want = oc.attention(q, w.sm_scale)
     assert np.abs(out.cpu().numpy().astype(np.float64) - want).max() <= ATTN_TOL
+    # q = 0: every token has the same probability, so every token contributes full-size digits to the int32 sums
+    # (the worst case for their range); the result is the mean of the dequantized values
+    q0 = np.zeros_like(q)
+    out0 = gpu.attention(torch.from_numpy(q0).cuda(), w.sm_scale, w.context + 64, n_splits=1)
+    torch.cuda.synchronize()
+    assert np.abs(out0.cpu().numpy().astype(np.float64) - oc.attention(q0, w.sm_scale)).max() <= ATTN_TOL
     assert int(gpu.status[0]) == 0
