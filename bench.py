@@ -278,7 +278,7 @@ def main():
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     w = sharding.rank_workload(w0, rank, world)
-    n_steps_total = 3 * (args.warmup + args.steps) + 8
+    n_steps_total = 4 * (args.warmup + args.steps) + 8      # warm-up, three passes of the steps, the end-to-end pass
     cache, prefill_ms, prefill_in = build_gpu_cache(w, n_steps_total + 64, torch, binding)
     lengths0 = w.lengths()
     hint = int(lengths0.max()) + n_steps_total
@@ -358,8 +358,8 @@ def main():
         if flush is None:
             e0.record()
             for i in range(args.steps):
-                step(args.warmup + i, args_plain, ev_call[i])
-            e1.record()
+                step(args.warmup + i, args_plain)      # nothing but the calls: an event between two calls would
+            e1.record()                                # keep the dependent launches from overlapping
             barrier()
             elapsed_ms = e0.elapsed_time(e1)
         else:   # small cache: flush L2 before every step and time each step on its own
@@ -367,20 +367,26 @@ def main():
             for i in range(args.steps):
                 flush.fill_(i & 1)
                 e0.record()
-                step(args.warmup + i, args_plain, ev_call[i])
+                step(args.warmup + i, args_plain)
                 e1.record()
                 torch.cuda.synchronize()
                 per.append(e0.elapsed_time(e1))
             barrier()
             elapsed_ms = sum(per)
         launches = binding.skvq_launch_count() - launches0
-        # the same steps once more with the library's own events around the partition kernel (an event between
+        # the same steps again with the library's own events around the partition kernel (an event between
         # the two kernels keeps the merge kernel from overlapping the partition kernel's tail, so this pass
         # measures the dominant kernel alone and the pass above measures the step as a user runs it)
         for i in range(args.steps):
             if flush is not None:
                 flush.fill_(i & 1)
             step(args.warmup + i, args_timed[i])
+        torch.cuda.synchronize()
+        # and once more with events around the attention call (partition + merge)
+        for i in range(args.steps):
+            if flush is not None:
+                flush.fill_(i & 1)
+            step(args.warmup + i, args_plain, ev_call[i])
         torch.cuda.synchronize()
         # keep the same kernels running (untimed) until the sampler has seen them under load
         t_end = time.perf_counter() + 3.0
@@ -420,7 +426,10 @@ def main():
     e1.record()
     barrier()
     e2e_ms = max(e0.elapsed_time(e1), 0.0)
-    e2e_tokens = (float(lengths0.sum()) + w.batch * (n_in + args.warmup + (args.steps + 1) / 2.0)) * args.steps
+    if int(cache.status[0].item()) != 0:      # capacity overflow or a copy that never completed: the numbers would be void
+        raise SystemExit(f"the cache's status word is {int(cache.status[0].item())} after the timed passes")
+    # lengths at the end-to-end pass: warm-up and three passes of the steps are already in the cache
+    e2e_tokens = (float(lengths0.sum()) + w.batch * (2 * args.warmup + 3 * args.steps + (args.steps + 1) / 2.0)) * args.steps
     e2e_ms, e2e_tokens = sharding.reduce_job(e2e_ms, e2e_tokens,
                                              device=torch.device("cuda", local_rank) if world > 1 else None)
     kv_bytes = w.batch * w.n_kv_heads * w.head_dim * 2
