@@ -207,8 +207,13 @@ int skvq_decode_step_host(const skvq_config *cfg, const skvq_cache *cache, const
  *   - Shapes whose partials need more than SKVQ_NOALLOC_SCRATCH_BYTES (that is,
  *     skvq_workspace_size(cfg, max_len_hint, n_splits) > SKVQ_NOALLOC_SCRATCH_BYTES) are refused with
  *     SKVQ_ERR_SCRATCH_LIMIT before anything is launched; ask for fewer splits or use the workspace variant.
- *   - The first call on each device looks up the array's device address (with that device current).  Make
- *     that first call outside any stream capture.
+ *   - The first call on each device looks up the array's device address (with that device current).  The CUDA
+ *     runtime loads a library's device image lazily, so this first lookup is also the moment the image, and the
+ *     array in it, is placed in that device's memory: on a device that is already full it fails with
+ *     SKVQ_ERR_CUDA.  Make the first call on every device at start-up -- before the engine sizes its KV cache to
+ *     the remaining memory, and outside any stream capture; later calls only launch kernels.
+ *   - The looked-up address is kept until the process exits.  cudaDeviceReset() (or anything else that destroys
+ *     the device's primary context) invalidates it; this entry point must not be used on that device afterwards.
  *   - All calls on a device share the one array, and it keeps whatever the last call left there.  Nothing
  *     needs clearing (a call writes every partial before it reads it), but two calls that overlap on the GPU
  *     -- different streams, no ordering between them -- race on it.  Keep them stream-ordered.

@@ -241,10 +241,12 @@ int skvq_decode_step_host(const skvq_config *cfg, const skvq_cache *cache, const
 static __device__ __align__(256) unsigned char g_noalloc_scratch[SKVQ_NOALLOC_SCRATCH_BYTES];
 
 namespace {
-constexpr int kMaxDevices = 64;
 std::atomic<float *> g_noalloc_ptr[kMaxDevices];
 
-// Device address of the array on the current device, looked up once per device.
+// Device address of the array on the current device, looked up once per device.  With CUDA's lazy module loading
+// this lookup is also what places the library's image -- and with it the array -- on that device, so it can fail
+// on a device whose memory is already full; callers make their first call at start-up.  The address is kept for
+// the life of the process: a cudaDeviceReset() invalidates it (documented in skvq.h).
 int noalloc_scratch(float **out)
 {
     int dev = -1;

@@ -50,8 +50,11 @@ __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
     const Shape &s = a.s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int rep = s.rep, G = s.G, ng = s.ng;
-    asm volatile("griddepcontrol.launch_dependents;");      // the merge kernel may start its window part early
+    // Order matters: the merge kernel reads the lengths, the sinks and the window BEFORE its own wait, so it may only be
+    // scheduled once everything in front of this grid (append, bookkeeping, plan) has completed and is visible.  Waiting
+    // first and triggering afterwards gives exactly that; the merge kernel still runs under this kernel's body.
     asm volatile("griddepcontrol.wait;" ::: "memory");      // the lengths, and the plan kernel's header when there is one
+    asm volatile("griddepcontrol.launch_dependents;");      // the merge kernel may start its window part now
 
     __shared__ __align__(16) Segment seg_sh;
     __shared__ int more_sh;
@@ -228,8 +231,8 @@ __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
 // prefix array, their total over all KV heads, and the units per slot.  One warp; B is small next to the cache.
 __global__ void plan_kernel(AttnArgs a)
 {
-    asm volatile("griddepcontrol.launch_dependents;");      // the partition kernel may start its launch now; it waits for this grid
     asm volatile("griddepcontrol.wait;" ::: "memory");      // whatever wrote the lengths (the append kernels, typically)
+    asm volatile("griddepcontrol.launch_dependents;");      // the partition kernel may be scheduled; it waits for this grid before it reads the header
     int *hdr = reinterpret_cast<int *>(a.ws);
     int *pre = hdr + kPlanHdrInts;
     const int lane = threadIdx.x & 31;
@@ -281,6 +284,9 @@ __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
     const Shape &s = a.s;
     const int hk = hq / s.rep;
     const int W = s.W;
+    // Read before this kernel's own griddepcontrol.wait: safe because every partition kernel (and the plan kernel) waits for
+    // its predecessors BEFORE it lets its dependents be scheduled, so by the time a CTA of this grid runs, the append and
+    // bookkeeping kernels in front of the partition kernel have completed and their writes (lengths, ring, sinks) are visible.
     const int L = a.c.lengths[b];
     const int Lq = max(L - W, 0);
     __shared__ float sq[kHeadDim];
@@ -424,19 +430,29 @@ static int partition_ctas_per_sm(const Shape &s)
     return 8;                                                                  // scalar kernel
 }
 
-static int sm_count()
+int current_device()
 {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess &&
-            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
-            n = v;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) {
+        (void)cudaGetLastError();
+        dev = 0;
+    }
+    return dev;
+}
+
+int sm_count()
+{
+    static int n[kMaxDevices] = {};        // per device: a process may drive GPUs of different sizes
+    const int dev = current_device() & (kMaxDevices - 1);
+    if (n[dev] == 0) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+            n[dev] = v;
         else
-            n = 148;
+            n[dev] = 148;
         (void)cudaGetLastError();
     }
-    return n;
+    return n[dev];
 }
 
 SplitPlan plan_splits(const Shape &s, int max_len, int requested_splits)

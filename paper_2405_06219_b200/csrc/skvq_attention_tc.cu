@@ -190,8 +190,11 @@ __global__ void __launch_bounds__(kTile + 32, kCtasPerSm) partition_tc_kernel(Mm
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool control = warp == kWarps;      // warp 4 issues every copy and MMA; warps 0-3 own one token each
     const int R = min(kHeads, s.rep - a.head0);      // query heads of every KV head served by this launch
-    asm volatile("griddepcontrol.launch_dependents;");      // the merge kernel may start its window part early
+    // Order matters: the merge kernel reads the lengths, the sinks and the window BEFORE its own wait, so it may only be
+    // scheduled once everything in front of this grid (append, bookkeeping, plan) has completed and is visible.  Waiting
+    // first and triggering afterwards gives exactly that; the merge kernel still runs under this kernel's body.
     asm volatile("griddepcontrol.wait;" ::: "memory");      // the lengths, and the plan kernel's header when there is one
+    asm volatile("griddepcontrol.launch_dependents;");      // the merge kernel may start its window part now
 
     __shared__ __align__(16) Segment seg_sh;
     __shared__ int more_sh;
@@ -630,13 +633,10 @@ template <int G, bool F8>
 cudaError_t launch_g(const MmaArgs &a, cudaStream_t stream, bool overlap)
 {
     using C = TCfg<G, F8>;
-    static bool configured = false;
+    static unsigned long long configured = 0;      // one bit per device
     auto kern = partition_tc_kernel<G, F8>;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    const cudaError_t ec = configure_smem_once(kern, C::kSmemBytes, configured);
+    if (ec != cudaSuccess) return ec;
     return launch_dependent(kern, dim3(a.plan.n_slots), dim3(kTile + 32), C::kSmemBytes, stream, overlap, a);
 }
 

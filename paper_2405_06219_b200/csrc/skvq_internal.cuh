@@ -162,4 +162,22 @@ cudaError_t launch_partition_tc(const Shape &s, const CachePtrs &c, const __half
 
 void count_launch(int n = 1);
 
+// Per-device state of the host side: function attributes (the dynamic shared-memory opt-in) belong to a device, so a
+// process that drives several GPUs has to set them once on each.
+constexpr int kMaxDevices = 64;
+int current_device();                      // cudaGetDevice, or 0 when that fails
+int sm_count();                            // multiprocessors of the current device
+
+// Sets the dynamic shared-memory limit of `kern` once per device.  `done` is a bit mask owned by the caller (one per kernel).
+template <typename Kern>
+inline cudaError_t configure_smem_once(Kern kern, int bytes, unsigned long long &done)
+{
+    const int dev = current_device();
+    const unsigned long long bit = 1ull << (dev & (kMaxDevices - 1));
+    if (done & bit) return cudaSuccess;
+    const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) done |= bit;     // racing host threads set the same attribute twice: harmless
+    return e;
+}
+
 }  // namespace skvq

@@ -12,7 +12,7 @@ constexpr int kWarps = 4;
 constexpr int kThreads = kWarps * 32;
 constexpr int kTileTok = 64;                 // tokens per warp tile
 constexpr int kRowBytes = 32;                // 128 channels x 2 bits
-constexpr uint32_t kWaitLimit = 1u << 22;    // bounded mbarrier polling
+constexpr unsigned long long kWaitLimitNs = 100ull * 1000 * 1000;   // a shared-memory copy that has not landed after 0.1 s never will
 
 struct MmaArgs {
     Shape s;
@@ -90,12 +90,24 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
                  : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Poll with an iteration limit; false means the copy never completed (reported, never spun on forever).
+__device__ __forceinline__ unsigned long long global_timer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Poll with a limit on elapsed time (a try_wait may itself suspend for a hardware-defined interval, so an iteration
+// count alone bounds nothing); false means the copy never completed (reported, never spun on forever).
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
 {
-    for (uint32_t i = 0; i < kWaitLimit; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
+    if (mbar_try_wait(bar, parity)) return true;          // the common case: the copy landed long ago
+    const unsigned long long t0 = global_timer_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 32; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (global_timer_ns() - t0 > kWaitLimitNs) return false;
+    }
 }
 // Bulk asynchronous copy global -> this CTA's shared memory; 16-byte aligned addresses, size % 16 == 0.
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)

@@ -33,3 +33,29 @@ def reduce_job(elapsed_ms: float, units: float, device=None):
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     dist.all_reduce(u, op=dist.ReduceOp.SUM)
     return float(t.item()), float(u.item())
+
+
+def _reduce(values, op_name: str, device=None):
+    """Element-wise reduction of a list of floats over the ranks; identity without a process group."""
+    import torch
+    import torch.distributed as dist
+    vals = [float(x) for x in values]
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return vals
+    t = torch.tensor(vals, dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=getattr(dist.ReduceOp, op_name))
+    return [float(x) for x in t.tolist()]
+
+
+def reduce_max_list(values, device=None):
+    """Per-pass timings: every entry becomes the slowest rank's."""
+    return _reduce(values, "MAX", device)
+
+
+def reduce_max(value: float, device=None) -> float:
+    return _reduce([value], "MAX", device)[0]
+
+
+def reduce_sum(value: float, device=None) -> float:
+    """Units of work: the whole job's."""
+    return _reduce([value], "SUM", device)[0]

@@ -19,6 +19,7 @@ long sequence can be regenerated without producing the rest.
 from __future__ import annotations
 
 import dataclasses
+import os
 from concurrent.futures import ThreadPoolExecutor
 
 import numpy as np
@@ -102,7 +103,7 @@ class Workload:
         if len(chunks) == 1:
             fill(chunks[0])
         else:
-            with ThreadPoolExecutor(max_workers=8) as ex:
+            with ThreadPoolExecutor(max_workers=min(32, max(8, os.cpu_count() or 8))) as ex:
                 list(ex.map(fill, chunks))
         return out
 

@@ -4,7 +4,7 @@ The GPU cache is prefilled chunk by chunk with the library's own quantize_append
 it, a few single-token decode appends follow, and decode attention runs with the default partition.  The CPU
 oracle cannot redo a whole configuration in reasonable time, so it redoes SAMPLED (sequence, KV head) pairs in
 full: every stored row of those pairs must be bit-exact and the attention output of their query heads within
-the tolerance.  The 1M-token case keeps the context of configuration 3 and reduces the head count.
+the tolerance.  Configurations 1 to 4 run at their full sizes (configuration 3 also once with two heads).
 """
 import numpy as np
 import pytest
@@ -51,13 +51,26 @@ def oracle_for_pairs(w, b, kv_heads, n_steps):
     return oc
 
 
-@pytest.mark.parametrize("cfg_i,kw,b,kv_heads", [
-    (1, dict(), 7, [0, 31]),                                        # 32k x batch 8, one query head per KV head
-    (2, dict(), 3, [5]),                                            # 128k x batch 4, four query heads per KV head, group 32
-    (2, dict(n_q_heads=24, meta_fp8=True, n_sink=5), 1, [2]),       # the tcgen05 kernel, FP8 parameters, sinks
-    (3, dict(n_q_heads=2, n_kv_heads=2), 0, [1]),                   # one sequence of 1M tokens (two heads instead of 32)
+def pick_sequence(lengths, which):
+    """An index into the batch: an int as it is, or the longest / shortest / median-length sequence."""
+    if isinstance(which, int):
+        return which
+    order = np.argsort(lengths, kind="stable")
+    return int({"longest": order[-1], "shortest": order[0], "median": order[len(order) // 2]}[which])
+
+
+@pytest.mark.parametrize("cfg_i,kw,picks", [
+    (1, dict(), [(7, [0, 31])]),                                    # 32k x batch 8, one query head per KV head
+    (2, dict(), [(3, [5])]),                                        # 128k x batch 4, four query heads per KV head, group 32
+    (2, dict(n_q_heads=24, meta_fp8=True, n_sink=5), [(1, [2])]),   # the tcgen05 kernel, FP8 parameters, sinks
+    (3, dict(n_q_heads=2, n_kv_heads=2), [(0, [1])]),               # one sequence of 1M tokens (two heads instead of 32)
+    # configuration 3 as the benchmark runs it: 32 heads, so a CTA's run of the flat partition is 18.5 heads' worth of
+    # slots and head boundaries fall inside runs; head 1 starts inside a run, head 18 ends inside one
+    (3, dict(), [(0, [1, 18])]),
+    # configuration 4 in full: 64 ragged sequences (plan kernel + header in the workspace), 4-bit codes, group 64, window 256
+    (4, dict(), [("longest", [0]), ("shortest", [31]), ("median", [13])]),
 ])
-def test_full_size_sampled_pairs_match_oracle(cfg_i, kw, b, kv_heads):
+def test_full_size_sampled_pairs_match_oracle(cfg_i, kw, picks):
     from paper_2405_06219_b200 import binding as B
     w = workloads.configs()[cfg_i].scaled(**kw)
     n_steps = 3
@@ -65,40 +78,41 @@ def test_full_size_sampled_pairs_match_oracle(cfg_i, kw, b, kv_heads):
     lengths = w.lengths()
     gpu = B.SkvqCache.for_workload(w, int(lengths.max()) + n_steps + 64)
     prefill_like_the_benchmark(w, gpu)
-    oc = oracle_for_pairs(w, b, kv_heads, n_steps)
-    for s in range(n_steps):                                        # decode steps: one token per sequence
-        kn, vn = w.new_token("k", s), w.new_token("v", s)
+    new_tokens = [(w.new_token("k", s), w.new_token("v", s)) for s in range(n_steps)]
+    for kn, vn in new_tokens:                                       # decode steps: one token per sequence
         gpu.append(torch.from_numpy(kn).cuda(), torch.from_numpy(vn).cuda())
-        oc.append(np.ascontiguousarray(kn[b:b + 1][:, :, kv_heads]), np.ascontiguousarray(vn[b:b + 1][:, :, kv_heads]))
+    q = w.query(11)
+    out = gpu.attention(torch.from_numpy(q).cuda(), w.sm_scale, int(lengths.max()) + n_steps)      # default partition
     torch.cuda.synchronize()
-    L = int(lengths[b]) + n_steps
-    assert int(gpu.lengths[b]) == L and int(gpu.status[0]) == 0
-    lq, ns = max(L - w.window, 0), min(w.n_sink, max(L - w.window, 0))
+    assert np.isfinite(out.cpu().numpy()).all()
+    assert int(gpu.status[0]) == 0
 
     def bits(t):        # fp16 bit patterns, or one E4M3 byte per parameter (kept in a uint16 by the oracle)
         x = t.cpu().numpy()
         return x.astype(np.uint16) if w.meta_fp8 else x.view(np.uint16)
 
-    for i, hk in enumerate(kv_heads):
-        assert np.array_equal(gpu.k_codes[b, hk, ns:lq].cpu().numpy(), oc.k_codes[0, i, ns:lq]), f"k codes, head {hk}"
-        assert np.array_equal(gpu.v_codes[b, hk, ns:lq].cpu().numpy(), oc.v_codes[0, i, ns:lq]), f"v codes, head {hk}"
-        assert np.array_equal(bits(gpu.k_meta[b, hk, ns:lq]), oc.k_meta.view(np.uint16)[0, i, ns:lq]), f"k scale/zero, head {hk}"
-        assert np.array_equal(bits(gpu.v_meta[b, hk, ns:lq]), oc.v_meta.view(np.uint16)[0, i, ns:lq]), f"v scale/zero, head {hk}"
-        assert np.array_equal(gpu.k_sink[b, hk, :ns].cpu().numpy().view(np.uint16), oc.k_sink.view(np.uint16)[0, i, :ns])
-        if w.window:
-            slots = sorted({t % w.window for t in range(lq, L)})
-            assert np.array_equal(gpu.k_win[b, hk][slots].cpu().numpy().view(np.uint16), oc.k_win.view(np.uint16)[0, i][slots])
-            assert np.array_equal(gpu.v_win[b, hk][slots].cpu().numpy().view(np.uint16), oc.v_win.view(np.uint16)[0, i][slots])
-
-    q = w.query(11)
-    out = gpu.attention(torch.from_numpy(q).cuda(), w.sm_scale, int(lengths.max()) + n_steps)      # default partition
-    torch.cuda.synchronize()
-    q_heads = [hk * rep + r for hk in kv_heads for r in range(rep)]
-    want = oc.attention(np.ascontiguousarray(q[b:b + 1][:, q_heads]), w.sm_scale)[0]
-    got = out[b, q_heads].cpu().numpy().astype(np.float64)
-    assert np.isfinite(out.cpu().numpy()).all()
-    assert np.abs(got - want).max() <= ATTN_TOL
-    assert int(gpu.status[0]) == 0
+    for which, kv_heads in picks:
+        b = pick_sequence(lengths, which)
+        oc = oracle_for_pairs(w, b, kv_heads, n_steps)
+        for kn, vn in new_tokens:
+            oc.append(np.ascontiguousarray(kn[b:b + 1][:, :, kv_heads]), np.ascontiguousarray(vn[b:b + 1][:, :, kv_heads]))
+        L = int(lengths[b]) + n_steps
+        assert int(gpu.lengths[b]) == L
+        lq, ns = max(L - w.window, 0), min(w.n_sink, max(L - w.window, 0))
+        for i, hk in enumerate(kv_heads):
+            assert np.array_equal(gpu.k_codes[b, hk, ns:lq].cpu().numpy(), oc.k_codes[0, i, ns:lq]), f"k codes, head {hk}"
+            assert np.array_equal(gpu.v_codes[b, hk, ns:lq].cpu().numpy(), oc.v_codes[0, i, ns:lq]), f"v codes, head {hk}"
+            assert np.array_equal(bits(gpu.k_meta[b, hk, ns:lq]), oc.k_meta.view(np.uint16)[0, i, ns:lq]), f"k scale/zero, head {hk}"
+            assert np.array_equal(bits(gpu.v_meta[b, hk, ns:lq]), oc.v_meta.view(np.uint16)[0, i, ns:lq]), f"v scale/zero, head {hk}"
+            assert np.array_equal(gpu.k_sink[b, hk, :ns].cpu().numpy().view(np.uint16), oc.k_sink.view(np.uint16)[0, i, :ns])
+            if w.window:
+                slots = sorted({t % w.window for t in range(lq, L)})
+                assert np.array_equal(gpu.k_win[b, hk][slots].cpu().numpy().view(np.uint16), oc.k_win.view(np.uint16)[0, i][slots])
+                assert np.array_equal(gpu.v_win[b, hk][slots].cpu().numpy().view(np.uint16), oc.v_win.view(np.uint16)[0, i][slots])
+        q_heads = [hk * rep + r for hk in kv_heads for r in range(rep)]
+        want = oc.attention(np.ascontiguousarray(q[b:b + 1][:, q_heads]), w.sm_scale)[0]
+        got = out[b, q_heads].cpu().numpy().astype(np.float64)
+        assert np.abs(got - want).max() <= ATTN_TOL, f"sequence {b} (length {L}), KV heads {kv_heads}"
 
 
 @pytest.mark.parametrize("kw", [

@@ -241,6 +241,44 @@ def test_decode_loop_append_then_attend():
     assert_cache_bit_exact(gpu, ora)
 
 
+@pytest.mark.parametrize("cfg_i,kw", [
+    (0, dict(context=300, n_q_heads=2, n_kv_heads=2)),                       # one or two partition CTAs: room for the merge CTAs beside them
+    (2, dict(context=400, batch=2, n_q_heads=8, n_kv_heads=2)),              # grouped-query kernel
+    (2, dict(context=700, batch=1, n_q_heads=6, n_kv_heads=2)),              # tcgen05 kernel
+    (4, dict(context=600, batch=40, ragged=(1, 600), n_q_heads=2, n_kv_heads=2)),   # plan kernel in the chain, 4-bit
+])
+def test_back_to_back_steps_without_synchronisation(cfg_i, kw):
+    """Many decode steps (append one token, attend) enqueued with no host synchronisation in between, on contexts so
+    short that only a few partition CTAs exist and merge CTAs can be resident beside them: every step's output must
+    see that step's appended token in the window and that step's lengths (the kernels of a step are chained with
+    programmatic dependent launches, so this is the ordering guarantee of the chain)."""
+    w = small(cfg_i, **kw)
+    n_steps = 48
+    lengths = w.lengths()
+    n = int(lengths.max())
+    gpu, ora = both_caches(w, n + n_steps + 64)
+    k, v = w.prefill("k", n), w.prefill("v", n)
+    gpu.append(dev(k), dev(v), dev(lengths))
+    ora.append(k, v, lengths)
+    kn = [w.new_token("k", s) for s in range(n_steps)]
+    vn = [w.new_token("v", s) for s in range(n_steps)]
+    qs = [w.query(s) for s in range(n_steps)]
+    dk, dv, dq = dev(np.stack(kn)), dev(np.stack(vn)), dev(np.stack(qs))
+    outs = torch.zeros_like(dq)
+    args = gpu.attn_args(w.sm_scale, n + n_steps)
+    torch.cuda.synchronize()
+    for s in range(n_steps):
+        gpu.append(dk[s], dv[s])
+        B.skvq_decode_attention(gpu.cfg, gpu.struct, dq[s], outs[s], args)
+    torch.cuda.synchronize()
+    got = outs.cpu().numpy().astype(np.float64)
+    for s in range(n_steps):
+        ora.append(kn[s], vn[s])
+        want = ora.attention(qs[s], w.sm_scale)
+        assert np.abs(got[s] - want).max() <= ATTN_TOL, f"step {s}"
+    assert_cache_bit_exact(gpu, ora)
+
+
 @pytest.mark.parametrize("cfg_i,kw", [(1, dict(context=3000, batch=2, n_q_heads=4, n_kv_heads=4)),       # integer kernel
                                        (2, dict(context=2500, batch=2)),                                 # grouped-query kernel
                                        (2, dict(context=2500, batch=1, n_q_heads=24))])                  # tcgen05 kernel
@@ -324,3 +362,4 @@ def test_adversarial_values_stay_bit_exact():
     assert_cache_bit_exact(gpu, ora)
     got, want = attention_both(gpu, ora, w)
     assert np.isfinite(got).all()
+    assert np.abs(got - want).max() <= ATTN_TOL

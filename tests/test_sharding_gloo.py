@@ -22,7 +22,10 @@ def _worker(rank, world, port, q):
     tokens = float(w.lengths().sum())
     t, u = sharding.reduce_job(10.0 + rank, tokens)
     first = w.tokens("k", 0, 0, 4).astype(np.float32).sum()
-    q.put((rank, t, u, float(first), list(sharding.split_sequences(5, rank, world))))
+    passes = sharding.reduce_max_list([1.0 + rank, 5.0 - rank, 2.0])      # per-pass timings: the slowest rank each
+    est = sharding.reduce_max(3.0 * (rank + 1))
+    job = sharding.reduce_sum(tokens)
+    q.put((rank, t, u, float(first), list(sharding.split_sequences(5, rank, world)), passes, est, job))
     dist.barrier()
     dist.destroy_process_group()
 
@@ -42,9 +45,16 @@ def test_two_ranks_reduce_max_time_and_sum_units():
     assert [r[2] for r in res] == [256.0, 256.0]               # 2 ranks x 2 sequences x 64 tokens
     assert res[0][3] != res[1][3]                              # ranks draw different data
     assert res[0][4] == [0, 1, 2] and res[1][4] == [3, 4]      # contiguous sequence blocks cover the batch
+    assert res[0][5] == res[1][5] == [2.0, 5.0, 2.0]           # element-wise max over the ranks
+    assert res[0][6] == res[1][6] == 6.0
+    assert res[0][7] == res[1][7] == 256.0
 
 
 def test_single_process_is_identity():
     assert sharding.reduce_job(3.5, 7.0) == (3.5, 7.0)
-    assert sharding.rank_workload(workloads.configs()[0], 0, 1) is workloads.configs()[0] or True
+    w = workloads.configs()[0]
+    assert sharding.rank_workload(w, 0, 1) is w
+    assert sharding.rank_workload(w, 1, 2).seed == w.seed + 1000
+    assert sharding.reduce_max_list([1.0, 2.0]) == [1.0, 2.0] and sharding.reduce_max(4.0) == 4.0
+    assert sharding.reduce_sum(9.0) == 9.0
     assert [list(sharding.split_sequences(8, r, 4)) for r in range(4)] == [[0, 1], [2, 3], [4, 5], [6, 7]]
