@@ -47,6 +47,7 @@ L2_BYTES = 126 * 1024 * 1024
 MIN_TIMED_MS = 500.0          # the timed passes of the headline configuration cover at least this much device time
 MIN_TIMED_MS_OTHER = 300.0
 MAX_TIMED_STEPS = 4096        # ... but never more steps than this (each step appends a token to the cache)
+MAX_E2E_STEPS = 1024
 # DRAM bytes (read + write) per launch of the partition kernel from ncu captures of reduced cases, scaled to the full
 # configuration by the tokens streamed (traffic is proportional to them); None where the kernel has changed since.
 NCU_TRAFFIC_BYTES = {1: None, 2: None, 3: None, 4: None}
@@ -66,7 +67,7 @@ def measured_peak():
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed regions run."""
     Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap,power.draw")
 
     def __init__(self, gpu_id: str):
         self.index, self.samples, self._stop, self._t = gpu_id, [], threading.Event(), None
@@ -96,26 +97,29 @@ class ClockSampler:
         windows (all samples when none is given or none falls inside)."""
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
-        def inside(s):
-            return any(s[0] >= a and s[1] <= b for a, b in windows)
+        def inside(s):      # the query overlapped a timed pass
+            return any(s[1] >= a and s[0] <= b for a, b in windows)
         chosen = [s for s in self.samples if windows and inside(s)]
-        scope = "inside the timed passes"
+        scope = "samples overlapping the timed passes"
         if not chosen:
             chosen, scope = self.samples, "whole run (no sample fell inside a timed pass)"
-        mhz, mx, reasons = [], None, set()
+        mhz, mx, reasons, watts = [], None, set(), []
         for _, _, s in chosen:
             if len(s) < 6:
                 continue
             try:
                 mhz.append(float(s[0]))
                 mx = float(s[1])
+                if len(s) > 6:
+                    watts.append(float(s[6]))
             except ValueError:
                 continue
             for n, v in zip(names, s[2:6]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
         return {"sm_mhz": statistics.median(mhz) if mhz else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
-                "samples": len(mhz), "scope": scope}
+                "samples": len(mhz), "scope": scope, "sm_mhz_min": min(mhz) if mhz else None,
+                "power_w": statistics.median(watts) if watts else None}
 
 
 # ---------------------------------------------------------------------------------------------- the oracle's sample
@@ -254,7 +258,7 @@ def run_config(cfg_i, w0, args, env, main):
     rank, world, local_rank, clocks = env["rank"], env["world"], env["local_rank"], env["clocks"]
     w = sharding.rank_workload(w0, rank, world)
     K, W_ = args.steps, args.warmup
-    extra = W_ + MAX_TIMED_STEPS + 4 * K + 64
+    extra = 3 * W_ + MAX_TIMED_STEPS + MAX_E2E_STEPS + 5 * K + 64      # every step of every pass appends a token
     lengths0 = w.lengths()
     dev = torch.device("cuda", local_rank) if world > 1 else None
 
@@ -426,7 +430,7 @@ def run_config(cfg_i, w0, args, env, main):
         for i in range(W_):
             host_step(i)
         e2e_ms, e2e_tok = [], []
-        n_e2e = int(min(max(1, -(-(MIN_TIMED_MS / 2) // max(est * 1.3, 1e-3))), max(1, 1024 // K)))
+        n_e2e = int(min(max(1, -(-(MIN_TIMED_MS / 2) // max(est * 1.3, 1e-3))), max(1, MAX_E2E_STEPS // K)))
         for _ in range(n_e2e):
             before = state["appended"]
             barrier()
@@ -468,7 +472,7 @@ def run_config(cfg_i, w0, args, env, main):
                    "parallelism": f"replica per GPU x{world}" if world > 1 else "single GPU"},
         "value": value, "unit": UNIT, "steps": K, "passes": len(pass_ms),
         "ms_per_step": med_ms / K, "ms_per_step_min": min(pass_ms) / K, "ms_per_step_max": max(pass_ms) / K,
-        "timed_ms_total": sum(pass_ms),
+        "timed_ms_total": sum(pass_ms), "pass_ms_per_step": [round(x / K, 5) for x in pass_ms],
         "step_bytes_per_s_gb": alg_bytes / (med_ms / K * 1e-3) / 1e9,
         "clocks": clocks.summary(windows),
         "gpu_launches": int(launches),

@@ -276,8 +276,10 @@ __global__ void plan_kernel(AttnArgs a)
 }
 
 // One CTA per (query head, sequence): walks the fp16 rows -- the attention sinks that have left the window, then
-// the window (thread = token for the scores, 16 lanes per row for P.V) -- then combines that with the split
-// partials of the quantized prefix.
+// the window -- and then combines that with the split partials of the quantized prefix.  Every row is read with
+// coalesced 16-byte loads (16 lanes per 256-byte row, two rows per warp instruction), keys and values alike; a lane
+// keeps its eight channels of the permuted query and of the running value sums in registers.
+constexpr int kMergeTile = 64;      // rows per pass: 4 warps x 8 row pairs, all 16 loads of a lane in flight at once
 __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
 {
     const int hq = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -289,8 +291,8 @@ __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
     // bookkeeping kernels in front of the partition kernel have completed and their writes (lengths, ring, sinks) are visible.
     const int L = a.c.lengths[b];
     const int Lq = max(L - W, 0);
-    __shared__ float sq[kHeadDim];
-    __shared__ float sp[kThreads];
+    __shared__ __align__(16) float sq[kHeadDim];
+    __shared__ float sp[kMergeTile];
     __shared__ float sred[kThreads / 32];
     __shared__ __align__(16) int hdr_sh[kPlanSmemInts];
     if (a.plan.in_kernel && warp == 0)      // the same header the partition CTAs derived; published by the barriers below
@@ -299,81 +301,72 @@ __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
     sq[tid] = __half2float(a.q[((size_t)b * s.Hq + hq) * kHeadDim + (a.c.reorder_k[(size_t)hk * kHeadDim + tid] & (kHeadDim - 1))]) *
               a.scale_log2;
     __syncthreads();
-    // P.V layout: a warp instruction reads two rows (16 lanes x 8 channels each); warp w takes row pairs w, w+4, ...
     __shared__ __align__(16) float sacc[kThreads / 32][kHeadDim];      // written with 16-byte stores
+    const int vsub = lane >> 4, vchunk = lane & 15;                    // row of the pair, 16-byte piece of the row
+    float q8[8];
+    {
+        const float4 qa = *reinterpret_cast<const float4 *>(&sq[8 * vchunk]), qb = *reinterpret_cast<const float4 *>(&sq[8 * vchunk + 4]);
+        q8[0] = qa.x; q8[1] = qa.y; q8[2] = qa.z; q8[3] = qa.w; q8[4] = qb.x; q8[5] = qb.y; q8[6] = qb.z; q8[7] = qb.w;
+    }
     float m_run = -CUDART_INF_F, l_thread = 0.f;
     float a8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-    const int vsub = lane >> 4, vchunk = lane & 15;
     // Online softmax over the fp16 rows of tokens [t_begin, t_end): row of token t = t % ring (ring > 0) or t.
     auto walk = [&](const __half *k_rows, const __half *v_rows, int t_begin, int t_end, int ring) {
-    for (int tile0 = t_begin; tile0 < t_end; tile0 += kThreads) {
-        const int t = tile0 + tid;
-        const bool valid = t < t_end;
-        float sc = valid ? 0.f : -CUDART_INF_F;
-        uint4 vu[kThreads / 8];
-        if (!valid) {
+    for (int tile0 = t_begin; tile0 < t_end; tile0 += kMergeTile) {
+        // this lane's rows of the tile: tt = 2 * (warp + 4 i) + vsub, i = 0..7
+        const int tt0 = 2 * warp + vsub;
+        int r0 = tile0 + tt0;
+        if (ring) r0 %= ring;
+        uint4 ku[kMergeTile / 8], vu[kMergeTile / 8];
+        int rows[kMergeTile / 8];
 #pragma unroll
-            for (int i = 0; i < kThreads / 8; ++i) {
-                const int tt = 8 * i + 2 * warp + vsub;
-                vu[i] = make_uint4(0u, 0u, 0u, 0u);
-                if (tile0 + tt < t_end)
-                    vu[i] = __ldg(reinterpret_cast<const uint4 *>(v_rows + (size_t)(ring ? (tile0 + tt) % ring : (tile0 + tt)) * kHeadDim) + vchunk);
-            }
+        for (int i = 0; i < kMergeTile / 8; ++i) {
+            int r = r0 + 8 * i;
+            if (ring) r = ring >= kMergeTile ? (r >= ring ? r - ring : r) : r % ring;
+            rows[i] = r;
+            ku[i] = make_uint4(0u, 0u, 0u, 0u);
+            if (tile0 + tt0 + 8 * i < t_end) ku[i] = __ldg(reinterpret_cast<const uint4 *>(k_rows + (size_t)r * kHeadDim) + vchunk);
         }
-        if (valid) {
-            const uint4 *row = reinterpret_cast<const uint4 *>(k_rows + (size_t)(ring ? t % ring : t) * kHeadDim);
-            uint4 u[kHeadDim / 8];
+        // the value rows do not depend on the scores: fetch them behind the key rows
 #pragma unroll
-            for (int j8 = 0; j8 < kHeadDim / 8; ++j8) u[j8] = __ldg(row + j8);      // all 16 loads in flight
-            // the value rows this thread will need do not depend on the scores: fetch them behind the key rows
-#pragma unroll
-            for (int i = 0; i < kThreads / 8; ++i) {
-                const int tt = 8 * i + 2 * warp + vsub;
-                vu[i] = make_uint4(0u, 0u, 0u, 0u);
-                if (tile0 + tt < t_end)
-                    vu[i] = __ldg(reinterpret_cast<const uint4 *>(v_rows + (size_t)(ring ? (tile0 + tt) % ring : (tile0 + tt)) * kHeadDim) + vchunk);
-            }
-#pragma unroll
-            for (int j8 = 0; j8 < kHeadDim / 8; ++j8) {
-                const __half2 *h2 = reinterpret_cast<const __half2 *>(&u[j8]);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const float2 kv = __half22float2(h2[i]);
-                    sc = fmaf(sq[8 * j8 + 2 * i], kv.x, fmaf(sq[8 * j8 + 2 * i + 1], kv.y, sc));
-                }
-            }
+        for (int i = 0; i < kMergeTile / 8; ++i) {
+            vu[i] = make_uint4(0u, 0u, 0u, 0u);
+            if (tile0 + tt0 + 8 * i < t_end) vu[i] = __ldg(reinterpret_cast<const uint4 *>(v_rows + (size_t)rows[i] * kHeadDim) + vchunk);
         }
-        const float wm = warp_max(sc);
-        if (lane == 0) sred[warp] = wm;
+#pragma unroll
+        for (int i = 0; i < kMergeTile / 8; ++i) {
+            const __half2 *h2 = reinterpret_cast<const __half2 *>(&ku[i]);
+            float d = 0.f;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float2 kv = __half22float2(h2[e]);
+                d = fmaf(q8[2 * e], kv.x, fmaf(q8[2 * e + 1], kv.y, d));
+            }
+#pragma unroll
+            for (int msk = 8; msk > 0; msk >>= 1) d += __shfl_xor_sync(0xffffffffu, d, msk);      // over the 16 lanes of the row
+            if (vchunk == 0) sp[tt0 + 8 * i] = (tile0 + tt0 + 8 * i < t_end) ? d : -CUDART_INF_F;
+        }
         __syncthreads();
-        float tm = sred[0];
-#pragma unroll
-        for (int w = 1; w < kThreads / 32; ++w) tm = fmaxf(tm, sred[w]);
+        const float tm = warp_max(fmaxf(sp[lane], sp[lane + 32]));      // every warp finds the same tile maximum
         const float m_new = fmaxf(m_run, tm);               // finite: the tile has a valid token
         const float corr = exp2f(m_run - m_new);            // exp2(-inf) = 0 on the first tile
-        const float p = valid ? exp2f(sc - m_new) : 0.f;
-        sp[tid] = p;
-        l_thread = l_thread * corr + p;
+        l_thread *= corr;
         m_run = m_new;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) a8[i] *= corr;
-        __syncthreads();
-        const int n_tok = min(kThreads, t_end - tile0);
+        for (int e = 0; e < 8; ++e) a8[e] *= corr;
 #pragma unroll
-        for (int i = 0; i < kThreads / 8; ++i) {            // 16 independent 16-byte loads per thread
-            const int tt = 8 * i + 2 * warp + vsub;
-            if (tt < n_tok) {
-                const __half2 *h2 = reinterpret_cast<const __half2 *>(&vu[i]);
-                const float pt = sp[tt];
+        for (int i = 0; i < kMergeTile / 8; ++i) {
+            const float pt = exp2f(sp[tt0 + 8 * i] - m_new);      // 0 past the end (score -inf); the 16 lanes of a row agree
+            if (vchunk == 0) l_thread += pt;                      // once per row
+            const __half2 *h2 = reinterpret_cast<const __half2 *>(&vu[i]);
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const float2 vv = __half22float2(h2[e]);
-                    a8[2 * e] = fmaf(pt, vv.x, a8[2 * e]);
-                    a8[2 * e + 1] = fmaf(pt, vv.y, a8[2 * e + 1]);
-                }
+            for (int e = 0; e < 4; ++e) {
+                const float2 vv = __half22float2(h2[e]);
+                a8[2 * e] = fmaf(pt, vv.x, a8[2 * e]);
+                a8[2 * e + 1] = fmaf(pt, vv.y, a8[2 * e + 1]);
             }
         }
-        __syncthreads();   // sp and sred are rewritten by the next tile
+        __syncthreads();   // sp is rewritten by the next tile
     }
     };
     // attention sinks that have left the window (fp16 copies), then the window itself

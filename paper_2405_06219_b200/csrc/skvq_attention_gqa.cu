@@ -465,17 +465,28 @@ __global__ void __launch_bounds__(kThreads, 2) partition_gqa_kernel(MmaArgs a)
             hmax_bits = mx & 0xFFFFu;                          // scales are non-negative: fp16 order = integer order
         }
         bool moved = hmax_bits >= h_thr || ++tiles_since_fold * kTileTok >= 32768;
+        const bool whole = n_valid == kTileTok && n_skip == 0;      // all but the first and last tiles of a segment
         float arg[4][2];
         float amax = -CUDART_INF_F;
+        if (whole) {
 #pragma unroll
-        for (int mt = 0; mt < 4; ++mt)
+            for (int mt = 0; mt < 4; ++mt)
 #pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                const int tok_in = 32 * (mt >> 1) + own[2 * (mt & 1) + e];
-                const bool valid = tok_in < n_valid && tok_in >= n_skip;
-                arg[mt][e] = valid ? fmaf(sraw[mt][e], cs, -m_ref) : -CUDART_INF_F;
-                amax = fmaxf(amax, arg[mt][e]);
-            }
+                for (int e = 0; e < 2; ++e) {
+                    arg[mt][e] = fmaf(sraw[mt][e], cs, -m_ref);
+                    amax = fmaxf(amax, arg[mt][e]);
+                }
+        } else {
+#pragma unroll
+            for (int mt = 0; mt < 4; ++mt)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const int tok_in = 32 * (mt >> 1) + own[2 * (mt & 1) + e];
+                    const bool valid = tok_in < n_valid && tok_in >= n_skip;
+                    arg[mt][e] = valid ? fmaf(sraw[mt][e], cs, -m_ref) : -CUDART_INF_F;
+                    amax = fmaxf(amax, arg[mt][e]);
+                }
+        }
         moved |= amax > kRefSlack;
         if (__any_sync(0xffffffffu, moved)) {
             // Raise the reference of every head to its running maximum (and the bound on h); fold what was accumulated.
