@@ -20,10 +20,13 @@
  *   - attention: fp64 everywhere; dequantized values are never rounded.
  *
  * Layout (all row-major, host memory)
- *   codes  uint8  [B][Hkv][cap_q][D*bits/8]   code j of a row sits in bits
- *                                             [(j*bits) mod 8, +bits) of byte (j*bits)/8
- *   meta   uint16 [B][Hkv][cap_q][D/G][2]     {h, z} as fp16 bit patterns; in FP8 mode the
- *                                             E4M3 byte of each in the low 8 bits
+ *   codes  uint8  [B][Hkv][cap_q][D*bits/8]   a row is a little-endian bit stream: code j
+ *                                             sits in bits [j*bits, (j+1)*bits) of the row, i.e.
+ *                                             from bit (j*bits) mod 8 of byte (j*bits)/8 on
+ *                                             (a 3-bit code may run into the next byte)
+ *   meta   uint16 [B][Hkv][cap_q][ng][2]      {h, z} as fp16 bit patterns; in FP8 mode the
+ *                                             E4M3 byte of each in the low 8 bits; ng groups
+ *                                             per row (D/G equal ones, or the given boundaries)
  *   win    uint16 [B][Hkv][W][D]              ring: token t lives in slot t mod W,
  *                                             channels already in reordered order
  *   lengths int32 [B]                         tokens appended so far
@@ -33,7 +36,10 @@
  * single-append == bulk-append, brute-force attention, convexity, q = 0 mean,
  * attention sinks (exact rows, brute force over the three segments, all-sink
  * case against a library attention), FP8 E4M3 conversions against a library's
- * (all 256 bytes, random and midpoint inputs) and the paper's 2.5-bit average.
+ * (all 256 bytes, random and midpoint inputs) and the paper's 2.5-bit average;
+ * unequal groups (equal boundaries reproduce the equal-group result, one-channel
+ * groups are lossless, parameters recomputed per boundary slice), 3-bit codes
+ * (golden stream bytes, nearest level, the paper's 3.25-bit average).
  * End-to-end accuracy versus the paper's benchmark tables: parity unpinned (the
  * datasets and model weights those tables need are not available).
  */
@@ -139,22 +145,28 @@ uint8_t orc_f32_to_e4m3(float f)
 /*
  * Clipped dynamic asymmetric quantization of one already-reordered row
  * (Sec. 3.1 uniform quantizer, Eq. 2, and clipping_quant of Algorithm 1):
- * per group of G consecutive channels take min and max, multiply both by the
+ * per group of consecutive channels take min and max, multiply both by the
  * group's clip factor, derive scale h and zero point z, round both to fp16
  * (to FP8 E4M3 if meta_fp8), then code = clamp(rint((x - z) / h), 0, 2^bits - 1).
+ * Groups (split_groups(X, group_indices) of Algorithm 1; Sec. 3.1: channels
+ * with similar ranges share a group, so after the reorder a group is a run of
+ * consecutive channels and the runs need not have the same length, Sec. 4.2):
+ * group g covers channels [bounds[g], bounds[g+1]) when bounds is given
+ * (bounds[0] = 0, bounds[ng] = D), else [g*G, (g+1)*G) with ng = D/G.
  * A zero is canonicalised to +0 before it is used so that the sign of a zero
  * minimum or maximum (which depends on the order elements are visited) cannot
  * leak into the stored parameters.
  */
 void orc_quantize_reordered_row(const uint16_t *xr, const float *alpha, int D, int G, int bits,
-                                uint8_t *codes, uint16_t *meta, int meta_fp8)
+                                uint8_t *codes, uint16_t *meta, int meta_fp8, const int32_t *bounds, int ng)
 {
     const int qmax = (1 << bits) - 1;
-    const int ng = D / G;
+    if (!bounds) ng = D / G;
     memset(codes, 0, (size_t)(D * bits / 8));
     for (int g = 0; g < ng; ++g) {
+        const int j0 = bounds ? bounds[g] : g * G, j1 = bounds ? bounds[g + 1] : (g + 1) * G;
         float mn = INFINITY, mx = -INFINITY;
-        for (int j = g * G; j < (g + 1) * G; ++j) {
+        for (int j = j0; j < j1; ++j) {
             float v = orc_f16_to_f32(xr[j]);
             if (v < mn) mn = v;
             if (v > mx) mx = v;
@@ -178,7 +190,7 @@ void orc_quantize_reordered_row(const uint16_t *xr, const float *alpha, int D, i
             meta[2 * g + 0] = h16;
             meta[2 * g + 1] = z16;
         }
-        for (int j = g * G; j < (g + 1) * G; ++j) {
+        for (int j = j0; j < j1; ++j) {
             int c = 0;
             if (hf != 0.0f) {
                 float x = orc_f16_to_f32(xr[j]);
@@ -190,22 +202,28 @@ void orc_quantize_reordered_row(const uint16_t *xr, const float *alpha, int D, i
             }
             int bit = j * bits;
             codes[bit >> 3] |= (uint8_t)(c << (bit & 7));
+            if ((bit & 7) + bits > 8) codes[(bit >> 3) + 1] |= (uint8_t)(c >> (8 - (bit & 7)));   /* the part in the next byte */
         }
     }
 }
 
-/* Code j of a packed row. */
+/* Code j of a packed row (a little-endian bit stream of bits-wide fields). */
 static int orc_code_at(const uint8_t *codes, int j, int bits)
 {
     int bit = j * bits;
-    return (codes[bit >> 3] >> (bit & 7)) & ((1 << bits) - 1);
+    int v = codes[bit >> 3] >> (bit & 7);
+    if ((bit & 7) + bits > 8) v |= (int)codes[(bit >> 3) + 1] << (8 - (bit & 7));
+    return v & ((1 << bits) - 1);
 }
 
-/* Dequantize one row to fp64 without rounding: x^ = h*c + z. */
-void orc_dequant_row(const uint8_t *codes, const uint16_t *meta, int D, int G, int bits, int meta_fp8, double *out)
+/* Dequantize one row to fp64 without rounding: x^ = h*c + z with the parameters of the channel's group. */
+void orc_dequant_row(const uint8_t *codes, const uint16_t *meta, int D, int G, int bits, int meta_fp8, double *out,
+                     const int32_t *bounds, int ng)
 {
     for (int j = 0; j < D; ++j) {
-        int g = j / G;
+        int g = 0;
+        if (bounds) { while (g + 1 < ng && j >= bounds[g + 1]) ++g; }
+        else g = j / G;
         double h = (double)(meta_fp8 ? orc_e4m3_to_f32((uint8_t)meta[2 * g + 0]) : orc_f16_to_f32(meta[2 * g + 0]));
         double z = (double)(meta_fp8 ? orc_e4m3_to_f32((uint8_t)meta[2 * g + 1]) : orc_f16_to_f32(meta[2 * g + 1]));
         out[j] = h * (double)orc_code_at(codes, j, bits) + z;
@@ -214,13 +232,14 @@ void orc_dequant_row(const uint8_t *codes, const uint16_t *meta, int D, int G, i
 
 /* Reorder then quantize n independent rows (no cache state); for unit tests. */
 void orc_quantize_rows(const uint16_t *x, int n, const int32_t *idx, const float *alpha, int D, int G,
-                       int bits, int meta_fp8, uint8_t *codes, uint16_t *meta)
+                       int bits, int meta_fp8, uint8_t *codes, uint16_t *meta, const int32_t *bounds, int ng)
 {
     uint16_t *tmp = (uint16_t *)malloc(sizeof(uint16_t) * (size_t)D);
+    if (!bounds) ng = D / G;
     for (int r = 0; r < n; ++r) {
         orc_reorder_row(x + (size_t)r * D, idx, D, tmp);
         orc_quantize_reordered_row(tmp, alpha, D, G, bits, codes + (size_t)r * (D * bits / 8),
-                                   meta + (size_t)r * (D / G) * 2, meta_fp8);
+                                   meta + (size_t)r * ng * 2, meta_fp8, bounds, ng);
     }
     free(tmp);
 }
@@ -239,6 +258,8 @@ typedef struct {
     int n_sink;                           /* first n_sink positions are never quantized (Sec. 3.2, filter rules) */
     uint16_t *k_sink, *v_sink;            /* fp16 bits [B][Hkv][n_sink][D], reordered channel order */
     int meta_fp8;                         /* scale and zero point stored as FP8 E4M3 instead of fp16 */
+    int ng;                               /* groups per row: D/G, or the number of boundary intervals */
+    const int32_t *bounds_k, *bounds_v;   /* [Hkv][ng+1] group boundaries in reordered channel order, or NULL = equal groups of G */
 } orc_cache;
 
 static size_t orc_row_index(const orc_cache *c, int b, int h, int t, int rows)
@@ -262,7 +283,7 @@ static size_t orc_row_index(const orc_cache *c, int b, int h, int t, int rows)
  */
 int orc_append(orc_cache *c, const uint16_t *k, const uint16_t *v, const int32_t *n_new, int n_stride)
 {
-    const int D = c->D, W = c->W, ng = c->D / c->G;
+    const int D = c->D, W = c->W, ng = c->ng;
     int status = 0;
     for (int b = 0; b < c->B; ++b) {
         const int L0 = c->lengths[b];
@@ -297,10 +318,12 @@ int orc_append(orc_cache *c, const uint16_t *k, const uint16_t *v, const int32_t
                 size_t r = orc_row_index(c, b, h, t, c->cap_q);
                 orc_quantize_reordered_row(rowk, c->alpha_k + (size_t)h * ng, D, c->G, c->k_bits,
                                            c->k_codes + r * (size_t)(D * c->k_bits / 8),
-                                           c->k_meta + r * (size_t)ng * 2, c->meta_fp8);
+                                           c->k_meta + r * (size_t)ng * 2, c->meta_fp8,
+                                           c->bounds_k ? c->bounds_k + (size_t)h * (ng + 1) : NULL, ng);
                 orc_quantize_reordered_row(rowv, c->alpha_v + (size_t)h * ng, D, c->G, c->v_bits,
                                            c->v_codes + r * (size_t)(D * c->v_bits / 8),
-                                           c->v_meta + r * (size_t)ng * 2, c->meta_fp8);
+                                           c->v_meta + r * (size_t)ng * 2, c->meta_fp8,
+                                           c->bounds_v ? c->bounds_v + (size_t)h * (ng + 1) : NULL, ng);
             }
             /* 2. the new tokens that remain inside the window go to the ring */
             int first_kept = q_end > L0 ? q_end : L0;
@@ -332,7 +355,7 @@ int orc_append(orc_cache *c, const uint16_t *k, const uint16_t *v, const int32_t
  */
 void orc_attention(const orc_cache *c, int Hq, const uint16_t *q, double sm_scale, double *out)
 {
-    const int D = c->D, W = c->W, ng = c->D / c->G;
+    const int D = c->D, W = c->W, ng = c->ng;
     const int rep = Hq / c->Hkv;
 #pragma omp parallel for collapse(2) schedule(dynamic, 1)
     for (int b = 0; b < c->B; ++b) {
@@ -359,7 +382,8 @@ void orc_attention(const orc_cache *c, int Hq, const uint16_t *q, double sm_scal
                 } else if (t < Lq) {
                     size_t r = orc_row_index(c, b, hk, t, c->cap_q);
                     orc_dequant_row(c->k_codes + r * (size_t)(D * c->k_bits / 8),
-                                    c->k_meta + r * (size_t)ng * 2, D, c->G, c->k_bits, c->meta_fp8, row);
+                                    c->k_meta + r * (size_t)ng * 2, D, c->G, c->k_bits, c->meta_fp8, row,
+                                    c->bounds_k ? c->bounds_k + (size_t)hk * (ng + 1) : NULL, ng);
                 } else {
                     size_t w = orc_row_index(c, b, hk, t % W, W) * (size_t)D;
                     for (int j = 0; j < D; ++j) row[j] = (double)orc_f16_to_f32(c->k_win[w + j]);
@@ -381,7 +405,8 @@ void orc_attention(const orc_cache *c, int Hq, const uint16_t *q, double sm_scal
                 } else if (t < Lq) {
                     size_t r = orc_row_index(c, b, hk, t, c->cap_q);
                     orc_dequant_row(c->v_codes + r * (size_t)(D * c->v_bits / 8),
-                                    c->v_meta + r * (size_t)ng * 2, D, c->G, c->v_bits, c->meta_fp8, row);
+                                    c->v_meta + r * (size_t)ng * 2, D, c->G, c->v_bits, c->meta_fp8, row,
+                                    c->bounds_v ? c->bounds_v + (size_t)hk * (ng + 1) : NULL, ng);
                 } else {
                     size_t w = orc_row_index(c, b, hk, t % W, W) * (size_t)D;
                     for (int j = 0; j < D; ++j) row[j] = (double)orc_f16_to_f32(c->v_win[w + j]);

@@ -41,6 +41,7 @@ class _Cache(ctypes.Structure):
         ("alpha_k", ctypes.c_void_p), ("alpha_v", ctypes.c_void_p),
         ("n_sink", ctypes.c_int), ("k_sink", ctypes.c_void_p), ("v_sink", ctypes.c_void_p),
         ("meta_fp8", ctypes.c_int),
+        ("ng", ctypes.c_int), ("bounds_k", ctypes.c_void_p), ("bounds_v", ctypes.c_void_p),
     ]
 
 
@@ -55,10 +56,10 @@ def lib():
         _lib.orc_quantize_rows.restype = None
         _lib.orc_quantize_rows.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p,
                                            ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_void_p,
-                                           ctypes.c_void_p]
+                                           ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int]
         _lib.orc_dequant_row.restype = None
         _lib.orc_dequant_row.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
-                                         ctypes.c_int, ctypes.c_int, ctypes.c_void_p]
+                                         ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int]
         _lib.orc_e4m3_to_f32.restype = ctypes.c_float
         _lib.orc_e4m3_to_f32.argtypes = [ctypes.c_uint8]
         _lib.orc_f32_to_e4m3.restype = ctypes.c_uint8
@@ -98,33 +99,49 @@ def e4m3_bits_to_f32(b: int) -> float:
     return float(lib().orc_e4m3_to_f32(ctypes.c_uint8(b)))
 
 
-def quantize_rows(x: np.ndarray, idx: np.ndarray, alpha: np.ndarray, bits: int, group: int, meta_fp8: bool = False):
+def _bounds(bounds, D):
+    """Group boundaries as a contiguous int32 array [ng+1] (0 ... D, strictly increasing), or None."""
+    if bounds is None:
+        return None
+    b = np.ascontiguousarray(bounds, dtype=np.int32)
+    assert b.ndim == 1 and b[0] == 0 and b[-1] == D and np.all(np.diff(b) > 0)
+    return b
+
+
+def quantize_rows(x: np.ndarray, idx: np.ndarray, alpha: np.ndarray, bits: int, group: int, meta_fp8: bool = False,
+                  bounds=None):
     """Reorder + clipped group quantization of independent rows.
 
-    x: float16 [n, D] in original channel order; idx: int32 [D]; alpha: float32 [D/group].
-    Returns (codes uint8 [n, D*bits/8], meta float16 [n, D/group, 2] = {h, z}); with meta_fp8 the
-    meta array holds the E4M3 byte of h and z as uint16 [n, D/group, 2].
+    x: float16 [n, D] in original channel order; idx: int32 [D]; alpha: float32 [ng].  Groups are D/group equal runs of
+    ``group`` reordered channels, or, with ``bounds`` (int [ng+1], 0 ... D), the runs [bounds[g], bounds[g+1]).
+    Returns (codes uint8 [n, D*bits/8], meta float16 [n, ng, 2] = {h, z}); with meta_fp8 the
+    meta array holds the E4M3 byte of h and z as uint16 [n, ng, 2].
     """
     x = np.ascontiguousarray(x, dtype=np.float16)
     n, D = x.shape
     idx = np.ascontiguousarray(idx, dtype=np.int32)
     alpha = np.ascontiguousarray(alpha, dtype=np.float32)
-    assert idx.shape == (D,) and alpha.shape == (D // group,)
+    b = _bounds(bounds, D)
+    ng = D // group if b is None else len(b) - 1
+    assert idx.shape == (D,) and alpha.shape == (ng,) and (D * bits) % 8 == 0
     codes = np.zeros((n, D * bits // 8), dtype=np.uint8)
-    meta = np.zeros((n, D // group, 2), dtype=np.uint16 if meta_fp8 else np.float16)
-    lib().orc_quantize_rows(_ptr(x), n, _ptr(idx), _ptr(alpha), D, group, bits, int(meta_fp8), _ptr(codes), _ptr(meta))
+    meta = np.zeros((n, ng, 2), dtype=np.uint16 if meta_fp8 else np.float16)
+    lib().orc_quantize_rows(_ptr(x), n, _ptr(idx), _ptr(alpha), D, group, bits, int(meta_fp8), _ptr(codes), _ptr(meta),
+                            None if b is None else _ptr(b), ng)
     return codes, meta
 
 
-def dequant_rows(codes: np.ndarray, meta: np.ndarray, bits: int, group: int, meta_fp8: bool = False) -> np.ndarray:
+def dequant_rows(codes: np.ndarray, meta: np.ndarray, bits: int, group: int, meta_fp8: bool = False, bounds=None) -> np.ndarray:
     """fp64 dequantization x^ = h*c + z of packed rows (no rounding)."""
     codes = np.ascontiguousarray(codes, dtype=np.uint8)
     meta = np.ascontiguousarray(meta, dtype=np.uint16 if meta_fp8 else np.float16)
     n = codes.shape[0]
     D = codes.shape[1] * 8 // bits
+    b = _bounds(bounds, D)
     out = np.zeros((n, D), dtype=np.float64)
     for r in range(n):
-        lib().orc_dequant_row(_ptr(codes[r]), _ptr(meta[r]), D, group, bits, int(meta_fp8), _ptr(out[r]))
+        lib().orc_dequant_row(_ptr(codes[r]), _ptr(meta[r]), D, group, bits, int(meta_fp8), _ptr(out[r]),
+                              None if b is None else _ptr(b), meta.shape[1])
     return out
 
 
@@ -132,10 +149,19 @@ class OracleCache:
     """Host-side SKVQ cache in the canonical layout, driven by the C oracle."""
 
     def __init__(self, batch, n_q_heads, n_kv_heads, head_dim, k_bits, v_bits, group_size, window,
-                 max_tokens, reorder_k, reorder_v, alpha_k, alpha_v, n_sink=0, meta_fp8=False):
+                 max_tokens, reorder_k, reorder_v, alpha_k, alpha_v, n_sink=0, meta_fp8=False, bounds_k=None,
+                 bounds_v=None):
         self.B, self.Hq, self.Hkv, self.D = batch, n_q_heads, n_kv_heads, head_dim
         self.k_bits, self.v_bits, self.G, self.W = k_bits, v_bits, group_size, window
         self.ng = head_dim // group_size
+        # unequal groups: boundaries [Hkv][ng+1] in reordered channel order (None = equal runs of group_size channels)
+        self.bounds_k = None if bounds_k is None else np.ascontiguousarray(bounds_k, dtype=np.int32).reshape(n_kv_heads, -1)
+        self.bounds_v = None if bounds_v is None else np.ascontiguousarray(bounds_v, dtype=np.int32).reshape(n_kv_heads, -1)
+        for bd in (self.bounds_k, self.bounds_v):
+            if bd is not None:
+                assert np.all(bd[:, 0] == 0) and np.all(bd[:, -1] == head_dim) and np.all(np.diff(bd, axis=1) > 0)
+                self.ng = bd.shape[1] - 1
+        assert self.bounds_k is None or self.bounds_v is None or self.bounds_k.shape == self.bounds_v.shape
         self.cap_q = max(max_tokens - window, 0)
         B, H, D, W = batch, n_kv_heads, head_dim, window
         self.k_codes = np.zeros((B, H, self.cap_q, D * k_bits // 8), dtype=np.uint8)
@@ -160,7 +186,9 @@ class OracleCache:
                       _ptr(self.k_codes), _ptr(self.v_codes), _ptr(self.k_meta), _ptr(self.v_meta),
                       _ptr(self.k_win), _ptr(self.v_win), _ptr(self.lengths),
                       _ptr(self.reorder_k), _ptr(self.reorder_v), _ptr(self.alpha_k), _ptr(self.alpha_v),
-                      self.n_sink, _ptr(self.k_sink), _ptr(self.v_sink), int(self.meta_fp8))
+                      self.n_sink, _ptr(self.k_sink), _ptr(self.v_sink), int(self.meta_fp8), self.ng,
+                      None if self.bounds_k is None else _ptr(self.bounds_k),
+                      None if self.bounds_v is None else _ptr(self.bounds_v))
 
     def append(self, k: np.ndarray, v: np.ndarray, n_new=None) -> int:
         """k, v: float16 [B, n, Hkv, D], original channel order; n_new: per-sequence counts or None."""

@@ -16,15 +16,18 @@ from test_oracle_quantizer import unpack_codes
 D = 128
 
 
-def make_cache(B, Hq, Hkv, W, cap, bits=2, group=128, alpha=0.9, seed=0, identity=False, n_sink=0, meta_fp8=False):
+def make_cache(B, Hq, Hkv, W, cap, bits=2, group=128, alpha=0.9, seed=0, identity=False, n_sink=0, meta_fp8=False,
+               bounds_k=None, bounds_v=None, v_bits=None):
     rng = np.random.default_rng(seed)
     if identity:
         rk = rv = np.tile(np.arange(D, dtype=np.int32), (Hkv, 1))
     else:
         rk = np.stack([rng.permutation(D) for _ in range(Hkv)]).astype(np.int32)
         rv = np.stack([rng.permutation(D) for _ in range(Hkv)]).astype(np.int32)
-    a = np.full((Hkv, D // group), alpha, np.float32)
-    return orc.OracleCache(B, Hq, Hkv, D, bits, bits, group, W, cap, rk, rv, a, a, n_sink=n_sink, meta_fp8=meta_fp8)
+    ng = D // group if bounds_k is None else np.asarray(bounds_k).shape[-1] - 1
+    a = np.full((Hkv, ng), alpha, np.float32)
+    return orc.OracleCache(B, Hq, Hkv, D, bits, bits if v_bits is None else v_bits, group, W, cap, rk, rv, a, a,
+                           n_sink=n_sink, meta_fp8=meta_fp8, bounds_k=bounds_k, bounds_v=bounds_v)
 
 
 def rand_kv(B, n, Hkv, seed):
@@ -46,16 +49,17 @@ def mixed_cache_dense(c, b, hk):
     L = int(c.lengths[b])
     Lq = max(L - c.W, 0)
     out = []
-    for codes, meta, win, sink, bits in ((c.k_codes, c.k_meta, c.k_win, c.k_sink, c.k_bits),
-                                         (c.v_codes, c.v_meta, c.v_win, c.v_sink, c.v_bits)):
+    for codes, meta, win, sink, bits, bounds in ((c.k_codes, c.k_meta, c.k_win, c.k_sink, c.k_bits, c.bounds_k),
+                                                 (c.v_codes, c.v_meta, c.v_win, c.v_sink, c.v_bits, c.bounds_v)):
         code = unpack_codes(codes[b, hk, :Lq], bits).astype(np.float64)
+        widths = np.full(c.ng, c.G) if bounds is None else np.diff(bounds[hk])      # channels per group
         if c.meta_fp8:                               # E4M3 bytes: decoded by a library, not by the oracle
             import torch
             meta = torch.from_numpy(meta[b, hk, :Lq].astype(np.uint8)).view(torch.float8_e4m3fn).to(torch.float64).numpy()
         else:
             meta = meta[b, hk, :Lq]
-        h = np.repeat(meta[:, :, 0].astype(np.float64), c.G, axis=1)
-        z = np.repeat(meta[:, :, 1].astype(np.float64), c.G, axis=1)
+        h = np.repeat(meta[:, :, 0].astype(np.float64), widths, axis=1)
+        z = np.repeat(meta[:, :, 1].astype(np.float64), widths, axis=1)
         dense = np.zeros((L, D))
         dense[:Lq] = h * code + z
         ns = min(c.n_sink, Lq)                       # attention sinks: full-precision rows, never quantized
@@ -333,3 +337,32 @@ def test_algorithmic_bytes_match_stated_sizes():
     assert abs(workloads.algorithmic_bytes(cf[1]) / 1e6 - 618.5) < 0.5
     assert abs(workloads.algorithmic_bytes(cf[2]) / 1e6 - 404.4) < 0.5
     assert abs(workloads.algorithmic_bytes(cf[3]) / 1e6 - 2417.7) < 0.5
+
+
+# ------------------------------------------------------------------ unequal groups and 3-bit codes in the cache
+@pytest.mark.parametrize("bits,v_bits,bk,bv", [
+    (2, 2, [[0, 32, 128], [0, 96, 128]], [[0, 64, 128], [0, 32, 128]]),      # two groups per row, another split per head and tensor
+    (3, 3, None, None),                                                     # 3-bit codes, equal groups
+    (3, 2, [[0, 16, 40, 128], [0, 100, 120, 128]], [[0, 8, 64, 128], [0, 32, 64, 128]]),
+])
+def test_attention_with_unequal_groups_and_three_bit_codes_matches_brute_force(bits, v_bits, bk, bv):
+    """The cache path (append, single-token appends, attention) with group boundaries and 3-bit streams against the
+    numpy reconstruction above (library softmax + einsum over an independently unpacked and dequantized cache)."""
+    group = 64 if bk is None else 128 // (len(bk[0]) - 1) if 128 % (len(bk[0]) - 1) == 0 else 64
+    c = make_cache(2, 4, 2, 8, 96, bits=bits, v_bits=v_bits, group=group, seed=21, bounds_k=bk, bounds_v=bv)
+    k, v = rand_kv(2, 60, 2, 22)
+    c.append(k[:, :50], v[:, :50])
+    for t in range(50, 60):
+        c.append(k[:, t:t + 1], v[:, t:t + 1])
+    bulk = make_cache(2, 4, 2, 8, 96, bits=bits, v_bits=v_bits, group=group, seed=21, bounds_k=bk, bounds_v=bv)
+    bulk.append(k, v)
+    for a_, b_ in zip(cache_state(c), cache_state(bulk)):
+        assert np.array_equal(a_, b_)
+    q = np.random.default_rng(23).standard_normal((2, 4, D)).astype(np.float16)
+    got = c.attention(q, 0.0884)
+    want = brute_attention(c, q, 0.0884)
+    assert np.abs(got - want).max() < 1e-12
+    # rows of the quantized segment equal the stand-alone row quantizer with the head's own boundaries
+    for h in range(2):
+        ck, mk = orc.quantize_rows(k[0, :52, h], c.reorder_k[h], c.alpha_k[h], bits, group, bounds=None if bk is None else bk[h])
+        assert np.array_equal(c.k_codes[0, h, :52], ck) and np.array_equal(c.k_meta[0, h, :52].view(np.uint16), mk.view(np.uint16))

@@ -55,7 +55,7 @@ def test_f32_to_f16_matches_numpy_round_to_nearest_even():
 
 
 # ------------------------------------------------------------------ closed forms
-@pytest.mark.parametrize("bits", [2, 4])
+@pytest.mark.parametrize("bits", [2, 3, 4])
 def test_lossless_arithmetic_progression(bits):
     """A group holding exactly the 2^bits levels a + k*d (d a power of two), alpha = 1: h = d, z = a, code = k."""
     qmax = (1 << bits) - 1
@@ -79,7 +79,7 @@ def test_pack_layout_golden_bytes():
     assert codes.shape == (1, 64) and np.array_equal(codes[0], want)
 
 
-@pytest.mark.parametrize("bits", [2, 4])
+@pytest.mark.parametrize("bits", [2, 3, 4])
 def test_constant_group_is_degenerate(bits):
     x = np.full((1, D), 0.7314, dtype=np.float16)
     codes, meta = orc.quantize_rows(x, ident(), np.full(1, 1.0, np.float32), bits, D)
@@ -88,7 +88,7 @@ def test_constant_group_is_degenerate(bits):
     assert np.all(orc.dequant_rows(codes, meta, bits, D) == float(x[0, 0]))
 
 
-@pytest.mark.parametrize("bits", [2, 4])
+@pytest.mark.parametrize("bits", [2, 3, 4])
 def test_two_valued_group_hits_both_ends(bits):
     qmax = (1 << bits) - 1
     rng = np.random.default_rng(3)
@@ -119,7 +119,7 @@ def random_rows(n, seed, outliers=True):
     return (rng.standard_normal((n, D)).astype(np.float32) * sigma).astype(np.float16)
 
 
-@pytest.mark.parametrize("bits,group,alpha", [(2, 128, 0.9), (2, 32, 0.85), (4, 64, 0.95), (2, 64, 1.0), (4, 128, 1.0)])
+@pytest.mark.parametrize("bits,group,alpha", [(2, 128, 0.9), (2, 32, 0.85), (4, 64, 0.95), (2, 64, 1.0), (4, 128, 1.0), (3, 64, 0.9)])
 def test_stored_parameters_follow_eq2(bits, group, alpha):
     """h = alpha*(max-min)/qmax and z = alpha*min (Eq. 2 / clipping_quant), stored as fp16.
     The expected values are formed in fp64 straight from the definition; fp32 intermediate
@@ -142,7 +142,8 @@ def test_stored_parameters_follow_eq2(bits, group, alpha):
     assert np.all(h_got >= 0)
 
 
-@pytest.mark.parametrize("bits,group,alpha", [(2, 128, 0.9), (2, 32, 0.85), (4, 64, 0.95), (2, 128, 1.0), (4, 32, 1.0)])
+@pytest.mark.parametrize("bits,group,alpha", [(2, 128, 0.9), (2, 32, 0.85), (4, 64, 0.95), (2, 128, 1.0), (4, 32, 1.0), (3, 64, 0.9),
+                                              (3, 128, 1.0)])
 def test_codes_are_nearest_level_brute_force(bits, group, alpha):
     """Brute force over all 2^bits levels: the stored code is (one of) the nearest reconstruction
     levels h*c+z to x, which also gives |x^ - x| <= h/2 inside the clipped range and the end
@@ -171,7 +172,7 @@ def test_codes_are_nearest_level_brute_force(bits, group, alpha):
     assert np.array_equal(orc.dequant_rows(codes, meta, bits, group), h * c + z)
 
 
-@pytest.mark.parametrize("bits", [2, 4])
+@pytest.mark.parametrize("bits", [2, 3, 4])
 def test_alpha_one_full_group_is_textbook_per_token_minmax(bits):
     """alpha = 1, one group per token, identity order: plain per-token asymmetric min-max
     round-to-nearest (the dynamic quantization of Sec. 3.1).  Away from rounding ties the codes
@@ -343,3 +344,98 @@ def test_fp8_parameters_are_the_rounded_fp32_ones_and_codes_use_them(bits, group
     assert np.array_equal(xhat, h_all.astype(np.float64) * c + z_all.astype(np.float64))
     inside = (x >= z_all) & (x <= z_all + qmax * h_all)                    # inside the stored grid the error is half a step
     assert np.all(np.abs(x.astype(np.float64) - xhat)[inside] <= 0.5 * h_all[inside] * (1 + 1e-6))
+
+
+# ------------------------------------------------------------------ 3-bit codes (the 3-bit column of the KVQuant comparison, Sec. 4.3)
+def test_three_bit_pack_layout_golden_bytes():
+    """A row is a little-endian bit stream of 3-bit fields: codes 0..7 in order occupy three bytes
+    0x88 0xC6 0xFA (bits 000 100 010 110 001 101 011 111 read least significant first); eight codes per 3 bytes,
+    32 codes per 12 bytes, a 128-channel row is 48 bytes."""
+    x = (np.arange(D) % 8).astype(np.float16)[None]
+    codes, meta = orc.quantize_rows(x, ident(), np.ones(1, np.float32), 3, D)
+    assert codes.shape == (1, 48)
+    assert np.array_equal(codes[0], np.array([0x88, 0xC6, 0xFA] * 16, dtype=np.uint8))
+    assert float(meta[0, 0, 0]) == 1.0 and float(meta[0, 0, 1]) == 0.0
+    # the width-generic numpy unpack (bit j*3 .. j*3+2 of the stream) reads the same codes back
+    assert np.array_equal(unpack_codes(codes, 3)[0], np.arange(D) % 8)
+    # a code that straddles a byte boundary: only code 2 (bits 6..8) set to 7 -> 0xC0 0x01
+    y = np.zeros((1, D), np.float16)
+    y[0, 2] = 7.0
+    y[0, 127] = 7.0      # keeps max = 7 wherever code 2 sits; last code occupies bits 381..383 = top of byte 47
+    codes, _ = orc.quantize_rows(y, ident(), np.ones(1, np.float32), 3, D)
+    assert codes[0, 0] == 0xC0 and codes[0, 1] == 0x01 and codes[0, 47] == 0xE0 and not codes[0, 2:47].any()
+
+
+# ------------------------------------------------------------------ unequal groups (split_groups of Algorithm 1; Sec. 4.2)
+def test_equal_boundaries_reproduce_equal_groups_bit_for_bit():
+    x = random_rows(32, 40)
+    rng = np.random.default_rng(41)
+    idx = rng.permutation(D).astype(np.int32)
+    for bits, group in ((2, 32), (4, 64), (3, 64), (2, 128)):
+        ng = D // group
+        a = (0.8 + 0.05 * np.arange(ng)).astype(np.float32)
+        c_eq, m_eq = orc.quantize_rows(x, idx, a, bits, group)
+        c_bd, m_bd = orc.quantize_rows(x, idx, a, bits, group, bounds=np.arange(ng + 1) * group)
+        assert np.array_equal(c_eq, c_bd) and np.array_equal(m_eq.view(np.uint16), m_bd.view(np.uint16))
+        assert np.array_equal(orc.dequant_rows(c_eq, m_eq, bits, group),
+                              orc.dequant_rows(c_bd, m_bd, bits, group, bounds=np.arange(ng + 1) * group))
+
+
+@pytest.mark.parametrize("bits,bounds", [(2, [0, 32, 128]), (2, [0, 96, 128]), (4, [0, 16, 48, 128]), (3, [0, 8, 72, 100, 128]),
+                                         (2, [0, 1, 128])])
+def test_unequal_groups_use_their_own_slice(bits, bounds):
+    """Every group [b_g, b_{g+1}) is quantized exactly like a stand-alone row of that width would be: parameters
+    from its own min and max (Eq. 2, recomputed here in fp64 on the slice), codes nearest to its own levels, and
+    nothing of a group depends on the channels outside it."""
+    qmax = (1 << bits) - 1
+    x = random_rows(48, 50 + bits + len(bounds))
+    ng = len(bounds) - 1
+    alpha = (0.85 + 0.05 * np.arange(ng)).clip(max=1.0).astype(np.float32)
+    codes, meta = orc.quantize_rows(x, ident(), alpha, bits, D, bounds=bounds)
+    assert meta.shape == (48, ng, 2) and codes.shape == (48, D * bits // 8)
+    c = unpack_codes(codes, bits)
+    xd = x.astype(np.float64)
+    deq = orc.dequant_rows(codes, meta, bits, D, bounds=bounds)
+    for g in range(ng):
+        lo, hi = bounds[g], bounds[g + 1]
+        a = float(alpha[g])
+        h_want, z_want = a * (xd[:, lo:hi].max(1) - xd[:, lo:hi].min(1)) / qmax, a * xd[:, lo:hi].min(1)
+        h, z = meta[:, g, 0].astype(np.float64), meta[:, g, 1].astype(np.float64)
+        assert np.all(np.abs(h - h_want) <= 0.5 * np.spacing(np.abs(h_want).astype(np.float16)).astype(np.float64) * 1.01 + 1e-12)
+        assert np.all(np.abs(z - z_want) <= 0.5 * np.spacing(np.abs(z_want).astype(np.float16)).astype(np.float64) * 1.01 + 1e-12)
+        levels = h[:, None, None] * np.arange(qmax + 1) + z[:, None, None]
+        err = np.abs(h[:, None] * c[:, lo:hi] + z[:, None] - xd[:, lo:hi])
+        slack = 4 * np.finfo(np.float32).eps * (np.abs(xd[:, lo:hi]) + np.abs(z[:, None]) + qmax * h[:, None]) + 1e-30
+        assert np.all(err <= np.abs(levels - xd[:, lo:hi, None]).min(axis=2) + slack)
+        assert np.array_equal(deq[:, lo:hi], h[:, None] * c[:, lo:hi] + z[:, None])
+        # the same channels quantized on their own (one group spanning a row that repeats the slice) give the same codes
+        if (hi - lo) in (32, 64, 128):
+            rep = np.tile(x[:, lo:hi], (1, D // (hi - lo)))
+            c_alone, m_alone = orc.quantize_rows(rep, ident(), np.full(D // (hi - lo), alpha[g], np.float32), bits, hi - lo)
+            assert np.array_equal(unpack_codes(c_alone, bits)[:, :hi - lo], c[:, lo:hi])
+            assert np.array_equal(m_alone[:, 0].view(np.uint16), meta[:, g].view(np.uint16))
+
+
+def test_one_channel_group_is_lossless():
+    """An outlier channel in a group of its own: min = max, so h = 0, z = the value (alpha = 1), and it comes back exactly."""
+    rng = np.random.default_rng(60)
+    x = rng.standard_normal((16, D)).astype(np.float16)
+    x[:, 0] = (40 + rng.standard_normal(16)).astype(np.float16)           # one outlier channel
+    codes, meta = orc.quantize_rows(x, ident(), np.ones(2, np.float32), 2, D, bounds=[0, 1, D])
+    deq = orc.dequant_rows(codes, meta, 2, D, bounds=[0, 1, D])
+    assert np.array_equal(deq[:, 0], x[:, 0].astype(np.float64))
+    assert np.all(meta[:, 0, 0] == 0) and np.array_equal(meta[:, 0, 1], x[:, 0])
+    # and the rest of the row no longer pays for the outlier: its scale is that of the 127 ordinary channels
+    _, meta_one = orc.quantize_rows(x, ident(), np.ones(1, np.float32), 2, D)
+    assert np.all(meta[:, 1, 0].astype(np.float64) <= meta_one[:, 0, 0].astype(np.float64))
+    assert np.median(meta[:, 1, 0].astype(np.float64) / meta_one[:, 0, 0].astype(np.float64)) < 0.5
+
+
+def test_unequal_groups_cost_what_their_average_size_costs():
+    """The paper keeps the NUMBER of groups fixed so that the average group size, and with it the average bits, equals
+    the equal-group setting it compares with (Sec. 4.2): 2 groups of 32 + 96 channels store what 2 x 64 store."""
+    x = random_rows(4, 61)
+    c_u, m_u = orc.quantize_rows(x, ident(), np.ones(2, np.float32), 2, D, bounds=[0, 32, 128], meta_fp8=True)
+    c_e, m_e = orc.quantize_rows(x, ident(), np.ones(2, np.float32), 2, 64, meta_fp8=True)
+    assert c_u.shape == c_e.shape and m_u.shape == m_e.shape
+    assert (c_u[0].nbytes + m_u[0].size) * 8 / D == pytest.approx(2.25)      # the paper's figure for group 64, FP8 parameters
