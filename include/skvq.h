@@ -39,7 +39,7 @@ extern "C" {
 
 #define SKVQ_OK 0
 #define SKVQ_ERR_INVALID_ARG (-1) /* NULL where a buffer is required, negative size, ... */
-#define SKVQ_ERR_UNSUPPORTED (-2) /* head_dim != 128, bits not in {2,4}, G not in {32,64,128}, Hq % Hkv != 0, Hq/Hkv > 8 */
+#define SKVQ_ERR_UNSUPPORTED (-2) /* head_dim != 128, bits not in {2,3,4}, G not in {32,64,128}, Hq % Hkv != 0, Hq/Hkv > 8 */
 #define SKVQ_ERR_MISALIGNED (-3)  /* a device buffer is not 16-byte aligned */
 #define SKVQ_ERR_CAPACITY (-4)    /* host-visible overflow: n_new or max_len_hint beyond max_tokens */
 #define SKVQ_ERR_WORKSPACE (-5)   /* workspace missing or smaller than skvq_workspace_size() */
@@ -55,15 +55,20 @@ extern "C" {
  * that a kernel may stage whole tiles; see skvq_quant_capacity(). */
 #define SKVQ_TOKEN_ALIGN 64
 
+/* Group boundaries (skvq_cache::group_bounds_*) are multiples of this many channels. */
+#define SKVQ_GROUP_GRANULE 32
+
 /* Shape and quantization settings (host struct). */
 typedef struct skvq_config {
     int32_t batch;       /* B >= 1 */
     int32_t n_q_heads;   /* Hq */
     int32_t n_kv_heads;  /* Hkv */
     int32_t head_dim;    /* D, must be 128 */
-    int32_t k_bits;      /* 2 or 4 */
-    int32_t v_bits;      /* 2 or 4 */
-    int32_t group_size;  /* G: 32, 64 or 128 consecutive (reordered) channels share scale/zero */
+    int32_t k_bits;      /* 2, 3 or 4 (3: the 3-bit setting of the paper's comparison with KVQuant, Sec. 4.3) */
+    int32_t v_bits;      /* 2, 3 or 4 */
+    int32_t group_size;  /* G: 32, 64 or 128; a row has ng = D/G groups that share scale/zero: equal runs of G consecutive
+                            (reordered) channels, or, with skvq_cache::group_bounds_*, ng runs of unequal width whose
+                            AVERAGE width is G (Sec. 4.2: the number of groups is kept, not their size) */
     int32_t window;      /* W >= 0 latest tokens kept in fp16 (Sec. 3.2); 0 quantizes everything */
     int32_t max_tokens;  /* per-sequence capacity (quantized segment + window) */
     int32_t n_sink;      /* 0..64: the first n_sink positions of a sequence are never quantized (Sec. 3.2, filter
@@ -76,8 +81,9 @@ typedef struct skvq_config {
 /*
  * The cache (host struct of device pointers).  cap = skvq_quant_capacity(cfg).
  * Layouts are row-major:
- *   k_codes/v_codes  uint8   [B][Hkv][cap][D*bits/8]  code j of a row = bits [(j*bits)%8, +bits) of
- *                                                     byte (j*bits)/8, j counted in reordered order
+ *   k_codes/v_codes  uint8   [B][Hkv][cap][D*bits/8]  a row is a little-endian bit stream: code j = bits [j*bits, (j+1)*bits)
+ *                                                     of the row, j counted in reordered order (2- and 4-bit codes never
+ *                                                     cross a byte; a 3-bit code may: 8 codes per 3 bytes, 48-byte rows)
  *   k_meta/v_meta    half2   [B][Hkv][cap][ng]        {scale h, zero z}; dequantized x^ = h*code + z.  With meta_fp8:
  *                    uint8   [B][Hkv][cap][ng][2]     {E4M3 byte of h, E4M3 byte of z} (1 sign, 4 exponent bits with
  *                                                     bias 7, 3 mantissa bits, no infinities, largest finite 448;
@@ -90,6 +96,13 @@ typedef struct skvq_config {
  *   status           int32   [1]                      optional (may be NULL); SKVQ_STATUS_* bits are OR-ed in
  *   k_sink/v_sink    half    [B][Hkv][n_sink][D]      position t < n_sink once it has left the window, reordered
  *                                                     order; may be NULL when n_sink == 0
+ *   group_bounds_k/_v int32  [Hkv][ng+1]              optional (NULL = equal groups): group g of KV head h covers reordered
+ *                                                     channels [bounds[h][g], bounds[h][g+1]); bounds[h][0] = 0,
+ *                                                     bounds[h][ng] = D, strictly increasing, every entry a multiple of
+ *                                                     SKVQ_GROUP_GRANULE (Sec. 3.1: channels of similar range share a
+ *                                                     group; split_groups(X, group_indices) of Algorithm 1).  The arrays
+ *                                                     live on the device, so the library cannot check them: validate the
+ *                                                     host copy with skvq_check_group_bounds() before uploading it.
  * Rows at or beyond Lq_b, and rows below n_sink, of the quantized buffers hold unspecified bytes.  The buffers fully describe the state:
  * copying them is a checkpoint.
  */
@@ -102,6 +115,7 @@ typedef struct skvq_cache {
     const float *alpha_k, *alpha_v;
     int32_t *status;
     void *k_sink, *v_sink;
+    const int32_t *group_bounds_k, *group_bounds_v;
 } skvq_cache;
 
 /* Options of one decode-attention call (host struct). */
@@ -129,6 +143,11 @@ uint64_t skvq_launch_count(void);
 /* Validate cfg (host only).  Returns SKVQ_OK or the error a call with it would return. */
 int skvq_check_config(const skvq_config *cfg);
 
+/* Validate group boundaries on the host: bounds is int32 [n_kv_heads][ng+1] with ng = head_dim / group_size.  Returns
+ * SKVQ_OK, or SKVQ_ERR_INVALID_ARG when a row does not start at 0, end at head_dim, increase strictly, or holds an entry
+ * that is not a multiple of SKVQ_GROUP_GRANULE. */
+int skvq_check_group_bounds(const skvq_config *cfg, const int32_t *bounds_host);
+
 /* Rows per (sequence, KV head) in the quantized segment:
  * round_up(max(max_tokens - W, 0), SKVQ_TOKEN_ALIGN), at least SKVQ_TOKEN_ALIGN.  Negative on a bad cfg. */
 int32_t skvq_quant_capacity(const skvq_config *cfg);
@@ -146,6 +165,7 @@ size_t skvq_sink_bytes(const skvq_config *cfg);
  * (stored[j] = x[idx[j]]), split into groups of G channels and quantized per group:
  *   lo = alpha*min, hi = alpha*max, h = fp16((hi-lo)/(2^bits-1)), z = fp16(lo),
  *   code = clamp(rint((x - z)/h), 0, 2^bits-1)   (fp32, IEEE division, ties to even; h == 0 -> code 0)
+ * (min, max and alpha are those of the channel's group: equal runs of G channels, or the runs given by group_bounds_*)
  * the last min(L1, W) tokens are kept in fp16 in the ring, and lengths[b] becomes L1.
  * Exception (Sec. 3.2, the filter mask of Algorithm 1): a token at a position below n_sink is copied, reordered,
  * to k_sink/v_sink when it leaves the window instead of being quantized.

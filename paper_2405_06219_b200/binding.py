@@ -22,10 +22,11 @@ SKVQ_NOALLOC_SCRATCH_BYTES = 8 << 20
 SKVQ_STATUS_OVERFLOW = 1
 SKVQ_STATUS_COPY_TIMEOUT = 2
 SKVQ_TOKEN_ALIGN = 64
+SKVQ_GROUP_GRANULE = 32
 
 EXPORTS = ["skvq_version", "skvq_strerror", "skvq_launch_count", "skvq_check_config", "skvq_quant_capacity",
            "skvq_cache_sizes", "skvq_sink_bytes", "skvq_quantize_append", "skvq_workspace_size", "skvq_decode_attention",
-           "skvq_step_staging_size", "skvq_decode_step_host", "skvq_decode_attention_noalloc"]
+           "skvq_step_staging_size", "skvq_decode_step_host", "skvq_decode_attention_noalloc", "skvq_check_group_bounds"]
 
 
 class SkvqConfig(ctypes.Structure):
@@ -36,7 +37,7 @@ class SkvqConfig(ctypes.Structure):
 class SkvqCacheStruct(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in ("k_codes", "v_codes", "k_meta", "v_meta", "k_win", "v_win", "lengths",
                                                "reorder_k", "reorder_v", "alpha_k", "alpha_v", "status", "k_sink",
-                                               "v_sink")]
+                                               "v_sink", "group_bounds_k", "group_bounds_v")]
 
 
 class SkvqAttnArgs(ctypes.Structure):
@@ -66,6 +67,8 @@ def lib() -> ctypes.CDLL:
         L.skvq_launch_count.restype = ctypes.c_uint64
         L.skvq_check_config.restype = c_int
         L.skvq_check_config.argtypes = [P(SkvqConfig)]
+        L.skvq_check_group_bounds.restype = c_int
+        L.skvq_check_group_bounds.argtypes = [P(SkvqConfig), vp]
         L.skvq_quant_capacity.restype = ctypes.c_int32
         L.skvq_quant_capacity.argtypes = [P(SkvqConfig)]
         L.skvq_cache_sizes.restype = c_int
@@ -120,6 +123,11 @@ def skvq_check_config(cfg: SkvqConfig) -> int:
     return lib().skvq_check_config(ctypes.byref(cfg))
 
 
+def skvq_check_group_bounds(cfg: SkvqConfig, bounds_host) -> int:
+    """bounds_host: contiguous int32 numpy array [Hkv, ng+1] in host memory."""
+    return lib().skvq_check_group_bounds(ctypes.byref(cfg), bounds_host.ctypes.data)
+
+
 def skvq_quant_capacity(cfg: SkvqConfig) -> int:
     return lib().skvq_quant_capacity(ctypes.byref(cfg))
 
@@ -170,11 +178,13 @@ def skvq_decode_attention_noalloc(cfg, cache, q, out, sm_scale, max_len_hint, n_
 class SkvqCache:
     """Allocates the cache buffers as torch tensors (device memory only) and keeps the C structs.
 
-    reorder_k/_v: int32 [Hkv, D]; alpha_k/_v: float32 [Hkv, D/G] (host arrays or tensors).
+    reorder_k/_v: int32 [Hkv, D]; alpha_k/_v: float32 [Hkv, D/G] (host arrays or tensors); bounds_k/_v: optional
+    int32 [Hkv, D/G + 1] group boundaries (host arrays), checked with skvq_check_group_bounds before the upload.
     """
 
     def __init__(self, batch, n_q_heads, n_kv_heads, head_dim, k_bits, v_bits, group_size, window, max_tokens,
-                 reorder_k, reorder_v, alpha_k, alpha_v, device="cuda:0", n_sink=0, meta_fp8=False):
+                 reorder_k, reorder_v, alpha_k, alpha_v, device="cuda:0", n_sink=0, meta_fp8=False, bounds_k=None,
+                 bounds_v=None):
         self.cfg = SkvqConfig(batch, n_q_heads, n_kv_heads, head_dim, k_bits, v_bits, group_size, window, max_tokens,
                               n_sink, 1 if meta_fp8 else 0)
         _check(skvq_check_config(self.cfg), "skvq_check_config")
@@ -202,10 +212,21 @@ class SkvqCache:
         self.reorder_v = torch.as_tensor(reorder_v, dtype=torch.int32).reshape(H, D).contiguous().to(dev)
         self.alpha_k = torch.as_tensor(alpha_k, dtype=torch.float32).reshape(H, self.ng).contiguous().to(dev)
         self.alpha_v = torch.as_tensor(alpha_v, dtype=torch.float32).reshape(H, self.ng).contiguous().to(dev)
+        self.bounds_k = self._upload_bounds(bounds_k)
+        self.bounds_v = self._upload_bounds(bounds_v)
         self.struct = SkvqCacheStruct(*[t.data_ptr() for t in (
             self.k_codes, self.v_codes, self.k_meta, self.v_meta, self.k_win, self.v_win, self.lengths,
-            self.reorder_k, self.reorder_v, self.alpha_k, self.alpha_v, self.status, self.k_sink, self.v_sink)])
+            self.reorder_k, self.reorder_v, self.alpha_k, self.alpha_v, self.status, self.k_sink, self.v_sink)],
+            _dptr(self.bounds_k), _dptr(self.bounds_v))
         self._workspace = None
+
+    def _upload_bounds(self, bounds):
+        if bounds is None:
+            return None
+        import numpy as np
+        b = np.ascontiguousarray(bounds, dtype=np.int32).reshape(self.cfg.n_kv_heads, self.ng + 1)
+        _check(skvq_check_group_bounds(self.cfg, b), "skvq_check_group_bounds")
+        return torch.from_numpy(b).to(self.device)
 
     @classmethod
     def for_workload(cls, w, max_tokens=None, device="cuda:0"):
@@ -213,7 +234,7 @@ class SkvqCache:
         mt = w.context if max_tokens is None else max_tokens
         return cls(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.k_bits, w.v_bits, w.group_size, w.window, mt,
                    w.reorder_index("k"), w.reorder_index("v"), w.alphas(), w.alphas(), device=device, n_sink=w.n_sink,
-                   meta_fp8=w.meta_fp8)
+                   meta_fp8=w.meta_fp8, bounds_k=w.bounds(), bounds_v=w.bounds())
 
     def nbytes(self) -> int:
         return sum(t.numel() * t.element_size() for t in (self.k_codes, self.v_codes, self.k_meta, self.v_meta,

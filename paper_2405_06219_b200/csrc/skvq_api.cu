@@ -15,7 +15,7 @@ static int check_cfg(const skvq_config *c)
         return SKVQ_ERR_INVALID_ARG;
     if (c->batch > 65535 || c->n_kv_heads > 65535) return SKVQ_ERR_UNSUPPORTED;
     if (c->head_dim != kHeadDim) return SKVQ_ERR_UNSUPPORTED;
-    if ((c->k_bits != 2 && c->k_bits != 4) || (c->v_bits != 2 && c->v_bits != 4)) return SKVQ_ERR_UNSUPPORTED;
+    if (c->k_bits < 2 || c->k_bits > 4 || c->v_bits < 2 || c->v_bits > 4) return SKVQ_ERR_UNSUPPORTED;
     if (c->group_size != 32 && c->group_size != 64 && c->group_size != 128) return SKVQ_ERR_UNSUPPORTED;
     if (c->n_q_heads % c->n_kv_heads != 0) return SKVQ_ERR_UNSUPPORTED;
     if (c->n_q_heads / c->n_kv_heads > kMaxRep) return SKVQ_ERR_UNSUPPORTED;
@@ -50,6 +50,7 @@ static Shape make_shape(const skvq_config *c)
     s.max_tokens = c->max_tokens;
     s.n_sink = c->n_sink;
     s.meta_fp8 = c->meta_fp8;
+    s.bounded = 0;      // set by check_cache when the cache carries group boundaries
     return s;
 }
 
@@ -65,6 +66,7 @@ static int check_cache(const skvq_config *cfg, const skvq_cache *c, CachePtrs *o
     if (cfg->n_sink > 0 && (!c->k_sink || !c->v_sink)) return SKVQ_ERR_INVALID_ARG;
     const void *ptrs[] = {c->k_codes, c->v_codes, c->k_meta, c->v_meta, c->k_win, c->v_win,
                           c->lengths, c->reorder_k, c->reorder_v, c->alpha_k, c->alpha_v, c->k_sink, c->v_sink};
+    if ((reinterpret_cast<uintptr_t>(c->group_bounds_k) | reinterpret_cast<uintptr_t>(c->group_bounds_v)) & 3u) return SKVQ_ERR_MISALIGNED;
     for (const void *p : ptrs)
         if (p && misaligned(p)) return SKVQ_ERR_MISALIGNED;
     out->k_codes = static_cast<uint8_t *>(c->k_codes);
@@ -81,6 +83,8 @@ static int check_cache(const skvq_config *cfg, const skvq_cache *c, CachePtrs *o
     out->status = c->status;
     out->k_sink = static_cast<__half *>(c->k_sink);
     out->v_sink = static_cast<__half *>(c->v_sink);
+    out->bounds_k = c->group_bounds_k;
+    out->bounds_v = c->group_bounds_v;
     return SKVQ_OK;
 }
 
@@ -115,6 +119,21 @@ const char *skvq_strerror(int code)
 uint64_t skvq_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 int skvq_check_config(const skvq_config *cfg) { return check_cfg(cfg); }
+
+int skvq_check_group_bounds(const skvq_config *cfg, const int32_t *bounds_host)
+{
+    const int rc = check_cfg(cfg);
+    if (rc != SKVQ_OK) return rc;
+    if (!bounds_host) return SKVQ_ERR_INVALID_ARG;
+    const int ng = kHeadDim / cfg->group_size;
+    for (int h = 0; h < cfg->n_kv_heads; ++h) {
+        const int32_t *b = bounds_host + (size_t)h * (ng + 1);
+        if (b[0] != 0 || b[ng] != kHeadDim) return SKVQ_ERR_INVALID_ARG;
+        for (int g = 0; g < ng; ++g)
+            if (b[g + 1] <= b[g] || b[g + 1] % SKVQ_GROUP_GRANULE != 0) return SKVQ_ERR_INVALID_ARG;
+    }
+    return SKVQ_OK;
+}
 
 int32_t skvq_quant_capacity(const skvq_config *cfg)
 {
@@ -158,7 +177,8 @@ int skvq_quantize_append(const skvq_config *cfg, const skvq_cache *cache, const 
     if (misaligned(k) || misaligned(v) || (n_new_per_seq && (reinterpret_cast<uintptr_t>(n_new_per_seq) & 3u)))
         return SKVQ_ERR_MISALIGNED;
     if (n_new > cfg->max_tokens) return SKVQ_ERR_CAPACITY;
-    const Shape s = make_shape(cfg);
+    Shape s = make_shape(cfg);
+    s.bounded = (c.bounds_k || c.bounds_v) ? 1 : 0;
     const cudaError_t e = launch_append(s, c, static_cast<const __half *>(k), static_cast<const __half *>(v),
                                         n_new_per_seq, n_new, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? SKVQ_OK : SKVQ_ERR_CUDA;
@@ -184,7 +204,8 @@ int skvq_decode_attention(const skvq_config *cfg, const skvq_cache *cache, const
     if (misaligned(q) || misaligned(out)) return SKVQ_ERR_MISALIGNED;
     if (args->max_len_hint < 0 || args->n_splits < 0) return SKVQ_ERR_INVALID_ARG;
     if (args->max_len_hint > cfg->max_tokens) return SKVQ_ERR_CAPACITY;
-    const Shape s = make_shape(cfg);
+    Shape s = make_shape(cfg);
+    s.bounded = (c.bounds_k || c.bounds_v) ? 1 : 0;
     const SplitPlan plan = plan_splits(s, args->max_len_hint, args->n_splits);
     if (!args->workspace || args->workspace_bytes < workspace_bytes(s, plan)) return SKVQ_ERR_WORKSPACE;
     if (misaligned(args->workspace)) return SKVQ_ERR_MISALIGNED;
@@ -275,7 +296,8 @@ int skvq_decode_attention_noalloc(const skvq_config *cfg, const skvq_cache *cach
     if (misaligned(q) || misaligned(out)) return SKVQ_ERR_MISALIGNED;
     if (max_len_hint < 0 || n_splits < 0) return SKVQ_ERR_INVALID_ARG;
     if (max_len_hint > cfg->max_tokens) return SKVQ_ERR_CAPACITY;
-    const Shape s = make_shape(cfg);
+    Shape s = make_shape(cfg);
+    s.bounded = (c.bounds_k || c.bounds_v) ? 1 : 0;
     const SplitPlan plan = plan_splits(s, max_len_hint, n_splits);
     if (workspace_bytes(s, plan) > (size_t)SKVQ_NOALLOC_SCRATCH_BYTES) return SKVQ_ERR_SCRATCH_LIMIT;
     float *scratch = nullptr;

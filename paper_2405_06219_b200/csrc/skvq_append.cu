@@ -50,20 +50,21 @@ __device__ __forceinline__ void bulk_range(int L0, int n_sink, int q_end, int &f
 }
 
 // The codes of 16 elements by the defining formula (IEEE division, rintf); kept out of line: it runs only for the
-// few row segments that have a quotient next to a rounding boundary.
+// few row segments that have a quotient next to a rounding boundary, and for 3-bit codes.  The 16 fields are a
+// little-endian bit stream of 16 * BITS bits in words[0], words[1].
 template <int BITS>
 __device__ __noinline__ void quantize16_exact(const float (&x)[16], float zf, float hf, uint32_t (&words)[2])
 {
     constexpr int qmax = (1 << BITS) - 1;
-    words[0] = 0u;
-    words[1] = 0u;
+    unsigned long long stream = 0ull;
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
         float c = rintf(__fdiv_rn(__fsub_rn(x[j], zf), hf));
         c = fminf(fmaxf(c, 0.0f), (float)qmax);
-        const uint32_t code = (uint32_t)(int)c;
-        words[(j * BITS) >> 5] |= code << ((j * BITS) & 31);
+        stream |= (unsigned long long)(uint32_t)(int)c << (j * BITS);
     }
+    words[0] = (uint32_t)stream;
+    words[1] = (uint32_t)(stream >> 32);
 }
 
 // Quantize the 16 channels held by this lane; `lanes_per_group` lanes share the group statistics.
@@ -84,9 +85,10 @@ __device__ __forceinline__ __half2 from_e4m3x2(uint16_t b)
 
 // Writes what is stored per (token, group): a half2 {h, z}, or its two E4M3 bytes in the low 16 bits of hz_bits.
 // LPG > 0: lanes per group known at compile time (the shuffle rounds unroll); 0: taken from lanes_per_group.
+// lanes_per_group == 0 (with LPG == 0): the group is the lanes [lane_lo, lane_hi) of the row's 8 (groups of unequal width).
 template <int BITS, int LPG = 0>
 __device__ __forceinline__ void quantize16(const float (&x)[16], float alpha, int lanes_per_group, bool meta_fp8,
-                                           uint32_t (&words)[2], uint32_t &hz_bits)
+                                           uint32_t (&words)[2], uint32_t &hz_bits, int lane_lo = 0, int lane_hi = 0)
 {
     // The 8 lanes that own one row always take the same path, so they are the shuffle's member set
     // (K and V rows may use different bit widths and therefore different instantiations).
@@ -104,11 +106,22 @@ __device__ __forceinline__ void quantize16(const float (&x)[16], float alpha, in
             mn = fminf(mn, __shfl_xor_sync(seg_mask, mn, m));
             mx = fmaxf(mx, __shfl_xor_sync(seg_mask, mx, m));
         }
-    } else {
+    } else if (lanes_per_group > 0) {
         for (int m = 1; m < lanes_per_group; m <<= 1) {
             mn = fminf(mn, __shfl_xor_sync(seg_mask, mn, m));
             mx = fmaxf(mx, __shfl_xor_sync(seg_mask, mx, m));
         }
+    } else {
+        // a run of lanes that need not be a power of two nor aligned: look at all eight, keep those of the run
+        const int base = (threadIdx.x & 31) & 24;
+        float a = mn, b = mx;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const float vj = __shfl_sync(seg_mask, mn, base + j), wj = __shfl_sync(seg_mask, mx, base + j);
+            if (j >= lane_lo && j < lane_hi) { a = fminf(a, vj); b = fmaxf(b, wj); }
+        }
+        mn = a;
+        mx = b;
     }
     // Clip both ends (Eq. 2 / clipping_quant); "+ 0" turns a negative zero into +0.
     const float lo = __fadd_rn(__fmul_rn(alpha, mn), 0.0f);
@@ -127,7 +140,10 @@ __device__ __forceinline__ void quantize16(const float (&x)[16], float alpha, in
     const float zf = __high2float(hz);
     words[0] = 0u;
     words[1] = 0u;
-    if (hf != 0.0f) {
+    if constexpr (BITS == 3) {
+        // 3-bit fields do not tile a 32-bit word; this width takes the defining formula directly
+        if (hf != 0.0f) quantize16_exact<3>(x, zf, hf, words);
+    } else if (hf != 0.0f) {
         // The code is clamp(rint(RN((x - z) / h)), 0, qmax) with IEEE division.  One division per element makes
         // this path bound by the special-function unit, so the quotient is first formed as d * RN(1/h): that is
         // within 3 * 2^-24 relative of the IEEE quotient, so wherever every value within 2^-18 relative of it
@@ -197,6 +213,8 @@ __global__ void __launch_bounds__(kAppendThreads) append_kernel(AppendArgs a)
     const __half *src = (is_v ? a.v : a.k) + ((size_t)b * a.n_new * s.Hkv + h) * kHeadDim;   // token stride Hkv*D
     const size_t src_tok_stride = (size_t)s.Hkv * kHeadDim;
     const float *alpha_head = (is_v ? a.c.alpha_v : a.c.alpha_k) + (size_t)h * s.ng;
+    const int32_t *bounds = is_v ? a.c.bounds_v : a.c.bounds_k;      // groups of unequal width, or NULL
+    if (bounds) bounds += (size_t)h * (s.ng + 1);
 
     // This lane's 16 gather indices (stored[j] = source[idx[j]], j = 16*sub .. 16*sub+15).
     int idx[16];
@@ -258,13 +276,22 @@ __global__ void __launch_bounds__(kAppendThreads) append_kernel(AppendArgs a)
         }
         // Every lane of a row's 8-lane segment executes the shuffles inside; inactive rows store nothing.
         {
-            const int lanes_per_group = s.G >> 4;
-            const int g = (sub << 4) / s.G;
+            int lanes_per_group = s.G >> 4;
+            int g = (sub << 4) / s.G;
+            int lane_lo = g * lanes_per_group, lane_hi = lane_lo + lanes_per_group;
+            if (bounds) {      // groups of unequal width: this lane's 16 channels lie inside one of them (boundaries are multiples of 32)
+                g = 0;
+                for (int i = 1; i < s.ng; ++i) g += ((sub << 4) >= bounds[i]) ? 1 : 0;
+                lane_lo = bounds[g] >> 4;
+                lane_hi = bounds[g + 1] >> 4;
+                lanes_per_group = 0;
+            }
             const float alpha = alpha_head[g];
             uint32_t words[2];
             uint32_t hz;
-            if (bits == 2) quantize16<2>(x, alpha, lanes_per_group, f8, words, hz);
-            else quantize16<4>(x, alpha, lanes_per_group, f8, words, hz);
+            if (bits == 2) quantize16<2>(x, alpha, lanes_per_group, f8, words, hz, lane_lo, lane_hi);
+            else if (bits == 3) quantize16<3>(x, alpha, lanes_per_group, f8, words, hz, lane_lo, lane_hi);
+            else quantize16<4>(x, alpha, lanes_per_group, f8, words, hz, lane_lo, lane_hi);
             if (do_quant && t < s.n_sink) {
                 // an attention sink (Sec. 3.2 filter rule): its reordered fp16 row is kept as it is
                 __align__(16) __half xh16[16];
@@ -276,9 +303,17 @@ __global__ void __launch_bounds__(kAppendThreads) append_kernel(AppendArgs a)
                 p[1] = *reinterpret_cast<const uint4 *>(&xh16[8]);
             } else if (do_quant) {
                 uint8_t *codes_row = codes + (size_t)t * row_bytes;
-                if (bits == 2) reinterpret_cast<uint32_t *>(codes_row)[sub] = words[0];
-                else reinterpret_cast<uint2 *>(codes_row)[sub] = make_uint2(words[0], words[1]);
-                if ((sub & (lanes_per_group - 1)) == 0) {
+                if (bits == 2) {
+                    reinterpret_cast<uint32_t *>(codes_row)[sub] = words[0];
+                } else if (bits == 3) {      // 48 bits per lane: the row stream continues without padding
+                    uint16_t *p = reinterpret_cast<uint16_t *>(codes_row) + 3 * sub;
+                    p[0] = (uint16_t)words[0];
+                    p[1] = (uint16_t)(words[0] >> 16);
+                    p[2] = (uint16_t)words[1];
+                } else {
+                    reinterpret_cast<uint2 *>(codes_row)[sub] = make_uint2(words[0], words[1]);
+                }
+                if (sub == lane_lo) {
                     const size_t mi = meta0 + (size_t)t * s.ng + g;
                     if (f8) reinterpret_cast<uint16_t *>(meta)[mi] = (uint16_t)hz;
                     else reinterpret_cast<uint32_t *>(meta)[mi] = hz;
@@ -407,7 +442,8 @@ cudaError_t launch_append(const Shape &s, const CachePtrs &c, const __half *k, c
                           const int32_t *n_new_per_seq, int n_new, cudaStream_t stream)
 {
     if (n_new <= 0) return cudaSuccess;
-    const bool bulk = n_new >= kBulkTok;
+    // the tile kernel serves 2- and 4-bit codes in equal groups; everything else goes through append_kernel
+    const bool bulk = n_new >= kBulkTok && !s.bounded && s.k_bits != 3 && s.v_bits != 3;
     AppendArgs a{s, c, k, v, n_new_per_seq, n_new, bulk ? 1 : 0};
     // what append_kernel keeps: evictions (at most W), and new tokens outside the bulk tiles (fewer than W + 128
     // when there are bulk tiles, all of them otherwise)

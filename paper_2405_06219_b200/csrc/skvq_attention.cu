@@ -11,6 +11,8 @@
 // the softmax denominator, undoes the value permutation and writes fp16.
 #include <math_constants.h>
 
+#include <type_traits>
+
 #include "skvq_internal.cuh"
 
 namespace skvq {
@@ -42,14 +44,26 @@ __device__ __forceinline__ float warp_sum(float v)
     return v;
 }
 
-// Scalar partition kernel (configurations the tensor-core kernel does not cover: 4-bit codes, mixed
-// widths, 8 query heads per KV head): one thread per token for the scores, one per channel for P.V.
+// Field j (BITS wide) of a row held as 32-bit words of a little-endian bit stream; a 3-bit field may span two words.
+template <int BITS>
+__device__ __forceinline__ uint32_t stream_field(const uint32_t *w, int j)
+{
+    const int bit = j * BITS, i = bit >> 5, sh = bit & 31;
+    uint32_t v = w[i] >> sh;
+    if (sh + BITS > 32) v |= w[i + 1] << (32 - sh);      // never past the row: 128 * BITS is a multiple of 32
+    return v & ((1u << BITS) - 1u);
+}
+
+// Scalar partition kernel (what the tensor-core kernels do not cover: 3-bit codes, groups of unequal width, 4-bit
+// codes with several query heads per KV head or groups of 32): one thread per token for the scores, one per channel
+// for P.V.  Scale and zero point are applied per 32-channel granule, whose group comes from a small map, so equal and
+// unequal groups take the same path.
 template <int KBITS, int VBITS>
 __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
 {
     const Shape &s = a.s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int rep = s.rep, G = s.G, ng = s.ng;
+    const int rep = s.rep, ng = s.ng;
     // Order matters: the merge kernel reads the lengths, the sinks and the window BEFORE its own wait, so it may only be
     // scheduled once everything in front of this grid (append, bookkeeping, plan) has completed and is visible.  Waiting
     // first and triggering afterwards gives exactly that; the merge kernel still runs under this kernel's body.
@@ -72,7 +86,7 @@ __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
     float *partials = a.ws + a.plan.hdr_ints;
 
     __shared__ float sq[kMaxRep][kHeadDim];        // permuted query, times sm_scale*log2(e)
-    __shared__ float sqsum[kMaxRep][4];            // per-group sums of the above
+    __shared__ float sqsum[kMaxRep][kGranules];    // per-granule sums of the above
     __shared__ float sp[kMaxRep][kTile];           // probabilities of the current tile
     __shared__ float sred[kMaxRep][kThreads / 32];
 
@@ -87,16 +101,16 @@ __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
         sq[r][tid] = __half2float(qrow[idx_k[tid] & (kHeadDim - 1)]) * a.scale_log2;
     }
     __syncthreads();
-    if (tid < rep * ng) {
-        const int r = tid / ng, g = tid % ng;
+    if (tid < rep * kGranules) {
+        const int r = tid / kGranules, gr = tid % kGranules;
         float acc = 0.f;
-        for (int j = g * G; j < (g + 1) * G; ++j) acc += sq[r][j];
-        sqsum[r][g] = acc;
+        for (int j = gr * kGranule; j < (gr + 1) * kGranule; ++j) acc += sq[r][j];
+        sqsum[r][gr] = acc;
     }
+    const uint32_t kmap = granule_groups(a.c.bounds_k, hk, s.G, ng), vmap = granule_groups(a.c.bounds_v, hk, s.G, ng);
     __syncthreads();
 
     constexpr int KROW = kHeadDim * KBITS / 8, VROW = kHeadDim * VBITS / 8;
-    constexpr int KQMAX = (1 << KBITS) - 1, VQMAX = (1 << VBITS) - 1;
     const uint8_t *k_codes = a.c.k_codes + bh * (size_t)s.cap * KROW;
     const uint8_t *v_codes = a.c.v_codes + bh * (size_t)s.cap * VROW;
     // {h, z} of row r, group g: a half2, or two E4M3 bytes (every E4M3 value is an fp16 value)
@@ -126,29 +140,31 @@ __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
             if (valid) {
 #pragma unroll
                 for (int r = 0; r < kMaxRep; ++r) sc[r] = 0.f;
-                {
-                    const uint32_t *row = reinterpret_cast<const uint32_t *>(k_codes + (size_t)t * KROW);
-                    constexpr int PER_WORD = 32 / KBITS;
-                    for (int g = 0; g < ng; ++g) {
-                        float part[kMaxRep];
+                const uint4 *row4 = reinterpret_cast<const uint4 *>(k_codes + (size_t)t * KROW);      // rows are multiples of 16 bytes
+                constexpr int GW = kGranule * KBITS / 32;      // words per granule: its 32 fields start on a word boundary
 #pragma unroll
-                        for (int r = 0; r < kMaxRep; ++r) part[r] = 0.f;
-                        for (int w = g * G / PER_WORD; w < (g + 1) * G / PER_WORD; ++w) {
-                            const uint32_t word = __ldg(row + w);
+                for (int gr = 0; gr < kGranules; ++gr) {
+                    uint32_t w[GW];
 #pragma unroll
-                            for (int i = 0; i < PER_WORD; ++i) {
-                                const float code = (float)((word >> (i * KBITS)) & KQMAX);
-                                const int j = w * PER_WORD + i;
+                    for (int i = 0; i < GW; ++i) {
+                        const int wi = gr * GW + i;
+                        const uint4 x = __ldg(row4 + (wi >> 2));
+                        w[i] = (wi & 3) == 0 ? x.x : (wi & 3) == 1 ? x.y : (wi & 3) == 2 ? x.z : x.w;
+                    }
+                    float part[kMaxRep];
 #pragma unroll
-                                for (int r = 0; r < kMaxRep; ++r)
-                                    if (r < rep) part[r] = fmaf(sq[r][j], code, part[r]);
-                            }
-                        }
-                        const float2 hz = load_hz(k_meta, meta0 + (size_t)t * ng + g);
+                    for (int r = 0; r < kMaxRep; ++r) part[r] = 0.f;
+#pragma unroll
+                    for (int jj = 0; jj < kGranule; ++jj) {
+                        const float code = (float)stream_field<KBITS>(w, jj);
 #pragma unroll
                         for (int r = 0; r < kMaxRep; ++r)
-                            if (r < rep) sc[r] += hz.x * part[r] + hz.y * sqsum[r][g];
+                            if (r < rep) part[r] = fmaf(sq[r][gr * kGranule + jj], code, part[r]);
                     }
+                    const float2 hz = load_hz(k_meta, meta0 + (size_t)t * ng + ((kmap >> (2 * gr)) & 3u));
+#pragma unroll
+                    for (int r = 0; r < kMaxRep; ++r)
+                        if (r < rep) sc[r] += hz.x * part[r] + hz.y * sqsum[r][gr];
                 }
             }
             // Online softmax update per query head.
@@ -181,14 +197,16 @@ __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
             // P.V: this thread owns (reordered) channel tid.
             const int n_tok = min(kTile, t_end - tile0);
             {
-                constexpr int PER_WORD = 32 / VBITS;
-                const int g = tid / G;
-                const int w = tid / PER_WORD, sh = (tid % PER_WORD) * VBITS;
+                const int g = (vmap >> (2 * (tid >> 5))) & 3u;
+                const int bit = tid * VBITS, wi = bit >> 5, sh = bit & 31;
+                const bool two = sh + VBITS > 32;      // a 3-bit field that runs into the next word of its row
                 for (int tt = max(s.n_sink - tile0, 0); tt < n_tok; ++tt) {      // rows of sinks hold unspecified bytes
                     const size_t row = (size_t)(tile0 + tt);
-                    const uint32_t word = __ldg(reinterpret_cast<const uint32_t *>(v_codes + row * VROW) + w);
+                    const uint32_t *rw = reinterpret_cast<const uint32_t *>(v_codes + row * VROW);
+                    uint32_t word = __ldg(rw + wi) >> sh;
+                    if (two) word |= __ldg(rw + wi + 1) << (32 - sh);
                     const float2 hz = load_hz(v_meta, meta0 + row * ng + g);
-                    const float val = fmaf(hz.x, (float)((word >> sh) & VQMAX), hz.y);
+                    const float val = fmaf(hz.x, (float)(word & ((1u << VBITS) - 1u)), hz.y);
 #pragma unroll
                     for (int r = 0; r < kMaxRep; ++r)
                         if (r < rep) acc[r] = fmaf(sp[r][tt], val, acc[r]);
@@ -414,8 +432,11 @@ __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
 }  // namespace
 
 // Resident CTAs per SM of the partition kernel that serves this shape (sets how many CTAs make one wave).
+// Resident CTAs per SM of the partition kernel that serves this shape (sets how many CTAs make one wave).  It must not
+// depend on whether group boundaries are given: the workspace is sized from the configuration alone.
 static int partition_ctas_per_sm(const Shape &s)
 {
+    if (s.k_bits == 3 || s.v_bits == 3) return 8;                              // scalar kernel
     if (s.rep == 1 && s.G >= 64) return s.k_bits == s.v_bits ? 4 : 3;           // integer kernel
     if (s.k_bits == 2 && s.v_bits == 2 && (s.rep == 3 || (s.rep > 4 && s.rep <= 8)) && (s.G == 128 || s.G == 64 || s.G == 32))
         return 3;                                                              // tcgen05 kernel: 128 tensor-memory columns, 69 KB
@@ -509,21 +530,40 @@ cudaError_t launch_attention(const Shape &s, const CachePtrs &c, const __half *q
     const bool overlap = !ev_begin;      // an event between two kernels serialises them anyway
     dim3 grid(plan.n_slots);
     bool handled = false;
-    cudaError_t em = launch_partition_mma(s, c, q, a.scale_log2, plan, workspace, stream, overlap, &handled);
-    if (em != cudaSuccess) return em;
-    if (!handled) {
-        em = launch_partition_gqa(s, c, q, a.scale_log2, plan, workspace, stream, overlap, &handled);
+    cudaError_t em = cudaSuccess;
+    // the tensor-core kernels serve 2- and 4-bit codes in equal groups; 3-bit streams and groups of unequal width take
+    // the scalar kernel
+    const bool plain = !s.bounded && s.k_bits != 3 && s.v_bits != 3;
+    if (plain) {
+        em = launch_partition_mma(s, c, q, a.scale_log2, plan, workspace, stream, overlap, &handled);
         if (em != cudaSuccess) return em;
+        if (!handled) {
+            em = launch_partition_gqa(s, c, q, a.scale_log2, plan, workspace, stream, overlap, &handled);
+            if (em != cudaSuccess) return em;
+        }
+        if (!handled) {
+            em = launch_partition_tc(s, c, q, a.scale_log2, plan, workspace, stream, overlap, &handled);
+            if (em != cudaSuccess) return em;
+        }
     }
     if (!handled) {
-        em = launch_partition_tc(s, c, q, a.scale_log2, plan, workspace, stream, overlap, &handled);
-        if (em != cudaSuccess) return em;
+        auto launch_scalar = [&](auto kb, auto vb) {
+            return launch_dependent(partition_kernel<decltype(kb)::value, decltype(vb)::value>, grid, dim3(kThreads), 0, stream,
+                                    overlap, a);
+        };
+        auto with_k = [&](auto kb) {
+            switch (s.v_bits) {
+                case 2: return launch_scalar(kb, std::integral_constant<int, 2>{});
+                case 3: return launch_scalar(kb, std::integral_constant<int, 3>{});
+                default: return launch_scalar(kb, std::integral_constant<int, 4>{});
+            }
+        };
+        switch (s.k_bits) {
+            case 2: em = with_k(std::integral_constant<int, 2>{}); break;
+            case 3: em = with_k(std::integral_constant<int, 3>{}); break;
+            default: em = with_k(std::integral_constant<int, 4>{}); break;
+        }
     }
-    if (handled) { /* tensor-core kernel launched */ }
-    else if (s.k_bits == 2 && s.v_bits == 2) em = launch_dependent(partition_kernel<2, 2>, grid, dim3(kThreads), 0, stream, overlap, a);
-    else if (s.k_bits == 4 && s.v_bits == 4) em = launch_dependent(partition_kernel<4, 4>, grid, dim3(kThreads), 0, stream, overlap, a);
-    else if (s.k_bits == 4 && s.v_bits == 2) em = launch_dependent(partition_kernel<4, 2>, grid, dim3(kThreads), 0, stream, overlap, a);
-    else em = launch_dependent(partition_kernel<2, 4>, grid, dim3(kThreads), 0, stream, overlap, a);
     if (em != cudaSuccess) return em;
     if (ev_end) cudaEventRecord(ev_end, stream);
     // merge CTAs may be scheduled while the last partition CTAs still run: they do the window part first and

@@ -12,6 +12,8 @@ namespace skvq {
 constexpr int kHeadDim = 128;
 constexpr int kMaxRep = 8;            // query heads per KV head supported by the kernels
 constexpr int kPartialStride = 132;   // floats per split partial: o'[128], m (log2 domain), l, 2 pad
+constexpr int kGranule = SKVQ_GROUP_GRANULE;          // group boundaries are multiples of this many channels
+constexpr int kGranules = kHeadDim / kGranule;
 
 // Everything the kernels need, by value.
 struct Shape {
@@ -20,6 +22,7 @@ struct Shape {
     int W, cap, max_tokens;
     int n_sink;            // positions below this are kept fp16 in the sink store when they leave the window
     int meta_fp8;          // scale/zero stored as two E4M3 bytes per (token, group) instead of a half2
+    int bounded;           // group boundaries of unequal width are given (CachePtrs::bounds_k / bounds_v)
 };
 
 struct CachePtrs {
@@ -31,6 +34,7 @@ struct CachePtrs {
     const float *alpha_k, *alpha_v;
     int32_t *status;
     __half *k_sink, *v_sink;
+    const int32_t *bounds_k, *bounds_v;      // [Hkv][ng+1] or NULL
 };
 
 // Flat partition of the quantized prefixes.  The unit is 256 tokens of one (sequence, KV head); all units of a
@@ -61,6 +65,23 @@ struct Segment {
 };
 
 #ifdef __CUDACC__
+// Group of every 32-channel granule of KV head hk, packed two bits per granule: equal groups of G channels, or the
+// boundaries in bounds[hk][0..ng] (multiples of 32; an entry that is not is treated as the next multiple below).
+__device__ inline uint32_t granule_groups(const int32_t *bounds, int hk, int G, int ng)
+{
+    uint32_t map = 0;
+#pragma unroll
+    for (int gr = 0; gr < kGranules; ++gr) {
+        int g = (gr * kGranule) / G;
+        if (bounds) {
+            g = 0;
+            for (int i = 1; i < ng; ++i) g += (gr * kGranule >= bounds[(size_t)hk * (ng + 1) + i]) ? 1 : 0;
+        }
+        map |= (uint32_t)g << (2 * gr);
+    }
+    return map;
+}
+
 // One thread walks the segments of slot w.  hdr is the workspace header written by the plan kernel.
 struct SlotWalker {
     const int *pre;     // units (per KV head) of the sequences before b, [B+1]

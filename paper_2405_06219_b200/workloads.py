@@ -48,6 +48,8 @@ class Workload:
     calib_tokens: int = 512
     n_sink: int = 0              # first positions kept fp16 for good (attention sinks; the paper's experiments use 5)
     meta_fp8: bool = False       # scale and zero point stored in FP8 E4M3 instead of fp16
+    group_bounds: tuple | None = None   # boundaries of groups of unequal width (0, ..., head_dim), same for every head and
+                                        # for keys and values; len - 1 must equal head_dim / group_size
 
     @property
     def sm_scale(self) -> float:
@@ -132,6 +134,13 @@ class Workload:
         x = self.tokens(tensor, 0, 0, self.calib_tokens).astype(np.float32)
         rng_c = x.max(axis=0) - x.min(axis=0)                       # [Hkv, D]
         return np.argsort(rng_c, axis=1, kind="stable").astype(np.int32)
+
+    def bounds(self):
+        """int32 [Hkv, ng+1] group boundaries, or None for equal groups."""
+        if self.group_bounds is None:
+            return None
+        assert len(self.group_bounds) - 1 == self.head_dim // self.group_size
+        return np.tile(np.asarray(self.group_bounds, dtype=np.int32), (self.n_kv_heads, 1))
 
     def alphas(self) -> np.ndarray:
         """float32 [Hkv, D/G] clip factors (one scalar broadcast)."""

@@ -9,7 +9,8 @@ ATTN_TOL = 2e-3   # max-abs error of the fp16 attention output against the oracl
 def oracle_cache_for(w, max_tokens):
     a = w.alphas()
     return orc.OracleCache(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.k_bits, w.v_bits, w.group_size,
-                           w.window, max_tokens, w.reorder_index("k"), w.reorder_index("v"), a, a, n_sink=w.n_sink, meta_fp8=w.meta_fp8)
+                           w.window, max_tokens, w.reorder_index("k"), w.reorder_index("v"), a, a, n_sink=w.n_sink, meta_fp8=w.meta_fp8,
+                           bounds_k=w.bounds(), bounds_v=w.bounds())
 
 
 def assert_cache_bit_exact(gpu, ora, lengths=None):

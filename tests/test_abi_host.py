@@ -48,7 +48,7 @@ def test_version_and_strerror(lib):
 
 
 @pytest.mark.parametrize("kw,code", [
-    (dict(head_dim=64), B.SKVQ_ERR_UNSUPPORTED), (dict(k_bits=3), B.SKVQ_ERR_UNSUPPORTED),
+    (dict(head_dim=64), B.SKVQ_ERR_UNSUPPORTED), (dict(k_bits=3), B.SKVQ_OK), (dict(k_bits=1), B.SKVQ_ERR_UNSUPPORTED), (dict(v_bits=5), B.SKVQ_ERR_UNSUPPORTED),
     (dict(v_bits=8), B.SKVQ_ERR_UNSUPPORTED), (dict(group_size=16), B.SKVQ_ERR_UNSUPPORTED),
     (dict(n_q_heads=7), B.SKVQ_ERR_UNSUPPORTED), (dict(n_q_heads=32, n_kv_heads=2), B.SKVQ_ERR_UNSUPPORTED),
     (dict(batch=0), B.SKVQ_ERR_INVALID_ARG), (dict(window=-1), B.SKVQ_ERR_INVALID_ARG),
@@ -128,3 +128,23 @@ def test_calls_reject_bad_arguments_before_any_launch(lib):
     assert lib.skvq_decode_attention(ctypes.byref(c), ctypes.byref(fake), 0x1000, 0x1000, ctypes.byref(toolong), None) \
         == B.SKVQ_ERR_CAPACITY
     assert B.skvq_launch_count() == before
+
+
+def test_three_bit_rows_are_48_bytes(lib):
+    sizes = B.skvq_cache_sizes(cfg(k_bits=3, v_bits=2, group_size=64))
+    cap = B.skvq_quant_capacity(cfg(k_bits=3, v_bits=2, group_size=64))
+    assert sizes[0] == 2 * 2 * cap * 48 and sizes[1] == 2 * 2 * cap * 32      # 128 three-bit fields = 48 bytes
+
+
+def test_group_bounds_are_validated_on_the_host(lib):
+    import numpy as np
+    c = cfg(group_size=64)                                   # two groups per row, two KV heads
+    ok = np.array([[0, 32, 128], [0, 96, 128]], np.int32)
+    assert B.skvq_check_group_bounds(c, ok) == B.SKVQ_OK
+    for bad in ([[0, 32, 128], [0, 48, 128]],                # not a multiple of the 32-channel granule
+                [[0, 128, 128], [0, 64, 128]],               # an empty group
+                [[32, 64, 128], [0, 64, 128]],               # does not start at 0
+                [[0, 64, 96], [0, 64, 128]]):                # does not end at head_dim
+        assert B.skvq_check_group_bounds(c, np.array(bad, np.int32)) == B.SKVQ_ERR_INVALID_ARG
+    assert lib.skvq_check_group_bounds(ctypes.byref(c), None) == B.SKVQ_ERR_INVALID_ARG
+    assert B.SKVQ_GROUP_GRANULE == 32

@@ -363,3 +363,56 @@ def test_adversarial_values_stay_bit_exact():
     got, want = attention_both(gpu, ora, w)
     assert np.isfinite(got).all()
     assert np.abs(got - want).max() <= ATTN_TOL
+
+
+# ------------------------------------------------------------------ groups of unequal width (split_groups of Algorithm 1) and 3-bit codes
+@pytest.mark.parametrize("cfg_i,kw,n", [
+    (1, dict(context=2300, batch=2, n_q_heads=4, n_kv_heads=4, group_size=64, group_bounds=(0, 32, 128)), 2300),    # one head per KV head
+    (2, dict(context=1900, batch=1, group_size=64, group_bounds=(0, 96, 128)), 1900),                              # 4 heads per KV head
+    (4, dict(context=1200, batch=2, ragged=None, n_q_heads=4, n_kv_heads=4, group_bounds=(0, 32, 128)), 1200),     # 4-bit, window 256
+    (2, dict(context=1500, batch=1, group_size=64, group_bounds=(0, 32, 128), meta_fp8=True, n_sink=5), 1500),     # FP8 parameters, sinks
+    (1, dict(context=2100, batch=1, n_q_heads=4, n_kv_heads=4, k_bits=3, v_bits=3, group_size=64), 2100),          # 3-bit, the setting of Sec. 4.3
+    (2, dict(context=1700, batch=2, k_bits=3, v_bits=2), 1700),                                                    # 3-bit keys, 2-bit values, g32, GQA
+    (4, dict(context=1300, batch=1, ragged=None, n_q_heads=8, n_kv_heads=4, k_bits=4, v_bits=3, group_bounds=(0, 96, 128)), 1300),
+    (0, dict(context=700, k_bits=3, v_bits=3, meta_fp8=True), 700),
+])
+def test_unequal_groups_and_three_bit_codes_bit_exact_cache_and_attention(cfg_i, kw, n):
+    w = small(cfg_i, **kw)
+    gpu, ora = both_caches(w, n + 64)
+    k, v = w.prefill("k", n), w.prefill("v", n)
+    cut = (n * 3) // 5
+    gpu.append(dev(k[:, :cut]), dev(v[:, :cut]))                      # bulk-sized pieces, ragged ends, evictions from the ring
+    gpu.append(dev(k[:, cut:]), dev(v[:, cut:]))
+    ora.append(k, v)
+    assert_cache_bit_exact(gpu, ora)
+    got, want = attention_both(gpu, ora, w)
+    assert np.abs(got - want).max() <= ATTN_TOL
+    for s in range(5):                                                # decode steps: single-token appends
+        kn, vn = w.new_token("k", s), w.new_token("v", s)
+        gpu.append(dev(kn), dev(vn))
+        ora.append(kn, vn)
+    assert_cache_bit_exact(gpu, ora)
+    got, want = attention_both(gpu, ora, w, step=1, n_splits=3)
+    assert np.abs(got - want).max() <= ATTN_TOL
+    assert int(gpu.status[0].item()) == 0
+
+
+def test_calibrated_reorder_groups_and_clip_factors_through_the_library():
+    """The offline calibrator's arrays (per-head reorder index, boundaries that differ between heads and between keys
+    and values, per-group clip factors) fed to the library and to the oracle alike."""
+    from oracle import skvq_oracle as orc
+    from paper_2405_06219_b200 import calibrate as cal
+    w = small(2, context=1600, batch=2, n_kv_heads=4, n_q_heads=8, group_size=64)
+    k, v = w.prefill("k", 1600), w.prefill("v", 1600)
+    q_cal = np.stack([w.query(100 + s)[0] for s in range(3)])
+    res = cal.calibrate(q_cal, k[0, :384], v[0, :384], n_groups=2, k_bits=2, v_bits=2, sm_scale=w.sm_scale, grid=[0.8, 0.9, 1.0])
+    assert len({tuple(b) for b in res["bounds_k"].tolist()} | {tuple(b) for b in res["bounds_v"].tolist()}) >= 2
+    gpu = B.SkvqCache(w.batch, w.n_q_heads, w.n_kv_heads, 128, 2, 2, 64, w.window, 1700, res["reorder_k"], res["reorder_v"],
+                      res["alpha_k"], res["alpha_v"], bounds_k=res["bounds_k"], bounds_v=res["bounds_v"])
+    ora = orc.OracleCache(w.batch, w.n_q_heads, w.n_kv_heads, 128, 2, 2, 64, w.window, 1700, res["reorder_k"], res["reorder_v"],
+                          res["alpha_k"], res["alpha_v"], bounds_k=res["bounds_k"], bounds_v=res["bounds_v"])
+    gpu.append(dev(k), dev(v))
+    ora.append(k, v)
+    assert_cache_bit_exact(gpu, ora)
+    got, want = attention_both(gpu, ora, w)
+    assert np.abs(got - want).max() <= ATTN_TOL
