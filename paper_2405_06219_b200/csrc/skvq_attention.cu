@@ -531,17 +531,16 @@ cudaError_t launch_attention(const Shape &s, const CachePtrs &c, const __half *q
     dim3 grid(plan.n_slots);
     bool handled = false;
     cudaError_t em = cudaSuccess;
-    // the tensor-core kernels serve 2- and 4-bit codes in equal groups; 3-bit streams and groups of unequal width take
-    // the scalar kernel
-    const bool plain = !s.bounded && s.k_bits != 3 && s.v_bits != 3;
-    if (plain) {
+    // the tensor-core kernels serve 2- and 4-bit codes; groups of unequal width when there are two per row (the integer
+    // and the grouped-query kernel).  3-bit streams and the other unequal-group shapes take the scalar kernel.
+    if (s.k_bits != 3 && s.v_bits != 3) {
         em = launch_partition_mma(s, c, q, a.scale_log2, plan, workspace, stream, overlap, &handled);
         if (em != cudaSuccess) return em;
         if (!handled) {
             em = launch_partition_gqa(s, c, q, a.scale_log2, plan, workspace, stream, overlap, &handled);
             if (em != cudaSuccess) return em;
         }
-        if (!handled) {
+        if (!handled && !s.bounded) {
             em = launch_partition_tc(s, c, q, a.scale_log2, plan, workspace, stream, overlap, &handled);
             if (em != cudaSuccess) return em;
         }

@@ -161,11 +161,14 @@ __device__ __forceinline__ int owned_token(int kk, int q, int gg) { return 32 * 
 
 // Two CTAs per SM (up to 255 registers per thread) measured faster than three (168 registers): the compiler needs
 // the registers to overlap the four 16-token score blocks and the two value blocks of a tile.
-template <int G, int R, bool F8>
+// UNEQ: two groups of unequal width per row (boundaries on multiples of 32 channels, read from the cache); the group of
+// a 32-channel block then comes from a map instead of from its position.
+template <int G, int R, bool F8, bool UNEQ>
 __global__ void __launch_bounds__(kThreads, 2) partition_gqa_kernel(MmaArgs a)
 {
     using C = GCfg<G, F8>;
     constexpr int NG = C::NG;
+    static_assert(!UNEQ || NG == 2, "unequal groups: two per row");
     static_assert(R <= kHeadSlots, "rows of the P.V MMAs are 4 heads x 4 digits");
     extern __shared__ __align__(128) uint8_t smem[];
     const Shape &s = a.s;
@@ -273,7 +276,12 @@ __global__ void __launch_bounds__(kThreads, 2) partition_gqa_kernel(MmaArgs a)
     if (tid < kHeadSlots * NG) {
         const int r = tid / NG, gg = tid % NG;
         float sq = 0.f, sw = 0.f;
-        for (int j = gg * G; j < (gg + 1) * G; ++j) {
+        int j0 = gg * G, j1 = (gg + 1) * G;
+        if (UNEQ && a.c.bounds_k) {
+            j0 = a.c.bounds_k[(size_t)hk * (NG + 1) + gg] & ~(kGranule - 1);
+            j1 = min(a.c.bounds_k[(size_t)hk * (NG + 1) + gg + 1] & ~(kGranule - 1), kHeadDim);
+        }
+        for (int j = j0; j < j1; ++j) {
             const float v = qs[r * kHeadDim + j];
             sq += v;
             sw += v * field_weight_inv(j & 7);
@@ -282,6 +290,9 @@ __global__ void __launch_bounds__(kThreads, 2) partition_gqa_kernel(MmaArgs a)
         cst[r * 4 + gg] = -64.0f * sw;
     }
     __syncthreads();
+
+    // group of every 32-channel block (two bits each) for keys and values
+    const uint32_t kmap = UNEQ ? granule_groups(a.c.bounds_k, hk, G, NG) : 0u, vmap = UNEQ ? granule_groups(a.c.bounds_v, hk, G, NG) : 0u;
 
     // B operands of the score MMAs.  ldmatrix hands lane t words t and 4+t of a token row; all sixteen fields of a
     // word are used, so k-step sx of channel half hf covers, in lane t, fields 2sx and 2sx+1 (+8) of word 4hf+t.
@@ -445,9 +456,15 @@ __global__ void __launch_bounds__(kThreads, 2) partition_gqa_kernel(MmaArgs a)
             for (int hf = 0; hf < 2; ++hf)
 #pragma unroll
                 for (int par = 0; par < 2; ++par) {
-                    const int gg = (64 * hf + 32 * par) / G;
-                    s0 = fmaf(lo_half(mw0[gg]), ak[hf][par], s0);
-                    s1 = fmaf(lo_half(mw1[gg]), ak[hf][2 + par], s1);
+                    if constexpr (UNEQ) {
+                        const bool g1 = (kmap >> (2 * (2 * hf + par))) & 1u;
+                        s0 = fmaf(lo_half(g1 ? mw0[1] : mw0[0]), ak[hf][par], s0);
+                        s1 = fmaf(lo_half(g1 ? mw1[1] : mw1[0]), ak[hf][2 + par], s1);
+                    } else {
+                        const int gg = (64 * hf + 32 * par) / G;
+                        s0 = fmaf(lo_half(mw0[gg]), ak[hf][par], s0);
+                        s1 = fmaf(lo_half(mw1[gg]), ak[hf][2 + par], s1);
+                    }
                 }
             sraw[mt][0] = s0;
             sraw[mt][1] = s1;
@@ -567,12 +584,19 @@ __global__ void __launch_bounds__(kThreads, 2) partition_gqa_kernel(MmaArgs a)
                 ldmatrix_b8_trans_x2(rr, vaddr + kk * 32 * kRowBytes + hh * 16);
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
-                    const int gg = (64 * hh + 32 * half) / G;
+                    uint32_t A0, A1, A2, A3;      // the digits of this 32-channel block's group
+                    if constexpr (UNEQ) {
+                        const bool g1 = (vmap >> (2 * (2 * hh + half))) & 1u;
+                        A0 = g1 ? Ag[1][0] : Ag[0][0]; A1 = g1 ? Ag[1][1] : Ag[0][1];
+                        A2 = g1 ? Ag[1][2] : Ag[0][2]; A3 = g1 ? Ag[1][3] : Ag[0][3];
+                    } else {
+                        const int gg = (64 * hh + 32 * half) / G;
+                        A0 = Ag[gg][0]; A1 = Ag[gg][1]; A2 = Ag[gg][2]; A3 = Ag[gg][3];
+                    }
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         const uint32_t m = 0x03030303u << (2 * j);
-                        imma16832_uu(acc[hh * 8 + half * 4 + j], Ag[gg][0], Ag[gg][1], Ag[gg][2], Ag[gg][3], rr[half] & m,
-                                     rr[2 + half] & m);
+                        imma16832_uu(acc[hh * 8 + half * 4 + j], A0, A1, A2, A3, rr[half] & m, rr[2 + half] & m);
                     }
                 }
             }
@@ -612,7 +636,7 @@ __global__ void __launch_bounds__(kThreads, 2) partition_gqa_kernel(MmaArgs a)
             const int d = lane + 32 * q4;
             const int j = d & 3;                                             // channel d carries the weight 4^j
             const float winv = j == 0 ? 1.0f : (j == 1 ? 0.25f : (j == 2 ? 0.0625f : 0.015625f));
-            const float o = Os[r * kHeadDim + d] * winv + Zs[r * 4 + d / G];
+            const float o = Os[r * kHeadDim + d] * winv + Zs[r * 4 + (UNEQ ? (int)((vmap >> (2 * (d >> 5))) & 1u) : d / G)];
             Ow[r * kPartialStride + d] = dead ? 0.f : o;
         }
     }
@@ -653,25 +677,25 @@ __global__ void __launch_bounds__(kThreads, 2) partition_gqa_kernel(MmaArgs a)
     }
 }
 
-template <int G, int R, bool F8>
+template <int G, int R, bool F8, bool UNEQ>
 cudaError_t launch_one(const MmaArgs &a, cudaStream_t stream, bool overlap)
 {
     using C = GCfg<G, F8>;
     static unsigned long long configured = 0;      // one bit per device
-    auto kern = partition_gqa_kernel<G, R, F8>;
+    auto kern = partition_gqa_kernel<G, R, F8, UNEQ>;
     const cudaError_t ec = configure_smem_once(kern, C::kSmemBytes, configured);
     if (ec != cudaSuccess) return ec;
     return launch_dependent(kern, dim3(a.plan.n_slots), dim3(kThreads), C::kSmemBytes, stream, overlap, a);
 }
 
-template <int G, bool F8>
+template <int G, bool F8, bool UNEQ>
 cudaError_t launch_g(const MmaArgs &a, cudaStream_t stream, bool overlap, bool *handled)
 {
     *handled = true;
     switch (a.s.rep) {
-        case 1: return launch_one<G, 1, F8>(a, stream, overlap);
-        case 2: return launch_one<G, 2, F8>(a, stream, overlap);
-        case 4: return launch_one<G, 4, F8>(a, stream, overlap);
+        case 1: return launch_one<G, 1, F8, UNEQ>(a, stream, overlap);
+        case 2: return launch_one<G, 2, F8, UNEQ>(a, stream, overlap);
+        case 4: return launch_one<G, 4, F8, UNEQ>(a, stream, overlap);
         default: *handled = false; return cudaSuccess;
     }
 }
@@ -679,25 +703,27 @@ cudaError_t launch_g(const MmaArgs &a, cudaStream_t stream, bool overlap, bool *
 }  // namespace
 
 // Launches the kernel above when the configuration is covered (2-bit K and V, 1, 2 or 4 query heads per KV
-// head); *handled tells the caller whether it did.
+// head; groups of unequal width with two groups per row); *handled tells the caller whether it did.
 cudaError_t launch_partition_gqa(const Shape &s, const CachePtrs &c, const __half *q, float scale_log2,
                                  const SplitPlan &plan, float *workspace, cudaStream_t stream, bool overlap, bool *handled)
 {
     *handled = false;
     if (s.k_bits != 2 || s.v_bits != 2) return cudaSuccess;
+    if (s.bounded && s.G != 64) return cudaSuccess;
     MmaArgs a{s, c, q, scale_log2, plan, workspace};
+    if (s.bounded) return s.meta_fp8 ? launch_g<64, true, true>(a, stream, overlap, handled) : launch_g<64, false, true>(a, stream, overlap, handled);
     if (s.meta_fp8) {
         switch (s.G) {
-            case 128: return launch_g<128, true>(a, stream, overlap, handled);
-            case 64: return launch_g<64, true>(a, stream, overlap, handled);
-            case 32: return launch_g<32, true>(a, stream, overlap, handled);
+            case 128: return launch_g<128, true, false>(a, stream, overlap, handled);
+            case 64: return launch_g<64, true, false>(a, stream, overlap, handled);
+            case 32: return launch_g<32, true, false>(a, stream, overlap, handled);
             default: return cudaSuccess;
         }
     }
     switch (s.G) {
-        case 128: return launch_g<128, false>(a, stream, overlap, handled);
-        case 64: return launch_g<64, false>(a, stream, overlap, handled);
-        case 32: return launch_g<32, false>(a, stream, overlap, handled);
+        case 128: return launch_g<128, false, false>(a, stream, overlap, handled);
+        case 64: return launch_g<64, false, false>(a, stream, overlap, handled);
+        case 32: return launch_g<32, false, false>(a, stream, overlap, handled);
         default: return cudaSuccess;
     }
 }

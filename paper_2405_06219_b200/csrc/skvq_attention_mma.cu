@@ -51,10 +51,13 @@ struct Cfg {
     static_assert(kKTile % 16 == 0 && kVTile % 16 == 0 && kMetaTile % 16 == 0, "bulk copies move multiples of 16 bytes");
 };
 
-template <int G, int KB, int VB, bool F8>
+// UNEQ: two groups of unequal width per row (boundaries on multiples of 32 channels, read from the cache); the group of
+// a 32-channel block then comes from a map instead of from its position.
+template <int G, int KB, int VB, bool F8, bool UNEQ>
 __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB, F8>::kCtasPerSm) partition_mma_kernel(MmaArgs a)
 {
     using C = Cfg<G, KB, VB, F8>;
+    static_assert(!UNEQ || C::NG == 2, "unequal groups: two per row");
     constexpr int NG = C::NG, KROW = C::KROW, VROW = C::VROW, T = C::T;
     extern __shared__ __align__(128) uint8_t smem[];
     const Shape &s = a.s;
@@ -158,10 +161,17 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB, F8>::kCtasPerSm) part
     }
     if (tid >= 32 && tid < 32 + NG) {
         const int gg = tid - 32;
+        int j0 = gg * G, j1 = (gg + 1) * G;
+        if (UNEQ && a.c.bounds_k) {
+            j0 = a.c.bounds_k[(size_t)hk * (NG + 1) + gg] & ~(kGranule - 1);
+            j1 = a.c.bounds_k[(size_t)hk * (NG + 1) + gg + 1] & ~(kGranule - 1);
+        }
         float sq = 0.f;
-        for (int j = gg * G; j < (gg + 1) * G; ++j) sq += qs[j];
+        for (int j = j0; j < j1 && j < kHeadDim; ++j) sq += qs[j];
         sqs[gg] = sq * a.scale_log2;
     }
+    // group of every 32-channel block (two bits each) for keys and values
+    const uint32_t kmap = UNEQ ? granule_groups(a.c.bounds_k, hk, G, NG) : 0u, vmap = UNEQ ? granule_groups(a.c.bounds_v, hk, G, NG) : 0u;
     __syncthreads();
 
     // B operand of the score MMAs (s8).  k-step ks contracts 32 channels; lane t supplies two registers of four
@@ -276,7 +286,12 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB, F8>::kCtasPerSm) part
                 // byte bb of (word & kmask) = weight * code: four channels per AND, no shift
                 const uint32_t a0 = w0[2 * ks] & kmask, a1 = w1[2 * ks] & kmask;
                 const uint32_t a2 = w0[2 * ks + 1] & kmask, a3 = w1[2 * ks + 1] & kmask;
-                imma16832(acc[(32 * ks) / G], a0, a1, a2, a3, bq[ks][0], bq[ks][1]);
+                if constexpr (UNEQ) {
+                    if ((kmap >> (2 * ks)) & 1u) imma16832(acc[1], a0, a1, a2, a3, bq[ks][0], bq[ks][1]);
+                    else imma16832(acc[0], a0, a1, a2, a3, bq[ks][0], bq[ks][1]);
+                } else {
+                    imma16832(acc[(32 * ks) / G], a0, a1, a2, a3, bq[ks][0], bq[ks][1]);
+                }
             }
             // lane (g,t) holds columns 2t, 2t+1 = two adjacent digits for tokens 16mt+g and 16mt+g+8
             if (t < 2) {
@@ -433,11 +448,12 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB, F8>::kCtasPerSm) part
             const int d = lane + 32 * q4;
             const int j = d % C::VCPB;                                 // channel d = VCPB*(byte column) + j carries weight 2^(VB*j)
             const float winv = __int_as_float((127 - VB * j) << 23);
+            const int gd = UNEQ ? (int)((vmap >> (2 * (d >> 5))) & 1u) : d / G;      // group of channel d
             float zg = 0.f;
 #pragma unroll
             for (int gg = 0; gg < NG; ++gg)
-                if (d / G == gg) zg = z_part[gg];
-            const float o = Ot[(d / G) * kHeadDim + d] * winv + zg;
+                if (gd == gg) zg = z_part[gg];
+            const float o = Ot[gd * kHeadDim + d] * winv + zg;
             Ow[d] = failed ? 0.f : o;
         }
     }
@@ -477,38 +493,40 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB, F8>::kCtasPerSm) part
     }
 }
 
-template <int G, int KB, int VB, bool F8>
+template <int G, int KB, int VB, bool F8, bool UNEQ>
 cudaError_t launch_one(const MmaArgs &a, cudaStream_t stream, bool overlap)
 {
     using C = Cfg<G, KB, VB, F8>;
     static unsigned long long configured = 0;      // one bit per device
-    auto kern = partition_mma_kernel<G, KB, VB, F8>;
+    auto kern = partition_mma_kernel<G, KB, VB, F8, UNEQ>;
     const cudaError_t ec = configure_smem_once(kern, C::kSmemBytes, configured);
     if (ec != cudaSuccess) return ec;
     return launch_dependent(kern, dim3(a.plan.n_slots), dim3(kThreads), C::kSmemBytes, stream, overlap, a);
 }
 
-template <int G, bool F8>
+template <int G, bool F8, bool UNEQ>
 cudaError_t launch_g(const MmaArgs &a, cudaStream_t stream, bool overlap)
 {
     if (a.s.k_bits == 2)
-        return a.s.v_bits == 2 ? launch_one<G, 2, 2, F8>(a, stream, overlap) : launch_one<G, 2, 4, F8>(a, stream, overlap);
-    return a.s.v_bits == 2 ? launch_one<G, 4, 2, F8>(a, stream, overlap) : launch_one<G, 4, 4, F8>(a, stream, overlap);
+        return a.s.v_bits == 2 ? launch_one<G, 2, 2, F8, UNEQ>(a, stream, overlap) : launch_one<G, 2, 4, F8, UNEQ>(a, stream, overlap);
+    return a.s.v_bits == 2 ? launch_one<G, 4, 2, F8, UNEQ>(a, stream, overlap) : launch_one<G, 4, 4, F8, UNEQ>(a, stream, overlap);
 }
 
 }  // namespace
 
-// Launches the integer kernel when the configuration is covered (one query head per KV head, G = 64 or 128);
-// *handled tells the caller whether it did.
+// Launches the integer kernel when the configuration is covered (one query head per KV head, 2- or 4-bit codes, G = 64 or
+// 128; groups of unequal width with two groups per row); *handled tells the caller whether it did.
 cudaError_t launch_partition_mma(const Shape &s, const CachePtrs &c, const __half *q, float scale_log2,
                                  const SplitPlan &plan, float *workspace, cudaStream_t stream, bool overlap, bool *handled)
 {
     *handled = false;
-    if (s.rep != 1 || (s.G != 64 && s.G != 128)) return cudaSuccess;
+    if (s.rep != 1 || (s.G != 64 && s.G != 128) || s.k_bits == 3 || s.v_bits == 3) return cudaSuccess;
+    if (s.bounded && s.G != 64) return cudaSuccess;
     MmaArgs a{s, c, q, scale_log2, plan, workspace};
     *handled = true;
-    if (s.meta_fp8) return s.G == 128 ? launch_g<128, true>(a, stream, overlap) : launch_g<64, true>(a, stream, overlap);
-    return s.G == 128 ? launch_g<128, false>(a, stream, overlap) : launch_g<64, false>(a, stream, overlap);
+    if (s.bounded) return s.meta_fp8 ? launch_g<64, true, true>(a, stream, overlap) : launch_g<64, false, true>(a, stream, overlap);
+    if (s.meta_fp8) return s.G == 128 ? launch_g<128, true, false>(a, stream, overlap) : launch_g<64, true, false>(a, stream, overlap);
+    return s.G == 128 ? launch_g<128, false, false>(a, stream, overlap) : launch_g<64, false, false>(a, stream, overlap);
 }
 
 }  // namespace skvq
