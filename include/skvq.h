@@ -50,6 +50,8 @@ extern "C" {
 #define SKVQ_STATUS_OVERFLOW 1    /* bit set in *status when a sequence would have exceeded max_tokens */
 #define SKVQ_STATUS_COPY_TIMEOUT 2 /* bit set when a shared-memory copy inside decode attention never completed (bounded
                                      wait ran out); the affected tokens contribute nothing to the result */
+#define SKVQ_STATUS_BOUNDS 4       /* only from a library built with -DSKVQ_CHECKED (a debugging build): a kernel was about to
+                                     use a row, slot or partial index outside its buffer; the access was skipped */
 
 /* Rows of the quantized segment are allocated in multiples of this many tokens so
  * that a kernel may stage whole tiles; see skvq_quant_capacity(). */

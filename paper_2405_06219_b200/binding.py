@@ -21,6 +21,7 @@ SKVQ_ERR_SCRATCH_LIMIT = -7
 SKVQ_NOALLOC_SCRATCH_BYTES = 8 << 20
 SKVQ_STATUS_OVERFLOW = 1
 SKVQ_STATUS_COPY_TIMEOUT = 2
+SKVQ_STATUS_BOUNDS = 4
 SKVQ_TOKEN_ALIGN = 64
 SKVQ_GROUP_GRANULE = 32
 
@@ -50,6 +51,14 @@ class SkvqError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = code
         super().__init__(f"{where}: {skvq_strerror(code)} ({code})")
+
+
+def use_library(path: str | None) -> None:
+    """Make the wrappers call the library at ``path`` from now on (None = the default libskvq.so): the debugging build
+    libskvq_checked.so exports the same entry points."""
+    global _lib, _LIB_PATH
+    _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libskvq.so") if path is None else path
+    _lib = None
 
 
 def lib() -> ctypes.CDLL:

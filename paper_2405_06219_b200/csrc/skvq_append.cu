@@ -294,6 +294,7 @@ __global__ void __launch_bounds__(kAppendThreads) append_kernel(AppendArgs a)
             if (bits == 2) quantize16<2>(x, alpha, lanes_per_group, f8, words, hz, lane_lo, lane_hi);
             else if (bits == 3) quantize16<3>(x, alpha, lanes_per_group, f8, words, hz, lane_lo, lane_hi);
             else quantize16<4>(x, alpha, lanes_per_group, f8, words, hz, lane_lo, lane_hi);
+            if (do_quant && !SKVQ_IN_BOUNDS(t >= 0 && t < s.cap && (from_ring || (t - L0 >= 0 && t - L0 < a.n_new)), a.c.status)) do_quant = false;
             if (do_quant && t < s.n_sink) {
                 // an attention sink (Sec. 3.2 filter rule): its reordered fp16 row is kept as it is
                 __align__(16) __half xh16[16];
@@ -322,6 +323,7 @@ __global__ void __launch_bounds__(kAppendThreads) append_kernel(AppendArgs a)
                 }
             }
         }
+        if (do_ring_write && !SKVQ_IN_BOUNDS(W > 0 && ring_token - L0 >= 0 && ring_token - L0 < a.n_new, a.c.status)) do_ring_write = false;
         if (do_ring_write) {
             const __half *row = src + (size_t)(ring_token - L0) * src_tok_stride;
 #pragma unroll
@@ -357,6 +359,7 @@ __global__ void __launch_bounds__(kAppendThreads) append_bulk_kernel(AppendArgs 
     bulk_range(L0, s.n_sink, max(L1 - s.W, 0), f0, f1);
     const int t0 = f0 + kBulkTok * blockIdx.x;
     if (t0 >= f1) return;
+    if (!SKVQ_IN_BOUNDS(t0 >= L0 && t0 + kBulkTok <= s.cap && t0 + kBulkTok - L0 <= a.n_new, a.c.status)) return;
 
     __shared__ __align__(16) __half xs[2][kBulkTok][kBulkStride];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;

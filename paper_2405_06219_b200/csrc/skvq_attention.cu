@@ -94,6 +94,7 @@ __global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
     if (tid == 0) seg_sh = walk.next(a.c.lengths, s.W, a.plan.lq_cap);
     __syncthreads();
     const int b = seg_sh.b, hk = seg_sh.hk, q_begin = seg_sh.tok_begin, q_end = seg_sh.tok_end, part_idx = seg_sh.part;
+    if (!segment_in_bounds(seg_sh, s, a.plan, a.c.status)) break;      // checked build only; uniform: every thread reads the same segment
     const size_t bh = (size_t)b * s.Hkv + hk;
     const int32_t *idx_k = a.c.reorder_k + (size_t)hk * kHeadDim;
     for (int r = 0; r < rep; ++r) {
@@ -408,7 +409,8 @@ __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
     // (a no-op unless this kernel was launched with programmatic stream serialization).
     asm volatile("griddepcontrol.wait;" ::: "memory");
     // log-sum-exp merge: the window and the S split partials; thread d owns reordered channel d
-    const int S = pair_partials(a.plan.in_kernel ? hdr_sh : reinterpret_cast<const int *>(a.ws), s.Hkv, b, hk);
+    int S = pair_partials(a.plan.in_kernel ? hdr_sh : reinterpret_cast<const int *>(a.ws), s.Hkv, b, hk);
+    if (!SKVQ_IN_BOUNDS(S >= 0 && S <= a.plan.s_max, a.c.status)) S = 0;
     const float *part = a.ws + a.plan.hdr_ints + ((size_t)b * s.Hq + hq) * a.plan.s_max * kPartialStride;
     float M = m_run;
     for (int i = 0; i < S; ++i) M = fmaxf(M, part[(size_t)i * kPartialStride + kHeadDim]);

@@ -102,6 +102,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB, F8>::kCtasPerSm) part
     if (tid == 0) seg_sh = walk.next(a.c.lengths, s.W, a.plan.lq_cap);
     __syncthreads();
     const int b = seg_sh.b, hk = seg_sh.hk, q_begin = seg_sh.tok_begin, q_end = seg_sh.tok_end, part = seg_sh.part;
+    if (!segment_in_bounds(seg_sh, s, a.plan, a.c.status)) break;      // checked build only; uniform: every thread reads the same segment
     const int n_parts = a.plan.s_max;
 
     uint8_t *stage_base = warp_base;

@@ -64,7 +64,23 @@ struct Segment {
     int part;                  // index of its partial among the pair's partials
 };
 
+// Checked build (-DSKVQ_CHECKED, a debugging aid where no memory checker can be run): every row, slot and partial index
+// is compared with the size of the buffer it addresses before it is used; a violation ORs SKVQ_STATUS_BOUNDS into the
+// status word and the access is skipped.  In the normal build the macro is the constant true and costs nothing.
+#ifdef SKVQ_CHECKED
+#define SKVQ_IN_BOUNDS(cond, status) ((cond) ? true : (((status) != nullptr ? (void)atomicOr((status), SKVQ_STATUS_BOUNDS) : (void)0), false))
+#else
+#define SKVQ_IN_BOUNDS(cond, status) (true)
+#endif
+
 #ifdef __CUDACC__
+// What a partition kernel is about to work on lies inside the cache and the workspace (checked build only).
+__device__ inline bool segment_in_bounds(const Segment &sg, const Shape &s, const SplitPlan &p, int32_t *status)
+{
+    return SKVQ_IN_BOUNDS(sg.b >= 0 && sg.b < s.B && sg.hk >= 0 && sg.hk < s.Hkv && sg.tok_begin >= 0 && sg.tok_begin <= sg.tok_end &&
+                          ((sg.tok_end + SKVQ_TOKEN_ALIGN - 1) & ~(SKVQ_TOKEN_ALIGN - 1)) <= s.cap && sg.part >= 0 && sg.part < p.s_max, status);
+}
+
 // Group of every 32-channel granule of KV head hk, packed two bits per granule: equal groups of G channels, or the
 // boundaries in bounds[hk][0..ng] (multiples of 32; an entry that is not is treated as the next multiple below).
 __device__ inline uint32_t granule_groups(const int32_t *bounds, int hk, int G, int ng)
