@@ -5,6 +5,7 @@ import glob
 import os
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 
 PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
@@ -31,17 +32,27 @@ def needs_build(lib: str = LIB) -> bool:
 def build_library(force: bool = False, verbose: bool = False, checked: bool = False) -> str:
     """Compile every .cu under csrc/ into paper_2405_06219_b200/libskvq.so; with ``checked`` the debugging build
     (-DSKVQ_CHECKED: every index is compared with its buffer's size, violations set SKVQ_STATUS_BOUNDS) into
-    libskvq_checked.so."""
+    libskvq_checked.so.  The translation units are compiled side by side (objects under _build/), then linked."""
     lib = LIB_CHECKED if checked else LIB
     if not force and not needs_build(lib):
         return lib
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    cmd = [nvcc, *NVCC_FLAGS, "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", lib, *sources()]
+    objdir = os.path.join(ROOT, "_build", "checked" if checked else "plain")
+    os.makedirs(objdir, exist_ok=True)
+    flags = [f for f in NVCC_FLAGS if f != "-shared"] + ["-I", os.path.join(ROOT, "include"), "-I", CSRC]
     if checked:
-        cmd += ["-DSKVQ_CHECKED=1"]
+        flags += ["-DSKVQ_CHECKED=1"]
     if verbose:
-        cmd += ["-Xptxas", "-v"]
-    subprocess.run(cmd, check=True)
+        flags += ["-Xptxas", "-v"]
+
+    def compile_one(src):
+        obj = os.path.join(objdir, os.path.basename(src)[:-3] + ".o")
+        subprocess.run([nvcc, *flags, "-c", "-o", obj, src], check=True)
+        return obj
+
+    with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as ex:
+        objs = list(ex.map(compile_one, sources()))
+    subprocess.run([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-Xcompiler", "-fPIC", "-o", lib, *objs], check=True)
     return lib
 
 

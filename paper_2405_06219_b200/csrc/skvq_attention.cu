@@ -2,16 +2,15 @@
 // [packed quantized prefix || fp16 window] (Eq. 1, Algorithm 1), split along the sequence
 // (flash-decoding) with a log-sum-exp merge.  Dequantization happens in registers.
 //
-// Per (sequence, KV head, split) one CTA serves all rep = Hq/Hkv query heads that share the
-// KV head.  It never forms h*code+z per element for the scores: with q' the permuted query,
+// This file holds what all partition kernels share -- the host side of the flat partition (plan_splits), the plan
+// kernel, the dispatch -- and the merge kernel.  The partition kernels themselves (skvq_attention_mma.cu, _gqa.cu,
+// _tc.cu) write partials (o'[128], m, l) of the quantized prefix to the caller's workspace; they never form
+// h*code+z per element for the scores: with q' the permuted query,
 //   q'.K~_t = sum_g h_{t,g} (sum_{j in g} q'_j c_{t,j}) + sum_g z_{t,g} (sum_{j in g} q'_j)
-// so the zero points cost one multiply-add per group.  Scores live in the log2 domain
-// (sm_scale*log2(e) folded into q').  Partials (o'[128], m, l) of the quantized prefix go to the
-// caller's workspace; merge_kernel walks the fp16 window itself, combines everything, divides by
-// the softmax denominator, undoes the value permutation and writes fp16.
+// so the zero points cost one multiply-add per group.  Scores live in the log2 domain (sm_scale*log2(e) folded into
+// q').  merge_kernel walks the fp16 window itself, combines everything, divides by the softmax denominator, undoes
+// the value permutation and writes fp16.
 #include <math_constants.h>
-
-#include <type_traits>
 
 #include "skvq_internal.cuh"
 
@@ -19,7 +18,6 @@ namespace skvq {
 namespace {
 
 constexpr int kThreads = 128;
-constexpr int kTile = 128;   // tokens per tile = threads
 
 struct AttnArgs {
     Shape s;
@@ -42,208 +40,6 @@ __device__ __forceinline__ float warp_sum(float v)
 #pragma unroll
     for (int m = 16; m > 0; m >>= 1) v += __shfl_xor_sync(0xffffffffu, v, m);
     return v;
-}
-
-// Field j (BITS wide) of a row held as 32-bit words of a little-endian bit stream; a 3-bit field may span two words.
-template <int BITS>
-__device__ __forceinline__ uint32_t stream_field(const uint32_t *w, int j)
-{
-    const int bit = j * BITS, i = bit >> 5, sh = bit & 31;
-    uint32_t v = w[i] >> sh;
-    if (sh + BITS > 32) v |= w[i + 1] << (32 - sh);      // never past the row: 128 * BITS is a multiple of 32
-    return v & ((1u << BITS) - 1u);
-}
-
-// Scalar partition kernel (what the tensor-core kernels do not cover: 3-bit codes, groups of unequal width, 4-bit
-// codes with several query heads per KV head or groups of 32): one thread per token for the scores, one per channel
-// for P.V.  Scale and zero point are applied per 32-channel granule, whose group comes from a small map, so equal and
-// unequal groups take the same path.
-template <int KBITS, int VBITS>
-__global__ void __launch_bounds__(kThreads) partition_kernel(AttnArgs a)
-{
-    const Shape &s = a.s;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int rep = s.rep, ng = s.ng;
-    // Order matters: the merge kernel reads the lengths, the sinks and the window BEFORE its own wait, so it may only be
-    // scheduled once everything in front of this grid (append, bookkeeping, plan) has completed and is visible.  Waiting
-    // first and triggering afterwards gives exactly that; the merge kernel still runs under this kernel's body.
-    asm volatile("griddepcontrol.wait;" ::: "memory");      // the lengths, and the plan kernel's header when there is one
-    asm volatile("griddepcontrol.launch_dependents;");      // the merge kernel may start its window part now
-
-    __shared__ __align__(16) Segment seg_sh;
-    __shared__ int more_sh;
-    __shared__ SlotWalker walk;      // only thread 0 touches it; shared memory keeps it out of everybody's registers
-    __shared__ __align__(16) int hdr_sh[kPlanSmemInts];
-    if (a.plan.in_kernel) {
-        if (warp == 0) plan_in_warp(a.c.lengths, s.B, s.Hkv, s.W, a.plan.lq_cap, a.plan.n_slots, hdr_sh);
-        __syncthreads();
-    }
-    if (tid == 0)
-        more_sh = walk.start(a.plan.in_kernel ? hdr_sh : reinterpret_cast<const int *>(a.ws), !a.plan.in_kernel, s.B, s.Hkv,
-                             blockIdx.x) ? 1 : 0;
-    __syncthreads();
-    if (!more_sh) return;
-    float *partials = a.ws + a.plan.hdr_ints;
-
-    __shared__ float sq[kMaxRep][kHeadDim];        // permuted query, times sm_scale*log2(e)
-    __shared__ float sqsum[kMaxRep][kGranules];    // per-granule sums of the above
-    __shared__ float sp[kMaxRep][kTile];           // probabilities of the current tile
-    __shared__ float sred[kMaxRep][kThreads / 32];
-
-    for (;;) {
-    if (tid == 0) seg_sh = walk.next(a.c.lengths, s.W, a.plan.lq_cap);
-    __syncthreads();
-    const int b = seg_sh.b, hk = seg_sh.hk, q_begin = seg_sh.tok_begin, q_end = seg_sh.tok_end, part_idx = seg_sh.part;
-    if (!segment_in_bounds(seg_sh, s, a.plan, a.c.status)) break;      // checked build only; uniform: every thread reads the same segment
-    const size_t bh = (size_t)b * s.Hkv + hk;
-    const int32_t *idx_k = a.c.reorder_k + (size_t)hk * kHeadDim;
-    for (int r = 0; r < rep; ++r) {
-        const __half *qrow = a.q + ((size_t)b * s.Hq + hk * rep + r) * kHeadDim;
-        sq[r][tid] = __half2float(qrow[idx_k[tid] & (kHeadDim - 1)]) * a.scale_log2;
-    }
-    __syncthreads();
-    if (tid < rep * kGranules) {
-        const int r = tid / kGranules, gr = tid % kGranules;
-        float acc = 0.f;
-        for (int j = gr * kGranule; j < (gr + 1) * kGranule; ++j) acc += sq[r][j];
-        sqsum[r][gr] = acc;
-    }
-    const uint32_t kmap = granule_groups(a.c.bounds_k, hk, s.G, ng), vmap = granule_groups(a.c.bounds_v, hk, s.G, ng);
-    __syncthreads();
-
-    constexpr int KROW = kHeadDim * KBITS / 8, VROW = kHeadDim * VBITS / 8;
-    const uint8_t *k_codes = a.c.k_codes + bh * (size_t)s.cap * KROW;
-    const uint8_t *v_codes = a.c.v_codes + bh * (size_t)s.cap * VROW;
-    // {h, z} of row r, group g: a half2, or two E4M3 bytes (every E4M3 value is an fp16 value)
-    const bool f8 = s.meta_fp8 != 0;
-    auto load_hz = [&](const __half2 *base, size_t idx) -> float2 {
-        if (!f8) return __half22float2(base[idx]);
-        const uint16_t b = reinterpret_cast<const uint16_t *>(base)[idx];
-        uint32_t r;
-        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(r) : "h"(b));
-        return __half22float2(*reinterpret_cast<const __half2 *>(&r));
-    };
-    const size_t meta0 = bh * (size_t)s.cap * ng;
-    const __half2 *k_meta = a.c.k_meta, *v_meta = a.c.v_meta;
-
-    float m_run[kMaxRep], l_thread[kMaxRep], acc[kMaxRep];
-#pragma unroll
-    for (int r = 0; r < kMaxRep; ++r) { m_run[r] = -CUDART_INF_F; l_thread[r] = 0.f; acc[r] = 0.f; }
-
-    {
-        const int t_begin = q_begin, t_end = q_end;
-        for (int tile0 = t_begin; tile0 < t_end; tile0 += kTile) {
-            const int t = tile0 + tid;
-            const bool valid = t < t_end && t >= s.n_sink;      // sinks belong to the merge kernel
-            float sc[kMaxRep];
-#pragma unroll
-            for (int r = 0; r < kMaxRep; ++r) sc[r] = -CUDART_INF_F;
-            if (valid) {
-#pragma unroll
-                for (int r = 0; r < kMaxRep; ++r) sc[r] = 0.f;
-                const uint4 *row4 = reinterpret_cast<const uint4 *>(k_codes + (size_t)t * KROW);      // rows are multiples of 16 bytes
-                constexpr int GW = kGranule * KBITS / 32;      // words per granule: its 32 fields start on a word boundary
-#pragma unroll
-                for (int gr = 0; gr < kGranules; ++gr) {
-                    uint32_t w[GW];
-#pragma unroll
-                    for (int i = 0; i < GW; ++i) {
-                        const int wi = gr * GW + i;
-                        const uint4 x = __ldg(row4 + (wi >> 2));
-                        w[i] = (wi & 3) == 0 ? x.x : (wi & 3) == 1 ? x.y : (wi & 3) == 2 ? x.z : x.w;
-                    }
-                    float part[kMaxRep];
-#pragma unroll
-                    for (int r = 0; r < kMaxRep; ++r) part[r] = 0.f;
-#pragma unroll
-                    for (int jj = 0; jj < kGranule; ++jj) {
-                        const float code = (float)stream_field<KBITS>(w, jj);
-#pragma unroll
-                        for (int r = 0; r < kMaxRep; ++r)
-                            if (r < rep) part[r] = fmaf(sq[r][gr * kGranule + jj], code, part[r]);
-                    }
-                    const float2 hz = load_hz(k_meta, meta0 + (size_t)t * ng + ((kmap >> (2 * gr)) & 3u));
-#pragma unroll
-                    for (int r = 0; r < kMaxRep; ++r)
-                        if (r < rep) sc[r] += hz.x * part[r] + hz.y * sqsum[r][gr];
-                }
-            }
-            // Online softmax update per query head.
-            float corr[kMaxRep];
-#pragma unroll
-            for (int r = 0; r < kMaxRep; ++r) {
-                corr[r] = 1.f;
-                if (r < rep) {
-                    const float wm = warp_max(sc[r]);
-                    if (lane == 0) sred[r][warp] = wm;
-                }
-            }
-            __syncthreads();
-#pragma unroll
-            for (int r = 0; r < kMaxRep; ++r) {
-                if (r < rep) {
-                    float tm = sred[r][0];
-#pragma unroll
-                    for (int w = 1; w < kThreads / 32; ++w) tm = fmaxf(tm, sred[r][w]);
-                    const float m_new = fmaxf(m_run[r], tm);    // finite: the tile has a valid token
-                    corr[r] = m_new == -CUDART_INF_F ? 1.f : exp2f(m_run[r] - m_new);   // 0 on the first tile with a token
-                    const float p = valid ? exp2f(sc[r] - m_new) : 0.f;
-                    sp[r][tid] = p;
-                    l_thread[r] = l_thread[r] * corr[r] + p;
-                    m_run[r] = m_new;
-                    acc[r] *= corr[r];
-                }
-            }
-            __syncthreads();
-            // P.V: this thread owns (reordered) channel tid.
-            const int n_tok = min(kTile, t_end - tile0);
-            {
-                const int g = (vmap >> (2 * (tid >> 5))) & 3u;
-                const int bit = tid * VBITS, wi = bit >> 5, sh = bit & 31;
-                const bool two = sh + VBITS > 32;      // a 3-bit field that runs into the next word of its row
-                for (int tt = max(s.n_sink - tile0, 0); tt < n_tok; ++tt) {      // rows of sinks hold unspecified bytes
-                    const size_t row = (size_t)(tile0 + tt);
-                    const uint32_t *rw = reinterpret_cast<const uint32_t *>(v_codes + row * VROW);
-                    uint32_t word = __ldg(rw + wi) >> sh;
-                    if (two) word |= __ldg(rw + wi + 1) << (32 - sh);
-                    const float2 hz = load_hz(v_meta, meta0 + row * ng + g);
-                    const float val = fmaf(hz.x, (float)(word & ((1u << VBITS) - 1u)), hz.y);
-#pragma unroll
-                    for (int r = 0; r < kMaxRep; ++r)
-                        if (r < rep) acc[r] = fmaf(sp[r][tt], val, acc[r]);
-                }
-            }
-            __syncthreads();   // sp and sred are rewritten by the next tile
-        }
-    }
-
-    // Write the partial: o'[d], m, l per query head.
-#pragma unroll
-    for (int r = 0; r < kMaxRep; ++r) {
-        if (r < rep) {
-            const float ws_ = warp_sum(l_thread[r]);
-            if (lane == 0) sred[r][warp] = ws_;
-        }
-    }
-    __syncthreads();
-#pragma unroll
-    for (int r = 0; r < kMaxRep; ++r) {
-        if (r < rep) {
-            float *part = partials + (((size_t)b * s.Hq + hk * rep + r) * a.plan.s_max + part_idx) * kPartialStride;
-            part[tid] = acc[r];
-            if (tid == 0) {
-                float l = 0.f;
-                for (int w = 0; w < kThreads / 32; ++w) l += sred[r][w];
-                part[kHeadDim] = m_run[r];
-                part[kHeadDim + 1] = l;
-            }
-        }
-    }
-    __syncthreads();          // the segment's shared data is dead; thread 0 decides whether there is another one
-    if (tid == 0) more_sh = walk.done() ? 0 : 1;
-    __syncthreads();
-    if (!more_sh) break;
-    }
 }
 
 // Writes the workspace header of the flat partition: units (256 quantized tokens) per sequence as an exclusive
@@ -438,12 +234,10 @@ __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
 // depend on whether group boundaries are given: the workspace is sized from the configuration alone.
 static int partition_ctas_per_sm(const Shape &s)
 {
-    if (s.k_bits == 3 || s.v_bits == 3) return 8;                              // scalar kernel
-    if (s.rep == 1 && s.G >= 64) return s.k_bits == s.v_bits ? 4 : 3;           // integer kernel
-    if (s.k_bits == 2 && s.v_bits == 2 && (s.rep == 3 || (s.rep > 4 && s.rep <= 8)) && (s.G == 128 || s.G == 64 || s.G == 32))
-        return 3;                                                              // tcgen05 kernel: 128 tensor-memory columns, 69 KB
-    if (s.k_bits == 2 && s.v_bits == 2 && s.rep <= 4) return 2;                // grouped-query kernel, 244 registers
-    return 8;                                                                  // scalar kernel
+    const bool three = s.k_bits == 3 || s.v_bits == 3;
+    if (!three && s.rep == 1 && s.G >= 64) return s.k_bits == s.v_bits ? 4 : 3;           // integer kernel
+    if (s.k_bits == 2 && s.v_bits == 2 && (s.rep == 1 || s.rep == 2 || s.rep == 4)) return 2;   // grouped-query kernel, 244 registers
+    return (s.k_bits == 2 && s.v_bits == 2) ? 3 : 2;      // tcgen05 kernel: 128 tensor-memory columns, 69-85 KB of shared memory
 }
 
 int current_device()
@@ -533,8 +327,9 @@ cudaError_t launch_attention(const Shape &s, const CachePtrs &c, const __half *q
     dim3 grid(plan.n_slots);
     bool handled = false;
     cudaError_t em = cudaSuccess;
-    // the tensor-core kernels serve 2- and 4-bit codes; groups of unequal width when there are two per row (the integer
-    // and the grouped-query kernel).  3-bit streams and the other unequal-group shapes take the scalar kernel.
+    // the integer and the grouped-query kernel serve 2- and 4-bit codes in equal groups, or in two groups of unequal
+    // width per row; everything else (3-bit streams, 4-bit with several query heads or groups of 32, other unequal
+    // groups, 3 and 5-8 query heads per KV head) goes to the tcgen05 kernel
     if (s.k_bits != 3 && s.v_bits != 3) {
         em = launch_partition_mma(s, c, q, a.scale_log2, plan, workspace, stream, overlap, &handled);
         if (em != cudaSuccess) return em;
@@ -542,29 +337,12 @@ cudaError_t launch_attention(const Shape &s, const CachePtrs &c, const __half *q
             em = launch_partition_gqa(s, c, q, a.scale_log2, plan, workspace, stream, overlap, &handled);
             if (em != cudaSuccess) return em;
         }
-        if (!handled && !s.bounded) {
-            em = launch_partition_tc(s, c, q, a.scale_log2, plan, workspace, stream, overlap, &handled);
-            if (em != cudaSuccess) return em;
-        }
     }
     if (!handled) {
-        auto launch_scalar = [&](auto kb, auto vb) {
-            return launch_dependent(partition_kernel<decltype(kb)::value, decltype(vb)::value>, grid, dim3(kThreads), 0, stream,
-                                    overlap, a);
-        };
-        auto with_k = [&](auto kb) {
-            switch (s.v_bits) {
-                case 2: return launch_scalar(kb, std::integral_constant<int, 2>{});
-                case 3: return launch_scalar(kb, std::integral_constant<int, 3>{});
-                default: return launch_scalar(kb, std::integral_constant<int, 4>{});
-            }
-        };
-        switch (s.k_bits) {
-            case 2: em = with_k(std::integral_constant<int, 2>{}); break;
-            case 3: em = with_k(std::integral_constant<int, 3>{}); break;
-            default: em = with_k(std::integral_constant<int, 4>{}); break;
-        }
+        em = launch_partition_tc(s, c, q, a.scale_log2, plan, workspace, stream, overlap, &handled);
+        if (em != cudaSuccess) return em;
     }
+    if (!handled) return cudaErrorInvalidValue;      // every configuration skvq_check_config accepts has a kernel above
     if (em != cudaSuccess) return em;
     if (ev_end) cudaEventRecord(ev_end, stream);
     // merge CTAs may be scheduled while the last partition CTAs still run: they do the window part first and

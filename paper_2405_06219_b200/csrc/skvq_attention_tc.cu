@@ -1,6 +1,7 @@
 // Partition kernel of skvq_decode_attention on the fifth-generation tensor cores (tcgen05.mma, accumulators in
-// tensor memory) for 2-bit K and V with up to 4 query heads per KV head per launch and any group size (Eq. 1,
-// Algorithm 1); scale and zero point stored as fp16 pairs or as E4M3 byte pairs.
+// tensor memory) for 2-, 3- or 4-bit K and V in any mix, up to 4 query heads per KV head per launch, any group size and
+// groups of unequal width (Eq. 1, Algorithm 1); scale and zero point stored as fp16 pairs or as E4M3 byte pairs.  It is
+// the general tensor-core path: whatever the two mma.sync kernels do not cover runs here.
 //
 //   q'.K~_t            = sum_g h_{t,g} (sum_{j in g} q'_j c_{t,j}) + sum_g z_{t,g} (sum_{j in g} q'_j)
 //   sum_t p_t V~_{t,d} = sum_t (p_t h_{t,g(d)}) c_{t,d} + sum_t p_t z_{t,g(d)}
@@ -8,8 +9,9 @@
 // One CTA = 128 token threads (one tile of 128 tokens at a time, one thread per token) and one control warp; three
 // CTAs per SM (128 tensor-memory columns and 69 KB of shared memory each).  The token threads only unpack and do the
 // per-(token, head, group) arithmetic; both contractions run asynchronously on the tensor core:
-//   * a thread turns its token's 32 packed bytes into 128 bytes "4^j * code" (one AND per four codes) and stores them
-//     as a row of the A operand of the score MMA (u8, K-major).  The B operand holds the permuted query of every head
+//   * a thread turns its token's packed row into 128 bytes "weight * code" -- one AND per four codes for 2- and 4-bit
+//     codes (weights 4^j and 16^j: the codes stay where they are in the word), shifts for the 3-bit stream (weight 1) --
+//     and stores them as a row of the A operand of the score MMA (u8, K-major).  The B operand holds the permuted query of every head
 //     as four signed byte digits of a 31-bit fixed-point number with the weight 4^j divided out, so the int32
 //     accumulators are the exact group dot products: one MMA k-step (32 channels) per 32 channels, a fresh set of
 //     16 columns (head, digit) per quantization group.
@@ -40,22 +42,21 @@ constexpr int kSlackLog2 = 8;           // the softmax reference moves only when
 constexpr int kRing = 2;                // slots of each of the two copy rings
 constexpr int kTmemCols = 128;          // allocation: scores in columns [0, 64), value sums in [64, 128)
 constexpr int kScoreCol = 0, kPvCol = 64;
-constexpr int kCtasPerSm = 3;           // by tensor memory (512 columns), shared memory and registers
-constexpr int kFoldTiles = 256;         // 255 * 192 * 128 * 256 < 2^31: the int32 value sums are folded at least this often
+constexpr int kFoldTiles = 256;         // 255 * 240 * 128 * 256 < 2^31: the int32 value sums are folded at least this often
 constexpr uint32_t kLbo = 128;          // bytes between core matrices along K (all operands)
 constexpr uint32_t kSboK = 1024;        // K-major operands: bytes between groups of 8 rows
 constexpr uint32_t kSboMN = 2048;       // MN-major operands: bytes between 16-byte chunks of the M/N extent (128 tokens)
 
 // Shared memory.  The K codes of a tile are needed one tile before everything else of it (its score MMA is issued
 // that far ahead), so they travel in a ring of their own.
-template <int G, bool F8>
+template <int G, int KB, int VB>
 struct TCfg {
     static constexpr int NG = kHeadDim / G;
-    static constexpr int kMetaBytes = F8 ? 2 : 4;                        // {scale, zero} per (token, group): E4M3 bytes or a half2
-    static constexpr int kCodeTile = kTile * kRowBytes;                  // 4096
-    static constexpr int kMetaTile = kTile * NG * kMetaBytes;
-    static constexpr int kVmBytes = kCodeTile + 2 * kMetaTile;           // V codes, K scale/zero, V scale/zero
-    static constexpr int kOffVm = kRing * kCodeTile;
+    static constexpr int kKRow = kHeadDim * KB / 8, kVRow = kHeadDim * VB / 8;   // bytes per packed token row
+    static constexpr int kKTile = kTile * kKRow, kVTile = kTile * kVRow;
+    static constexpr int kMetaTile = kTile * NG * 4;                     // room for half2 pairs; E4M3 pairs use half of it
+    static constexpr int kVmBytes = kVTile + 2 * kMetaTile;              // V codes, K scale/zero, V scale/zero
+    static constexpr int kOffVm = kRing * kKTile;
     static constexpr int kOffKA = kOffVm + kRing * kVmBytes;             // A of the score MMA: [128 tokens][128 bytes]
     static constexpr int kOffQB = kOffKA + kTile * 128;                  // B of the score MMA: [16 (head, digit)][128 bytes]
     static constexpr int kOffVB = kOffQB + 16 * 128;                     // A of the value MMA: [128 tokens][128 byte columns]
@@ -63,7 +64,9 @@ struct TCfg {
     static constexpr int kOffOs = kOffPA + kTile * 64;                   // folded value sums [4][128] fp32, by byte column
     static constexpr int kOffMisc = kOffOs + kHeads * kHeadDim * 4;      // small arrays, see the kernel
     static constexpr int kSmemBytes = kOffMisc + 1024;
+    static constexpr int kCtasPerSm = (KB == 2 && VB == 2) ? 3 : 2;      // by shared memory (69 KB at 2 bits, up to 85 KB otherwise)
     static_assert(kTile * 128 >= kHeads * kHeadDim * 4, "the V operand buffer doubles as query scratch in the prologue");
+    static_assert(kKTile % 16 == 0 && kVTile % 16 == 0, "bulk copies move multiples of 16 bytes");
 };
 
 // ---------------------------------------------------------------- tcgen05 wrappers
@@ -127,11 +130,13 @@ __device__ __forceinline__ void load_words32(const uint32_t *p, uint32_t (&w)[NG
     }
 }
 
-// The {h, z} words of one token as fp16 pairs, from fp16 pairs or from E4M3 byte pairs.
-template <int NG, bool F8>
-__device__ __forceinline__ void load_words(const uint8_t *p, uint32_t (&w)[NG])
+// The {h, z} words of one token as fp16 pairs, from fp16 pairs or (f8) from E4M3 byte pairs; tile = the token rows as
+// they lie in the cache (NG pairs per token).
+template <int NG>
+__device__ __forceinline__ void load_words(const uint8_t *tile, int tok, bool f8, uint32_t (&w)[NG])
 {
-    if constexpr (F8) {
+    if (f8) {
+        const uint8_t *p = tile + tok * NG * 2;
         uint16_t b[NG];
         if constexpr (NG == 4) {
             const uint2 x = *reinterpret_cast<const uint2 *>(p);
@@ -145,26 +150,66 @@ __device__ __forceinline__ void load_words(const uint8_t *p, uint32_t (&w)[NG])
 #pragma unroll
         for (int i = 0; i < NG; ++i) asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(w[i]) : "h"(b[i]));
     } else {
-        load_words32<NG>(reinterpret_cast<const uint32_t *>(p), w);
+        load_words32<NG>(reinterpret_cast<const uint32_t *>(tile + tok * NG * 4), w);
     }
 }
 
-// One token's 32 packed bytes -> 128 bytes 4^j * code.  Byte 16w + 4j + b of the row is code j + 4b of word w (channel
-// 16w + j + 4b) times 4^j; chunk w (16 bytes) goes to dst + w * chunk_stride.
+// One token's packed row -> 128 bytes "weight * code", one per channel, in eight chunks of 16 byte columns; chunk i goes
+// to dst + i * chunk_stride.  Which channel and which weight a byte column carries: column_channel / column_shift.
+//   2 bits: chunk i = word i under the four masks 0x03030303 << 2j: byte 16i + 4j + b = code j + 4b of the word, times 4^j.
+//   4 bits: chunk i = words 2i, 2i+1 under the masks 0x0F0F0F0F, 0xF0F0F0F0: byte 16i + 8v + 4j + b = code 2b + j of word
+//           2i + v, times 16^j.
+//   3 bits: the row is a bit stream; chunk i = channels 16i .. 16i+15 in order, four 3-bit fields spread into the four
+//           bytes of a register (weight 1).
+template <int BITS>
 __device__ __forceinline__ void unpack_row(const uint8_t *packed, uint8_t *dst, uint32_t chunk_stride)
 {
-    const uint4 x0 = *reinterpret_cast<const uint4 *>(packed), x1 = *reinterpret_cast<const uint4 *>(packed + 16);
-    const uint32_t w[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+    constexpr int NW = kHeadDim * BITS / 32;
+    uint32_t w[NW];
 #pragma unroll
-    for (int i = 0; i < 8; ++i)
-        *reinterpret_cast<uint4 *>(dst + i * chunk_stride) =
-            make_uint4(w[i] & 0x03030303u, w[i] & 0x0C0C0C0Cu, w[i] & 0x30303030u, w[i] & 0xC0C0C0C0u);
+    for (int i = 0; i < NW / 4; ++i) {
+        const uint4 x = *reinterpret_cast<const uint4 *>(packed + 16 * i);
+        w[4 * i] = x.x; w[4 * i + 1] = x.y; w[4 * i + 2] = x.z; w[4 * i + 3] = x.w;
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        uint4 o;
+        if constexpr (BITS == 2) {
+            o = make_uint4(w[i] & 0x03030303u, w[i] & 0x0C0C0C0Cu, w[i] & 0x30303030u, w[i] & 0xC0C0C0C0u);
+        } else if constexpr (BITS == 4) {
+            o = make_uint4(w[2 * i] & 0x0F0F0F0Fu, w[2 * i] & 0xF0F0F0F0u, w[2 * i + 1] & 0x0F0F0F0Fu, w[2 * i + 1] & 0xF0F0F0F0u);
+        } else {
+            uint32_t r[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int p = 48 * i + 12 * k, wi = p >> 5, sh = p & 31;      // twelve stream bits from bit p on
+                uint32_t f = w[wi] >> sh;
+                if (sh > 20) f |= w[wi + 1] << (32 - sh);                      // never past the row: p + 12 <= 384
+                f &= 0xFFFu;
+                r[k] = (f & 0x7u) | ((f & 0x38u) << 5) | ((f & 0x1C0u) << 10) | ((f & 0xE00u) << 15);
+            }
+            o = make_uint4(r[0], r[1], r[2], r[3]);
+        }
+        *reinterpret_cast<uint4 *>(dst + i * chunk_stride) = o;
+    }
 }
 
-// Channel and weight exponent of byte column n of an unpacked row (the K index of the score MMA, the N index of the
-// value MMA).
-__device__ __forceinline__ int column_channel(int n) { return 16 * (n >> 4) + ((n >> 2) & 3) + 4 * (n & 3); }
-__device__ __forceinline__ int column_shift(int n) { return 2 * ((n >> 2) & 3); }
+// Channel and weight exponent of byte column n of an unpacked row (the K index of the score MMA, the M index of the
+// value MMA).  A 32-column block always holds the 32 channels of one granule, whatever the width.
+template <int BITS>
+__device__ __forceinline__ int column_channel(int n)
+{
+    if constexpr (BITS == 2) return 16 * (n >> 4) + ((n >> 2) & 3) + 4 * (n & 3);
+    else if constexpr (BITS == 4) return 16 * (n >> 4) + 8 * ((n >> 3) & 1) + 2 * (n & 3) + ((n >> 2) & 1);
+    else return n;
+}
+template <int BITS>
+__device__ __forceinline__ int column_shift(int n)
+{
+    if constexpr (BITS == 2) return 2 * ((n >> 2) & 3);
+    else if constexpr (BITS == 4) return 4 * ((n >> 2) & 1);
+    else return 0;
+}
 
 // Barrier 1: the 128 token threads only (the control warp never joins it).
 __device__ __forceinline__ void token_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
@@ -180,11 +225,13 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
-template <int G, bool F8>
-__global__ void __launch_bounds__(kTile + 32, kCtasPerSm) partition_tc_kernel(MmaArgs a)
+template <int G, int KB, int VB>
+__global__ void __launch_bounds__(kTile + 32, TCfg<G, KB, VB>::kCtasPerSm) partition_tc_kernel(MmaArgs a)
 {
-    using C = TCfg<G, F8>;
+    using C = TCfg<G, KB, VB>;
     constexpr int NG = C::NG;
+    const bool f8 = a.s.meta_fp8 != 0;                    // scale/zero as E4M3 byte pairs
+    const int meta_row = NG * (f8 ? 2 : 4);               // bytes of scale/zero per token and tensor
     extern __shared__ __align__(128) uint8_t smem[];
     const Shape &s = a.s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -217,9 +264,9 @@ __global__ void __launch_bounds__(kTile + 32, kCtasPerSm) partition_tc_kernel(Mm
     float *partials = a.ws + a.plan.hdr_ints;
 
     // ---- shared memory
-    uint8_t *QB = smem + C::kOffQB, *VB = smem + C::kOffVB;
+    uint8_t *QB = smem + C::kOffQB, *VOp = smem + C::kOffVB;
     float *Os = reinterpret_cast<float *>(smem + C::kOffOs);         // [4][128] by MMA column
-    float *qs = reinterpret_cast<float *>(VB);                       // [4][128] permuted query (prologue only)
+    float *qs = reinterpret_cast<float *>(VOp);                      // [4][128] permuted query (prologue only)
     float *sqs_sh = reinterpret_cast<float *>(smem + C::kOffMisc);   // [4][4]  sm_scale*log2(e) * sum_{j in g} q'_j
     float *csc_sh = sqs_sh + 16;                                     // [4]     sm_scale*log2(e) * 2^(e_r - 30)
     int *fexp = reinterpret_cast<int *>(csc_sh + 4);                 // [4]
@@ -274,24 +321,24 @@ __global__ void __launch_bounds__(kTile + 32, kCtasPerSm) partition_tc_kernel(Mm
     // The control warp starts the first copies meanwhile.
     auto rows_of = [&](int i) { return (uint32_t)min(kTile, (q_end - (q_begin + i * kTile) + 63) & ~63); };
     auto issue_k = [&](int i) {       // control lane only (the cache's capacity is a multiple of 64 rows)
-        const uint8_t *k_codes = a.c.k_codes + bh * (size_t)s.cap * kRowBytes;
+        const uint8_t *k_codes = a.c.k_codes + bh * (size_t)s.cap * C::kKRow;
         const uint32_t slot = (tiles_done + i) % kRing, rows = rows_of(i);
-        mbar_expect_tx(bar_k + 8 * slot, rows * kRowBytes);
-        bulk_g2s(smem_u32(smem + slot * C::kCodeTile), k_codes + (size_t)(q_begin + i * kTile) * kRowBytes, rows * kRowBytes,
+        mbar_expect_tx(bar_k + 8 * slot, rows * C::kKRow);
+        bulk_g2s(smem_u32(smem + slot * C::kKTile), k_codes + (size_t)(q_begin + i * kTile) * C::kKRow, rows * C::kKRow,
                  bar_k + 8 * slot);
     };
     auto issue_v = [&](int i) {       // control lane only
-        const uint8_t *v_codes = a.c.v_codes + bh * (size_t)s.cap * kRowBytes;
-        constexpr uint32_t kRowMeta = NG * C::kMetaBytes;
+        const uint8_t *v_codes = a.c.v_codes + bh * (size_t)s.cap * C::kVRow;
+        const uint32_t kRowMeta = (uint32_t)meta_row;
         const uint8_t *k_meta = reinterpret_cast<const uint8_t *>(a.c.k_meta) + bh * (size_t)s.cap * kRowMeta;
         const uint8_t *v_meta = reinterpret_cast<const uint8_t *>(a.c.v_meta) + bh * (size_t)s.cap * kRowMeta;
         const uint32_t slot = (tiles_done + i) % kRing, rows = rows_of(i);
         const int tok0 = q_begin + i * kTile;
         const uint32_t dst = smem_u32(smem + C::kOffVm + slot * C::kVmBytes), bar = bar_v + 8 * slot;
-        mbar_expect_tx(bar, rows * (kRowBytes + 2 * kRowMeta));
-        bulk_g2s(dst, v_codes + (size_t)tok0 * kRowBytes, rows * kRowBytes, bar);
-        bulk_g2s(dst + C::kCodeTile, k_meta + (size_t)tok0 * kRowMeta, rows * kRowMeta, bar);
-        bulk_g2s(dst + C::kCodeTile + C::kMetaTile, v_meta + (size_t)tok0 * kRowMeta, rows * kRowMeta, bar);
+        mbar_expect_tx(bar, rows * (C::kVRow + 2 * kRowMeta));
+        bulk_g2s(dst, v_codes + (size_t)tok0 * C::kVRow, rows * C::kVRow, bar);
+        bulk_g2s(dst + C::kVTile, k_meta + (size_t)tok0 * kRowMeta, rows * kRowMeta, bar);
+        bulk_g2s(dst + C::kVTile + C::kMetaTile, v_meta + (size_t)tok0 * kRowMeta, rows * kRowMeta, bar);
     };
     auto wait_ring = [&](uint32_t bar0, int i) {
         const uint32_t t = tiles_done + i;
@@ -323,10 +370,13 @@ __global__ void __launch_bounds__(kTile + 32, kCtasPerSm) partition_tc_kernel(Mm
         fexp[tid] = e;
         csc_sh[tid] = ldexpf(a.scale_log2, e - 30);
     }
+    // group of every 32-channel granule (two bits each): position / G, or the cache's boundaries
+    const uint32_t kmap = granule_groups(a.c.bounds_k, hk, G, NG), vmap = granule_groups(a.c.bounds_v, hk, G, NG);
     if (tid >= 32 && tid < 32 + kHeads * NG) {
         const int r = (tid - 32) / NG, gg = (tid - 32) % NG;
         float sq = 0.f;
-        for (int j = gg * G; j < (gg + 1) * G; ++j) sq += qs[r * kHeadDim + j];
+        for (int j = 0; j < kHeadDim; ++j)
+            if ((int)((kmap >> (2 * (j >> 5))) & 3u) == gg) sq += qs[r * kHeadDim + j];
         sqs_sh[r * 4 + gg] = sq * a.scale_log2;
     }
     __syncthreads();
@@ -336,16 +386,18 @@ __global__ void __launch_bounds__(kTile + 32, kCtasPerSm) partition_tc_kernel(Mm
         // in which the token threads finish the operands
         if (lane == 0 && n_tiles > 0) {
             const uint64_t dKA = smem_desc(smem_u32(smem + C::kOffKA), kLbo, kSboK), dQB = smem_desc(smem_u32(QB), kLbo, kSboK);
-            const uint64_t dVB = smem_desc(smem_u32(VB), kLbo, kSboMN), dPA = smem_desc(smem_u32(smem + C::kOffPA), kLbo, kSboMN);
+            const uint64_t dVB = smem_desc(smem_u32(VOp), kLbo, kSboMN), dPA = smem_desc(smem_u32(smem + C::kOffPA), kLbo, kSboMN);
             bool ok = true;
             auto scores = [&](int j) {      // score MMA of tile j, once its A operand is complete and the old scores are read
                 const uint32_t n = s_count + j;
                 if (!mbar_wait_bounded(bar_ka, n & 1u)) { ok = false; return; }
                 tc_fence_after();
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    umma_i8(tmem + kScoreCol + 16 * ((32 * ks) / G), dKA + ((ks * 2 * kLbo) >> 4), dQB + ((ks * 2 * kLbo) >> 4), kIdescS,
-                            ((32 * ks) % G) != 0 ? 1u : 0u);
+                for (int ks = 0; ks < 4; ++ks) {      // one k-step = one granule; a group's granules are consecutive
+                    const uint32_t gk = (kmap >> (2 * ks)) & 3u;
+                    const uint32_t acc = (ks > 0 && ((kmap >> (2 * (ks - 1))) & 3u) == gk) ? 1u : 0u;
+                    umma_i8(tmem + kScoreCol + 16 * gk, dKA + ((ks * 2 * kLbo) >> 4), dQB + ((ks * 2 * kLbo) >> 4), kIdescS, acc);
+                }
                 umma_commit(bar_s);
                 if (j + kRing < n_tiles) { proxy_fence(); issue_k(j + kRing); }      // the token threads are done with that slot
             };
@@ -371,8 +423,8 @@ __global__ void __launch_bounds__(kTile + 32, kCtasPerSm) partition_tc_kernel(Mm
     } else {
         // ================================================================ token threads
         {
-            // thread = byte column k of the operand: channel column_channel(k), weight 4^j divided out of the query
-            const int ch = column_channel(tid), sh = column_shift(tid);
+            // thread = byte column k of the operand: channel column_channel(k), its weight divided out of the query
+            const int ch = column_channel<KB>(tid), sh = column_shift<KB>(tid);
             uint8_t *col = QB + (tid >> 4) * kLbo + (tid & 15);
 #pragma unroll
             for (int r = 0; r < kHeads; ++r) {
@@ -420,8 +472,8 @@ __global__ void __launch_bounds__(kTile + 32, kCtasPerSm) partition_tc_kernel(Mm
         // every thread: its token's row of tile i -> A operand of the score MMA, then tell the control warp
         auto build_k = [&](int i) {
             wait_ring(bar_k, i);
-            unpack_row(smem + ((tiles_done + i) % kRing) * C::kCodeTile + tid * kRowBytes,
-                       smem + C::kOffKA + (tid >> 3) * kSboK + (tid & 7) * 16, kLbo);
+            unpack_row<KB>(smem + ((tiles_done + i) % kRing) * C::kKTile + tid * C::kKRow,
+                           smem + C::kOffKA + (tid >> 3) * kSboK + (tid & 7) * 16, kLbo);
             proxy_fence();
             mbar_arrive(bar_ka);
         };
@@ -433,7 +485,7 @@ __global__ void __launch_bounds__(kTile + 32, kCtasPerSm) partition_tc_kernel(Mm
             if (!pv_fresh) {
                 // tensor-memory lane tid = byte column tid of the V rows; its group's 16 columns are (head, digit)
                 int v[16];
-                tmem_ld16(tmem_row + kPvCol + 16 * ((warp * 32) / G), v);
+                tmem_ld16(tmem_row + kPvCol + 16 * ((vmap >> (2 * warp)) & 3u), v);      // the 32 byte columns of warp w are granule w
                 tmem_wait_ld();
                 const float sa = h_bound * (1.0f / (float)(1u << (32 - kSlackLog2)));
 #pragma unroll
@@ -453,8 +505,8 @@ __global__ void __launch_bounds__(kTile + 32, kCtasPerSm) partition_tc_kernel(Mm
         for (int i = 0; i < n_tiles; ++i) {
             const uint32_t n = s_count + i;
             const uint8_t *vm = smem + C::kOffVm + ((tiles_done + i) % kRing) * C::kVmBytes;
-            const uint8_t *Km = vm + C::kCodeTile;                      // [128][NG] {h, z}
-            const uint8_t *Vm = vm + C::kCodeTile + C::kMetaTile;
+            const uint8_t *Km = vm + C::kVTile;                         // [128][NG] {h, z}
+            const uint8_t *Vm = vm + C::kVTile + C::kMetaTile;
             uint8_t *PA = smem + C::kOffPA;
             const int tok = q_begin + i * kTile + tid;
             const bool valid = tok < q_end && tok >= s.n_sink;      // sinks belong to the merge kernel
@@ -470,8 +522,8 @@ __global__ void __launch_bounds__(kTile + 32, kCtasPerSm) partition_tc_kernel(Mm
             for (int gg = 0; gg < H0; ++gg) tmem_ld16(tmem_row + kScoreCol + 16 * gg, va[gg]);
             wait_ring(bar_v, i);
             uint32_t kw[NG], vw[NG];
-            load_words<NG, F8>(Km + tid * NG * C::kMetaBytes, kw);
-            load_words<NG, F8>(Vm + tid * NG * C::kMetaBytes, vw);
+            load_words<NG>(Km, tid, f8, kw);
+            load_words<NG>(Vm, tid, f8, vw);
             tmem_wait_ld();
             int vb[NG - H0 > 0 ? NG - H0 : 1][16];
 #pragma unroll
@@ -566,7 +618,7 @@ __global__ void __launch_bounds__(kTile + 32, kCtasPerSm) partition_tc_kernel(Mm
             }
 
             // ---------------- V tile -> A operand of the value MMA
-            unpack_row(vm + tid * kRowBytes, VB + (tid >> 3) * kLbo + (tid & 7) * 16, kSboMN);
+            unpack_row<VB>(vm + tid * C::kVRow, VOp + (tid >> 3) * kLbo + (tid & 7) * 16, kSboMN);
             fresh_sh = pv_fresh ? 1 : 0;      // every thread writes the same value
             proxy_fence();
             mbar_arrive(bar_pa);
@@ -593,15 +645,15 @@ __global__ void __launch_bounds__(kTile + 32, kCtasPerSm) partition_tc_kernel(Mm
         }
         token_sync();
         {
-            const int ch = column_channel(tid);
-            const float winv = __int_as_float((127 - column_shift(tid)) << 23);      // 4^-j
+            const int ch = column_channel<VB>(tid);
+            const float winv = __int_as_float((127 - column_shift<VB>(tid)) << 23);      // the weight of this byte column, undone
 #pragma unroll
             for (int r = 0; r < kHeads; ++r) {
                 if (r >= R) break;
                 float l = 0.f, z = 0.f;
                 for (int w = 0; w < kWarps; ++w) {
                     l += red[w * 24 + r];
-                    z += red[w * 24 + 8 + r * 4 + ch / G];
+                    z += red[w * 24 + 8 + r * 4 + ((vmap >> (2 * (ch >> 5))) & 3u)];
                 }
                 const bool dead = failed || m_ref[r] == -CUDART_INF_F;
                 float *dst = partials + (((size_t)b * s.Hq + hk * s.rep + a.head0 + r) * n_parts + part) * kPartialStride;
@@ -630,35 +682,50 @@ __global__ void __launch_bounds__(kTile + 32, kCtasPerSm) partition_tc_kernel(Mm
     if (control) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
 }
 
-template <int G, bool F8>
-cudaError_t launch_g(const MmaArgs &a, cudaStream_t stream, bool overlap)
+template <int G, int KB, int VB>
+cudaError_t launch_one(const MmaArgs &a, cudaStream_t stream, bool overlap)
 {
-    using C = TCfg<G, F8>;
+    using C = TCfg<G, KB, VB>;
     static unsigned long long configured = 0;      // one bit per device
-    auto kern = partition_tc_kernel<G, F8>;
+    auto kern = partition_tc_kernel<G, KB, VB>;
     const cudaError_t ec = configure_smem_once(kern, C::kSmemBytes, configured);
     if (ec != cudaSuccess) return ec;
     return launch_dependent(kern, dim3(a.plan.n_slots), dim3(kTile + 32), C::kSmemBytes, stream, overlap, a);
 }
 
+template <int G>
+cudaError_t launch_g(const MmaArgs &a, cudaStream_t stream, bool overlap)
+{
+    switch (a.s.k_bits * 10 + a.s.v_bits) {
+        case 22: return launch_one<G, 2, 2>(a, stream, overlap);
+        case 23: return launch_one<G, 2, 3>(a, stream, overlap);
+        case 24: return launch_one<G, 2, 4>(a, stream, overlap);
+        case 32: return launch_one<G, 3, 2>(a, stream, overlap);
+        case 33: return launch_one<G, 3, 3>(a, stream, overlap);
+        case 34: return launch_one<G, 3, 4>(a, stream, overlap);
+        case 42: return launch_one<G, 4, 2>(a, stream, overlap);
+        case 43: return launch_one<G, 4, 3>(a, stream, overlap);
+        default: return launch_one<G, 4, 4>(a, stream, overlap);
+    }
+}
+
 }  // namespace
 
-// Launches the kernel above when the configuration is covered (2-bit K and V, up to 8 query heads per KV head: one
-// launch per four heads); *handled tells the caller whether it did.
+// Launches the kernel above: every configuration the library accepts is covered (2-, 3- or 4-bit K and V, groups of 32,
+// 64 or 128 channels or of unequal width, up to 8 query heads per KV head: one launch per four heads); *handled tells the
+// caller whether it did.
 cudaError_t launch_partition_tc(const Shape &s, const CachePtrs &c, const __half *q, float scale_log2, const SplitPlan &plan,
                                 float *workspace, cudaStream_t stream, bool overlap, bool *handled)
 {
     *handled = false;
-    if (s.k_bits != 2 || s.v_bits != 2 || s.rep > 2 * kHeads || (s.G != 128 && s.G != 64 && s.G != 32)) return cudaSuccess;
+    if (s.rep > 2 * kHeads || (s.G != 128 && s.G != 64 && s.G != 32)) return cudaSuccess;
     *handled = true;
     for (int head0 = 0; head0 < s.rep; head0 += kHeads) {
         MmaArgs a{s, c, q, scale_log2, plan, workspace};
         a.head0 = head0;
         // a second launch reads the same cache again for the next four heads; it starts when the first has finished
         const bool ov = overlap && head0 == 0;
-        cudaError_t e;
-        if (s.meta_fp8) e = s.G == 128 ? launch_g<128, true>(a, stream, ov) : s.G == 64 ? launch_g<64, true>(a, stream, ov) : launch_g<32, true>(a, stream, ov);
-        else e = s.G == 128 ? launch_g<128, false>(a, stream, ov) : s.G == 64 ? launch_g<64, false>(a, stream, ov) : launch_g<32, false>(a, stream, ov);
+        const cudaError_t e = s.G == 128 ? launch_g<128>(a, stream, ov) : s.G == 64 ? launch_g<64>(a, stream, ov) : launch_g<32>(a, stream, ov);
         if (e != cudaSuccess) return e;
         if (head0 > 0) count_launch(1);
     }

@@ -35,7 +35,7 @@ def test_checked_library_exports_the_same_entry_points(checked_library):
     (2, dict(context=1800, batch=2, n_sink=5), [1800, 1800]),                                       # grouped-query kernel, sinks
     (4, dict(context=900, batch=40, ragged=(1, 900), n_q_heads=2, n_kv_heads=2), None),             # plan kernel, 4-bit, window 256
     (2, dict(context=1000, batch=1, n_q_heads=24, meta_fp8=True), [1000]),                          # tcgen05 kernel
-    (1, dict(context=900, batch=1, n_q_heads=4, n_kv_heads=4, k_bits=3, v_bits=3, group_size=64, group_bounds=(0, 32, 128)), [900]),   # scalar kernel
+    (1, dict(context=900, batch=1, n_q_heads=4, n_kv_heads=4, k_bits=3, v_bits=3, group_size=64, group_bounds=(0, 32, 128)), [900]),   # tcgen05 kernel: 3-bit streams, groups of unequal width
 ])
 def test_decode_path_stays_in_bounds(cfg_i, kw, lens):
     w = CF[cfg_i].scaled(**kw)

@@ -120,7 +120,7 @@ def test_ragged_append_and_overflow_flag():
     (4, dict(context=2777, batch=2, ragged=None, n_q_heads=4, n_kv_heads=4, k_bits=4, v_bits=2), 2777),     # mixed widths
     (4, dict(context=2777, batch=2, ragged=None, n_q_heads=4, n_kv_heads=4, k_bits=2, v_bits=4, group_size=128), 2777),
     (4, dict(context=3100, batch=1, ragged=None, n_q_heads=4, n_kv_heads=4, group_size=128, window=128), 3100),   # 4-bit, one group
-    (4, dict(context=2000, batch=1, ragged=None, n_q_heads=8, n_kv_heads=4), 2000),      # 4-bit with 2 heads per KV head: scalar kernel
+    (4, dict(context=2000, batch=1, ragged=None, n_q_heads=8, n_kv_heads=4), 2000),      # 4-bit with 2 heads per KV head: tcgen05 kernel
     (2, dict(context=5300, batch=2, ragged=None, n_q_heads=12, n_kv_heads=4), 5300),     # 3 heads per KV head, g32: tcgen05 kernel
     (1, dict(context=70000, batch=1, n_q_heads=6, n_kv_heads=2), 70000),                 # 3 heads per KV head, g128, many tiles per CTA
     (2, dict(context=1000, batch=33, ragged=(1, 1000), n_q_heads=3, n_kv_heads=1, group_size=64), 1000),   # 3 heads, g64, plan kernel, short and empty prefixes
@@ -143,9 +143,9 @@ def test_attention_matches_oracle(cfg_i, kw, n):
     (1, dict(context=3000, batch=2, n_kv_heads=4, n_q_heads=4, n_sink=5), 3000),              # integer kernel, 5 sinks as in the paper
     (2, dict(context=2900, batch=1, n_sink=5), 2900),                                         # grouped-query kernel
     (4, dict(context=1400, batch=2, ragged=None, n_kv_heads=4, n_q_heads=4, n_sink=64), 1400),   # 4-bit, a whole tile of sinks
-    (2, dict(context=800, batch=1, n_q_heads=16, n_kv_heads=2, n_sink=7), 800),               # scalar kernel
+    (2, dict(context=800, batch=1, n_q_heads=16, n_kv_heads=2, n_sink=7), 800),               # 8 heads per KV head: two tcgen05 launches
     (2, dict(context=900, batch=2, ragged=None, n_sink=64), 900),                             # grouped-query kernel, first tile all sinks
-    (2, dict(context=700, batch=1, n_q_heads=16, n_kv_heads=2, n_sink=64), 700),              # scalar kernel, first tile all sinks
+    (2, dict(context=700, batch=1, n_q_heads=16, n_kv_heads=2, n_sink=64), 700),              # 8 heads per KV head (two tcgen05 launches), first tile all sinks
     (2, dict(context=1900, batch=1, n_q_heads=6, n_kv_heads=2, n_sink=9), 1900),              # tcgen05 kernel (3 heads per KV head)
     (0, dict(context=130, n_sink=5), 130),                                                    # fewer tokens out of the window than sinks
     (0, dict(context=300, window=0, n_sink=3), 300),
@@ -176,7 +176,7 @@ def test_sinks_stay_fp16_and_attention_matches_oracle(cfg_i, kw, n):
     (1, dict(context=2500, batch=2, n_q_heads=4, n_kv_heads=4, meta_fp8=True), 2500),          # one head per KV head, g128
     (1, dict(context=2100, batch=1, n_q_heads=16, n_kv_heads=2, group_size=64, meta_fp8=True, n_sink=5), 2100),   # 8 heads, g64, sinks
     (4, dict(context=1300, batch=2, ragged=None, n_q_heads=4, n_kv_heads=4, meta_fp8=True), 1300),   # 4-bit g64, integer kernel
-    (4, dict(context=1100, batch=1, ragged=None, n_q_heads=8, n_kv_heads=4, meta_fp8=True), 1100),   # 4-bit, 2 heads per KV head: scalar kernel
+    (4, dict(context=1100, batch=1, ragged=None, n_q_heads=8, n_kv_heads=4, meta_fp8=True), 1100),   # 4-bit, 2 heads per KV head: tcgen05 kernel
     (2, dict(context=1500, batch=1, n_q_heads=24, meta_fp8=True), 1500),                             # 3 heads per KV head: tcgen05 kernel
     (4, dict(context=1500, batch=1, ragged=None, n_q_heads=4, n_kv_heads=4, k_bits=4, v_bits=2, group_size=128, meta_fp8=True), 1500),   # mixed widths
     (0, dict(context=200, meta_fp8=True), 200),
