@@ -375,6 +375,11 @@ def test_adversarial_values_stay_bit_exact():
     (2, dict(context=1700, batch=2, k_bits=3, v_bits=2), 1700),                                                    # 3-bit keys, 2-bit values, g32, GQA
     (4, dict(context=1300, batch=1, ragged=None, n_q_heads=8, n_kv_heads=4, k_bits=4, v_bits=3, group_bounds=(0, 96, 128)), 1300),
     (0, dict(context=700, k_bits=3, v_bits=3, meta_fp8=True), 700),
+    (2, dict(context=2600, batch=1, n_q_heads=24, group_size=64, group_bounds=(0, 96, 128)), 2600),               # 3 heads per KV head, unequal groups
+    (2, dict(context=1400, batch=2, n_q_heads=40, group_size=64, group_bounds=(0, 32, 128), k_bits=3, v_bits=4), 1400),   # 5 heads: two launches, 3-bit keys, 4-bit values
+    (4, dict(context=2300, batch=2, ragged=None, n_q_heads=8, n_kv_heads=2, group_size=32), 2300),               # 4-bit, 4 heads per KV head, group 32
+    (4, dict(context=1900, batch=1, ragged=None, n_q_heads=4, n_kv_heads=4, group_size=32, k_bits=4, v_bits=2), 1900),   # 4-bit keys, 2-bit values, group 32, one head per KV head
+    (1, dict(context=70000, batch=1, n_q_heads=2, n_kv_heads=1, k_bits=3, v_bits=3), 70000),                     # 3-bit, many tiles per CTA: the int32 value sums fold on their own
 ])
 def test_unequal_groups_and_three_bit_codes_bit_exact_cache_and_attention(cfg_i, kw, n):
     w = small(cfg_i, **kw)
