@@ -29,12 +29,13 @@ def needs_build(lib: str = LIB) -> bool:
     return any(os.path.getmtime(p) > t for p in deps)
 
 
-def build_library(force: bool = False, verbose: bool = False, checked: bool = False) -> str:
+def build_library(force: bool = False, verbose: bool = False, checked: bool = False, nvtx: bool = False) -> str:
     """Compile every .cu under csrc/ into paper_2405_06219_b200/libskvq.so; with ``checked`` the debugging build
     (-DSKVQ_CHECKED: every index is compared with its buffer's size, violations set SKVQ_STATUS_BOUNDS) into
-    libskvq_checked.so.  The translation units are compiled side by side (objects under _build/), then linked."""
+    libskvq_checked.so.  ``nvtx`` (with force) compiles NVTX ranges around the entry points into the library being built.
+    The translation units are compiled side by side (objects under _build/), then linked."""
     lib = LIB_CHECKED if checked else LIB
-    if not force and not needs_build(lib):
+    if not force and not nvtx and not needs_build(lib):
         return lib
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     objdir = os.path.join(ROOT, "_build", "checked" if checked else "plain")
@@ -42,6 +43,8 @@ def build_library(force: bool = False, verbose: bool = False, checked: bool = Fa
     flags = [f for f in NVCC_FLAGS if f != "-shared"] + ["-I", os.path.join(ROOT, "include"), "-I", CSRC]
     if checked:
         flags += ["-DSKVQ_CHECKED=1"]
+    if nvtx:
+        flags += ["-DSKVQ_NVTX=1"]
     if verbose:
         flags += ["-Xptxas", "-v"]
 

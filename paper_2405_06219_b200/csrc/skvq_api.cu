@@ -3,6 +3,21 @@
 
 #include "skvq_internal.cuh"
 
+// Profiler ranges around the entry points (header-only NVTX 3), compiled in with -DSKVQ_NVTX: a timeline then shows
+// which kernels belong to which call.  Without the define the macro is empty.
+#ifdef SKVQ_NVTX
+#include <nvtx3/nvToolsExt.h>
+namespace {
+struct NvtxRange {
+    explicit NvtxRange(const char *name) { nvtxRangePushA(name); }
+    ~NvtxRange() { nvtxRangePop(); }
+};
+}  // namespace
+#define SKVQ_RANGE(name) NvtxRange skvq_nvtx_range_(name)
+#else
+#define SKVQ_RANGE(name) do {} while (0)
+#endif
+
 namespace skvq {
 
 static std::atomic<uint64_t> g_launches{0};
@@ -166,6 +181,7 @@ size_t skvq_sink_bytes(const skvq_config *cfg)
 int skvq_quantize_append(const skvq_config *cfg, const skvq_cache *cache, const void *k, const void *v,
                          const int32_t *n_new_per_seq, int32_t n_new, void *cuda_stream)
 {
+    SKVQ_RANGE("skvq_quantize_append");
     int rc = check_cfg(cfg);
     if (rc != SKVQ_OK) return rc;
     CachePtrs c;
@@ -195,6 +211,7 @@ size_t skvq_workspace_size(const skvq_config *cfg, int32_t max_len_hint, int32_t
 int skvq_decode_attention(const skvq_config *cfg, const skvq_cache *cache, const void *q, void *out,
                           const skvq_attn_args *args, void *cuda_stream)
 {
+    SKVQ_RANGE("skvq_decode_attention");
     int rc = check_cfg(cfg);
     if (rc != SKVQ_OK) return rc;
     CachePtrs c;
@@ -229,6 +246,7 @@ int skvq_decode_step_host(const skvq_config *cfg, const skvq_cache *cache, const
                           const void *v_new_host, const void *q_host, void *out_host, void *staging,
                           const skvq_attn_args *args, void *cuda_stream)
 {
+    SKVQ_RANGE("skvq_decode_step_host");
     int rc = check_cfg(cfg);
     if (rc != SKVQ_OK) return rc;
     if (!k_new_host || !v_new_host || !q_host || !out_host || !staging || !args) return SKVQ_ERR_INVALID_ARG;
@@ -287,6 +305,7 @@ int noalloc_scratch(float **out)
 int skvq_decode_attention_noalloc(const skvq_config *cfg, const skvq_cache *cache, const void *q, void *out,
                                   float sm_scale, int32_t max_len_hint, int32_t n_splits, void *cuda_stream)
 {
+    SKVQ_RANGE("skvq_decode_attention_noalloc");
     int rc = check_cfg(cfg);
     if (rc != SKVQ_OK) return rc;
     CachePtrs c;
