@@ -74,6 +74,18 @@ def lib():
     return _lib
 
 
+BITS_TERNARY = 15      # the "1.5-bit" three-level code: five base-3 digits per byte
+
+
+def row_bytes(D: int, bits: int) -> int:
+    """Bytes of one packed row of D codes."""
+    return (D + 4) // 5 if bits == BITS_TERNARY else D * bits // 8
+
+
+def qmax(bits: int) -> int:
+    return 2 if bits == BITS_TERNARY else (1 << bits) - 1
+
+
 def _ptr(a: np.ndarray) -> int:
     assert a.flags["C_CONTIGUOUS"]
     return a.ctypes.data
@@ -123,8 +135,8 @@ def quantize_rows(x: np.ndarray, idx: np.ndarray, alpha: np.ndarray, bits: int, 
     alpha = np.ascontiguousarray(alpha, dtype=np.float32)
     b = _bounds(bounds, D)
     ng = D // group if b is None else len(b) - 1
-    assert idx.shape == (D,) and alpha.shape == (ng,) and (D * bits) % 8 == 0
-    codes = np.zeros((n, D * bits // 8), dtype=np.uint8)
+    assert idx.shape == (D,) and alpha.shape == (ng,) and (bits == BITS_TERNARY or (D * bits) % 8 == 0)
+    codes = np.zeros((n, row_bytes(D, bits)), dtype=np.uint8)
     meta = np.zeros((n, ng, 2), dtype=np.uint16 if meta_fp8 else np.float16)
     lib().orc_quantize_rows(_ptr(x), n, _ptr(idx), _ptr(alpha), D, group, bits, int(meta_fp8), _ptr(codes), _ptr(meta),
                             None if b is None else _ptr(b), ng)
@@ -136,7 +148,7 @@ def dequant_rows(codes: np.ndarray, meta: np.ndarray, bits: int, group: int, met
     codes = np.ascontiguousarray(codes, dtype=np.uint8)
     meta = np.ascontiguousarray(meta, dtype=np.uint16 if meta_fp8 else np.float16)
     n = codes.shape[0]
-    D = codes.shape[1] * 8 // bits
+    D = (meta.shape[1] * group if bounds is None else int(np.asarray(bounds)[-1])) if bits == BITS_TERNARY else codes.shape[1] * 8 // bits
     b = _bounds(bounds, D)
     out = np.zeros((n, D), dtype=np.float64)
     for r in range(n):
@@ -164,8 +176,8 @@ class OracleCache:
         assert self.bounds_k is None or self.bounds_v is None or self.bounds_k.shape == self.bounds_v.shape
         self.cap_q = max(max_tokens - window, 0)
         B, H, D, W = batch, n_kv_heads, head_dim, window
-        self.k_codes = np.zeros((B, H, self.cap_q, D * k_bits // 8), dtype=np.uint8)
-        self.v_codes = np.zeros((B, H, self.cap_q, D * v_bits // 8), dtype=np.uint8)
+        self.k_codes = np.zeros((B, H, self.cap_q, row_bytes(D, k_bits)), dtype=np.uint8)
+        self.v_codes = np.zeros((B, H, self.cap_q, row_bytes(D, v_bits)), dtype=np.uint8)
         self.meta_fp8 = bool(meta_fp8)      # scale/zero as FP8 E4M3: the arrays then hold the byte of each as uint16
         meta_t = np.uint16 if self.meta_fp8 else np.float16
         self.k_meta = np.zeros((B, H, self.cap_q, self.ng, 2), dtype=meta_t)

@@ -344,6 +344,8 @@ def test_algorithmic_bytes_match_stated_sizes():
     (2, 2, [[0, 32, 128], [0, 96, 128]], [[0, 64, 128], [0, 32, 128]]),      # two groups per row, another split per head and tensor
     (3, 3, None, None),                                                     # 3-bit codes, equal groups
     (3, 2, [[0, 16, 40, 128], [0, 100, 120, 128]], [[0, 8, 64, 128], [0, 32, 64, 128]]),
+    (2, 15, None, None),                                                    # 2-bit keys, three-level values (the paper's K2 V1.5)
+    (2, 15, [[0, 32, 128], [0, 96, 128]], [[0, 64, 128], [0, 32, 128]]),
 ])
 def test_attention_with_unequal_groups_and_three_bit_codes_matches_brute_force(bits, v_bits, bk, bv):
     """The cache path (append, single-token appends, attention) with group boundaries and 3-bit streams against the

@@ -18,6 +18,9 @@ GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 def unpack_codes(codes: np.ndarray, bits: int) -> np.ndarray:
     """Independent numpy unpack: code j = bits [(j*bits) mod 8, +bits) of byte (j*bits)//8."""
     n, nbytes = codes.shape
+    if bits == 15:                                                     # three levels, five base-3 digits per byte
+        digits = np.stack([(codes.astype(np.int64) // 3 ** i) % 3 for i in range(5)], axis=2)      # [n, nbytes, 5]
+        return digits.reshape(n, nbytes * 5)[:, :D]
     bitsarr = np.unpackbits(codes, axis=1, bitorder="little")          # [n, nbytes*8], LSB first
     bitsarr = bitsarr.reshape(n, nbytes * 8 // bits, bits)
     weights = (1 << np.arange(bits)).astype(np.int64)
@@ -439,3 +442,50 @@ def test_unequal_groups_cost_what_their_average_size_costs():
     c_e, m_e = orc.quantize_rows(x, ident(), np.ones(2, np.float32), 2, 64, meta_fp8=True)
     assert c_u.shape == c_e.shape and m_u.shape == m_e.shape
     assert (c_u[0].nbytes + m_u[0].size) * 8 / D == pytest.approx(2.25)      # the paper's figure for group 64, FP8 parameters
+
+
+# ------------------------------------------------------------------ the three-level ("1.5-bit") value code (abstract, Sec. 4.2)
+def test_three_level_code_golden_bytes_and_closed_forms():
+    """Five codes per byte in base 3: codes 0,1,2,0,1 -> 0 + 1*3 + 2*9 + 0*27 + 1*81 = 102, and so on with the pattern
+    j mod 3 continuing across bytes; 128 codes take 26 bytes (the last byte holds codes 125, 126, 127 and two zero digits)."""
+    x = (np.arange(D) % 3).astype(np.float16)[None]
+    codes, meta = orc.quantize_rows(x, ident(), np.ones(1, np.float32), 15, D)
+    assert codes.shape == (1, 26) and orc.row_bytes(D, 15) == 26 and orc.qmax(15) == 2
+    want = [sum(((5 * b + i) % 3) * 3 ** i for i in range(5) if 5 * b + i < D) for b in range(26)]
+    assert codes[0].tolist() == want and want[0] == 102
+    assert float(meta[0, 0, 0]) == 1.0 and float(meta[0, 0, 1]) == 0.0            # h = (2 - 0) / 2, z = 0
+    assert np.array_equal(unpack_codes(codes, 15)[0], np.arange(D) % 3)
+    assert np.array_equal(orc.dequant_rows(codes, meta, 15, D)[0], x[0].astype(np.float64))      # three exact levels: lossless
+    # a two-valued group sits on codes 0 and 2; a constant group is degenerate (h = 0)
+    y = np.where(np.arange(D) % 2 == 0, -1.5, 3.0).astype(np.float16)[None]
+    c2, _ = orc.quantize_rows(y, ident(), np.ones(1, np.float32), 15, D)
+    assert np.array_equal(unpack_codes(c2, 15)[0], (np.arange(D) % 2) * 2)
+    c3, m3 = orc.quantize_rows(np.full((1, D), 0.37, np.float16), ident(), np.ones(1, np.float32), 15, D)
+    assert not c3.any() and float(m3[0, 0, 0]) == 0.0
+
+
+@pytest.mark.parametrize("group,alpha,bounds", [(128, 1.0, None), (64, 0.9, None), (32, 0.85, None), (64, 0.9, [0, 32, 128])])
+def test_three_level_codes_are_nearest_level_and_parameters_follow_eq2(group, alpha, bounds):
+    """h = alpha (max - min) / 2, z = alpha min; the code is the nearest of the three levels z, z + h, z + 2h."""
+    x = random_rows(64, 70 + group)
+    ng = D // group
+    codes, meta = orc.quantize_rows(x, ident(), np.full(ng, alpha, np.float32), 15, group, bounds=bounds)
+    c = unpack_codes(codes, 15)
+    assert c.min() >= 0 and c.max() <= 2
+    widths = np.full(ng, group) if bounds is None else np.diff(bounds)
+    h = np.repeat(meta[..., 0].astype(np.float64), widths, axis=1)
+    z = np.repeat(meta[..., 1].astype(np.float64), widths, axis=1)
+    xd = x.astype(np.float64)
+    err = np.abs(h * c + z - xd)
+    best = np.abs(h[..., None] * np.arange(3) + z[..., None] - xd[..., None]).min(axis=2)
+    slack = 4 * np.finfo(np.float32).eps * (np.abs(xd) + np.abs(z) + 2 * h) + 1e-30
+    assert np.all(err <= best + slack)
+    edges = np.concatenate([[0], np.cumsum(widths)])
+    a = float(np.float32(alpha))
+    for g in range(ng):
+        seg = xd[:, edges[g]:edges[g + 1]]
+        h_want = a * (seg.max(1) - seg.min(1)) / 2
+        assert np.all(np.abs(meta[:, g, 0].astype(np.float64) - h_want) <= 0.5 * np.spacing(np.abs(h_want).astype(np.float16)).astype(np.float64) * 1.01 + 1e-12)
+    assert np.array_equal(orc.dequant_rows(codes, meta, 15, group, bounds=bounds), h * c + z)
+    # storage: 26 bytes for 128 codes = 1.625 bits per code (the paper's nominal figure is 1.5)
+    assert codes.shape[1] * 8 / D == 1.625
