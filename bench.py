@@ -464,7 +464,7 @@ def run_config(cfg_i, w0, args, env, main):
     kavg_ms = sum(kern_ms) / len(kern_ms)
     achieved = part_bytes / (kavg_ms * 1e-3) / 1e9
     cavg_ms = sum(call_ms) / len(call_ms)
-    plain = not (args.batch or args.context or args.sinks or args.q_heads or args.meta_fp8 or args.splits)
+    plain = not (args.batch or args.context or args.sinks or args.q_heads or args.meta_fp8 or args.splits or args.k_bits or args.v_bits)
     rec = {
         "workload": f"configs[{cfg_i}] {w.name}",
         "config": {"workload": f"configs[{cfg_i}] {w.name}", "batch": w.batch, "n_q_heads": w.n_q_heads,
@@ -519,6 +519,8 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (small profiling cases)")
     ap.add_argument("--context", type=int, default=0, help="override the context length (small profiling cases)")
     ap.add_argument("--q-heads", type=int, default=0, help="override the number of query heads (other grouped-query ratios)")
+    ap.add_argument("--k-bits", type=int, default=0, help="override the key code width (2, 3, 4)")
+    ap.add_argument("--v-bits", type=int, default=0, help="override the value code width (2, 3, 4; 15 = three-level '1.5-bit' codes)")
     ap.add_argument("--meta-fp8", action="store_true",
                     help="scale and zero point stored in FP8 E4M3 instead of fp16 (Sec. 4.1; 2.5 bits per element at g32)")
     ap.add_argument("--sinks", type=int, default=0,
@@ -551,6 +553,10 @@ def main():
             w0 = w0.scaled(n_q_heads=args.q_heads)
         if args.meta_fp8:
             w0 = w0.scaled(meta_fp8=True)
+        if args.k_bits:
+            w0 = w0.scaled(k_bits=args.k_bits)
+        if args.v_bits:
+            w0 = w0.scaled(v_bits=args.v_bits)
         return w0
 
     if args.impl == "reference":
@@ -572,7 +578,7 @@ def main():
         gpu_id = "GPU-" + str(torch.cuda.get_device_properties(local_rank).uuid)
     except Exception:
         gpu_id = str(local_rank)
-    others = [] if (args.config >= 0 or args.no_others or world > 1 or args.batch or args.context or args.q_heads) \
+    others = [] if (args.config >= 0 or args.no_others or world > 1 or args.batch or args.context or args.q_heads or args.k_bits or args.v_bits) \
         else list(OTHER_CONFIGS)
     with ClockSampler(gpu_id) as clocks:
         env = {"torch": torch, "dist": dist, "binding": binding, "sharding": sharding, "workloads": workloads,

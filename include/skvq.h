@@ -39,7 +39,7 @@ extern "C" {
 
 #define SKVQ_OK 0
 #define SKVQ_ERR_INVALID_ARG (-1) /* NULL where a buffer is required, negative size, ... */
-#define SKVQ_ERR_UNSUPPORTED (-2) /* head_dim != 128, bits not in {2,3,4}, G not in {32,64,128}, Hq % Hkv != 0, Hq/Hkv > 8 */
+#define SKVQ_ERR_UNSUPPORTED (-2) /* head_dim != 128, k_bits not in {2,3,4}, v_bits not in {2,3,4,15}, G not in {32,64,128}, Hq % Hkv != 0, Hq/Hkv > 8 */
 #define SKVQ_ERR_MISALIGNED (-3)  /* a device buffer is not 16-byte aligned */
 #define SKVQ_ERR_CAPACITY (-4)    /* host-visible overflow: n_new or max_len_hint beyond max_tokens */
 #define SKVQ_ERR_WORKSPACE (-5)   /* workspace missing or smaller than skvq_workspace_size() */
@@ -60,6 +60,11 @@ extern "C" {
 /* Group boundaries (skvq_cache::group_bounds_*) are multiples of this many channels. */
 #define SKVQ_GROUP_GRANULE 32
 
+/* v_bits value of the "1.5-bit" setting for values (abstract; Sec. 4.2: keys at 2 bits, values at 1.5 bits): three
+ * levels per code (2^1.5 = 2.83 rounds to 3), five codes per byte in base 3.  The paper gives neither the levels nor the
+ * storage of that setting; this is the library's reading of it. */
+#define SKVQ_BITS_TERNARY 15
+
 /* Shape and quantization settings (host struct). */
 typedef struct skvq_config {
     int32_t batch;       /* B >= 1 */
@@ -67,7 +72,7 @@ typedef struct skvq_config {
     int32_t n_kv_heads;  /* Hkv */
     int32_t head_dim;    /* D, must be 128 */
     int32_t k_bits;      /* 2, 3 or 4 (3: the 3-bit setting of the paper's comparison with KVQuant, Sec. 4.3) */
-    int32_t v_bits;      /* 2, 3 or 4 */
+    int32_t v_bits;      /* 2, 3, 4 or SKVQ_BITS_TERNARY (three-level codes, 1.625 bits per element stored) */
     int32_t group_size;  /* G: 32, 64 or 128; a row has ng = D/G groups that share scale/zero: equal runs of G consecutive
                             (reordered) channels, or, with skvq_cache::group_bounds_*, ng runs of unequal width whose
                             AVERAGE width is G (Sec. 4.2: the number of groups is kept, not their size) */
@@ -85,7 +90,10 @@ typedef struct skvq_config {
  * Layouts are row-major:
  *   k_codes/v_codes  uint8   [B][Hkv][cap][D*bits/8]  a row is a little-endian bit stream: code j = bits [j*bits, (j+1)*bits)
  *                                                     of the row, j counted in reordered order (2- and 4-bit codes never
- *                                                     cross a byte; a 3-bit code may: 8 codes per 3 bytes, 48-byte rows)
+ *                                                     cross a byte; a 3-bit code may: 8 codes per 3 bytes, 48-byte rows).
+ *                                                     v_bits = SKVQ_BITS_TERNARY: (D+4)/5 = 26 bytes per row, code j is
+ *                                                     base-3 digit j % 5 (weight 3^(j % 5)) of byte j / 5; the two unused
+ *                                                     digits of the last byte are 0
  *   k_meta/v_meta    half2   [B][Hkv][cap][ng]        {scale h, zero z}; dequantized x^ = h*code + z.  With meta_fp8:
  *                    uint8   [B][Hkv][cap][ng][2]     {E4M3 byte of h, E4M3 byte of z} (1 sign, 4 exponent bits with
  *                                                     bias 7, 3 mantissa bits, no infinities, largest finite 448;
@@ -165,8 +173,9 @@ size_t skvq_sink_bytes(const skvq_config *cfg);
  * Sequence b receives n_b = n_new_per_seq ? n_new_per_seq[b] : n_new tokens (0 <= n_b <= n_new).
  * With L0 = lengths[b], L1 = L0 + n_b: every token in [max(L0-W,0), max(L1-W,0)) is reordered
  * (stored[j] = x[idx[j]]), split into groups of G channels and quantized per group:
- *   lo = alpha*min, hi = alpha*max, h = fp16((hi-lo)/(2^bits-1)), z = fp16(lo),
- *   code = clamp(rint((x - z)/h), 0, 2^bits-1)   (fp32, IEEE division, ties to even; h == 0 -> code 0)
+ *   lo = alpha*min, hi = alpha*max, h = fp16((hi-lo)/qmax), z = fp16(lo),
+ *   code = clamp(rint((x - z)/h), 0, qmax)   (fp32, IEEE division, ties to even; h == 0 -> code 0;
+ *                                             qmax = 2^bits-1, or 2 for the three-level codes)
  * (min, max and alpha are those of the channel's group: equal runs of G channels, or the runs given by group_bounds_*)
  * the last min(L1, W) tokens are kept in fp16 in the ring, and lengths[b] becomes L1.
  * Exception (Sec. 3.2, the filter mask of Algorithm 1): a token at a position below n_sink is copied, reordered,

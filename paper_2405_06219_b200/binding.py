@@ -24,6 +24,7 @@ SKVQ_STATUS_COPY_TIMEOUT = 2
 SKVQ_STATUS_BOUNDS = 4
 SKVQ_TOKEN_ALIGN = 64
 SKVQ_GROUP_GRANULE = 32
+SKVQ_BITS_TERNARY = 15
 
 EXPORTS = ["skvq_version", "skvq_strerror", "skvq_launch_count", "skvq_check_config", "skvq_quant_capacity",
            "skvq_cache_sizes", "skvq_sink_bytes", "skvq_quantize_append", "skvq_workspace_size", "skvq_decode_attention",
@@ -203,8 +204,9 @@ class SkvqCache:
         sizes = skvq_cache_sizes(self.cfg)
         B, H, W, D = batch, n_kv_heads, window, head_dim
         dev = self.device
-        self.k_codes = torch.zeros((B, H, self.cap, D * k_bits // 8), dtype=torch.uint8, device=dev)
-        self.v_codes = torch.zeros((B, H, self.cap, D * v_bits // 8), dtype=torch.uint8, device=dev)
+        rows = B * H * self.cap
+        self.k_codes = torch.zeros((B, H, self.cap, sizes[0] // rows), dtype=torch.uint8, device=dev)
+        self.v_codes = torch.zeros((B, H, self.cap, sizes[1] // rows), dtype=torch.uint8, device=dev)
         meta_t = torch.uint8 if meta_fp8 else torch.float16      # {h, z} per (token, group): E4M3 bytes or fp16
         self.k_meta = torch.zeros((B, H, self.cap, self.ng, 2), dtype=meta_t, device=dev)
         self.v_meta = torch.zeros((B, H, self.cap, self.ng, 2), dtype=meta_t, device=dev)

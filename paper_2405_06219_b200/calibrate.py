@@ -90,7 +90,7 @@ def fake_quant(xr: np.ndarray, bounds: np.ndarray, alpha: np.ndarray, bits: int)
     uses: lo = alpha*min, hi = alpha*max, h = fp16((hi - lo)/qmax), z = fp16(lo), code = clip(rint((x - z)/h)),
     x^ = h*code + z; fp32 throughout, returned as float64."""
     xr = np.asarray(xr, dtype=np.float16).astype(np.float32)
-    qmax = np.float32((1 << bits) - 1)
+    qmax = np.float32(2 if bits == 15 else (1 << bits) - 1)      # 15: the three-level code
     out = np.empty(xr.shape, dtype=np.float64)
     for g in range(len(bounds) - 1):
         a, b = int(bounds[g]), int(bounds[g + 1])

@@ -30,7 +30,7 @@ static int check_cfg(const skvq_config *c)
         return SKVQ_ERR_INVALID_ARG;
     if (c->batch > 65535 || c->n_kv_heads > 65535) return SKVQ_ERR_UNSUPPORTED;
     if (c->head_dim != kHeadDim) return SKVQ_ERR_UNSUPPORTED;
-    if (c->k_bits < 2 || c->k_bits > 4 || c->v_bits < 2 || c->v_bits > 4) return SKVQ_ERR_UNSUPPORTED;
+    if (c->k_bits < 2 || c->k_bits > 4 || ((c->v_bits < 2 || c->v_bits > 4) && c->v_bits != kTernary)) return SKVQ_ERR_UNSUPPORTED;
     if (c->group_size != 32 && c->group_size != 64 && c->group_size != 128) return SKVQ_ERR_UNSUPPORTED;
     if (c->n_q_heads % c->n_kv_heads != 0) return SKVQ_ERR_UNSUPPORTED;
     if (c->n_q_heads / c->n_kv_heads > kMaxRep) return SKVQ_ERR_UNSUPPORTED;
@@ -163,8 +163,8 @@ int skvq_cache_sizes(const skvq_config *cfg, size_t bytes_out[6])
     if (!bytes_out) return SKVQ_ERR_INVALID_ARG;
     const Shape s = make_shape(cfg);
     const size_t rows = (size_t)s.B * s.Hkv * s.cap;
-    bytes_out[0] = rows * (kHeadDim * s.k_bits / 8);
-    bytes_out[1] = rows * (kHeadDim * s.v_bits / 8);
+    bytes_out[0] = rows * packed_row_bytes(s.k_bits);
+    bytes_out[1] = rows * packed_row_bytes(s.v_bits);
     bytes_out[2] = rows * s.ng * (s.meta_fp8 ? 2 : sizeof(__half2));
     bytes_out[3] = bytes_out[2];
     bytes_out[4] = (size_t)s.B * s.Hkv * s.W * kHeadDim * sizeof(__half);

@@ -1,5 +1,5 @@
 // skvq_quantize_append: channel reorder, group-wise clipped dynamic asymmetric quantization,
-// 2/4-bit packing and sliding-window bookkeeping (Sec. 3.1 Eq. 2, Sec. 3.2, Algorithm 1).
+// 2/3/4-bit and three-level packing and sliding-window bookkeeping (Sec. 3.1 Eq. 2, Sec. 3.2, Algorithm 1).
 //
 // Work decomposition.  For sequence b with L0 tokens before and L1 = L0 + n_b after the call:
 //   "evict" items   tokens t in [max(L0-W,0), min(L0, L1-W)): still in the fp16 ring (already in
@@ -53,17 +53,17 @@ __device__ __forceinline__ void bulk_range(int L0, int n_sink, int q_end, int &f
 // that have a quotient next to a rounding boundary, and for 3-bit codes.  Inlined on purpose: as a separate function
 // it takes the 16 values through local memory, which every caller then pays for on the fast path too (measured:
 // 1.88 -> 2.13 TB/s of prefill input).  The 16 fields are a little-endian bit stream of 16 * BITS bits in words[0],
-// words[1].
+// words[1]; the three-level codes come out as 16 two-bit fields (the caller packs them in base 3).
 template <int BITS>
 __device__ __forceinline__ void quantize16_exact(const float (&x)[16], float zf, float hf, uint32_t (&words)[2])
 {
-    constexpr int qmax = (1 << BITS) - 1;
+    constexpr int qmax = code_max(BITS), FIELD = BITS == kTernary ? 2 : BITS;
     unsigned long long stream = 0ull;
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
         float c = rintf(__fdiv_rn(__fsub_rn(x[j], zf), hf));
         c = fminf(fmaxf(c, 0.0f), (float)qmax);
-        stream |= (unsigned long long)(uint32_t)(int)c << (j * BITS);
+        stream |= (unsigned long long)(uint32_t)(int)c << (j * FIELD);
     }
     words[0] = (uint32_t)stream;
     words[1] = (uint32_t)(stream >> 32);
@@ -95,7 +95,7 @@ __device__ __forceinline__ void quantize16(const float (&x)[16], float alpha, in
     // The 8 lanes that own one row always take the same path, so they are the shuffle's member set
     // (K and V rows may use different bit widths and therefore different instantiations).
     const uint32_t seg_mask = 0xFFu << ((threadIdx.x & 31) & 24);
-    constexpr int qmax = (1 << BITS) - 1;
+    constexpr int qmax = code_max(BITS);
     float mn = x[0], mx = x[0];
 #pragma unroll
     for (int j = 1; j < 16; ++j) {
@@ -142,9 +142,10 @@ __device__ __forceinline__ void quantize16(const float (&x)[16], float alpha, in
     const float zf = __high2float(hz);
     words[0] = 0u;
     words[1] = 0u;
-    if constexpr (BITS == 3) {
-        // 3-bit fields do not tile a 32-bit word; this width takes the defining formula directly
-        if (hf != 0.0f) quantize16_exact<3>(x, zf, hf, words);
+    if constexpr (BITS == 3 || BITS == kTernary) {
+        // 3-bit fields do not tile a 32-bit word, three-level codes are packed across lanes afterwards; these widths
+        // take the defining formula directly
+        if (hf != 0.0f) quantize16_exact<BITS>(x, zf, hf, words);
     } else if (hf != 0.0f) {
         // The code is clamp(rint(RN((x - z) / h)), 0, qmax) with IEEE division.  One division per element makes
         // this path bound by the special-function unit, so the quotient is first formed as d * RN(1/h): that is
@@ -205,7 +206,7 @@ __global__ void __launch_bounds__(kAppendThreads) append_kernel(AppendArgs a)
     const int tok_sel = lane >> 4;
 
     const int bits = is_v ? s.v_bits : s.k_bits;
-    const int row_bytes = kHeadDim * bits / 8;
+    const int row_bytes = packed_row_bytes(bits);
     const size_t bh = (size_t)b * s.Hkv + h;
     uint8_t *codes = (is_v ? a.c.v_codes : a.c.k_codes) + bh * (size_t)s.cap * row_bytes;
     __half2 *meta = (is_v ? a.c.v_meta : a.c.k_meta);      // two bytes per (token, group) with FP8 parameters
@@ -293,7 +294,25 @@ __global__ void __launch_bounds__(kAppendThreads) append_kernel(AppendArgs a)
             uint32_t hz;
             if (bits == 2) quantize16<2>(x, alpha, lanes_per_group, f8, words, hz, lane_lo, lane_hi);
             else if (bits == 3) quantize16<3>(x, alpha, lanes_per_group, f8, words, hz, lane_lo, lane_hi);
+            else if (bits == kTernary) quantize16<kTernary>(x, alpha, lanes_per_group, f8, words, hz, lane_lo, lane_hi);
             else quantize16<4>(x, alpha, lanes_per_group, f8, words, hz, lane_lo, lane_hi);
+            uint32_t tern = 0u;      // three-level codes: bytes 4*sub .. 4*sub+3 of the row
+            if (bits == kTernary) {
+                // Byte n carries codes 5n .. 5n+4 as base-3 digits.  They lie in the two-bit fields of at most two
+                // neighbouring lanes of the row; all 8 lanes of the row take part in the shuffles.
+                const uint32_t seg_mask = 0xFFu << (lane & 24);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int first = 5 * (4 * sub + k);                  // first code of the byte; beyond the row for bytes >= 26
+                    const int src = min(first >> 4, 7);
+                    const uint32_t lo = __shfl_sync(seg_mask, words[0], (lane & 24) + src);
+                    uint32_t hi = __shfl_sync(seg_mask, words[0], (lane & 24) + min(src + 1, 7));
+                    if (src == 7) hi = 0u;                                // codes past channel 127 do not exist: digits 0
+                    const uint32_t f = (uint32_t)((((unsigned long long)hi << 32) | lo) >> (2 * (first & 15))) & 0x3FFu;
+                    const uint32_t byte = (f & 3u) + 3u * ((f >> 2) & 3u) + 9u * ((f >> 4) & 3u) + 27u * ((f >> 6) & 3u) + 81u * ((f >> 8) & 3u);
+                    tern |= byte << (8 * k);
+                }
+            }
             if (do_quant && !SKVQ_IN_BOUNDS(t >= 0 && t < s.cap && (from_ring || (t - L0 >= 0 && t - L0 < a.n_new)), a.c.status)) do_quant = false;
             if (do_quant && t < s.n_sink) {
                 // an attention sink (Sec. 3.2 filter rule): its reordered fp16 row is kept as it is
@@ -313,6 +332,10 @@ __global__ void __launch_bounds__(kAppendThreads) append_kernel(AppendArgs a)
                     p[0] = (uint16_t)words[0];
                     p[1] = (uint16_t)(words[0] >> 16);
                     p[2] = (uint16_t)words[1];
+                } else if (bits == kTernary) {      // 26 bytes per row, rows 2-byte aligned: lanes 0-5 hold four bytes, lane 6 two
+                    uint16_t *p = reinterpret_cast<uint16_t *>(codes_row) + 2 * sub;
+                    if (sub < 7) p[0] = (uint16_t)tern;
+                    if (sub < 6) p[1] = (uint16_t)(tern >> 16);
                 } else {
                     reinterpret_cast<uint2 *>(codes_row)[sub] = make_uint2(words[0], words[1]);
                 }
@@ -456,7 +479,7 @@ cudaError_t launch_append(const Shape &s, const CachePtrs &c, const __half *k, c
 {
     if (n_new <= 0) return cudaSuccess;
     // the tile kernel serves 2- and 4-bit codes in equal groups; everything else goes through append_kernel
-    const bool bulk = n_new >= kBulkTok && !s.bounded && s.k_bits != 3 && s.v_bits != 3;
+    const bool bulk = n_new >= kBulkTok && !s.bounded && plain_width(s.k_bits) && plain_width(s.v_bits);
     AppendArgs a{s, c, k, v, n_new_per_seq, n_new, bulk ? 1 : 0};
     // what append_kernel keeps: evictions (at most W), and new tokens outside the bulk tiles (fewer than W + 128
     // when there are bulk tiles, all of them otherwise)

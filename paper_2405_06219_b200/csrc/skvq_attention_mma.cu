@@ -521,7 +521,7 @@ cudaError_t launch_partition_mma(const Shape &s, const CachePtrs &c, const __hal
                                  const SplitPlan &plan, float *workspace, cudaStream_t stream, bool overlap, bool *handled)
 {
     *handled = false;
-    if (s.rep != 1 || (s.G != 64 && s.G != 128) || s.k_bits == 3 || s.v_bits == 3) return cudaSuccess;
+    if (s.rep != 1 || (s.G != 64 && s.G != 128) || !plain_width(s.k_bits) || !plain_width(s.v_bits)) return cudaSuccess;
     if (s.bounded && s.G != 64) return cudaSuccess;
     MmaArgs a{s, c, q, scale_log2, plan, workspace};
     *handled = true;

@@ -1,6 +1,7 @@
 // Partition kernel of skvq_decode_attention on the fifth-generation tensor cores (tcgen05.mma, accumulators in
-// tensor memory) for 2-, 3- or 4-bit K and V in any mix, up to 4 query heads per KV head per launch, any group size and
-// groups of unequal width (Eq. 1, Algorithm 1); scale and zero point stored as fp16 pairs or as E4M3 byte pairs.  It is
+// tensor memory) for 2-, 3- or 4-bit K and V in any mix and three-level ("1.5-bit") V, up to 4 query heads per KV head
+// per launch, any group size and groups of unequal width (Eq. 1, Algorithm 1); scale and zero point stored as fp16 pairs
+// or as E4M3 byte pairs.  It is
 // the general tensor-core path: whatever the two mma.sync kernels do not cover runs here.
 //
 //   q'.K~_t            = sum_g h_{t,g} (sum_{j in g} q'_j c_{t,j}) + sum_g z_{t,g} (sum_{j in g} q'_j)
@@ -52,7 +53,7 @@ constexpr uint32_t kSboMN = 2048;       // MN-major operands: bytes between 16-b
 template <int G, int KB, int VB>
 struct TCfg {
     static constexpr int NG = kHeadDim / G;
-    static constexpr int kKRow = kHeadDim * KB / 8, kVRow = kHeadDim * VB / 8;   // bytes per packed token row
+    static constexpr int kKRow = packed_row_bytes(KB), kVRow = packed_row_bytes(VB);   // bytes per packed token row
     static constexpr int kKTile = kTile * kKRow, kVTile = kTile * kVRow;
     static constexpr int kMetaTile = kTile * NG * 4;                     // room for half2 pairs; E4M3 pairs use half of it
     static constexpr int kVmBytes = kVTile + 2 * kMetaTile;              // V codes, K scale/zero, V scale/zero
@@ -194,6 +195,39 @@ __device__ __forceinline__ void unpack_row(const uint8_t *packed, uint8_t *dst, 
     }
 }
 
+// Three-level codes: one token's 26 bytes (five base-3 digits each; the row is only 2-byte aligned) -> 128 code bytes in
+// channel order (weight 1), through a table of the five digits of every byte value: lut[v] = {digits 0-3 in the four
+// bytes of .x, digit 4 in the low byte of .y}.  The table's 5-byte pieces are joined into 4-byte registers by byte
+// permutes whose selectors are compile-time constants after unrolling.
+__device__ __forceinline__ void unpack_row_ternary(const uint8_t *packed, uint8_t *dst, uint32_t chunk_stride, const uint2 *lut)
+{
+    constexpr int NB = packed_row_bytes(kTernary);      // 26
+    uint32_t lo[NB], hi[NB];
+    const uint16_t *p = reinterpret_cast<const uint16_t *>(packed);
+#pragma unroll
+    for (int i = 0; i < NB / 2; ++i) {
+        const uint32_t two = p[i];
+        const uint2 e0 = lut[two & 255u], e1 = lut[two >> 8];
+        lo[2 * i] = e0.x; hi[2 * i] = e0.y;
+        lo[2 * i + 1] = e1.x; hi[2 * i + 1] = e1.y;
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        uint32_t r[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int pos = 16 * i + 4 * k, n = pos / 5, off = pos % 5;      // channels pos .. pos+3 = digits off .. of byte n, then of byte n+1
+            const int n1 = n + 1 < NB ? n + 1 : n;                          // off > 1 implies n + 1 < NB (pos + 3 <= 127)
+            r[k] = off == 0 ? lo[n]
+                 : off == 1 ? __byte_perm(lo[n], hi[n], 0x4321)
+                 : off == 2 ? __byte_perm(__byte_perm(lo[n], hi[n], 0x0432), lo[n1], 0x4210)
+                 : off == 3 ? __byte_perm(__byte_perm(lo[n], hi[n], 0x0043), lo[n1], 0x5410)
+                            : __byte_perm(hi[n], lo[n1], 0x6540);
+        }
+        *reinterpret_cast<uint4 *>(dst + i * chunk_stride) = make_uint4(r[0], r[1], r[2], r[3]);
+    }
+}
+
 // Channel and weight exponent of byte column n of an unpacked row (the K index of the score MMA, the M index of the
 // value MMA).  A 32-column block always holds the 32 channels of one granule, whatever the width.
 template <int BITS>
@@ -250,6 +284,11 @@ __global__ void __launch_bounds__(kTile + 32, TCfg<G, KB, VB>::kCtasPerSm) parti
     __shared__ uint32_t tmem_sh;
     __shared__ SlotWalker walk;      // only thread 0 touches it
     __shared__ __align__(16) int hdr_sh[kPlanSmemInts];
+    __shared__ uint2 digits_sh[VB == kTernary ? 256 : 1];      // the five base-3 digits of every byte value
+    if constexpr (VB == kTernary) {
+        for (int v = tid; v < 256; v += kTile + 32)
+            digits_sh[v] = make_uint2((v % 3) | ((v / 3 % 3) << 8) | ((v / 9 % 3) << 16) | ((v / 27 % 3) << 24), v / 81);
+    }
     if (a.plan.in_kernel) {
         if (warp == 0) plan_in_warp(a.c.lengths, s.B, s.Hkv, s.W, a.plan.lq_cap, a.plan.n_slots, hdr_sh);
         __syncthreads();
@@ -618,7 +657,8 @@ __global__ void __launch_bounds__(kTile + 32, TCfg<G, KB, VB>::kCtasPerSm) parti
             }
 
             // ---------------- V tile -> A operand of the value MMA
-            unpack_row<VB>(vm + tid * C::kVRow, VOp + (tid >> 3) * kLbo + (tid & 7) * 16, kSboMN);
+            if constexpr (VB == kTernary) unpack_row_ternary(vm + tid * C::kVRow, VOp + (tid >> 3) * kLbo + (tid & 7) * 16, kSboMN, digits_sh);
+            else unpack_row<VB>(vm + tid * C::kVRow, VOp + (tid >> 3) * kLbo + (tid & 7) * 16, kSboMN);
             fresh_sh = pv_fresh ? 1 : 0;      // every thread writes the same value
             proxy_fence();
             mbar_arrive(bar_pa);
@@ -696,22 +736,26 @@ cudaError_t launch_one(const MmaArgs &a, cudaStream_t stream, bool overlap)
 template <int G>
 cudaError_t launch_g(const MmaArgs &a, cudaStream_t stream, bool overlap)
 {
-    switch (a.s.k_bits * 10 + a.s.v_bits) {
-        case 22: return launch_one<G, 2, 2>(a, stream, overlap);
-        case 23: return launch_one<G, 2, 3>(a, stream, overlap);
-        case 24: return launch_one<G, 2, 4>(a, stream, overlap);
-        case 32: return launch_one<G, 3, 2>(a, stream, overlap);
-        case 33: return launch_one<G, 3, 3>(a, stream, overlap);
-        case 34: return launch_one<G, 3, 4>(a, stream, overlap);
-        case 42: return launch_one<G, 4, 2>(a, stream, overlap);
-        case 43: return launch_one<G, 4, 3>(a, stream, overlap);
-        default: return launch_one<G, 4, 4>(a, stream, overlap);
+    switch (a.s.k_bits * 100 + a.s.v_bits) {
+        case 202: return launch_one<G, 2, 2>(a, stream, overlap);
+        case 203: return launch_one<G, 2, 3>(a, stream, overlap);
+        case 204: return launch_one<G, 2, 4>(a, stream, overlap);
+        case 215: return launch_one<G, 2, kTernary>(a, stream, overlap);
+        case 302: return launch_one<G, 3, 2>(a, stream, overlap);
+        case 303: return launch_one<G, 3, 3>(a, stream, overlap);
+        case 304: return launch_one<G, 3, 4>(a, stream, overlap);
+        case 315: return launch_one<G, 3, kTernary>(a, stream, overlap);
+        case 402: return launch_one<G, 4, 2>(a, stream, overlap);
+        case 403: return launch_one<G, 4, 3>(a, stream, overlap);
+        case 404: return launch_one<G, 4, 4>(a, stream, overlap);
+        case 415: return launch_one<G, 4, kTernary>(a, stream, overlap);
+        default: return cudaErrorInvalidValue;
     }
 }
 
 }  // namespace
 
-// Launches the kernel above: every configuration the library accepts is covered (2-, 3- or 4-bit K and V, groups of 32,
+// Launches the kernel above: every configuration the library accepts is covered (2-, 3- or 4-bit K and V, three-level V, groups of 32,
 // 64 or 128 channels or of unequal width, up to 8 query heads per KV head: one launch per four heads); *handled tells the
 // caller whether it did.
 cudaError_t launch_partition_tc(const Shape &s, const CachePtrs &c, const __half *q, float scale_log2, const SplitPlan &plan,

@@ -14,6 +14,12 @@ constexpr int kMaxRep = 8;            // query heads per KV head supported by th
 constexpr int kPartialStride = 132;   // floats per split partial: o'[128], m (log2 domain), l, 2 pad
 constexpr int kGranule = SKVQ_GROUP_GRANULE;          // group boundaries are multiples of this many channels
 constexpr int kGranules = kHeadDim / kGranule;
+constexpr int kTernary = SKVQ_BITS_TERNARY;           // the width value of the three-level code
+
+// Bytes of one packed row of kHeadDim codes; largest code; is the width one of the plain power-of-two fields (2, 4)?
+__host__ __device__ constexpr int packed_row_bytes(int bits) { return bits == kTernary ? (kHeadDim + 4) / 5 : kHeadDim * bits / 8; }
+__host__ __device__ constexpr int code_max(int bits) { return bits == kTernary ? 2 : (1 << bits) - 1; }
+__host__ __device__ constexpr bool plain_width(int bits) { return bits == 2 || bits == 4; }
 
 // Everything the kernels need, by value.
 struct Shape {

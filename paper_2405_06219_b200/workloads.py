@@ -160,13 +160,21 @@ def configs() -> list[Workload]:
     ]
 
 
+BITS_TERNARY = 15      # v_bits of the three-level ("1.5-bit") value codes: five base-3 digits per byte
+
+
+def packed_row_bytes(D: int, bits: int) -> int:
+    """Bytes of one packed row of D codes in the cache."""
+    return (D + 4) // 5 if bits == BITS_TERNARY else D * bits // 8
+
+
 def algorithmic_bytes(w: Workload, lengths=None) -> int:
     """Bytes one decode-attention call must move: packed codes + scale/zero of the quantized
     prefix, the fp16 window and sinks, and q/out.  Split scratch is not counted."""
     lengths = w.lengths() if lengths is None else np.asarray(lengths)
     D, ng = w.head_dim, w.head_dim // w.group_size
     mb = 2 if w.meta_fp8 else 4      # bytes of {scale, zero} per (token, group)
-    per_tok = (D * w.k_bits // 8 + mb * ng) + (D * w.v_bits // 8 + mb * ng)
+    per_tok = (packed_row_bytes(D, w.k_bits) + mb * ng) + (packed_row_bytes(D, w.v_bits) + mb * ng)
     total = 0
     for L in lengths.tolist():
         lq = max(L - w.window, 0)
@@ -182,6 +190,6 @@ def partition_kernel_bytes(w: Workload, lengths=None) -> int:
     lengths = w.lengths() if lengths is None else np.asarray(lengths)
     D, ng = w.head_dim, w.head_dim // w.group_size
     mb = 2 if w.meta_fp8 else 4      # bytes of {scale, zero} per (token, group)
-    per_tok = (D * w.k_bits // 8 + mb * ng) + (D * w.v_bits // 8 + mb * ng)
+    per_tok = (packed_row_bytes(D, w.k_bits) + mb * ng) + (packed_row_bytes(D, w.v_bits) + mb * ng)
     total = sum(w.n_kv_heads * max(L - w.window - w.n_sink, 0) * per_tok for L in lengths.tolist())
     return int(total + w.batch * w.n_q_heads * D * 2)

@@ -136,6 +136,16 @@ def test_three_bit_rows_are_48_bytes(lib):
     assert sizes[0] == 2 * 2 * cap * 48 and sizes[1] == 2 * 2 * cap * 32      # 128 three-bit fields = 48 bytes
 
 
+def test_three_level_value_rows_are_26_bytes_and_keys_stay_binary(lib):
+    c = cfg(k_bits=2, v_bits=B.SKVQ_BITS_TERNARY, group_size=64)
+    assert B.skvq_check_config(c) == B.SKVQ_OK
+    sizes, cap = B.skvq_cache_sizes(c), B.skvq_quant_capacity(c)
+    assert sizes[0] == 2 * 2 * cap * 32 and sizes[1] == 2 * 2 * cap * 26      # five base-3 digits per byte: ceil(128 / 5)
+    assert B.skvq_check_config(cfg(k_bits=B.SKVQ_BITS_TERNARY, v_bits=2)) == B.SKVQ_ERR_UNSUPPORTED
+    for v in (5, 8, 14, 16):
+        assert B.skvq_check_config(cfg(v_bits=v)) == B.SKVQ_ERR_UNSUPPORTED
+
+
 def test_group_bounds_are_validated_on_the_host(lib):
     import numpy as np
     c = cfg(group_size=64)                                   # two groups per row, two KV heads

@@ -65,6 +65,8 @@ def guarded_cache(w, max_tokens):
     (4, dict(context=1100, batch=3, ragged=None, n_q_heads=4, n_kv_heads=4), 1100, [1100, 0, 300]),   # 4-bit g64, window 256
     (2, dict(context=900, batch=1, n_q_heads=24), 900, [900]),                                    # tcgen05 kernel
     (4, dict(context=700, batch=1, ragged=None, n_q_heads=8, n_kv_heads=4), 700, [650]),          # 4-bit with 2 heads per KV head: tcgen05 kernel
+    (2, dict(context=1000, batch=2, v_bits=15, n_sink=3), 1000, [1000, 333]),                     # three-level values: 26-byte rows, 2-byte aligned
+    (1, dict(context=800, batch=1, n_q_heads=4, n_kv_heads=4, k_bits=3, v_bits=3), 800, [800]),   # 3-bit streams: 48-byte rows
 ])
 def test_nothing_is_written_outside_the_buffers(cfg_i, kw, n, lens):
     w = CF[cfg_i].scaled(**kw)

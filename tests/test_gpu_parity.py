@@ -380,6 +380,12 @@ def test_adversarial_values_stay_bit_exact():
     (4, dict(context=2300, batch=2, ragged=None, n_q_heads=8, n_kv_heads=2, group_size=32), 2300),               # 4-bit, 4 heads per KV head, group 32
     (4, dict(context=1900, batch=1, ragged=None, n_q_heads=4, n_kv_heads=4, group_size=32, k_bits=4, v_bits=2), 1900),   # 4-bit keys, 2-bit values, group 32, one head per KV head
     (1, dict(context=70000, batch=1, n_q_heads=2, n_kv_heads=1, k_bits=3, v_bits=3), 70000),                     # 3-bit, many tiles per CTA: the int32 value sums fold on their own
+    # three-level ("1.5-bit") values, the K2 V1.5 setting of the abstract and Sec. 4.2: 26-byte rows, five base-3 digits per byte
+    (1, dict(context=2200, batch=2, n_q_heads=4, n_kv_heads=4, v_bits=15), 2200),                                 # group 128, one head per KV head
+    (2, dict(context=1800, batch=2, v_bits=15, n_sink=5), 1800),                                                  # group 32, 4 heads per KV head, sinks
+    (2, dict(context=1500, batch=1, v_bits=15, group_size=64, group_bounds=(0, 96, 128), meta_fp8=True), 1500),   # unequal groups, FP8 parameters
+    (4, dict(context=1300, batch=3, ragged=None, n_q_heads=12, n_kv_heads=2, k_bits=4, v_bits=15), 1300),         # 4-bit keys, 6 heads per KV head: two launches
+    (1, dict(context=40000, batch=1, n_q_heads=2, n_kv_heads=1, k_bits=3, v_bits=15, group_size=64), 40000),      # 3-bit keys, many tiles per CTA
 ])
 def test_unequal_groups_and_three_bit_codes_bit_exact_cache_and_attention(cfg_i, kw, n):
     w = small(cfg_i, **kw)
