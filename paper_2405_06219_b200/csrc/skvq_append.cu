@@ -8,46 +8,21 @@
 //                   the final window, so the read and the overwrite of a slot never race.
 //   "new" items     tokens t in [L0, L1): quantized straight from the input if t < L1-W, else
 //                   written to the ring unless an evict item refills that slot.
-// Bulk appends (prefill) send every whole, 64-aligned tile of tokens that goes straight from the input to the
-// quantized segment through append_bulk_kernel (rows staged in shared memory by cp.async, gathered from
-// there); append_kernel takes the rest: evictions from the ring, ring writes and the ragged ends.
+// Bulk appends (prefill) send every whole, 64-aligned run of tokens that goes straight from the input to the
+// quantized segment through the tile kernel (skvq_append_tc.cu: reorder on the tensor core, one thread per token
+// row); append_kernel takes the rest: evictions from the ring, ring writes and the ragged ends.
 // Eight lanes own one 128-channel row (16 channels each); a warp handles two tokens at a time,
 // K rows on lanes 0-7/16-23 and V rows on lanes 8-15/24-31.  Group statistics are reduced with
 // xor-shuffles over G/16 lanes.  All quantizer arithmetic uses explicitly rounded fp32 intrinsics
 // so the codes, scales and zeros do not depend on compiler contraction.
-#include <type_traits>
 
-#include "skvq_internal.cuh"
+#include "skvq_append_common.cuh"
 
 namespace skvq {
 namespace {
 
 constexpr int kItemsPerCta = 64;
 constexpr int kAppendThreads = 128;
-
-struct AppendArgs {
-    Shape s;
-    CachePtrs c;
-    const __half *k, *v;
-    const int32_t *n_new_per_seq;
-    int n_new;
-    int use_bulk;   // append_bulk_kernel runs alongside
-};
-
-__device__ __forceinline__ int seq_new_count(const AppendArgs &a, int b)
-{
-    int n = a.n_new_per_seq ? a.n_new_per_seq[b] : a.n_new;
-    return min(max(n, 0), a.n_new);
-}
-
-// Tokens [f0, f1) of a sequence (multiples of 64, possibly empty) are quantized by append_bulk_kernel: they are
-// new, they end up below the window, and they form whole aligned tiles.
-__device__ __forceinline__ void bulk_range(int L0, int n_sink, int q_end, int &f0, int &f1)
-{
-    f0 = (max(L0, n_sink) + 63) & ~63;      // attention sinks are not quantized: they stay with append_kernel
-    f1 = q_end & ~63;
-    if (f1 < f0) f1 = f0;
-}
 
 // The codes of 16 elements by the defining formula (IEEE division, rintf): it runs only for the few row segments
 // that have a quotient next to a rounding boundary, and for 3-bit codes.  Inlined on purpose: as a separate function
@@ -70,21 +45,6 @@ __device__ __forceinline__ void quantize16_exact(const float (&x)[16], float zf,
 }
 
 // Quantize the 16 channels held by this lane; `lanes_per_group` lanes share the group statistics.
-// fp32 scale and zero point -> the two E4M3 bytes {h, z} (round to nearest even, saturating at 448) ...
-__device__ __forceinline__ uint16_t to_e4m3x2(float h, float z)
-{
-    uint16_t r;
-    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(z), "f"(h));      // first operand -> upper byte
-    return r;
-}
-// ... and back: {h, z} as a half2 (every E4M3 value is an fp16 value)
-__device__ __forceinline__ __half2 from_e4m3x2(uint16_t b)
-{
-    uint32_t r;
-    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(r) : "h"(b));
-    return *reinterpret_cast<const __half2 *>(&r);
-}
-
 // Writes what is stored per (token, group): a half2 {h, z}, or its two E4M3 bytes in the low 16 bits of hz_bits.
 // LPG > 0: lanes per group known at compile time (the shuffle rounds unroll); 0: taken from lanes_per_group.
 // lanes_per_group == 0 (with LPG == 0): the group is the lanes [lane_lo, lane_hi) of the row's 8 (groups of unequal width).
@@ -197,7 +157,7 @@ __global__ void __launch_bounds__(kAppendThreads) append_kernel(AppendArgs a)
     const int n_evict = max(min(L0, q_end) - t_lo, 0);
     int f0, f1;
     bulk_range(L0, s.n_sink, q_end, f0, f1);
-    const int n_bulk = a.use_bulk ? f1 - f0 : 0;   // new tokens the bulk kernel takes: skipped here
+    const int n_bulk = a.use_bulk ? f1 - f0 : 0;   // new tokens the tile kernel takes: skipped here
     const int n_items = n_evict + n_b - n_bulk;
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -358,103 +318,7 @@ __global__ void __launch_bounds__(kAppendThreads) append_kernel(AppendArgs a)
     }
 }
 
-constexpr int kBulkTok = 64;
-constexpr int kBulkStride = kHeadDim + 8;   // halfs per staged row: 16 bytes of padding spread the rows over the banks
-
-__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc)
-{
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc)
-                 : "memory");
-}
-
-// One CTA = one (sequence, KV head, 64-token tile) of bulk_range(): 64 K rows and 64 V rows are copied to
-// shared memory in 16-byte pieces (coalesced 256-byte rows), then gathered by the reorder index from there.
-template <int G>
-__global__ void __launch_bounds__(kAppendThreads) append_bulk_kernel(AppendArgs a)
-{
-    const Shape &s = a.s;
-    const int b = blockIdx.z, h = blockIdx.y;
-    const int L0 = a.c.lengths[b];
-    const int n_b = seq_new_count(a, b);
-    const int L1 = L0 + n_b;
-    if (n_b == 0 || L1 > s.max_tokens) return;
-    int f0, f1;
-    bulk_range(L0, s.n_sink, max(L1 - s.W, 0), f0, f1);
-    const int t0 = f0 + kBulkTok * blockIdx.x;
-    if (t0 >= f1) return;
-    if (!SKVQ_IN_BOUNDS(t0 >= L0 && t0 + kBulkTok <= s.cap && t0 + kBulkTok - L0 <= a.n_new, a.c.status)) return;
-
-    __shared__ __align__(16) __half xs[2][kBulkTok][kBulkStride];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const size_t tok_stride = (size_t)s.Hkv * kHeadDim;
-    const size_t src0 = ((size_t)b * a.n_new + (t0 - L0)) * tok_stride + (size_t)h * kHeadDim;
-    // two copy groups: the value rows are still on their way while the key rows are quantized
-#pragma unroll
-    for (int tensor = 0; tensor < 2; ++tensor) {
-#pragma unroll
-        for (int c = tid; c < kBulkTok * 16; c += kAppendThreads) {
-            const int tok = c >> 4, piece = c & 15;
-            cp_async16(&xs[tensor][tok][piece * 8], (tensor ? a.v : a.k) + src0 + (size_t)tok * tok_stride + piece * 8);
-        }
-        asm volatile("cp.async.commit_group;" ::: "memory");
-    }
-    asm volatile("cp.async.wait_group 1;" ::: "memory");
-    __syncthreads();
-
-    const int sub = lane & 7, rsel = lane >> 3;
-    const size_t bh = (size_t)b * s.Hkv + h;
-    constexpr int lanes_per_group = G >> 4;
-    const int g = (sub << 4) / G;
-    const bool f8 = s.meta_fp8 != 0;
-    // One tensor's 64 rows; the code width is a template parameter so that nothing inside branches on it.
-    auto quantize_tile = [&](auto bits_tag, int tensor) {
-        constexpr int BITS = decltype(bits_tag)::value;
-        constexpr int row_bytes = kHeadDim * BITS / 8;
-        uint8_t *codes = (tensor ? a.c.v_codes : a.c.k_codes) + (bh * (size_t)s.cap + t0) * row_bytes;
-        __half2 *meta = (tensor ? a.c.v_meta : a.c.k_meta);      // two bytes per (token, group) with FP8 parameters
-        const size_t meta0 = (bh * (size_t)s.cap + t0) * s.ng + g;
-        const float alpha = ((tensor ? a.c.alpha_v : a.c.alpha_k) + (size_t)h * s.ng)[g];
-        // this lane's 16 gather addresses (shared-memory window) in its first row; later rows are constant offsets
-        uint32_t src_j[16];
-        {
-            const int32_t *ip = (tensor ? a.c.reorder_v : a.c.reorder_k) + (size_t)h * kHeadDim + (sub << 4);
-            const uint32_t row0 = (uint32_t)__cvta_generic_to_shared(&xs[tensor][warp * 4 + rsel][0]);
-#pragma unroll
-            for (int j = 0; j < 16; ++j) src_j[j] = row0 + 2u * (uint32_t)(ip[j] & (kHeadDim - 1));
-        }
-#pragma unroll
-        for (int it = 0; it < kBulkTok / 16; ++it) {
-            const int tok = it * 16 + warp * 4 + rsel;
-            float x[16];
-#pragma unroll
-            for (int j = 0; j < 16; ++j) {
-                unsigned short v;
-                asm("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(src_j[j] + (uint32_t)(it * 16 * kBulkStride * 2)));
-                x[j] = __half2float(__ushort_as_half(v));
-            }
-            uint32_t words[2];
-            uint32_t hz;
-            quantize16<BITS, lanes_per_group>(x, alpha, lanes_per_group, f8, words, hz);
-            uint8_t *codes_row = codes + (size_t)tok * row_bytes;
-            if constexpr (BITS == 2) reinterpret_cast<uint32_t *>(codes_row)[sub] = words[0];
-            else reinterpret_cast<uint2 *>(codes_row)[sub] = make_uint2(words[0], words[1]);
-            if ((sub & (lanes_per_group - 1)) == 0) {
-                const size_t mi = meta0 + (size_t)tok * s.ng;
-                if (f8) reinterpret_cast<uint16_t *>(meta)[mi] = (uint16_t)hz;
-                else reinterpret_cast<uint32_t *>(meta)[mi] = hz;
-            }
-        }
-    };
-#pragma unroll 1
-    for (int tensor = 0; tensor < 2; ++tensor) {
-        if (tensor) {
-            asm volatile("cp.async.wait_group 0;" ::: "memory");
-            __syncthreads();
-        }
-        if ((tensor ? s.v_bits : s.k_bits) == 2) quantize_tile(std::integral_constant<int, 2>{}, tensor);
-        else quantize_tile(std::integral_constant<int, 4>{}, tensor);
-    }
-}
+constexpr int kBulkTok = 64;      // the smallest append that goes through the tile kernel
 
 // lengths[b] += n_b, or flag an overflow and leave the sequence alone.
 __global__ void append_bookkeeping_kernel(AppendArgs a)
@@ -478,8 +342,8 @@ cudaError_t launch_append(const Shape &s, const CachePtrs &c, const __half *k, c
                           const int32_t *n_new_per_seq, int n_new, cudaStream_t stream)
 {
     if (n_new <= 0) return cudaSuccess;
-    // the tile kernel serves 2- and 4-bit codes in equal groups; everything else goes through append_kernel
-    const bool bulk = n_new >= kBulkTok && !s.bounded && plain_width(s.k_bits) && plain_width(s.v_bits);
+    // the tile kernel serves 2- and 4-bit codes (equal or unequal groups); the other widths go through append_kernel
+    const bool bulk = n_new >= kBulkTok && plain_width(s.k_bits) && plain_width(s.v_bits);
     AppendArgs a{s, c, k, v, n_new_per_seq, n_new, bulk ? 1 : 0};
     // what append_kernel keeps: evictions (at most W), and new tokens outside the bulk tiles (fewer than W + 128
     // when there are bulk tiles, all of them otherwise)
@@ -488,11 +352,7 @@ cudaError_t launch_append(const Shape &s, const CachePtrs &c, const __half *k, c
     const int max_items = n_evict_max + n_rest_max;
     int launched = 0;
     if (bulk) {
-        dim3 gridb((n_new + kBulkTok - 1) / kBulkTok, s.Hkv, s.B);
-        if (s.G == 128) append_bulk_kernel<128><<<gridb, kAppendThreads, 0, stream>>>(a);
-        else if (s.G == 64) append_bulk_kernel<64><<<gridb, kAppendThreads, 0, stream>>>(a);
-        else append_bulk_kernel<32><<<gridb, kAppendThreads, 0, stream>>>(a);
-        cudaError_t e = cudaGetLastError();
+        cudaError_t e = launch_append_tiles(a, stream);
         if (e != cudaSuccess) return e;
         ++launched;
     }

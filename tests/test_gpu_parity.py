@@ -85,6 +85,37 @@ def test_chunked_and_single_token_appends_bit_exact():
     assert_cache_bit_exact(gpu, bulk)
 
 
+@pytest.mark.parametrize("cfg_i,kw,chunks", [
+    (1, dict(context=5000, batch=2, n_q_heads=4, n_kv_heads=4), (37, 3000, 64, 1500, 399)),                # g128: runs of more than 8 tiles, a 64-row tail
+    (4, dict(context=3000, batch=2, ragged=None, n_q_heads=4, n_kv_heads=4), (1000, 1, 1300, 699)),        # 4-bit g64, window 256
+    (2, dict(context=2600, batch=1, meta_fp8=True, n_sink=5), (700, 1900)),                                 # g32, FP8 parameters, sinks
+    (2, dict(context=2100, batch=2, group_size=64, group_bounds=(0, 96, 128)), (1100, 1000)),               # two groups of unequal width
+    (4, dict(context=1700, batch=1, ragged=None, n_q_heads=4, n_kv_heads=4, k_bits=4, v_bits=2, group_size=32,
+             group_bounds=(0, 32, 64, 96, 128)), (900, 800)),                                               # mixed widths, boundaries given but equal
+])
+def test_bulk_appends_on_top_of_existing_tokens_bit_exact(cfg_i, kw, chunks):
+    """The tile kernel of bulk appends: chunks that start at any length, several CTA runs, ragged per-sequence counts."""
+    w = small(cfg_i, **kw)
+    n = sum(chunks)
+    gpu, ora = both_caches(w, n + 64)
+    k, v = w.prefill("k", n), w.prefill("v", n)
+    t = 0
+    for step in chunks:
+        gpu.append(dev(k[:, t:t + step]), dev(v[:, t:t + step]))
+        ora.append(k[:, t:t + step], v[:, t:t + step])
+        t += step
+        assert_cache_bit_exact(gpu, ora)
+    assert int(gpu.status[0].item()) == 0
+    # the same tokens with per-sequence counts: sequence b takes only part of the chunk
+    gpu2, ora2 = both_caches(w, n + 64)
+    counts = np.array([n - 517 * b for b in range(w.batch)], np.int32)
+    gpu2.append(dev(k), dev(v), dev(counts))
+    ora2.append(k, v, counts)
+    assert_cache_bit_exact(gpu2, ora2)
+    got, want = attention_both(gpu2, ora2, w)
+    assert np.abs(got - want).max() <= ATTN_TOL
+
+
 def test_ragged_append_and_overflow_flag():
     w = small(4, context=600, batch=4, ragged=None)
     gpu, ora = both_caches(w, 640)
