@@ -1,23 +1,32 @@
 // Tile kernel of skvq_quantize_append for bulk appends (prefill): channel reorder on the tensor core, then group-wise
-// clipped dynamic asymmetric quantization with one thread per token row (Sec. 3.1 Eq. 1 and Eq. 2, Algorithm 1).
+// clipped dynamic asymmetric quantization with two threads per token row (Sec. 3.1 Eq. 1 and Eq. 2, Algorithm 1).
 //
 // The reorder stored[j] = x[idx[j]] of a tile of 128 tokens is the product X * P^T with the 0/1 matrix
 // P[j][k] = (k == idx[j]): every output is one input times 1.0 plus zeros, so fp16 operands with fp32 accumulation give
 // the reordered values exactly.  One tcgen05.mma chain (M = 128 tokens, N = 128 stored channels, K = 128 source
-// channels, fp16 in, fp32 accumulators in tensor memory) replaces 16384 two-byte gathers, and it hands every thread
-// its token's whole reordered row: lane m of the tensor memory is token m of the tile.  Group minimum and maximum,
-// scale and zero point, the codes and their packing are then register arithmetic of one thread, without shuffles.
+// channels, fp16 in, fp32 accumulators in tensor memory) replaces 16384 two-byte gathers, and it lays every token's
+// reordered row along one lane of the tensor memory: lane m is token m of the tile.  Group minimum and maximum, scale
+// and zero point, the codes and their packing are then register arithmetic without shuffles.
 //
-// One CTA = 128 threads = one (sequence, KV head, tensor K or V) and a run of consecutive 128-token tiles:
-//   copy      16-byte cp.async pieces of the next tile straight into the canonical K-major operand layout
-//             (8-row x 16-byte core matrices), issued as soon as the MMAs of the current tile have read the buffer;
-//   MMA       thread 0 issues 8 k-steps, commits them to an mbarrier (bounded wait);
-//   quantize  every thread reads its row from tensor memory 32 channels at a time: one pass for the extremes of every
-//             32-channel granule (groups are unions of granules), one pass that quantizes, then 16-byte stores of the
-//             packed row and of the {scale, zero} words.
-// Three CTAs per SM (64 KB of shared memory and 128 tensor-memory columns each) keep copies, MMAs and arithmetic of
-// different tiles in flight.  The quantizer arithmetic is that of append_kernel (explicitly rounded fp32 operations),
-// so both kernels produce the same bits.
+// One CTA = one (sequence, KV head, tensor K or V) and a run of consecutive 128-token tiles; 256 arithmetic threads and
+// one control warp.  Arithmetic warps w and w + 4 share the 32 tokens of lane quadrant w & 3: the first takes stored
+// channels 0-63 of each, the second 64-127 (a group that spans both halves has its extremes exchanged through shared
+// memory).  Nothing but mbarriers orders the two sides:
+//   copy      the control lane brings a tile in with two tensor-map copies (cp.async.bulk.tensor, 64 channels x 128
+//             tokens each, 128-byte swizzle: the K-major operand layout of the MMA), two tiles ahead of the arithmetic;
+//             rows past the end of the input are filled with zeros by the copy engine;
+//   MMA       the control lane issues 8 k-steps per tile and commits them to an mbarrier; two accumulators in tensor
+//             memory, so the MMAs of tile t+1 run under the arithmetic of tile t;
+//   quantize  every arithmetic thread reads its half row (64 values) from tensor memory into registers once: the
+//             extremes of its two 32-channel granules (groups are unions of granules), scale and zero point, the
+//             codes, then one 16-byte store of its half of the packed row, and the {scale, zero} words; its arrival on
+//             the accumulator's mbarrier lets the control lane reuse it.
+// Every wait is bounded; a wait that ran out is reported through the cache's status word, the threads then run to the end
+// of their loops without waiting or storing.  Two CTAs per SM (96 KB of shared memory and 256 tensor-memory columns
+// each).  The quantizer arithmetic is that of append_kernel (explicitly rounded fp32 operations), so both kernels
+// produce the same bits.
+#include <cuda.h>
+
 #include <type_traits>
 
 #include "skvq_append_common.cuh"
@@ -30,13 +39,16 @@ namespace {
 using namespace mmak;
 using namespace tc5;
 
-constexpr int kTileRows = 128;                       // tokens per tile = rows of the MMA = threads per CTA
+constexpr int kTileRows = 128;                       // tokens per tile = rows of the MMA
+constexpr int kArithThreads = 2 * kTileRows;         // two threads per token row
+constexpr int kTileThreads = kArithThreads + 32;     // and the control warp
 constexpr int kTilesPerCta = 8;                      // consecutive tiles one CTA works through
 constexpr int kOperandBytes = kTileRows * kHeadDim * 2;      // 32 KB: a 128 x 128 fp16 operand
-constexpr int kSmemBytes = 2 * kOperandBytes;        // P and one tile of X
-constexpr uint32_t kLboBytes = 128;                  // between core matrices along K
-constexpr uint32_t kSboBytes = 16 * 128;             // between groups of 8 rows: 16 core matrices of 128 bytes
-constexpr int kTmemColumns = 128;                    // one 128 x 128 fp32 accumulator
+constexpr int kSmemBytes = 3 * kOperandBytes + 1024;      // P and two tiles of X, and room to align them to 1024 bytes
+constexpr uint32_t kLboBytes = 128;                  // P (no swizzle): between core matrices along K
+constexpr uint32_t kSboBytes = 16 * 128;             // P: between groups of 8 rows: 16 core matrices of 128 bytes
+constexpr int kHalfTileBytes = kTileRows * 128;      // X: 64 channels of 128 tokens, 128-byte rows (swizzled)
+constexpr int kTmemColumns = 256;                    // two 128 x 128 fp32 accumulators
 
 // Byte offset of the 16-byte piece (row, piece) of a K-major operand without swizzle: piece = 8 consecutive K elements.
 __device__ __forceinline__ uint32_t operand_offset(int row, int piece)
@@ -44,10 +56,24 @@ __device__ __forceinline__ uint32_t operand_offset(int row, int piece)
     return (uint32_t)((row >> 3) * kSboBytes + piece * kLboBytes + (row & 7) * 16);
 }
 
-__device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void *gsrc)
+// One box of a three-dimensional tensor map -> shared memory, completion counted in bytes on an mbarrier.
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2, uint32_t bar)
 {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gsrc) : "memory");
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
 }
+// Shared-memory matrix descriptor of a K-major operand in the 128-byte swizzle: rows of 128 bytes, 8-row atoms of 1024
+// bytes (stride offset), start address inside the atom for a k-step; descriptor version 1, layout type 2.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
+{
+    return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// Barrier 1: the arithmetic threads only (the control warp never joins it).
+__device__ __forceinline__ void arith_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 // Stored scale and zero point of a group from its extremes (Eq. 2; both ends clipped by alpha): the words that go to
 // the cache, and the values the codes are computed against.
@@ -77,74 +103,97 @@ __device__ __forceinline__ float mul_sat(float a, float b)      // clamp(RN(a * 
     return r;
 }
 
-// Codes of 32 consecutive stored channels against (hf, zf): BITS words, code j in bits [j*BITS, (j+1)*BITS) of the run.
-// code = clamp(rint(RN((x - z) / h)), 0, qmax) with IEEE division.  Instead of dividing, u = sat(d * RN(RN(1/h) / qmax))
-// is the clamped quotient on the scale [0, 1], within 5 * 2^-24 relative of the IEEE quotient / qmax; wherever every
-// value within 2^-18 relative of it rounds to the same integer, that integer is the code.  The test is two FMAs onto
-// 1.5 * 2^23 (the low mantissa bits of the sum are then the rounded integer, ties to even, like rintf), one with the
-// quotient scaled down and one scaled up by 2^-18; both results are packed, and fields in which the two packed rows
-// differ are elements in doubt (a quotient next to k + 0.5, exact ties included).  Those are redone by the defining
-// formula: the warp walks the union of its doubtful columns, re-reads each from tensor memory (taddr = this warp's
-// lanes, first column of the run) and the lanes concerned patch their field.  Every lane of the warp must call this.
+// Codes of 16 consecutive stored channels against (hf, zf): BITS / 2 words, code j in bits [j*BITS, (j+1)*BITS) of the run.
+// code = clamp(rint(RN((x - z) / h)), 0, qmax) with IEEE division.  Instead of dividing, u = sat(d * r) with
+// r = RN(RN(1/h) / qmax) is the clamped quotient on the scale [0, 1], within 5 * 2^-24 relative of the IEEE quotient / qmax;
+// wherever every value within 2^-18 relative of it rounds to the same integer, that integer is the code.  The test is two
+// FMAs onto 1.5 * 2^23 (the low mantissa bits of the sum are then the rounded integer, ties to even, like rintf), one with
+// the quotient scaled down and one scaled up by 2^-18; both results are packed (four partial sums each, so that no
+// addition waits for the one before), and fields in which the two packed runs differ are elements in doubt (a quotient
+// next to k + 0.5, exact ties included): doubt[] has their bits set and repair16 redoes them.
 template <int BITS>
-__device__ __forceinline__ void quantize32(const float (&x)[32], float hf, float zf, uint32_t taddr, uint32_t (&words)[BITS])
+__device__ __forceinline__ void pack16(const float (&x)[16], float zf, float r, uint32_t (&words)[BITS / 2], uint32_t (&doubt)[BITS / 2])
 {
-    constexpr int qmax = (1 << BITS) - 1, PER_WORD = 32 / BITS;
+    constexpr int qmax = (1 << BITS) - 1, PER_WORD = 32 / BITS, NW = BITS / 2, LANES = 4 / NW;      // partial sums per word
     constexpr float MAGIC = 12582912.0f;                       // 0x4B400000
     constexpr float UP = (float)qmax * (1.0f + 3.814697265625e-06f), DN = (float)qmax * (1.0f - 3.814697265625e-06f);   // exact products
     uint32_t kconst = 0u;
 #pragma unroll
     for (int j = 0; j < PER_WORD; ++j) kconst += 0x4B400000u << (j * BITS);
-    const float r = hf != 0.0f ? __fmul_rn(__frcp_rn(hf), 1.0f / (float)qmax) : 0.0f;      // degenerate group (h == 0): every code is 0
-    uint32_t wb[BITS];
+    uint32_t wa[NW][LANES], wb[NW][LANES];
 #pragma unroll
-    for (int i = 0; i < BITS; ++i) {
-        words[i] = 0u - kconst;      // the constant bits of 1.5 * 2^23 come out of the sums (modulo 2^32)
-        wb[i] = 0u - kconst;
-    }
+    for (int i = 0; i < NW; ++i)
 #pragma unroll
-    for (int j = 0; j < 32; ++j) {
+        for (int l = 0; l < LANES; ++l) { wa[i][l] = 0u; wb[i][l] = 0u; }
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
         const float u = mul_sat(__fsub_rn(x[j], zf), r);
-        words[j / PER_WORD] += __float_as_uint(__fmaf_rn(u, DN, MAGIC)) << ((j % PER_WORD) * BITS);
-        wb[j / PER_WORD] += __float_as_uint(__fmaf_rn(u, UP, MAGIC)) << ((j % PER_WORD) * BITS);
+        wa[j / PER_WORD][j % LANES] += __float_as_uint(__fmaf_rn(u, DN, MAGIC)) << ((j % PER_WORD) * BITS);
+        wb[j / PER_WORD][j % LANES] += __float_as_uint(__fmaf_rn(u, UP, MAGIC)) << ((j % PER_WORD) * BITS);
     }
-    uint32_t any = 0u;
 #pragma unroll
-    for (int i = 0; i < BITS; ++i) {
-        wb[i] ^= words[i];           // non-zero fields: elements in doubt
-        any |= wb[i];
+    for (int i = 0; i < NW; ++i) {
+        uint32_t sa = 0u - kconst, sb = 0u - kconst;      // the constant bits of 1.5 * 2^23 come out of the sums (modulo 2^32)
+#pragma unroll
+        for (int l = 0; l < LANES; ++l) { sa += wa[i][l]; sb += wb[i][l]; }
+        words[i] = sa;
+        doubt[i] = sa ^ sb;
     }
-    if (__any_sync(0xffffffffu, any != 0u)) {
+}
+
+// The elements of a 16-column run that pack16 left in doubt, redone by the defining formula: the warp walks the union of
+// its doubtful columns, re-reads each from tensor memory (taddr = this warp's lanes, first column of the run) and the
+// lanes concerned patch their field.  Every lane of the warp must call this.
+template <int BITS>
+__device__ __forceinline__ void repair16(float hf, float zf, uint32_t taddr, uint32_t (&words)[BITS / 2], const uint32_t (&doubt)[BITS / 2])
+{
+    constexpr int qmax = (1 << BITS) - 1, PER_WORD = 32 / BITS, NW = BITS / 2;
 #pragma unroll
-        for (int i = 0; i < BITS; ++i) {
-            uint32_t todo = __reduce_or_sync(0xffffffffu, wb[i]);      // the same for every lane: the loop is uniform
-            while (todo) {
-                const int f = (__ffs(todo) - 1) / BITS;                // field of this word = column i * PER_WORD + f of the run
-                const uint32_t field = (uint32_t)qmax << (f * BITS);
-                todo &= ~field;
-                float xv;
-                tmem_ld1(taddr + i * PER_WORD + f, xv);
-                tmem_wait_ld();
-                if (wb[i] & field) {
-                    float c = hf != 0.0f ? rintf(__fdiv_rn(__fsub_rn(xv, zf), hf)) : 0.0f;
-                    c = fminf(fmaxf(c, 0.0f), (float)qmax);
-                    words[i] = (words[i] & ~field) | ((uint32_t)(int)c << (f * BITS));
-                }
+    for (int i = 0; i < NW; ++i) {
+        uint32_t todo = __reduce_or_sync(0xffffffffu, doubt[i]);      // the same for every lane: the loop is uniform
+        while (todo) {
+            const int f = (__ffs(todo) - 1) / BITS;                    // field of this word = column i * PER_WORD + f of the run
+            const uint32_t field = (uint32_t)qmax << (f * BITS);
+            todo &= ~field;
+            float xv;
+            tmem_ld1(taddr + i * PER_WORD + f, xv);
+            tmem_wait_ld();
+            if (doubt[i] & field) {
+                float c = hf != 0.0f ? rintf(__fdiv_rn(__fsub_rn(xv, zf), hf)) : 0.0f;
+                c = fminf(fmaxf(c, 0.0f), (float)qmax);
+                words[i] = (words[i] & ~field) | ((uint32_t)(int)c << (f * BITS));
             }
         }
     }
 }
 
+// Minimum and maximum of 16 values.
+__device__ __forceinline__ void extremes16(const float (&x)[16], float &lo, float &hi)
+{
+    lo = x[0];
+    hi = x[0];
+#pragma unroll
+    for (int j = 1; j < 16; ++j) {
+        lo = fminf(lo, x[j]);
+        hi = fmaxf(hi, x[j]);
+    }
+}
+
 template <int G>
-__global__ void __launch_bounds__(kTileRows, 3) append_tile_kernel(AppendArgs a)
+__global__ void __maxnreg__(112)      // two CTAs of nine warps per SM
+append_tile_kernel(AppendArgs a, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v)
 {
     constexpr int NG = kHeadDim / G;
-    extern __shared__ __align__(128) uint8_t smem[];
-    __shared__ __align__(8) uint64_t bar_sh;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    __shared__ __align__(8) uint64_t bar_sh[6];
     __shared__ uint32_t tmem_sh;
     __shared__ int fail_sh;
+    __shared__ __align__(16) float4 ext_sh[2][kTileRows];      // {min, max} of a half row's two granules, for the thread of the other half
     const Shape &s = a.s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const bool control = warp == kArithThreads / 32;
+    const int quad = warp & 3, half = (warp >> 2) & 1;         // tensor-memory lanes 32*quad .. +31; stored channels 64*half .. +63
+    const int row = 32 * quad + lane;                          // this thread's token of every tile
     const int b = blockIdx.z, tensor = blockIdx.x & 1, h = blockIdx.y;
     const int L0 = a.c.lengths[b];
     const int n_b = seq_new_count(a, b);
@@ -156,159 +205,280 @@ __global__ void __launch_bounds__(kTileRows, 3) append_tile_kernel(AppendArgs a)
     const int t_begin = (blockIdx.x >> 1) * kTilesPerCta, t_end = min(n_tiles, t_begin + kTilesPerCta);
     if (t_begin >= t_end) return;
     if (!SKVQ_IN_BOUNDS(f0 >= L0 && f1 <= s.cap && f1 - L0 <= a.n_new, a.c.status)) return;
+    const int T = t_end - t_begin;
 
-    const int bits = tensor ? s.v_bits : s.k_bits;
-    const bool f8 = s.meta_fp8 != 0;
-    const size_t bh = (size_t)b * s.Hkv + h;
-    const size_t tok_stride = (size_t)s.Hkv * kHeadDim;
-    const __half *src = (tensor ? a.v : a.k) + ((size_t)b * a.n_new * s.Hkv + h) * kHeadDim;      // token L0 of this sequence and head
-    const int32_t *idx = (tensor ? a.c.reorder_v : a.c.reorder_k) + (size_t)h * kHeadDim;
-    const float *alpha = (tensor ? a.c.alpha_v : a.c.alpha_k) + (size_t)h * NG;
-    const uint32_t gmap = granule_groups(tensor ? a.c.bounds_v : a.c.bounds_k, h, G, NG);      // group of every 32-channel granule
-    uint8_t *codes = (tensor ? a.c.v_codes : a.c.k_codes) + bh * (size_t)s.cap * packed_row_bytes(bits);
-    uint8_t *meta = reinterpret_cast<uint8_t *>(tensor ? a.c.v_meta : a.c.k_meta) + bh * (size_t)s.cap * NG * (f8 ? 2 : 4);
+    uint8_t *base = smem + ((1024u - (smem_u32(smem) & 1023u)) & 1023u);      // the swizzle pattern repeats every 1024 bytes
+    uint8_t *P = base, *X = base + kOperandBytes;      // X: two tile buffers of two half tiles each
+    const uint32_t bar_full = smem_u32(&bar_sh[0]);    // + 8 * (t & 1): the copies of tile t have landed
+    const uint32_t bar_mma = bar_full + 16;            // + 8 * (t & 1): the MMAs of tile t have completed
+    const uint32_t bar_free = bar_full + 32;           // + 8 * (t & 1): every arithmetic thread is done with the accumulator of tile t
 
-    uint8_t *P = smem, *X = smem + kOperandBytes;
-    const uint32_t bar = smem_u32(&bar_sh);
-
-    // ---- once per CTA: the permutation operand, the tensor memory, the barrier
-    {
+    // ---- once per CTA: the permutation operand, the tensor memory, the barriers
+    if (!control) {
         uint4 *p4 = reinterpret_cast<uint4 *>(P);
 #pragma unroll
-        for (int i = 0; i < kOperandBytes / 16 / kTileRows; ++i) p4[tid + i * kTileRows] = make_uint4(0u, 0u, 0u, 0u);
-    }
-    if (warp == 0) tmem_alloc(smem_u32(&tmem_sh), kTmemColumns);
-    if (tid == 0) {
-        mbar_init(bar, 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        fail_sh = 0;
+        for (int i = 0; i < kOperandBytes / 16 / kArithThreads; ++i) p4[tid + i * kArithThreads] = make_uint4(0u, 0u, 0u, 0u);
+    } else {
+        tmem_alloc(smem_u32(&tmem_sh), kTmemColumns);
+        if (lane == 0) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) mbar_init(bar_full + 8 * i, 1);
+            mbar_init(bar_free, kArithThreads);
+            mbar_init(bar_free + 8, kArithThreads);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            fail_sh = 0;
+        }
     }
     __syncthreads();
-    {
+    if (tid < kHeadDim) {
+        const int32_t *idx = (tensor ? a.c.reorder_v : a.c.reorder_k) + (size_t)h * kHeadDim;
         const int k = idx[tid] & (kHeadDim - 1);      // stored channel tid takes source channel k: P[tid][k] = 1
         *reinterpret_cast<__half *>(P + operand_offset(tid, k >> 3) + (k & 7) * 2) = __float2half(1.0f);
     }
+    proxy_fence();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = tmem_sh;
-    const uint32_t tmem_row = tmem + ((uint32_t)(warp * 32) << 16);      // this warp's 32 lanes
+    volatile int *fail = &fail_sh;
 
-    // Copies of tile t: warp w moves pieces 4w .. 4w+3 (64 consecutive bytes) of every row; a warp instruction covers 8
-    // rows x 4 pieces = four whole core matrices in shared memory.  Rows past the end of the range are left as they are
-    // (their products only reach their own accumulator rows, which nobody stores).
-    auto issue_copies = [&](int t) {
-        const int tok0 = f0 + (t_begin + t) * kTileRows;
-        const int rows = min(kTileRows, f1 - tok0);
-        const int piece = 4 * warp + (lane >> 3);
-        const __half *g = src + (size_t)(tok0 - L0 + (lane & 7)) * tok_stride + piece * 8;
-        const uint32_t dst = smem_u32(X) + operand_offset(lane & 7, piece);
+    if (control) {
+        // ================================================================ control warp: one lane copies and issues
+        if (lane == 0) {
+            const CUtensorMap *map = tensor ? &map_v : &map_k;
+            const uint64_t dP = smem_desc(smem_u32(P), kLboBytes, kSboBytes);
+            constexpr uint32_t kIdesc = idesc_f16_f32(kTileRows, kHeadDim);
+            bool alive = true;
+            auto copy_tile = [&](int t) {      // both halves of tile t into buffer t & 1
+                const uint32_t dst = smem_u32(X) + (t & 1) * kOperandBytes, bar = bar_full + 8 * (t & 1);
+                const int tok = f0 + (t_begin + t) * kTileRows - L0;      // row of the input
+                mbar_expect_tx(bar, kOperandBytes);
+                tma_load_3d(dst, map, h * kHeadDim, tok, b, bar);
+                tma_load_3d(dst + kHalfTileBytes, map, h * kHeadDim + 64, tok, b, bar);
+            };
+            copy_tile(0);
+            if (T > 1) copy_tile(1);
+            for (int t = 0; t < T; ++t) {
+                if (*fail) alive = false;
+                const uint32_t ph = (uint32_t)(t >> 1) & 1u;
+                if (alive && !mbar_wait_bounded(bar_full + 8 * (t & 1), ph)) { alive = false; *fail = 1; }
+                if (t >= 2 && alive && !mbar_wait_bounded(bar_free + 8 * (t & 1), ph ^ 1u)) { alive = false; *fail = 1; }      // tile t-2 has been read
+                tc_fence_after();
+                const uint32_t xb = smem_u32(X) + (t & 1) * kOperandBytes;
 #pragma unroll
-        for (int i = 0; i < kTileRows / 8; ++i)
-            if (8 * i < rows) cp_async16(dst + i * kSboBytes, g + (size_t)(8 * i) * tok_stride);      // rows is a multiple of 64
-        asm volatile("cp.async.commit_group;" ::: "memory");
-    };
+                for (int ks = 0; ks < kHeadDim / 16; ++ks) {      // 16 source channels = 32 bytes of a swizzled row per k-step
+                    const uint64_t dX = smem_desc_sw128(xb + (ks >> 2) * kHalfTileBytes + (ks & 3) * 32);
+                    umma_f16(tmem + (uint32_t)(t & 1) * kHeadDim, dX, dP + ((ks * 2 * kLboBytes) >> 4), kIdesc, ks > 0 ? 1u : 0u);
+                }
+                umma_commit(bar_mma + 8 * (t & 1));
+                if (t + 2 < T) {      // the buffer is free once these MMAs have read it
+                    if (alive && !mbar_wait_bounded(bar_mma + 8 * (t & 1), ph)) { alive = false; *fail = 1; }
+                    copy_tile(t + 2);
+                }
+            }
+            // nothing of this lane's may be in flight when the CTA leaves: the last copies and MMAs
+            for (int t = max(T - 2, 0); t < T; ++t) {
+                const uint32_t ph = (uint32_t)(t >> 1) & 1u;
+                if (alive && !mbar_wait_bounded(bar_full + 8 * (t & 1), ph)) alive = false;
+                if (alive && !mbar_wait_bounded(bar_mma + 8 * (t & 1), ph)) alive = false;
+            }
+        }
+        __syncwarp();
+    } else {
+        // ================================================================ arithmetic threads
+        const int bits = tensor ? s.v_bits : s.k_bits;
+        const bool f8 = s.meta_fp8 != 0;
+        const size_t bh = (size_t)b * s.Hkv + h;
+        const float *alpha = (tensor ? a.c.alpha_v : a.c.alpha_k) + (size_t)h * NG;
+        float alpha_g[NG];
+#pragma unroll
+        for (int g = 0; g < NG; ++g) alpha_g[g] = alpha[g];
+        const uint32_t gmap = granule_groups(tensor ? a.c.bounds_v : a.c.bounds_k, h, G, NG);      // group of every 32-channel granule
+        // Does a group reach into both halves of the row?  Then the two threads of a token exchange their extremes.
+        const bool spans = ((gmap >> 2) & 3u) == ((gmap >> 4) & 3u);
+        uint8_t *codes = (tensor ? a.c.v_codes : a.c.k_codes) + bh * (size_t)s.cap * packed_row_bytes(bits);
+        uint8_t *meta = reinterpret_cast<uint8_t *>(tensor ? a.c.v_meta : a.c.k_meta) + bh * (size_t)s.cap * NG * (f8 ? 2 : 4);
+        const uint32_t tmem_half = tmem + ((uint32_t)(quad * 32) << 16) + 64 * half;      // this thread's lane, its first column
+        const float qmaxf = (float)code_max(bits);
+        bool alive = true;
 
-    const int T = t_end - t_begin;
-    const uint64_t dX = smem_desc(smem_u32(X), kLboBytes, kSboBytes), dP = smem_desc(smem_u32(P), kLboBytes, kSboBytes);
-    constexpr uint32_t kIdesc = idesc_f16_f32(kTileRows, kHeadDim);
-    issue_copies(0);
-
-    for (int t = 0; t < T; ++t) {
-        // ---- tile t has landed: make it visible to the tensor core, which also has finished with the accumulators'
-        // previous contents once every thread is here
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
-        proxy_fence();
-        tc_fence_before();
-        __syncthreads();
-        if (tid == 0) {
+        for (int t = 0; t < T; ++t) {
+            if (*fail) alive = false;
+            if (alive && !mbar_wait_bounded(bar_mma + 8 * (t & 1), (uint32_t)(t >> 1) & 1u)) { alive = false; *fail = 1; }
             tc_fence_after();
-#pragma unroll
-            for (int ks = 0; ks < kHeadDim / 16; ++ks)      // 16 source channels = two core matrices per k-step
-                umma_f16(tmem, dX + ((ks * 2 * kLboBytes) >> 4), dP + ((ks * 2 * kLboBytes) >> 4), kIdesc, ks > 0 ? 1u : 0u);
-            umma_commit(bar);
-        }
-        if (!mbar_wait_bounded(bar, (uint32_t)t & 1u)) fail_sh = 1;
-        tc_fence_after();
-        if (__syncthreads_or(fail_sh)) break;                 // a uniform decision; also: every thread knows the buffer is free
-        if (t + 1 < T) issue_copies(t + 1);                   // in flight while this tile is quantized
+            const uint32_t trow = tmem_half + (uint32_t)(t & 1) * kHeadDim;
+            const int tok = f0 + (t_begin + t) * kTileRows + row;
+            const bool valid = alive && tok < f1;
 
-        // ---- this thread's token
-        const int tok = f0 + (t_begin + t) * kTileRows + tid;
-        const bool valid = tok < f1;
-        float x[32];
-        float mn[kGranules], mx[kGranules];
-#pragma unroll
-        for (int gr = 0; gr < kGranules; ++gr) {
-            tmem_ld32(tmem_row + 32 * gr, x);
-            tmem_wait_ld();
-            float lo = x[0], hi = x[0];
-#pragma unroll
-            for (int j = 1; j < 32; ++j) {
-                lo = fminf(lo, x[j]);
-                hi = fmaxf(hi, x[j]);
+            // ---- the thread's half row into registers, the extremes of its two 32-channel granules
+            float x0[16], x1[16], x2[16], x3[16];
+            tmem_ld16f(trow, x0);
+            tmem_ld16f(trow + 16, x1);
+            tmem_ld16f(trow + 32, x2);
+            tmem_ld16f(trow + 48, x3);
+            tmem_wait_ld16f(x0);
+            tmem_wait_ld16f(x1);
+            tmem_wait_ld16f(x2);
+            tmem_wait_ld16f(x3);
+            float lo[2], hi[2];
+            {
+                float lo0, hi0, lo1, hi1;
+                extremes16(x0, lo0, hi0);
+                extremes16(x1, lo1, hi1);
+                lo[0] = fminf(lo0, lo1);
+                hi[0] = fmaxf(hi0, hi1);
+                extremes16(x2, lo0, hi0);
+                extremes16(x3, lo1, hi1);
+                lo[1] = fminf(lo0, lo1);
+                hi[1] = fmaxf(hi0, hi1);
             }
-            mn[gr] = lo;
-            mx[gr] = hi;
-        }
-        float hf[NG], zf[NG];
-        uint32_t hz[NG];
+            float mn[kGranules], mx[kGranules];      // the row's four granules; the other half's only when a group spans both
 #pragma unroll
-        for (int g = 0; g < NG; ++g) {
-            float lo = CUDART_INF_F, hi = -CUDART_INF_F;
-#pragma unroll
-            for (int gr = 0; gr < kGranules; ++gr)
-                if (((gmap >> (2 * gr)) & 3u) == (uint32_t)g) {
-                    lo = fminf(lo, mn[gr]);
-                    hi = fmaxf(hi, mx[gr]);
-                }
-            group_parameters(lo, hi, alpha[g], (float)code_max(bits), f8, hz[g], hf[g], zf[g]);
-        }
-        // second pass: the codes, 32 channels at a time, and the packed row (the code width is a compile-time constant
-        // inside, so that the row stays in registers)
-        auto quantize_row = [&](auto bits_tag) {
-            constexpr int BITS = decltype(bits_tag)::value;
-            uint32_t *crow = reinterpret_cast<uint32_t *>(codes + (size_t)tok * packed_row_bytes(BITS));
-#pragma unroll 1      // rolled on purpose: one copy of the arithmetic in the instruction cache
             for (int gr = 0; gr < kGranules; ++gr) {
-                tmem_ld32(tmem_row + 32 * gr, x);
-                tmem_wait_ld();
-                const uint32_t g = (gmap >> (2 * gr)) & 3u;
-                float hg = hf[0], zg = zf[0];
-#pragma unroll
-                for (int i = 1; i < NG; ++i)
-                    if (g == (uint32_t)i) { hg = hf[i]; zg = zf[i]; }
-                uint32_t cw[BITS];
-                quantize32<BITS>(x, hg, zg, tmem_row + 32 * gr, cw);
-                if (valid) {
-                    if constexpr (BITS == 2) *reinterpret_cast<uint2 *>(crow + 2 * gr) = make_uint2(cw[0], cw[1]);
-                    else *reinterpret_cast<uint4 *>(crow + 4 * gr) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
-                }
+                mn[gr] = (gr >> 1) == half ? lo[gr & 1] : CUDART_INF_F;
+                mx[gr] = (gr >> 1) == half ? hi[gr & 1] : -CUDART_INF_F;
             }
-        };
-        if (bits == 2) quantize_row(std::integral_constant<int, 2>{});
-        else quantize_row(std::integral_constant<int, 4>{});
-        tc_fence_before();
-        if (valid) {
-            if (f8) {
-                uint16_t *m = reinterpret_cast<uint16_t *>(meta + (size_t)tok * NG * 2);
+            if (spans) {      // uniform: a property of the KV head
+                ext_sh[half][row] = make_float4(lo[0], hi[0], lo[1], hi[1]);
+                arith_sync();
+                const float4 o = ext_sh[half ^ 1][row];
 #pragma unroll
-                for (int g = 0; g < NG; ++g) m[g] = (uint16_t)hz[g];
-            } else {
-                uint32_t *m = reinterpret_cast<uint32_t *>(meta + (size_t)tok * NG * 4);
-                if constexpr (NG == 4) *reinterpret_cast<uint4 *>(m) = make_uint4(hz[0], hz[1], hz[2], hz[3]);
-                else if constexpr (NG == 2) *reinterpret_cast<uint2 *>(m) = make_uint2(hz[0], hz[1]);
-                else m[0] = hz[0];
+                for (int gr = 0; gr < kGranules; ++gr)
+                    if ((gr >> 1) != half) {
+                        mn[gr] = (gr & 1) ? o.z : o.x;
+                        mx[gr] = (gr & 1) ? o.w : o.y;
+                    }
+                arith_sync();      // the buffer is rewritten for the next tile
+            }
+
+            // ---- scale and zero point of the groups this thread has a part in
+            float hf[NG], zf[NG], rq[NG];
+            uint32_t hz[NG];
+#pragma unroll
+            for (int g = 0; g < NG; ++g) {
+                float glo = CUDART_INF_F, ghi = -CUDART_INF_F;
+#pragma unroll
+                for (int gr = 0; gr < kGranules; ++gr)
+                    if (((gmap >> (2 * gr)) & 3u) == (uint32_t)g) {
+                        glo = fminf(glo, mn[gr]);
+                        ghi = fmaxf(ghi, mx[gr]);
+                    }
+                if (glo > ghi) {      // a group of the other half alone: not this thread's business (uniform over the warp)
+                    hz[g] = 0u; hf[g] = 0.f; zf[g] = 0.f; rq[g] = 0.f;
+                    continue;
+                }
+                group_parameters(glo, ghi, alpha_g[g], qmaxf, f8, hz[g], hf[g], zf[g]);
+                // degenerate group (h == 0): every quotient is taken as 0.  1/qmax is 1/3 or 1/15 rounded: see pack16
+                rq[g] = hf[g] != 0.0f ? __fmul_rn(__frcp_rn(hf[g]), bits == 2 ? 1.0f / 3.0f : 1.0f / 15.0f) : 0.0f;
+            }
+
+            // ---- the codes of the thread's two granules, one store of its half of the packed row
+            auto quantize_half = [&](auto bits_tag) {
+                constexpr int BITS = decltype(bits_tag)::value;      // a compile-time constant inside
+                constexpr int NW = BITS / 2;
+                uint32_t cw[2][2][NW];                               // [granule][chunk][word]
+#pragma unroll
+                for (int gr = 0; gr < 2; ++gr) {
+                    const uint32_t g = (gmap >> (2 * (2 * half + gr))) & 3u;
+                    float hg = hf[0], zg = zf[0], rg = rq[0];
+#pragma unroll
+                    for (int i = 1; i < NG; ++i)
+                        if (g == (uint32_t)i) { hg = hf[i]; zg = zf[i]; rg = rq[i]; }
+                    uint32_t d0[NW], d1[NW];
+                    pack16<BITS>(gr == 0 ? x0 : x2, zg, rg, cw[gr][0], d0);
+                    pack16<BITS>(gr == 0 ? x1 : x3, zg, rg, cw[gr][1], d1);
+                    uint32_t any = 0u;
+#pragma unroll
+                    for (int i = 0; i < NW; ++i) any |= d0[i] | d1[i];
+                    if (__any_sync(0xffffffffu, any != 0u)) {      // rare: some quotient of the warp lies next to a rounding boundary
+                        repair16<BITS>(hg, zg, trow + 32 * gr, cw[gr][0], d0);
+                        repair16<BITS>(hg, zg, trow + 32 * gr + 16, cw[gr][1], d1);
+                    }
+                }
+                if (valid) {
+                    uint32_t *chalf = reinterpret_cast<uint32_t *>(codes + (size_t)tok * packed_row_bytes(BITS)) + half * (2 * BITS);
+                    if constexpr (BITS == 2) {
+                        *reinterpret_cast<uint4 *>(chalf) = make_uint4(cw[0][0][0], cw[0][1][0], cw[1][0][0], cw[1][1][0]);
+                    } else {
+                        *reinterpret_cast<uint4 *>(chalf) = make_uint4(cw[0][0][0], cw[0][0][1], cw[0][1][0], cw[0][1][1]);
+                        *reinterpret_cast<uint4 *>(chalf + 4) = make_uint4(cw[1][0][0], cw[1][0][1], cw[1][1][0], cw[1][1][1]);
+                    }
+                }
+            };
+            if (bits == 2) quantize_half(std::integral_constant<int, 2>{});
+            else quantize_half(std::integral_constant<int, 4>{});
+            // the accumulator may be overwritten: the last tensor-memory read of this tile (a repair) is behind us
+            tc_fence_before();
+            mbar_arrive(bar_free + 8 * (t & 1));
+            // {scale, zero}: group g is written by the half that holds its first granule
+            if (valid) {
+#pragma unroll
+                for (int g = 0; g < NG; ++g) {
+                    int first = 0;
+#pragma unroll
+                    for (int gr = kGranules - 1; gr >= 0; --gr)
+                        if (((gmap >> (2 * gr)) & 3u) == (uint32_t)g) first = gr;
+                    if ((first >> 1) == half) {
+                        if (f8) reinterpret_cast<uint16_t *>(meta + (size_t)tok * NG * 2)[g] = (uint16_t)hz[g];
+                        else reinterpret_cast<uint32_t *>(meta + (size_t)tok * NG * 4)[g] = hz[g];
+                    }
+                }
             }
         }
     }
 
-    // ---- leave: nothing of this CTA is in flight any more (a failed wait still drains its own copies)
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    if (fail_sh && tid == 0 && a.c.status) atomicOr(a.c.status, SKVQ_STATUS_COPY_TIMEOUT);
+    // ---- leave: nothing of this CTA is in flight any more
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, kTmemColumns);
+    if (tid == 0 && fail_sh && a.c.status) atomicOr(a.c.status, SKVQ_STATUS_COPY_TIMEOUT);
+    if (control) tmem_dealloc(tmem, kTmemColumns);
+}
+
+}  // namespace
+
+namespace {
+
+// cuTensorMapEncodeTiled through the runtime's driver entry point (the library does not link against the driver).
+using EncodeTiled = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                 const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiled encode_tiled()
+{
+    static EncodeTiled fn = [] {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeTiled>(p);
+    }();
+    return fn;
+}
+
+// The input [B][n_new][Hkv][D] as a tensor of (channel of the token row, token, sequence); a box is 64 channels of 128
+// tokens of one sequence, stored in the 128-byte swizzle.  Tokens past n_new read as zeros.
+cudaError_t make_input_map(CUtensorMap *map, const __half *x, const Shape &s, int n_new)
+{
+    const EncodeTiled enc = encode_tiled();
+    if (!enc) return cudaErrorNotSupported;
+    const cuuint64_t row_elems = (cuuint64_t)s.Hkv * kHeadDim;
+    const cuuint64_t dims[3] = {row_elems, (cuuint64_t)n_new, (cuuint64_t)s.B};
+    const cuuint64_t strides[2] = {row_elems * 2, row_elems * 2 * (cuuint64_t)n_new};      // bytes: token, sequence
+    const cuuint32_t box[3] = {64, (cuuint32_t)kTileRows, 1};
+    const cuuint32_t elem[3] = {1, 1, 1};
+    const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<__half *>(x), dims, strides, box, elem,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+template <int G>
+cudaError_t launch_g(const AppendArgs &a, const CUtensorMap &mk, const CUtensorMap &mv, dim3 grid, cudaStream_t stream)
+{
+    static unsigned long long configured = 0;      // one bit per device
+    const cudaError_t e = configure_smem_once(append_tile_kernel<G>, kSmemBytes, configured);
+    if (e != cudaSuccess) return e;
+    append_tile_kernel<G><<<grid, kTileThreads, kSmemBytes, stream>>>(a, mk, mv);
+    return cudaGetLastError();
 }
 
 }  // namespace
@@ -316,24 +486,16 @@ __global__ void __launch_bounds__(kTileRows, 3) append_tile_kernel(AppendArgs a)
 cudaError_t launch_append_tiles(const AppendArgs &a, cudaStream_t stream)
 {
     const Shape &s = a.s;
+    alignas(64) CUtensorMap mk, mv;
+    cudaError_t e = make_input_map(&mk, a.k, s, a.n_new);
+    if (e != cudaSuccess) return e;
+    e = make_input_map(&mv, a.v, s, a.n_new);
+    if (e != cudaSuccess) return e;
     const int max_tiles = (a.n_new + kTileRows - 1) / kTileRows;
     dim3 grid(2 * ((max_tiles + kTilesPerCta - 1) / kTilesPerCta), s.Hkv, s.B);      // x: (run of tiles, tensor)
-    static unsigned long long configured[3] = {0, 0, 0};      // one bit per device, per instantiation
-    cudaError_t e;
-    if (s.G == 128) {
-        e = configure_smem_once(append_tile_kernel<128>, kSmemBytes, configured[0]);
-        if (e != cudaSuccess) return e;
-        append_tile_kernel<128><<<grid, kTileRows, kSmemBytes, stream>>>(a);
-    } else if (s.G == 64) {
-        e = configure_smem_once(append_tile_kernel<64>, kSmemBytes, configured[1]);
-        if (e != cudaSuccess) return e;
-        append_tile_kernel<64><<<grid, kTileRows, kSmemBytes, stream>>>(a);
-    } else {
-        e = configure_smem_once(append_tile_kernel<32>, kSmemBytes, configured[2]);
-        if (e != cudaSuccess) return e;
-        append_tile_kernel<32><<<grid, kTileRows, kSmemBytes, stream>>>(a);
-    }
-    return cudaGetLastError();
+    if (s.G == 128) return launch_g<128>(a, mk, mv, grid, stream);
+    if (s.G == 64) return launch_g<64>(a, mk, mv, grid, stream);
+    return launch_g<32>(a, mk, mv, grid, stream);
 }
 
 }  // namespace skvq
