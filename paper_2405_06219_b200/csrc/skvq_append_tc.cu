@@ -8,19 +8,18 @@
 // reordered row along one lane of the tensor memory: lane m is token m of the tile.  Group minimum and maximum, scale
 // and zero point, the codes and their packing are then register arithmetic without shuffles.
 //
-// One CTA = one (sequence, KV head, tensor K or V) and a run of consecutive 128-token tiles; 256 arithmetic threads and
-// one control warp.  Arithmetic warps w and w + 4 share the 32 tokens of lane quadrant w & 3: the first takes stored
+// One CTA = 256 threads = one (sequence, KV head, tensor K or V) and a run of consecutive 128-token tiles.  Warps w and w + 4 share the 32 tokens of lane quadrant w & 3: the first takes stored
 // channels 0-63 of each, the second 64-127 (a group that spans both halves has its extremes exchanged through shared
 // memory).  Nothing but mbarriers orders the two sides:
-//   copy      the control lane brings a tile in with two tensor-map copies (cp.async.bulk.tensor, 64 channels x 128
+//   copy      thread 0 brings a tile in with two tensor-map copies (cp.async.bulk.tensor, 64 channels x 128
 //             tokens each, 128-byte swizzle: the K-major operand layout of the MMA), two tiles ahead of the arithmetic;
 //             rows past the end of the input are filled with zeros by the copy engine;
-//   MMA       the control lane issues 8 k-steps per tile and commits them to an mbarrier; two accumulators in tensor
+//   MMA       thread 0 issues 8 k-steps per tile, before it starts on its own share of the tile in front, and commits them to an mbarrier; two accumulators in tensor
 //             memory, so the MMAs of tile t+1 run under the arithmetic of tile t;
-//   quantize  every arithmetic thread reads its half row (64 values) from tensor memory into registers once: the
+//   quantize  every thread reads its half row (64 values) from tensor memory into registers once: the
 //             extremes of its two 32-channel granules (groups are unions of granules), scale and zero point, the
 //             codes, then one 16-byte store of its half of the packed row, and the {scale, zero} words; its arrival on
-//             the accumulator's mbarrier lets the control lane reuse it.
+//             the accumulator's mbarrier lets thread 0 reuse it.
 // Every wait is bounded; a wait that ran out is reported through the cache's status word, the threads then run to the end
 // of their loops without waiting or storing.  Two CTAs per SM (96 KB of shared memory and 256 tensor-memory columns
 // each).  The quantizer arithmetic is that of append_kernel (explicitly rounded fp32 operations), so both kernels
@@ -40,8 +39,7 @@ using namespace mmak;
 using namespace tc5;
 
 constexpr int kTileRows = 128;                       // tokens per tile = rows of the MMA
-constexpr int kArithThreads = 2 * kTileRows;         // two threads per token row
-constexpr int kTileThreads = kArithThreads + 32;     // and the control warp
+constexpr int kTileThreads = 2 * kTileRows;          // two threads per token row
 constexpr int kTilesPerCta = 8;                      // consecutive tiles one CTA works through
 constexpr int kOperandBytes = kTileRows * kHeadDim * 2;      // 32 KB: a 128 x 128 fp16 operand
 constexpr int kSmemBytes = 3 * kOperandBytes + 1024;      // P and two tiles of X, and room to align them to 1024 bytes
@@ -72,8 +70,7 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-// Barrier 1: the arithmetic threads only (the control warp never joins it).
-__device__ __forceinline__ void arith_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+__device__ __forceinline__ void arith_sync() { __syncthreads(); }
 
 // Stored scale and zero point of a group from its extremes (Eq. 2; both ends clipped by alpha): the words that go to
 // the cache, and the values the codes are computed against.
@@ -180,7 +177,7 @@ __device__ __forceinline__ void extremes16(const float (&x)[16], float &lo, floa
 }
 
 template <int G>
-__global__ void __maxnreg__(112)      // two CTAs of nine warps per SM
+__global__ void __launch_bounds__(kTileThreads, 2)
 append_tile_kernel(AppendArgs a, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v)
 {
     constexpr int NG = kHeadDim / G;
@@ -191,7 +188,7 @@ append_tile_kernel(AppendArgs a, const __grid_constant__ CUtensorMap map_k, cons
     __shared__ __align__(16) float4 ext_sh[2][kTileRows];      // {min, max} of a half row's two granules, for the thread of the other half
     const Shape &s = a.s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const bool control = warp == kArithThreads / 32;
+    const bool control = tid == 0;      // thread 0 also copies and issues the MMAs
     const int quad = warp & 3, half = (warp >> 2) & 1;         // tensor-memory lanes 32*quad .. +31; stored channels 64*half .. +63
     const int row = 32 * quad + lane;                          // this thread's token of every tile
     const int b = blockIdx.z, tensor = blockIdx.x & 1, h = blockIdx.y;
@@ -214,20 +211,19 @@ append_tile_kernel(AppendArgs a, const __grid_constant__ CUtensorMap map_k, cons
     const uint32_t bar_free = bar_full + 32;           // + 8 * (t & 1): every arithmetic thread is done with the accumulator of tile t
 
     // ---- once per CTA: the permutation operand, the tensor memory, the barriers
-    if (!control) {
+    {
         uint4 *p4 = reinterpret_cast<uint4 *>(P);
 #pragma unroll
-        for (int i = 0; i < kOperandBytes / 16 / kArithThreads; ++i) p4[tid + i * kArithThreads] = make_uint4(0u, 0u, 0u, 0u);
-    } else {
-        tmem_alloc(smem_u32(&tmem_sh), kTmemColumns);
-        if (lane == 0) {
+        for (int i = 0; i < kOperandBytes / 16 / kTileThreads; ++i) p4[tid + i * kTileThreads] = make_uint4(0u, 0u, 0u, 0u);
+    }
+    if (warp == 0) tmem_alloc(smem_u32(&tmem_sh), kTmemColumns);
+    if (control) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) mbar_init(bar_full + 8 * i, 1);
-            mbar_init(bar_free, kArithThreads);
-            mbar_init(bar_free + 8, kArithThreads);
-            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-            fail_sh = 0;
-        }
+        for (int i = 0; i < 4; ++i) mbar_init(bar_full + 8 * i, 1);
+        mbar_init(bar_free, kTileThreads);
+        mbar_init(bar_free + 8, kTileThreads);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fail_sh = 0;
     }
     __syncthreads();
     if (tid < kHeadDim) {
@@ -242,50 +238,46 @@ append_tile_kernel(AppendArgs a, const __grid_constant__ CUtensorMap map_k, cons
     const uint32_t tmem = tmem_sh;
     volatile int *fail = &fail_sh;
 
-    if (control) {
-        // ================================================================ control warp: one lane copies and issues
-        if (lane == 0) {
-            const CUtensorMap *map = tensor ? &map_v : &map_k;
-            const uint64_t dP = smem_desc(smem_u32(P), kLboBytes, kSboBytes);
-            constexpr uint32_t kIdesc = idesc_f16_f32(kTileRows, kHeadDim);
-            bool alive = true;
-            auto copy_tile = [&](int t) {      // both halves of tile t into buffer t & 1
-                const uint32_t dst = smem_u32(X) + (t & 1) * kOperandBytes, bar = bar_full + 8 * (t & 1);
-                const int tok = f0 + (t_begin + t) * kTileRows - L0;      // row of the input
-                mbar_expect_tx(bar, kOperandBytes);
-                tma_load_3d(dst, map, h * kHeadDim, tok, b, bar);
-                tma_load_3d(dst + kHalfTileBytes, map, h * kHeadDim + 64, tok, b, bar);
-            };
-            copy_tile(0);
-            if (T > 1) copy_tile(1);
-            for (int t = 0; t < T; ++t) {
-                if (*fail) alive = false;
-                const uint32_t ph = (uint32_t)(t >> 1) & 1u;
-                if (alive && !mbar_wait_bounded(bar_full + 8 * (t & 1), ph)) { alive = false; *fail = 1; }
-                if (t >= 2 && alive && !mbar_wait_bounded(bar_free + 8 * (t & 1), ph ^ 1u)) { alive = false; *fail = 1; }      // tile t-2 has been read
-                tc_fence_after();
-                const uint32_t xb = smem_u32(X) + (t & 1) * kOperandBytes;
+    // ---- thread 0's second job: copies and MMAs, one tile ahead of the arithmetic
+    const CUtensorMap *map = tensor ? &map_v : &map_k;
+    const uint64_t dP = smem_desc(smem_u32(P), kLboBytes, kSboBytes);
+    constexpr uint32_t kIdesc = idesc_f16_f32(kTileRows, kHeadDim);
+    bool alive = true;
+    auto copy_tile = [&](int t) {      // both halves of tile t into buffer t & 1
+        const uint32_t dst = smem_u32(X) + (t & 1) * kOperandBytes, bar = bar_full + 8 * (t & 1);
+        const int tok = f0 + (t_begin + t) * kTileRows - L0;      // row of the input
+        mbar_expect_tx(bar, kOperandBytes);
+        tma_load_3d(dst, map, h * kHeadDim, tok, b, bar);
+        tma_load_3d(dst + kHalfTileBytes, map, h * kHeadDim + 64, tok, b, bar);
+    };
+    auto issue_mmas = [&](int t) {     // once tile t has landed and the arithmetic is done with tile t-2, which had the same accumulator
+        const uint32_t ph = (uint32_t)(t >> 1) & 1u;
+        if (alive && !mbar_wait_bounded(bar_full + 8 * (t & 1), ph)) { alive = false; *fail = 1; }
+        if (t >= 2 && alive && !mbar_wait_bounded(bar_free + 8 * (t & 1), ph ^ 1u)) { alive = false; *fail = 1; }
+        tc_fence_after();
+        const uint32_t xb = smem_u32(X) + (t & 1) * kOperandBytes;
 #pragma unroll
-                for (int ks = 0; ks < kHeadDim / 16; ++ks) {      // 16 source channels = 32 bytes of a swizzled row per k-step
-                    const uint64_t dX = smem_desc_sw128(xb + (ks >> 2) * kHalfTileBytes + (ks & 3) * 32);
-                    umma_f16(tmem + (uint32_t)(t & 1) * kHeadDim, dX, dP + ((ks * 2 * kLboBytes) >> 4), kIdesc, ks > 0 ? 1u : 0u);
-                }
-                umma_commit(bar_mma + 8 * (t & 1));
-                if (t + 2 < T) {      // the buffer is free once these MMAs have read it
-                    if (alive && !mbar_wait_bounded(bar_mma + 8 * (t & 1), ph)) { alive = false; *fail = 1; }
-                    copy_tile(t + 2);
-                }
-            }
-            // nothing of this lane's may be in flight when the CTA leaves: the last copies and MMAs
-            for (int t = max(T - 2, 0); t < T; ++t) {
-                const uint32_t ph = (uint32_t)(t >> 1) & 1u;
-                if (alive && !mbar_wait_bounded(bar_full + 8 * (t & 1), ph)) alive = false;
-                if (alive && !mbar_wait_bounded(bar_mma + 8 * (t & 1), ph)) alive = false;
-            }
+        for (int ks = 0; ks < kHeadDim / 16; ++ks) {      // 16 source channels = 32 bytes of a swizzled row per k-step
+            const uint64_t dX = smem_desc_sw128(xb + (ks >> 2) * kHalfTileBytes + (ks & 3) * 32);
+            umma_f16(tmem + (uint32_t)(t & 1) * kHeadDim, dX, dP + ((ks * 2 * kLboBytes) >> 4), kIdesc, ks > 0 ? 1u : 0u);
         }
-        __syncwarp();
-    } else {
-        // ================================================================ arithmetic threads
+        umma_commit(bar_mma + 8 * (t & 1));
+    };
+    auto refill = [&](int t) {         // the buffer of tile t takes tile t+2 once the MMAs of tile t have read it
+        if (t + 2 >= T) return;
+        if (alive && !mbar_wait_bounded(bar_mma + 8 * (t & 1), (uint32_t)(t >> 1) & 1u)) { alive = false; *fail = 1; }
+        copy_tile(t + 2);
+    };
+    if (control) {
+        copy_tile(0);
+        if (T > 1) copy_tile(1);
+        issue_mmas(0);
+        refill(0);
+    }
+    __syncwarp();
+
+    {
+        // ================================================================ the arithmetic
         const int bits = tensor ? s.v_bits : s.k_bits;
         const bool f8 = s.meta_fp8 != 0;
         const size_t bh = (size_t)b * s.Hkv + h;
@@ -300,10 +292,10 @@ append_tile_kernel(AppendArgs a, const __grid_constant__ CUtensorMap map_k, cons
         uint8_t *meta = reinterpret_cast<uint8_t *>(tensor ? a.c.v_meta : a.c.k_meta) + bh * (size_t)s.cap * NG * (f8 ? 2 : 4);
         const uint32_t tmem_half = tmem + ((uint32_t)(quad * 32) << 16) + 64 * half;      // this thread's lane, its first column
         const float qmaxf = (float)code_max(bits);
-        bool alive = true;
-
         for (int t = 0; t < T; ++t) {
             if (*fail) alive = false;
+            if (control && t + 1 < T) issue_mmas(t + 1);      // they run under this tile's arithmetic
+            __syncwarp();
             if (alive && !mbar_wait_bounded(bar_mma + 8 * (t & 1), (uint32_t)(t >> 1) & 1u)) { alive = false; *fail = 1; }
             tc_fence_after();
             const uint32_t trow = tmem_half + (uint32_t)(t & 1) * kHeadDim;
@@ -424,6 +416,8 @@ append_tile_kernel(AppendArgs a, const __grid_constant__ CUtensorMap map_k, cons
                     }
                 }
             }
+            if (control) refill(t + 1);
+            __syncwarp();
         }
     }
 
@@ -431,7 +425,7 @@ append_tile_kernel(AppendArgs a, const __grid_constant__ CUtensorMap map_k, cons
     tc_fence_before();
     __syncthreads();
     if (tid == 0 && fail_sh && a.c.status) atomicOr(a.c.status, SKVQ_STATUS_COPY_TIMEOUT);
-    if (control) tmem_dealloc(tmem, kTmemColumns);
+    if (warp == 0) tmem_dealloc(tmem, kTmemColumns);
 }
 
 }  // namespace
@@ -475,6 +469,12 @@ template <int G>
 cudaError_t launch_g(const AppendArgs &a, const CUtensorMap &mk, const CUtensorMap &mv, dim3 grid, cudaStream_t stream)
 {
     static unsigned long long configured = 0;      // one bit per device
+    if (!(configured & (1ull << (current_device() & (kMaxDevices - 1))))) {
+        // two CTAs of 97 KB each only fit the largest shared-memory carveout
+        const cudaError_t ec = cudaFuncSetAttribute(append_tile_kernel<G>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                                    (int)cudaSharedmemCarveoutMaxShared);
+        if (ec != cudaSuccess) return ec;
+    }
     const cudaError_t e = configure_smem_once(append_tile_kernel<G>, kSmemBytes, configured);
     if (e != cudaSuccess) return e;
     append_tile_kernel<G><<<grid, kTileThreads, kSmemBytes, stream>>>(a, mk, mv);
