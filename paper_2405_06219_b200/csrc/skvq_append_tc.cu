@@ -70,7 +70,8 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void arith_sync() { __syncthreads(); }
+// Barrier 1 + quad: the two warps that share the tokens of lane quadrant quad (64 threads).
+__device__ __forceinline__ void pair_sync(int quad) { asm volatile("bar.sync %0, 64;" ::"r"(1 + quad) : "memory"); }
 
 // Stored scale and zero point of a group from its extremes (Eq. 2; both ends clipped by alpha): the words that go to
 // the cache, and the values the codes are computed against.
@@ -185,7 +186,7 @@ append_tile_kernel(AppendArgs a, const __grid_constant__ CUtensorMap map_k, cons
     __shared__ __align__(8) uint64_t bar_sh[6];
     __shared__ uint32_t tmem_sh;
     __shared__ int fail_sh;
-    __shared__ __align__(16) float4 ext_sh[2][kTileRows];      // {min, max} of a half row's two granules, for the thread of the other half
+    __shared__ __align__(16) float4 ext_sh[2][2][kTileRows];   // [tile & 1][half][token]: {min, max} of a half row's two granules, for the thread of the other half
     const Shape &s = a.s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool control = tid == 0;      // thread 0 also copies and issues the MMAs
@@ -331,16 +332,17 @@ append_tile_kernel(AppendArgs a, const __grid_constant__ CUtensorMap map_k, cons
                 mx[gr] = (gr >> 1) == half ? hi[gr & 1] : -CUDART_INF_F;
             }
             if (spans) {      // uniform: a property of the KV head
-                ext_sh[half][row] = make_float4(lo[0], hi[0], lo[1], hi[1]);
-                arith_sync();
-                const float4 o = ext_sh[half ^ 1][row];
+                // Two buffers and one barrier per tile: a thread rewrites the entry of tile t when it works on tile t+2, behind
+                // the barrier of tile t+1, which its partner reaches only after it has read the entry of tile t.
+                ext_sh[t & 1][half][row] = make_float4(lo[0], hi[0], lo[1], hi[1]);
+                pair_sync(quad);
+                const float4 o = ext_sh[t & 1][half ^ 1][row];
 #pragma unroll
                 for (int gr = 0; gr < kGranules; ++gr)
                     if ((gr >> 1) != half) {
                         mn[gr] = (gr & 1) ? o.z : o.x;
                         mx[gr] = (gr & 1) ? o.w : o.y;
                     }
-                arith_sync();      // the buffer is rewritten for the next tile
             }
 
             // ---- scale and zero point of the groups this thread has a part in
