@@ -40,7 +40,6 @@ using namespace tc5;
 
 constexpr int kTileRows = 128;                       // tokens per tile = rows of the MMA
 constexpr int kTileThreads = 2 * kTileRows;          // two threads per token row
-constexpr int kTilesPerCta = 8;                      // consecutive tiles one CTA works through
 constexpr int kOperandBytes = kTileRows * kHeadDim * 2;      // 32 KB: a 128 x 128 fp16 operand
 constexpr int kSmemBytes = 3 * kOperandBytes + 1024;      // P and two tiles of X, and room to align them to 1024 bytes
 constexpr uint32_t kLboBytes = 128;                  // P (no swizzle): between core matrices along K
@@ -179,7 +178,7 @@ __device__ __forceinline__ void extremes16(const float (&x)[16], float &lo, floa
 
 template <int G>
 __global__ void __launch_bounds__(kTileThreads, 2)
-append_tile_kernel(AppendArgs a, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v)
+append_tile_kernel(AppendArgs a, int tiles_per_cta, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v)
 {
     constexpr int NG = kHeadDim / G;
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -200,7 +199,7 @@ append_tile_kernel(AppendArgs a, const __grid_constant__ CUtensorMap map_k, cons
     int f0, f1;
     bulk_range(L0, s.n_sink, max(L1 - s.W, 0), f0, f1);
     const int n_tiles = (f1 - f0 + kTileRows - 1) / kTileRows;
-    const int t_begin = (blockIdx.x >> 1) * kTilesPerCta, t_end = min(n_tiles, t_begin + kTilesPerCta);
+    const int t_begin = (blockIdx.x >> 1) * tiles_per_cta, t_end = min(n_tiles, t_begin + tiles_per_cta);      // this CTA's run of tiles
     if (t_begin >= t_end) return;
     if (!SKVQ_IN_BOUNDS(f0 >= L0 && f1 <= s.cap && f1 - L0 <= a.n_new, a.c.status)) return;
     const int T = t_end - t_begin;
@@ -468,7 +467,7 @@ cudaError_t make_input_map(CUtensorMap *map, const __half *x, const Shape &s, in
 }
 
 template <int G>
-cudaError_t launch_g(const AppendArgs &a, const CUtensorMap &mk, const CUtensorMap &mv, dim3 grid, cudaStream_t stream)
+cudaError_t launch_g(const AppendArgs &a, int tiles_per_cta, const CUtensorMap &mk, const CUtensorMap &mv, dim3 grid, cudaStream_t stream)
 {
     static unsigned long long configured = 0;      // one bit per device
     if (!(configured & (1ull << (current_device() & (kMaxDevices - 1))))) {
@@ -479,7 +478,7 @@ cudaError_t launch_g(const AppendArgs &a, const CUtensorMap &mk, const CUtensorM
     }
     const cudaError_t e = configure_smem_once(append_tile_kernel<G>, kSmemBytes, configured);
     if (e != cudaSuccess) return e;
-    append_tile_kernel<G><<<grid, kTileThreads, kSmemBytes, stream>>>(a, mk, mv);
+    append_tile_kernel<G><<<grid, kTileThreads, kSmemBytes, stream>>>(a, tiles_per_cta, mk, mv);
     return cudaGetLastError();
 }
 
@@ -494,10 +493,16 @@ cudaError_t launch_append_tiles(const AppendArgs &a, cudaStream_t stream)
     e = make_input_map(&mv, a.v, s, a.n_new);
     if (e != cudaSuccess) return e;
     const int max_tiles = (a.n_new + kTileRows - 1) / kTileRows;
-    dim3 grid(2 * ((max_tiles + kTilesPerCta - 1) / kTilesPerCta), s.Hkv, s.B);      // x: (run of tiles, tensor)
-    if (s.G == 128) return launch_g<128>(a, mk, mv, grid, stream);
-    if (s.G == 64) return launch_g<64>(a, mk, mv, grid, stream);
-    return launch_g<32>(a, mk, mv, grid, stream);
+    // A CTA's set-up (the permutation operand, the tensor memory, the first copies) costs about two tiles' time: long runs
+    // of tiles per CTA, as long as the grid still has several waves of the two CTAs an SM holds.
+    const long total_tiles = (long)max_tiles * 2 * s.Hkv * s.B;
+    const long want_ctas = 8L * 2 * sm_count();      // measured: 32 tiles per CTA 3.55, 16: 3.49, 8: 3.37, 4: 3.10 TB/s on a 1 GiB chunk
+    int tiles_per_cta = (int)(total_tiles / want_ctas);
+    tiles_per_cta = tiles_per_cta < 4 ? 4 : (tiles_per_cta > 32 ? 32 : tiles_per_cta);
+    dim3 grid(2 * ((max_tiles + tiles_per_cta - 1) / tiles_per_cta), s.Hkv, s.B);      // x: (run of tiles, tensor)
+    if (s.G == 128) return launch_g<128>(a, tiles_per_cta, mk, mv, grid, stream);
+    if (s.G == 64) return launch_g<64>(a, tiles_per_cta, mk, mv, grid, stream);
+    return launch_g<32>(a, tiles_per_cta, mk, mv, grid, stream);
 }
 
 }  // namespace skvq
