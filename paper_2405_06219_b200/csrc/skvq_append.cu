@@ -342,8 +342,7 @@ cudaError_t launch_append(const Shape &s, const CachePtrs &c, const __half *k, c
                           const int32_t *n_new_per_seq, int n_new, cudaStream_t stream)
 {
     if (n_new <= 0) return cudaSuccess;
-    // the tile kernel serves 2- and 4-bit codes (equal or unequal groups); the other widths go through append_kernel
-    const bool bulk = n_new >= kBulkTok && plain_width(s.k_bits) && plain_width(s.v_bits);
+    const bool bulk = n_new >= kBulkTok;
     AppendArgs a{s, c, k, v, n_new_per_seq, n_new, bulk ? 1 : 0};
     // what append_kernel keeps: evictions (at most W), and new tokens outside the bulk tiles (fewer than W + 128
     // when there are bulk tiles, all of them otherwise)

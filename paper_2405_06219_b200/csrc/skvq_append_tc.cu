@@ -7,6 +7,8 @@
 // channels, fp16 in, fp32 accumulators in tensor memory) replaces 16384 two-byte gathers, and it lays every token's
 // reordered row along one lane of the tensor memory: lane m is token m of the tile.  Group minimum and maximum, scale
 // and zero point, the codes and their packing are then register arithmetic without shuffles.
+// All code widths: 2- and 4-bit fields as they are, 3-bit codes closed up from 4-bit fields into the row's bit stream,
+// three-level codes from 2-bit fields into base-3 bytes.
 //
 // One CTA = 256 threads = one (sequence, KV head, tensor K or V) and a run of consecutive 128-token tiles.  Warps w and w + 4 share the 32 tokens of lane quadrant w & 3: the first takes stored
 // channels 0-63 of each, the second 64-127 (a group that spans both halves has its extremes exchanged through shared
@@ -100,7 +102,9 @@ __device__ __forceinline__ float mul_sat(float a, float b)      // clamp(RN(a * 
     return r;
 }
 
-// Codes of 16 consecutive stored channels against (hf, zf): BITS / 2 words, code j in bits [j*BITS, (j+1)*BITS) of the run.
+// Codes of 16 consecutive stored channels against (hf, zf) in fields of FIELD bits (2 or 4; QMAX = the largest code, which
+// need not fill the field: 3-bit codes travel in 4-bit fields, three-level codes in 2-bit fields until the row is
+// packed): FIELD / 2 words, code j in bits [j*FIELD, (j+1)*FIELD) of the run.
 // code = clamp(rint(RN((x - z) / h)), 0, qmax) with IEEE division.  Instead of dividing, u = sat(d * r) with
 // r = RN(RN(1/h) / qmax) is the clamped quotient on the scale [0, 1], within 5 * 2^-24 relative of the IEEE quotient / qmax;
 // wherever every value within 2^-18 relative of it rounds to the same integer, that integer is the code.  The test is two
@@ -108,10 +112,10 @@ __device__ __forceinline__ float mul_sat(float a, float b)      // clamp(RN(a * 
 // the quotient scaled down and one scaled up by 2^-18; both results are packed (four partial sums each, so that no
 // addition waits for the one before), and fields in which the two packed runs differ are elements in doubt (a quotient
 // next to k + 0.5, exact ties included): doubt[] has their bits set and repair16 redoes them.
-template <int BITS>
+template <int BITS, int QMAX>
 __device__ __forceinline__ void pack16(const float (&x)[16], float zf, float r, uint32_t (&words)[BITS / 2], uint32_t (&doubt)[BITS / 2])
 {
-    constexpr int qmax = (1 << BITS) - 1, PER_WORD = 32 / BITS, NW = BITS / 2, LANES = 4 / NW;      // partial sums per word
+    constexpr int qmax = QMAX, PER_WORD = 32 / BITS, NW = BITS / 2, LANES = 4 / NW;      // BITS = field width; partial sums per word
     constexpr float MAGIC = 12582912.0f;                       // 0x4B400000
     constexpr float UP = (float)qmax * (1.0f + 3.814697265625e-06f), DN = (float)qmax * (1.0f - 3.814697265625e-06f);   // exact products
     uint32_t kconst = 0u;
@@ -141,16 +145,16 @@ __device__ __forceinline__ void pack16(const float (&x)[16], float zf, float r, 
 // The elements of a 16-column run that pack16 left in doubt, redone by the defining formula: the warp walks the union of
 // its doubtful columns, re-reads each from tensor memory (taddr = this warp's lanes, first column of the run) and the
 // lanes concerned patch their field.  Every lane of the warp must call this.
-template <int BITS>
+template <int BITS, int QMAX>
 __device__ __forceinline__ void repair16(float hf, float zf, uint32_t taddr, uint32_t (&words)[BITS / 2], const uint32_t (&doubt)[BITS / 2])
 {
-    constexpr int qmax = (1 << BITS) - 1, PER_WORD = 32 / BITS, NW = BITS / 2;
+    constexpr int qmax = QMAX, PER_WORD = 32 / BITS, NW = BITS / 2;      // BITS = field width
 #pragma unroll
     for (int i = 0; i < NW; ++i) {
         uint32_t todo = __reduce_or_sync(0xffffffffu, doubt[i]);      // the same for every lane: the loop is uniform
         while (todo) {
             const int f = (__ffs(todo) - 1) / BITS;                    // field of this word = column i * PER_WORD + f of the run
-            const uint32_t field = (uint32_t)qmax << (f * BITS);
+            const uint32_t field = ((1u << BITS) - 1u) << (f * BITS);
             todo &= ~field;
             float xv;
             tmem_ld1(taddr + i * PER_WORD + f, xv);
@@ -185,6 +189,7 @@ append_tile_kernel(AppendArgs a, int tiles_per_cta, const __grid_constant__ CUte
     __shared__ __align__(8) uint64_t bar_sh[6];
     __shared__ uint32_t tmem_sh;
     __shared__ int fail_sh;
+    __shared__ uint32_t tern_sh[2][kTileRows];                 // [tile & 1][token]: code 64 of a three-level row, for the thread of the first half
     __shared__ __align__(16) float4 ext_sh[2][2][kTileRows];   // [tile & 1][half][token]: {min, max} of a half row's two granules, for the thread of the other half
     const Shape &s = a.s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -292,6 +297,7 @@ append_tile_kernel(AppendArgs a, int tiles_per_cta, const __grid_constant__ CUte
         uint8_t *meta = reinterpret_cast<uint8_t *>(tensor ? a.c.v_meta : a.c.k_meta) + bh * (size_t)s.cap * NG * (f8 ? 2 : 4);
         const uint32_t tmem_half = tmem + ((uint32_t)(quad * 32) << 16) + 64 * half;      // this thread's lane, its first column
         const float qmaxf = (float)code_max(bits);
+        const float qmax_inv = bits == 2 ? 1.0f / 3.0f : (bits == 4 ? 1.0f / 15.0f : (bits == 3 ? 1.0f / 7.0f : 0.5f));
         for (int t = 0; t < T; ++t) {
             if (*fail) alive = false;
             if (control && t + 1 < T) issue_mmas(t + 1);      // they run under this tile's arithmetic
@@ -361,15 +367,16 @@ append_tile_kernel(AppendArgs a, int tiles_per_cta, const __grid_constant__ CUte
                     continue;
                 }
                 group_parameters(glo, ghi, alpha_g[g], qmaxf, f8, hz[g], hf[g], zf[g]);
-                // degenerate group (h == 0): every quotient is taken as 0.  1/qmax is 1/3 or 1/15 rounded: see pack16
-                rq[g] = hf[g] != 0.0f ? __fmul_rn(__frcp_rn(hf[g]), bits == 2 ? 1.0f / 3.0f : 1.0f / 15.0f) : 0.0f;
+                // degenerate group (h == 0): every quotient is taken as 0.  1/qmax is a rounded constant: see pack16
+                rq[g] = hf[g] != 0.0f ? __fmul_rn(__frcp_rn(hf[g]), qmax_inv) : 0.0f;
             }
 
-            // ---- the codes of the thread's two granules, one store of its half of the packed row
-            auto quantize_half = [&](auto bits_tag) {
-                constexpr int BITS = decltype(bits_tag)::value;      // a compile-time constant inside
-                constexpr int NW = BITS / 2;
-                uint32_t cw[2][2][NW];                               // [granule][chunk][word]
+            // ---- the codes of the thread's two granules, then its half of the packed row.  WIDTH is the cache's code width
+            // (2, 3, 4, or kTernary); the codes are formed in fields of 2 or 4 bits.
+            auto quantize_half = [&](auto width_tag) {
+                constexpr int WIDTH = decltype(width_tag)::value;      // a compile-time constant inside
+                constexpr int FIELD = (WIDTH == 2 || WIDTH == kTernary) ? 2 : 4, QMAX = code_max(WIDTH), NW = FIELD / 2;
+                uint32_t cw[2][2][NW];                                 // [granule][chunk][word]
 #pragma unroll
                 for (int gr = 0; gr < 2; ++gr) {
                     const uint32_t g = (gmap >> (2 * (2 * half + gr))) & 3u;
@@ -378,28 +385,80 @@ append_tile_kernel(AppendArgs a, int tiles_per_cta, const __grid_constant__ CUte
                     for (int i = 1; i < NG; ++i)
                         if (g == (uint32_t)i) { hg = hf[i]; zg = zf[i]; rg = rq[i]; }
                     uint32_t d0[NW], d1[NW];
-                    pack16<BITS>(gr == 0 ? x0 : x2, zg, rg, cw[gr][0], d0);
-                    pack16<BITS>(gr == 0 ? x1 : x3, zg, rg, cw[gr][1], d1);
+                    pack16<FIELD, QMAX>(gr == 0 ? x0 : x2, zg, rg, cw[gr][0], d0);
+                    pack16<FIELD, QMAX>(gr == 0 ? x1 : x3, zg, rg, cw[gr][1], d1);
                     uint32_t any = 0u;
 #pragma unroll
                     for (int i = 0; i < NW; ++i) any |= d0[i] | d1[i];
                     if (__any_sync(0xffffffffu, any != 0u)) {      // rare: some quotient of the warp lies next to a rounding boundary
-                        repair16<BITS>(hg, zg, trow + 32 * gr, cw[gr][0], d0);
-                        repair16<BITS>(hg, zg, trow + 32 * gr + 16, cw[gr][1], d1);
+                        repair16<FIELD, QMAX>(hg, zg, trow + 32 * gr, cw[gr][0], d0);
+                        repair16<FIELD, QMAX>(hg, zg, trow + 32 * gr + 16, cw[gr][1], d1);
                     }
                 }
-                if (valid) {
-                    uint32_t *chalf = reinterpret_cast<uint32_t *>(codes + (size_t)tok * packed_row_bytes(BITS)) + half * (2 * BITS);
-                    if constexpr (BITS == 2) {
-                        *reinterpret_cast<uint4 *>(chalf) = make_uint4(cw[0][0][0], cw[0][1][0], cw[1][0][0], cw[1][1][0]);
+                uint8_t *crow = codes + (size_t)tok * packed_row_bytes(WIDTH);
+                if constexpr (WIDTH == 2) {
+                    if (valid) *reinterpret_cast<uint4 *>(crow + 16 * half) = make_uint4(cw[0][0][0], cw[0][1][0], cw[1][0][0], cw[1][1][0]);
+                } else if constexpr (WIDTH == 4) {
+                    if (valid) {
+                        *reinterpret_cast<uint4 *>(crow + 32 * half) = make_uint4(cw[0][0][0], cw[0][0][1], cw[0][1][0], cw[0][1][1]);
+                        *reinterpret_cast<uint4 *>(crow + 32 * half + 16) = make_uint4(cw[1][0][0], cw[1][0][1], cw[1][1][0], cw[1][1][1]);
+                    }
+                } else if constexpr (WIDTH == 3) {
+                    // eight 4-bit fields of a word -> 24 bits of the row's bit stream (code j in bits [3j, 3j+3)): pairs of
+                    // fields close up inside their byte, then the four bytes close up; 64 codes = 24 bytes per half row
+                    uint32_t r[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const uint32_t w = cw[i >> 2][(i >> 1) & 1][i & 1];
+                        const uint32_t p = (w & 0x07070707u) | ((w >> 1) & 0x38383838u);
+                        r[i] = (p & 0x3Fu) | ((p >> 2) & 0xFC0u) | ((p >> 4) & 0x3F000u) | ((p >> 6) & 0xFC0000u);
+                    }
+                    if (valid) {
+                        uint2 *o = reinterpret_cast<uint2 *>(crow + 24 * half);
+                        o[0] = make_uint2(r[0] | (r[1] << 24), (r[1] >> 8) | (r[2] << 16));
+                        o[1] = make_uint2((r[2] >> 16) | (r[3] << 8), r[4] | (r[5] << 24));
+                        o[2] = make_uint2((r[5] >> 8) | (r[6] << 16), (r[6] >> 16) | (r[7] << 8));
+                    }
+                } else {
+                    // three-level codes: byte n of the row = codes 5n .. 5n+4 as base-3 digits.  Bytes 0-12 belong to the
+                    // first half of the row, which needs code 64 from the second (handed over through shared memory);
+                    // bytes 13-25 to the second half (local codes 1 .. 63, then nothing: the last digits are 0).
+                    auto code = [&](int j) -> uint32_t {      // j: compile-time index into the thread's 64 codes
+                        return j < 64 ? (cw[j >> 5][(j >> 4) & 1][0] >> (2 * (j & 15))) & 3u : 0u;
+                    };
+                    if (half == 1) tern_sh[t & 1][row] = code(0);
+                    pair_sync(quad);      // two buffers, one barrier per tile: as for the extremes
+                    const uint32_t c64 = half == 0 ? tern_sh[t & 1][row] : 0u;
+                    uint32_t by[13];
+                    if (half == 0) {
+#pragma unroll
+                        for (int n = 0; n < 13; ++n) {
+                            const uint32_t last = 5 * n + 4 < 64 ? code(5 * n + 4) : c64;
+                            by[n] = code(5 * n) + 3u * code(5 * n + 1) + 9u * code(5 * n + 2) + 27u * code(5 * n + 3) + 81u * last;
+                        }
                     } else {
-                        *reinterpret_cast<uint4 *>(chalf) = make_uint4(cw[0][0][0], cw[0][0][1], cw[0][1][0], cw[0][1][1]);
-                        *reinterpret_cast<uint4 *>(chalf + 4) = make_uint4(cw[1][0][0], cw[1][0][1], cw[1][1][0], cw[1][1][1]);
+#pragma unroll
+                        for (int n = 0; n < 13; ++n)
+                            by[n] = code(5 * n + 1) + 3u * code(5 * n + 2) + 9u * code(5 * n + 3) + 27u * code(5 * n + 4) + 81u * code(5 * n + 5);
+                    }
+                    if (valid) {      // rows of 26 bytes are 2-byte aligned; the second half starts at an odd byte
+                        uint8_t *o = crow + 13 * half;
+                        if (half == 0) {
+#pragma unroll
+                            for (int n = 0; n < 6; ++n) *reinterpret_cast<uint16_t *>(o + 2 * n) = (uint16_t)(by[2 * n] | (by[2 * n + 1] << 8));
+                            o[12] = (uint8_t)by[12];
+                        } else {
+                            o[0] = (uint8_t)by[0];
+#pragma unroll
+                            for (int n = 0; n < 6; ++n) *reinterpret_cast<uint16_t *>(o + 1 + 2 * n) = (uint16_t)(by[2 * n + 1] | (by[2 * n + 2] << 8));
+                        }
                     }
                 }
             };
             if (bits == 2) quantize_half(std::integral_constant<int, 2>{});
-            else quantize_half(std::integral_constant<int, 4>{});
+            else if (bits == 4) quantize_half(std::integral_constant<int, 4>{});
+            else if (bits == 3) quantize_half(std::integral_constant<int, 3>{});
+            else quantize_half(std::integral_constant<int, kTernary>{});
             // the accumulator may be overwritten: the last tensor-memory read of this tile (a repair) is behind us
             tc_fence_before();
             mbar_arrive(bar_free + 8 * (t & 1));

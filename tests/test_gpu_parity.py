@@ -92,6 +92,9 @@ def test_chunked_and_single_token_appends_bit_exact():
     (2, dict(context=2100, batch=2, group_size=64, group_bounds=(0, 96, 128)), (1100, 1000)),               # two groups of unequal width
     (4, dict(context=1700, batch=1, ragged=None, n_q_heads=4, n_kv_heads=4, k_bits=4, v_bits=2, group_size=32,
              group_bounds=(0, 32, 64, 96, 128)), (900, 800)),                                               # mixed widths, boundaries given but equal
+    (1, dict(context=2500, batch=2, n_q_heads=4, n_kv_heads=4, k_bits=3, v_bits=3, group_size=64), (1300, 70, 1130)),  # 3-bit streams closed up from 4-bit fields
+    (2, dict(context=2300, batch=2, k_bits=3, v_bits=15, group_size=64, group_bounds=(0, 32, 128)), (1000, 1300)),     # three-level values: base-3 bytes, a code handed across the row's halves
+    (1, dict(context=1900, batch=1, n_q_heads=4, n_kv_heads=4, v_bits=15, meta_fp8=True), (900, 1000)),
 ])
 def test_bulk_appends_on_top_of_existing_tokens_bit_exact(cfg_i, kw, chunks):
     """The tile kernel of bulk appends: chunks that start at any length, several CTA runs, ragged per-sequence counts."""
