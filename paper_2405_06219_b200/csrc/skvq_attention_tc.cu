@@ -67,7 +67,8 @@ struct TCfg {
     static constexpr int kOffOs = kOffPA + kTile * 64;                   // folded value sums [4][128] fp32, by byte column
     static constexpr int kOffMisc = kOffOs + kHeads * kHeadDim * 4;      // small arrays, see the kernel
     static constexpr int kSmemBytes = kOffMisc + 1024;
-    static constexpr int kCtasPerSm = (KB == 2 && VB == 2) ? 3 : 2;      // by shared memory (69 KB at 2 bits, up to 85 KB otherwise)
+    static constexpr int kCtasPerSm = tc_ctas_per_sm(G, KB, VB);         // by shared memory (62-73 KB: three; up to 85 KB: two)
+    static_assert(kSmemBytes == tc_smem_bytes(G, KB, VB), "the host sizes the grid from the same figure");
     static_assert(kTile * 128 >= kHeads * kHeadDim * 4, "the V operand buffer doubles as query scratch in the prologue");
     static_assert(kKTile % 16 == 0 && kVTile % 16 == 0, "bulk copies move multiples of 16 bytes");
 };
