@@ -287,12 +287,20 @@ append_tile_kernel(AppendArgs a, int tiles_per_cta, const __grid_constant__ CUte
         const bool f8 = s.meta_fp8 != 0;
         const size_t bh = (size_t)b * s.Hkv + h;
         const float *alpha = (tensor ? a.c.alpha_v : a.c.alpha_k) + (size_t)h * NG;
-        float alpha_g[NG];
-#pragma unroll
-        for (int g = 0; g < NG; ++g) alpha_g[g] = alpha[g];
         const uint32_t gmap = granule_groups(tensor ? a.c.bounds_v : a.c.bounds_k, h, G, NG);      // group of every 32-channel granule
+        auto group_of = [&](int granule) { return (gmap >> (2 * granule)) & 3u; };
         // Does a group reach into both halves of the row?  Then the two threads of a token exchange their extremes.
-        const bool spans = ((gmap >> 2) & 3u) == ((gmap >> 4) & 3u);
+        const bool spans = group_of(1) == group_of(2);
+        // This thread's two granules belong to one or two groups: parameter set 0 is the group of its first granule, set 1
+        // that of its second when it is another one.  The other half's granules feed a set only when their group spans.
+        const uint32_t g0 = group_of(2 * half), g1 = group_of(2 * half + 1);
+        const bool two_sets = g1 != g0;
+        const float alpha0 = alpha[g0], alpha1 = alpha[g1];
+        const uint32_t p0 = group_of(2 * (half ^ 1)), p1 = group_of(2 * (half ^ 1) + 1);      // the partner's granules
+        const bool p0_in0 = spans && p0 == g0, p1_in0 = spans && p1 == g0, p0_in1 = spans && two_sets && p0 == g1,
+                   p1_in1 = spans && two_sets && p1 == g1;
+        // {scale, zero} of a group are written by the thread that holds its first granule
+        const bool writes0 = half == 0 || group_of(1) != g0;
         uint8_t *codes = (tensor ? a.c.v_codes : a.c.k_codes) + bh * (size_t)s.cap * packed_row_bytes(bits);
         uint8_t *meta = reinterpret_cast<uint8_t *>(tensor ? a.c.v_meta : a.c.k_meta) + bh * (size_t)s.cap * NG * (f8 ? 2 : 4);
         const uint32_t tmem_half = tmem + ((uint32_t)(quad * 32) << 16) + 64 * half;      // this thread's lane, its first column
@@ -330,11 +338,10 @@ append_tile_kernel(AppendArgs a, int tiles_per_cta, const __grid_constant__ CUte
                 lo[1] = fminf(lo0, lo1);
                 hi[1] = fmaxf(hi0, hi1);
             }
-            float mn[kGranules], mx[kGranules];      // the row's four granules; the other half's only when a group spans both
-#pragma unroll
-            for (int gr = 0; gr < kGranules; ++gr) {
-                mn[gr] = (gr >> 1) == half ? lo[gr & 1] : CUDART_INF_F;
-                mx[gr] = (gr >> 1) == half ? hi[gr & 1] : -CUDART_INF_F;
+            float slo[2] = {lo[0], lo[1]}, shi[2] = {hi[0], hi[1]};      // extremes of the two parameter sets
+            if (!two_sets) {
+                slo[0] = fminf(lo[0], lo[1]);
+                shi[0] = fmaxf(hi[0], hi[1]);
             }
             if (spans) {      // uniform: a property of the KV head
                 // Two buffers and one barrier per tile: a thread rewrites the entry of tile t when it works on tile t+2, behind
@@ -342,33 +349,22 @@ append_tile_kernel(AppendArgs a, int tiles_per_cta, const __grid_constant__ CUte
                 ext_sh[t & 1][half][row] = make_float4(lo[0], hi[0], lo[1], hi[1]);
                 pair_sync(quad);
                 const float4 o = ext_sh[t & 1][half ^ 1][row];
-#pragma unroll
-                for (int gr = 0; gr < kGranules; ++gr)
-                    if ((gr >> 1) != half) {
-                        mn[gr] = (gr & 1) ? o.z : o.x;
-                        mx[gr] = (gr & 1) ? o.w : o.y;
-                    }
+                if (p0_in0) { slo[0] = fminf(slo[0], o.x); shi[0] = fmaxf(shi[0], o.y); }
+                if (p1_in0) { slo[0] = fminf(slo[0], o.z); shi[0] = fmaxf(shi[0], o.w); }
+                if (p0_in1) { slo[1] = fminf(slo[1], o.x); shi[1] = fmaxf(shi[1], o.y); }
+                if (p1_in1) { slo[1] = fminf(slo[1], o.z); shi[1] = fmaxf(shi[1], o.w); }
             }
 
-            // ---- scale and zero point of the groups this thread has a part in
-            float hf[NG], zf[NG], rq[NG];
-            uint32_t hz[NG];
-#pragma unroll
-            for (int g = 0; g < NG; ++g) {
-                float glo = CUDART_INF_F, ghi = -CUDART_INF_F;
-#pragma unroll
-                for (int gr = 0; gr < kGranules; ++gr)
-                    if (((gmap >> (2 * gr)) & 3u) == (uint32_t)g) {
-                        glo = fminf(glo, mn[gr]);
-                        ghi = fmaxf(ghi, mx[gr]);
-                    }
-                if (glo > ghi) {      // a group of the other half alone: not this thread's business (uniform over the warp)
-                    hz[g] = 0u; hf[g] = 0.f; zf[g] = 0.f; rq[g] = 0.f;
-                    continue;
-                }
-                group_parameters(glo, ghi, alpha_g[g], qmaxf, f8, hz[g], hf[g], zf[g]);
-                // degenerate group (h == 0): every quotient is taken as 0.  1/qmax is a rounded constant: see pack16
-                rq[g] = hf[g] != 0.0f ? __fmul_rn(__frcp_rn(hf[g]), qmax_inv) : 0.0f;
+            // ---- scale and zero point of the thread's one or two groups
+            float hf[2], zf[2], rq[2];
+            uint32_t hz[2];
+            group_parameters(slo[0], shi[0], alpha0, qmaxf, f8, hz[0], hf[0], zf[0]);
+            // degenerate group (h == 0): every quotient is taken as 0.  1/qmax is a rounded constant: see pack16
+            rq[0] = hf[0] != 0.0f ? __fmul_rn(__frcp_rn(hf[0]), qmax_inv) : 0.0f;
+            hz[1] = hz[0]; hf[1] = hf[0]; zf[1] = zf[0]; rq[1] = rq[0];
+            if (two_sets) {      // uniform over the warp
+                group_parameters(slo[1], shi[1], alpha1, qmaxf, f8, hz[1], hf[1], zf[1]);
+                rq[1] = hf[1] != 0.0f ? __fmul_rn(__frcp_rn(hf[1]), qmax_inv) : 0.0f;
             }
 
             // ---- the codes of the thread's two granules, then its half of the packed row.  WIDTH is the cache's code width
@@ -379,11 +375,7 @@ append_tile_kernel(AppendArgs a, int tiles_per_cta, const __grid_constant__ CUte
                 uint32_t cw[2][2][NW];                                 // [granule][chunk][word]
 #pragma unroll
                 for (int gr = 0; gr < 2; ++gr) {
-                    const uint32_t g = (gmap >> (2 * (2 * half + gr))) & 3u;
-                    float hg = hf[0], zg = zf[0], rg = rq[0];
-#pragma unroll
-                    for (int i = 1; i < NG; ++i)
-                        if (g == (uint32_t)i) { hg = hf[i]; zg = zf[i]; rg = rq[i]; }
+                    const float hg = hf[gr], zg = zf[gr], rg = rq[gr];      // set 1 equals set 0 when both granules share a group
                     uint32_t d0[NW], d1[NW];
                     pack16<FIELD, QMAX>(gr == 0 ? x0 : x2, zg, rg, cw[gr][0], d0);
                     pack16<FIELD, QMAX>(gr == 0 ? x1 : x3, zg, rg, cw[gr][1], d1);
@@ -462,18 +454,15 @@ append_tile_kernel(AppendArgs a, int tiles_per_cta, const __grid_constant__ CUte
             // the accumulator may be overwritten: the last tensor-memory read of this tile (a repair) is behind us
             tc_fence_before();
             mbar_arrive(bar_free + 8 * (t & 1));
-            // {scale, zero}: group g is written by the half that holds its first granule
             if (valid) {
-#pragma unroll
-                for (int g = 0; g < NG; ++g) {
-                    int first = 0;
-#pragma unroll
-                    for (int gr = kGranules - 1; gr >= 0; --gr)
-                        if (((gmap >> (2 * gr)) & 3u) == (uint32_t)g) first = gr;
-                    if ((first >> 1) == half) {
-                        if (f8) reinterpret_cast<uint16_t *>(meta + (size_t)tok * NG * 2)[g] = (uint16_t)hz[g];
-                        else reinterpret_cast<uint32_t *>(meta + (size_t)tok * NG * 4)[g] = hz[g];
-                    }
+                const size_t mrow = (size_t)tok * NG;
+                if (writes0) {
+                    if (f8) reinterpret_cast<uint16_t *>(meta)[mrow + g0] = (uint16_t)hz[0];
+                    else reinterpret_cast<uint32_t *>(meta)[mrow + g0] = hz[0];
+                }
+                if (two_sets) {
+                    if (f8) reinterpret_cast<uint16_t *>(meta)[mrow + g1] = (uint16_t)hz[1];
+                    else reinterpret_cast<uint32_t *>(meta)[mrow + g1] = hz[1];
                 }
             }
             if (control) refill(t + 1);
