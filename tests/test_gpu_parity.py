@@ -442,6 +442,37 @@ def test_unequal_groups_and_three_bit_codes_bit_exact_cache_and_attention(cfg_i,
     assert int(gpu.status[0].item()) == 0
 
 
+@pytest.mark.parametrize("seed", [11, 12, 13])
+def test_random_shapes_widths_groups_windows_and_chunkings(seed):
+    """A seeded sweep over the options of the cache: group size and boundaries, code widths (2, 3, 4 bits, three-level
+    values), KV heads and query heads per KV head, batch, window, sinks, FP8 parameters, and how the tokens arrive."""
+    rng = np.random.default_rng(seed)
+    for _ in range(12):
+        G = int(rng.choice([32, 64, 128]))
+        ng = 128 // G
+        kw = dict(batch=int(rng.choice([1, 2, 3])), ragged=None, n_kv_heads=int(rng.choice([1, 2, 3, 5])), k_bits=int(rng.choice([2, 3, 4])),
+                  v_bits=int(rng.choice([2, 3, 4, 15])), group_size=G, window=int(rng.choice([0, 64, 128, 256])),
+                  n_sink=int(rng.choice([0, 0, 5])), meta_fp8=bool(rng.random() < 0.3))
+        kw["n_q_heads"] = kw["n_kv_heads"] * int(rng.choice([1, 2, 4]))
+        if ng >= 2 and rng.random() < 0.4:
+            cuts = sorted(rng.choice(np.arange(1, 4), size=ng - 1, replace=False).tolist())
+            kw["group_bounds"] = tuple([0] + [32 * c for c in cuts] + [128])
+        chunks = [int(x) for x in rng.integers(1, 1500, size=int(rng.integers(1, 5)))]
+        n = sum(chunks)
+        w = small(1, context=n, **kw)
+        gpu, ora = both_caches(w, n + 64)
+        k, v = w.prefill("k", n), w.prefill("v", n)
+        t = 0
+        for step in chunks:
+            gpu.append(dev(k[:, t:t + step]), dev(v[:, t:t + step]))
+            ora.append(k[:, t:t + step], v[:, t:t + step])
+            t += step
+        assert_cache_bit_exact(gpu, ora)
+        assert int(gpu.status[0].item()) == 0, (kw, chunks)
+        got, want = attention_both(gpu, ora, w)
+        assert np.abs(got - want).max() <= ATTN_TOL, (kw, chunks)
+
+
 def test_calibrated_reorder_groups_and_clip_factors_through_the_library():
     """The offline calibrator's arrays (per-head reorder index, boundaries that differ between heads and between keys
     and values, per-group clip factors) fed to the library and to the oracle alike."""
