@@ -237,7 +237,7 @@ static int partition_ctas_per_sm(const Shape &s)
     const bool plain = plain_width(s.k_bits) && plain_width(s.v_bits);
     if (plain && s.rep == 1 && s.G >= 64) return s.k_bits == s.v_bits ? 4 : 3;           // integer kernel
     if (s.k_bits == 2 && s.v_bits == 2 && (s.rep == 1 || s.rep == 2 || s.rep == 4)) return 2;   // grouped-query kernel, 244 registers
-    return tc_ctas_per_sm(s.G, s.k_bits, s.v_bits);      // tcgen05 kernel: 128 tensor-memory columns, 62-85 KB of shared memory
+    return kTcCtasPerSm;      // tcgen05 kernel: 128 tensor-memory columns, at most 73 KB of shared memory
 }
 
 int current_device()

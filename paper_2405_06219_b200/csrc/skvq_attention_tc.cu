@@ -62,12 +62,18 @@ struct TCfg {
     static constexpr int kOffVm = kRing * kKTile;
     static constexpr int kOffKA = kOffVm + kRing * kVmBytes;             // A of the score MMA: [128 tokens][128 bytes]
     static constexpr int kOffQB = kOffKA + kTile * 128;                  // B of the score MMA: [16 (head, digit)][128 bytes]
-    static constexpr int kOffVB = kOffQB + 16 * 128;                     // A of the value MMA: [128 tokens][128 byte columns]
-    static constexpr int kOffPA = kOffVB + kTile * 128;                  // B of the value MMA: [128 tokens][64 (group, head, digit)]
+    // A of the value MMA: [128 tokens][128 byte columns].  Where both operand buffers would leave room for only two CTAs
+    // per SM (the wider codes), it lives in the buffer of A of the score MMA: the two are built and consumed in turn (K of
+    // tile i+1 in the middle of tile i, V of tile i at its end), each once the MMA that read the other has completed
+    // (measured: the third CTA is worth 9-14 %, the extra waits cost 2 %).
+    static constexpr bool kShared = tc_shared_operand(G, KB, VB);
+    static constexpr int kOffVB = kShared ? kOffKA : kOffQB + 16 * 128;
+    static constexpr int kOffPA = kShared ? kOffQB + 16 * 128 : kOffVB + kTile * 128;      // B of the value MMA: [128 tokens][64 (group, head, digit)]
     static constexpr int kOffOs = kOffPA + kTile * 64;                   // folded value sums [4][128] fp32, by byte column
     static constexpr int kOffMisc = kOffOs + kHeads * kHeadDim * 4;      // small arrays, see the kernel
     static constexpr int kSmemBytes = kOffMisc + 1024;
-    static constexpr int kCtasPerSm = tc_ctas_per_sm(G, KB, VB);         // by shared memory (62-73 KB: three; up to 85 KB: two)
+    static constexpr int kCtasPerSm = kTcCtasPerSm;                      // by shared memory (at most 73 KB)
+    static_assert(kSmemBytes <= 74752, "three CTAs per SM");
     static_assert(kSmemBytes == tc_smem_bytes(G, KB, VB), "the host sizes the grid from the same figure");
     static_assert(kTile * 128 >= kHeads * kHeadDim * 4, "the V operand buffer doubles as query scratch in the prologue");
     static_assert(kKTile % 16 == 0 && kVTile % 16 == 0, "bulk copies move multiples of 16 bytes");
@@ -475,6 +481,7 @@ __global__ void __launch_bounds__(kTile + 32, TCfg<G, KB, VB>::kCtasPerSm) parti
         };
         // every thread: its token's row of tile i -> A operand of the score MMA, then tell the control warp
         auto build_k = [&](int i) {
+            if (C::kShared) wait_pv();      // the value MMA of the tile before has read the buffer (as the V operand)
             wait_ring(bar_k, i);
             unpack_row<KB>(smem + ((tiles_done + i) % kRing) * C::kKTile + tid * C::kKRow,
                            smem + C::kOffKA + (tid >> 3) * kSboK + (tid & 7) * 16, kLbo);
@@ -621,7 +628,9 @@ __global__ void __launch_bounds__(kTile + 32, TCfg<G, KB, VB>::kCtasPerSm) parti
                                    to_fixed_u32(ps[3] * hv[gg]));
             }
 
-            // ---------------- V tile -> A operand of the value MMA
+            // ---------------- V tile -> A operand of the value MMA, once the score MMA of the next tile has read the buffer
+            // (as its K operand; it was issued when that operand was complete, in the middle of this tile)
+            if (C::kShared && i + 1 < n_tiles && !mbar_wait_bounded(bar_s, (n + 1) & 1u)) fail_sh = 1;
             if constexpr (VB == kTernary) unpack_row_ternary(vm + tid * C::kVRow, VOp + (tid >> 3) * kLbo + (tid & 7) * 16, kSboMN, digits_sh);
             else unpack_row<VB>(vm + tid * C::kVRow, VOp + (tid >> 3) * kLbo + (tid & 7) * 16, kSboMN);
             fresh_sh = pv_fresh ? 1 : 0;      // every thread writes the same value

@@ -22,16 +22,23 @@ __host__ __device__ constexpr int code_max(int bits) { return bits == kTernary ?
 __host__ __device__ constexpr bool plain_width(int bits) { return bits == 2 || bits == 4; }
 
 // Dynamic shared memory of the tcgen05 partition kernel (two-slot rings of K codes and of V codes with both tensors'
-// scale/zero, the four MMA operands, folded sums, small arrays) for 128-token tiles, and the CTAs of it an SM holds.
+// scale/zero, the MMA operands, folded sums, small arrays) for 128-token tiles.  Three CTAs of it fit an SM (3 x (73 KB +
+// 1 KB reserved + statics) is what 227 KB hold); where the K and the V operand would not both fit beside the rings, they
+// share one buffer (tc_shared_operand).
+__host__ __device__ constexpr int tc_ring_bytes(int G, int k_bits, int v_bits)
+{
+    return 2 * 128 * packed_row_bytes(k_bits) + 2 * (128 * packed_row_bytes(v_bits) + 2 * 128 * (kHeadDim / G) * 4);
+}
+__host__ __device__ constexpr bool tc_shared_operand(int G, int k_bits, int v_bits)
+{
+    return tc_ring_bytes(G, k_bits, v_bits) + 2 * 128 * 128 + 16 * 128 + 128 * 64 + 4 * kHeadDim * 4 + 1024 > 74752;
+}
 __host__ __device__ constexpr int tc_smem_bytes(int G, int k_bits, int v_bits)
 {
-    return 2 * 128 * packed_row_bytes(k_bits) + 2 * (128 * packed_row_bytes(v_bits) + 2 * 128 * (kHeadDim / G) * 4) + 128 * 128 + 16 * 128 +
-           128 * 128 + 128 * 64 + 4 * kHeadDim * 4 + 1024;
+    return tc_ring_bytes(G, k_bits, v_bits) + (tc_shared_operand(G, k_bits, v_bits) ? 1 : 2) * 128 * 128 + 16 * 128 + 128 * 64 +
+           4 * kHeadDim * 4 + 1024;
 }
-__host__ __device__ constexpr int tc_ctas_per_sm(int G, int k_bits, int v_bits)
-{
-    return tc_smem_bytes(G, k_bits, v_bits) <= 74752 ? 3 : 2;      // 3 x (73 KB + 1 KB reserved + statics) is what 227 KB hold
-}
+constexpr int kTcCtasPerSm = 3;
 
 // Everything the kernels need, by value.
 struct Shape {
