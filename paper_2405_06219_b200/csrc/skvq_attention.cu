@@ -234,8 +234,8 @@ __global__ void __launch_bounds__(kHeadDim) merge_kernel(AttnArgs a)
 // depend on whether group boundaries are given: the workspace is sized from the configuration alone.
 static int partition_ctas_per_sm(const Shape &s)
 {
-    const bool plain = plain_width(s.k_bits) && plain_width(s.v_bits);
-    if (plain && s.rep == 1 && s.G >= 64) return s.k_bits == s.v_bits ? 4 : 3;           // integer kernel
+    const bool integer = plain_width(s.k_bits) && (plain_width(s.v_bits) || s.v_bits == kTernary) && s.rep == 1 && s.G >= 64;
+    if (integer) return s.k_bits == s.v_bits ? 4 : 3;           // integer kernel (three-level values are rewritten as 2-bit rows)
     if (s.k_bits == 2 && s.v_bits == 2 && (s.rep == 1 || s.rep == 2 || s.rep == 4)) return 2;   // grouped-query kernel, 244 registers
     return kTcCtasPerSm;      // tcgen05 kernel: 128 tensor-memory columns, at most 73 KB of shared memory
 }
@@ -330,7 +330,7 @@ cudaError_t launch_attention(const Shape &s, const CachePtrs &c, const __half *q
     // the integer and the grouped-query kernel serve 2- and 4-bit codes in equal groups, or in two groups of unequal
     // width per row; everything else (3-bit streams, three-level values, 4-bit with several query heads or groups of 32,
     // other unequal groups, 3 and 5-8 query heads per KV head) goes to the tcgen05 kernel
-    if (plain_width(s.k_bits) && plain_width(s.v_bits)) {
+    if (plain_width(s.k_bits) && (plain_width(s.v_bits) || s.v_bits == kTernary)) {
         em = launch_partition_mma(s, c, q, a.scale_log2, plan, workspace, stream, overlap, &handled);
         if (em != cudaSuccess) return em;
         if (!handled) {

@@ -1,5 +1,5 @@
 // Integer tensor-core partition kernel of skvq_decode_attention for one query head per KV head and at most two
-// groups per row (G = 64 or 128), 2- or 4-bit K and V in any combination (Eq. 1, Algorithm 1).
+// groups per row (G = 64 or 128), 2- or 4-bit K and V in any combination, or three-level V (Eq. 1, Algorithm 1).
 //
 // Why tensor cores on an HBM-bound path: at 2 bits a cache element costs 0.28 bytes, so streaming at several
 // TB/s leaves fewer than two issue slots per element, and the logic pipe that does the bit work retires half
@@ -34,16 +34,22 @@ struct Cfg {
     static constexpr int NG = kHeadDim / G;
     static_assert(NG <= 2, "(group, byte digit) has to fit the 8 MMA columns");
     static constexpr int T = (KB == 4 && VB == 4) ? 32 : 64;             // tokens per warp tile
-    static constexpr int KROW = kHeadDim * KB / 8, VROW = kHeadDim * VB / 8;   // bytes per token row
-    static constexpr int VCPB = 8 / VB;                                   // codes per byte = masks per register
-    static constexpr int kKTile = T * KROW, kVTile = T * VROW;
+    // Three-level V rows (VB = kTernary: five base-3 digits per byte) arrive as they are stored and are rewritten per
+    // tile, by the warp, as rows of 2-bit fields in a buffer of their own; from there on they are 2-bit rows (VBE).
+    static constexpr bool kTern = VB == kTernary;
+    static constexpr int VBE = kTern ? 2 : VB;
+    static constexpr int KROW = kHeadDim * KB / 8, VROW = kHeadDim * VBE / 8;  // bytes per token row in shared memory
+    static constexpr int VRAW = packed_row_bytes(VB);                     // bytes per V row in the cache
+    static constexpr int VCPB = 8 / VBE;                                  // codes per byte = masks per register
+    static constexpr int kKTile = T * KROW, kVTile = T * VRAW;
+    static constexpr int kVdBytes = kTern ? T * VROW : 0;                 // the rewritten V tile
     static constexpr int kMetaBytes = F8 ? 2 : 4;      // {scale, zero} per (token, group): two E4M3 bytes or a half2
     static constexpr int kMetaTile = T * NG * kMetaBytes;
     static constexpr int kStageBytes = kKTile + kVTile + 2 * kMetaTile;
     static constexpr int kStages = 2;
     static constexpr int kScBytes = T * NG * 8;                           // per (token, group): low and high digit pairs
     static constexpr int kPBytes = (T / 32) * 8 * 32;                     // P operand tile: [k-block][8 columns][32 tokens] bytes
-    static constexpr int kWarpBytes = kStages * kStageBytes + kScBytes + kPBytes + 64;   // + mbarriers
+    static constexpr int kWarpBytes = kStages * kStageBytes + kScBytes + kPBytes + 64 + kVdBytes;   // + mbarriers (+ the rewritten V tile)
     static constexpr int kQBytes = (kHeadDim * 4 + NG * 4 + 2 * 4 + 64 + 127) / 128 * 128 + 512;   // + the B operand image
     static constexpr int kSmemBytes = kQBytes + kWarps * kWarpBytes;
     static constexpr int kCtasPerSm = (KB == VB) ? 4 : 3;      // three measured slower for the equal-width kernels
@@ -58,7 +64,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB, F8>::kCtasPerSm) part
 {
     using C = Cfg<G, KB, VB, F8>;
     static_assert(!UNEQ || C::NG == 2, "unequal groups: two per row");
-    constexpr int NG = C::NG, KROW = C::KROW, VROW = C::VROW, T = C::T;
+    constexpr int NG = C::NG, KROW = C::KROW, VROW = C::VROW, T = C::T, VBE = C::VBE;
     extern __shared__ __align__(128) uint8_t smem[];
     const Shape &s = a.s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -73,6 +79,11 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB, F8>::kCtasPerSm) part
     __shared__ int more_sh;
     __shared__ SlotWalker walk;      // only thread 0 touches it; shared memory keeps it out of everybody's registers
     __shared__ __align__(16) int hdr_sh[kPlanSmemInts];
+    __shared__ uint16_t digits_sh[C::kTern ? 256 : 1];      // byte value -> its five base-3 digits as 2-bit fields
+    if constexpr (C::kTern) {
+        for (int v = tid; v < 256; v += kThreads)
+            digits_sh[v] = (uint16_t)((v % 3) | ((v / 3 % 3) << 2) | ((v / 9 % 3) << 4) | ((v / 27 % 3) << 6) | ((v / 81) << 8));
+    }
     if (a.plan.in_kernel) {
         if (warp == 0) plan_in_warp(a.c.lengths, s.B, s.Hkv, s.W, a.plan.lq_cap, a.plan.n_slots, hdr_sh);
         __syncthreads();
@@ -108,7 +119,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB, F8>::kCtasPerSm) part
     uint8_t *stage_base = warp_base;
     const size_t bh = (size_t)b * s.Hkv + hk;
     const uint8_t *k_codes = a.c.k_codes + bh * (size_t)s.cap * KROW;
-    const uint8_t *v_codes = a.c.v_codes + bh * (size_t)s.cap * VROW;
+    const uint8_t *v_codes = a.c.v_codes + bh * (size_t)s.cap * C::VRAW;
     const uint8_t *k_meta = reinterpret_cast<const uint8_t *>(a.c.k_meta) + bh * (size_t)s.cap * NG * C::kMetaBytes;
     const uint8_t *v_meta = reinterpret_cast<const uint8_t *>(a.c.v_meta) + bh * (size_t)s.cap * NG * C::kMetaBytes;
 
@@ -122,7 +133,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB, F8>::kCtasPerSm) part
         const uint32_t bar = bar0 + 8 * st;
         mbar_expect_tx(bar, C::kStageBytes);
         bulk_g2s(dst, k_codes + (size_t)tok0 * KROW, C::kKTile, bar);
-        bulk_g2s(dst + C::kKTile, v_codes + (size_t)tok0 * VROW, C::kVTile, bar);
+        bulk_g2s(dst + C::kKTile, v_codes + (size_t)tok0 * C::VRAW, C::kVTile, bar);
         bulk_g2s(dst + C::kKTile + C::kVTile, k_meta + (size_t)tok0 * NG * C::kMetaBytes, C::kMetaTile, bar);
         bulk_g2s(dst + C::kKTile + C::kVTile + C::kMetaTile, v_meta + (size_t)tok0 * NG * C::kMetaBytes, C::kMetaTile, bar);
     };
@@ -242,6 +253,31 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB, F8>::kCtasPerSm) part
         if (!mbar_wait_bounded(bar0 + 8 * st, parity)) { failed = true; break; }
         const uint8_t *Kc = stage_base + st * C::kStageBytes;
         const uint8_t *Vc = Kc + C::kKTile;
+        if constexpr (C::kTern) {
+            // Rewrite the tile's V rows (26 bytes of base-3 digits) as rows of 2-bit fields: a lane takes tokens lane and
+            // lane + 32; a byte's five digits come from the table as ten bits and are ORed into the row's bit stream.
+            uint8_t *Vd = stage_base + C::kWarpBytes - C::kVdBytes;
+#pragma unroll
+            for (int hf = 0; hf < T / 32; ++hf) {
+                const uint16_t *raw = reinterpret_cast<const uint16_t *>(Vc + (lane + 32 * hf) * C::VRAW);      // rows are 2-byte aligned
+                uint32_t w[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+#pragma unroll
+                for (int n2 = 0; n2 < C::VRAW / 2; ++n2) {
+                    const uint32_t two = raw[n2];
+#pragma unroll
+                    for (int k = 0; k < 2; ++k) {
+                        const int pos = 10 * (2 * n2 + k), wi = pos >> 5, sh = pos & 31;      // ten bits from bit pos of the row on
+                        const uint32_t e = digits_sh[k ? (two >> 8) : (two & 255u)];
+                        w[wi] |= e << sh;
+                        if (sh > 22 && wi + 1 < 8) w[wi + 1] |= e >> (32 - sh);
+                    }
+                }
+                uint4 *o = reinterpret_cast<uint4 *>(Vd + (lane + 32 * hf) * VROW);
+                o[0] = make_uint4(w[0], w[1], w[2], w[3]);
+                o[1] = make_uint4(w[4], w[5], w[6], w[7]);
+            }
+            Vc = Vd;      // visible to the other lanes behind the __syncwarp() calls in front of the value MMAs
+        }
         const uint8_t *Km = Kc + C::kKTile + C::kVTile;                      // [T][NG] {h, z}
         const uint8_t *Vm = Kc + C::kKTile + C::kVTile + C::kMetaTile;
         // {h, z} of (token, group) as floats: a half2, or two E4M3 bytes (every E4M3 value is an fp16 value)
@@ -397,7 +433,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB, F8>::kCtasPerSm) part
                     ldmatrix_b8_trans_x2(rr, vaddr + kk * 32 * VROW + hh * 16);
 #pragma unroll
                     for (int j = 0; j < C::VCPB; ++j) {
-                        const uint32_t m = VB == 2 ? (0x03030303u << (2 * j)) : (0x0F0F0F0Fu << (4 * j));
+                        const uint32_t m = VBE == 2 ? (0x03030303u << (2 * j)) : (0x0F0F0F0Fu << (4 * j));
                         imma16832_uu(iacc[hh * C::VCPB + j], rr[0] & m, rr[1] & m, rr[2] & m, rr[3] & m, pb.x, pb.y);
                     }
                 }
@@ -448,7 +484,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<G, KB, VB, F8>::kCtasPerSm) part
         for (int q4 = 0; q4 < 4; ++q4) {
             const int d = lane + 32 * q4;
             const int j = d % C::VCPB;                                 // channel d = VCPB*(byte column) + j carries weight 2^(VB*j)
-            const float winv = __int_as_float((127 - VB * j) << 23);
+            const float winv = __int_as_float((127 - VBE * j) << 23);
             const int gd = UNEQ ? (int)((vmap >> (2 * (d >> 5))) & 1u) : d / G;      // group of channel d
             float zg = 0.f;
 #pragma unroll
@@ -509,8 +545,10 @@ template <int G, bool F8, bool UNEQ>
 cudaError_t launch_g(const MmaArgs &a, cudaStream_t stream, bool overlap)
 {
     if (a.s.k_bits == 2)
-        return a.s.v_bits == 2 ? launch_one<G, 2, 2, F8, UNEQ>(a, stream, overlap) : launch_one<G, 2, 4, F8, UNEQ>(a, stream, overlap);
-    return a.s.v_bits == 2 ? launch_one<G, 4, 2, F8, UNEQ>(a, stream, overlap) : launch_one<G, 4, 4, F8, UNEQ>(a, stream, overlap);
+        return a.s.v_bits == 2 ? launch_one<G, 2, 2, F8, UNEQ>(a, stream, overlap)
+             : a.s.v_bits == 4 ? launch_one<G, 2, 4, F8, UNEQ>(a, stream, overlap) : launch_one<G, 2, kTernary, F8, UNEQ>(a, stream, overlap);
+    return a.s.v_bits == 2 ? launch_one<G, 4, 2, F8, UNEQ>(a, stream, overlap)
+         : a.s.v_bits == 4 ? launch_one<G, 4, 4, F8, UNEQ>(a, stream, overlap) : launch_one<G, 4, kTernary, F8, UNEQ>(a, stream, overlap);
 }
 
 }  // namespace
@@ -521,7 +559,7 @@ cudaError_t launch_partition_mma(const Shape &s, const CachePtrs &c, const __hal
                                  const SplitPlan &plan, float *workspace, cudaStream_t stream, bool overlap, bool *handled)
 {
     *handled = false;
-    if (s.rep != 1 || (s.G != 64 && s.G != 128) || !plain_width(s.k_bits) || !plain_width(s.v_bits)) return cudaSuccess;
+    if (s.rep != 1 || (s.G != 64 && s.G != 128) || !plain_width(s.k_bits) || !(plain_width(s.v_bits) || s.v_bits == kTernary)) return cudaSuccess;
     if (s.bounded && s.G != 64) return cudaSuccess;
     MmaArgs a{s, c, q, scale_log2, plan, workspace};
     *handled = true;
