@@ -236,7 +236,7 @@ static int partition_ctas_per_sm(const Shape &s)
 {
     const bool integer = plain_width(s.k_bits) && (plain_width(s.v_bits) || s.v_bits == kTernary) && s.rep == 1 && s.G >= 64;
     if (integer) return s.k_bits == s.v_bits ? 4 : 3;           // integer kernel (three-level values are rewritten as 2-bit rows)
-    if (s.k_bits == 2 && s.v_bits == 2 && (s.rep == 1 || s.rep == 2 || s.rep == 4)) return 2;   // grouped-query kernel, 244 registers
+    if (s.k_bits == 2 && (s.v_bits == 2 || s.v_bits == kTernary) && (s.rep == 1 || s.rep == 2 || s.rep == 4)) return 2;   // grouped-query kernel, 244 registers
     return kTcCtasPerSm;      // tcgen05 kernel: 128 tensor-memory columns, at most 73 KB of shared memory
 }
 

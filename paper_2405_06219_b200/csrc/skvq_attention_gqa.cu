@@ -33,18 +33,23 @@ constexpr int kHeadSlots = 4;           // query heads per KV head this kernel s
 constexpr int kRefSlackLog2 = 12;       // the softmax reference moves only when a score exceeds it by this (log2)
 constexpr float kRefSlack = (float)kRefSlackLog2;
 
-template <int G, bool F8>
+// TERN: three-level V rows (five base-3 digits per byte, 26 bytes) arrive as they are stored and are rewritten per tile, by
+// the warp, as rows of 2-bit fields in a buffer of their own; from there on they are 2-bit rows.
+template <int G, bool F8, bool TERN>
 struct GCfg {
     static constexpr int NG = kHeadDim / G;
     static constexpr int kCodeTile = kTileTok * kRowBytes;               // 2048 B
     static constexpr int kMetaBytes = F8 ? 2 : 4;                        // {scale, zero} per (token, group): two E4M3 bytes or a half2
     static constexpr int kMetaTile = kTileTok * NG * kMetaBytes;
+    static constexpr int kVRaw = TERN ? packed_row_bytes(kTernary) : kRowBytes;      // bytes per V row in the cache
+    static constexpr int kVCopy = kTileTok * kVRaw;                      // bytes of V codes copied per tile (the slot keeps its size)
     static constexpr int kStageBytes = 2 * kCodeTile + 2 * kMetaTile;
+    static constexpr int kVdBytes = TERN ? kCodeTile : 0;                // the rewritten V tile
     static constexpr int kStages = 2;
     static constexpr int kXBytes = NG * 2 * 32 * 8;                      // digit registers on their way to the A fragments
     static constexpr int kOBytes = kHeadSlots * kHeadDim * 4;            // folded P.V sums
     static constexpr int kZBytes = kHeadSlots * 4 * 4;                   // sum p*z per (head, group)
-    static constexpr int kWarpBytes = kStages * kStageBytes + kXBytes + kOBytes + kZBytes + 64;
+    static constexpr int kWarpBytes = kStages * kStageBytes + kXBytes + kOBytes + kZBytes + 64 + kVdBytes;
     static constexpr int kQFloats = kHeadSlots * kHeadDim + 2 * kHeadSlots * 4 + 2 * kHeadSlots + kWarps * kHeadSlots;
     static constexpr int kQBytes = (kQFloats * 4 + 127) / 128 * 128;
     static constexpr int kSmemBytes = kQBytes + kWarps * kWarpBytes;
@@ -163,10 +168,10 @@ __device__ __forceinline__ int owned_token(int kk, int q, int gg) { return 32 * 
 // the registers to overlap the four 16-token score blocks and the two value blocks of a tile.
 // UNEQ: two groups of unequal width per row (boundaries on multiples of 32 channels, read from the cache); the group of
 // a 32-channel block then comes from a map instead of from its position.
-template <int G, int R, bool F8, bool UNEQ>
+template <int G, int R, bool F8, bool UNEQ, bool TERN>
 __global__ void __launch_bounds__(kThreads, 2) partition_gqa_kernel(MmaArgs a)
 {
-    using C = GCfg<G, F8>;
+    using C = GCfg<G, F8, TERN>;
     constexpr int NG = C::NG;
     static_assert(!UNEQ || NG == 2, "unequal groups: two per row");
     static_assert(R <= kHeadSlots, "rows of the P.V MMAs are 4 heads x 4 digits");
@@ -184,6 +189,11 @@ __global__ void __launch_bounds__(kThreads, 2) partition_gqa_kernel(MmaArgs a)
     __shared__ int more_sh;
     __shared__ SlotWalker walk;      // only thread 0 touches it; shared memory keeps it out of everybody's registers
     __shared__ __align__(16) int hdr_sh[kPlanSmemInts];
+    __shared__ uint16_t digits_sh[TERN ? 256 : 1];      // byte value -> its five base-3 digits as 2-bit fields
+    if constexpr (TERN) {
+        for (int v = tid; v < 256; v += kThreads)
+            digits_sh[v] = (uint16_t)((v % 3) | ((v / 3 % 3) << 2) | ((v / 9 % 3) << 4) | ((v / 27 % 3) << 6) | ((v / 81) << 8));
+    }
     if (a.plan.in_kernel) {
         if (warp == 0) plan_in_warp(a.c.lengths, s.B, s.Hkv, s.W, a.plan.lq_cap, a.plan.n_slots, hdr_sh);
         __syncthreads();
@@ -219,7 +229,7 @@ __global__ void __launch_bounds__(kThreads, 2) partition_gqa_kernel(MmaArgs a)
     uint8_t *stage_base = warp_base;
     const size_t bh = (size_t)b * s.Hkv + hk;
     const uint8_t *k_codes = a.c.k_codes + bh * (size_t)s.cap * kRowBytes;
-    const uint8_t *v_codes = a.c.v_codes + bh * (size_t)s.cap * kRowBytes;
+    const uint8_t *v_codes = a.c.v_codes + bh * (size_t)s.cap * C::kVRaw;
     const uint8_t *k_meta = reinterpret_cast<const uint8_t *>(a.c.k_meta) + bh * (size_t)s.cap * NG * C::kMetaBytes;
     const uint8_t *v_meta = reinterpret_cast<const uint8_t *>(a.c.v_meta) + bh * (size_t)s.cap * NG * C::kMetaBytes;
 
@@ -231,9 +241,9 @@ __global__ void __launch_bounds__(kThreads, 2) partition_gqa_kernel(MmaArgs a)
         const int tok0 = q_begin + (warp + i * kWarps) * kTileTok;
         const uint32_t dst = smem_u32(stage_base + st * C::kStageBytes);
         const uint32_t bar = bar0 + 8 * st;
-        mbar_expect_tx(bar, C::kStageBytes);
+        mbar_expect_tx(bar, C::kStageBytes - C::kCodeTile + C::kVCopy);
         bulk_g2s(dst, k_codes + (size_t)tok0 * kRowBytes, C::kCodeTile, bar);
-        bulk_g2s(dst + C::kCodeTile, v_codes + (size_t)tok0 * kRowBytes, C::kCodeTile, bar);
+        bulk_g2s(dst + C::kCodeTile, v_codes + (size_t)tok0 * C::kVRaw, C::kVCopy, bar);
         bulk_g2s(dst + 2 * C::kCodeTile, k_meta + (size_t)tok0 * NG * C::kMetaBytes, C::kMetaTile, bar);
         bulk_g2s(dst + 2 * C::kCodeTile + C::kMetaTile, v_meta + (size_t)tok0 * NG * C::kMetaBytes, C::kMetaTile, bar);
     };
@@ -398,6 +408,31 @@ __global__ void __launch_bounds__(kThreads, 2) partition_gqa_kernel(MmaArgs a)
         if (!mbar_wait_bounded(bar0 + 8 * st, parity)) { failed = true; break; }
         uint8_t *Kc = stage_base + st * C::kStageBytes;
         uint8_t *Vc = Kc + C::kCodeTile;
+        if constexpr (TERN) {
+            // a lane takes tokens lane and lane + 32: a byte's five digits come from the table as ten bits and are ORed
+            // into the row's stream of 2-bit fields
+            uint8_t *Vd = warp_base + C::kWarpBytes - C::kVdBytes;
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+                const uint16_t *raw = reinterpret_cast<const uint16_t *>(Vc + (lane + 32 * hf) * C::kVRaw);      // rows are 2-byte aligned
+                uint32_t w[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+#pragma unroll
+                for (int n2 = 0; n2 < C::kVRaw / 2; ++n2) {
+                    const uint32_t two = raw[n2];
+#pragma unroll
+                    for (int k = 0; k < 2; ++k) {
+                        const int pos = 10 * (2 * n2 + k), wi = pos >> 5, sh = pos & 31;      // ten bits from bit pos of the row on
+                        const uint32_t e = digits_sh[k ? (two >> 8) : (two & 255u)];
+                        w[wi] |= e << sh;
+                        if (sh > 22 && wi + 1 < 8) w[wi + 1] |= e >> (32 - sh);
+                    }
+                }
+                uint4 *o = reinterpret_cast<uint4 *>(Vd + (lane + 32 * hf) * kRowBytes);
+                o[0] = make_uint4(w[0], w[1], w[2], w[3]);
+                o[1] = make_uint4(w[4], w[5], w[6], w[7]);
+            }
+            Vc = Vd;      // visible to the other lanes behind the __syncwarp() calls in front of the value MMAs
+        }
         uint8_t *Km = Kc + 2 * C::kCodeTile;                        // [64][NG] {h, z}
         uint8_t *Vm = Kc + 2 * C::kCodeTile + C::kMetaTile;
         const int tok0 = q_begin + (warp + i * kWarps) * kTileTok;
@@ -678,15 +713,21 @@ __global__ void __launch_bounds__(kThreads, 2) partition_gqa_kernel(MmaArgs a)
     }
 }
 
-template <int G, int R, bool F8, bool UNEQ>
-cudaError_t launch_one(const MmaArgs &a, cudaStream_t stream, bool overlap)
+template <int G, int R, bool F8, bool UNEQ, bool TERN>
+cudaError_t launch_t(const MmaArgs &a, cudaStream_t stream, bool overlap)
 {
-    using C = GCfg<G, F8>;
+    using C = GCfg<G, F8, TERN>;
     static unsigned long long configured = 0;      // one bit per device
-    auto kern = partition_gqa_kernel<G, R, F8, UNEQ>;
+    auto kern = partition_gqa_kernel<G, R, F8, UNEQ, TERN>;
     const cudaError_t ec = configure_smem_once(kern, C::kSmemBytes, configured);
     if (ec != cudaSuccess) return ec;
     return launch_dependent(kern, dim3(a.plan.n_slots), dim3(kThreads), C::kSmemBytes, stream, overlap, a);
+}
+
+template <int G, int R, bool F8, bool UNEQ>
+cudaError_t launch_one(const MmaArgs &a, cudaStream_t stream, bool overlap)
+{
+    return a.s.v_bits == kTernary ? launch_t<G, R, F8, UNEQ, true>(a, stream, overlap) : launch_t<G, R, F8, UNEQ, false>(a, stream, overlap);
 }
 
 template <int G, bool F8, bool UNEQ>
@@ -703,13 +744,13 @@ cudaError_t launch_g(const MmaArgs &a, cudaStream_t stream, bool overlap, bool *
 
 }  // namespace
 
-// Launches the kernel above when the configuration is covered (2-bit K and V, 1, 2 or 4 query heads per KV
+// Launches the kernel above when the configuration is covered (2-bit K, 2-bit or three-level V, 1, 2 or 4 query heads per KV
 // head; groups of unequal width with two groups per row); *handled tells the caller whether it did.
 cudaError_t launch_partition_gqa(const Shape &s, const CachePtrs &c, const __half *q, float scale_log2,
                                  const SplitPlan &plan, float *workspace, cudaStream_t stream, bool overlap, bool *handled)
 {
     *handled = false;
-    if (s.k_bits != 2 || s.v_bits != 2) return cudaSuccess;
+    if (s.k_bits != 2 || (s.v_bits != 2 && s.v_bits != kTernary)) return cudaSuccess;
     if (s.bounded && s.G != 64) return cudaSuccess;
     MmaArgs a{s, c, q, scale_log2, plan, workspace};
     if (s.bounded) return s.meta_fp8 ? launch_g<64, true, true>(a, stream, overlap, handled) : launch_g<64, false, true>(a, stream, overlap, handled);
