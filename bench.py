@@ -50,9 +50,9 @@ MAX_TIMED_STEPS = 4096        # ... but never more steps than this (each step ap
 MAX_E2E_STEPS = 1024
 # DRAM bytes (read + write) per launch of the partition kernel from ncu captures of reduced cases, scaled to the full
 # configuration by the tokens streamed (traffic is proportional to them); None where the kernel has changed since.
-NCU_TRAFFIC_BYTES = {1: 609.5e6, 2: 410.6e6, 3: 2447.0e6, 4: 2549.0e6}
+NCU_TRAFFIC_BYTES = {1: 609.2e6, 2: 409.7e6, 3: 2445.6e6, 4: 2548.7e6}
 NCU_TRAFFIC_SOURCE = {
-    1: "same kernel as configuration 3 (partition_mma_kernel<128,2,2>): its capture's DRAM bytes / algorithmic bytes = 1.013, times this configuration's algorithmic bytes",
+    1: "same kernel as configuration 3 (partition_mma_kernel<128,2,2>): its capture's DRAM bytes / algorithmic bytes = 1.0124, times this configuration's algorithmic bytes",
     2: "ncu capture of configuration 2 at batch 2 (profiles/partition_gqa_K2V2_g32_r4_config2_batch2.md), scaled x 2 by the tokens streamed",
     3: "ncu capture of configuration 3 at a 131072-token context (profiles/partition_mma_K2V2_g128_config3_context128k.md), scaled x 8.006 by the tokens streamed",
     4: "ncu capture of configuration 4 at batch 16 (profiles/partition_mma_K4V4_g64_and_merge_config4_batch16.md), scaled x 4.014 by the tokens streamed",
