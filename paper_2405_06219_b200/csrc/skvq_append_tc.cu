@@ -10,14 +10,16 @@
 // All code widths: 2- and 4-bit fields as they are, 3-bit codes closed up from 4-bit fields into the row's bit stream,
 // three-level codes from 2-bit fields into base-3 bytes.
 //
-// One CTA = 256 threads = one (sequence, KV head, tensor K or V) and a run of consecutive 128-token tiles.  Warps w and w + 4 share the 32 tokens of lane quadrant w & 3: the first takes stored
-// channels 0-63 of each, the second 64-127 (a group that spans both halves has its extremes exchanged through shared
-// memory).  Nothing but mbarriers orders the two sides:
+// One CTA = 256 threads = one (sequence, KV head, tensor K or V) and a run of consecutive 128-token tiles.  Warps w and
+// w + 4 share the 32 tokens of lane quadrant w & 3: the first takes stored channels 0-63 of each, the second 64-127 (a
+// group that spans both halves has its extremes exchanged through shared memory).  Nothing but mbarriers orders copies,
+// MMAs and arithmetic:
 //   copy      thread 0 brings a tile in with two tensor-map copies (cp.async.bulk.tensor, 64 channels x 128
 //             tokens each, 128-byte swizzle: the K-major operand layout of the MMA), two tiles ahead of the arithmetic;
 //             rows past the end of the input are filled with zeros by the copy engine;
-//   MMA       thread 0 issues 8 k-steps per tile, before it starts on its own share of the tile in front, and commits them to an mbarrier; two accumulators in tensor
-//             memory, so the MMAs of tile t+1 run under the arithmetic of tile t;
+//   MMA       thread 0 issues 8 k-steps per tile, before it starts on its own share of the tile in front, and commits
+//             them to an mbarrier; two accumulators in tensor memory, so the MMAs of tile t+1 run under the arithmetic
+//             of tile t;
 //   quantize  every thread reads its half row (64 values) from tensor memory into registers once: the
 //             extremes of its two 32-channel granules (groups are unions of granules), scale and zero point, the
 //             codes, then one 16-byte store of its half of the packed row, and the {scale, zero} words; its arrival on
