@@ -69,6 +69,10 @@ def pick_sequence(lengths, which):
     (3, dict(), [(0, [1, 18])]),
     # configuration 4 in full: 64 ragged sequences (plan kernel + header in the workspace), 4-bit codes, group 64, window 256
     (4, dict(), [("longest", [0]), ("shortest", [31]), ("median", [13])]),
+    # three-level ("1.5-bit") values at full size: rewritten to 2-bit rows inside the integer kernel (configuration 1) and the
+    # grouped-query kernel (configuration 2), prefilled by the tile kernel's base-3 packing
+    (1, dict(v_bits=15), [(6, [17])]),
+    (2, dict(v_bits=15), [(2, [3])]),
 ])
 def test_full_size_sampled_pairs_match_oracle(cfg_i, kw, picks):
     from paper_2405_06219_b200 import binding as B
